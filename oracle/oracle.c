@@ -1,0 +1,277 @@
+/*
+ * oracle.c - plain, slow, fp64 CPU definitions (see oracle.h).
+ * TEST INFRASTRUCTURE ONLY: used by tests, the smoke check and the benchmark's
+ * CPU-baseline leg.  Shares nothing with the CUDA library.
+ *
+ * Build: gcc -O2 -std=c99 -fopenmp -fPIC -shared oracle.c -o liboracle.so -lm
+ * (no -ffast-math: the compensated sums and the NaN / inf rules rely on IEEE).
+ */
+#include "oracle.h"
+
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+static int g_last_threads = 1;
+
+/* ---- Neumaier-compensated accumulation ------------------------------------ */
+typedef struct { double s, c; } nsum;
+
+static void nsum_add(nsum* a, double v) {
+  double t = a->s + v;
+  if (fabs(a->s) >= fabs(v)) a->c += (a->s - t) + v;
+  else                       a->c += (v - t) + a->s;
+  a->s = t;
+}
+static double nsum_get(const nsum* a) { return a->s + a->c; }
+
+/* ---- exact widening of stored elements to double --------------------------- */
+static double widen(const void* base, int dtype, int64_t idx) {
+  if (dtype == ORACLE_F32) return (double)((const float*)base)[idx];
+  if (dtype == ORACLE_F64) return ((const double*)base)[idx];
+  /* bf16: the 16 stored bits are the high half of an IEEE binary32 */
+  uint32_t bits = (uint32_t)((const uint16_t*)base)[idx] << 16;
+  float f;
+  memcpy(&f, &bits, sizeof f);
+  return (double)f;
+}
+
+/* ---- softmax family --------------------------------------------------------- */
+
+/* classify the row: 0 = ordinary (m finite), 1 = NaN row, 2 = no live entry */
+static int softmax_stats(const double* z, int64_t n, double* m_out, double* s_out) {
+  double m = -INFINITY;
+  int has_nan = 0;
+  for (int64_t c = 0; c < n; ++c) {
+    if (isnan(z[c])) has_nan = 1;
+    else if (z[c] > m) m = z[c];
+  }
+  if (has_nan || m == INFINITY) return 1;
+  if (m == -INFINITY) return 2;
+  nsum s = {0.0, 0.0};
+  for (int64_t c = 0; c < n; ++c) nsum_add(&s, exp(z[c] - m)); /* exp(-inf) = 0 */
+  *m_out = m;
+  *s_out = nsum_get(&s);
+  return 0;
+}
+
+void oracle_softmax_row(const double* z, int64_t n, double* y) {
+  double m = 0.0, s = 0.0;
+  int kind = softmax_stats(z, n, &m, &s);
+  if (kind == 1) { for (int64_t c = 0; c < n; ++c) y[c] = NAN; return; }
+  if (kind == 2) { for (int64_t c = 0; c < n; ++c) y[c] = 0.0; return; }
+  for (int64_t c = 0; c < n; ++c) y[c] = exp(z[c] - m) / s;
+}
+
+void oracle_log_softmax_row(const double* z, int64_t n, double* y) {
+  double m = 0.0, s = 0.0;
+  int kind = softmax_stats(z, n, &m, &s);
+  if (kind == 1) { for (int64_t c = 0; c < n; ++c) y[c] = NAN; return; }
+  if (kind == 2) { for (int64_t c = 0; c < n; ++c) y[c] = -INFINITY; return; }
+  double ls = log(s);
+  for (int64_t c = 0; c < n; ++c) y[c] = (z[c] - m) - ls; /* -inf stays -inf */
+}
+
+double oracle_logsumexp_row(const double* z, int64_t n) {
+  double m = 0.0, s = 0.0;
+  int kind = softmax_stats(z, n, &m, &s);
+  if (kind == 1) return NAN;
+  if (kind == 2) return -INFINITY;
+  return m + log(s);
+}
+
+/* ---- normalisations --------------------------------------------------------- */
+
+void oracle_layernorm_row(const double* x, int64_t n, const double* gamma,
+                          const double* beta, double eps, double* y) {
+  nsum a = {0.0, 0.0};
+  for (int64_t c = 0; c < n; ++c) nsum_add(&a, x[c]);
+  double mu = nsum_get(&a) / (double)n;
+  nsum q = {0.0, 0.0};
+  for (int64_t c = 0; c < n; ++c) { double d = x[c] - mu; nsum_add(&q, d * d); }
+  double var = nsum_get(&q) / (double)n;
+  double sd = sqrt(var + eps);
+  for (int64_t c = 0; c < n; ++c) {
+    double g = gamma ? gamma[c] : 1.0;
+    double b = beta ? beta[c] : 0.0;
+    y[c] = (x[c] - mu) / sd * g + b;
+  }
+}
+
+void oracle_rmsnorm_row(const double* x, int64_t n, const double* w,
+                        double eps, double* y) {
+  nsum q = {0.0, 0.0};
+  for (int64_t c = 0; c < n; ++c) nsum_add(&q, x[c] * x[c]);
+  double ms = nsum_get(&q) / (double)n;
+  double rms = sqrt(ms + eps);
+  for (int64_t c = 0; c < n; ++c) y[c] = x[c] / rms * (w ? w[c] : 1.0);
+}
+
+/* ---- array drivers ------------------------------------------------------------ */
+
+static int bad_shape(const void* x, int dtype, int64_t rows, int64_t cols,
+                     int64_t stride, const double* out) {
+  if (rows < 0 || cols < 0) return 1;
+  if (rows == 0 || cols == 0) return 0;
+  if (!x || !out) return 1;
+  if (stride < cols) return 1;
+  if (dtype != ORACLE_F32 && dtype != ORACLE_BF16 && dtype != ORACLE_F64) return 1;
+  return 0;
+}
+
+static int use_threads(int nthreads) {
+#ifdef _OPENMP
+  int t = nthreads > 1 ? nthreads : 1;
+#else
+  int t = 1; (void)nthreads;
+#endif
+  g_last_threads = t;
+  return t;
+}
+
+/* z for one row: widen, add the additive mask, apply the causal rule */
+static void masked_row(const void* x, int dtype, int64_t cols, int64_t x_off,
+                       int64_t grow, const oracle_mask* mask, double* z) {
+  for (int64_t c = 0; c < cols; ++c) z[c] = widen(x, dtype, x_off + c);
+  if (!mask) return;
+  if (mask->additive) {
+    int64_t mr = grow % mask->add_rows;
+    for (int64_t c = 0; c < cols; ++c)
+      z[c] += widen(mask->additive, dtype, mr * mask->add_row_stride + c);
+  }
+  if (mask->causal) {
+    int64_t last_live = grow % mask->causal_period + mask->causal_offset;
+    for (int64_t c = 0; c < cols; ++c)
+      if (c > last_live) z[c] = -INFINITY;
+  }
+}
+
+static int softmax_driver(const void* x, int dtype, int64_t rows, int64_t cols,
+                          int64_t x_stride, const int64_t* row_ids,
+                          const oracle_mask* mask, double* out, int nthreads,
+                          int want_log) {
+  if (bad_shape(x, dtype, rows, cols, x_stride, out)) return 1;
+  if (mask) {
+    if (mask->additive && (mask->add_rows < 1 || mask->add_row_stride < cols)) return 1;
+    if (mask->causal && mask->causal_period < 1) return 1;
+  }
+  int t = use_threads(nthreads);
+  if (rows == 0 || cols == 0) return 0;
+  int failed = 0;
+#pragma omp parallel num_threads(t)
+  {
+    double* z = (double*)malloc((size_t)cols * sizeof(double));
+    if (!z) {
+#pragma omp atomic write
+      failed = 1;
+    }
+#pragma omp for schedule(static)
+    for (int64_t i = 0; i < rows; ++i) {
+      if (!z) continue;
+      int64_t grow = row_ids ? row_ids[i] : i;
+      masked_row(x, dtype, cols, i * x_stride, grow, mask, z);
+      if (want_log) oracle_log_softmax_row(z, cols, out + i * cols);
+      else          oracle_softmax_row(z, cols, out + i * cols);
+    }
+    free(z);
+  }
+  return failed;
+}
+
+int oracle_softmax(const void* x, int dtype, int64_t rows, int64_t cols,
+                   int64_t x_stride, const int64_t* row_ids,
+                   const oracle_mask* mask, double* out, int nthreads) {
+  return softmax_driver(x, dtype, rows, cols, x_stride, row_ids, mask, out, nthreads, 0);
+}
+
+int oracle_log_softmax(const void* x, int dtype, int64_t rows, int64_t cols,
+                       int64_t x_stride, const int64_t* row_ids,
+                       const oracle_mask* mask, double* out, int nthreads) {
+  return softmax_driver(x, dtype, rows, cols, x_stride, row_ids, mask, out, nthreads, 1);
+}
+
+static double* widen_vector(const void* v, int dtype, int64_t n) {
+  double* d = (double*)malloc((size_t)n * sizeof(double));
+  if (d) for (int64_t c = 0; c < n; ++c) d[c] = widen(v, dtype, c);
+  return d;
+}
+
+int oracle_layernorm(const void* x, int dtype, int64_t rows, int64_t cols,
+                     int64_t x_stride, const void* gamma, const void* beta,
+                     double eps, double* out, int nthreads) {
+  if (bad_shape(x, dtype, rows, cols, x_stride, out)) return 1;
+  if (!(eps >= 0.0)) return 1;
+  int t = use_threads(nthreads);
+  if (rows == 0 || cols == 0) return 0;
+  double* g = gamma ? widen_vector(gamma, dtype, cols) : NULL;
+  double* b = beta ? widen_vector(beta, dtype, cols) : NULL;
+  int failed = (gamma && !g) || (beta && !b);
+#pragma omp parallel num_threads(t)
+  {
+    double* xr = (double*)malloc((size_t)cols * sizeof(double));
+    if (!xr) {
+#pragma omp atomic write
+      failed = 1;
+    }
+#pragma omp for schedule(static)
+    for (int64_t i = 0; i < rows; ++i) {
+      if (!xr || failed) continue;
+      for (int64_t c = 0; c < cols; ++c) xr[c] = widen(x, dtype, i * x_stride + c);
+      oracle_layernorm_row(xr, cols, g, b, eps, out + i * cols);
+    }
+    free(xr);
+  }
+  free(g);
+  free(b);
+  return failed;
+}
+
+int oracle_rmsnorm(const void* x, int dtype, int64_t rows, int64_t cols,
+                   int64_t x_stride, const void* weight, double eps,
+                   double* out, int nthreads) {
+  if (bad_shape(x, dtype, rows, cols, x_stride, out)) return 1;
+  if (!(eps >= 0.0)) return 1;
+  int t = use_threads(nthreads);
+  if (rows == 0 || cols == 0) return 0;
+  double* w = weight ? widen_vector(weight, dtype, cols) : NULL;
+  int failed = (weight && !w);
+#pragma omp parallel num_threads(t)
+  {
+    double* xr = (double*)malloc((size_t)cols * sizeof(double));
+    if (!xr) {
+#pragma omp atomic write
+      failed = 1;
+    }
+#pragma omp for schedule(static)
+    for (int64_t i = 0; i < rows; ++i) {
+      if (!xr || failed) continue;
+      for (int64_t c = 0; c < cols; ++c) xr[c] = widen(x, dtype, i * x_stride + c);
+      oracle_rmsnorm_row(xr, cols, w, eps, out + i * cols);
+    }
+    free(xr);
+  }
+  free(w);
+  return failed;
+}
+
+/* ---- the paper's verifier criterion (Section 3.2.3, Eq. 2-3) ------------------ */
+
+double oracle_verifier_fraction(const double* gen, const double* ref, int64_t n,
+                                double eps_switch, double tau) {
+  if (n <= 0) return 0.0;
+  int64_t over = 0;
+  for (int64_t i = 0; i < n; ++i) {
+    double g = gen[i], r = ref[i];
+    if (isnan(g) || isnan(r)) { if (!(isnan(g) && isnan(r))) ++over; continue; }
+    if (isinf(g) || isinf(r)) { if (g != r) ++over; continue; }
+    double e = fabs(g - r);
+    if (fabs(r) > eps_switch) e /= fabs(r);
+    if (e > tau) ++over;
+  }
+  return (double)over / (double)n;
+}
+
+int oracle_last_threads(void) { return g_last_threads; }

@@ -1,0 +1,108 @@
+/*
+ * oracle.h - plain fp64 CPU definitions of the last-axis reduce-then-normalise
+ * operators (softmax, log-softmax, LayerNorm, RMSNorm, additive / causal mask).
+ *
+ * THIS IS TEST INFRASTRUCTURE, NOT THE PRODUCT.  Only the test-suite, the smoke
+ * check and the benchmark's CPU-baseline leg may call it.  It shares no code,
+ * header, table or helper with the CUDA library and neither includes the other.
+ *
+ * Every function works on host memory, one row at a time, in double precision,
+ * as the textbook definition written out (sums are Neumaier-compensated so the
+ * oracle's own rounding stays near 1e-16 relative).  Where the paper speaks
+ * (RMSNorm: sum of squares over the reduced axis, divided by its length, eps
+ * added to that mean, square root, then divide - the Unified Sketch figure of
+ * Section 3.2.1) the oracle follows it; softmax and LayerNorm are only named by
+ * the paper (Section 3.6, Section 4.3) and take their textbook definitions;
+ * log-softmax and masking come from the build contract.
+ *
+ * Parity status: every function below is pinned by tests that run without a GPU
+ * (hand-derived worked examples, closed forms, invariants, fp64 library
+ * routines, 40-digit brute force).  Nothing here is "parity unpinned".
+ */
+#ifndef ORACLE_H_
+#define ORACLE_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* storage types of the input arrays */
+enum { ORACLE_F32 = 0, ORACLE_BF16 = 1, ORACLE_F64 = 2 };
+
+/* Mask descriptor (NULL pointer = no mask).
+ *   z[r,c] = x[r,c] + additive[(r % add_rows) * add_row_stride + c]   (if additive != NULL)
+ *   z[r,c] = -inf  where  c > (r % causal_period) + causal_offset      (if causal != 0)
+ * r is the GLOBAL row index (row_ids[i] when row_ids is given).
+ * The additive array has the same storage type as x. */
+typedef struct oracle_mask {
+  const void* additive;
+  int64_t add_rows;
+  int64_t add_row_stride;
+  int32_t causal;
+  int64_t causal_period;
+  int64_t causal_offset;
+} oracle_mask;
+
+/* ---- single-row cores on doubles (n >= 1) ------------------------------- */
+
+/* softmax of z[0..n): live set L = {c : z_c > -inf}.
+ *   any NaN in z, or max z = +inf  -> every output NaN
+ *   L empty                        -> every output +0
+ *   else m = max z, s = sum exp(z_c - m), y_c = exp(z_c - m) / s           */
+void oracle_softmax_row(const double* z, int64_t n, double* y);
+
+/* log-softmax: y_c = (z_c - m) - ln s; -inf where z_c = -inf;
+ *   L empty -> every output -inf; NaN rule as for softmax.                 */
+void oracle_log_softmax_row(const double* z, int64_t n, double* y);
+
+/* logsumexp(z) = m + ln s (same special cases: -inf if L empty, NaN rule). */
+double oracle_logsumexp_row(const double* z, int64_t n);
+
+/* LayerNorm: mu = sum x / n; var = sum (x-mu)^2 / n (biased);
+ *   y_c = (x_c - mu) / sqrt(var + eps) * gamma_c + beta_c
+ *   gamma == NULL -> 1, beta == NULL -> 0.                                 */
+void oracle_layernorm_row(const double* x, int64_t n, const double* gamma,
+                          const double* beta, double eps, double* y);
+
+/* RMSNorm (Unified Sketch figure, Section 3.2.1): ms = sum x^2 / n;
+ *   y_c = x_c / sqrt(ms + eps) * w_c;  w == NULL -> 1.                     */
+void oracle_rmsnorm_row(const double* x, int64_t n, const double* w,
+                        double eps, double* y);
+
+/* ---- array drivers -------------------------------------------------------
+ * x: rows x cols elements of storage type dtype, row i starts at x + i*x_stride
+ * (elements).  row_ids: NULL -> global row index of row i is i; otherwise
+ * row_ids[i] (used only by the mask).  out: rows x cols doubles, contiguous.
+ * nthreads <= 1: serial; > 1: rows are divided among that many OpenMP threads
+ * (rows are independent; the per-row arithmetic is unchanged).
+ * Return 0 on success, 1 on a malformed argument.                          */
+int oracle_softmax(const void* x, int dtype, int64_t rows, int64_t cols,
+                   int64_t x_stride, const int64_t* row_ids,
+                   const oracle_mask* mask, double* out, int nthreads);
+int oracle_log_softmax(const void* x, int dtype, int64_t rows, int64_t cols,
+                       int64_t x_stride, const int64_t* row_ids,
+                       const oracle_mask* mask, double* out, int nthreads);
+int oracle_layernorm(const void* x, int dtype, int64_t rows, int64_t cols,
+                     int64_t x_stride, const void* gamma, const void* beta,
+                     double eps, double* out, int nthreads);
+int oracle_rmsnorm(const void* x, int dtype, int64_t rows, int64_t cols,
+                   int64_t x_stride, const void* weight, double eps,
+                   double* out, int nthreads);
+
+/* The paper's correctness criterion (Section 3.2.3, Eq. 2-3): element error is
+ * |gen-ref|/|ref| when |ref| > eps_switch, else |gen-ref|; returns the fraction
+ * of elements whose error exceeds tau (the kernel passes iff that fraction is
+ * <= tau).  Elements where both are NaN, or both the same infinity, count as
+ * error 0; a NaN/inf mismatch counts as exceeding tau.                     */
+double oracle_verifier_fraction(const double* gen, const double* ref, int64_t n,
+                                double eps_switch, double tau);
+
+/* number of OpenMP threads the last array driver call actually used */
+int oracle_last_threads(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ORACLE_H_ */

@@ -1,0 +1,168 @@
+"""Seeded synthetic inputs for the five benchmark configurations.
+
+This module holds input generation only - none of the operators' arithmetic -
+so that the CPU oracle and the CUDA library can consume the very same bytes.
+Everything is numpy on the host; bf16 arrays are ``uint16`` holding raw bits.
+
+The operator workloads (row-wise softmax / LayerNorm / RMSNorm over LLM-like
+hidden sizes, a vocabulary-like axis, and an attention-score block) stand in for
+the paper's operator benchmark (Section 3.6) and the third-party suite of
+Section 4.1, neither of which is reproduced here.
+
+Seeding: configuration k (1-based) uses base seed k-1; independent sub-streams
+come from ``numpy.random.SeedSequence(seed).spawn(4)`` in the fixed order
+x, gamma/weight, beta, positions, each driving a ``Generator(PCG64)``.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+from typing import Dict, Optional
+
+import numpy as np
+
+F32, BF16 = 0, 1
+
+
+def f32_to_bf16_bits(a: np.ndarray) -> np.ndarray:
+    """Round float32 to bfloat16 (nearest, ties to even); returns uint16 bits.
+    NaN inputs map to a quiet NaN."""
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    bits = a.view(np.uint32)
+    rounded = ((bits + (np.uint32(0x7FFF) + ((bits >> np.uint32(16)) & np.uint32(1))))
+               >> np.uint32(16)).astype(np.uint16)
+    nan = np.isnan(a)
+    if nan.any():
+        rounded = np.where(nan, np.uint16(0x7FC0), rounded)
+    return rounded
+
+
+def bf16_bits_to_f32(b: np.ndarray) -> np.ndarray:
+    """Exact widening of raw bf16 bits to float32."""
+    b = np.ascontiguousarray(b, dtype=np.uint16)
+    return (b.astype(np.uint32) << np.uint32(16)).view(np.float32)
+
+
+@dataclass
+class Workload:
+    """One operator call: what to run and the host arrays it runs on."""
+    name: str
+    op: str                      # softmax | log_softmax | layernorm | rmsnorm
+    dtype: int                   # F32 | BF16
+    rows: int
+    cols: int
+    x: np.ndarray                # [rows, cols] float32, or uint16 bf16 bits
+    eps: float = 0.0
+    gamma: Optional[np.ndarray] = None   # LayerNorm gamma or RMSNorm weight
+    beta: Optional[np.ndarray] = None
+    causal_period: int = 0       # > 0: entry (r, c) masked iff c > r % period
+    extra: Dict[str, object] = field(default_factory=dict)
+
+    @property
+    def itemsize(self) -> int:
+        return 4 if self.dtype == F32 else 2
+
+    def algorithmic_bytes(self) -> int:
+        """Bytes the method must move: every live input element read once,
+        every output element written once, gamma / beta / weight once."""
+        e = self.itemsize
+        if self.causal_period > 0:
+            p = self.causal_period
+            full, rem = divmod(self.rows, p)
+            # row r has min(cols, r % p + 1) live entries
+            per_period = sum(min(self.cols, i + 1) for i in range(p)) if p <= 1 << 16 else None
+            if per_period is None:
+                raise ValueError("causal period too large for the byte count")
+            live = full * per_period + sum(min(self.cols, i + 1) for i in range(rem))
+        else:
+            live = self.rows * self.cols
+        vec = sum(self.cols for v in (self.gamma, self.beta) if v is not None)
+        return (live + vec + self.rows * self.cols) * e
+
+
+_SHAPES = {
+    1: ("softmax", F32, 64, 1024),
+    2: ("layernorm", F32, 4096, 4096),
+    3: ("rmsnorm", BF16, 16384, 8192),
+    4: ("log_softmax", F32, 256, 262144),
+    5: ("softmax", BF16, 32 * 4096, 4096),
+}
+
+CONFIG_NAMES = {
+    1: "softmax_f32_64x1024",
+    2: "layernorm_f32_4096x4096",
+    3: "rmsnorm_bf16_16384x8192",
+    4: "log_softmax_f32_256x262144",
+    5: "causal_softmax_bf16_32x4096x4096",
+}
+
+
+def _normal_f32(rng: np.random.Generator, rows: int, cols: int) -> np.ndarray:
+    out = np.empty((rows, cols), dtype=np.float32)
+    block = max(1, (1 << 24) // max(cols, 1))
+    for r0 in range(0, rows, block):
+        r1 = min(rows, r0 + block)
+        out[r0:r1] = rng.standard_normal((r1 - r0, cols), dtype=np.float32)
+    return out
+
+
+def make_config(k: int, rows: Optional[int] = None, seed_offset: int = 0) -> Workload:
+    """Build configuration k (1..5).  ``rows`` truncates the row count (the
+    column count, value distribution and seeds are unchanged, so the first rows
+    of a truncated workload equal the first rows of the full one for k != 5's
+    blockwise generator as well).  ``seed_offset`` shifts the base seed (used to
+    give each rank of a multi-GPU run its own rows)."""
+    op, dtype, full_rows, cols = _SHAPES[k]
+    rows = full_rows if rows is None else int(rows)
+    seed = (k - 1) + 1000 * int(seed_offset)
+    s_x, s_g, s_b, s_p = np.random.SeedSequence(seed).spawn(4)
+    rx, rg, rb, rp = (np.random.Generator(np.random.PCG64(s)) for s in (s_x, s_g, s_b, s_p))
+    name = CONFIG_NAMES[k]
+    if k == 1:
+        return Workload(name, op, dtype, rows, cols, _normal_f32(rx, rows, cols))
+    if k == 2:
+        x = _normal_f32(rx, rows, cols)
+        x *= np.float32(2.0)
+        x += np.float32(3.0)
+        gamma = rg.uniform(0.5, 1.5, cols).astype(np.float32)
+        beta = (rb.standard_normal(cols) * 0.1).astype(np.float32)
+        return Workload(name, op, dtype, rows, cols, x, eps=1e-5, gamma=gamma, beta=beta)
+    if k == 3:
+        x = f32_to_bf16_bits(_normal_f32(rx, rows, cols))
+        w = f32_to_bf16_bits(rg.uniform(0.5, 1.5, cols).astype(np.float32))
+        return Workload(name, op, dtype, rows, cols, x, eps=1e-6, gamma=w)
+    if k == 4:
+        x = _normal_f32(rx, rows, cols)
+        x *= np.float32(4.0)
+        n_out = (cols * 1) // 10000          # 0.01 % of the row, rounded down
+        pos = np.empty((rows, n_out), dtype=np.int64)
+        for r in range(rows):
+            pos[r] = rp.choice(cols, size=n_out, replace=False)
+            x[r, pos[r]] = np.float32(30.0)
+        return Workload(name, op, dtype, rows, cols, x, extra={"outlier_cols": pos})
+    if k == 5:
+        scale = np.float32(1.0 / np.sqrt(128.0))
+        x = _normal_f32(rx, rows, cols)
+        x *= scale
+        return Workload(name, op, dtype, rows, cols, f32_to_bf16_bits(x), causal_period=4096)
+    raise ValueError(f"unknown configuration {k}")
+
+
+def make_random(op: str, dtype: int, rows: int, cols: int, seed: int,
+                loc: float = 0.0, scale: float = 1.0, affine: bool = True,
+                eps: float = 1e-5) -> Workload:
+    """Free-form seeded workload for shape sweeps."""
+    s_x, s_g, s_b = np.random.SeedSequence(seed).spawn(3)
+    rx, rg, rb = (np.random.Generator(np.random.PCG64(s)) for s in (s_x, s_g, s_b))
+    x = _normal_f32(rx, rows, cols) * np.float32(scale) + np.float32(loc)
+    gamma = beta = None
+    if op in ("layernorm", "rmsnorm") and affine:
+        gamma = rg.uniform(0.5, 1.5, cols).astype(np.float32)
+        if op == "layernorm":
+            beta = (rb.standard_normal(cols) * 0.1).astype(np.float32)
+    if dtype == BF16:
+        x = f32_to_bf16_bits(x)
+        gamma = None if gamma is None else f32_to_bf16_bits(gamma)
+        beta = None if beta is None else f32_to_bf16_bits(beta)
+    return Workload(f"{op}_{'f32' if dtype == F32 else 'bf16'}_{rows}x{cols}", op, dtype,
+                    rows, cols, x, eps=eps if op in ("layernorm", "rmsnorm") else 0.0,
+                    gamma=gamma, beta=beta)
