@@ -1,0 +1,411 @@
+#!/usr/bin/env python
+"""Benchmark of the row-operator library on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+A step is one launch of the headline operator (LayerNorm fp32 [4096, 4096], the
+second benchmark configuration) through the C ABI on inputs already resident in
+HBM; successive steps rotate over four buffer pairs so the working set (512 MiB)
+exceeds L2.  The one JSON line printed by rank 0 carries the headline number,
+the same figure for every configuration (`per_config`), the roofline fraction,
+the end-to-end figure with host buffers, and the fp64 CPU oracle's timing.
+
+With N > 1 (launched by torch.distributed.run) every rank runs the same
+per-GPU workload on its own seed: rows are independent, there is no collective
+on the data path ("weak" scaling, replicas).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2512_23424_b200 import workloads as wl  # noqa: E402
+
+METRIC = "achieved HBM GB/s (fraction of B200 peak) and rows/s per op and shape"
+HEADLINE = 2
+FALLBACK_HBM_GBS = 6650.0
+NOMINAL_HBM_GBS = 8000.0
+L2_BYTES = 126 * 1000 * 1000
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as fh:
+            return float(json.load(fh)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def profiled_traffic(name: str):
+    """DRAM bytes per launch from the committed ncu summary, if one exists."""
+    path = os.path.join(ROOT, "profiles", "traffic.json")
+    try:
+        with open(path) as fh:
+            return json.load(fh).get(name)
+    except Exception:
+        return None
+
+
+# --------------------------------------------------------------------------------------------
+# clocks
+# --------------------------------------------------------------------------------------------
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML in a background thread."""
+
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
+               0x4: "sw_power_cap", 0x80: "hw_power_brake", 0x2: "applications_clocks_setting"}
+
+    def __init__(self, device_index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        self._h = None
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+            if not uuid.startswith("GPU-"):
+                uuid = "GPU-" + uuid
+            try:
+                self._h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+            except Exception:
+                self._h = pynvml.nvmlDeviceGetHandleByIndex(device_index)
+            self._nv = pynvml
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._h = None
+
+    def _loop(self):
+        nv = self._nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                bits = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+                for bit, name in self.REASONS.items():
+                    if bits & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.002)
+
+    def start(self):
+        if self._h is not None:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self, note: str):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0,
+                    "note": "NVML unavailable"}
+        return {"sm_mhz": int(np.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples), "note": note}
+
+
+# --------------------------------------------------------------------------------------------
+# our arm
+# --------------------------------------------------------------------------------------------
+class DeviceWorkload:
+    """A workload resident in HBM, with `pairs` rotating (x, y) buffer pairs."""
+
+    def __init__(self, w: wl.Workload, pairs: int):
+        import torch
+        from paper_2512_23424_b200 import binding
+        self.w, self.binding, self.torch = w, binding, torch
+        tdt = torch.float32 if w.dtype == wl.F32 else torch.bfloat16
+
+        def dev(a):
+            if a is None:
+                return None
+            if w.dtype == wl.F32:
+                return torch.from_numpy(a).cuda()
+            return torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
+
+        x0 = dev(w.x)
+        self.xs = [x0] + [x0.clone() for _ in range(pairs - 1)]
+        self.ys = [torch.empty((w.rows, w.cols), dtype=tdt, device="cuda") for _ in range(pairs)]
+        self.gamma, self.beta = dev(w.gamma), dev(w.beta)
+        self.mask = binding.make_mask(x0, causal=w.causal_period > 0, causal_period=max(w.causal_period, 1))
+        # arguments marshalled once per buffer pair: a step is then one C-ABI call
+        self.calls = [binding.prepare(w.op, x, y, gamma=self.gamma, beta=self.beta, eps=w.eps,
+                                      mask=self.mask) for x, y in zip(self.xs, self.ys)]
+        self.i = 0
+
+    def launch(self):
+        call = self.calls[self.i % len(self.calls)]
+        self.i += 1
+        return call.launch()
+
+
+def pairs_for(w: wl.Workload) -> int:
+    one = 2 * w.rows * w.cols * w.itemsize
+    if one >= 3 * L2_BYTES:
+        return 1
+    return max(2, int(np.ceil(4 * L2_BYTES / one)))
+
+
+def time_launches(dw: DeviceWorkload, steps: int, warmup: int, barrier=None):
+    """Device time of `steps` back-to-back launches (CUDA events on the launch stream)."""
+    torch = dw.torch
+    for _ in range(max(warmup, 3)):
+        dw.launch()
+    torch.cuda.synchronize()
+    if barrier is not None:
+        barrier()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    start.record()
+    for _ in range(steps):
+        dw.launch()
+    stop.record()
+    torch.cuda.synchronize()
+    if barrier is not None:
+        barrier()
+    return start.elapsed_time(stop) * 1e-3          # seconds
+
+
+def e2e_steps(w: wl.Workload, steps: int, warmup: int):
+    """Same operator with HOST buffers: every step copies the inputs host->device from
+    pinned memory, runs the kernel and copies the result back, inside the timed region."""
+    import torch
+    from paper_2512_23424_b200 import binding
+    tdt = torch.float32 if w.dtype == wl.F32 else torch.bfloat16
+    host_x = torch.from_numpy(w.x if w.dtype == wl.F32 else w.x.view(np.int16))
+    host_x = (host_x if w.dtype == wl.F32 else host_x.view(torch.bfloat16)).pin_memory()
+    host_y = torch.empty((w.rows, w.cols), dtype=tdt).pin_memory()
+    dx = torch.empty((w.rows, w.cols), dtype=tdt, device="cuda")
+    dy = torch.empty_like(dx)
+    gamma = None if w.gamma is None else (torch.from_numpy(w.gamma) if w.dtype == wl.F32 else
+                                          torch.from_numpy(w.gamma.view(np.int16)).view(torch.bfloat16)).cuda()
+    beta = None if w.beta is None else (torch.from_numpy(w.beta) if w.dtype == wl.F32 else
+                                        torch.from_numpy(w.beta.view(np.int16)).view(torch.bfloat16)).cuda()
+    mask = binding.make_mask(dx, causal=w.causal_period > 0, causal_period=max(w.causal_period, 1))
+
+    def step():
+        dx.copy_(host_x, non_blocking=True)
+        if w.op == "softmax":
+            binding.softmax(dx, out=dy, mask=mask)
+        elif w.op == "log_softmax":
+            binding.log_softmax(dx, out=dy, mask=mask)
+        elif w.op == "layernorm":
+            binding.layernorm(dx, gamma, beta, eps=w.eps, out=dy)
+        else:
+            binding.rmsnorm(dx, gamma, eps=w.eps, out=dy)
+        host_y.copy_(dy, non_blocking=True)
+
+    for _ in range(max(1, min(warmup, 3))):
+        step()
+    torch.cuda.synchronize()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    for _ in range(steps):
+        step()
+    stop.record()
+    torch.cuda.synchronize()
+    secs = start.elapsed_time(stop) * 1e-3
+    nbytes = w.rows * w.cols * w.itemsize
+    return secs / steps, nbytes, nbytes
+
+
+def oracle_baseline(w: wl.Workload, budget_s: float = 12.0):
+    """Time the fp64 oracle, as it stands, on a bounded row sample of the workload."""
+    import oracle
+    cores = os.cpu_count() or 1
+
+    def run(rows):
+        sub = wl.Workload(w.name, w.op, w.dtype, rows, w.cols, w.x[:rows], eps=w.eps, gamma=w.gamma,
+                          beta=w.beta, causal_period=w.causal_period)
+        t0 = time.perf_counter()
+        if w.op in ("softmax", "log_softmax"):
+            mask = oracle.Mask(causal=True, causal_period=w.causal_period) if w.causal_period else None
+            getattr(oracle, w.op)(sub.x, mask=mask, nthreads=cores)
+        elif w.op == "layernorm":
+            oracle.layernorm(sub.x, w.gamma, w.beta, eps=float(np.float32(w.eps)), nthreads=cores)
+        else:
+            oracle.rmsnorm(sub.x, w.gamma, eps=float(np.float32(w.eps)), nthreads=cores)
+        return time.perf_counter() - t0, sub.algorithmic_bytes()
+
+    probe_rows = max(1, min(w.rows, max(cores, (1 << 22) // w.cols)))
+    run(probe_rows)                                           # page-in / thread start-up
+    t_probe, _ = run(probe_rows)
+    rows = int(min(w.rows, max(probe_rows, probe_rows * budget_s / max(t_probe, 1e-4))))
+    secs, nbytes = run(rows)
+    return {"value": nbytes / secs / 1e9, "unit": "GB/s", "cores": oracle.last_threads(),
+            "kind": "oracle", "seconds": round(secs, 3), "rows_per_s": rows / secs,
+            "sample": f"first {rows} of {w.rows} rows of {w.name}, OpenMP over rows"}
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2512_23424_b200 import binding
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    else:
+        torch.cuda.set_device(0)
+    dev = torch.cuda.current_device()
+    binding.lib()                                             # fail loudly if the library is missing
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+
+    def max_over_ranks(v: float) -> float:
+        if world == 1:
+            return v
+        t = torch.tensor([v], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    peak, peak_kind = measured_peak()
+    w = wl.make_config(HEADLINE, seed_offset=rank)
+    dw = DeviceWorkload(w, pairs_for(w))
+    sampler = ClockSampler(dev)
+    sampler.start()
+    secs = max_over_ranks(time_launches(dw, args.steps, args.warmup, barrier))
+    note = "timed region"
+    if len(sampler.samples) < 5:                             # short region: keep the same kernel running
+        t_end = time.perf_counter() + 0.25
+        while time.perf_counter() < t_end:
+            for _ in range(50):
+                dw.launch()
+            torch.cuda.synchronize()
+        note = "timed region plus 0.25 s of the same launches"
+    sampler.stop()
+    kernel = binding.last_kernel()
+    per_step = secs / args.steps
+    nbytes = w.algorithmic_bytes()
+    gbs_one = nbytes / per_step / 1e9
+    value = gbs_one * world
+
+    line = {
+        "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": per_step * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": wl.CONFIG_NAMES[HEADLINE], "op": w.op, "rows": w.rows, "cols": w.cols,
+                   "io_dtype": "f32", "rows_per_s": w.rows * world / per_step, "kernel": kernel,
+                   "l2": f"rotating {len(dw.xs)} buffer pairs ({len(dw.xs) * 2 * w.rows * w.cols * w.itemsize >> 20} MiB > L2)",
+                   "parallelism": f"replicas x{world}, no collective"},
+        "gpu_launches": args.steps,
+        "clocks": sampler.summary(note),
+    }
+    if rank == 0 and world == 1:
+        line["roofline"] = {"bound": "hbm", "achieved": gbs_one, "peak": peak, "unit": "GB/s",
+                            "frac": gbs_one / peak, "frac_nominal": gbs_one / NOMINAL_HBM_GBS,
+                            "peak_kind": peak_kind, "traffic": profiled_traffic(wl.CONFIG_NAMES[HEADLINE]),
+                            "algorithmic_bytes": nbytes, "kernel": kernel}
+    # end to end with host buffers
+    e2e_k = max(3, min(args.steps, 20))
+    t_e2e, h2d, d2h = e2e_steps(w, e2e_k, args.warmup)
+    t_e2e = max_over_ranks(t_e2e)
+    line["e2e"] = {"value": nbytes * world / t_e2e / 1e9, "unit": "GB/s", "h2d_bytes_per_step": h2d,
+                   "d2h_bytes_per_step": d2h, "ms_per_step": t_e2e * 1e3, "steps": e2e_k}
+    del dw
+    torch.cuda.empty_cache()
+
+    if rank == 0 and world == 1 and not args.headline_only:
+        table = []
+        for k in (1, 2, 3, 4, 5):
+            wk = w if k == HEADLINE else wl.make_config(k)
+            dwk = DeviceWorkload(wk, pairs_for(wk))
+            reps = {1: 2000, 2: 1000, 3: 300, 4: 300, 5: 100}[k]
+            sk = time_launches(dwk, reps, 10) / reps
+            bk = wk.algorithmic_bytes()
+            row = {"workload": wl.CONFIG_NAMES[k], "kernel": binding.last_kernel(), "us": sk * 1e6,
+                   "rows_per_s": wk.rows / sk, "launches": reps}
+            if k == 1:
+                row["note"] = "latency-bound (0.5 MiB, L2-resident); GB/s not meaningful"
+            else:
+                row.update({"gbs": bk / sk / 1e9, "frac_measured": bk / sk / 1e9 / peak,
+                            "frac_nominal": bk / sk / 1e9 / NOMINAL_HBM_GBS, "algorithmic_bytes": bk,
+                            "traffic": profiled_traffic(wl.CONFIG_NAMES[k])})
+            table.append(row)
+            del dwk, wk
+            torch.cuda.empty_cache()
+        line["per_config"] = table
+    if rank == 0 and world == 1:
+        line["cpu_baseline"] = oracle_baseline(w)
+    assert binding.device_status() == 0, "a device-side bounded wait expired"
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+# --------------------------------------------------------------------------------------------
+# reference arm: the fp64 oracle on the host cores
+# --------------------------------------------------------------------------------------------
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if rank != 0:
+        return
+    import oracle
+    w = wl.make_config(HEADLINE, rows=256)                   # bounded sample of the workload per step
+    cores = os.cpu_count() or 1
+    eps = float(np.float32(w.eps))
+
+    def step():
+        oracle.layernorm(w.x, w.gamma, w.beta, eps=eps, nthreads=cores)
+
+    for _ in range(max(args.warmup, 1)):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    per_step = (time.perf_counter() - t0) / args.steps
+    gbs = w.algorithmic_bytes() / per_step / 1e9
+    sample = f"first 256 of 4096 rows of {wl.CONFIG_NAMES[HEADLINE]} per step, OpenMP over rows"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_step * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic",
+        "config": {"workload": wl.CONFIG_NAMES[HEADLINE], "op": w.op, "rows": w.rows, "cols": w.cols,
+                   "io_dtype": "f32", "sample": sample},
+        "gpu_launches": 0,
+        "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": oracle.last_threads(), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--headline-only", action="store_true",
+                    help="skip the per-configuration table (the headline line is unchanged)")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

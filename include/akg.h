@@ -1,0 +1,151 @@
+/*
+ * akg.h - C ABI of the B200 (sm_100a) row-operator library.
+ *
+ * Last-axis reduce-then-normalise operators over a row-major matrix
+ * X[rows, cols]: softmax, log-softmax, LayerNorm, RMSNorm, with optional
+ * additive and/or causal masking for the softmax pair.  One fused kernel per
+ * call: every live input element is read from HBM once and every output
+ * element written once.  fp32 or bf16 storage; all arithmetic in fp32; a bf16
+ * result is rounded once (nearest-even) at the store.
+ *
+ * General rules for every entry point
+ *   - Pointers named x, y, gamma, beta, weight and akg_mask.additive are DEVICE
+ *     pointers on the current device unless the function name ends in _host.
+ *     The caller owns every buffer; the library allocates no device memory.
+ *   - Strides are in ELEMENTS and must be >= cols.  Vectors (gamma, beta,
+ *     weight) hold cols contiguous elements of the same dtype as x.
+ *   - The call validates its arguments, enqueues work on `stream` (a
+ *     cudaStream_t passed as void*; NULL = the legacy default stream) and
+ *     returns without synchronising.  It never throws, aborts or changes the
+ *     current device.  Calls from several host threads are safe.
+ *   - rows == 0 or cols == 0 is AKG_OK with nothing launched.  Any alignment of
+ *     pointers and strides is accepted: 16-byte aligned rows select vectorised
+ *     kernels, anything else a scalar kernel with the same results.
+ *   - In place (y == x with equal strides) is allowed; any other overlap of the
+ *     x and y ranges is AKG_ERR_INVALID_ARG.
+ *   - On AKG_ERR_INVALID_ARG / AKG_ERR_UNSUPPORTED nothing has been launched.
+ *     AKG_ERR_CUDA reports a failed launch (the CUDA error is consumed; its
+ *     text is available from akg_last_error_string on the same thread).
+ */
+#ifndef AKG_H_
+#define AKG_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum akg_status {
+  AKG_OK = 0,
+  AKG_ERR_INVALID_ARG = 1,
+  AKG_ERR_UNSUPPORTED = 2,
+  AKG_ERR_CUDA = 3,
+  AKG_ERR_DEVICE_TIMEOUT = 4
+} akg_status;
+
+typedef enum akg_dtype { AKG_F32 = 0, AKG_BF16 = 1 } akg_dtype;
+
+/* Kernel families (for akg_set_variant; AKG_VARIANT_AUTO lets the library choose).
+ *   STREAM  scalar loads, any alignment, statistics pass + second read of the row
+ *   REG     row held in registers, 128-bit loads, warp- or CTA-per-row
+ *   TMA     persistent CTAs, rows staged in a shared-memory ring by bulk-copy engine
+ *   CLUSTER one thread-block cluster per row, row resident in the cluster's shared
+ *           memory, partial statistics exchanged through distributed shared memory */
+typedef enum akg_variant {
+  AKG_VARIANT_AUTO = 0,
+  AKG_VARIANT_STREAM = 1,
+  AKG_VARIANT_REG = 2,
+  AKG_VARIANT_TMA = 3,
+  AKG_VARIANT_CLUSTER = 4
+} akg_variant;
+
+/* Mask for the softmax pair (pass NULL for "no mask").  Not part of the paper;
+ * defined by this library:
+ *   z[r,c] = x[r,c] + additive[(r % add_rows) * add_row_stride + c]    if additive != NULL
+ *   z[r,c] = -inf   where  c > (r % causal_period) + causal_offset     if causal != 0
+ * The causal rule is applied from indices: masked input elements are never read
+ * and may hold anything.  additive has the dtype of x; -inf entries are allowed. */
+typedef struct akg_mask {
+  const void* additive;     /* device pointer or NULL                              */
+  int64_t add_rows;         /* >= 1 when additive != NULL                          */
+  int64_t add_row_stride;   /* elements, >= cols                                   */
+  int32_t causal;           /* 0 or 1                                              */
+  int64_t causal_period;    /* P >= 1 when causal                                  */
+  int64_t causal_offset;    /* normally 0; may be negative                         */
+} akg_mask;
+
+/* Softmax over the last axis ("Softmax" in the reduction category, Section 3.6;
+ * textbook definition).  Per row, with z the masked input and L = {c: z_c > -inf}:
+ *   y_c = exp(z_c - max z) / sum_c exp(z_c - max z);   y_c = +0 for c not in L.
+ * A row with no live entry yields +0 everywhere, bit-exactly.  A live NaN, or a
+ * +inf maximum, makes the whole row NaN. */
+akg_status akg_softmax(const void* x, void* y, int64_t rows, int64_t cols,
+                       int64_t x_row_stride, int64_t y_row_stride, akg_dtype dtype,
+                       const akg_mask* mask, void* stream);
+
+/* Log-softmax over the last axis: y_c = (z_c - max z) - ln sum_c exp(z_c - max z),
+ * i.e. x - logsumexp(x); y_c = -inf for masked entries; a row with no live entry
+ * yields -inf everywhere.  NaN rule as for akg_softmax.  Same arguments. */
+akg_status akg_log_softmax(const void* x, void* y, int64_t rows, int64_t cols,
+                           int64_t x_row_stride, int64_t y_row_stride, akg_dtype dtype,
+                           const akg_mask* mask, void* stream);
+
+/* LayerNorm over the last axis ("LayerNorm ... mean, variance, and normalization
+ * steps" fused into one kernel, Section 4.3):
+ *   mu = mean(x), var = mean((x - mu)^2) (biased),
+ *   y_c = (x_c - mu) / sqrt(var + eps) * gamma_c + beta_c.
+ * gamma == NULL means 1, beta == NULL means 0.  eps >= 0 (NaN is rejected). */
+akg_status akg_layernorm(const void* x, void* y, int64_t rows, int64_t cols,
+                         int64_t x_row_stride, int64_t y_row_stride, akg_dtype dtype,
+                         const void* gamma, const void* beta, float eps, void* stream);
+
+/* RMSNorm over the last axis (the Unified Sketch figure of Section 3.2.1: sum of
+ * squares, divided by the axis length, eps added, square root, divide):
+ *   y_c = x_c / sqrt(mean(x^2) + eps) * weight_c;  weight == NULL means 1. */
+akg_status akg_rmsnorm(const void* x, void* y, int64_t rows, int64_t cols,
+                       int64_t x_row_stride, int64_t y_row_stride, akg_dtype dtype,
+                       const void* weight, float eps, void* stream);
+
+/* Human-readable name of a status code (static storage, never NULL). */
+const char* akg_status_string(akg_status status);
+
+/* Text of the most recent failure on the calling thread ("" if none). */
+const char* akg_last_error_string(void);
+
+/* Library version: major * 10000 + minor * 100 + patch. */
+int akg_version(void);
+
+/* Force a kernel family for subsequent calls from any thread (testing and
+ * benchmarking aid).  A forced family that cannot run the given call (alignment,
+ * row length) makes that call return AKG_ERR_UNSUPPORTED.  Returns
+ * AKG_ERR_INVALID_ARG for an unknown value.  AKG_VARIANT_AUTO restores choice. */
+akg_status akg_set_variant(akg_variant variant);
+
+/* Override one launch-geometry choice for subsequent calls (benchmarking aid; 0
+ * restores the library's own choice).  Keys: "reg_threads", "reg_vpt" (CTA size and
+ * 16-byte vectors per thread of the register-resident family; both must be set),
+ * "reg_group" (32 = a warp per row, 1 = a CTA per row), "grid_cap" (maximum CTAs;
+ * rows beyond it are taken in a grid-stride loop); for the shared-memory ring
+ * families "cluster_size" (CTAs per row: 1, 2, 4, 8, 16), "smem_nbuf" (ring depth
+ * limit), "smem_threads" (256, 512, 1024), "smem_ctas" (CTAs per SM the ring is
+ * sized for).  A geometry the library was not
+ * built for makes the next call return AKG_ERR_CUDA.  Unknown key:
+ * AKG_ERR_INVALID_ARG. */
+akg_status akg_set_tuning(const char* key, int value);
+
+/* Name of the kernel family and geometry the last successful call on this thread
+ * launched, e.g. "reg<f32,t256,v4>" (static/thread-local storage). */
+const char* akg_last_kernel_name(void);
+
+/* Reads the device-side status word of the current device (synchronises with
+ * the device).  0 = clean; non-zero = a bounded wait on a bulk copy expired in
+ * some kernel since the last call (the word is reset to 0 by this call).
+ * Returns AKG_OK, AKG_ERR_DEVICE_TIMEOUT, or AKG_ERR_CUDA. */
+akg_status akg_device_status(int* word_out);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AKG_H_ */

@@ -1,1 +1,10 @@
-"""B200-native last-axis softmax / log-softmax / LayerNorm / RMSNorm."""
+"""B200-native last-axis softmax / log-softmax / LayerNorm / RMSNorm.
+
+The operators live in ``libakg.so`` (hand-written sm_100a CUDA behind the C ABI of
+``include/akg.h``); ``binding`` marshals torch tensors into it and ``workloads``
+generates the seeded benchmark inputs.  There is no CPU implementation here.
+"""
+from . import workloads  # noqa: F401
+from .binding import (AkgError, Mask, device_status, last_error, last_kernel, layernorm,  # noqa: F401
+                      lib, log_softmax, make_mask, rmsnorm, set_tuning, set_variant, softmax,
+                      status_string)

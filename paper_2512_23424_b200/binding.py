@@ -1,0 +1,265 @@
+"""Thin ctypes binding of ``libakg.so`` - argument marshalling only.
+
+Every operator runs in the CUDA library; this module turns torch tensors into
+(device pointer, rows, cols, strides, dtype, stream) and checks the returned
+status.  There is no CPU path: a missing library raises, it is never replaced.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+from . import build as _build
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_DEVICE_TIMEOUT = range(5)
+F32, BF16 = 0, 1
+VARIANT_AUTO, VARIANT_STREAM, VARIANT_REG, VARIANT_TMA, VARIANT_CLUSTER = range(5)
+VARIANTS = {"auto": 0, "stream": 1, "reg": 2, "tma": 3, "cluster": 4}
+
+
+class AkgError(RuntimeError):
+    def __init__(self, status: int, where: str, detail: str):
+        super().__init__(f"{where}: {status_string(status)} - {detail}")
+        self.status = status
+
+
+class Mask(ctypes.Structure):
+    """Mirror of ``akg_mask`` (see include/akg.h)."""
+    _fields_ = [("additive", ctypes.c_void_p), ("add_rows", ctypes.c_int64),
+                ("add_row_stride", ctypes.c_int64), ("causal", ctypes.c_int32),
+                ("causal_period", ctypes.c_int64), ("causal_offset", ctypes.c_int64)]
+
+
+_lib: Optional[ctypes.CDLL] = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load ``libakg.so`` (the in-tree build); raises if it is not there."""
+    global _lib
+    if _lib is None:
+        path = _build.LIB_PATH
+        if not os.path.exists(path):
+            raise FileNotFoundError(
+                f"{path} is missing: build it with `python -m paper_2512_23424_b200.build` "
+                "(nvcc, sm_100a); there is no fallback path")
+        L = ctypes.CDLL(path)
+        vp, i64, ci, cf = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_float
+        mp = ctypes.POINTER(Mask)
+        for name in ("akg_softmax", "akg_log_softmax"):
+            getattr(L, name).argtypes = [vp, vp, i64, i64, i64, i64, ci, mp, vp]
+            getattr(L, name).restype = ci
+        L.akg_layernorm.argtypes = [vp, vp, i64, i64, i64, i64, ci, vp, vp, cf, vp]
+        L.akg_layernorm.restype = ci
+        L.akg_rmsnorm.argtypes = [vp, vp, i64, i64, i64, i64, ci, vp, cf, vp]
+        L.akg_rmsnorm.restype = ci
+        L.akg_status_string.argtypes = [ci]
+        L.akg_status_string.restype = ctypes.c_char_p
+        L.akg_last_error_string.argtypes = []
+        L.akg_last_error_string.restype = ctypes.c_char_p
+        L.akg_last_kernel_name.argtypes = []
+        L.akg_last_kernel_name.restype = ctypes.c_char_p
+        L.akg_version.argtypes = []
+        L.akg_version.restype = ci
+        L.akg_set_variant.argtypes = [ci]
+        L.akg_set_variant.restype = ci
+        L.akg_set_tuning.argtypes = [ctypes.c_char_p, ci]
+        L.akg_set_tuning.restype = ci
+        L.akg_device_status.argtypes = [ctypes.POINTER(ci)]
+        L.akg_device_status.restype = ci
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().akg_status_string(int(status)).decode()
+
+
+def last_error() -> str:
+    return lib().akg_last_error_string().decode()
+
+
+def last_kernel() -> str:
+    return lib().akg_last_kernel_name().decode()
+
+
+def set_variant(variant) -> None:
+    code = VARIANTS[variant] if isinstance(variant, str) else int(variant)
+    _check(lib().akg_set_variant(code), "akg_set_variant")
+
+
+def set_tuning(key: str, value: int) -> None:
+    _check(lib().akg_set_tuning(key.encode(), int(value)), "akg_set_tuning")
+
+
+def device_status() -> int:
+    word = ctypes.c_int(0)
+    st = lib().akg_device_status(ctypes.byref(word))
+    if st not in (OK, ERR_DEVICE_TIMEOUT):
+        _check(st, "akg_device_status")
+    return word.value
+
+
+def _check(status: int, where: str) -> None:
+    if status != OK:
+        raise AkgError(status, where, last_error())
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError(f"unsupported dtype {t.dtype}: the library handles float32 and bfloat16")
+
+
+def _matrix(t: torch.Tensor, what: str):
+    if t.dim() != 2:
+        raise ValueError(f"{what} must be 2-D [rows, cols]")
+    if not t.is_cuda:
+        raise ValueError(f"{what} must live on a CUDA device")
+    rows, cols = t.shape
+    if cols > 1 and t.stride(1) != 1:
+        raise ValueError(f"{what}: the last axis must be contiguous")
+    return rows, cols, (t.stride(0) if rows > 1 else cols)
+
+
+def _vector(v: Optional[torch.Tensor], like: torch.Tensor, cols: int, what: str):
+    if v is None:
+        return None
+    if v.dtype != like.dtype or v.dim() != 1 or v.numel() != cols or not v.is_contiguous() \
+            or v.device != like.device:
+        raise ValueError(f"{what} must be a contiguous {like.dtype} vector of cols elements on x's device")
+    return v.data_ptr()
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def make_mask(x: torch.Tensor, additive: Optional[torch.Tensor] = None, causal: bool = False,
+              causal_period: int = 1, causal_offset: int = 0) -> Optional[Mask]:
+    if additive is None and not causal:
+        return None
+    m = Mask()
+    if additive is not None:
+        if additive.dim() != 2 or additive.dtype != x.dtype or additive.device != x.device:
+            raise ValueError("additive mask must be a 2-D tensor of x's dtype on x's device")
+        if additive.shape[1] > 1 and additive.stride(1) != 1:
+            raise ValueError("additive mask: the last axis must be contiguous")
+        m.additive = additive.data_ptr()
+        m.add_rows = additive.shape[0]
+        m.add_row_stride = additive.stride(0) if additive.shape[0] > 1 else max(additive.shape[1], 1)
+        m._keep = additive
+    m.causal = 1 if causal else 0
+    m.causal_period = int(causal_period)
+    m.causal_offset = int(causal_offset)
+    return m
+
+
+class PreparedCall:
+    """One operator call with its arguments marshalled once; ``launch()`` only makes
+    the C call (about a microsecond of host time), for loops that re-issue the same
+    call.  The tensors are kept alive by the object; the stream is fixed at creation."""
+
+    def __init__(self, fn_name: str, args: tuple, keep: tuple, out: torch.Tensor):
+        self._fn = getattr(lib(), fn_name)
+        self._name, self._args, self._keep, self.out = fn_name, args, keep, out
+
+    def launch(self) -> torch.Tensor:
+        st = self._fn(*self._args)
+        if st != OK:
+            raise AkgError(st, self._name, last_error())
+        return self.out
+
+
+def prepare(op: str, x: torch.Tensor, out: Optional[torch.Tensor] = None, *,
+            gamma: Optional[torch.Tensor] = None, beta: Optional[torch.Tensor] = None,
+            eps: float = 1e-5, mask: Optional[Mask] = None, stream=None) -> PreparedCall:
+    """Marshal a call of ``op`` (softmax | log_softmax | layernorm | rmsnorm) once."""
+    rows, cols, xs = _matrix(x, "x")
+    if out is None:
+        out = torch.empty_like(x)
+    orow, ocol, ys = _matrix(out, "out")
+    if (orow, ocol) != (rows, cols) or out.dtype != x.dtype or out.device != x.device:
+        raise ValueError("out must match x in shape, dtype and device")
+    with torch.cuda.device(x.device):
+        s = ctypes.c_void_p(_stream(stream))
+    vp, i64 = ctypes.c_void_p, ctypes.c_int64
+    head = (vp(x.data_ptr()), vp(out.data_ptr()), i64(rows), i64(cols), i64(xs), i64(ys),
+            ctypes.c_int(_dtype_code(x)))
+    if op in ("softmax", "log_softmax"):
+        args = head + (ctypes.byref(mask) if mask is not None else None, s)
+        return PreparedCall("akg_" + op, args, (x, mask), out)
+    if op == "layernorm":
+        args = head + (vp(_vector(gamma, x, cols, "gamma")), vp(_vector(beta, x, cols, "beta")),
+                       ctypes.c_float(eps), s)
+        return PreparedCall("akg_layernorm", args, (x, gamma, beta), out)
+    if op == "rmsnorm":
+        args = head + (vp(_vector(gamma, x, cols, "weight")), ctypes.c_float(eps), s)
+        return PreparedCall("akg_rmsnorm", args, (x, gamma), out)
+    raise ValueError(f"unknown operator {op}")
+
+
+def _softmax_like(fn_name, x, out, mask, stream):
+    rows, cols, xs = _matrix(x, "x")
+    if out is None:
+        out = torch.empty_like(x)
+    orow, ocol, ys = _matrix(out, "out")
+    if (orow, ocol) != (rows, cols) or out.dtype != x.dtype or out.device != x.device:
+        raise ValueError("out must match x in shape, dtype and device")
+    with torch.cuda.device(x.device):
+        st = getattr(lib(), fn_name)(x.data_ptr(), out.data_ptr(), rows, cols, xs, ys,
+                                     _dtype_code(x), ctypes.byref(mask) if mask is not None else None,
+                                     _stream(stream))
+    _check(st, fn_name)
+    return out
+
+
+def softmax(x: torch.Tensor, out: Optional[torch.Tensor] = None, mask: Optional[Mask] = None,
+            stream=None) -> torch.Tensor:
+    """akg_softmax over the last axis of a 2-D CUDA tensor."""
+    return _softmax_like("akg_softmax", x, out, mask, stream)
+
+
+def log_softmax(x: torch.Tensor, out: Optional[torch.Tensor] = None, mask: Optional[Mask] = None,
+                stream=None) -> torch.Tensor:
+    """akg_log_softmax over the last axis of a 2-D CUDA tensor."""
+    return _softmax_like("akg_log_softmax", x, out, mask, stream)
+
+
+def layernorm(x: torch.Tensor, gamma: Optional[torch.Tensor] = None, beta: Optional[torch.Tensor] = None,
+              eps: float = 1e-5, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """akg_layernorm over the last axis of a 2-D CUDA tensor."""
+    rows, cols, xs = _matrix(x, "x")
+    if out is None:
+        out = torch.empty_like(x)
+    orow, ocol, ys = _matrix(out, "out")
+    if (orow, ocol) != (rows, cols) or out.dtype != x.dtype or out.device != x.device:
+        raise ValueError("out must match x in shape, dtype and device")
+    with torch.cuda.device(x.device):
+        st = lib().akg_layernorm(x.data_ptr(), out.data_ptr(), rows, cols, xs, ys, _dtype_code(x),
+                                 _vector(gamma, x, cols, "gamma"), _vector(beta, x, cols, "beta"),
+                                 float(eps), _stream(stream))
+    _check(st, "akg_layernorm")
+    return out
+
+
+def rmsnorm(x: torch.Tensor, weight: Optional[torch.Tensor] = None, eps: float = 1e-6,
+            out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """akg_rmsnorm over the last axis of a 2-D CUDA tensor."""
+    rows, cols, xs = _matrix(x, "x")
+    if out is None:
+        out = torch.empty_like(x)
+    orow, ocol, ys = _matrix(out, "out")
+    if (orow, ocol) != (rows, cols) or out.dtype != x.dtype or out.device != x.device:
+        raise ValueError("out must match x in shape, dtype and device")
+    with torch.cuda.device(x.device):
+        st = lib().akg_rmsnorm(x.data_ptr(), out.data_ptr(), rows, cols, xs, ys, _dtype_code(x),
+                               _vector(weight, x, cols, "weight"), float(eps), _stream(stream))
+    _check(st, "akg_rmsnorm")
+    return out

@@ -1,0 +1,355 @@
+// C ABI of the row-operator library: argument validation, kernel-family choice,
+// launch.  No device memory is allocated here and nothing synchronises.
+#include <atomic>
+#include <climits>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+
+#include "../../include/akg.h"
+#include "launch.cuh"
+
+namespace akg {
+namespace {
+
+thread_local char t_error[256] = "";
+thread_local char t_kernel[96] = "";
+std::atomic<int> g_forced_variant{V_AUTO};
+std::atomic<int> g_tune_reg_threads{0};   // 0 = planner's choice
+std::atomic<int> g_tune_reg_vpt{0};
+std::atomic<int> g_tune_reg_group{0};     // 0 = planner's choice, 32 = warp per row, 1 = CTA per row
+std::atomic<int> g_tune_grid_cap{0};      // 0 = one CTA per row group
+std::atomic<int> g_tune_cluster_size{0};  // shared-memory ring family: CTAs per row
+std::atomic<int> g_tune_smem_nbuf{0};     //   ring depth limit
+std::atomic<int> g_tune_smem_threads{0};  //   CTA size (256 / 512 / 1024)
+std::atomic<int> g_tune_smem_ctas{0};     //   CTAs per SM the ring is sized for
+
+__device__ int g_status_word = 0;
+
+akg_status fail(akg_status st, const char* fmt, const char* a = "", long long b = 0) {
+  std::snprintf(t_error, sizeof t_error, fmt, a, b);
+  return st;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+struct Call {
+  int op;
+  const void* x; void* y;
+  int64_t rows, cols, xs, ys;
+  int dtype;
+  const akg_mask* mask;
+  const void* gamma; const void* beta;
+  float eps;
+  void* stream;
+};
+
+akg_status validate(const Call& c, const char* name) {
+  if (c.dtype != AKG_F32 && c.dtype != AKG_BF16) return fail(AKG_ERR_INVALID_ARG, "%s: unknown dtype", name);
+  if (c.rows < 0 || c.cols < 0) return fail(AKG_ERR_INVALID_ARG, "%s: negative rows or cols", name);
+  const bool norm = (c.op == OP_LAYERNORM || c.op == OP_RMSNORM);
+  if (norm && !(c.eps >= 0.f)) return fail(AKG_ERR_INVALID_ARG, "%s: eps must be >= 0 and not NaN", name);
+  if (norm && std::isinf(c.eps)) return fail(AKG_ERR_INVALID_ARG, "%s: eps must be finite", name);
+  if (c.mask != nullptr) {
+    const akg_mask& m = *c.mask;
+    if (m.causal != 0 && m.causal != 1) return fail(AKG_ERR_INVALID_ARG, "%s: mask.causal must be 0 or 1", name);
+    if (m.causal && m.causal_period < 1) return fail(AKG_ERR_INVALID_ARG, "%s: mask.causal_period must be >= 1", name);
+    if (m.additive != nullptr && (m.add_rows < 1 || m.add_row_stride < c.cols))
+      return fail(AKG_ERR_INVALID_ARG, "%s: additive mask needs add_rows >= 1 and add_row_stride >= cols", name);
+  }
+  if (c.rows == 0 || c.cols == 0) return AKG_OK;
+  if (c.x == nullptr || c.y == nullptr) return fail(AKG_ERR_INVALID_ARG, "%s: x and y must not be NULL", name);
+  if (c.xs < c.cols || c.ys < c.cols) return fail(AKG_ERR_INVALID_ARG, "%s: row stride smaller than cols", name);
+  if (c.cols > INT_MAX / 2) return fail(AKG_ERR_UNSUPPORTED, "%s: cols above 2^30 - 1", name);
+  const int64_t es = (c.dtype == AKG_F32) ? 4 : 2;
+  // extent of each matrix in bytes; reject anything that would overflow pointer arithmetic
+  const long double lim = 9.0e18L;
+  if (static_cast<long double>(c.rows) * c.xs * es > lim || static_cast<long double>(c.rows) * c.ys * es > lim)
+    return fail(AKG_ERR_INVALID_ARG, "%s: rows * stride overflows", name);
+  const uintptr_t x0 = reinterpret_cast<uintptr_t>(c.x), y0 = reinterpret_cast<uintptr_t>(c.y);
+  const uintptr_t x1 = x0 + static_cast<uintptr_t>(((c.rows - 1) * c.xs + c.cols) * es);
+  const uintptr_t y1 = y0 + static_cast<uintptr_t>(((c.rows - 1) * c.ys + c.cols) * es);
+  const bool overlap = x0 < y1 && y0 < x1;
+  if (overlap && !(x0 == y0 && c.xs == c.ys))
+    return fail(AKG_ERR_INVALID_ARG, "%s: x and y overlap without being the same matrix", name);
+  return AKG_OK;
+}
+
+bool is_pow2(long long v) { return v > 0 && (v & (v - 1)) == 0; }
+
+int pow2_ceil(int v) { int r = 1; while (r < v) r <<= 1; return r; }
+
+// Can the vectorised families run this call?  (16-byte aligned rows and vectors.)
+bool vector_ok(const Call& c) {
+  const int64_t es = (c.dtype == AKG_F32) ? 4 : 2;
+  const int64_t epv = 16 / es;
+  if (c.cols % epv) return false;
+  if (!aligned16(c.x) || !aligned16(c.y)) return false;
+  if (c.rows > 1 && ((c.xs * es) % 16 || (c.ys * es) % 16)) return false;
+  if (c.gamma && !aligned16(c.gamma)) return false;
+  if (c.beta && !aligned16(c.beta)) return false;
+  if (c.mask && c.mask->additive) {
+    if (!aligned16(c.mask->additive)) return false;
+    if (c.mask->add_rows > 1 && (c.mask->add_row_stride * es) % 16) return false;
+  }
+  return true;
+}
+
+// Register-resident plan, or false if the row does not fit.
+bool plan_reg(const Call& c, LaunchPlan* plan) {
+  const int64_t epv = (c.dtype == AKG_F32) ? 4 : 8;
+  const int64_t nvec = c.cols / epv;
+  int group = 0, vpt = 0, threads = 0;
+  const int t_group = g_tune_reg_group.load(), t_threads = g_tune_reg_threads.load(), t_vpt = g_tune_reg_vpt.load();
+  const bool many_rows = c.rows >= 4096;
+  const bool want_warp = (t_group == 32) || (t_group == 0 && nvec <= 256 && many_rows);
+  if (want_warp && nvec <= 256) {
+    group = 32; threads = 128;
+    vpt = pow2_ceil(static_cast<int>((nvec + 31) / 32));
+  } else if (t_threads > 0 && t_vpt > 0) {
+    group = threads = t_threads; vpt = t_vpt;
+    if (static_cast<int64_t>(threads) * vpt < nvec) return false;
+  } else {
+    // widest vectors-per-thread of 4 until the CTA is full, then 8
+    if (nvec <= 128) { threads = 128; vpt = 1; }
+    else if (nvec <= 256) { threads = 128; vpt = 2; }
+    else if (nvec <= 512) { threads = 128; vpt = 4; }
+    else if (nvec <= 1024) { threads = 256; vpt = 4; }
+    else if (nvec <= 2048) { threads = 512; vpt = 4; }
+    else if (nvec <= 4096) { threads = (c.dtype == AKG_F32) ? 512 : 1024; vpt = (c.dtype == AKG_F32) ? 8 : 4; }
+    else if (nvec <= 8192 && c.dtype == AKG_F32) { threads = 1024; vpt = 8; }
+    else return false;
+    group = threads;
+  }
+  const int64_t rpc = threads / group;
+  int64_t grid = (c.rows + rpc - 1) / rpc;
+  const int cap = g_tune_grid_cap.load();
+  if (cap > 0 && grid > cap) grid = cap;
+  if (grid > INT_MAX) grid = INT_MAX;
+  plan->variant = V_REG; plan->threads = threads; plan->group = group; plan->vpt = vpt;
+  plan->grid = static_cast<unsigned>(grid); plan->cluster = 1; plan->stages = 0; plan->smem = 0;
+  return true;
+}
+
+// Shared-memory ring plan with a cluster of cs CTAs per row, cs_min <= cs <= cs_max
+// (cs = 1 is the plain TMA ring).  Picks the smallest cluster whose slice leaves room
+// for at least two ring buffers, else the smallest with one.  False if nothing fits.
+bool plan_smem(const Call& c, int cs_min, int cs_max, LaunchPlan* plan) {
+  const int64_t epv = (c.dtype == AKG_F32) ? 4 : 8;
+  const int64_t nvec = c.cols / epv;
+  const int t_cs = g_tune_cluster_size.load(), t_nbuf = g_tune_smem_nbuf.load();
+  const int t_threads = g_tune_smem_threads.load(), t_ctas = g_tune_smem_ctas.load();
+  if (t_cs > 0) {
+    if (t_cs < cs_min || t_cs > cs_max) return false;
+    cs_min = cs_max = t_cs;
+  }
+  int best_cs = 0, best_nbuf = 0, best_threads = 0;
+  int64_t best_slice = 0;
+  for (int want = 2; want >= 1 && best_cs == 0; --want) {
+    for (int cs = cs_min; cs <= cs_max; cs *= 2) {
+      const int64_t slice = (nvec + cs - 1) / cs;
+      if (slice < 1) continue;
+      int threads = t_threads > 0 ? t_threads : (slice <= 1024 ? 256 : (slice <= 8192 ? 512 : 1024));
+      if (threads != 256 && threads != 512 && threads != 1024) return false;
+      const int64_t buf = (slice * 16 + 127) & ~int64_t(127);
+      // rows of up to 32 KiB share an SM between two CTAs so that one row's reduction
+      // overlaps the other's copies and stores
+      const int ctas = t_ctas > 0 ? t_ctas : ((cs == 1 && buf <= 32768) ? 2 : 1);
+      const int64_t budget = static_cast<int64_t>(kMaxDynSmem) / ctas - (ctas > 1 ? 1024 : 0) -
+                             smem_header_bytes(threads);
+      int64_t nbuf = budget / buf;
+      if (nbuf > kMaxBuf) nbuf = kMaxBuf;
+      if (t_nbuf > 0 && nbuf > t_nbuf) nbuf = t_nbuf;
+      if (nbuf >= want) { best_cs = cs; best_nbuf = static_cast<int>(nbuf); best_threads = threads; best_slice = slice; break; }
+    }
+  }
+  if (best_cs == 0) return false;
+  const int64_t buf = (best_slice * 16 + 127) & ~int64_t(127);
+  plan->variant = (best_cs == 1) ? V_TMA : V_CLUSTER;
+  plan->threads = best_threads; plan->group = best_threads; plan->vpt = static_cast<int>(best_slice);
+  plan->cluster = best_cs; plan->stages = best_nbuf;
+  plan->smem = smem_header_bytes(best_threads) + static_cast<size_t>(best_nbuf) * buf;
+  const int cap = g_tune_grid_cap.load();
+  plan->grid = cap > 0 ? static_cast<unsigned>((cap / best_cs > 0 ? cap / best_cs : 1) * best_cs) : 0u;
+  return true;
+}
+
+// Device address of the status word on the current device (cached per device).
+int* status_word_ptr() {
+  static std::atomic<int*> cache[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  int* ptr = cache[dev].load();
+  if (ptr == nullptr) {
+    void* sym = nullptr;
+    if (cudaGetSymbolAddress(&sym, g_status_word) != cudaSuccess) { (void)cudaGetLastError(); return nullptr; }
+    ptr = static_cast<int*>(sym);
+    cache[dev].store(ptr);
+  }
+  return ptr;
+}
+
+void plan_stream(const Call& c, LaunchPlan* plan) {
+  int64_t grid = c.rows;
+  const int cap = g_tune_grid_cap.load();
+  if (cap > 0 && grid > cap) grid = cap;
+  if (grid > INT_MAX) grid = INT_MAX;
+  plan->variant = V_STREAM; plan->threads = 256; plan->group = 256; plan->vpt = 0;
+  plan->grid = static_cast<unsigned>(grid); plan->cluster = 1; plan->stages = 0; plan->smem = 0;
+}
+
+akg_status run(const Call& c, const char* name) {
+  t_error[0] = '\0';
+  akg_status st = validate(c, name);
+  if (st != AKG_OK) return st;
+  if (c.rows == 0 || c.cols == 0) return AKG_OK;
+
+  RowParams p;
+  std::memset(&p, 0, sizeof p);
+  p.x = c.x; p.y = c.y; p.rows = c.rows; p.cols = c.cols; p.xs = c.xs; p.ys = c.ys;
+  p.gamma = c.gamma; p.beta = c.beta; p.eps = c.eps;
+  p.period = 1;
+  p.add_rows = 1;
+  if (c.mask != nullptr) {
+    p.add = c.mask->additive;
+    if (p.add) {
+      p.add_rows = c.mask->add_rows; p.add_stride = c.mask->add_row_stride;
+      p.add_mode = (p.add_rows == 1) ? 1 : (p.add_rows >= c.rows ? 2 : 0);
+    }
+    p.causal = c.mask->causal;
+    if (p.causal) {
+      p.period = c.mask->causal_period; p.offset = c.mask->causal_offset;
+      p.period_pow2 = is_pow2(p.period) ? 1 : 0;
+    }
+  }
+  p.status = nullptr;
+
+  const int forced = g_forced_variant.load();
+  const bool vec = vector_ok(c);
+  LaunchPlan plan;
+  std::memset(&plan, 0, sizeof plan);
+  bool planned = false;
+  if ((forced == V_AUTO || forced == V_REG) && vec) planned = plan_reg(c, &plan);
+  if (!planned && vec) {
+    if (forced == V_AUTO) planned = plan_smem(c, 1, kMaxCluster, &plan);
+    else if (forced == V_TMA) planned = plan_smem(c, 1, 1, &plan);
+    else if (forced == V_CLUSTER) planned = plan_smem(c, 2, kMaxCluster, &plan);
+    if (planned) p.status = status_word_ptr();
+  }
+  if (!planned && (forced == V_AUTO || forced == V_STREAM)) { plan_stream(c, &plan); planned = true; }
+  if (!planned) return fail(AKG_ERR_UNSUPPORTED, "%s: the forced kernel family cannot run this call", name);
+
+  cudaStream_t stream = static_cast<cudaStream_t>(c.stream);
+  cudaError_t err;
+  switch (c.op) {
+    case OP_SOFTMAX: err = launch_op<OP_SOFTMAX>(plan, c.dtype, p, stream); break;
+    case OP_LOG_SOFTMAX: err = launch_op<OP_LOG_SOFTMAX>(plan, c.dtype, p, stream); break;
+    case OP_LAYERNORM: err = launch_op<OP_LAYERNORM>(plan, c.dtype, p, stream); break;
+    default: err = launch_op<OP_RMSNORM>(plan, c.dtype, p, stream); break;
+  }
+  if (err != cudaSuccess) {
+    (void)cudaGetLastError();
+    std::snprintf(t_error, sizeof t_error, "%s: launch failed: %s", name, cudaGetErrorString(err));
+    return AKG_ERR_CUDA;
+  }
+  const char* dt = (c.dtype == AKG_F32) ? "f32" : "bf16";
+  if (plan.variant == V_REG)
+    std::snprintf(t_kernel, sizeof t_kernel, "reg<%s,g%d,t%d,v%d>", dt, plan.group, plan.threads, plan.vpt);
+  else if (plan.variant == V_TMA || plan.variant == V_CLUSTER)
+    std::snprintf(t_kernel, sizeof t_kernel, "%s<%s,t%d,cs%d,nbuf%d,slice%d>",
+                  plan.variant == V_TMA ? "tma" : "cluster", dt, plan.threads, plan.cluster, plan.stages, plan.vpt);
+  else
+    std::snprintf(t_kernel, sizeof t_kernel, "stream<%s,t%d>", dt, plan.threads);
+  return AKG_OK;
+}
+
+}  // namespace
+}  // namespace akg
+
+using namespace akg;
+
+extern "C" {
+
+akg_status akg_softmax(const void* x, void* y, int64_t rows, int64_t cols, int64_t x_row_stride,
+                       int64_t y_row_stride, akg_dtype dtype, const akg_mask* mask, void* stream) {
+  Call c{OP_SOFTMAX, x, y, rows, cols, x_row_stride, y_row_stride, static_cast<int>(dtype), mask,
+         nullptr, nullptr, 0.f, stream};
+  return run(c, "akg_softmax");
+}
+
+akg_status akg_log_softmax(const void* x, void* y, int64_t rows, int64_t cols, int64_t x_row_stride,
+                           int64_t y_row_stride, akg_dtype dtype, const akg_mask* mask, void* stream) {
+  Call c{OP_LOG_SOFTMAX, x, y, rows, cols, x_row_stride, y_row_stride, static_cast<int>(dtype), mask,
+         nullptr, nullptr, 0.f, stream};
+  return run(c, "akg_log_softmax");
+}
+
+akg_status akg_layernorm(const void* x, void* y, int64_t rows, int64_t cols, int64_t x_row_stride,
+                         int64_t y_row_stride, akg_dtype dtype, const void* gamma, const void* beta,
+                         float eps, void* stream) {
+  Call c{OP_LAYERNORM, x, y, rows, cols, x_row_stride, y_row_stride, static_cast<int>(dtype), nullptr,
+         gamma, beta, eps, stream};
+  return run(c, "akg_layernorm");
+}
+
+akg_status akg_rmsnorm(const void* x, void* y, int64_t rows, int64_t cols, int64_t x_row_stride,
+                       int64_t y_row_stride, akg_dtype dtype, const void* weight, float eps, void* stream) {
+  Call c{OP_RMSNORM, x, y, rows, cols, x_row_stride, y_row_stride, static_cast<int>(dtype), nullptr,
+         weight, nullptr, eps, stream};
+  return run(c, "akg_rmsnorm");
+}
+
+const char* akg_status_string(akg_status status) {
+  switch (status) {
+    case AKG_OK: return "AKG_OK";
+    case AKG_ERR_INVALID_ARG: return "AKG_ERR_INVALID_ARG";
+    case AKG_ERR_UNSUPPORTED: return "AKG_ERR_UNSUPPORTED";
+    case AKG_ERR_CUDA: return "AKG_ERR_CUDA";
+    case AKG_ERR_DEVICE_TIMEOUT: return "AKG_ERR_DEVICE_TIMEOUT";
+  }
+  return "AKG_ERR_UNKNOWN";
+}
+
+const char* akg_last_error_string(void) { return t_error; }
+
+int akg_version(void) { return 100; }
+
+akg_status akg_set_variant(akg_variant variant) {
+  if (variant < AKG_VARIANT_AUTO || variant > AKG_VARIANT_CLUSTER)
+    return fail(AKG_ERR_INVALID_ARG, "%s: unknown variant", "akg_set_variant");
+  g_forced_variant.store(static_cast<int>(variant));
+  return AKG_OK;
+}
+
+akg_status akg_set_tuning(const char* key, int value) {
+  if (key == nullptr) return fail(AKG_ERR_INVALID_ARG, "%s: NULL key", "akg_set_tuning");
+  if (!std::strcmp(key, "reg_threads")) g_tune_reg_threads.store(value);
+  else if (!std::strcmp(key, "reg_vpt")) g_tune_reg_vpt.store(value);
+  else if (!std::strcmp(key, "reg_group")) g_tune_reg_group.store(value);
+  else if (!std::strcmp(key, "grid_cap")) g_tune_grid_cap.store(value);
+  else if (!std::strcmp(key, "cluster_size")) g_tune_cluster_size.store(value);
+  else if (!std::strcmp(key, "smem_nbuf")) g_tune_smem_nbuf.store(value);
+  else if (!std::strcmp(key, "smem_threads")) g_tune_smem_threads.store(value);
+  else if (!std::strcmp(key, "smem_ctas")) g_tune_smem_ctas.store(value);
+  else return fail(AKG_ERR_INVALID_ARG, "akg_set_tuning: unknown key %s", key);
+  return AKG_OK;
+}
+
+const char* akg_last_kernel_name(void) { return t_kernel; }
+
+akg_status akg_device_status(int* word_out) {
+  int word = 0;
+  cudaError_t err = cudaMemcpyFromSymbol(&word, g_status_word, sizeof(int));
+  if (err == cudaSuccess && word != 0) {
+    const int zero = 0;
+    err = cudaMemcpyToSymbol(g_status_word, &zero, sizeof(int));
+  }
+  if (err != cudaSuccess) {
+    (void)cudaGetLastError();
+    return fail(AKG_ERR_CUDA, "akg_device_status: %s", cudaGetErrorString(err));
+  }
+  if (word_out) *word_out = word;
+  return word == 0 ? AKG_OK : AKG_ERR_DEVICE_TIMEOUT;
+}
+
+}  // extern "C"

@@ -1,0 +1,263 @@
+// Device-side building blocks shared by every kernel family of the row-operator
+// library: parameter block, element packing, streaming loads / stores, and the
+// per-operator statistics (online max / rescaled sum for the softmax pair,
+// count-mean-M2 with Chan's merge for LayerNorm, sum of squares for RMSNorm).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace akg {
+
+enum Op : int { OP_SOFTMAX = 0, OP_LOG_SOFTMAX = 1, OP_LAYERNORM = 2, OP_RMSNORM = 3 };
+enum DType : int { DT_F32 = 0, DT_BF16 = 1 };
+
+// One operator call.  Strides in elements.  gamma doubles as the RMSNorm weight.
+struct RowParams {
+  const void* x;
+  void* y;
+  long long rows, cols, xs, ys;
+  const void* gamma;
+  const void* beta;
+  float eps;
+  const void* add;          // additive mask or nullptr
+  long long add_rows, add_stride;
+  int causal;
+  long long period, offset;
+  int period_pow2;          // 1: period is a power of two (row & (period - 1))
+  int add_mode;             // 0: row % add_rows, 1: add_rows == 1, 2: add_rows >= rows
+  int* status;              // device status word (bounded waits report here)
+};
+
+// Shared-memory ring kernels: limits and the size of the bookkeeping area that
+// precedes the ring buffers (mbarriers, CTA reduction slots, cluster exchange slots).
+constexpr int kMaxCluster = 16;
+constexpr int kMaxBuf = 16;
+constexpr unsigned kMaxDynSmem = 232448;      // 227 KiB opt-in limit per CTA
+__host__ __device__ constexpr unsigned smem_header_bytes(int threads) {
+  return (kMaxBuf * 8u + (2u * (threads / 32) + 2u * kMaxCluster) * 12u + 127u) & ~127u;
+}
+
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kNegInf = -__builtin_huge_valf();
+
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+// e^(a - b) for a <= b (or NaN / inf operands, which propagate as IEEE says)
+__device__ __forceinline__ float exp_diff(float a, float b) { return ex2_approx((a - b) * kLog2e); }
+
+// 128-bit streaming accesses: the row data is touched once, keep it out of L1.
+__device__ __forceinline__ uint4 ld_stream(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_stream(void* p, const uint4& v) {
+  asm volatile("st.global.cs.v4.u32 [%0], {%1, %2, %3, %4};"
+               :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+// read-only, cached (gamma / beta / weight are reused by every row)
+__device__ __forceinline__ uint4 ld_cached(const void* p) {
+  return __ldg(reinterpret_cast<const uint4*>(p));
+}
+
+template <typename T> struct Elem;
+
+template <> struct Elem<float> {
+  static constexpr int EPV = 4;                    // elements per 16-byte vector
+  static constexpr int DT = DT_F32;
+  static __device__ __forceinline__ void unpack(const uint4& u, float (&f)[4]) {
+    f[0] = __uint_as_float(u.x); f[1] = __uint_as_float(u.y);
+    f[2] = __uint_as_float(u.z); f[3] = __uint_as_float(u.w);
+  }
+  static __device__ __forceinline__ uint4 pack(const float (&f)[4]) {
+    return make_uint4(__float_as_uint(f[0]), __float_as_uint(f[1]),
+                      __float_as_uint(f[2]), __float_as_uint(f[3]));
+  }
+  static __device__ __forceinline__ float load1(const void* base, long long i) {
+    return reinterpret_cast<const float*>(base)[i];
+  }
+  static __device__ __forceinline__ void store1(void* base, long long i, float v) {
+    reinterpret_cast<float*>(base)[i] = v;
+  }
+};
+
+template <> struct Elem<__nv_bfloat16> {
+  static constexpr int EPV = 8;
+  static constexpr int DT = DT_BF16;
+  static __device__ __forceinline__ void unpack(const uint4& u, float (&f)[8]) {
+    const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      f[2 * i] = __uint_as_float(w[i] << 16);            // low half = even element
+      f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+  }
+  static __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
+    __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);   // round-to-nearest-even, once
+    return *reinterpret_cast<uint32_t*>(&h);
+  }
+  static __device__ __forceinline__ uint4 pack(const float (&f)[8]) {
+    return make_uint4(pack2(f[0], f[1]), pack2(f[2], f[3]), pack2(f[4], f[5]), pack2(f[6], f[7]));
+  }
+  static __device__ __forceinline__ float load1(const void* base, long long i) {
+    return __uint_as_float(static_cast<uint32_t>(reinterpret_cast<const uint16_t*>(base)[i]) << 16);
+  }
+  static __device__ __forceinline__ void store1(void* base, long long i, float v) {
+    reinterpret_cast<__nv_bfloat16*>(base)[i] = __float2bfloat16_rn(v);
+  }
+};
+
+template <int OP> struct OpTraits {
+  static constexpr bool kSoftmaxLike = (OP == OP_SOFTMAX || OP == OP_LOG_SOFTMAX);
+};
+
+// Number of leading live columns of a row (the rest is masked by the causal rule).
+__device__ __forceinline__ long long live_cols(const RowParams& p, long long row) {
+  if (!p.causal) return p.cols;
+  const long long rp = p.period_pow2 ? (row & (p.period - 1)) : (row % p.period);
+  long long l = rp + p.offset + 1;
+  return l < 0 ? 0 : (l > p.cols ? p.cols : l);
+}
+
+// Row of the additive mask that row `row` uses.
+__device__ __forceinline__ long long add_row(const RowParams& p, long long row) {
+  return p.add_mode == 1 ? 0 : (p.add_mode == 2 ? row : row % p.add_rows);
+}
+
+// ---------------------------------------------------------------------------------
+// Per-row statistics.  Field use:
+//   softmax pair : a = running max m, b = sum of exp(z - m)
+//   LayerNorm    : a = count, b = mean, c = sum of squared deviations (M2)
+//   RMSNorm      : a = sum of squares
+// ---------------------------------------------------------------------------------
+struct Stat { float a, b, c; };
+
+template <int OP> __device__ __forceinline__ Stat stat_identity() {
+  if (OpTraits<OP>::kSoftmaxLike) return Stat{kNegInf, 0.f, 0.f};
+  return Stat{0.f, 0.f, 0.f};
+}
+
+template <int OP> __device__ __forceinline__ Stat stat_merge(const Stat& x, const Stat& y) {
+  Stat r;
+  if (OpTraits<OP>::kSoftmaxLike) {
+    // (m, s) (+) (m', s') = (M, s e^(m-M) + s' e^(m'-M)); equal maxima (also both
+    // -inf, or both +inf) take factor 1 so that no inf - inf is formed here.
+    const float M = fmaxf(x.a, y.a);
+    const float fx = (x.a == M) ? 1.f : exp_diff(x.a, M);
+    const float fy = (y.a == M) ? 1.f : exp_diff(y.a, M);
+    r.a = M; r.b = x.b * fx + y.b * fy; r.c = 0.f;
+  } else if (OP == OP_LAYERNORM) {
+    // Chan's pairwise update of (count, mean, M2)
+    const float n = x.a + y.a;
+    const float w = (n > 0.f) ? __fdividef(y.a, n) : 0.f;
+    const float d = y.b - x.b;
+    r.a = n; r.b = x.b + d * w; r.c = x.c + y.c + d * d * x.a * w;
+  } else {
+    r.a = x.a + y.a; r.b = 0.f; r.c = 0.f;
+  }
+  return r;
+}
+
+template <int OP> __device__ __forceinline__ Stat stat_shfl_xor(const Stat& s, int lane_mask) {
+  Stat r;
+  r.a = __shfl_xor_sync(0xffffffffu, s.a, lane_mask);
+  r.b = (OP != OP_RMSNORM) ? __shfl_xor_sync(0xffffffffu, s.b, lane_mask) : 0.f;
+  r.c = (OP == OP_LAYERNORM) ? __shfl_xor_sync(0xffffffffu, s.c, lane_mask) : 0.f;
+  return r;
+}
+
+template <int OP> __device__ __forceinline__ Stat warp_reduce(Stat s) {
+#pragma unroll
+  for (int m = 16; m >= 1; m >>= 1) s = stat_merge<OP>(s, stat_shfl_xor<OP>(s, m));
+  return s;
+}
+
+// Reduce over a whole CTA of NW warps.  `slots` points at NW Stat entries of shared
+// memory reserved for this call; callers alternate between two slot sets on
+// successive rows so one barrier per row is enough.  Every thread gets the result,
+// combined in the same order, hence bit-identical across the CTA.
+template <int OP, int NW> __device__ __forceinline__ Stat cta_reduce(Stat s, Stat* slots) {
+  s = warp_reduce<OP>(s);
+  if (NW == 1) return s;
+  if ((threadIdx.x & 31) == 0) slots[threadIdx.x >> 5] = s;
+  __syncthreads();
+  Stat r = slots[0];
+#pragma unroll
+  for (int w = 1; w < NW; ++w) r = stat_merge<OP>(r, slots[w]);
+  return r;
+}
+
+// Row scalars derived from the reduced statistics.
+//   softmax     : p = M (row max, or 0 if no live entry), q = 1 / S (0 if no live entry)
+//   log-softmax : p = M, q = ln S; dead = no live entry
+//   LayerNorm   : p = mean, q = 1 / sqrt(var + eps)
+//   RMSNorm     : q = 1 / sqrt(mean square + eps)
+struct RowScalars { float p, q; bool dead; };
+
+template <int OP> __device__ __forceinline__ RowScalars finalize(const Stat& s, long long cols, float eps) {
+  RowScalars r;
+  r.dead = false;
+  if (OP == OP_SOFTMAX) {
+    r.dead = (s.a == kNegInf);
+    r.p = r.dead ? 0.f : s.a;
+    r.q = r.dead ? 0.f : 1.0f / s.b;
+  } else if (OP == OP_LOG_SOFTMAX) {
+    r.dead = (s.a == kNegInf);
+    r.p = s.a;
+    r.q = logf(s.b);
+  } else if (OP == OP_LAYERNORM) {
+    r.p = s.b;
+    r.q = 1.0f / sqrtf(s.c / static_cast<float>(cols) + eps);
+  } else {
+    r.p = 0.f;
+    r.q = 1.0f / sqrtf(s.a / static_cast<float>(cols) + eps);
+  }
+  return r;
+}
+
+// Statistics of a register tile of N already-masked values (n_valid of them count).
+// For softmax the values are replaced by exp(z - m_local) so that the exponential
+// is evaluated once per element; the caller later scales by exp(m_local - M) / S.
+template <int OP, int N>
+__device__ __forceinline__ Stat tile_stats(float (&v)[N], int n_valid, float& m_local) {
+  Stat s = stat_identity<OP>();
+  m_local = 0.f;
+  if (OpTraits<OP>::kSoftmaxLike) {
+    float m = kNegInf;
+#pragma unroll
+    for (int i = 0; i < N; ++i) m = fmaxf(m, v[i]);
+    const float ms = (m == kNegInf) ? 0.f : m;      // keeps -inf - -inf out of the exponent
+    float acc = 0.f;
+#pragma unroll
+    for (int i = 0; i < N; ++i) {
+      const float e = exp_diff(v[i], ms);
+      acc += e;
+      if (OP == OP_SOFTMAX) v[i] = e;
+    }
+    s.a = m; s.b = acc; m_local = m;
+  } else if (OP == OP_LAYERNORM) {
+    float sum = 0.f;
+#pragma unroll
+    for (int i = 0; i < N; ++i) sum += (i < n_valid) ? v[i] : 0.f;
+    const float n = static_cast<float>(n_valid);
+    const float mean = (n_valid > 0) ? sum / n : 0.f;
+    float m2 = 0.f;
+#pragma unroll
+    for (int i = 0; i < N; ++i) { const float d = v[i] - mean; m2 += (i < n_valid) ? d * d : 0.f; }
+    s.a = n; s.b = mean; s.c = m2;
+  } else {
+    float ss = 0.f;
+#pragma unroll
+    for (int i = 0; i < N; ++i) ss += (i < n_valid) ? v[i] * v[i] : 0.f;
+    s.a = ss;
+  }
+  return s;
+}
+
+}  // namespace akg

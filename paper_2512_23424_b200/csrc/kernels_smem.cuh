@@ -1,0 +1,276 @@
+// smem_kernel: rows staged in shared memory by the bulk-copy engine (TMA, untiled
+// cp.async.bulk, no multicast), for rows that do not fit the register file.
+//
+// A cluster of CS CTAs (CS = 1 for the "TMA" family, 2..16 for the "CLUSTER" family)
+// owns one row at a time; CTA k of the cluster keeps slice k of the row in shared
+// memory.  Each CTA has a ring of NBUF slice buffers: while the slice of row i is being
+// reduced, normalised and stored, the copies for rows i+1 .. i+NBUF-1 are in flight.
+// Per row: wait for the slice -> pass 1 over shared memory (thread-local statistics)
+// -> CTA reduction -> partial statistics written into every peer's shared memory
+// (distributed shared memory) -> cluster barrier -> pass 2 over shared memory
+// (normalise, 128-bit stores) -> refill the buffer.  HBM traffic stays at one read and
+// one write per element; 12 bytes per CTA cross the cluster per row.
+#pragma once
+
+#include "kernels_basic.cuh"
+
+namespace akg {
+
+
+
+constexpr uint32_t kWaitLimit = 1u << 22;     // bounded mbarrier wait (each try blocks for a while)
+constexpr int kStatusTimeout = 1;
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+               "selp.u32 %0, 1, 0, p;\n\t}" : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Wait for a phase with an iteration limit; on expiry the status word is set and the
+// caller carries on (its output for that row is then undefined, never out of bounds).
+__device__ __forceinline__ void mbar_wait_bounded(uint32_t bar, uint32_t parity, int* status) {
+  for (uint32_t i = 0; i < kWaitLimit; ++i)
+    if (mbar_try_wait(bar, parity)) return;
+  if (status != nullptr) atomicExch(status, kStatusTimeout);
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               :: "r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t cluster_rank() {
+  uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r;
+}
+__device__ __forceinline__ uint32_t cluster_size() {
+  uint32_t r; asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r)); return r;
+}
+__device__ __forceinline__ uint32_t cluster_id() {
+  uint32_t r; asm volatile("mov.u32 %0, %%clusterid.x;" : "=r"(r)); return r;
+}
+__device__ __forceinline__ uint32_t cluster_count() {
+  uint32_t r; asm volatile("mov.u32 %0, %%nclusterid.x;" : "=r"(r)); return r;
+}
+__device__ __forceinline__ void cluster_arrive() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void cluster_wait() {
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void st_remote_f32(uint32_t local_addr, uint32_t rank, float v) {
+  uint32_t remote;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
+  asm volatile("st.shared::cluster.f32 [%0], %1;" :: "r"(remote), "f"(v) : "memory");
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+  return v;
+}
+
+// Fold one vector of EPV (masked) values into the running thread statistics.
+template <int OP, int EPV>
+__device__ __forceinline__ void fold_vector(Stat& st, const float (&z)[EPV]) {
+  if (OpTraits<OP>::kSoftmaxLike) {
+    float mv = z[0];
+#pragma unroll
+    for (int j = 1; j < EPV; ++j) mv = fmaxf(mv, z[j]);
+    const float mn = fmaxf(st.a, mv);
+    const float ms = (mn == kNegInf) ? 0.f : mn;
+    float acc = st.b * exp_diff(st.a, ms);
+#pragma unroll
+    for (int j = 0; j < EPV; ++j) acc += exp_diff(z[j], ms);
+    st.a = mn; st.b = acc;
+  } else if (OP == OP_LAYERNORM) {
+    float sum = 0.f;
+#pragma unroll
+    for (int j = 0; j < EPV; ++j) sum += z[j];
+    const float mean = sum * (1.0f / EPV);
+    float m2 = 0.f;
+#pragma unroll
+    for (int j = 0; j < EPV; ++j) { const float d = z[j] - mean; m2 += d * d; }
+    st = stat_merge<OP>(st, Stat{static_cast<float>(EPV), mean, m2});
+  } else {
+#pragma unroll
+    for (int j = 0; j < EPV; ++j) st.a += z[j] * z[j];
+  }
+}
+
+struct SmemGeom {
+  int nbuf;               // ring depth
+  int slice_vecs;         // 16-byte vectors per CTA slice (last slice may be shorter)
+  unsigned buf_bytes;     // bytes reserved per ring buffer (multiple of 128)
+};
+
+template <int OP, typename T, int THREADS>
+__global__ void __launch_bounds__(THREADS) smem_kernel(const RowParams p, const SmemGeom g) {
+  using E = Elem<T>;
+  constexpr int EPV = E::EPV;
+  constexpr int NW = THREADS / 32;
+  constexpr bool SM = OpTraits<OP>::kSoftmaxLike;
+
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem_raw);                       // [kMaxBuf]
+  Stat* red = reinterpret_cast<Stat*>(smem_raw + kMaxBuf * sizeof(uint64_t));    // [2][NW]
+  Stat* peers = red + 2 * NW;                                                     // [2][kMaxCluster]
+  constexpr unsigned kHeader = smem_header_bytes(THREADS);
+  unsigned char* bufs = smem_raw + kHeader;
+
+  const uint32_t cs = cluster_size();
+  const uint32_t rank = cluster_rank();
+  const long long first_row = cluster_id();
+  const long long row_step = cluster_count();
+  const int nvec = static_cast<int>(p.cols / EPV);
+  const int v0 = static_cast<int>(rank) * g.slice_vecs;                          // my first vector
+  const int my_vecs = max(0, min(g.slice_vecs, nvec - v0));
+
+  if (threadIdx.x == 0) {
+    for (int b = 0; b < g.nbuf; ++b) mbar_init(smem_addr(&bars[b]), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if (cs > 1) {            // every CTA of the cluster is running before any remote store
+    cluster_arrive();
+    cluster_wait();
+  }
+
+  // number of live vectors of my slice for a given row
+  auto live_in_slice = [&](long long row, int& live) -> int {
+    live = SM ? static_cast<int>(live_cols(p, row)) : static_cast<int>(p.cols);
+    const int live_vecs = (live + EPV - 1) / EPV;
+    return max(0, min(my_vecs, live_vecs - v0));
+  };
+  auto issue = [&](long long row, int b) {
+    int live;
+    const int lv = live_in_slice(row, live);
+    const uint32_t bar = smem_addr(&bars[b]);
+    if (lv == 0) {
+      // nothing to fetch (slice fully masked): complete the phase so parities stay in step
+      asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(bar) : "memory");
+    } else {
+      const uint32_t bytes = static_cast<uint32_t>(lv) * 16u;
+      mbar_expect_tx(bar, bytes);
+      const unsigned char* src = reinterpret_cast<const unsigned char*>(
+          reinterpret_cast<const T*>(p.x) + row * p.xs + static_cast<long long>(v0) * EPV);
+      const uint32_t dst = smem_addr(bufs + static_cast<size_t>(b) * g.buf_bytes);
+      constexpr uint32_t kChunk = 32768;
+      for (uint32_t off = 0; off < bytes; off += kChunk)
+        bulk_load(dst + off, src + off, min(kChunk, bytes - off), bar);
+    }
+  };
+
+  if (threadIdx.x == 0) {
+    long long r = first_row;
+    for (int b = 0; b < g.nbuf && r < p.rows; ++b, r += row_step) issue(r, b);
+  }
+
+  long long it = 0;
+  for (long long row = first_row; row < p.rows; row += row_step, ++it) {
+    const int b = static_cast<int>(it % g.nbuf);
+    const uint32_t phase = static_cast<uint32_t>((it / g.nbuf) & 1);
+    const int par = static_cast<int>(it & 1);
+    int live;
+    const int lv = live_in_slice(row, live);
+    const uint32_t buf = smem_addr(bufs + static_cast<size_t>(b) * g.buf_bytes);
+    const T* ar = (SM && p.add != nullptr)
+                      ? reinterpret_cast<const T*>(p.add) + add_row(p, row) * p.add_stride
+                      : nullptr;
+    mbar_wait_bounded(smem_addr(&bars[b]), phase, p.status);
+
+    // ---- pass 1: thread-local statistics over my slice
+    Stat st = stat_identity<OP>();
+    for (int v = threadIdx.x; v < lv; v += THREADS) {
+      float z[EPV];
+      E::unpack(lds128(buf + static_cast<uint32_t>(v) * 16u), z);
+      if (SM) {
+        const int c0 = (v0 + v) * EPV;
+        if (ar != nullptr) {
+          float a[EPV];
+          E::unpack(ld_stream(ar + c0), a);
+#pragma unroll
+          for (int j = 0; j < EPV; ++j) z[j] += a[j];
+        }
+        if (c0 + EPV > live) {
+#pragma unroll
+          for (int j = 0; j < EPV; ++j) if (c0 + j >= live) z[j] = kNegInf;
+        }
+      }
+      fold_vector<OP, EPV>(st, z);
+    }
+    st = cta_reduce<OP, NW>(st, red + par * NW);
+
+    // ---- combine across the cluster through distributed shared memory
+    if (cs > 1) {
+      if (threadIdx.x < cs) {
+        const uint32_t slot = smem_addr(&peers[par * kMaxCluster + rank]);
+        st_remote_f32(slot, threadIdx.x, st.a);
+        st_remote_f32(slot + 4, threadIdx.x, st.b);
+        st_remote_f32(slot + 8, threadIdx.x, st.c);
+      }
+      cluster_arrive();
+      cluster_wait();
+      Stat r = peers[par * kMaxCluster];
+      for (uint32_t k = 1; k < cs; ++k) r = stat_merge<OP>(r, peers[par * kMaxCluster + k]);
+      st = r;
+    }
+    const RowScalars rs = finalize<OP>(st, p.cols, p.eps);
+    const float fill = SM ? masked_fill<OP>(rs) : 0.f;
+
+    // ---- pass 2: normalise from shared memory, 128-bit stores
+    T* yr = reinterpret_cast<T*>(p.y) + row * p.ys + static_cast<long long>(v0) * EPV;
+    for (int v = threadIdx.x; v < my_vecs; v += THREADS) {
+      float o[EPV];
+      if (v < lv) {
+        float z[EPV];
+        E::unpack(lds128(buf + static_cast<uint32_t>(v) * 16u), z);
+        const int c0 = (v0 + v) * EPV;
+        float ga[EPV], be[EPV];
+#pragma unroll
+        for (int j = 0; j < EPV; ++j) { ga[j] = 1.f; be[j] = 0.f; }
+        if (SM) {
+          if (ar != nullptr) {
+            float a[EPV];
+            E::unpack(ld_stream(ar + c0), a);
+#pragma unroll
+            for (int j = 0; j < EPV; ++j) z[j] += a[j];
+          }
+        } else {
+          if (p.gamma != nullptr) E::unpack(ld_cached(reinterpret_cast<const T*>(p.gamma) + c0), ga);
+          if (OP == OP_LAYERNORM && p.beta != nullptr)
+            E::unpack(ld_cached(reinterpret_cast<const T*>(p.beta) + c0), be);
+        }
+#pragma unroll
+        for (int j = 0; j < EPV; ++j) {
+          if (SM && c0 + j >= live) o[j] = fill;
+          else if (OP == OP_SOFTMAX) o[j] = exp_diff(z[j], rs.p) * rs.q;
+          else o[j] = apply_one<OP>(z[j], rs, 0.f, ga[j], be[j]);
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < EPV; ++j) o[j] = fill;
+      }
+      st_stream(yr + static_cast<long long>(v) * EPV, E::pack(o));
+    }
+
+    // ---- the buffer is free once every thread has read it: refill for row it + nbuf
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      const long long next = row + row_step * g.nbuf;
+      if (next < p.rows) issue(next, b);
+    }
+  }
+  // Peers write into this CTA's shared memory only before the cluster barrier of a row
+  // this CTA also takes part in, so leaving after the last row is safe; every bulk copy
+  // issued was waited for above (each issued row is consumed by the loop).
+}
+
+}  // namespace akg

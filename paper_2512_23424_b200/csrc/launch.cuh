@@ -1,0 +1,33 @@
+// Host-side launch plan and the per-operator launcher template.  Each operator's
+// translation unit instantiates launch_op<OP> once, so the four operators compile in
+// parallel; api.cu sees only the declarations.
+#pragma once
+
+#include <cuda_runtime.h>
+
+#include "common.cuh"
+
+namespace akg {
+
+enum Variant : int { V_AUTO = 0, V_STREAM = 1, V_REG = 2, V_TMA = 3, V_CLUSTER = 4 };
+
+struct LaunchPlan {
+  int variant;        // V_STREAM .. V_CLUSTER
+  int threads;        // CTA size
+  int group;          // threads per row (32 or threads) for V_REG
+  int vpt;            // 16-byte vectors per thread for V_REG
+  unsigned grid;      // CTAs (V_CLUSTER: a multiple of cluster)
+  int cluster;        // CTAs per cluster (V_CLUSTER), else 1
+  int stages;         // ring depth (V_TMA)
+  size_t smem;        // dynamic shared memory per CTA
+};
+
+template <int OP>
+cudaError_t launch_op(const LaunchPlan& plan, int dtype, const RowParams& p, cudaStream_t stream);
+
+extern template cudaError_t launch_op<OP_SOFTMAX>(const LaunchPlan&, int, const RowParams&, cudaStream_t);
+extern template cudaError_t launch_op<OP_LOG_SOFTMAX>(const LaunchPlan&, int, const RowParams&, cudaStream_t);
+extern template cudaError_t launch_op<OP_LAYERNORM>(const LaunchPlan&, int, const RowParams&, cudaStream_t);
+extern template cudaError_t launch_op<OP_RMSNORM>(const LaunchPlan&, int, const RowParams&, cudaStream_t);
+
+}  // namespace akg

@@ -1,0 +1,110 @@
+// Definition of launch_op<OP>; included only by the per-operator translation units.
+#pragma once
+
+#include <map>
+#include <mutex>
+#include <tuple>
+
+#include "kernels_basic.cuh"
+#include "kernels_smem.cuh"
+#include "launch.cuh"
+
+namespace akg {
+
+// The (threads-per-row, vectors-per-thread, CTA size) shapes reg_kernel is built for.
+// api.cu's planner only ever asks for one of these.
+#define AKG_REG_SHAPES(X) \
+  X(32, 1, 128) X(32, 2, 128) X(32, 4, 128) X(32, 8, 128) \
+  X(128, 1, 128) X(128, 2, 128) X(128, 4, 128) \
+  X(256, 1, 256) X(256, 2, 256) X(256, 4, 256) \
+  X(512, 4, 512) X(512, 8, 512) X(1024, 4, 1024) X(1024, 8, 1024)
+
+// Launch smem_kernel (TMA ring, optionally clustered).  plan.grid == 0 asks for as many
+// clusters as can be co-resident (capped by the number of rows).
+template <int OP, typename T, int THREADS>
+cudaError_t launch_smem(const LaunchPlan& plan, const RowParams& p, cudaStream_t s) {
+  auto kernel = smem_kernel<OP, T, THREADS>;
+  static std::mutex mu;
+  static std::map<std::tuple<int, int, size_t>, int> resident;   // (device, cluster, smem) -> clusters
+  static std::map<int, bool> prepared;                             // device -> attributes set
+  int dev = 0;
+  cudaError_t err = cudaGetDevice(&dev);
+  if (err != cudaSuccess) return err;
+
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = static_cast<unsigned>(plan.cluster);
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.blockDim = dim3(THREADS);
+  cfg.dynamicSmemBytes = plan.smem;
+  cfg.stream = s;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+
+  int max_clusters = 0;
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    if (!prepared[dev]) {
+      err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448);
+      if (err != cudaSuccess) return err;
+      err = cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+      if (err != cudaSuccess) return err;
+      prepared[dev] = true;
+    }
+    auto key = std::make_tuple(dev, plan.cluster, plan.smem);
+    auto it = resident.find(key);
+    if (it == resident.end()) {
+      cfg.gridDim = dim3(static_cast<unsigned>(plan.cluster) * 1024u);
+      int n = 0;
+      err = cudaOccupancyMaxActiveClusters(&n, kernel, &cfg);
+      if (err != cudaSuccess) return err;
+      it = resident.emplace(key, n).first;
+    }
+    max_clusters = it->second;
+  }
+  if (max_clusters < 1) return cudaErrorLaunchOutOfResources;
+  long long clusters = plan.grid ? plan.grid / plan.cluster : max_clusters;
+  if (clusters > p.rows) clusters = p.rows;
+  if (clusters < 1) clusters = 1;
+  cfg.gridDim = dim3(static_cast<unsigned>(clusters * plan.cluster));
+  SmemGeom g;
+  g.nbuf = plan.stages;
+  g.slice_vecs = plan.vpt;          // V_TMA / V_CLUSTER reuse the field: vectors per CTA slice
+  g.buf_bytes = static_cast<unsigned>((static_cast<size_t>(plan.vpt) * 16 + 127) & ~static_cast<size_t>(127));
+  return cudaLaunchKernelEx(&cfg, kernel, p, g);
+}
+
+template <int OP, typename T>
+cudaError_t launch_typed(const LaunchPlan& plan, const RowParams& p, cudaStream_t s) {
+  if (plan.variant == V_STREAM) {
+    stream_kernel<OP, T, 256><<<plan.grid, 256, 0, s>>>(p);
+    return cudaGetLastError();
+  }
+  if (plan.variant == V_REG) {
+#define AKG_REG_CASE(G_, V_, T_)                                              \
+  if (plan.group == (G_) && plan.vpt == (V_) && plan.threads == (T_)) {       \
+    reg_kernel<OP, T, G_, V_, T_><<<plan.grid, T_, 0, s>>>(p);                \
+    return cudaGetLastError();                                                \
+  }
+    AKG_REG_SHAPES(AKG_REG_CASE)
+#undef AKG_REG_CASE
+    return cudaErrorInvalidConfiguration;
+  }
+  if (plan.variant == V_TMA || plan.variant == V_CLUSTER) {
+    if (plan.threads == 256) return launch_smem<OP, T, 256>(plan, p, s);
+    if (plan.threads == 512) return launch_smem<OP, T, 512>(plan, p, s);
+    if (plan.threads == 1024) return launch_smem<OP, T, 1024>(plan, p, s);
+    return cudaErrorInvalidConfiguration;
+  }
+  return cudaErrorInvalidConfiguration;
+}
+
+template <int OP>
+cudaError_t launch_op(const LaunchPlan& plan, int dtype, const RowParams& p, cudaStream_t stream) {
+  if (dtype == DT_F32) return launch_typed<OP, float>(plan, p, stream);
+  return launch_typed<OP, __nv_bfloat16>(plan, p, stream);
+}
+
+}  // namespace akg
