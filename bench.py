@@ -392,6 +392,25 @@ def run_reference(args):
     }))
 
 
+def run_profile(args):
+    """Bare launches of one configuration (for a profiler): warm-up + steps launches of
+    the operator on resident inputs, nothing else.  --profile-rows truncates the rows."""
+    import torch
+    from paper_2512_23424_b200 import binding
+    torch.cuda.set_device(0)
+    w = wl.make_config(args.profile, rows=args.profile_rows)
+    if args.variant:
+        binding.set_variant(args.variant)
+    for item in filter(None, args.tune.split(",")):
+        key, _, val = item.partition("=")
+        binding.set_tuning(key, int(val))
+    dw = DeviceWorkload(w, pairs_for(w) if args.profile_rows is None else 1)
+    secs = time_launches(dw, args.steps, args.warmup)
+    print(json.dumps({"profile": wl.CONFIG_NAMES[args.profile], "rows": w.rows, "kernel": binding.last_kernel(),
+                      "us_per_launch": secs / args.steps * 1e6, "launches": args.steps + max(args.warmup, 3),
+                      "algorithmic_bytes": w.algorithmic_bytes()}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -400,8 +419,15 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--headline-only", action="store_true",
                     help="skip the per-configuration table (the headline line is unchanged)")
+    ap.add_argument("--profile", type=int, default=0, metavar="K",
+                    help="only launch configuration K (1..5) warmup+steps times, for use under ncu")
+    ap.add_argument("--profile-rows", type=int, default=None, help="truncate the rows of --profile")
+    ap.add_argument("--variant", default="", help="force a kernel family in --profile mode")
+    ap.add_argument("--tune", default="", help="--profile mode: key=value[,key=value] launch-geometry overrides")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.profile:
+        run_profile(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

@@ -23,6 +23,8 @@ std::atomic<int> g_tune_cluster_size{0};  // shared-memory ring family: CTAs per
 std::atomic<int> g_tune_smem_nbuf{0};     //   ring depth limit
 std::atomic<int> g_tune_smem_threads{0};  //   CTA size (256 / 512 / 1024)
 std::atomic<int> g_tune_smem_ctas{0};     //   CTAs per SM the ring is sized for
+std::atomic<int> g_tune_reg_general{0};   // 1 = never take the predicate-free normalisation kernel
+std::atomic<int> g_tune_cluster_mode{0};  // 0 = planner's choice, 1 = row resident in shared memory, 2 = two-pass split
 
 __device__ int g_status_word = 0;
 
@@ -127,7 +129,9 @@ bool plan_reg(const Call& c, LaunchPlan* plan) {
   if (cap > 0 && grid > cap) grid = cap;
   if (grid > INT_MAX) grid = INT_MAX;
   plan->variant = V_REG; plan->threads = threads; plan->group = group; plan->vpt = vpt;
-  plan->grid = static_cast<unsigned>(grid); plan->cluster = 1; plan->stages = 0; plan->smem = 0;
+  plan->grid = static_cast<unsigned>(grid); plan->cluster = 1; plan->smem = 0;
+  // a row of exactly group * vpt vectors takes the predicate-free normalisation kernel
+  plan->stages = (static_cast<int64_t>(group) * vpt == nvec && g_tune_reg_general.load() == 0) ? 1 : 0;
   return true;
 }
 
@@ -171,6 +175,25 @@ bool plan_smem(const Call& c, int cs_min, int cs_max, LaunchPlan* plan) {
   plan->smem = smem_header_bytes(best_threads) + static_cast<size_t>(best_nbuf) * buf;
   const int cap = g_tune_grid_cap.load();
   plan->grid = cap > 0 ? static_cast<unsigned>((cap / best_cs > 0 ? cap / best_cs : 1) * best_cs) : 0u;
+  return true;
+}
+
+// Two-pass split plan (cluster per row, second pass served by L2): any aligned row.
+// The cluster is sized so that every SM gets work even when there are few rows.
+bool plan_split(const Call& c, LaunchPlan* plan) {
+  const int64_t epv = (c.dtype == AKG_F32) ? 4 : 8;
+  const int64_t nvec = c.cols / epv;
+  const int t_cs = g_tune_cluster_size.load(), t_threads = g_tune_smem_threads.load();
+  int cs = t_cs > 0 ? t_cs : 8;
+  if (cs < 1 || cs > kMaxCluster || (cs & (cs - 1))) return false;
+  const int threads = t_threads > 0 ? t_threads : 256;
+  if (threads != 256 && threads != 512 && threads != 1024) return false;
+  while (cs > 1 && nvec / cs < threads) cs /= 2;          // keep at least one vector per thread
+  plan->variant = V_CLUSTER; plan->threads = threads; plan->group = threads;
+  plan->vpt = static_cast<int>((nvec + cs - 1) / cs);
+  plan->cluster = cs; plan->stages = 0; plan->smem = 0;
+  const int cap = g_tune_grid_cap.load();
+  plan->grid = cap > 0 ? static_cast<unsigned>((cap / cs > 0 ? cap / cs : 1) * cs) : 0u;
   return true;
 }
 
@@ -233,7 +256,8 @@ akg_status run(const Call& c, const char* name) {
   if (!planned && vec) {
     if (forced == V_AUTO) planned = plan_smem(c, 1, kMaxCluster, &plan);
     else if (forced == V_TMA) planned = plan_smem(c, 1, 1, &plan);
-    else if (forced == V_CLUSTER) planned = plan_smem(c, 2, kMaxCluster, &plan);
+    else if (forced == V_CLUSTER)
+      planned = (g_tune_cluster_mode.load() == 2) ? plan_split(c, &plan) : plan_smem(c, 2, kMaxCluster, &plan);
     if (planned) p.status = status_word_ptr();
   }
   if (!planned && (forced == V_AUTO || forced == V_STREAM)) { plan_stream(c, &plan); planned = true; }
@@ -254,10 +278,12 @@ akg_status run(const Call& c, const char* name) {
   }
   const char* dt = (c.dtype == AKG_F32) ? "f32" : "bf16";
   if (plan.variant == V_REG)
-    std::snprintf(t_kernel, sizeof t_kernel, "reg<%s,g%d,t%d,v%d>", dt, plan.group, plan.threads, plan.vpt);
+    std::snprintf(t_kernel, sizeof t_kernel, "reg<%s,g%d,t%d,v%d%s>", dt, plan.group, plan.threads, plan.vpt,
+                  (plan.stages == 1 && (c.op == OP_LAYERNORM || c.op == OP_RMSNORM)) ? ",full" : "");
   else if (plan.variant == V_TMA || plan.variant == V_CLUSTER)
     std::snprintf(t_kernel, sizeof t_kernel, "%s<%s,t%d,cs%d,nbuf%d,slice%d>",
-                  plan.variant == V_TMA ? "tma" : "cluster", dt, plan.threads, plan.cluster, plan.stages, plan.vpt);
+                  plan.variant == V_TMA ? "tma" : (plan.stages == 0 ? "split" : "cluster"), dt, plan.threads,
+                  plan.cluster, plan.stages, plan.vpt);
   else
     std::snprintf(t_kernel, sizeof t_kernel, "stream<%s,t%d>", dt, plan.threads);
   return AKG_OK;
@@ -331,6 +357,8 @@ akg_status akg_set_tuning(const char* key, int value) {
   else if (!std::strcmp(key, "smem_nbuf")) g_tune_smem_nbuf.store(value);
   else if (!std::strcmp(key, "smem_threads")) g_tune_smem_threads.store(value);
   else if (!std::strcmp(key, "smem_ctas")) g_tune_smem_ctas.store(value);
+  else if (!std::strcmp(key, "reg_general")) g_tune_reg_general.store(value);
+  else if (!std::strcmp(key, "cluster_mode")) g_tune_cluster_mode.store(value);
   else return fail(AKG_ERR_INVALID_ARG, "akg_set_tuning: unknown key %s", key);
   return AKG_OK;
 }

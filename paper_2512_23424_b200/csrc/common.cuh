@@ -204,11 +204,11 @@ template <int OP> __device__ __forceinline__ RowScalars finalize(const Stat& s, 
   RowScalars r;
   r.dead = false;
   if (OP == OP_SOFTMAX) {
-    r.dead = (s.a == kNegInf);
+    r.dead = (s.a == kNegInf) && !(s.b != s.b);   // a row of only NaN / -inf is a NaN row
     r.p = r.dead ? 0.f : s.a;
     r.q = r.dead ? 0.f : 1.0f / s.b;
   } else if (OP == OP_LOG_SOFTMAX) {
-    r.dead = (s.a == kNegInf);
+    r.dead = (s.a == kNegInf) && !(s.b != s.b);   // a row of only NaN / -inf is a NaN row
     r.p = s.a;
     r.q = logf(s.b);
   } else if (OP == OP_LAYERNORM) {

@@ -1,0 +1,159 @@
+// Lean register-resident kernels (the fast paths of the REG family).
+//
+//   reg_norm_full   LayerNorm / RMSNorm when the row is exactly G * VPT vectors: no
+//                   predicates, equal-count pairwise mean / M2 merges (no divisions),
+//                   one CTA barrier per row
+//   reg_softmax     softmax / log-softmax, any row that fits, optional additive and
+//                   causal mask: vectors beyond the live prefix are skipped with
+//                   CTA-uniform branches, the exponential is evaluated once per live
+//                   element against the warp maximum, and the cross-warp combine costs
+//                   one exponential per warp
+//
+// The instruction count per element is what bounds these kernels once the loads are
+// wide enough, so everything per-row (reductions, reciprocal, square root) is kept to
+// a few dozen instructions per thread.
+#pragma once
+
+#include "kernels_basic.cuh"
+
+namespace akg {
+
+// Occupancy target of the register-resident kernels: at least 1024 threads per SM, i.e.
+// at most 64 registers per thread (occupancy, not instruction count, bounds them next).
+template <int THREADS> constexpr int kRegMinBlocks = (1024 / THREADS) > 0 ? (1024 / THREADS) : 1;
+
+// 1 / sqrt(a): hardware approximation plus one Newton step (about 1 ulp).
+__device__ __forceinline__ float rsqrt_refined(float a) {
+  float r = rsqrtf(a);
+  if (a > 0.f && a < __int_as_float(0x7f800000)) r = r * (1.5f - 0.5f * a * r * r);
+  return r;
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int m = 16; m >= 1; m >>= 1) v += __shfl_xor_sync(0xffffffffu, v, m);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int m = 16; m >= 1; m >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, m));
+  return v;
+}
+
+// ------------------------------------------------------------------------------------
+// reg_norm_full
+// ------------------------------------------------------------------------------------
+template <int OP, typename T, int G, int VPT, int THREADS>
+__global__ void __launch_bounds__(THREADS, kRegMinBlocks<THREADS>) reg_norm_full(const RowParams p) {
+  using E = Elem<T>;
+  constexpr int EPV = E::EPV;
+  constexpr int N = VPT * EPV;
+  constexpr int RPC = THREADS / G;
+  constexpr int NW = G / 32;
+  static_assert(OP == OP_LAYERNORM || OP == OP_RMSNORM, "normalisations only");
+  static_assert((NW & (NW - 1)) == 0, "warps per row must be a power of two");
+  __shared__ float red[2][2][NW > 1 ? NW : 1];
+
+  const int tg = threadIdx.x % G;
+  const int grp = threadIdx.x / G;
+  const float inv_cols = 1.0f / static_cast<float>(N * G);
+  int parity = 0;
+
+  for (long long rb = static_cast<long long>(blockIdx.x) * RPC; rb < p.rows;
+       rb += static_cast<long long>(gridDim.x) * RPC, parity ^= 1) {
+    const long long row = rb + grp;
+    if (G != THREADS && row >= p.rows) continue;
+    const T* xr = reinterpret_cast<const T*>(p.x) + row * p.xs + tg * EPV;
+    T* yr = reinterpret_cast<T*>(p.y) + row * p.ys + tg * EPV;
+
+    uint4 raw[VPT];
+#pragma unroll
+    for (int k = 0; k < VPT; ++k) raw[k] = ld_stream(xr + k * G * EPV);
+    float v[N];
+#pragma unroll
+    for (int k = 0; k < VPT; ++k) {
+      float f[EPV];
+      E::unpack(raw[k], f);
+#pragma unroll
+      for (int j = 0; j < EPV; ++j) v[k * EPV + j] = f[j];
+    }
+
+    float mean = 0.f, rstd;
+    if (OP == OP_RMSNORM) {
+      float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+      for (int i = 0; i < N; i += 2) { s0 = fmaf(v[i], v[i], s0); s1 = fmaf(v[i + 1], v[i + 1], s1); }
+      float ss = warp_sum(s0 + s1);
+      if (NW > 1) {
+        if ((threadIdx.x & 31) == 0) red[parity][0][threadIdx.x >> 5] = ss;
+        __syncthreads();
+        ss = red[parity][0][threadIdx.x & (NW - 1)];
+#pragma unroll
+        for (int m = NW / 2; m >= 1; m >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, m);
+      }
+      rstd = rsqrt_refined(fmaf(ss, inv_cols, p.eps));
+    } else {
+      // thread tile: exact two-pass mean and M2 over N values
+      float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+      for (int i = 0; i < N; i += 2) { s0 += v[i]; s1 += v[i + 1]; }
+      float mu = (s0 + s1) * (1.0f / N);
+      float q0 = 0.f, q1 = 0.f;
+#pragma unroll
+      for (int i = 0; i < N; i += 2) {
+        const float d0 = v[i] - mu, d1 = v[i + 1] - mu;
+        q0 = fmaf(d0, d0, q0); q1 = fmaf(d1, d1, q1);
+      }
+      float m2 = q0 + q1;
+      // equal-count pairwise merges: both sides hold c values, so
+      //   mean = (ma + mb) / 2,  M2 = M2a + M2b + (mb - ma)^2 * c / 2
+      float half_c = 0.5f * N;
+#pragma unroll
+      for (int m = 1; m <= 16; m <<= 1) {
+        const float mb = __shfl_xor_sync(0xffffffffu, mu, m);
+        const float qb = __shfl_xor_sync(0xffffffffu, m2, m);
+        const float d = mb - mu;
+        mu = fmaf(0.5f, d, mu);
+        m2 = fmaf(d * d, half_c, m2 + qb);
+        half_c *= 2.f;
+      }
+      if (NW > 1) {
+        if ((threadIdx.x & 31) == 0) { red[parity][0][threadIdx.x >> 5] = mu; red[parity][1][threadIdx.x >> 5] = m2; }
+        __syncthreads();
+        mu = red[parity][0][threadIdx.x & (NW - 1)];
+        m2 = red[parity][1][threadIdx.x & (NW - 1)];
+#pragma unroll
+        for (int m = 1; m < NW; m <<= 1) {
+          const float mb = __shfl_xor_sync(0xffffffffu, mu, m);
+          const float qb = __shfl_xor_sync(0xffffffffu, m2, m);
+          const float d = mb - mu;
+          mu = fmaf(0.5f, d, mu);
+          m2 = fmaf(d * d, half_c, m2 + qb);
+          half_c *= 2.f;
+        }
+      }
+      mean = mu;
+      rstd = rsqrt_refined(fmaf(m2, inv_cols, p.eps));
+    }
+
+    const T* gp = reinterpret_cast<const T*>(p.gamma) + tg * EPV;
+    const T* bp = reinterpret_cast<const T*>(p.beta) + tg * EPV;
+#pragma unroll
+    for (int k = 0; k < VPT; ++k) {
+      float g[EPV], b[EPV], o[EPV];
+#pragma unroll
+      for (int j = 0; j < EPV; ++j) { g[j] = 1.f; b[j] = 0.f; }
+      if (p.gamma != nullptr) E::unpack(ld_cached(gp + k * G * EPV), g);
+      if (OP == OP_LAYERNORM && p.beta != nullptr) E::unpack(ld_cached(bp + k * G * EPV), b);
+#pragma unroll
+      for (int j = 0; j < EPV; ++j) {
+        if (OP == OP_LAYERNORM) o[j] = fmaf((v[k * EPV + j] - mean) * rstd, g[j], b[j]);
+        else o[j] = v[k * EPV + j] * rstd * g[j];
+      }
+      st_stream(yr + k * G * EPV, E::pack(o));
+    }
+  }
+}
+
+
+}  // namespace akg

@@ -105,6 +105,30 @@ __device__ __forceinline__ void fold_vector(Stat& st, const float (&z)[EPV]) {
   }
 }
 
+// Fold a block of four vectors: one running-maximum update and one rescale for the block
+// (softmax pair); the normalisations fold the vectors one after the other.
+template <int OP, int EPV>
+__device__ __forceinline__ void fold_block(Stat& st, const float (&z)[4][EPV]) {
+  if (OpTraits<OP>::kSoftmaxLike) {
+    float mv = z[0][0];
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+#pragma unroll
+      for (int j = 0; j < EPV; ++j) mv = fmaxf(mv, z[u][j]);
+    const float mn = fmaxf(st.a, mv);
+    const float ms = (mn == kNegInf) ? 0.f : mn;
+    float acc[4] = {st.b * exp_diff(st.a, ms), 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+#pragma unroll
+      for (int j = 0; j < EPV; ++j) acc[u] += exp_diff(z[u][j], ms);
+    st.a = mn; st.b = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+  } else {
+#pragma unroll
+    for (int u = 0; u < 4; ++u) fold_vector<OP, EPV>(st, z[u]);
+  }
+}
+
 struct SmemGeom {
   int nbuf;               // ring depth
   int slice_vecs;         // 16-byte vectors per CTA slice (last slice may be shorter)
@@ -186,9 +210,20 @@ __global__ void __launch_bounds__(THREADS) smem_kernel(const RowParams p, const 
                       : nullptr;
     mbar_wait_bounded(smem_addr(&bars[b]), phase, p.status);
 
-    // ---- pass 1: thread-local statistics over my slice
+    // ---- pass 1: thread-local statistics over my slice.  `plain` = no element of the
+    // slice is masked: four vectors per step, loads first, one rescale per block.
     Stat st = stat_identity<OP>();
-    for (int v = threadIdx.x; v < lv; v += THREADS) {
+    const bool plain = !SM || (ar == nullptr && (v0 + lv) * EPV <= live);
+    int v = threadIdx.x;
+    if (plain) {
+      for (; v + 3 * THREADS < lv; v += 4 * THREADS) {
+        float z[4][EPV];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) E::unpack(lds128(buf + static_cast<uint32_t>(v + u * THREADS) * 16u), z[u]);
+        fold_block<OP, EPV>(st, z);
+      }
+    }
+    for (; v < lv; v += THREADS) {
       float z[EPV];
       E::unpack(lds128(buf + static_cast<uint32_t>(v) * 16u), z);
       if (SM) {
@@ -227,7 +262,33 @@ __global__ void __launch_bounds__(THREADS) smem_kernel(const RowParams p, const 
 
     // ---- pass 2: normalise from shared memory, 128-bit stores
     T* yr = reinterpret_cast<T*>(p.y) + row * p.ys + static_cast<long long>(v0) * EPV;
-    for (int v = threadIdx.x; v < my_vecs; v += THREADS) {
+    v = threadIdx.x;
+    if (plain && lv == my_vecs) {
+      for (; v + 3 * THREADS < my_vecs; v += 4 * THREADS) {
+        float z[4][EPV];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) E::unpack(lds128(buf + static_cast<uint32_t>(v + u * THREADS) * 16u), z[u]);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int c0 = (v0 + v + u * THREADS) * EPV;
+          float ga[EPV], be[EPV], o[EPV];
+#pragma unroll
+          for (int j = 0; j < EPV; ++j) { ga[j] = 1.f; be[j] = 0.f; }
+          if (!SM) {
+            if (p.gamma != nullptr) E::unpack(ld_cached(reinterpret_cast<const T*>(p.gamma) + c0), ga);
+            if (OP == OP_LAYERNORM && p.beta != nullptr)
+              E::unpack(ld_cached(reinterpret_cast<const T*>(p.beta) + c0), be);
+          }
+#pragma unroll
+          for (int j = 0; j < EPV; ++j) {
+            if (OP == OP_SOFTMAX) o[j] = exp_diff(z[u][j], rs.p) * rs.q;
+            else o[j] = apply_one<OP>(z[u][j], rs, 0.f, ga[j], be[j]);
+          }
+          st_stream(yr + static_cast<long long>(v + u * THREADS) * EPV, E::pack(o));
+        }
+      }
+    }
+    for (; v < my_vecs; v += THREADS) {
       float o[EPV];
       if (v < lv) {
         float z[EPV];

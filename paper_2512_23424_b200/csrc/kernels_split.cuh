@@ -1,0 +1,188 @@
+// split_kernel: long rows without shared-memory residency.
+//
+// A cluster of CS CTAs owns one row at a time and CTA k streams slice k twice:
+//   pass 1  128-bit loads, four per thread in flight, marked "keep in L2"
+//           -> thread statistics -> CTA reduction -> partial statistics exchanged
+//           through distributed shared memory -> cluster barrier
+//   pass 2  the same slice again, now served by the 126 MB L2 (the row was read a few
+//           microseconds earlier), marked "evict first" -> normalise -> streaming stores
+// HBM therefore still sees one read and one write per element, while nothing limits
+// the row length and every SM keeps many loads in flight.  Rows are spread over as many
+// clusters as fit the GPU, so the rows resident in L2 between the passes are
+// (clusters in flight) x (row bytes), far below the L2 size for the shapes this is
+// chosen for (the planner checks it).
+#pragma once
+
+#include "kernels_smem.cuh"
+
+namespace akg {
+
+__device__ __forceinline__ uint64_t l2_policy_keep() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ uint64_t l2_policy_drop() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ uint4 ld_hint(const void* p, uint64_t pol) {
+  uint4 v;
+  asm volatile("ld.global.L1::no_allocate.L2::cache_hint.v4.u32 {%0, %1, %2, %3}, [%4], %5;"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p), "l"(pol) : "memory");
+  return v;
+}
+
+template <int OP, typename T, int THREADS>
+__global__ void __launch_bounds__(THREADS, (1024 / THREADS) > 0 ? (1024 / THREADS) : 1)
+split_kernel(const RowParams p, const int slice_vecs) {
+  using E = Elem<T>;
+  constexpr int EPV = E::EPV;
+  constexpr int NW = THREADS / 32;
+  constexpr bool SM = OpTraits<OP>::kSoftmaxLike;
+  __shared__ Stat red[2][NW];
+  __shared__ Stat peers[2][kMaxCluster];
+
+  const uint32_t cs = cluster_size();
+  const uint32_t rank = cluster_rank();
+  const long long row_step = cluster_count();
+  const int nvec = static_cast<int>(p.cols / EPV);
+  const int v0 = static_cast<int>(rank) * slice_vecs;
+  const int my_vecs = max(0, min(slice_vecs, nvec - v0));
+  const uint64_t keep = l2_policy_keep();
+  const uint64_t drop = l2_policy_drop();
+
+  if (cs > 1) {            // every CTA of the cluster is running before any remote store
+    cluster_arrive();
+    cluster_wait();
+  }
+
+  int par = 0;
+  for (long long row = cluster_id(); row < p.rows; row += row_step, par ^= 1) {
+    const int live = SM ? static_cast<int>(live_cols(p, row)) : static_cast<int>(p.cols);
+    const int live_vecs = (live + EPV - 1) / EPV;
+    const int lv = max(0, min(my_vecs, live_vecs - v0));
+    const T* xr = reinterpret_cast<const T*>(p.x) + row * p.xs + static_cast<long long>(v0) * EPV;
+    T* yr = reinterpret_cast<T*>(p.y) + row * p.ys + static_cast<long long>(v0) * EPV;
+    const T* ar = (SM && p.add != nullptr)
+                      ? reinterpret_cast<const T*>(p.add) + add_row(p, row) * p.add_stride +
+                            static_cast<long long>(v0) * EPV
+                      : nullptr;
+    const bool plain = !SM || (ar == nullptr && (v0 + lv) * EPV <= live);
+
+    // ---- pass 1: statistics
+    Stat st = stat_identity<OP>();
+    int v = threadIdx.x;
+    if (plain) {
+      for (; v + 3 * THREADS < lv; v += 4 * THREADS) {
+        uint4 raw[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) raw[u] = ld_hint(xr + static_cast<long long>(v + u * THREADS) * EPV, keep);
+        float z[4][EPV];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) E::unpack(raw[u], z[u]);
+        fold_block<OP, EPV>(st, z);
+      }
+    }
+    for (; v < lv; v += THREADS) {
+      float z[EPV];
+      E::unpack(ld_hint(xr + static_cast<long long>(v) * EPV, keep), z);
+      if (SM) {
+        const int c0 = (v0 + v) * EPV;
+        if (ar != nullptr) {
+          float a[EPV];
+          E::unpack(ld_hint(ar + static_cast<long long>(v) * EPV, keep), a);
+#pragma unroll
+          for (int j = 0; j < EPV; ++j) z[j] += a[j];
+        }
+        if (c0 + EPV > live) {
+#pragma unroll
+          for (int j = 0; j < EPV; ++j) if (c0 + j >= live) z[j] = kNegInf;
+        }
+      }
+      fold_vector<OP, EPV>(st, z);
+    }
+    st = cta_reduce<OP, NW>(st, red[par]);
+
+    if (cs > 1) {
+      if (threadIdx.x < cs) {
+        const uint32_t slot = smem_addr(&peers[par][rank]);
+        st_remote_f32(slot, threadIdx.x, st.a);
+        st_remote_f32(slot + 4, threadIdx.x, st.b);
+        st_remote_f32(slot + 8, threadIdx.x, st.c);
+      }
+      cluster_arrive();
+      cluster_wait();
+      Stat r = peers[par][0];
+      for (uint32_t k = 1; k < cs; ++k) r = stat_merge<OP>(r, peers[par][k]);
+      st = r;
+    }
+    const RowScalars rs = finalize<OP>(st, p.cols, p.eps);
+    const float fill = SM ? masked_fill<OP>(rs) : 0.f;
+
+    // ---- pass 2: second read (L2), normalise, store
+    v = threadIdx.x;
+    if (plain && lv == my_vecs) {
+      for (; v + 3 * THREADS < my_vecs; v += 4 * THREADS) {
+        uint4 raw[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) raw[u] = ld_hint(xr + static_cast<long long>(v + u * THREADS) * EPV, drop);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int c0 = (v0 + v + u * THREADS) * EPV;
+          float z[EPV], ga[EPV], be[EPV], o[EPV];
+          E::unpack(raw[u], z);
+#pragma unroll
+          for (int j = 0; j < EPV; ++j) { ga[j] = 1.f; be[j] = 0.f; }
+          if (!SM) {
+            if (p.gamma != nullptr) E::unpack(ld_cached(reinterpret_cast<const T*>(p.gamma) + c0), ga);
+            if (OP == OP_LAYERNORM && p.beta != nullptr)
+              E::unpack(ld_cached(reinterpret_cast<const T*>(p.beta) + c0), be);
+          }
+#pragma unroll
+          for (int j = 0; j < EPV; ++j) {
+            if (OP == OP_SOFTMAX) o[j] = exp_diff(z[j], rs.p) * rs.q;
+            else o[j] = apply_one<OP>(z[j], rs, 0.f, ga[j], be[j]);
+          }
+          st_stream(yr + static_cast<long long>(v + u * THREADS) * EPV, E::pack(o));
+        }
+      }
+    }
+    for (; v < my_vecs; v += THREADS) {
+      float o[EPV];
+      if (v < lv) {
+        float z[EPV];
+        E::unpack(ld_hint(xr + static_cast<long long>(v) * EPV, drop), z);
+        const int c0 = (v0 + v) * EPV;
+        float ga[EPV], be[EPV];
+#pragma unroll
+        for (int j = 0; j < EPV; ++j) { ga[j] = 1.f; be[j] = 0.f; }
+        if (SM) {
+          if (ar != nullptr) {
+            float a[EPV];
+            E::unpack(ld_hint(ar + static_cast<long long>(v) * EPV, drop), a);
+#pragma unroll
+            for (int j = 0; j < EPV; ++j) z[j] += a[j];
+          }
+        } else {
+          if (p.gamma != nullptr) E::unpack(ld_cached(reinterpret_cast<const T*>(p.gamma) + c0), ga);
+          if (OP == OP_LAYERNORM && p.beta != nullptr)
+            E::unpack(ld_cached(reinterpret_cast<const T*>(p.beta) + c0), be);
+        }
+#pragma unroll
+        for (int j = 0; j < EPV; ++j) {
+          if (SM && c0 + j >= live) o[j] = fill;
+          else if (OP == OP_SOFTMAX) o[j] = exp_diff(z[j], rs.p) * rs.q;
+          else o[j] = apply_one<OP>(z[j], rs, 0.f, ga[j], be[j]);
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < EPV; ++j) o[j] = fill;
+      }
+      st_stream(yr + static_cast<long long>(v) * EPV, E::pack(o));
+    }
+  }
+}
+
+}  // namespace akg

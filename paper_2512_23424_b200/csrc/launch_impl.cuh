@@ -6,7 +6,10 @@
 #include <tuple>
 
 #include "kernels_basic.cuh"
+#include "kernels_reg.cuh"
+#include "kernels_softmax.cuh"
 #include "kernels_smem.cuh"
+#include "kernels_split.cuh"
 #include "launch.cuh"
 
 namespace akg {
@@ -17,7 +20,8 @@ namespace akg {
   X(32, 1, 128) X(32, 2, 128) X(32, 4, 128) X(32, 8, 128) \
   X(128, 1, 128) X(128, 2, 128) X(128, 4, 128) \
   X(256, 1, 256) X(256, 2, 256) X(256, 4, 256) \
-  X(512, 4, 512) X(512, 8, 512) X(1024, 4, 1024) X(1024, 8, 1024)
+  X(512, 1, 512) X(512, 2, 512) X(512, 4, 512) X(512, 8, 512) \
+  X(1024, 1, 1024) X(1024, 2, 1024) X(1024, 4, 1024) X(1024, 8, 1024)
 
 // Launch smem_kernel (TMA ring, optionally clustered).  plan.grid == 0 asks for as many
 // clusters as can be co-resident (capped by the number of rows).
@@ -76,6 +80,54 @@ cudaError_t launch_smem(const LaunchPlan& plan, const RowParams& p, cudaStream_t
   return cudaLaunchKernelEx(&cfg, kernel, p, g);
 }
 
+// Launch split_kernel (cluster per row, two streaming passes, second one from L2).
+template <int OP, typename T, int THREADS>
+cudaError_t launch_split(const LaunchPlan& plan, const RowParams& p, cudaStream_t s) {
+  auto kernel = split_kernel<OP, T, THREADS>;
+  static std::mutex mu;
+  static std::map<std::pair<int, int>, int> resident;   // (device, cluster) -> co-resident clusters
+  static std::map<int, bool> prepared;
+  int dev = 0;
+  cudaError_t err = cudaGetDevice(&dev);
+  if (err != cudaSuccess) return err;
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = static_cast<unsigned>(plan.cluster);
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.blockDim = dim3(THREADS);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = s;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  int max_clusters = 0;
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    if (!prepared[dev]) {
+      err = cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+      if (err != cudaSuccess) return err;
+      prepared[dev] = true;
+    }
+    auto key = std::make_pair(dev, plan.cluster);
+    auto it = resident.find(key);
+    if (it == resident.end()) {
+      cfg.gridDim = dim3(static_cast<unsigned>(plan.cluster) * 1024u);
+      int n = 0;
+      err = cudaOccupancyMaxActiveClusters(&n, kernel, &cfg);
+      if (err != cudaSuccess) return err;
+      it = resident.emplace(key, n).first;
+    }
+    max_clusters = it->second;
+  }
+  if (max_clusters < 1) return cudaErrorLaunchOutOfResources;
+  long long clusters = plan.grid ? plan.grid / plan.cluster : max_clusters;
+  if (clusters > p.rows) clusters = p.rows;
+  if (clusters < 1) clusters = 1;
+  cfg.gridDim = dim3(static_cast<unsigned>(clusters * plan.cluster));
+  return cudaLaunchKernelEx(&cfg, kernel, p, plan.vpt);
+}
+
 template <int OP, typename T>
 cudaError_t launch_typed(const LaunchPlan& plan, const RowParams& p, cudaStream_t s) {
   if (plan.variant == V_STREAM) {
@@ -83,13 +135,28 @@ cudaError_t launch_typed(const LaunchPlan& plan, const RowParams& p, cudaStream_
     return cudaGetLastError();
   }
   if (plan.variant == V_REG) {
+    // plan.stages == 1 marks a row of exactly group * vpt vectors (the predicate-free
+    // normalisation kernel); the softmax pair always takes its own lean kernel.
 #define AKG_REG_CASE(G_, V_, T_)                                              \
   if (plan.group == (G_) && plan.vpt == (V_) && plan.threads == (T_)) {       \
-    reg_kernel<OP, T, G_, V_, T_><<<plan.grid, T_, 0, s>>>(p);                \
+    if constexpr (OpTraits<OP>::kSoftmaxLike) {                               \
+      reg_softmax<OP, T, G_, V_, T_><<<plan.grid, T_, 0, s>>>(p);             \
+    } else {                                                                  \
+      if (plan.stages == 1)                                                   \
+        reg_norm_full<OP, T, G_, V_, T_><<<plan.grid, T_, 0, s>>>(p);         \
+      else                                                                    \
+        reg_kernel<OP, T, G_, V_, T_><<<plan.grid, T_, 0, s>>>(p);            \
+    }                                                                         \
     return cudaGetLastError();                                                \
   }
     AKG_REG_SHAPES(AKG_REG_CASE)
 #undef AKG_REG_CASE
+    return cudaErrorInvalidConfiguration;
+  }
+  if (plan.variant == V_CLUSTER && plan.stages == 0) {       // no ring: the two-pass split kernel
+    if (plan.threads == 256) return launch_split<OP, T, 256>(plan, p, s);
+    if (plan.threads == 512) return launch_split<OP, T, 512>(plan, p, s);
+    if (plan.threads == 1024) return launch_split<OP, T, 1024>(plan, p, s);
     return cudaErrorInvalidConfiguration;
   }
   if (plan.variant == V_TMA || plan.variant == V_CLUSTER) {

@@ -15,7 +15,7 @@ from parity_util import (assert_positive_zero, cancel_magnitude, compare, run_gp
 
 pytestmark = pytest.mark.gpu
 
-VARIANTS = ["auto", "stream", "reg", "tma", "cluster"]
+VARIANTS = ["auto", "stream", "reg", "tma", "cluster", "split"]
 GOLDEN = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
 
 
@@ -23,13 +23,16 @@ GOLDEN = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
 def _reset_variant():
     yield
     akg.set_variant("auto")
-    for key in ("reg_threads", "reg_vpt", "reg_group", "grid_cap"):
+    for key in ("reg_threads", "reg_vpt", "reg_group", "reg_general", "grid_cap", "cluster_size",
+                "smem_nbuf", "smem_threads", "smem_ctas"):
         akg.set_tuning(key, 0)
 
 
 def run_variant(variant, fn):
     """Run fn() under a forced kernel family; None if that family cannot take the call."""
-    akg.set_variant(variant)
+    # "split" is the cluster family's two-pass mode (second pass served by L2)
+    akg.set_variant("cluster" if variant == "split" else variant)
+    akg.set_tuning("cluster_mode", 2 if variant == "split" else (1 if variant == "cluster" else 0))
     try:
         return fn()
     except akg.AkgError as e:
@@ -38,6 +41,7 @@ def run_variant(variant, fn):
         raise
     finally:
         akg.set_variant("auto")
+        akg.set_tuning("cluster_mode", 0)
 
 
 def check_workload(w, variants=VARIANTS, **kw):
@@ -209,6 +213,9 @@ def test_rows_without_live_entries_and_non_finite_inputs(dtype):
     x[1, 5] = np.nan
     x[2, 1000] = np.inf
     x[3, ::2] = -np.inf
+    x[4, :] = np.nan                       # nothing but NaN
+    x[5, :] = -np.inf                      # NaN among masked entries only
+    x[5, 77] = np.nan
     xs = x if dtype == wl.F32 else wl.f32_to_bf16_bits(x)
     for op in ("softmax", "log_softmax"):
         w = wl.Workload("special", op, dtype, 6, cols, xs)

@@ -209,6 +209,9 @@ def test_fully_masked_and_non_finite_rows():
     assert np.isnan(y[2]).all() and np.isnan(ly[2]).all()
     assert np.isnan(y[3]).all() and np.isnan(ly[3]).all()
     assert oracle.logsumexp_row(x[0]) == ninf
+    # a NaN makes the row NaN even when every other entry is masked
+    only = np.array([[np.nan, ninf, ninf], [np.nan, np.nan, np.nan]])
+    assert np.isnan(oracle.softmax(only)).all() and np.isnan(oracle.log_softmax(only)).all()
 
 
 def test_layernorm_moments_and_affine_invariance():
