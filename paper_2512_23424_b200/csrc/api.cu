@@ -25,6 +25,8 @@ std::atomic<int> g_tune_smem_threads{0};  //   CTA size (256 / 512 / 1024)
 std::atomic<int> g_tune_smem_ctas{0};     //   CTAs per SM the ring is sized for
 std::atomic<int> g_tune_reg_general{0};   // 1 = never take the predicate-free normalisation kernel
 std::atomic<int> g_tune_cluster_mode{0};  // 0 = planner's choice, 1 = row resident in shared memory, 2 = two-pass split
+std::atomic<int> g_tune_tma_mode{0};      // 0 = planner's choice, 1 = ring-fed register kernel, 2 = shared-memory passes
+std::atomic<int> g_tune_interleave{0};    // 1 = visit causal rows short/long alternately (default: storage order)
 
 __device__ int g_status_word = 0;
 
@@ -79,6 +81,22 @@ akg_status validate(const Call& c, const char* name) {
 
 bool is_pow2(long long v) { return v > 0 && (v & (v - 1)) == 0; }
 
+// SMs of the current device (cached per device; 148 if the query fails).
+int sm_count() {
+  static std::atomic<int> cache[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { (void)cudaGetLastError(); return 148; }
+  int n = cache[dev].load();
+  if (n == 0) {
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) {
+      (void)cudaGetLastError();
+      n = 148;
+    }
+    cache[dev].store(n);
+  }
+  return n;
+}
+
 int pow2_ceil(int v) { int r = 1; while (r < v) r <<= 1; return r; }
 
 // Can the vectorised families run this call?  (16-byte aligned rows and vectors.)
@@ -125,7 +143,11 @@ bool plan_reg(const Call& c, LaunchPlan* plan) {
   }
   const int64_t rpc = threads / group;
   int64_t grid = (c.rows + rpc - 1) / rpc;
-  const int cap = g_tune_grid_cap.load();
+  int cap = g_tune_grid_cap.load();
+  // the softmax pair runs persistent (two resident waves of CTAs, grid-stride over rows):
+  // measured a little faster than one CTA per row, most under a causal mask
+  if (cap == 0 && group == threads && (c.op == OP_SOFTMAX || c.op == OP_LOG_SOFTMAX))
+    cap = sm_count() * (2048 / threads);
   if (cap > 0 && grid > cap) grid = cap;
   if (grid > INT_MAX) grid = INT_MAX;
   plan->variant = V_REG; plan->threads = threads; plan->group = group; plan->vpt = vpt;
@@ -178,13 +200,48 @@ bool plan_smem(const Call& c, int cs_min, int cs_max, LaunchPlan* plan) {
   return true;
 }
 
+// Ring-fed register plan: persistent CTAs, a CTA per row, the row prefetched by bulk
+// copies into a shared-memory ring.  Normalisations need a row of exactly threads * vpt
+// vectors; the softmax pair takes any row that fits.  False if the row does not fit.
+bool plan_ring(const Call& c, LaunchPlan* plan) {
+  const int64_t epv = (c.dtype == AKG_F32) ? 4 : 8;
+  const int64_t nvec = c.cols / epv;
+  const bool norm = (c.op == OP_LAYERNORM || c.op == OP_RMSNORM);
+  const int t_threads = g_tune_reg_threads.load(), t_vpt = g_tune_reg_vpt.load();
+  int threads = 0, vpt = 0;
+  if (t_threads > 0 && t_vpt > 0) { threads = t_threads; vpt = t_vpt; }
+  else if (nvec <= 128) { threads = 128; vpt = 1; }
+  else if (nvec <= 256) { threads = 128; vpt = 2; }
+  else if (nvec <= 512) { threads = 128; vpt = 4; }
+  else if (nvec <= 1024) { threads = 256; vpt = 4; }
+  else if (nvec <= 2048) { threads = 512; vpt = 4; }
+  else return false;
+  if (threads > 512 || vpt > 4 || static_cast<int64_t>(threads) * vpt < nvec) return false;
+  if (norm && static_cast<int64_t>(threads) * vpt != nvec) return false;
+  const int64_t buf = (nvec * 16 + 127) & ~int64_t(127);
+  // size the ring so that the CTAs the register budget allows (1024 threads per SM) fit
+  const int ctas = g_tune_smem_ctas.load() > 0 ? g_tune_smem_ctas.load() : (1024 / threads);
+  int64_t nbuf = (static_cast<int64_t>(kMaxDynSmem) + 1024) / ctas - 1024 - 256 - 128;
+  nbuf /= buf;
+  if (nbuf > kMaxBuf) nbuf = kMaxBuf;
+  const int t_nbuf = g_tune_smem_nbuf.load();
+  if (t_nbuf > 0 && nbuf > t_nbuf) nbuf = t_nbuf;
+  if (nbuf < 1) return false;
+  plan->variant = V_TMA; plan->mode = 1; plan->threads = threads; plan->group = threads; plan->vpt = vpt;
+  plan->cluster = 1; plan->stages = static_cast<int>(nbuf);
+  plan->smem = 128 + static_cast<size_t>(nbuf) * buf;
+  const int cap = g_tune_grid_cap.load();
+  plan->grid = cap > 0 ? static_cast<unsigned>(cap) : 0u;
+  return true;
+}
+
 // Two-pass split plan (cluster per row, second pass served by L2): any aligned row.
 // The cluster is sized so that every SM gets work even when there are few rows.
 bool plan_split(const Call& c, LaunchPlan* plan) {
   const int64_t epv = (c.dtype == AKG_F32) ? 4 : 8;
   const int64_t nvec = c.cols / epv;
   const int t_cs = g_tune_cluster_size.load(), t_threads = g_tune_smem_threads.load();
-  int cs = t_cs > 0 ? t_cs : 8;
+  int cs = t_cs > 0 ? t_cs : 16;
   if (cs < 1 || cs > kMaxCluster || (cs & (cs - 1))) return false;
   const int threads = t_threads > 0 ? t_threads : 256;
   if (threads != 256 && threads != 512 && threads != 1024) return false;
@@ -194,6 +251,15 @@ bool plan_split(const Call& c, LaunchPlan* plan) {
   plan->cluster = cs; plan->stages = 0; plan->smem = 0;
   const int cap = g_tune_grid_cap.load();
   plan->grid = cap > 0 ? static_cast<unsigned>((cap / cs > 0 ? cap / cs : 1) * cs) : 0u;
+  if (cap == 0) {
+    // rows in flight must stay resident in L2 between the two passes: at most 64 MB of
+    // them, but never fewer clusters than it takes to give every SM a CTA
+    const int64_t row_bytes = c.cols * ((c.dtype == AKG_F32) ? 4 : 2);
+    int64_t clusters = (int64_t(64) << 20) / (row_bytes > 0 ? row_bytes : 1);
+    const int64_t floor_clusters = (160 + cs - 1) / cs;
+    if (clusters < floor_clusters) clusters = floor_clusters;
+    if (clusters < 4096) plan->grid = static_cast<unsigned>(clusters * cs);   // else: the launcher's own limit is lower
+  }
   return true;
 }
 
@@ -243,6 +309,8 @@ akg_status run(const Call& c, const char* name) {
     if (p.causal) {
       p.period = c.mask->causal_period; p.offset = c.mask->causal_offset;
       p.period_pow2 = is_pow2(p.period) ? 1 : 0;
+      p.interleave = (p.period_pow2 && p.period >= 4 && c.rows % p.period == 0 &&
+                      g_tune_interleave.load() == 1) ? 1 : 0;   // opt-in: measured slower than storage order
     }
   }
   p.status = nullptr;
@@ -252,10 +320,29 @@ akg_status run(const Call& c, const char* name) {
   LaunchPlan plan;
   std::memset(&plan, 0, sizeof plan);
   bool planned = false;
-  if ((forced == V_AUTO || forced == V_REG) && vec) planned = plan_reg(c, &plan);
+  // Automatic choice (each rule is a measured preference on B200, see the profiles):
+  //   bf16 normalisation rows of exactly threads * vpt vectors, many rows -> ring-fed
+  //     register kernel (the load latency is hidden by the copy ring, not by occupancy)
+  //   every other row that fits a CTA's registers -> register kernel
+  //   longer aligned rows -> two-pass split cluster kernel (second pass from L2)
+  //   anything unaligned -> scalar stream kernel
+  if (forced == V_AUTO && vec && c.dtype == AKG_BF16 && (c.op == OP_LAYERNORM || c.op == OP_RMSNORM) &&
+      c.rows >= 2048 && c.cols >= 2048 && g_tune_tma_mode.load() != 2) {
+    planned = plan_ring(c, &plan);
+    if (planned) {
+      if (g_tune_smem_nbuf.load() == 0) {                  // one buffer per CTA measured best
+        plan.smem -= static_cast<size_t>(plan.stages - 1) * ((plan.smem - 128) / plan.stages);
+        plan.stages = 1;
+      }
+      p.status = status_word_ptr();
+    }
+  }
+  if (!planned && (forced == V_AUTO || forced == V_REG) && vec) planned = plan_reg(c, &plan);
   if (!planned && vec) {
-    if (forced == V_AUTO) planned = plan_smem(c, 1, kMaxCluster, &plan);
-    else if (forced == V_TMA) planned = plan_smem(c, 1, 1, &plan);
+    if (forced == V_AUTO) planned = (g_tune_cluster_mode.load() == 1) ? plan_smem(c, 1, kMaxCluster, &plan)
+                                                                      : plan_split(c, &plan);
+    else if (forced == V_TMA)
+      planned = (g_tune_tma_mode.load() != 2 && plan_ring(c, &plan)) || plan_smem(c, 1, 1, &plan);
     else if (forced == V_CLUSTER)
       planned = (g_tune_cluster_mode.load() == 2) ? plan_split(c, &plan) : plan_smem(c, 2, kMaxCluster, &plan);
     if (planned) p.status = status_word_ptr();
@@ -282,7 +369,8 @@ akg_status run(const Call& c, const char* name) {
                   (plan.stages == 1 && (c.op == OP_LAYERNORM || c.op == OP_RMSNORM)) ? ",full" : "");
   else if (plan.variant == V_TMA || plan.variant == V_CLUSTER)
     std::snprintf(t_kernel, sizeof t_kernel, "%s<%s,t%d,cs%d,nbuf%d,slice%d>",
-                  plan.variant == V_TMA ? "tma" : (plan.stages == 0 ? "split" : "cluster"), dt, plan.threads,
+                  plan.variant == V_TMA ? (plan.mode == 1 ? "ring" : "tma") : (plan.stages == 0 ? "split" : "cluster"),
+                  dt, plan.threads,
                   plan.cluster, plan.stages, plan.vpt);
   else
     std::snprintf(t_kernel, sizeof t_kernel, "stream<%s,t%d>", dt, plan.threads);
@@ -359,6 +447,8 @@ akg_status akg_set_tuning(const char* key, int value) {
   else if (!std::strcmp(key, "smem_ctas")) g_tune_smem_ctas.store(value);
   else if (!std::strcmp(key, "reg_general")) g_tune_reg_general.store(value);
   else if (!std::strcmp(key, "cluster_mode")) g_tune_cluster_mode.store(value);
+  else if (!std::strcmp(key, "tma_mode")) g_tune_tma_mode.store(value);
+  else if (!std::strcmp(key, "interleave")) g_tune_interleave.store(value);
   else return fail(AKG_ERR_INVALID_ARG, "akg_set_tuning: unknown key %s", key);
   return AKG_OK;
 }

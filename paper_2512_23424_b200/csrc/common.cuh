@@ -27,6 +27,7 @@ struct RowParams {
   long long period, offset;
   int period_pow2;          // 1: period is a power of two (row & (period - 1))
   int add_mode;             // 0: row % add_rows, 1: add_rows == 1, 2: add_rows >= rows
+  int interleave;           // 1: visit the rows of a causal period short/long alternately
   int* status;              // device status word (bounded waits report here)
 };
 
@@ -123,6 +124,19 @@ __device__ __forceinline__ long long live_cols(const RowParams& p, long long row
   const long long rp = p.period_pow2 ? (row & (p.period - 1)) : (row % p.period);
   long long l = rp + p.offset + 1;
   return l < 0 ? 0 : (l > p.cols ? p.cols : l);
+}
+
+// Under a causal mask the live length grows with the row's position in its period, so
+// neighbouring rows cost the same and an SM would see all-short then all-long rows.
+// With p.interleave set (period a power of two, rows a multiple of it) work item i of a
+// period is mapped to row i/2 (i even) or period-1-i/2 (i odd): CTAs resident together
+// then mix short and long rows, and load-heavy and store-heavy work overlap.  Rows are
+// independent, so any one-to-one order is valid.
+__device__ __forceinline__ long long balanced_row(const RowParams& p, long long i) {
+  if (!p.interleave) return i;
+  const long long r = i & (p.period - 1);
+  const long long h = r >> 1;
+  return (i - r) + ((r & 1) ? (p.period - 1 - h) : h);
 }
 
 // Row of the additive mask that row `row` uses.

@@ -1,20 +1,18 @@
-// Lean register-resident kernels (the fast paths of the REG family).
+// Lean register-resident normalisation (the fast path of the REG family).
 //
-//   reg_norm_full   LayerNorm / RMSNorm when the row is exactly G * VPT vectors: no
-//                   predicates, equal-count pairwise mean / M2 merges (no divisions),
-//                   one CTA barrier per row
-//   reg_softmax     softmax / log-softmax, any row that fits, optional additive and
-//                   causal mask: vectors beyond the live prefix are skipped with
-//                   CTA-uniform branches, the exponential is evaluated once per live
-//                   element against the warp maximum, and the cross-warp combine costs
-//                   one exponential per warp
+//   norm_row_full   one row of LayerNorm / RMSNorm when the row is exactly G * VPT
+//                   vectors: no predicates, equal-count pairwise mean / M2 merges (no
+//                   divisions), one CTA barrier per row.  The row comes either from
+//                   global memory or from a shared-memory buffer a bulk copy filled.
+//   reg_norm_full   the kernel around it: a warp or a CTA per row, grid-stride
 //
 // The instruction count per element is what bounds these kernels once the loads are
-// wide enough, so everything per-row (reductions, reciprocal, square root) is kept to
-// a few dozen instructions per thread.
+// wide enough, so everything per-row (reductions, reciprocal square root) is kept to a
+// few dozen instructions per thread.
 #pragma once
 
 #include "kernels_basic.cuh"
+#include "tma.cuh"
 
 namespace akg {
 
@@ -40,76 +38,80 @@ __device__ __forceinline__ float warp_max(float v) {
   return v;
 }
 
-// ------------------------------------------------------------------------------------
-// reg_norm_full
-// ------------------------------------------------------------------------------------
-template <int OP, typename T, int G, int VPT, int THREADS>
-__global__ void __launch_bounds__(THREADS, kRegMinBlocks<THREADS>) reg_norm_full(const RowParams p) {
+// red: [2][NW] floats of shared memory reserved for this row (callers alternate two sets).
+template <int OP, typename T, int G, int VPT, int THREADS, bool RING = false>
+__device__ __forceinline__ void norm_row_full(const RowParams& p, long long row, int tg,
+                                              float (*red)[(G / 32) > 1 ? (G / 32) : 1],
+                                              uint32_t ring_buf = 0) {
   using E = Elem<T>;
   constexpr int EPV = E::EPV;
   constexpr int N = VPT * EPV;
-  constexpr int RPC = THREADS / G;
   constexpr int NW = G / 32;
   static_assert(OP == OP_LAYERNORM || OP == OP_RMSNORM, "normalisations only");
   static_assert((NW & (NW - 1)) == 0, "warps per row must be a power of two");
-  __shared__ float red[2][2][NW > 1 ? NW : 1];
-
-  const int tg = threadIdx.x % G;
-  const int grp = threadIdx.x / G;
   const float inv_cols = 1.0f / static_cast<float>(N * G);
-  int parity = 0;
+  const T* xr = reinterpret_cast<const T*>(p.x) + row * p.xs + tg * EPV;
+  T* yr = reinterpret_cast<T*>(p.y) + row * p.ys + tg * EPV;
 
-  for (long long rb = static_cast<long long>(blockIdx.x) * RPC; rb < p.rows;
-       rb += static_cast<long long>(gridDim.x) * RPC, parity ^= 1) {
-    const long long row = rb + grp;
-    if (G != THREADS && row >= p.rows) continue;
-    const T* xr = reinterpret_cast<const T*>(p.x) + row * p.xs + tg * EPV;
-    T* yr = reinterpret_cast<T*>(p.y) + row * p.ys + tg * EPV;
+  uint4 raw[VPT];
+#pragma unroll
+  for (int k = 0; k < VPT; ++k)
+    raw[k] = RING ? lds128(ring_buf + static_cast<uint32_t>(tg + k * G) * 16u) : ld_stream(xr + k * G * EPV);
+  float v[N];
+#pragma unroll
+  for (int k = 0; k < VPT; ++k) {
+    float f[EPV];
+    E::unpack(raw[k], f);
+#pragma unroll
+    for (int j = 0; j < EPV; ++j) v[k * EPV + j] = f[j];
+  }
 
-    uint4 raw[VPT];
+  float mean = 0.f, rstd;
+  if (OP == OP_RMSNORM) {
+    float s0 = 0.f, s1 = 0.f;
 #pragma unroll
-    for (int k = 0; k < VPT; ++k) raw[k] = ld_stream(xr + k * G * EPV);
-    float v[N];
+    for (int i = 0; i < N; i += 2) { s0 = fmaf(v[i], v[i], s0); s1 = fmaf(v[i + 1], v[i + 1], s1); }
+    float ss = warp_sum(s0 + s1);
+    if (NW > 1) {
+      if ((threadIdx.x & 31) == 0) red[0][threadIdx.x >> 5] = ss;
+      __syncthreads();
+      ss = red[0][threadIdx.x & (NW - 1)];
 #pragma unroll
-    for (int k = 0; k < VPT; ++k) {
-      float f[EPV];
-      E::unpack(raw[k], f);
-#pragma unroll
-      for (int j = 0; j < EPV; ++j) v[k * EPV + j] = f[j];
+      for (int m = NW / 2; m >= 1; m >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, m);
     }
-
-    float mean = 0.f, rstd;
-    if (OP == OP_RMSNORM) {
-      float s0 = 0.f, s1 = 0.f;
+    rstd = rsqrt_refined(fmaf(ss, inv_cols, p.eps));
+  } else {
+    // thread tile: exact two-pass mean and M2 over N values
+    float s0 = 0.f, s1 = 0.f;
 #pragma unroll
-      for (int i = 0; i < N; i += 2) { s0 = fmaf(v[i], v[i], s0); s1 = fmaf(v[i + 1], v[i + 1], s1); }
-      float ss = warp_sum(s0 + s1);
-      if (NW > 1) {
-        if ((threadIdx.x & 31) == 0) red[parity][0][threadIdx.x >> 5] = ss;
-        __syncthreads();
-        ss = red[parity][0][threadIdx.x & (NW - 1)];
+    for (int i = 0; i < N; i += 2) { s0 += v[i]; s1 += v[i + 1]; }
+    float mu = (s0 + s1) * (1.0f / N);
+    float q0 = 0.f, q1 = 0.f;
 #pragma unroll
-        for (int m = NW / 2; m >= 1; m >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, m);
-      }
-      rstd = rsqrt_refined(fmaf(ss, inv_cols, p.eps));
-    } else {
-      // thread tile: exact two-pass mean and M2 over N values
-      float s0 = 0.f, s1 = 0.f;
+    for (int i = 0; i < N; i += 2) {
+      const float d0 = v[i] - mu, d1 = v[i + 1] - mu;
+      q0 = fmaf(d0, d0, q0); q1 = fmaf(d1, d1, q1);
+    }
+    float m2 = q0 + q1;
+    // equal-count pairwise merges: both sides hold c values, so
+    //   mean = (ma + mb) / 2,  M2 = M2a + M2b + (mb - ma)^2 * c / 2
+    float half_c = 0.5f * N;
 #pragma unroll
-      for (int i = 0; i < N; i += 2) { s0 += v[i]; s1 += v[i + 1]; }
-      float mu = (s0 + s1) * (1.0f / N);
-      float q0 = 0.f, q1 = 0.f;
+    for (int m = 1; m <= 16; m <<= 1) {
+      const float mb = __shfl_xor_sync(0xffffffffu, mu, m);
+      const float qb = __shfl_xor_sync(0xffffffffu, m2, m);
+      const float d = mb - mu;
+      mu = fmaf(0.5f, d, mu);
+      m2 = fmaf(d * d, half_c, m2 + qb);
+      half_c *= 2.f;
+    }
+    if (NW > 1) {
+      if ((threadIdx.x & 31) == 0) { red[0][threadIdx.x >> 5] = mu; red[1][threadIdx.x >> 5] = m2; }
+      __syncthreads();
+      mu = red[0][threadIdx.x & (NW - 1)];
+      m2 = red[1][threadIdx.x & (NW - 1)];
 #pragma unroll
-      for (int i = 0; i < N; i += 2) {
-        const float d0 = v[i] - mu, d1 = v[i + 1] - mu;
-        q0 = fmaf(d0, d0, q0); q1 = fmaf(d1, d1, q1);
-      }
-      float m2 = q0 + q1;
-      // equal-count pairwise merges: both sides hold c values, so
-      //   mean = (ma + mb) / 2,  M2 = M2a + M2b + (mb - ma)^2 * c / 2
-      float half_c = 0.5f * N;
-#pragma unroll
-      for (int m = 1; m <= 16; m <<= 1) {
+      for (int m = 1; m < NW; m <<= 1) {
         const float mb = __shfl_xor_sync(0xffffffffu, mu, m);
         const float qb = __shfl_xor_sync(0xffffffffu, m2, m);
         const float d = mb - mu;
@@ -117,43 +119,43 @@ __global__ void __launch_bounds__(THREADS, kRegMinBlocks<THREADS>) reg_norm_full
         m2 = fmaf(d * d, half_c, m2 + qb);
         half_c *= 2.f;
       }
-      if (NW > 1) {
-        if ((threadIdx.x & 31) == 0) { red[parity][0][threadIdx.x >> 5] = mu; red[parity][1][threadIdx.x >> 5] = m2; }
-        __syncthreads();
-        mu = red[parity][0][threadIdx.x & (NW - 1)];
-        m2 = red[parity][1][threadIdx.x & (NW - 1)];
-#pragma unroll
-        for (int m = 1; m < NW; m <<= 1) {
-          const float mb = __shfl_xor_sync(0xffffffffu, mu, m);
-          const float qb = __shfl_xor_sync(0xffffffffu, m2, m);
-          const float d = mb - mu;
-          mu = fmaf(0.5f, d, mu);
-          m2 = fmaf(d * d, half_c, m2 + qb);
-          half_c *= 2.f;
-        }
-      }
-      mean = mu;
-      rstd = rsqrt_refined(fmaf(m2, inv_cols, p.eps));
     }
+    mean = mu;
+    rstd = rsqrt_refined(fmaf(m2, inv_cols, p.eps));
+  }
 
-    const T* gp = reinterpret_cast<const T*>(p.gamma) + tg * EPV;
-    const T* bp = reinterpret_cast<const T*>(p.beta) + tg * EPV;
+  const T* gp = reinterpret_cast<const T*>(p.gamma) + tg * EPV;
+  const T* bp = reinterpret_cast<const T*>(p.beta) + tg * EPV;
 #pragma unroll
-    for (int k = 0; k < VPT; ++k) {
-      float g[EPV], b[EPV], o[EPV];
+  for (int k = 0; k < VPT; ++k) {
+    float g[EPV], b[EPV], o[EPV];
 #pragma unroll
-      for (int j = 0; j < EPV; ++j) { g[j] = 1.f; b[j] = 0.f; }
-      if (p.gamma != nullptr) E::unpack(ld_cached(gp + k * G * EPV), g);
-      if (OP == OP_LAYERNORM && p.beta != nullptr) E::unpack(ld_cached(bp + k * G * EPV), b);
+    for (int j = 0; j < EPV; ++j) { g[j] = 1.f; b[j] = 0.f; }
+    if (p.gamma != nullptr) E::unpack(ld_cached(gp + k * G * EPV), g);
+    if (OP == OP_LAYERNORM && p.beta != nullptr) E::unpack(ld_cached(bp + k * G * EPV), b);
 #pragma unroll
-      for (int j = 0; j < EPV; ++j) {
-        if (OP == OP_LAYERNORM) o[j] = fmaf((v[k * EPV + j] - mean) * rstd, g[j], b[j]);
-        else o[j] = v[k * EPV + j] * rstd * g[j];
-      }
-      st_stream(yr + k * G * EPV, E::pack(o));
+    for (int j = 0; j < EPV; ++j) {
+      if (OP == OP_LAYERNORM) o[j] = fmaf((v[k * EPV + j] - mean) * rstd, g[j], b[j]);
+      else o[j] = v[k * EPV + j] * rstd * g[j];
     }
+    st_stream(yr + k * G * EPV, E::pack(o));
   }
 }
 
+template <int OP, typename T, int G, int VPT, int THREADS>
+__global__ void __launch_bounds__(THREADS, kRegMinBlocks<THREADS>) reg_norm_full(const RowParams p) {
+  constexpr int RPC = THREADS / G;
+  constexpr int NW = G / 32;
+  __shared__ float red[2][2][NW > 1 ? NW : 1];
+  const int tg = threadIdx.x % G;
+  const int grp = threadIdx.x / G;
+  int parity = 0;
+  for (long long rb = static_cast<long long>(blockIdx.x) * RPC; rb < p.rows;
+       rb += static_cast<long long>(gridDim.x) * RPC, parity ^= 1) {
+    const long long row = rb + grp;
+    if (G != THREADS && row >= p.rows) continue;
+    norm_row_full<OP, T, G, VPT, THREADS>(p, row, tg, red[parity]);
+  }
+}
 
 }  // namespace akg

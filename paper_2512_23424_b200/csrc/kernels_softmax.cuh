@@ -13,9 +13,12 @@
 
 namespace akg {
 
-template <int OP, typename T, int G, int VPT, int THREADS, int NK>
+// RING = false: the row is read from global memory; RING = true: from the shared-memory
+// buffer at `ring_buf` that a bulk copy has filled with the row's live prefix.
+template <int OP, typename T, int G, int VPT, int THREADS, int NK, bool RING = false>
 __device__ __forceinline__ void softmax_row(const RowParams& p, long long row, int tg, int nvec, int live,
-                                            int live_vecs, float (*red)[(G / 32) > 1 ? (G / 32) : 1]) {
+                                            int live_vecs, float (*red)[(G / 32) > 1 ? (G / 32) : 1],
+                                            uint32_t ring_buf = 0) {
   using E = Elem<T>;
   constexpr int EPV = E::EPV;
   constexpr int NW = G / 32;
@@ -29,7 +32,8 @@ __device__ __forceinline__ void softmax_row(const RowParams& p, long long row, i
   uint4 raw[NKA];
 #pragma unroll
   for (int k = 0; k < NK; ++k)
-    if (k < NK - 1 || last_ok) raw[k] = ld_stream(xr + k * G * EPV);
+    if (k < NK - 1 || last_ok)
+      raw[k] = RING ? lds128(ring_buf + static_cast<uint32_t>(tg + k * G) * 16u) : ld_stream(xr + k * G * EPV);
   float v[NKA][EPV];
   float m_t = kNegInf;
 #pragma unroll
@@ -58,11 +62,15 @@ __device__ __forceinline__ void softmax_row(const RowParams& p, long long row, i
   const float m_w = warp_max(m_t);
   const float m_ws = (m_w == kNegInf) ? 0.f : m_w;        // keeps -inf - -inf out of the exponent
   float s_t = 0.f;
+  // bf16 storage: one fused multiply-add forms the exponent (its rounding, below 1e-5
+  // relative, is far inside the 2^-9 of the bf16 result); fp32 keeps the exact difference
+  constexpr bool kFusedExponent = (sizeof(T) == 2);
+  const float neg_m_l2 = -m_ws * kLog2e;
 #pragma unroll
   for (int k = 0; k < NK; ++k) {
 #pragma unroll
     for (int j = 0; j < EPV; ++j) {
-      const float e = exp_diff(v[k][j], m_ws);
+      const float e = kFusedExponent ? ex2_approx(fmaf(v[k][j], kLog2e, neg_m_l2)) : exp_diff(v[k][j], m_ws);
       s_t += e;
       if (OP == OP_SOFTMAX) v[k][j] = e;
     }
@@ -136,8 +144,8 @@ __global__ void __launch_bounds__(THREADS, kRegMinBlocks<THREADS>) reg_softmax(c
 
   for (long long rb = static_cast<long long>(blockIdx.x) * RPC; rb < p.rows;
        rb += static_cast<long long>(gridDim.x) * RPC, parity ^= 1) {
-    const long long row = rb + grp;
-    if (G != THREADS && row >= p.rows) continue;
+    if (G != THREADS && rb + grp >= p.rows) continue;
+    const long long row = balanced_row(p, rb + grp);
     const int live = static_cast<int>(live_cols(p, row));
     const int live_vecs = (live + EPV - 1) / EPV;
     const int nk = (live_vecs + G - 1) / G;             // uniform over the threads of the row

@@ -75,10 +75,23 @@ split_kernel(const RowParams p, const int slice_vecs) {
     Stat st = stat_identity<OP>();
     int v = threadIdx.x;
     if (plain) {
-      for (; v + 3 * THREADS < lv; v += 4 * THREADS) {
+      const uint4* px = reinterpret_cast<const uint4*>(xr) + v;
+      for (; v + 7 * THREADS < lv; v += 8 * THREADS, px += 8 * THREADS) {   // eight loads in flight
+        uint4 raw[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) raw[u] = ld_hint(px + u * THREADS, keep);
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          float z[4][EPV];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) E::unpack(raw[4 * h + u], z[u]);
+          fold_block<OP, EPV>(st, z);
+        }
+      }
+      for (; v + 3 * THREADS < lv; v += 4 * THREADS, px += 4 * THREADS) {
         uint4 raw[4];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) raw[u] = ld_hint(xr + static_cast<long long>(v + u * THREADS) * EPV, keep);
+        for (int u = 0; u < 4; ++u) raw[u] = ld_hint(px + u * THREADS, keep);
         float z[4][EPV];
 #pragma unroll
         for (int u = 0; u < 4; ++u) E::unpack(raw[u], z[u]);
@@ -124,10 +137,12 @@ split_kernel(const RowParams p, const int slice_vecs) {
     // ---- pass 2: second read (L2), normalise, store
     v = threadIdx.x;
     if (plain && lv == my_vecs) {
-      for (; v + 3 * THREADS < my_vecs; v += 4 * THREADS) {
+      const uint4* px = reinterpret_cast<const uint4*>(xr) + v;
+      uint4* py = reinterpret_cast<uint4*>(yr) + v;
+      for (; v + 3 * THREADS < my_vecs; v += 4 * THREADS, px += 4 * THREADS, py += 4 * THREADS) {
         uint4 raw[4];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) raw[u] = ld_hint(xr + static_cast<long long>(v + u * THREADS) * EPV, drop);
+        for (int u = 0; u < 4; ++u) raw[u] = ld_hint(px + u * THREADS, drop);
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
           const int c0 = (v0 + v + u * THREADS) * EPV;
@@ -145,7 +160,7 @@ split_kernel(const RowParams p, const int slice_vecs) {
             if (OP == OP_SOFTMAX) o[j] = exp_diff(z[j], rs.p) * rs.q;
             else o[j] = apply_one<OP>(z[j], rs, 0.f, ga[j], be[j]);
           }
-          st_stream(yr + static_cast<long long>(v + u * THREADS) * EPV, E::pack(o));
+          st_stream(py + u * THREADS, E::pack(o));
         }
       }
     }

@@ -20,6 +20,7 @@ struct LaunchPlan {
   int cluster;        // CTAs per cluster (V_CLUSTER), else 1
   int stages;         // ring depth (V_TMA)
   size_t smem;        // dynamic shared memory per CTA
+  int mode;           // V_TMA: 1 = register kernels fed by a ring, 0 = shared-memory-resident kernel
 };
 
 template <int OP>

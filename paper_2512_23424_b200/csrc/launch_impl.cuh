@@ -8,6 +8,7 @@
 #include "kernels_basic.cuh"
 #include "kernels_reg.cuh"
 #include "kernels_softmax.cuh"
+#include "kernels_ring.cuh"
 #include "kernels_smem.cuh"
 #include "kernels_split.cuh"
 #include "launch.cuh"
@@ -80,6 +81,40 @@ cudaError_t launch_smem(const LaunchPlan& plan, const RowParams& p, cudaStream_t
   return cudaLaunchKernelEx(&cfg, kernel, p, g);
 }
 
+// Launch a ring-fed register kernel (persistent; plan.grid == 0 asks for one full wave).
+template <typename Kernel>
+cudaError_t launch_ring(Kernel kernel, int threads, const LaunchPlan& plan, const RowParams& p, cudaStream_t s) {
+  static std::mutex mu;
+  static std::map<std::tuple<const void*, int, size_t>, int> wave;   // (kernel, device, smem) -> CTAs per wave
+  int dev = 0;
+  cudaError_t err = cudaGetDevice(&dev);
+  if (err != cudaSuccess) return err;
+  int ctas = 0;
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    auto key = std::make_tuple(reinterpret_cast<const void*>(kernel), dev, plan.smem);
+    auto it = wave.find(key);
+    if (it == wave.end()) {
+      // the kernels also hold a few hundred bytes of static shared memory
+      err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(kMaxDynSmem) - 2048);
+      if (err != cudaSuccess) return err;
+      int per_sm = 0, sms = 0;
+      err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, plan.smem);
+      if (err != cudaSuccess) return err;
+      err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+      if (err != cudaSuccess) return err;
+      it = wave.emplace(key, per_sm * sms).first;
+    }
+    ctas = it->second;
+  }
+  if (ctas < 1) return cudaErrorLaunchOutOfResources;
+  long long grid = plan.grid ? plan.grid : ctas;
+  if (grid > p.rows) grid = p.rows;
+  kernel<<<static_cast<unsigned>(grid), threads, plan.smem, s>>>(p, plan.stages);
+  return cudaGetLastError();
+}
+
 // Launch split_kernel (cluster per row, two streaming passes, second one from L2).
 template <int OP, typename T, int THREADS>
 cudaError_t launch_split(const LaunchPlan& plan, const RowParams& p, cudaStream_t s) {
@@ -121,7 +156,8 @@ cudaError_t launch_split(const LaunchPlan& plan, const RowParams& p, cudaStream_
     max_clusters = it->second;
   }
   if (max_clusters < 1) return cudaErrorLaunchOutOfResources;
-  long long clusters = plan.grid ? plan.grid / plan.cluster : max_clusters;
+  long long clusters = max_clusters;                     // one resident wave, optionally capped
+  if (plan.grid && plan.grid / plan.cluster < clusters) clusters = plan.grid / plan.cluster;
   if (clusters > p.rows) clusters = p.rows;
   if (clusters < 1) clusters = 1;
   cfg.gridDim = dim3(static_cast<unsigned>(clusters * plan.cluster));
@@ -151,6 +187,20 @@ cudaError_t launch_typed(const LaunchPlan& plan, const RowParams& p, cudaStream_
   }
     AKG_REG_SHAPES(AKG_REG_CASE)
 #undef AKG_REG_CASE
+    return cudaErrorInvalidConfiguration;
+  }
+  if (plan.variant == V_TMA && plan.mode == 1) {             // ring-fed register kernels
+#define AKG_RING_CASE(G_, V_, T_)                                                                  \
+  if ((G_) == (T_) && plan.vpt == (V_) && plan.threads == (T_)) {                                  \
+    if constexpr ((G_) == (T_) && (V_) <= 4 && (T_) <= 512) {                                      \
+      if constexpr (OpTraits<OP>::kSoftmaxLike)                                                    \
+        return launch_ring(ring_softmax<OP, T, V_, T_>, T_, plan, p, s);                           \
+      else                                                                                         \
+        return launch_ring(ring_norm_full<OP, T, V_, T_>, T_, plan, p, s);                         \
+    }                                                                                              \
+  }
+    AKG_REG_SHAPES(AKG_RING_CASE)
+#undef AKG_RING_CASE
     return cudaErrorInvalidConfiguration;
   }
   if (plan.variant == V_CLUSTER && plan.stages == 0) {       // no ring: the two-pass split kernel

@@ -15,7 +15,7 @@ from parity_util import (assert_positive_zero, cancel_magnitude, compare, run_gp
 
 pytestmark = pytest.mark.gpu
 
-VARIANTS = ["auto", "stream", "reg", "tma", "cluster", "split"]
+VARIANTS = ["auto", "stream", "reg", "tma", "tma_smem", "cluster", "split"]
 GOLDEN = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
 
 
@@ -31,8 +31,11 @@ def _reset_variant():
 def run_variant(variant, fn):
     """Run fn() under a forced kernel family; None if that family cannot take the call."""
     # "split" is the cluster family's two-pass mode (second pass served by L2)
-    akg.set_variant("cluster" if variant == "split" else variant)
+    # "tma" prefers the ring-fed register kernels; "tma_smem" forces the shared-memory passes
+    family = {"split": "cluster", "tma_smem": "tma"}.get(variant, variant)
+    akg.set_variant(family)
     akg.set_tuning("cluster_mode", 2 if variant == "split" else (1 if variant == "cluster" else 0))
+    akg.set_tuning("tma_mode", 2 if variant == "tma_smem" else 0)
     try:
         return fn()
     except akg.AkgError as e:
@@ -42,6 +45,7 @@ def run_variant(variant, fn):
     finally:
         akg.set_variant("auto")
         akg.set_tuning("cluster_mode", 0)
+        akg.set_tuning("tma_mode", 0)
 
 
 def check_workload(w, variants=VARIANTS, **kw):
