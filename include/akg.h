@@ -108,6 +108,41 @@ akg_status akg_rmsnorm(const void* x, void* y, int64_t rows, int64_t cols,
                        int64_t x_row_stride, int64_t y_row_stride, akg_dtype dtype,
                        const void* weight, float eps, void* stream);
 
+typedef enum akg_op {
+  AKG_OP_SOFTMAX = 0,
+  AKG_OP_LOG_SOFTMAX = 1,
+  AKG_OP_LAYERNORM = 2,
+  AKG_OP_RMSNORM = 3
+} akg_op;
+
+/* Any of the four operators above on HOST buffers (no counterpart in the paper; the
+ * operator definitions are the ones cited at akg_softmax .. akg_rmsnorm).
+ *   x_host, y_host, gamma_host, beta_host : HOST pointers (page-locked memory lets the
+ *     copies overlap; pageable memory works but serialises).  gamma_host is the
+ *     RMSNorm weight; beta_host is used by LayerNorm only; mask (softmax pair only)
+ *     may carry the causal rule, an additive mask is AKG_ERR_UNSUPPORTED here.
+ *   workspace : DEVICE pointer, 16-byte aligned, workspace_bytes long, owned by the
+ *     caller; the library allocates no device memory.  Any size from
+ *     3 * round_up(cols * element size, 256) (+ the vectors) works; the size returned
+ *     by akg_host_workspace_bytes lets copies and kernels overlap fully.
+ * The rows are cut into chunks; chunk i is copied host -> workspace slot (i mod 3),
+ * processed in place by the same kernels as the device entry points, and copied back,
+ * on one of three internal streams, so uploads, kernels and downloads of different
+ * chunks overlap.  The work is ordered after everything already enqueued on `stream`,
+ * and `stream` waits for it; the call itself returns without synchronising (the host
+ * buffers and the workspace must stay valid until `stream` has caught up).  In place
+ * (y_host == x_host, equal strides) is allowed.  Calls on the same device are
+ * serialised by an internal lock while they enqueue.  Errors as for the device entry
+ * points; a workspace that is NULL, misaligned or too small is AKG_ERR_INVALID_ARG. */
+akg_status akg_rowop_host(akg_op op, const void* x_host, void* y_host, int64_t rows, int64_t cols,
+                          int64_t x_row_stride, int64_t y_row_stride, akg_dtype dtype,
+                          const void* gamma_host, const void* beta_host, float eps,
+                          const akg_mask* mask, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Workspace size (bytes) with which akg_rowop_host pipelines about a dozen chunks of
+ * at least 4 MiB; 0 for a malformed shape. */
+size_t akg_host_workspace_bytes(int64_t rows, int64_t cols, akg_dtype dtype, int has_gamma, int has_beta);
+
 /* Human-readable name of a status code (static storage, never NULL). */
 const char* akg_status_string(akg_status status);
 
@@ -130,7 +165,11 @@ akg_status akg_set_variant(akg_variant variant);
  * rows beyond it are taken in a grid-stride loop); for the shared-memory ring
  * families "cluster_size" (CTAs per row: 1, 2, 4, 8, 16), "smem_nbuf" (ring depth
  * limit), "smem_threads" (256, 512, 1024), "smem_ctas" (CTAs per SM the ring is
- * sized for).  A geometry the library was not
+ * sized for), "tma_mode" (1 = ring-fed register kernels, 2 = shared-memory passes),
+ * "cluster_mode" (1 = row resident in the cluster's shared memory, 2 = two streaming
+ * passes with the second served by L2), "reg_general" (1 = never the predicate-free
+ * normalisation kernel), "interleave" (1 = visit causal rows short/long alternately).
+ * A geometry the library was not
  * built for makes the next call return AKG_ERR_CUDA.  Unknown key:
  * AKG_ERR_INVALID_ARG. */
 akg_status akg_set_tuning(const char* key, int value);

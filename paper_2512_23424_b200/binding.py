@@ -69,6 +69,11 @@ def lib() -> ctypes.CDLL:
         L.akg_set_tuning.restype = ci
         L.akg_device_status.argtypes = [ctypes.POINTER(ci)]
         L.akg_device_status.restype = ci
+        L.akg_rowop_host.argtypes = [ci, vp, vp, i64, i64, i64, i64, ci, vp, vp, cf, mp, vp,
+                                     ctypes.c_size_t, vp]
+        L.akg_rowop_host.restype = ci
+        L.akg_host_workspace_bytes.argtypes = [i64, i64, ci, ci, ci]
+        L.akg_host_workspace_bytes.restype = ctypes.c_size_t
         _lib = L
     return _lib
 
@@ -203,6 +208,47 @@ def prepare(op: str, x: torch.Tensor, out: Optional[torch.Tensor] = None, *,
         args = head + (vp(_vector(gamma, x, cols, "weight")), ctypes.c_float(eps), s)
         return PreparedCall("akg_rmsnorm", args, (x, gamma), out)
     raise ValueError(f"unknown operator {op}")
+
+
+OPS = {"softmax": 0, "log_softmax": 1, "layernorm": 2, "rmsnorm": 3}
+
+
+def host_workspace_bytes(rows: int, cols: int, dtype: torch.dtype, has_gamma: bool = False,
+                         has_beta: bool = False) -> int:
+    code = F32 if dtype == torch.float32 else BF16
+    return int(lib().akg_host_workspace_bytes(rows, cols, code, int(has_gamma), int(has_beta)))
+
+
+def rowop_host(op: str, x: torch.Tensor, out: torch.Tensor, workspace: torch.Tensor, *,
+               gamma: Optional[torch.Tensor] = None, beta: Optional[torch.Tensor] = None,
+               eps: float = 1e-5, causal_period: int = 0, causal_offset: int = 0, stream=None) -> torch.Tensor:
+    """akg_rowop_host: x, out, gamma, beta are HOST tensors (pinned for overlap), workspace
+    is a device byte tensor the caller owns.  Enqueues on the current stream and returns."""
+    if x.is_cuda or out.is_cuda or not workspace.is_cuda:
+        raise ValueError("x / out must be host tensors and workspace a device tensor")
+    if x.dim() != 2 or out.shape != x.shape or out.dtype != x.dtype:
+        raise ValueError("x and out must be 2-D host tensors of the same shape and dtype")
+    if x.shape[1] > 1 and (x.stride(1) != 1 or out.stride(1) != 1):
+        raise ValueError("the last axis must be contiguous")
+    rows, cols = x.shape
+    xs = x.stride(0) if rows > 1 else cols
+    ys = out.stride(0) if rows > 1 else cols
+    mask = None
+    if causal_period > 0:
+        mask = Mask()
+        mask.causal, mask.causal_period, mask.causal_offset = 1, int(causal_period), int(causal_offset)
+    for v, what in ((gamma, "gamma"), (beta, "beta")):
+        if v is not None and (v.is_cuda or v.dtype != x.dtype or v.numel() != cols or not v.is_contiguous()):
+            raise ValueError(f"{what} must be a contiguous host vector of cols elements of x's dtype")
+    with torch.cuda.device(workspace.device):
+        st = lib().akg_rowop_host(OPS[op], x.data_ptr(), out.data_ptr(), rows, cols, xs, ys, _dtype_code(x),
+                                  None if gamma is None else gamma.data_ptr(),
+                                  None if beta is None else beta.data_ptr(), float(eps),
+                                  ctypes.byref(mask) if mask is not None else None,
+                                  workspace.data_ptr(), workspace.numel() * workspace.element_size(),
+                                  _stream(stream))
+    _check(st, "akg_rowop_host")
+    return out
 
 
 def _softmax_like(fn_name, x, out, mask, stream):

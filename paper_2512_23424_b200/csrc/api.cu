@@ -5,6 +5,7 @@
 #include <cmath>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 
 #include "../../include/akg.h"
 #include "launch.cuh"
@@ -46,6 +47,7 @@ struct Call {
   const void* gamma; const void* beta;
   float eps;
   void* stream;
+  int64_t row_base = 0;      // global index of row 0 (host-buffer chunks)
 };
 
 akg_status validate(const Call& c, const char* name) {
@@ -314,6 +316,8 @@ akg_status run(const Call& c, const char* name) {
     }
   }
   p.status = nullptr;
+  p.row_base = c.row_base;
+  if (c.row_base != 0) { p.interleave = 0; if (p.add_mode == 2) p.add_mode = 0; }
 
   const int forced = g_forced_variant.load();
   const bool vec = vector_ok(c);
@@ -377,6 +381,118 @@ akg_status run(const Call& c, const char* name) {
   return AKG_OK;
 }
 
+// ---- host-buffer pipeline ------------------------------------------------------------
+// Three internal streams per device, each owning one slot of the caller's workspace:
+// chunk i goes host -> slot (i % 3) -> kernel in place -> host on stream (i % 3), so the
+// copy engines (both directions) and the SMs work on different chunks at the same time.
+constexpr int kHostSlots = 3;
+struct HostPipe {
+  cudaStream_t s[kHostSlots];
+  cudaEvent_t done[kHostSlots];
+  cudaEvent_t start, vectors;
+  bool ready = false;
+};
+std::mutex g_pipe_mu;
+HostPipe g_pipes[64];
+
+akg_status cuda_fail(const char* name, cudaError_t err) {
+  (void)cudaGetLastError();
+  std::snprintf(t_error, sizeof t_error, "%s: %s", name, cudaGetErrorString(err));
+  return AKG_ERR_CUDA;
+}
+
+size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+size_t host_vector_bytes(int64_t cols, int dtype, bool gamma, bool beta) {
+  const size_t one = round_up(static_cast<size_t>(cols) * ((dtype == AKG_F32) ? 4 : 2), 256);
+  return one * ((gamma ? 1 : 0) + (beta ? 1 : 0));
+}
+
+akg_status run_host(const Call& hc, const char* name, void* workspace, size_t ws_bytes) {
+  t_error[0] = '\0';
+  akg_status st = validate(hc, name);              // same rules; the pointers are host pointers here
+  if (st != AKG_OK) return st;
+  if (hc.rows == 0 || hc.cols == 0) return AKG_OK;
+  if (hc.mask != nullptr && hc.mask->additive != nullptr)
+    return fail(AKG_ERR_UNSUPPORTED, "%s: an additive mask is not supported with host buffers", name);
+  if (workspace == nullptr || !aligned16(workspace))
+    return fail(AKG_ERR_INVALID_ARG, "%s: workspace must be a 16-byte aligned device pointer", name);
+  const size_t es = (hc.dtype == AKG_F32) ? 4 : 2;
+  const size_t row_bytes = static_cast<size_t>(hc.cols) * es;
+  const size_t vec_bytes = host_vector_bytes(hc.cols, hc.dtype, hc.gamma != nullptr, hc.beta != nullptr);
+  if (ws_bytes < vec_bytes + kHostSlots * round_up(row_bytes, 256))
+    return fail(AKG_ERR_INVALID_ARG, "%s: workspace too small (see akg_host_workspace_bytes)", name);
+  const size_t slot_bytes = ((ws_bytes - vec_bytes) / kHostSlots) & ~static_cast<size_t>(255);
+  int64_t chunk_rows = static_cast<int64_t>(slot_bytes / row_bytes);
+  // about a dozen chunks so the pipeline fills, but no chunk under 4 MiB (copy efficiency)
+  int64_t want = (hc.rows + 11) / 12;
+  const int64_t min_rows = static_cast<int64_t>(((size_t(4) << 20) + row_bytes - 1) / row_bytes);
+  if (want < min_rows) want = min_rows;
+  if (chunk_rows > want) chunk_rows = want;
+  if (chunk_rows < 1) chunk_rows = 1;
+
+  int dev = 0;
+  cudaError_t err = cudaGetDevice(&dev);
+  if (err != cudaSuccess) return cuda_fail(name, err);
+  if (dev < 0 || dev >= 64) return fail(AKG_ERR_UNSUPPORTED, "%s: device index above 63", name);
+  std::lock_guard<std::mutex> lock(g_pipe_mu);
+  HostPipe& pipe = g_pipes[dev];
+  if (!pipe.ready) {
+    for (int k = 0; k < kHostSlots; ++k) {
+      if ((err = cudaStreamCreateWithFlags(&pipe.s[k], cudaStreamNonBlocking)) != cudaSuccess) return cuda_fail(name, err);
+      if ((err = cudaEventCreateWithFlags(&pipe.done[k], cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(name, err);
+    }
+    if ((err = cudaEventCreateWithFlags(&pipe.start, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(name, err);
+    if ((err = cudaEventCreateWithFlags(&pipe.vectors, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(name, err);
+    pipe.ready = true;
+  }
+  cudaStream_t user = static_cast<cudaStream_t>(hc.stream);
+  unsigned char* ws = static_cast<unsigned char*>(workspace);
+  void* d_gamma = nullptr;
+  void* d_beta = nullptr;
+  size_t off = 0;
+  if ((err = cudaEventRecord(pipe.start, user)) != cudaSuccess) return cuda_fail(name, err);
+  for (int k = 0; k < kHostSlots; ++k)
+    if ((err = cudaStreamWaitEvent(pipe.s[k], pipe.start, 0)) != cudaSuccess) return cuda_fail(name, err);
+  if (hc.gamma != nullptr) {
+    d_gamma = ws + off; off += round_up(row_bytes, 256);
+    if ((err = cudaMemcpyAsync(d_gamma, hc.gamma, row_bytes, cudaMemcpyHostToDevice, pipe.s[0])) != cudaSuccess) return cuda_fail(name, err);
+  }
+  if (hc.beta != nullptr) {
+    d_beta = ws + off; off += round_up(row_bytes, 256);
+    if ((err = cudaMemcpyAsync(d_beta, hc.beta, row_bytes, cudaMemcpyHostToDevice, pipe.s[0])) != cudaSuccess) return cuda_fail(name, err);
+  }
+  if (off > 0) {
+    if ((err = cudaEventRecord(pipe.vectors, pipe.s[0])) != cudaSuccess) return cuda_fail(name, err);
+    for (int k = 1; k < kHostSlots; ++k)
+      if ((err = cudaStreamWaitEvent(pipe.s[k], pipe.vectors, 0)) != cudaSuccess) return cuda_fail(name, err);
+  }
+  const unsigned char* hx = static_cast<const unsigned char*>(hc.x);
+  unsigned char* hy = static_cast<unsigned char*>(hc.y);
+  int64_t chunk = 0;
+  for (int64_t r0 = 0; r0 < hc.rows; r0 += chunk_rows, ++chunk) {
+    const int k = static_cast<int>(chunk % kHostSlots);
+    const int64_t n = (hc.rows - r0 < chunk_rows) ? hc.rows - r0 : chunk_rows;
+    unsigned char* slot = ws + vec_bytes + static_cast<size_t>(k) * slot_bytes;
+    err = cudaMemcpy2DAsync(slot, row_bytes, hx + static_cast<size_t>(r0) * hc.xs * es, static_cast<size_t>(hc.xs) * es,
+                            row_bytes, static_cast<size_t>(n), cudaMemcpyHostToDevice, pipe.s[k]);
+    if (err != cudaSuccess) return cuda_fail(name, err);
+    Call dc = hc;
+    dc.x = slot; dc.y = slot; dc.rows = n; dc.xs = hc.cols; dc.ys = hc.cols;
+    dc.gamma = d_gamma; dc.beta = d_beta; dc.stream = pipe.s[k]; dc.row_base = r0;
+    st = run(dc, name);
+    if (st != AKG_OK) return st;
+    err = cudaMemcpy2DAsync(hy + static_cast<size_t>(r0) * hc.ys * es, static_cast<size_t>(hc.ys) * es, slot, row_bytes,
+                            row_bytes, static_cast<size_t>(n), cudaMemcpyDeviceToHost, pipe.s[k]);
+    if (err != cudaSuccess) return cuda_fail(name, err);
+  }
+  for (int k = 0; k < kHostSlots; ++k) {
+    if ((err = cudaEventRecord(pipe.done[k], pipe.s[k])) != cudaSuccess) return cuda_fail(name, err);
+    if ((err = cudaStreamWaitEvent(user, pipe.done[k], 0)) != cudaSuccess) return cuda_fail(name, err);
+  }
+  return AKG_OK;
+}
+
 }  // namespace
 }  // namespace akg
 
@@ -411,6 +527,30 @@ akg_status akg_rmsnorm(const void* x, void* y, int64_t rows, int64_t cols, int64
   Call c{OP_RMSNORM, x, y, rows, cols, x_row_stride, y_row_stride, static_cast<int>(dtype), nullptr,
          weight, nullptr, eps, stream};
   return run(c, "akg_rmsnorm");
+}
+
+akg_status akg_rowop_host(akg_op op, const void* x_host, void* y_host, int64_t rows, int64_t cols,
+                          int64_t x_row_stride, int64_t y_row_stride, akg_dtype dtype, const void* gamma_host,
+                          const void* beta_host, float eps, const akg_mask* mask, void* workspace,
+                          size_t workspace_bytes, void* stream) {
+  if (op < AKG_OP_SOFTMAX || op > AKG_OP_RMSNORM)
+    return fail(AKG_ERR_INVALID_ARG, "%s: unknown operator", "akg_rowop_host");
+  const bool softmax_like = (op == AKG_OP_SOFTMAX || op == AKG_OP_LOG_SOFTMAX);
+  Call c{static_cast<int>(op), x_host, y_host, rows, cols, x_row_stride, y_row_stride, static_cast<int>(dtype),
+         softmax_like ? mask : nullptr, softmax_like ? nullptr : gamma_host,
+         op == AKG_OP_LAYERNORM ? beta_host : nullptr, softmax_like ? 0.f : eps, stream};
+  return run_host(c, "akg_rowop_host", workspace, workspace_bytes);
+}
+
+size_t akg_host_workspace_bytes(int64_t rows, int64_t cols, akg_dtype dtype, int has_gamma, int has_beta) {
+  if (rows <= 0 || cols <= 0 || (dtype != AKG_F32 && dtype != AKG_BF16)) return 0;
+  const size_t row_bytes = static_cast<size_t>(cols) * ((dtype == AKG_F32) ? 4 : 2);
+  size_t chunk_rows = (static_cast<size_t>(rows) + 11) / 12;
+  const size_t min_rows = ((size_t(4) << 20) + row_bytes - 1) / row_bytes;
+  if (chunk_rows < min_rows) chunk_rows = min_rows;
+  if (chunk_rows > static_cast<size_t>(rows)) chunk_rows = static_cast<size_t>(rows);
+  return host_vector_bytes(cols, dtype, has_gamma != 0, has_beta != 0) +
+         kHostSlots * round_up(chunk_rows * row_bytes, 256);
 }
 
 const char* akg_status_string(akg_status status) {

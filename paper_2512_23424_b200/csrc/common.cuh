@@ -28,6 +28,7 @@ struct RowParams {
   int period_pow2;          // 1: period is a power of two (row & (period - 1))
   int add_mode;             // 0: row % add_rows, 1: add_rows == 1, 2: add_rows >= rows
   int interleave;           // 1: visit the rows of a causal period short/long alternately
+  long long row_base;       // global index of row 0 (mask rules use row + row_base); 0 unless chunked
   int* status;              // device status word (bounded waits report here)
 };
 
@@ -121,7 +122,8 @@ template <int OP> struct OpTraits {
 // Number of leading live columns of a row (the rest is masked by the causal rule).
 __device__ __forceinline__ long long live_cols(const RowParams& p, long long row) {
   if (!p.causal) return p.cols;
-  const long long rp = p.period_pow2 ? (row & (p.period - 1)) : (row % p.period);
+  const long long g = row + p.row_base;
+  const long long rp = p.period_pow2 ? (g & (p.period - 1)) : (g % p.period);
   long long l = rp + p.offset + 1;
   return l < 0 ? 0 : (l > p.cols ? p.cols : l);
 }
@@ -141,7 +143,7 @@ __device__ __forceinline__ long long balanced_row(const RowParams& p, long long 
 
 // Row of the additive mask that row `row` uses.
 __device__ __forceinline__ long long add_row(const RowParams& p, long long row) {
-  return p.add_mode == 1 ? 0 : (p.add_mode == 2 ? row : row % p.add_rows);
+  return p.add_mode == 1 ? 0 : (p.add_mode == 2 ? row + p.row_base : (row + p.row_base) % p.add_rows);
 }
 
 // ---------------------------------------------------------------------------------
