@@ -391,7 +391,9 @@ def run_ours(args):
         for k in (1, 2, 3, 4, 5):
             wk = w if k == HEADLINE else wl.make_config(k)
             dwk = DeviceWorkload(wk, pairs_for(wk))
-            reps = {1: 2000, 2: 1000, 3: 300, 4: 300, 5: 100}[k]
+            # launches per configuration at the default --steps 1000; fewer steps scale them down
+            full = {1: 2000, 2: 1000, 3: 300, 4: 300, 5: 100}[k]
+            reps = max(10, min(full, full * args.steps // 1000))
             sk = time_launches(dwk, reps, 10) / reps
             bk = wk.algorithmic_bytes()
             row = {"workload": wl.CONFIG_NAMES[k], "kernel": binding.last_kernel(), "us": sk * 1e6,
@@ -399,7 +401,7 @@ def run_ours(args):
             if k == 1:
                 row["note"] = ("latency-bound (0.5 MiB, L2-resident); GB/s not meaningful; 'us' is paced by the "
                                "host's launch rate, 'graph_us' is one launch inside a CUDA graph of 256")
-                row["graph_us"] = graph_launch_us(wk)
+                row["graph_us"] = graph_launch_us(wk, replays=max(2, min(20, args.steps // 50)))
             else:
                 row.update({"gbs": bk / sk / 1e9, "frac_measured": bk / sk / 1e9 / peak,
                             "frac_nominal": bk / sk / 1e9 / NOMINAL_HBM_GBS, "algorithmic_bytes": bk,

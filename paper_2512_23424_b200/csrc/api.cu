@@ -28,6 +28,7 @@ std::atomic<int> g_tune_reg_general{0};   // 1 = never take the predicate-free n
 std::atomic<int> g_tune_cluster_mode{0};  // 0 = planner's choice, 1 = row resident in shared memory, 2 = two-pass split
 std::atomic<int> g_tune_tma_mode{0};      // 0 = planner's choice, 1 = ring-fed register kernel, 2 = shared-memory passes
 std::atomic<int> g_tune_interleave{0};    // 1 = visit causal rows short/long alternately (default: storage order)
+std::atomic<int> g_tune_pdl{0};           // 2 = launch without programmatic stream serialisation
 
 __device__ int g_status_word = 0;
 
@@ -355,6 +356,9 @@ akg_status run(const Call& c, const char* name) {
   if (!planned) return fail(AKG_ERR_UNSUPPORTED, "%s: the forced kernel family cannot run this call", name);
 
   cudaStream_t stream = static_cast<cudaStream_t>(c.stream);
+  // programmatic dependent launch hides the launch gap of back-to-back calls; cluster
+  // launches measured slower with it (dependent clusters take SMs from the tail), so not there
+  plan.pdl = (g_tune_pdl.load() == 2 || (plan.variant == V_CLUSTER && g_tune_pdl.load() != 1)) ? 0 : 1;
   cudaError_t err;
   switch (c.op) {
     case OP_SOFTMAX: err = launch_op<OP_SOFTMAX>(plan, c.dtype, p, stream); break;
@@ -589,6 +593,7 @@ akg_status akg_set_tuning(const char* key, int value) {
   else if (!std::strcmp(key, "cluster_mode")) g_tune_cluster_mode.store(value);
   else if (!std::strcmp(key, "tma_mode")) g_tune_tma_mode.store(value);
   else if (!std::strcmp(key, "interleave")) g_tune_interleave.store(value);
+  else if (!std::strcmp(key, "pdl")) g_tune_pdl.store(value);
   else return fail(AKG_ERR_INVALID_ARG, "akg_set_tuning: unknown key %s", key);
   return AKG_OK;
 }

@@ -41,6 +41,17 @@ __host__ __device__ constexpr unsigned smem_header_bytes(int threads) {
   return (kMaxBuf * 8u + (2u * (threads / 32) + 2u * kMaxCluster) * 12u + 127u) & ~127u;
 }
 
+// Programmatic dependent launch.  Every kernel starts with this: it waits until the
+// kernel launched before it on the stream has completed and its writes are visible
+// (so stream order is kept exactly), then lets the kernel launched after it begin to
+// place its CTAs while this one drains.  Both instructions do nothing when the launch
+// did not ask for programmatic serialisation.  What is gained is the launch latency
+// between back-to-back kernels (about 2.5 us on B200, a tenth of a 20 us kernel).
+__device__ __forceinline__ void pdl_prologue() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kNegInf = -__builtin_huge_valf();
 

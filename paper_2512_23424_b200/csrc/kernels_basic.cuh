@@ -32,6 +32,7 @@ template <int OP> __device__ __forceinline__ float masked_fill(const RowScalars&
 // ------------------------------------------------------------------------------------
 template <int OP, typename T, int G, int VPT, int THREADS>
 __global__ void __launch_bounds__(THREADS) reg_kernel(const RowParams p) {
+  pdl_prologue();
   using E = Elem<T>;
   constexpr int EPV = E::EPV;
   constexpr int N = VPT * EPV;
@@ -153,6 +154,7 @@ __global__ void __launch_bounds__(THREADS) reg_kernel(const RowParams p) {
 // ------------------------------------------------------------------------------------
 template <int OP, typename T, int THREADS>
 __global__ void __launch_bounds__(THREADS) stream_kernel(const RowParams p) {
+  pdl_prologue();
   using E = Elem<T>;
   constexpr int NW = THREADS / 32;
   constexpr bool SM = OpTraits<OP>::kSoftmaxLike;

@@ -144,6 +144,7 @@ __device__ __forceinline__ void norm_row_full(const RowParams& p, long long row,
 
 template <int OP, typename T, int G, int VPT, int THREADS>
 __global__ void __launch_bounds__(THREADS, kRegMinBlocks<THREADS>) reg_norm_full(const RowParams p) {
+  pdl_prologue();
   constexpr int RPC = THREADS / G;
   constexpr int NW = G / 32;
   __shared__ float red[2][2][NW > 1 ? NW : 1];

@@ -48,6 +48,7 @@ struct RowRing {
 
 template <int OP, typename T, int VPT, int THREADS>
 __global__ void __launch_bounds__(THREADS, kRegMinBlocks<THREADS>) ring_norm_full(const RowParams p, const int nbuf) {
+  pdl_prologue();
   constexpr int EPV = Elem<T>::EPV;
   constexpr int NW = THREADS / 32;
   constexpr uint32_t kRowBytes = THREADS * VPT * 16u;
@@ -78,6 +79,7 @@ __global__ void __launch_bounds__(THREADS, kRegMinBlocks<THREADS>) ring_norm_ful
 
 template <int OP, typename T, int VPT, int THREADS>
 __global__ void __launch_bounds__(THREADS, kRegMinBlocks<THREADS>) ring_softmax(const RowParams p, const int nbuf) {
+  pdl_prologue();
   constexpr int EPV = Elem<T>::EPV;
   constexpr int NW = THREADS / 32;
   static_assert(VPT <= 8, "row body is specialised for up to eight iterations");

@@ -79,6 +79,7 @@ struct SmemGeom {
 
 template <int OP, typename T, int THREADS>
 __global__ void __launch_bounds__(THREADS) smem_kernel(const RowParams p, const SmemGeom g) {
+  pdl_prologue();
   using E = Elem<T>;
   constexpr int EPV = E::EPV;
   constexpr int NW = THREADS / 32;

@@ -130,6 +130,7 @@ __device__ __forceinline__ void softmax_row(const RowParams& p, long long row, i
 
 template <int OP, typename T, int G, int VPT, int THREADS>
 __global__ void __launch_bounds__(THREADS, kRegMinBlocks<THREADS>) reg_softmax(const RowParams p) {
+  pdl_prologue();
   constexpr int EPV = Elem<T>::EPV;
   constexpr int RPC = THREADS / G;
   constexpr int NW = G / 32;

@@ -37,6 +37,7 @@ __device__ __forceinline__ uint4 ld_hint(const void* p, uint64_t pol) {
 template <int OP, typename T, int THREADS>
 __global__ void __launch_bounds__(THREADS, (1024 / THREADS) > 0 ? (1024 / THREADS) : 1)
 split_kernel(const RowParams p, const int slice_vecs) {
+  pdl_prologue();
   using E = Elem<T>;
   constexpr int EPV = E::EPV;
   constexpr int NW = THREADS / 32;

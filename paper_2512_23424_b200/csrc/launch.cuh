@@ -21,6 +21,7 @@ struct LaunchPlan {
   int stages;         // ring depth (V_TMA)
   size_t smem;        // dynamic shared memory per CTA
   int mode;           // V_TMA: 1 = register kernels fed by a ring, 0 = shared-memory-resident kernel
+  int pdl;            // 1 = launch with programmatic stream serialisation (see pdl_prologue)
 };
 
 template <int OP>

@@ -24,6 +24,40 @@ namespace akg {
   X(512, 1, 512) X(512, 2, 512) X(512, 4, 512) X(512, 8, 512) \
   X(1024, 1, 1024) X(1024, 2, 1024) X(1024, 4, 1024) X(1024, 8, 1024)
 
+// Fill the launch attributes: programmatic stream serialisation when the plan asks for
+// it, a cluster dimension when cluster > 1.  Returns the number of attributes set.
+inline unsigned launch_attrs(cudaLaunchAttribute* attr, const LaunchPlan& plan, int cluster) {
+  unsigned n = 0;
+  if (cluster > 1) {
+    attr[n].id = cudaLaunchAttributeClusterDimension;
+    attr[n].val.clusterDim.x = static_cast<unsigned>(cluster);
+    attr[n].val.clusterDim.y = 1;
+    attr[n].val.clusterDim.z = 1;
+    ++n;
+  }
+  if (plan.pdl) {
+    attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+  }
+  return n;
+}
+
+// A plain (non-cluster) launch with the plan's attributes.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_plain(void (*kernel)(KArgs...), const LaunchPlan& plan, unsigned grid, int threads, size_t smem,
+                         cudaStream_t s, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attr[2];
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(static_cast<unsigned>(threads));
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cfg.attrs = attr;
+  cfg.numAttrs = launch_attrs(attr, plan, 1);
+  return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
 // Launch smem_kernel (TMA ring, optionally clustered).  plan.grid == 0 asks for as many
 // clusters as can be co-resident (capped by the number of rows).
 template <int OP, typename T, int THREADS>
@@ -37,8 +71,8 @@ cudaError_t launch_smem(const LaunchPlan& plan, const RowParams& p, cudaStream_t
   if (err != cudaSuccess) return err;
 
   cudaLaunchConfig_t cfg = {};
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;       // always first: the occupancy query reads it
   attr[0].val.clusterDim.x = static_cast<unsigned>(plan.cluster);
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
@@ -78,6 +112,11 @@ cudaError_t launch_smem(const LaunchPlan& plan, const RowParams& p, cudaStream_t
   g.nbuf = plan.stages;
   g.slice_vecs = plan.vpt;          // V_TMA / V_CLUSTER reuse the field: vectors per CTA slice
   g.buf_bytes = static_cast<unsigned>((static_cast<size_t>(plan.vpt) * 16 + 127) & ~static_cast<size_t>(127));
+  if (plan.pdl) {
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.numAttrs = 2;
+  }
   return cudaLaunchKernelEx(&cfg, kernel, p, g);
 }
 
@@ -111,8 +150,7 @@ cudaError_t launch_ring(Kernel kernel, int threads, const LaunchPlan& plan, cons
   if (ctas < 1) return cudaErrorLaunchOutOfResources;
   long long grid = plan.grid ? plan.grid : ctas;
   if (grid > p.rows) grid = p.rows;
-  kernel<<<static_cast<unsigned>(grid), threads, plan.smem, s>>>(p, plan.stages);
-  return cudaGetLastError();
+  return launch_plain(kernel, plan, static_cast<unsigned>(grid), threads, plan.smem, s, p, plan.stages);
 }
 
 // Launch split_kernel (cluster per row, two streaming passes, second one from L2).
@@ -126,8 +164,8 @@ cudaError_t launch_split(const LaunchPlan& plan, const RowParams& p, cudaStream_
   cudaError_t err = cudaGetDevice(&dev);
   if (err != cudaSuccess) return err;
   cudaLaunchConfig_t cfg = {};
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;       // always first: the occupancy query reads it
   attr[0].val.clusterDim.x = static_cast<unsigned>(plan.cluster);
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
@@ -161,14 +199,18 @@ cudaError_t launch_split(const LaunchPlan& plan, const RowParams& p, cudaStream_
   if (clusters > p.rows) clusters = p.rows;
   if (clusters < 1) clusters = 1;
   cfg.gridDim = dim3(static_cast<unsigned>(clusters * plan.cluster));
+  if (plan.pdl) {
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.numAttrs = 2;
+  }
   return cudaLaunchKernelEx(&cfg, kernel, p, plan.vpt);
 }
 
 template <int OP, typename T>
 cudaError_t launch_typed(const LaunchPlan& plan, const RowParams& p, cudaStream_t s) {
   if (plan.variant == V_STREAM) {
-    stream_kernel<OP, T, 256><<<plan.grid, 256, 0, s>>>(p);
-    return cudaGetLastError();
+    return launch_plain(stream_kernel<OP, T, 256>, plan, plan.grid, 256, 0, s, p);
   }
   if (plan.variant == V_REG) {
     // plan.stages == 1 marks a row of exactly group * vpt vectors (the predicate-free
@@ -176,14 +218,12 @@ cudaError_t launch_typed(const LaunchPlan& plan, const RowParams& p, cudaStream_
 #define AKG_REG_CASE(G_, V_, T_)                                              \
   if (plan.group == (G_) && plan.vpt == (V_) && plan.threads == (T_)) {       \
     if constexpr (OpTraits<OP>::kSoftmaxLike) {                               \
-      reg_softmax<OP, T, G_, V_, T_><<<plan.grid, T_, 0, s>>>(p);             \
+      return launch_plain(reg_softmax<OP, T, G_, V_, T_>, plan, plan.grid, T_, 0, s, p);      \
     } else {                                                                  \
       if (plan.stages == 1)                                                   \
-        reg_norm_full<OP, T, G_, V_, T_><<<plan.grid, T_, 0, s>>>(p);         \
-      else                                                                    \
-        reg_kernel<OP, T, G_, V_, T_><<<plan.grid, T_, 0, s>>>(p);            \
+        return launch_plain(reg_norm_full<OP, T, G_, V_, T_>, plan, plan.grid, T_, 0, s, p);  \
+      return launch_plain(reg_kernel<OP, T, G_, V_, T_>, plan, plan.grid, T_, 0, s, p);       \
     }                                                                         \
-    return cudaGetLastError();                                                \
   }
     AKG_REG_SHAPES(AKG_REG_CASE)
 #undef AKG_REG_CASE
