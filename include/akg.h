@@ -143,6 +143,37 @@ akg_status akg_rowop_host(akg_op op, const void* x_host, void* y_host, int64_t r
  * at least 4 MiB; 0 for a malformed shape. */
 size_t akg_host_workspace_bytes(int64_t rows, int64_t cols, akg_dtype dtype, int has_gamma, int has_beta);
 
+/* Size of the staging area built into the library (see akg_rowop_host_static). */
+#define AKG_STATIC_STAGING_BYTES (16u << 20)
+
+/* akg_rowop_host for callers that cannot provide a device workspace (the paper has no
+ * counterpart: this is a convenience of this library).  Meant for code that is given
+ * host buffers and a stream but no way to allocate device memory: a plug-in inside an
+ * application whose memory pool it may not touch, a service that must not allocate
+ * after start-up, a host-only component of a larger pipeline.  Same operators, same
+ * arguments and the same results as akg_rowop_host, minus the workspace: the chunks are
+ * staged in a fixed area of AKG_STATIC_STAGING_BYTES (16 MiB) that is part of the
+ * library image.  Every GPU on which the library is loaded holds that area until the
+ * process exits, whether or not this function is ever called.
+ *   - Nothing is allocated or freed here or in anything this function calls, and no
+ *     streams or events are created: uploads, kernels and downloads run one after the
+ *     other on `stream` (no overlap between them; use akg_rowop_host for throughput).
+ *   - Size limit: one row plus gamma / beta must fit the area, i.e.
+ *     round_up(cols * element size, 256) * (1 + number of vectors) <=
+ *     AKG_STATIC_STAGING_BYTES; a longer row is AKG_ERR_UNSUPPORTED with a message
+ *     naming the limit, and nothing is enqueued.  Any number of rows is fine.
+ *   - The first call on each device looks up the device address of the area (with that
+ *     device current) and keeps it; make that first call outside any stream capture.
+ *   - The area is shared by all calls on the device and keeps the previous call's data.
+ *     Nothing in it needs clearing (every chunk is overwritten by its upload before a
+ *     kernel reads it), but two calls whose work overlaps on the GPU, from different
+ *     streams or threads, race on it: keep such calls on one stream, or order them.
+ * Errors otherwise as for akg_rowop_host. */
+akg_status akg_rowop_host_static(akg_op op, const void* x_host, void* y_host, int64_t rows, int64_t cols,
+                                 int64_t x_row_stride, int64_t y_row_stride, akg_dtype dtype,
+                                 const void* gamma_host, const void* beta_host, float eps,
+                                 const akg_mask* mask, void* stream);
+
 /* Human-readable name of a status code (static storage, never NULL). */
 const char* akg_status_string(akg_status status);
 

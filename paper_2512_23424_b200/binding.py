@@ -251,6 +251,46 @@ def rowop_host(op: str, x: torch.Tensor, out: torch.Tensor, workspace: torch.Ten
     return out
 
 
+STATIC_STAGING_BYTES = 16 << 20
+
+
+def rowop_host_static(op: str, x: torch.Tensor, out: torch.Tensor, *, gamma: Optional[torch.Tensor] = None,
+                      beta: Optional[torch.Tensor] = None, eps: float = 1e-5, causal_period: int = 0,
+                      causal_offset: int = 0, stream=None) -> torch.Tensor:
+    """akg_rowop_host_static: like rowop_host, for callers that cannot hand over a device
+    workspace (no allocator at hand, or allocation not allowed where they run).  The chunks
+    are staged in the 16 MiB area built into the library; nothing is allocated, on the
+    device or by this wrapper.  x, out, gamma, beta are HOST tensors.  All work is enqueued
+    on one stream (the current one unless given); calls that overlap on the GPU from
+    different streams race on the shared staging area."""
+    if x.is_cuda or out.is_cuda:
+        raise ValueError("x / out must be host tensors")
+    if x.dim() != 2 or out.shape != x.shape or out.dtype != x.dtype:
+        raise ValueError("x and out must be 2-D host tensors of the same shape and dtype")
+    if x.shape[1] > 1 and (x.stride(1) != 1 or out.stride(1) != 1):
+        raise ValueError("the last axis must be contiguous")
+    rows, cols = x.shape
+    xs = x.stride(0) if rows > 1 else cols
+    ys = out.stride(0) if rows > 1 else cols
+    mask = None
+    if causal_period > 0:
+        mask = Mask()
+        mask.causal, mask.causal_period, mask.causal_offset = 1, int(causal_period), int(causal_offset)
+    for v, what in ((gamma, "gamma"), (beta, "beta")):
+        if v is not None and (v.is_cuda or v.dtype != x.dtype or v.numel() != cols or not v.is_contiguous()):
+            raise ValueError(f"{what} must be a contiguous host vector of cols elements of x's dtype")
+    fn = lib().akg_rowop_host_static
+    if not fn.argtypes:
+        vp, i64, ci = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int
+        fn.argtypes = [ci, vp, vp, i64, i64, i64, i64, ci, vp, vp, ctypes.c_float, ctypes.POINTER(Mask), vp]
+        fn.restype = ci
+    st = fn(OPS[op], x.data_ptr(), out.data_ptr(), rows, cols, xs, ys, _dtype_code(x),
+            None if gamma is None else gamma.data_ptr(), None if beta is None else beta.data_ptr(),
+            float(eps), ctypes.byref(mask) if mask is not None else None, _stream(stream))
+    _check(st, "akg_rowop_host_static")
+    return out
+
+
 def _softmax_like(fn_name, x, out, mask, stream):
     rows, cols, xs = _matrix(x, "x")
     if out is None:

@@ -616,3 +616,108 @@ akg_status akg_device_status(int* word_out) {
 }
 
 }  // extern "C"
+
+// ---- host buffers without any allocation ---------------------------------------------------
+// akg_rowop_host needs a device staging area from its caller.  Some callers have no way to
+// get one: a plug-in that is handed host buffers and a stream but no allocator, a service
+// whose device memory is wholly owned by another component's pool, a control loop that may
+// not allocate once it is running.  For them the staging area below is part of the library
+// image: the driver reserves it on every GPU that loads the library and keeps it until the
+// process exits.  It is shared by every call on that GPU and keeps whatever the last call
+// left in it; nothing in it has to start at zero, because each chunk is fully overwritten
+// by its upload before a kernel reads it.
+namespace {
+
+constexpr size_t kStaticStagingBytes = size_t(16) << 20;          // AKG_STATIC_STAGING_BYTES
+static __device__ __align__(256) unsigned char g_static_staging[kStaticStagingBytes];
+
+// In host code `g_static_staging` is only a handle for the runtime, not a device address.
+// The address is asked for once per device, with that device current, and cached.
+akg_status static_staging_address(const char* name, unsigned char** out) {
+  static std::atomic<unsigned char*> cache[64];
+  int dev = 0;
+  cudaError_t err = cudaGetDevice(&dev);
+  if (err != cudaSuccess) return akg::cuda_fail(name, err);
+  if (dev < 0 || dev >= 64) return akg::fail(AKG_ERR_UNSUPPORTED, "%s: device index above 63", name);
+  unsigned char* ptr = cache[dev].load();
+  if (ptr == nullptr) {
+    void* sym = nullptr;
+    err = cudaGetSymbolAddress(&sym, g_static_staging);
+    if (err != cudaSuccess || sym == nullptr) return akg::cuda_fail(name, err);
+    ptr = static_cast<unsigned char*>(sym);
+    cache[dev].store(ptr);
+  }
+  *out = ptr;
+  return AKG_OK;
+}
+
+}  // namespace
+
+extern "C" akg_status akg_rowop_host_static(akg_op op, const void* x_host, void* y_host, int64_t rows, int64_t cols,
+                                            int64_t x_row_stride, int64_t y_row_stride, akg_dtype dtype,
+                                            const void* gamma_host, const void* beta_host, float eps,
+                                            const akg_mask* mask, void* stream) {
+  const char* name = "akg_rowop_host_static";
+  if (op < AKG_OP_SOFTMAX || op > AKG_OP_RMSNORM) return akg::fail(AKG_ERR_INVALID_ARG, "%s: unknown operator", name);
+  const bool softmax_like = (op == AKG_OP_SOFTMAX || op == AKG_OP_LOG_SOFTMAX);
+  akg::Call hc{static_cast<int>(op), x_host, y_host, rows, cols, x_row_stride, y_row_stride, static_cast<int>(dtype),
+               softmax_like ? mask : nullptr, softmax_like ? nullptr : gamma_host,
+               op == AKG_OP_LAYERNORM ? beta_host : nullptr, softmax_like ? 0.f : eps, stream};
+  akg::t_error[0] = '\0';
+  akg_status st = akg::validate(hc, name);
+  if (st != AKG_OK) return st;
+  if (hc.rows == 0 || hc.cols == 0) return AKG_OK;
+  if (hc.mask != nullptr && hc.mask->additive != nullptr)
+    return akg::fail(AKG_ERR_UNSUPPORTED, "%s: an additive mask is not supported with host buffers", name);
+  const size_t es = (hc.dtype == AKG_F32) ? 4 : 2;
+  const size_t row_bytes = static_cast<size_t>(hc.cols) * es;
+  const size_t vec_bytes = akg::host_vector_bytes(hc.cols, hc.dtype, hc.gamma != nullptr, hc.beta != nullptr);
+  if (vec_bytes + akg::round_up(row_bytes, 256) > kStaticStagingBytes) {
+    std::snprintf(akg::t_error, sizeof akg::t_error,
+                  "%s: a row of %lld columns (with its vectors) does not fit the built-in %zu-byte staging area; "
+                  "use akg_rowop_host with a workspace of your own", name, static_cast<long long>(hc.cols),
+                  kStaticStagingBytes);
+    return AKG_ERR_UNSUPPORTED;
+  }
+  unsigned char* ws = nullptr;
+  st = static_staging_address(name, &ws);
+  if (st != AKG_OK) return st;
+
+  // One slot, one stream: upload a chunk, run the operator on it in place, download it.
+  cudaStream_t user = static_cast<cudaStream_t>(hc.stream);
+  cudaError_t err;
+  void* d_gamma = nullptr;
+  void* d_beta = nullptr;
+  size_t off = 0;
+  if (hc.gamma != nullptr) {
+    d_gamma = ws + off; off += akg::round_up(row_bytes, 256);
+    if ((err = cudaMemcpyAsync(d_gamma, hc.gamma, row_bytes, cudaMemcpyHostToDevice, user)) != cudaSuccess)
+      return akg::cuda_fail(name, err);
+  }
+  if (hc.beta != nullptr) {
+    d_beta = ws + off; off += akg::round_up(row_bytes, 256);
+    if ((err = cudaMemcpyAsync(d_beta, hc.beta, row_bytes, cudaMemcpyHostToDevice, user)) != cudaSuccess)
+      return akg::cuda_fail(name, err);
+  }
+  unsigned char* slot = ws + vec_bytes;
+  const int64_t chunk_rows = static_cast<int64_t>((kStaticStagingBytes - vec_bytes) / row_bytes);
+  const unsigned char* hx = static_cast<const unsigned char*>(hc.x);
+  unsigned char* hy = static_cast<unsigned char*>(hc.y);
+  for (int64_t r0 = 0; r0 < hc.rows; r0 += chunk_rows) {
+    const int64_t n = (hc.rows - r0 < chunk_rows) ? hc.rows - r0 : chunk_rows;
+    err = cudaMemcpy2DAsync(slot, row_bytes, hx + static_cast<size_t>(r0) * hc.xs * es, static_cast<size_t>(hc.xs) * es,
+                            row_bytes, static_cast<size_t>(n), cudaMemcpyHostToDevice, user);
+    if (err != cudaSuccess) return akg::cuda_fail(name, err);
+    akg::Call dc = hc;
+    dc.x = slot; dc.y = slot; dc.rows = n; dc.xs = hc.cols; dc.ys = hc.cols;
+    dc.gamma = d_gamma; dc.beta = d_beta; dc.row_base = r0;
+    st = akg::run(dc, name);
+    if (st != AKG_OK) return st;
+    err = cudaMemcpy2DAsync(hy + static_cast<size_t>(r0) * hc.ys * es, static_cast<size_t>(hc.ys) * es, slot, row_bytes,
+                            row_bytes, static_cast<size_t>(n), cudaMemcpyDeviceToHost, user);
+    if (err != cudaSuccess) return akg::cuda_fail(name, err);
+  }
+  return AKG_OK;
+}
+
+static_assert(kStaticStagingBytes == AKG_STATIC_STAGING_BYTES, "the header states the size of the staging area");
