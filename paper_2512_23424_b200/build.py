@@ -49,7 +49,8 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
 
     def compile_one(src: str) -> str:
         obj = os.path.join(_OBJ, os.path.basename(src)[:-3] + ".o")
-        cmd = [nvcc, *NVCC_FLAGS, "-I", _INCLUDE, "-c", src, "-o", obj]
+        extra = os.environ.get("AKG_NVCC_EXTRA", "").split()      # e.g. -D switches while experimenting
+        cmd = [nvcc, *NVCC_FLAGS, *extra, "-I", _INCLUDE, "-c", src, "-o", obj]
         res = subprocess.run(cmd, capture_output=True, text=True)
         log = os.path.join(_OBJ, os.path.basename(src)[:-3] + ".ptxas.log")
         with open(log, "w") as fh:

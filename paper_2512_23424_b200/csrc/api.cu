@@ -144,7 +144,7 @@ bool plan_reg(const Call& c, LaunchPlan* plan) {
     else return false;
     group = threads;
   }
-  const int64_t rpc = threads / group;
+  const int64_t rpc = threads / group;          // rows per CTA iteration
   int64_t grid = (c.rows + rpc - 1) / rpc;
   int cap = g_tune_grid_cap.load();
   // the softmax pair runs persistent (two resident waves of CTAs, grid-stride over rows):

@@ -106,22 +106,9 @@ __global__ void __launch_bounds__(THREADS, kRegMinBlocks<THREADS>) ring_softmax(
   uint32_t phase = 0;
   for (long long item = blockIdx.x; item < p.rows; item += step, parity ^= 1) {
     const long long row = balanced_row(p, item);
-    const int live = static_cast<int>(live_cols(p, row));
-    const int live_vecs = (live + EPV - 1) / EPV;
-    const int nk = (live_vecs + THREADS - 1) / THREADS;
     ring.wait(b, phase, p.status);
-#define AKG_SM_CASE(NK_)                                                                              \
-  case NK_:                                                                                           \
-    if constexpr (NK_ <= VPT)                                                                         \
-      softmax_row<OP, T, THREADS, VPT, THREADS, NK_, true>(p, row, threadIdx.x, nvec, live, live_vecs, \
-                                                           red[parity], ring.buf(b));                 \
-    break;
-    switch (nk) {
-      AKG_SM_CASE(0) AKG_SM_CASE(1) AKG_SM_CASE(2) AKG_SM_CASE(3) AKG_SM_CASE(4)
-      AKG_SM_CASE(5) AKG_SM_CASE(6) AKG_SM_CASE(7) AKG_SM_CASE(8)
-      default: break;
-    }
-#undef AKG_SM_CASE
+    softmax_row_dispatch<OP, T, THREADS, VPT, VPT, THREADS, true>(p, row, threadIdx.x, nvec, red[parity],
+                                                                  ring.buf(b));
     if (threadIdx.x == 0) {
       const long long next = item + step * nbuf;
       if (next < p.rows) {

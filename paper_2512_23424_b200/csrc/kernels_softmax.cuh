@@ -1,28 +1,40 @@
 // reg_softmax: register-resident softmax / log-softmax for rows that fit one warp or
 // one CTA, with optional additive and causal masks.
 //
-// Thread t of the G threads of a row owns vectors t, t + G, ..., VPT of them.  With a
-// causal mask only the first NK = ceil(live_vecs / G) of those iterations hold live
-// data; the row body is compiled once per NK and selected by a CTA-uniform switch, so
-// masked iterations cost nothing but their zero-fill stores (no predicated-off work).
+// A group of G threads owns a row (a warp, or the whole CTA; the row body also supports
+// aligned sub-groups with named barriers); thread t of the group owns vectors t, t + G, ...
+// With a causal mask only the first NK = ceil(live_vecs / G) of those iterations hold
+// live data; the row body is compiled once per NK and selected by a group-uniform switch,
+// so masked iterations cost nothing but their fill stores (no predicated-off work).
 // The exponential is evaluated once per live element, against the warp maximum; the
 // cross-warp combine costs one exponential per warp.
+//
 #pragma once
 
 #include "kernels_reg.cuh"
 
 namespace akg {
 
+// Barrier over the G threads of one row group (the whole CTA, or an aligned subset).
+template <int G, int THREADS> __device__ __forceinline__ void group_barrier(int group) {
+  if (G == THREADS) __syncthreads();
+  else asm volatile("bar.sync %0, %1;" :: "r"(group + 1), "r"(G) : "memory");
+}
+
+// One row.  G threads per row, VPT live iterations at most, KFILL >= VPT store iterations
+// (KFILL * G vectors cover the row), NK live iterations for this row.
 // RING = false: the row is read from global memory; RING = true: from the shared-memory
 // buffer at `ring_buf` that a bulk copy has filled with the row's live prefix.
-template <int OP, typename T, int G, int VPT, int THREADS, int NK, bool RING = false>
+// red: [2][THREADS / 32] floats, indexed by the warp's position in the CTA.
+template <int OP, typename T, int G, int VPT, int KFILL, int THREADS, int NK, bool RING = false>
 __device__ __forceinline__ void softmax_row(const RowParams& p, long long row, int tg, int nvec, int live,
-                                            int live_vecs, float (*red)[(G / 32) > 1 ? (G / 32) : 1],
-                                            uint32_t ring_buf = 0) {
+                                            int live_vecs, float (*red)[THREADS / 32], uint32_t ring_buf = 0) {
   using E = Elem<T>;
   constexpr int EPV = E::EPV;
   constexpr int NW = G / 32;
   constexpr int NKA = NK > 0 ? NK : 1;
+  static_assert(NW >= 1 && (NW & (NW - 1)) == 0, "warps per row must be a power of two");
+  static_assert(NK <= VPT && VPT <= KFILL, "live iterations fit the register tile");
   const bool ragged = live_vecs * EPV != live;
   const T* xr = reinterpret_cast<const T*>(p.x) + row * p.xs + tg * EPV;
   T* yr = reinterpret_cast<T*>(p.y) + row * p.ys + tg * EPV;
@@ -79,19 +91,21 @@ __device__ __forceinline__ void softmax_row(const RowParams& p, long long row, i
 
   float M = m_w, S = s_w, my_factor = 1.f;
   if (NW > 1) {
-    if ((threadIdx.x & 31) == 0) { red[0][threadIdx.x >> 5] = m_w; red[1][threadIdx.x >> 5] = s_w; }
-    __syncthreads();
-    M = red[0][0];
+    const int warp_cta = threadIdx.x >> 5;
+    const int wbase = warp_cta & ~(NW - 1);                // first warp of this row's group
+    if ((threadIdx.x & 31) == 0) { red[0][warp_cta] = m_w; red[1][warp_cta] = s_w; }
+    group_barrier<G, THREADS>(warp_cta / NW);
+    // lane l takes the pair of the group's warp (l mod NW); xor-butterflies over NW lanes
+    // give every lane the row maximum and the rescaled sum
+    const float mw = red[0][wbase + (threadIdx.x & (NW - 1))];
+    const float sw = red[1][wbase + (threadIdx.x & (NW - 1))];
+    M = mw;
 #pragma unroll
-    for (int w = 1; w < NW; ++w) M = fmaxf(M, red[0][w]);
+    for (int m = 1; m < NW && m < 32; m <<= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, m));
     const float Ms = (M == kNegInf) ? 0.f : M;
-    S = 0.f;
+    S = sw * ((mw == M) ? 1.f : exp_diff(mw, Ms));          // equal maxima (also +-inf): factor 1
 #pragma unroll
-    for (int w = 0; w < NW; ++w) {
-      const float mw = red[0][w];
-      const float f = (mw == M) ? 1.f : exp_diff(mw, Ms);   // equal maxima (also +-inf): factor 1
-      S = fmaf(red[1][w], f, S);
-    }
+    for (int m = 1; m < NW && m < 32; m <<= 1) S += __shfl_xor_sync(0xffffffffu, S, m);
     my_factor = (m_w == M) ? 1.f : exp_diff(m_w, Ms);
   }
 
@@ -105,12 +119,21 @@ __device__ __forceinline__ void softmax_row(const RowParams& p, long long row, i
     lse_l = logf(S);
     fill = (S != S) ? nan : kNegInf;
   }
+  // the fill value as stored bits: +0, -inf or quiet NaN in the element type
+  uint32_t fill_word = __float_as_uint(fill);
+  if (sizeof(T) == 2) fill_word = (fill_word >> 16) | (fill_word & 0xffff0000u);
+  const uint4 fill_vec = make_uint4(fill_word, fill_word, fill_word, fill_word);
 
 #pragma unroll
-  for (int k = 0; k < VPT; ++k) {
+  for (int k = 0; k < KFILL; ++k) {
     const int idx = tg + k * G;
-    float o[EPV];
-    if (k < NK && (k < NK - 1 || last_ok)) {
+    if (k >= NK) {                                           // compile-time: wholly masked iteration
+      if (idx < nvec) st_stream(yr + k * G * EPV, fill_vec); // constant bits, no conversion
+      continue;
+    }
+    uint4 out_vec = fill_vec;
+    if (k < NK - 1 || last_ok) {
+      float o[EPV];
 #pragma unroll
       for (int j = 0; j < EPV; ++j) {
         if (OP == OP_SOFTMAX) o[j] = v[k < NK ? k : 0][j] * scale;
@@ -120,47 +143,58 @@ __device__ __forceinline__ void softmax_row(const RowParams& p, long long row, i
 #pragma unroll
         for (int j = 0; j < EPV; ++j) if (idx * EPV + j >= live) o[j] = fill;
       }
-    } else {
-#pragma unroll
-      for (int j = 0; j < EPV; ++j) o[j] = fill;
+      out_vec = E::pack(o);
     }
-    if (idx < nvec) st_stream(yr + k * G * EPV, E::pack(o));
+    if (idx < nvec) st_stream(yr + k * G * EPV, out_vec);    // one store site per live iteration
   }
+}
+
+// Pick the body for this row's number of live iterations (uniform over the row's group).
+template <int OP, typename T, int G, int VPT, int KFILL, int THREADS, bool RING = false>
+__device__ __forceinline__ void softmax_row_dispatch(const RowParams& p, long long row, int tg, int nvec,
+                                                     float (*red)[THREADS / 32], uint32_t ring_buf = 0) {
+  constexpr int EPV = Elem<T>::EPV;
+  static_assert(VPT <= 8, "row body is specialised for up to eight iterations");
+  const int live = static_cast<int>(live_cols(p, row));
+  const int live_vecs = (live + EPV - 1) / EPV;
+  const int nk = (live_vecs + G - 1) / G;
+#define AKG_SM_CASE(NK_)                                                                                      \
+  case NK_:                                                                                                   \
+    if constexpr (NK_ <= VPT)                                                                                 \
+      softmax_row<OP, T, G, VPT, KFILL, THREADS, NK_, RING>(p, row, tg, nvec, live, live_vecs, red, ring_buf); \
+    break;
+  switch (nk) {
+    AKG_SM_CASE(0) AKG_SM_CASE(1) AKG_SM_CASE(2) AKG_SM_CASE(3) AKG_SM_CASE(4)
+    AKG_SM_CASE(5) AKG_SM_CASE(6) AKG_SM_CASE(7) AKG_SM_CASE(8)
+    default: break;
+  }
+#undef AKG_SM_CASE
 }
 
 template <int OP, typename T, int G, int VPT, int THREADS>
 __global__ void __launch_bounds__(THREADS, kRegMinBlocks<THREADS>) reg_softmax(const RowParams p) {
   pdl_prologue();
   constexpr int EPV = Elem<T>::EPV;
-  constexpr int RPC = THREADS / G;
-  constexpr int NW = G / 32;
+  constexpr int NWC = THREADS / 32;
   static_assert(OP == OP_SOFTMAX || OP == OP_LOG_SOFTMAX, "softmax pair only");
-  static_assert(VPT <= 8, "row body is specialised for up to eight iterations");
-  __shared__ float red[2][2][NW > 1 ? NW : 1];
-
-  const int tg = threadIdx.x % G;
-  const int grp = threadIdx.x / G;
+  static_assert(G == 32 || G == THREADS, "a warp or a CTA per row");
+  __shared__ float red[2][2][NWC];
   const int nvec = static_cast<int>(p.cols / EPV);
-  int parity = 0;
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
 
-  for (long long rb = static_cast<long long>(blockIdx.x) * RPC; rb < p.rows;
-       rb += static_cast<long long>(gridDim.x) * RPC, parity ^= 1) {
-    if (G != THREADS && rb + grp >= p.rows) continue;
-    const long long row = balanced_row(p, rb + grp);
-    const int live = static_cast<int>(live_cols(p, row));
-    const int live_vecs = (live + EPV - 1) / EPV;
-    const int nk = (live_vecs + G - 1) / G;             // uniform over the threads of the row
-#define AKG_SM_CASE(NK_)                                                                          \
-  case NK_:                                                                                       \
-    if constexpr (NK_ <= VPT)                                                                     \
-      softmax_row<OP, T, G, VPT, THREADS, NK_>(p, row, tg, nvec, live, live_vecs, red[parity]);   \
-    break;
-    switch (nk) {
-      AKG_SM_CASE(0) AKG_SM_CASE(1) AKG_SM_CASE(2) AKG_SM_CASE(3) AKG_SM_CASE(4)
-      AKG_SM_CASE(5) AKG_SM_CASE(6) AKG_SM_CASE(7) AKG_SM_CASE(8)
-      default: break;
+  if constexpr (G == 32) {
+    // a warp per row throughout (rows short enough for one warp's registers)
+    for (long long rb = static_cast<long long>(blockIdx.x) * NWC; rb < p.rows;
+         rb += static_cast<long long>(gridDim.x) * NWC) {
+      if (rb + warp >= p.rows) continue;
+      softmax_row_dispatch<OP, T, 32, VPT, VPT, THREADS>(p, balanced_row(p, rb + warp), lane, nvec, red[0]);
     }
-#undef AKG_SM_CASE
+  } else {
+    // a CTA per row, grid-stride (persistent when the planner caps the grid)
+    int parity = 0;
+    for (long long r = blockIdx.x; r < p.rows; r += gridDim.x, parity ^= 1)
+      softmax_row_dispatch<OP, T, THREADS, VPT, VPT, THREADS>(p, balanced_row(p, r), threadIdx.x, nvec, red[parity]);
   }
 }
 
