@@ -242,33 +242,6 @@ def graph_launch_us(w: wl.Workload, launches: int = 256, replays: int = 20) -> f
     return start.elapsed_time(stop) * 1e3 / (launches * replays)
 
 
-def library_traffic_probes():
-    """Context for the write-heavy causal configuration: what plain library kernels reach on
-    this GPU for write-only traffic and for a copy (HBM writes alone run well below the
-    copy rate, so a 1-read : 2-write workload sits between the two)."""
-    import torch
-    n = 1 << 28                                         # 256 Mi bf16 = 512 MiB
-    src = torch.zeros(n // 2, dtype=torch.bfloat16, device="cuda")
-    dst = torch.empty(n, dtype=torch.bfloat16, device="cuda")
-
-    def timed(fn, reps=10):
-        for _ in range(3):
-            fn()
-        torch.cuda.synchronize()
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record()
-        for _ in range(reps):
-            fn()
-        b.record()
-        torch.cuda.synchronize()
-        return a.elapsed_time(b) * 1e-3 / reps
-
-    t_fill = timed(lambda: dst.fill_(1.0))
-    t_copy = timed(lambda: dst[: n // 2].copy_(src))
-    return {"write_only_fill_gbs": n * 2 / t_fill / 1e9, "copy_gbs": n * 2 / t_copy / 1e9,
-            "note": "torch fill_ (512 MiB written) and copy_ (256 MiB read + 256 MiB written), same run"}
-
-
 def oracle_baseline(w: wl.Workload, budget_s: float = 12.0):
     """Time the fp64 oracle, as it stands, on a bounded row sample of the workload."""
     import oracle
@@ -410,7 +383,6 @@ def run_ours(args):
             del dwk, wk
             torch.cuda.empty_cache()
         line["per_config"] = table
-        line["library_probes"] = library_traffic_probes()
     if rank == 0 and world == 1:
         line["cpu_baseline"] = oracle_baseline(w)
     assert binding.device_status() == 0, "a device-side bounded wait expired"
