@@ -29,6 +29,7 @@ std::atomic<int> g_tune_cluster_mode{0};  // 0 = planner's choice, 1 = row resid
 std::atomic<int> g_tune_tma_mode{0};      // 0 = planner's choice, 1 = ring-fed register kernel, 2 = shared-memory passes
 std::atomic<int> g_tune_interleave{0};    // 1 = visit causal rows short/long alternately (default: storage order)
 std::atomic<int> g_tune_pdl{0};           // 2 = launch without programmatic stream serialisation
+std::atomic<int> g_tune_reg_flex{0};      // 2 = never the runtime-thread-count normalisation kernel
 
 __device__ int g_status_word = 0;
 
@@ -157,6 +158,35 @@ bool plan_reg(const Call& c, LaunchPlan* plan) {
   plan->grid = static_cast<unsigned>(grid); plan->cluster = 1; plan->smem = 0;
   // a row of exactly group * vpt vectors takes the predicate-free normalisation kernel
   plan->stages = (static_cast<int64_t>(group) * vpt == nvec && g_tune_reg_general.load() == 0) ? 1 : 0;
+  // otherwise a normalisation row that splits exactly into (a multiple of 32 threads) x vpt
+  // vectors takes the runtime-thread-count variant of it (e.g. 5120, 6144, 7168 columns)
+  const bool norm = (c.op == OP_LAYERNORM || c.op == OP_RMSNORM);
+  // (also preferred over the 512- and 1024-thread exact fits: fatter threads measured faster)
+  if (norm && (plan->stages == 0 || threads >= 512 || g_tune_reg_flex.load() == 1) && group == threads &&
+      g_tune_reg_general.load() == 0 &&
+      !(t_threads > 0 && t_vpt > 0) && g_tune_reg_flex.load() != 2) {
+    const int max_vpt = (c.dtype == AKG_F32) ? 8 : 4;
+    int best_vpt = 0;
+    int64_t best_g = 0;
+    // fewer, fatter threads measured best (the per-row reduction is paid per thread): take
+    // the largest vectors-per-thread that leaves at least 128 threads, else whatever fits
+    for (int v = max_vpt; v >= 1 && best_vpt == 0; --v) {
+      if (nvec % v) continue;
+      const int64_t g = nvec / v;
+      if (g % 32 == 0 && g >= 128 && g <= 1024) { best_vpt = v; best_g = g; }
+    }
+    for (int v = max_vpt; v >= 1 && best_vpt == 0; --v) {
+      if (nvec % v) continue;
+      const int64_t g = nvec / v;
+      if (g % 32 == 0 && g >= 64 && g <= 1024) { best_vpt = v; best_g = g; }
+    }
+    if (best_vpt > 0) {
+      plan->mode = 2; plan->threads = static_cast<int>(best_g); plan->group = plan->threads; plan->vpt = best_vpt;
+      plan->grid = static_cast<unsigned>(c.rows > INT_MAX ? INT_MAX : c.rows);
+      if (g_tune_grid_cap.load() > 0 && plan->grid > static_cast<unsigned>(g_tune_grid_cap.load()))
+        plan->grid = static_cast<unsigned>(g_tune_grid_cap.load());
+    }
+  }
   return true;
 }
 
@@ -326,12 +356,13 @@ akg_status run(const Call& c, const char* name) {
   std::memset(&plan, 0, sizeof plan);
   bool planned = false;
   // Automatic choice (each rule is a measured preference on B200, see the profiles):
-  //   bf16 normalisation rows of exactly threads * vpt vectors, many rows -> ring-fed
-  //     register kernel (the load latency is hidden by the copy ring, not by occupancy)
+  //   bf16 RMSNorm rows of exactly threads * vpt vectors, many rows -> ring-fed register
+  //     kernel (the load latency is hidden by the copy ring, not by occupancy; bf16
+  //     LayerNorm, heavier per element, measured faster without the ring)
   //   every other row that fits a CTA's registers -> register kernel
   //   longer aligned rows -> two-pass split cluster kernel (second pass from L2)
   //   anything unaligned -> scalar stream kernel
-  if (forced == V_AUTO && vec && c.dtype == AKG_BF16 && (c.op == OP_LAYERNORM || c.op == OP_RMSNORM) &&
+  if (forced == V_AUTO && vec && c.dtype == AKG_BF16 && c.op == OP_RMSNORM &&
       c.rows >= 2048 && c.cols >= 2048 && g_tune_tma_mode.load() != 2) {
     planned = plan_ring(c, &plan);
     if (planned) {
@@ -374,7 +405,8 @@ akg_status run(const Call& c, const char* name) {
   const char* dt = (c.dtype == AKG_F32) ? "f32" : "bf16";
   if (plan.variant == V_REG)
     std::snprintf(t_kernel, sizeof t_kernel, "reg<%s,g%d,t%d,v%d%s>", dt, plan.group, plan.threads, plan.vpt,
-                  (plan.stages == 1 && (c.op == OP_LAYERNORM || c.op == OP_RMSNORM)) ? ",full" : "");
+                  plan.mode == 2 ? ",flex"
+                                 : ((plan.stages == 1 && (c.op == OP_LAYERNORM || c.op == OP_RMSNORM)) ? ",full" : ""));
   else if (plan.variant == V_TMA || plan.variant == V_CLUSTER)
     std::snprintf(t_kernel, sizeof t_kernel, "%s<%s,t%d,cs%d,nbuf%d,slice%d>",
                   plan.variant == V_TMA ? (plan.mode == 1 ? "ring" : "tma") : (plan.stages == 0 ? "split" : "cluster"),
@@ -594,6 +626,7 @@ akg_status akg_set_tuning(const char* key, int value) {
   else if (!std::strcmp(key, "tma_mode")) g_tune_tma_mode.store(value);
   else if (!std::strcmp(key, "interleave")) g_tune_interleave.store(value);
   else if (!std::strcmp(key, "pdl")) g_tune_pdl.store(value);
+  else if (!std::strcmp(key, "reg_flex")) g_tune_reg_flex.store(value);
   else return fail(AKG_ERR_INVALID_ARG, "akg_set_tuning: unknown key %s", key);
   return AKG_OK;
 }

@@ -142,6 +142,99 @@ __device__ __forceinline__ void norm_row_full(const RowParams& p, long long row,
   }
 }
 
+// reg_norm_flex: the same predicate-free scheme for rows of exactly blockDim.x * VPT
+// vectors where blockDim.x is any multiple of 32 (hidden sizes such as 5120, 6144, 7168).
+// A CTA per row.  Every warp holds the same number of values, so the warps' (mean, M2)
+// pairs combine without divisions:  mean = avg(mean_w),  M2 = sum(M2_w) + c * sum((mean_w - mean)^2)
+// with c = values per warp; every thread reads the NW pairs from shared memory.
+template <int OP, typename T, int VPT>
+__global__ void __launch_bounds__(1024, 1) reg_norm_flex(const RowParams p, const float inv_warps) {
+  pdl_prologue();
+  using E = Elem<T>;
+  constexpr int EPV = E::EPV;
+  constexpr int N = VPT * EPV;
+  static_assert(OP == OP_LAYERNORM || OP == OP_RMSNORM, "normalisations only");
+  __shared__ float red[2][2][32];
+  const int G = blockDim.x;
+  const int NW = G >> 5;
+  const int tg = threadIdx.x;
+  const float inv_cols = 1.0f / static_cast<float>(p.cols);
+  int parity = 0;
+  for (long long row = blockIdx.x; row < p.rows; row += gridDim.x, parity ^= 1) {
+    const T* xr = reinterpret_cast<const T*>(p.x) + row * p.xs + tg * EPV;
+    T* yr = reinterpret_cast<T*>(p.y) + row * p.ys + tg * EPV;
+    uint4 raw[VPT];
+#pragma unroll
+    for (int k = 0; k < VPT; ++k) raw[k] = ld_stream(xr + static_cast<long long>(k) * G * EPV);
+    float v[N];
+#pragma unroll
+    for (int k = 0; k < VPT; ++k) {
+      float f[EPV];
+      E::unpack(raw[k], f);
+#pragma unroll
+      for (int j = 0; j < EPV; ++j) v[k * EPV + j] = f[j];
+    }
+    float mean = 0.f, rstd;
+    if (OP == OP_RMSNORM) {
+      float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+      for (int i = 0; i < N; i += 2) { s0 = fmaf(v[i], v[i], s0); s1 = fmaf(v[i + 1], v[i + 1], s1); }
+      float ss = warp_sum(s0 + s1);
+      if ((threadIdx.x & 31) == 0) red[parity][0][threadIdx.x >> 5] = ss;
+      __syncthreads();
+      ss = 0.f;
+      for (int w = 0; w < NW; ++w) ss += red[parity][0][w];
+      rstd = rsqrt_refined(fmaf(ss, inv_cols, p.eps));
+    } else {
+      float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+      for (int i = 0; i < N; i += 2) { s0 += v[i]; s1 += v[i + 1]; }
+      float mu = (s0 + s1) * (1.0f / N);
+      float q0 = 0.f, q1 = 0.f;
+#pragma unroll
+      for (int i = 0; i < N; i += 2) {
+        const float d0 = v[i] - mu, d1 = v[i + 1] - mu;
+        q0 = fmaf(d0, d0, q0); q1 = fmaf(d1, d1, q1);
+      }
+      float m2 = q0 + q1;
+      float half_c = 0.5f * N;
+#pragma unroll
+      for (int m = 1; m <= 16; m <<= 1) {                 // equal-count merges inside the warp
+        const float mb = __shfl_xor_sync(0xffffffffu, mu, m);
+        const float qb = __shfl_xor_sync(0xffffffffu, m2, m);
+        const float d = mb - mu;
+        mu = fmaf(0.5f, d, mu);
+        m2 = fmaf(d * d, half_c, m2 + qb);
+        half_c *= 2.f;
+      }
+      if ((threadIdx.x & 31) == 0) { red[parity][0][threadIdx.x >> 5] = mu; red[parity][1][threadIdx.x >> 5] = m2; }
+      __syncthreads();
+      float msum = 0.f, qsum = 0.f;
+      for (int w = 0; w < NW; ++w) { msum += red[parity][0][w]; qsum += red[parity][1][w]; }
+      mean = msum * inv_warps;
+      float dev = 0.f;
+      for (int w = 0; w < NW; ++w) { const float d = red[parity][0][w] - mean; dev = fmaf(d, d, dev); }
+      rstd = rsqrt_refined(fmaf(fmaf(dev, 32.0f * N, qsum), inv_cols, p.eps));
+    }
+    const T* gp = reinterpret_cast<const T*>(p.gamma) + tg * EPV;
+    const T* bp = reinterpret_cast<const T*>(p.beta) + tg * EPV;
+#pragma unroll
+    for (int k = 0; k < VPT; ++k) {
+      float g[EPV], b[EPV], o[EPV];
+#pragma unroll
+      for (int j = 0; j < EPV; ++j) { g[j] = 1.f; b[j] = 0.f; }
+      if (p.gamma != nullptr) E::unpack(ld_cached(gp + static_cast<long long>(k) * G * EPV), g);
+      if (OP == OP_LAYERNORM && p.beta != nullptr) E::unpack(ld_cached(bp + static_cast<long long>(k) * G * EPV), b);
+#pragma unroll
+      for (int j = 0; j < EPV; ++j) {
+        if (OP == OP_LAYERNORM) o[j] = fmaf((v[k * EPV + j] - mean) * rstd, g[j], b[j]);
+        else o[j] = v[k * EPV + j] * rstd * g[j];
+      }
+      st_stream(yr + static_cast<long long>(k) * G * EPV, E::pack(o));
+    }
+  }
+}
+
 template <int OP, typename T, int G, int VPT, int THREADS>
 __global__ void __launch_bounds__(THREADS, kRegMinBlocks<THREADS>) reg_norm_full(const RowParams p) {
   pdl_prologue();

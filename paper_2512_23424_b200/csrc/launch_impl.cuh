@@ -212,6 +212,20 @@ cudaError_t launch_typed(const LaunchPlan& plan, const RowParams& p, cudaStream_
   if (plan.variant == V_STREAM) {
     return launch_plain(stream_kernel<OP, T, 256>, plan, plan.grid, 256, 0, s, p);
   }
+  if (plan.variant == V_REG && plan.mode == 2) {            // runtime thread count, exact fit
+    if constexpr (!OpTraits<OP>::kSoftmaxLike) {
+      const float inv_warps = 1.0f / static_cast<float>(plan.threads / 32);
+      switch (plan.vpt) {
+#define AKG_FLEX_CASE(V_) \
+  case V_: return launch_plain(reg_norm_flex<OP, T, V_>, plan, plan.grid, plan.threads, 0, s, p, inv_warps);
+        AKG_FLEX_CASE(1) AKG_FLEX_CASE(2) AKG_FLEX_CASE(3) AKG_FLEX_CASE(4)
+        AKG_FLEX_CASE(5) AKG_FLEX_CASE(6) AKG_FLEX_CASE(7) AKG_FLEX_CASE(8)
+#undef AKG_FLEX_CASE
+        default: break;
+      }
+    }
+    return cudaErrorInvalidConfiguration;
+  }
   if (plan.variant == V_REG) {
     // plan.stages == 1 marks a row of exactly group * vpt vectors (the predicate-free
     // normalisation kernel); the softmax pair always takes its own lean kernel.

@@ -112,7 +112,9 @@ def test_worked_examples_on_gpu(dtype):
 # ---- shape sweep: ragged sizes, strides, misaligned bases ---------------------------------------
 
 SWEEP_COLS = [1, 2, 3, 4, 5, 7, 8, 9, 31, 32, 33, 127, 128, 129, 1000, 1023, 1024, 1025, 4095, 4096,
-              4097, 8191, 8192, 32768 + 8]
+              4097, 8191, 8192, 32768 + 8,
+              # hidden sizes that are (a multiple of 32 threads) x (1..8 vectors), not a power of two
+              1536, 2560, 5120, 6144, 7168, 12288, 20480]
 SWEEP_ROWS = [1, 2, 3, 63, 65, 149]
 
 
