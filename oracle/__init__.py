@@ -188,6 +188,40 @@ def rmsnorm(x, weight=None, eps: float = 1e-6, nthreads: int = 1):
     return out
 
 
+AXIS_OPS = {"softmax": 0, "log_softmax": 1, "layernorm": 2, "rmsnorm": 3}
+
+
+def rowop_axis(op: str, x: np.ndarray, gamma=None, beta=None, eps: float = 1e-5, nthreads: int = 1):
+    """Operator `op` over axis 1 of a 3-D array [outer, reduce, inner] (inner contiguous):
+    the layout of the paper's RMSNorm sketch.  gamma / beta have `reduce` elements."""
+    if x.ndim != 3:
+        raise ValueError("oracle: x must be 3-D [outer, reduce, inner]")
+    if x.shape[2] > 1 and x.strides[2] != x.itemsize:
+        x = np.ascontiguousarray(x)
+    if any(s % x.itemsize for s in x.strides[:2]):
+        x = np.ascontiguousarray(x)
+    outer, reduce_n, inner = x.shape
+    so = x.strides[0] // x.itemsize if outer > 1 else reduce_n * max(x.strides[1] // x.itemsize, inner)
+    sf = x.strides[1] // x.itemsize if reduce_n > 1 else inner
+    if sf < inner or so < (reduce_n - 1) * sf + inner:
+        x = np.ascontiguousarray(x)
+        so, sf = reduce_n * inner, inner
+    out = np.empty((outer, reduce_n, inner), dtype=np.float64)
+    g, gp = _vec(gamma, x, reduce_n)
+    b, bp = _vec(beta, x, reduce_n)
+    L = lib()
+    if not L.oracle_rowop_axis.argtypes:
+        i64, vp, ci, cd = ctypes.c_int64, ctypes.c_void_p, ctypes.c_int, ctypes.c_double
+        L.oracle_rowop_axis.argtypes = [ci, vp, ci, i64, i64, i64, i64, i64, vp, vp, cd,
+                                        ctypes.POINTER(ctypes.c_double), ci]
+        L.oracle_rowop_axis.restype = ci
+    rc = L.oracle_rowop_axis(AXIS_OPS[op], x.ctypes.data, _dtype_code(x), outer, reduce_n, inner, so, sf,
+                             gp, bp, float(eps), _dptr(out), int(nthreads))
+    if rc != 0:
+        raise ValueError("oracle_rowop_axis: malformed argument")
+    return out
+
+
 def verifier_fraction(gen, ref, eps_switch: float = 1e-8, tau: float = 1e-3) -> float:
     """Fraction of elements whose error (Section 3.2.3, Eq. 2) exceeds tau."""
     g = np.ascontiguousarray(gen, dtype=np.float64).ravel()

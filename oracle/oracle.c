@@ -257,6 +257,50 @@ int oracle_rmsnorm(const void* x, int dtype, int64_t rows, int64_t cols,
   return failed;
 }
 
+/* ---- reduction over a non-last axis (layout of the Unified Sketch figure, Section 3.2.1) ---- */
+
+int oracle_rowop_axis(int op, const void* x, int dtype, int64_t outer, int64_t reduce, int64_t inner,
+                      int64_t outer_stride, int64_t reduce_stride, const void* gamma, const void* beta,
+                      double eps, double* out, int nthreads) {
+  if (op < 0 || op > 3) return 1;
+  if (outer < 0 || reduce < 0 || inner < 0) return 1;
+  if (dtype != ORACLE_F32 && dtype != ORACLE_BF16 && dtype != ORACLE_F64) return 1;
+  if ((op == 2 || op == 3) && !(eps >= 0.0)) return 1;
+  int t = use_threads(nthreads);
+  if (outer == 0 || reduce == 0 || inner == 0) return 0;
+  if (!x || !out) return 1;
+  if (reduce_stride < inner || outer_stride < (reduce - 1) * reduce_stride + inner) return 1;
+  double* g = (gamma && op >= 2) ? widen_vector(gamma, dtype, reduce) : NULL;
+  double* b = (beta && op == 2) ? widen_vector(beta, dtype, reduce) : NULL;
+  int failed = (gamma && op >= 2 && !g) || (beta && op == 2 && !b);
+  int64_t lines = outer * inner;                      /* one line per (b, d) */
+#pragma omp parallel num_threads(t)
+  {
+    double* z = (double*)malloc((size_t)reduce * sizeof(double));
+    double* y = (double*)malloc((size_t)reduce * sizeof(double));
+    if (!z || !y) {
+#pragma omp atomic write
+      failed = 1;
+    }
+#pragma omp for schedule(static)
+    for (int64_t l = 0; l < lines; ++l) {
+      if (!z || !y || failed) continue;
+      int64_t bb = l / inner, d = l % inner;
+      for (int64_t f = 0; f < reduce; ++f) z[f] = widen(x, dtype, bb * outer_stride + f * reduce_stride + d);
+      if (op == 0) oracle_softmax_row(z, reduce, y);
+      else if (op == 1) oracle_log_softmax_row(z, reduce, y);
+      else if (op == 2) oracle_layernorm_row(z, reduce, g, b, eps, y);
+      else oracle_rmsnorm_row(z, reduce, g, eps, y);
+      for (int64_t f = 0; f < reduce; ++f) out[(bb * reduce + f) * inner + d] = y[f];
+    }
+    free(z);
+    free(y);
+  }
+  free(g);
+  free(b);
+  return failed;
+}
+
 /* ---- the paper's verifier criterion (Section 3.2.3, Eq. 2-3) ------------------ */
 
 double oracle_verifier_fraction(const double* gen, const double* ref, int64_t n,

@@ -91,6 +91,19 @@ int oracle_rmsnorm(const void* x, int dtype, int64_t rows, int64_t cols,
                    int64_t x_stride, const void* weight, double eps,
                    double* out, int nthreads);
 
+/* ---- reduction over a NON-last axis -----------------------------------------
+ * The layout of the paper's RMSNorm sketch (Unified Sketch figure, Section 3.2.1):
+ * X[B, F, D1, D2] reduced over F.  Here x is [outer, reduce, inner] with inner
+ * (= D1 * D2) contiguous: element (b, f, d) sits at b*outer_stride + f*reduce_stride + d
+ * (strides in elements).  For every (b, d) the `reduce` values along f form one row of
+ * the operator op (0 softmax, 1 log-softmax, 2 LayerNorm, 3 RMSNorm; no masks);
+ * gamma / beta (LayerNorm) or gamma as the weight (RMSNorm) have `reduce` elements of x's
+ * storage type and are indexed by f; NULL means 1 / 0.
+ * out: outer x reduce x inner doubles, contiguous.  Returns 0, or 1 on a bad argument. */
+int oracle_rowop_axis(int op, const void* x, int dtype, int64_t outer, int64_t reduce, int64_t inner,
+                      int64_t outer_stride, int64_t reduce_stride, const void* gamma, const void* beta,
+                      double eps, double* out, int nthreads);
+
 /* The paper's correctness criterion (Section 3.2.3, Eq. 2-3): element error is
  * |gen-ref|/|ref| when |ref| > eps_switch, else |gen-ref|; returns the fraction
  * of elements whose error exceeds tau (the kernel passes iff that fraction is
