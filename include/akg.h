@@ -143,6 +143,27 @@ akg_status akg_rowop_host(akg_op op, const void* x_host, void* y_host, int64_t r
  * at least 4 MiB; 0 for a malformed shape. */
 size_t akg_host_workspace_bytes(int64_t rows, int64_t cols, akg_dtype dtype, int has_gamma, int has_beta);
 
+/* The same four operators over a NON-last axis: x and y are [outer, reduce, inner]
+ * DEVICE arrays with inner contiguous; element (b, f, d) is at
+ * b * outer_stride + f * reduce_stride + d (strides in elements,
+ * reduce_stride >= inner, outer_stride >= (reduce - 1) * reduce_stride + inner).
+ * This is the layout of the paper's RMSNorm sketch (Unified Sketch figure, Section
+ * 3.2.1: X[B, F, D1, D2] reduced over F, i.e. outer = B, reduce = F, inner = D1 * D2).
+ * For every (b, d) the `reduce` values along f are one row of the operator:
+ *   RMSNorm    y = x / sqrt(mean_f(x^2) + eps) * gamma[f]        (the sketch, gamma = NULL)
+ *   LayerNorm  y = (x - mean_f) / sqrt(var_f + eps) * gamma[f] + beta[f]
+ *   softmax / log-softmax over f (no masks on this entry point)
+ * gamma / beta: DEVICE vectors of `reduce` elements of x's dtype, indexed by f, or NULL
+ * (1 / 0); ignored by the softmax pair.  One kernel, two passes over the data, the second
+ * served by L2: HBM sees each element once in and once out.  16-byte aligned bases and
+ * strides with inner a multiple of the vector width take 128-bit accesses, anything else
+ * a scalar path with the same results.  In place (y == x, equal strides) is allowed.
+ * Enqueues on `stream` and returns; errors as for the last-axis entry points. */
+akg_status akg_rowop_axis(akg_op op, const void* x, void* y, int64_t outer, int64_t reduce, int64_t inner,
+                          int64_t x_outer_stride, int64_t x_reduce_stride, int64_t y_outer_stride,
+                          int64_t y_reduce_stride, akg_dtype dtype, const void* gamma, const void* beta,
+                          float eps, void* stream);
+
 /* Size of the staging area built into the library (see akg_rowop_host_static). */
 #define AKG_STATIC_STAGING_BYTES (16u << 20)
 

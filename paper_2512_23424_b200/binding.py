@@ -251,6 +251,41 @@ def rowop_host(op: str, x: torch.Tensor, out: torch.Tensor, workspace: torch.Ten
     return out
 
 
+def rowop_axis(op: str, x: torch.Tensor, out: Optional[torch.Tensor] = None, *,
+               gamma: Optional[torch.Tensor] = None, beta: Optional[torch.Tensor] = None,
+               eps: float = 1e-5, stream=None) -> torch.Tensor:
+    """akg_rowop_axis: `op` over axis 1 of a 3-D CUDA tensor [outer, reduce, inner] whose
+    last axis is contiguous (the layout of the paper's RMSNorm sketch).  gamma / beta are
+    device vectors of `reduce` elements."""
+    if x.dim() != 3 or not x.is_cuda:
+        raise ValueError("x must be a 3-D CUDA tensor [outer, reduce, inner]")
+    if out is None:
+        out = torch.empty_like(x)
+    if out.shape != x.shape or out.dtype != x.dtype or out.device != x.device:
+        raise ValueError("out must match x in shape, dtype and device")
+    outer, red, inner = x.shape
+    for t in (x, out):
+        if inner > 1 and t.stride(2) != 1:
+            raise ValueError("the last axis must be contiguous")
+
+    def strides(t):
+        sf = t.stride(1) if red > 1 else inner
+        so = t.stride(0) if outer > 1 else (red - 1) * sf + inner
+        return so, sf
+
+    (xso, xsf), (yso, ysf) = strides(x), strides(out)
+    fn = lib().akg_rowop_axis
+    if not fn.argtypes:
+        vp, i64, ci = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int
+        fn.argtypes = [ci, vp, vp, i64, i64, i64, i64, i64, i64, i64, ci, vp, vp, ctypes.c_float, vp]
+        fn.restype = ci
+    with torch.cuda.device(x.device):
+        st = fn(OPS[op], x.data_ptr(), out.data_ptr(), outer, red, inner, xso, xsf, yso, ysf, _dtype_code(x),
+                _vector(gamma, x, red, "gamma"), _vector(beta, x, red, "beta"), float(eps), _stream(stream))
+    _check(st, "akg_rowop_axis")
+    return out
+
+
 STATIC_STAGING_BYTES = 16 << 20
 
 

@@ -650,6 +650,71 @@ akg_status akg_device_status(int* word_out) {
 
 }  // extern "C"
 
+// ---- operators over a non-last axis ----------------------------------------------------------
+extern "C" akg_status akg_rowop_axis(akg_op op, const void* x, void* y, int64_t outer, int64_t reduce,
+                                     int64_t inner, int64_t x_outer_stride, int64_t x_reduce_stride,
+                                     int64_t y_outer_stride, int64_t y_reduce_stride, akg_dtype dtype,
+                                     const void* gamma, const void* beta, float eps, void* stream) {
+  const char* name = "akg_rowop_axis";
+  akg::t_error[0] = '\0';
+  if (op < AKG_OP_SOFTMAX || op > AKG_OP_RMSNORM) return akg::fail(AKG_ERR_INVALID_ARG, "%s: unknown operator", name);
+  if (dtype != AKG_F32 && dtype != AKG_BF16) return akg::fail(AKG_ERR_INVALID_ARG, "%s: unknown dtype", name);
+  if (outer < 0 || reduce < 0 || inner < 0) return akg::fail(AKG_ERR_INVALID_ARG, "%s: negative size", name);
+  const bool norm = (op == AKG_OP_LAYERNORM || op == AKG_OP_RMSNORM);
+  if (norm && (!(eps >= 0.f) || std::isinf(eps)))
+    return akg::fail(AKG_ERR_INVALID_ARG, "%s: eps must be finite and >= 0", name);
+  if (outer == 0 || reduce == 0 || inner == 0) return AKG_OK;
+  if (x == nullptr || y == nullptr) return akg::fail(AKG_ERR_INVALID_ARG, "%s: x and y must not be NULL", name);
+  if (x_reduce_stride < inner || y_reduce_stride < inner)
+    return akg::fail(AKG_ERR_INVALID_ARG, "%s: reduce stride smaller than inner", name);
+  const long double span_x = static_cast<long double>(reduce - 1) * x_reduce_stride + inner;
+  const long double span_y = static_cast<long double>(reduce - 1) * y_reduce_stride + inner;
+  if (x_outer_stride < span_x || y_outer_stride < span_y)
+    return akg::fail(AKG_ERR_INVALID_ARG, "%s: outer stride smaller than one [reduce, inner] slab", name);
+  const int64_t es = (dtype == AKG_F32) ? 4 : 2;
+  if (static_cast<long double>(outer) * x_outer_stride * es > 9.0e18L ||
+      static_cast<long double>(outer) * y_outer_stride * es > 9.0e18L)
+    return akg::fail(AKG_ERR_INVALID_ARG, "%s: outer * stride overflows", name);
+  if (reduce > INT_MAX / 2 || inner > (int64_t(1) << 40))
+    return akg::fail(AKG_ERR_UNSUPPORTED, "%s: reduce above 2^30 - 1 or inner above 2^40", name);
+  const uintptr_t x0 = reinterpret_cast<uintptr_t>(x), y0 = reinterpret_cast<uintptr_t>(y);
+  const uintptr_t x1 = x0 + static_cast<uintptr_t>(((outer - 1) * x_outer_stride + static_cast<int64_t>(span_x)) * es);
+  const uintptr_t y1 = y0 + static_cast<uintptr_t>(((outer - 1) * y_outer_stride + static_cast<int64_t>(span_y)) * es);
+  if (x0 < y1 && y0 < x1 && !(x0 == y0 && x_outer_stride == y_outer_stride && x_reduce_stride == y_reduce_stride))
+    return akg::fail(AKG_ERR_INVALID_ARG, "%s: x and y overlap without being the same array", name);
+
+  akg::AxisParams p;
+  p.x = x; p.y = y; p.outer = outer; p.reduce = reduce; p.inner = inner;
+  p.xso = x_outer_stride; p.xsf = x_reduce_stride; p.yso = y_outer_stride; p.ysf = y_reduce_stride;
+  p.gamma = norm ? gamma : nullptr;
+  p.beta = (op == AKG_OP_LAYERNORM) ? beta : nullptr;
+  p.eps = eps;
+  const int64_t epv = 16 / es;
+  const bool vec = (inner % epv == 0) && akg::aligned16(x) && akg::aligned16(y) &&
+                   (x_outer_stride * es) % 16 == 0 && (x_reduce_stride * es) % 16 == 0 &&
+                   (y_outer_stride * es) % 16 == 0 && (y_reduce_stride * es) % 16 == 0 &&
+                   akg::g_forced_variant.load() != akg::V_STREAM;
+  const int64_t w = vec ? epv : 1;
+  const int64_t strips_per_outer = (inner + 32 * w - 1) / (32 * w);
+  // strips in flight are re-read from L2 in the second pass: keep them within 64 MB
+  const long double strip_bytes = static_cast<long double>(reduce) * 32 * w * es;
+  int64_t cap = static_cast<int64_t>((64.0L * 1048576.0L) / strip_bytes);
+  const int64_t wave = static_cast<int64_t>(akg::sm_count()) * 8;
+  if (cap > wave) cap = wave;
+  if (cap < akg::sm_count()) cap = akg::sm_count();
+  const int tuned = akg::g_tune_grid_cap.load();
+  if (tuned > 0) cap = tuned;
+  long double strips = static_cast<long double>(outer) * strips_per_outer;
+  const unsigned grid = static_cast<unsigned>(strips < cap ? strips : cap);
+  const cudaError_t err = akg::launch_axis(static_cast<int>(op), static_cast<int>(dtype), vec, p, grid,
+                                          strips_per_outer, akg::g_tune_pdl.load() == 2 ? 0 : 1,
+                                          static_cast<cudaStream_t>(stream));
+  if (err != cudaSuccess) return akg::cuda_fail(name, err);
+  std::snprintf(akg::t_kernel, sizeof akg::t_kernel, "axis<%s,%s,t256,grid%u>", dtype == AKG_F32 ? "f32" : "bf16",
+                vec ? "vec" : "scalar", grid);
+  return AKG_OK;
+}
+
 // ---- host buffers without any allocation ---------------------------------------------------
 // akg_rowop_host needs a device staging area from its caller.  Some callers have no way to
 // get one: a plug-in that is handed host buffers and a stream but no allocator, a service

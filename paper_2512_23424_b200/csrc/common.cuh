@@ -32,6 +32,17 @@ struct RowParams {
   int* status;              // device status word (bounded waits report here)
 };
 
+// One call over a non-last axis: x[outer, reduce, inner], inner contiguous.
+struct AxisParams {
+  const void* x;
+  void* y;
+  long long outer, reduce, inner;
+  long long xso, xsf, yso, ysf;       // outer / reduce strides in elements (inner stride is 1)
+  const void* gamma;                  // [reduce] or nullptr (RMSNorm weight / LayerNorm gamma)
+  const void* beta;                   // [reduce] or nullptr
+  float eps;
+};
+
 // Shared-memory ring kernels: limits and the size of the bookkeeping area that
 // precedes the ring buffers (mbarriers, CTA reduction slots, cluster exchange slots).
 constexpr int kMaxCluster = 16;

@@ -27,6 +27,10 @@ struct LaunchPlan {
 template <int OP>
 cudaError_t launch_op(const LaunchPlan& plan, int dtype, const RowParams& p, cudaStream_t stream);
 
+// Non-last-axis kernel (op_axis.cu).  vec: 16-byte vectors along the inner axis are usable.
+cudaError_t launch_axis(int op, int dtype, bool vec, const AxisParams& p, unsigned grid,
+                        long long strips_per_outer, int pdl, cudaStream_t stream);
+
 extern template cudaError_t launch_op<OP_SOFTMAX>(const LaunchPlan&, int, const RowParams&, cudaStream_t);
 extern template cudaError_t launch_op<OP_LOG_SOFTMAX>(const LaunchPlan&, int, const RowParams&, cudaStream_t);
 extern template cudaError_t launch_op<OP_LAYERNORM>(const LaunchPlan&, int, const RowParams&, cudaStream_t);
