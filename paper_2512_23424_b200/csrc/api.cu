@@ -30,6 +30,8 @@ std::atomic<int> g_tune_tma_mode{0};      // 0 = planner's choice, 1 = ring-fed 
 std::atomic<int> g_tune_interleave{0};    // 1 = visit causal rows short/long alternately (default: storage order)
 std::atomic<int> g_tune_pdl{0};           // 2 = launch without programmatic stream serialisation
 std::atomic<int> g_tune_reg_flex{0};      // 2 = never the runtime-thread-count normalisation kernel
+std::atomic<int> g_tune_axis_r{0};        // non-last axis: rows per thread (2 / 4 / 8), -1 = two-pass kernel only
+std::atomic<int> g_tune_axis_nc{0};       //   column blocks per CTA
 
 __device__ int g_status_word = 0;
 
@@ -627,6 +629,8 @@ akg_status akg_set_tuning(const char* key, int value) {
   else if (!std::strcmp(key, "interleave")) g_tune_interleave.store(value);
   else if (!std::strcmp(key, "pdl")) g_tune_pdl.store(value);
   else if (!std::strcmp(key, "reg_flex")) g_tune_reg_flex.store(value);
+  else if (!std::strcmp(key, "axis_r")) g_tune_axis_r.store(value);
+  else if (!std::strcmp(key, "axis_nc")) g_tune_axis_nc.store(value);
   else return fail(AKG_ERR_INVALID_ARG, "akg_set_tuning: unknown key %s", key);
   return AKG_OK;
 }
@@ -695,6 +699,41 @@ extern "C" akg_status akg_rowop_axis(akg_op op, const void* x, void* y, int64_t 
                    (y_outer_stride * es) % 16 == 0 && (y_reduce_stride * es) % 16 == 0 &&
                    akg::g_forced_variant.load() != akg::V_STREAM;
   const int64_t w = vec ? epv : 1;
+  const int pdl = akg::g_tune_pdl.load() == 2 ? 0 : 1;
+  const int tuned = akg::g_tune_grid_cap.load();
+
+  // Register-resident kernel: nf warps x r rows cover the reduced axis (nf <= 16).  Of the
+  // three r, the one that wastes the fewest row slots wins, the larger r on a tie.
+  int r_best = 0, nf_best = 0;
+  const int t_r = akg::g_tune_axis_r.load();
+  for (int r = 8; r >= 2 && t_r >= 0; r >>= 1) {
+    if (t_r > 0 && r != t_r) continue;
+    const int64_t nf = (reduce + r - 1) / r;
+    if (nf > 16) continue;
+    if (r_best == 0 || nf * r < static_cast<int64_t>(nf_best) * r_best) { r_best = r; nf_best = static_cast<int>(nf); }
+  }
+  if (r_best > 0) {
+    const int64_t blocks = (inner + 32 * w - 1) / (32 * w);           // column blocks of one outer index
+    int64_t nc = std::max(1, 8 / nf_best);                            // about 256 threads
+    if (akg::g_tune_axis_nc.load() > 0) nc = std::min<int64_t>(akg::g_tune_axis_nc.load(), 16 / nf_best);
+    nc = std::max<int64_t>(1, std::min(nc, blocks));
+    const int64_t spo = (blocks + nc - 1) / nc;                       // <= 2^40 / 32 / 4 = 2^33
+    // one CTA per strip (more CTAs measured faster than a persistent grid); the loops in the
+    // kernel only run when a grid dimension is clipped
+    int64_t gx = std::min<int64_t>(spo, tuned > 0 ? tuned : (int64_t(1) << 30));
+    if (spo > UINT_MAX) return akg::fail(AKG_ERR_UNSUPPORTED, "%s: inner above 2^37 with a short reduced axis", name);
+    const int64_t gy = std::min<int64_t>(outer, 65535);
+    const dim3 grid(static_cast<unsigned>(gx), static_cast<unsigned>(gy));
+    const cudaError_t err = akg::launch_axis_reg(static_cast<int>(op), static_cast<int>(dtype), vec, r_best, p, grid,
+                                                 static_cast<unsigned>(spo), nf_best, static_cast<int>(nc), pdl,
+                                                 static_cast<cudaStream_t>(stream));
+    if (err != cudaSuccess) return akg::cuda_fail(name, err);
+    std::snprintf(akg::t_kernel, sizeof akg::t_kernel, "axis_reg<%s,%s,r%d,nf%d,nc%d,grid%ux%u>",
+                  dtype == AKG_F32 ? "f32" : "bf16", vec ? "vec" : "scalar", r_best, nf_best, static_cast<int>(nc),
+                  grid.x, grid.y);
+    return AKG_OK;
+  }
+
   const int64_t strips_per_outer = (inner + 32 * w - 1) / (32 * w);
   // strips in flight are re-read from L2 in the second pass: keep them within 64 MB
   const long double strip_bytes = static_cast<long double>(reduce) * 32 * w * es;
@@ -702,12 +741,11 @@ extern "C" akg_status akg_rowop_axis(akg_op op, const void* x, void* y, int64_t 
   const int64_t wave = static_cast<int64_t>(akg::sm_count()) * 8;
   if (cap > wave) cap = wave;
   if (cap < akg::sm_count()) cap = akg::sm_count();
-  const int tuned = akg::g_tune_grid_cap.load();
   if (tuned > 0) cap = tuned;
   long double strips = static_cast<long double>(outer) * strips_per_outer;
   const unsigned grid = static_cast<unsigned>(strips < cap ? strips : cap);
   const cudaError_t err = akg::launch_axis(static_cast<int>(op), static_cast<int>(dtype), vec, p, grid,
-                                          strips_per_outer, akg::g_tune_pdl.load() == 2 ? 0 : 1,
+                                          strips_per_outer, pdl,
                                           static_cast<cudaStream_t>(stream));
   if (err != cudaSuccess) return akg::cuda_fail(name, err);
   std::snprintf(akg::t_kernel, sizeof akg::t_kernel, "axis<%s,%s,t256,grid%u>", dtype == AKG_F32 ? "f32" : "bf16",

@@ -31,6 +31,13 @@ cudaError_t launch_op(const LaunchPlan& plan, int dtype, const RowParams& p, cud
 cudaError_t launch_axis(int op, int dtype, bool vec, const AxisParams& p, unsigned grid,
                         long long strips_per_outer, int pdl, cudaStream_t stream);
 
+// Register-resident non-last-axis kernel (op_axis_reg.cu): a CTA of nf x nc warps, nf
+// along the reduced axis with r rows per thread (reduce <= nf * r, r in {2, 4, 8}), nc
+// column blocks of 32 vectors (or 32 elements when !vec); strips_per_outer counts strips of
+// nc * 32 vectors; grid = (strips of one outer index, outer indices), either may be smaller.
+cudaError_t launch_axis_reg(int op, int dtype, bool vec, int r, const AxisParams& p, dim3 grid,
+                            unsigned strips_per_outer, int nf, int nc, int pdl, cudaStream_t stream);
+
 extern template cudaError_t launch_op<OP_SOFTMAX>(const LaunchPlan&, int, const RowParams&, cudaStream_t);
 extern template cudaError_t launch_op<OP_LOG_SOFTMAX>(const LaunchPlan&, int, const RowParams&, cudaStream_t);
 extern template cudaError_t launch_op<OP_LAYERNORM>(const LaunchPlan&, int, const RowParams&, cudaStream_t);
