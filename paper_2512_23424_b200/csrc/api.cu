@@ -32,6 +32,8 @@ std::atomic<int> g_tune_pdl{0};           // 2 = launch without programmatic str
 std::atomic<int> g_tune_reg_flex{0};      // 2 = never the runtime-thread-count normalisation kernel
 std::atomic<int> g_tune_axis_r{0};        // non-last axis: rows per thread (2 / 4 / 8), -1 = two-pass kernel only
 std::atomic<int> g_tune_axis_nc{0};       //   column blocks per CTA
+std::atomic<int> g_tune_axis_lc{0};       //   two-pass kernel: 1 + log2 of the lanes along the columns
+std::atomic<int> g_tune_axis_mode{0};     //   1 = 16-byte vectors, 2 = bf16 8-byte vectors widened, 3 = elements
 
 __device__ int g_status_word = 0;
 
@@ -631,6 +633,8 @@ akg_status akg_set_tuning(const char* key, int value) {
   else if (!std::strcmp(key, "reg_flex")) g_tune_reg_flex.store(value);
   else if (!std::strcmp(key, "axis_r")) g_tune_axis_r.store(value);
   else if (!std::strcmp(key, "axis_nc")) g_tune_axis_nc.store(value);
+  else if (!std::strcmp(key, "axis_mode")) g_tune_axis_mode.store(value);
+  else if (!std::strcmp(key, "axis_lc")) g_tune_axis_lc.store(value);
   else return fail(AKG_ERR_INVALID_ARG, "akg_set_tuning: unknown key %s", key);
   return AKG_OK;
 }
@@ -694,13 +698,28 @@ extern "C" akg_status akg_rowop_axis(akg_op op, const void* x, void* y, int64_t 
   p.beta = (op == AKG_OP_LAYERNORM) ? beta : nullptr;
   p.eps = eps;
   const int64_t epv = 16 / es;
-  const bool vec = (inner % epv == 0) && akg::aligned16(x) && akg::aligned16(y) &&
-                   (x_outer_stride * es) % 16 == 0 && (x_reduce_stride * es) % 16 == 0 &&
-                   (y_outer_stride * es) % 16 == 0 && (y_reduce_stride * es) % 16 == 0 &&
-                   akg::g_forced_variant.load() != akg::V_STREAM;
-  const int64_t w = vec ? epv : 1;
+  auto multiples_of = [&](int64_t bytes) {
+    return (inner * es) % bytes == 0 && reinterpret_cast<uintptr_t>(x) % bytes == 0 &&
+           reinterpret_cast<uintptr_t>(y) % bytes == 0 && (x_outer_stride * es) % bytes == 0 &&
+           (x_reduce_stride * es) % bytes == 0 && (y_outer_stride * es) % bytes == 0 &&
+           (y_reduce_stride * es) % bytes == 0;
+  };
+  const bool scalar_only = akg::g_forced_variant.load() == akg::V_STREAM;
+  const bool vec = !scalar_only && multiples_of(16);
   const int pdl = akg::g_tune_pdl.load() == 2 ? 0 : 1;
   const int tuned = akg::g_tune_grid_cap.load();
+
+  // What a lane holds of a row in the register-resident kernel.  bf16 in 16-byte vectors is
+  // unpacked at every use and softmax then needs a second exponential; 8-byte vectors widened
+  // to floats avoid both but move 256-byte row segments.  Measured on the sketch's shape:
+  // softmax is faster widened, the other three packed.
+  int mode = vec ? 1 : 0;
+  if (dtype == AKG_BF16 && !scalar_only && multiples_of(8) && (!vec || op == AKG_OP_SOFTMAX)) mode = 2;
+  const int t_mode = akg::g_tune_axis_mode.load();
+  if (t_mode == 3) mode = 0;
+  if (t_mode == 1 && vec) mode = 1;
+  if (t_mode == 2 && dtype == AKG_BF16 && !scalar_only && multiples_of(8)) mode = 2;
+  const int64_t w = akg::axis_reg_width(static_cast<int>(dtype), mode);
 
   // Register-resident kernel: nf warps x r rows cover the reduced axis (nf <= 16).  Of the
   // three r, the one that wastes the fewest row slots wins, the larger r on a tie.
@@ -724,32 +743,39 @@ extern "C" akg_status akg_rowop_axis(akg_op op, const void* x, void* y, int64_t 
     if (spo > UINT_MAX) return akg::fail(AKG_ERR_UNSUPPORTED, "%s: inner above 2^37 with a short reduced axis", name);
     const int64_t gy = std::min<int64_t>(outer, 65535);
     const dim3 grid(static_cast<unsigned>(gx), static_cast<unsigned>(gy));
-    const cudaError_t err = akg::launch_axis_reg(static_cast<int>(op), static_cast<int>(dtype), vec, r_best, p, grid,
+    const cudaError_t err = akg::launch_axis_reg(static_cast<int>(op), static_cast<int>(dtype), mode, r_best, p, grid,
                                                  static_cast<unsigned>(spo), nf_best, static_cast<int>(nc), pdl,
                                                  static_cast<cudaStream_t>(stream));
     if (err != cudaSuccess) return akg::cuda_fail(name, err);
     std::snprintf(akg::t_kernel, sizeof akg::t_kernel, "axis_reg<%s,%s,r%d,nf%d,nc%d,grid%ux%u>",
-                  dtype == AKG_F32 ? "f32" : "bf16", vec ? "vec" : "scalar", r_best, nf_best, static_cast<int>(nc),
-                  grid.x, grid.y);
+                  dtype == AKG_F32 ? "f32" : "bf16", mode == 1 ? "vec" : (mode == 2 ? "wide8" : "scalar"), r_best,
+                  nf_best, static_cast<int>(nc), grid.x, grid.y);
     return AKG_OK;
   }
 
-  const int64_t strips_per_outer = (inner + 32 * w - 1) / (32 * w);
-  // strips in flight are re-read from L2 in the second pass: keep them within 64 MB
-  const long double strip_bytes = static_cast<long double>(reduce) * 32 * w * es;
-  int64_t cap = static_cast<int64_t>((64.0L * 1048576.0L) / strip_bytes);
-  const int64_t wave = static_cast<int64_t>(akg::sm_count()) * 8;
-  if (cap > wave) cap = wave;
-  if (cap < akg::sm_count()) cap = akg::sm_count();
-  if (tuned > 0) cap = tuned;
-  long double strips = static_cast<long double>(outer) * strips_per_outer;
-  const unsigned grid = static_cast<unsigned>(strips < cap ? strips : cap);
+  // Two-pass kernel.  The strips in flight (4 CTAs per SM) are read again from L2 in the second
+  // pass: long reduced axes take narrower strips (fewer lanes of a warp along the columns, down
+  // to 128-byte row segments) to keep them within 64 MB.
+  const int64_t w2 = vec ? epv : 1;
+  const int64_t lane_bytes = w2 * es;
+  int lc_shift = 5;
+  const int min_shift = vec ? 3 : 5;
+  while (lc_shift > min_shift &&
+         static_cast<long double>(reduce) * (int64_t(1) << lc_shift) * lane_bytes * akg::sm_count() * 4 > 64.0L * 1048576.0L)
+    --lc_shift;
+  while (lc_shift > 0 && (int64_t(1) << (lc_shift - 1)) * w2 >= inner) --lc_shift;   // no more lanes than columns
+  const int t_lc = akg::g_tune_axis_lc.load();
+  if (t_lc > 0) lc_shift = std::min(5, t_lc - 1);
+  const int64_t cw = (int64_t(1) << lc_shift) * w2;
+  const int64_t spo = (inner + cw - 1) / cw;
+  if (spo > UINT_MAX) return akg::fail(AKG_ERR_UNSUPPORTED, "%s: inner above 2^32 strips", name);
+  const dim3 grid(static_cast<unsigned>(std::min<int64_t>(spo, tuned > 0 ? tuned : (int64_t(1) << 30))),
+                  static_cast<unsigned>(std::min<int64_t>(outer, 65535)));
   const cudaError_t err = akg::launch_axis(static_cast<int>(op), static_cast<int>(dtype), vec, p, grid,
-                                          strips_per_outer, pdl,
-                                          static_cast<cudaStream_t>(stream));
+                                          static_cast<unsigned>(spo), lc_shift, pdl, static_cast<cudaStream_t>(stream));
   if (err != cudaSuccess) return akg::cuda_fail(name, err);
-  std::snprintf(akg::t_kernel, sizeof akg::t_kernel, "axis<%s,%s,t256,grid%u>", dtype == AKG_F32 ? "f32" : "bf16",
-                vec ? "vec" : "scalar", grid);
+  std::snprintf(akg::t_kernel, sizeof akg::t_kernel, "axis<%s,%s,t256,lc%d,grid%ux%u>", dtype == AKG_F32 ? "f32" : "bf16",
+                vec ? "vec" : "scalar", 1 << lc_shift, grid.x, grid.y);
   return AKG_OK;
 }
 

@@ -16,16 +16,45 @@
 #pragma once
 
 #include "kernels_reg.cuh"
+#include "kernels_split.cuh"
 
 namespace akg {
 
-template <typename T, bool VEC> struct AxisRaw;
+// How a thread holds one row of its columns (MODE):
+//   0  one element, widened to float (any alignment)
+//   1  one 16-byte vector as loaded (4 floats / 8 packed bf16); bf16 is unpacked at each use
+//   2  bf16 only: one 8-byte vector widened to 4 floats at the load - the register picture of
+//      fp32 mode 1, so a bf16 value is unpacked once and softmax evaluates one exponential
+//      per element; rows are 256-byte segments per warp
+template <typename T, int MODE> struct AxisRaw;
 
-template <typename T> struct AxisRaw<T, true> {
+template <> struct AxisRaw<__nv_bfloat16, 2> {
+  using T = __nv_bfloat16;
+  using Raw = float4;
+  static constexpr int W = 4;
+  static constexpr bool kFloatRaw = true;
+  static __device__ __forceinline__ Raw load(const T* p) {
+    uint32_t a, b;
+    asm volatile("ld.global.L1::no_allocate.v2.u32 {%0, %1}, [%2];" : "=r"(a), "=r"(b) : "l"(p) : "memory");
+    return make_float4(__uint_as_float(a << 16), __uint_as_float(a & 0xffff0000u),
+                       __uint_as_float(b << 16), __uint_as_float(b & 0xffff0000u));
+  }
+  static __device__ __forceinline__ Raw fill(float v) { return make_float4(v, v, v, v); }
+  static __device__ __forceinline__ void unpack(const Raw& r, float (&f)[4]) { f[0] = r.x; f[1] = r.y; f[2] = r.z; f[3] = r.w; }
+  static __device__ __forceinline__ Raw pack(const float (&f)[4]) { return make_float4(f[0], f[1], f[2], f[3]); }
+  static __device__ __forceinline__ void store(T* p, const Raw& r) {
+    const uint32_t a = Elem<T>::pack2(r.x, r.y), b = Elem<T>::pack2(r.z, r.w);
+    asm volatile("st.global.cs.v2.u32 [%0], {%1, %2};" :: "l"(p), "r"(a), "r"(b) : "memory");
+  }
+};
+
+template <typename T> struct AxisRaw<T, 1> {
   using E = Elem<T>;
   using Raw = uint4;
   static constexpr int W = E::EPV;
+  static constexpr bool kFloatRaw = (sizeof(T) == 4);
   static __device__ __forceinline__ Raw load(const T* p) { return ld_stream(p); }
+  static __device__ __forceinline__ Raw load_hint(const T* p, uint64_t policy) { return ld_hint(p, policy); }
   static __device__ __forceinline__ Raw fill(float v) {
     float t[W];
 #pragma unroll
@@ -37,11 +66,13 @@ template <typename T> struct AxisRaw<T, true> {
   static __device__ __forceinline__ void store(T* p, const Raw& r) { st_stream(p, r); }
 };
 
-template <typename T> struct AxisRaw<T, false> {
+template <typename T> struct AxisRaw<T, 0> {
   using E = Elem<T>;
   using Raw = float;                        // a bf16 value widens exactly
   static constexpr int W = 1;
+  static constexpr bool kFloatRaw = true;
   static __device__ __forceinline__ Raw load(const T* p) { return E::load1(p, 0); }
+  static __device__ __forceinline__ Raw load_hint(const T* p, uint64_t) { return E::load1(p, 0); }
   static __device__ __forceinline__ Raw fill(float v) { return v; }
   static __device__ __forceinline__ void unpack(const Raw& r, float (&f)[1]) { f[0] = r; }
   static __device__ __forceinline__ Raw pack(const float (&f)[1]) { return f[0]; }
@@ -56,7 +87,8 @@ __host__ __device__ constexpr unsigned axis_reg_smem_floats(int ks, int nf, int 
 }
 
 // The two scalars of a column from its merged statistics:
-//   softmax     : p = M (0 for a column without live entry), q = 1 / S (0 for such a column)
+//   softmax     : p = C = round(M log2e) (0 for a column without live entry), q = 1 / S (0 for
+//                 such a column)
 //   log-softmax : p = M, q = ln S (both 0 for such a column: x - 0 - 0 = -inf)
 //   LayerNorm   : p = mean, q = 1 / sqrt(M2 / F + eps)
 //   RMSNorm     : q = 1 / sqrt(sum of squares / F + eps)
@@ -75,18 +107,61 @@ __device__ __forceinline__ void axis_scalars(float a, float b, float inv_f, floa
   }
 }
 
+// Merge the nf partials of one column (q0[i * CW], q1[i * CW]: partial i) and derive the
+// column's two scalars.  Warp-row i holds nbase + (i < nrem) rows of the reduced axis.
+template <int OP, int CW>
+__device__ __forceinline__ void axis_merge_column(const float* q0, const float* q1, int nf, int nbase, int nrem,
+                                                  float inv_f, float eps, float& sp, float& sq) {
+  float a = 0.f, bb = 0.f;
+  if (OpTraits<OP>::kSoftmaxLike) {
+    a = kNegInf;
+#pragma unroll 4
+    for (int i = 0; i < nf; ++i) a = fmaxf(a, q0[i * CW]);
+    const float ms = (a == kNegInf) ? 0.f : a;
+#pragma unroll 4
+    for (int i = 0; i < nf; ++i)
+      bb = fmaf(q1[i * CW], OP == OP_SOFTMAX ? ex2_approx(q0[i * CW] - ms) : exp_diff(q0[i * CW], ms), bb);
+  } else if (OP == OP_LAYERNORM) {
+    if (nrem == 0) {                       // equal counts: mean of means, M2 = sum M2_i + n sum d_i^2
+#pragma unroll 4
+      for (int i = 0; i < nf; ++i) a += q0[i * CW];
+      const float nb = static_cast<float>(nbase);
+      a *= nb * inv_f;
+      float dd = 0.f;
+#pragma unroll 4
+      for (int i = 0; i < nf; ++i) {
+        const float d = q0[i * CW] - a;
+        bb += q1[i * CW];
+        dd = fmaf(d, d, dd);
+      }
+      bb = fmaf(nb, dd, bb);
+    } else {
+      for (int i = 0; i < nf; ++i) a = fmaf(static_cast<float>(nbase + (i < nrem ? 1 : 0)), q0[i * CW], a);
+      a *= inv_f;
+      for (int i = 0; i < nf; ++i) {
+        const float d = q0[i * CW] - a;
+        bb += fmaf(static_cast<float>(nbase + (i < nrem ? 1 : 0)) * d, d, q1[i * CW]);
+      }
+    }
+  } else {
+#pragma unroll 4
+    for (int i = 0; i < nf; ++i) a += q0[i * CW];
+  }
+  axis_scalars<OP>(a, bb, inv_f, eps, sp, sq);
+}
+
 // Phase 1 of a strip: load this thread's rows and fold them into per-column partials
 // ((m, s), (mean, M2) or the sum of squares).  FULL: all R rows exist and the columns are
 // inside the array, so nothing is predicated (the case of every thread but those of a
 // ragged last warp-row or column block).
-template <int OP, typename T, bool VEC, int R, bool FULL>
+template <int OP, typename T, int MODE, int R, bool FULL>
 __device__ __forceinline__ void axis_reg_load(const T* px, long long xstep, bool active, int nt,
-                                              typename AxisRaw<T, VEC>::Raw (&raw)[R],
-                                              float (&sa)[AxisRaw<T, VEC>::W], float (&sb)[AxisRaw<T, VEC>::W]) {
-  using A = AxisRaw<T, VEC>;
+                                              typename AxisRaw<T, MODE>::Raw (&raw)[R],
+                                              float (&sa)[AxisRaw<T, MODE>::W], float (&sb)[AxisRaw<T, MODE>::W]) {
+  using A = AxisRaw<T, MODE>;
   constexpr int W = A::W;
   constexpr bool SM = OpTraits<OP>::kSoftmaxLike;
-  constexpr bool KEEP = (OP == OP_SOFTMAX) && (sizeof(T) == 4);
+  constexpr bool KEEP = (OP == OP_SOFTMAX) && A::kFloatRaw;
 #pragma unroll
   for (int r = 0; r < R; ++r, px += xstep) {
     if (FULL) raw[r] = A::load(px);
@@ -102,15 +177,27 @@ __device__ __forceinline__ void axis_reg_load(const T* px, long long xstep, bool
 #pragma unroll
       for (int j = 0; j < W; ++j) sa[j] = fmaxf(sa[j], v[j]);
     }
+    // softmax works in the base-2 domain: its partial maximum is c = round(m log2e), and every
+    // exponential is exp2(x log2e - c) in one multiply-add.  Partials are later rescaled by
+    // exp2(c - C) with the same rounded numbers, so the rounding of m log2e cancels exactly
+    // between numerator and denominator.  log-softmax keeps (x - m) exact instead.
     float ms[W];
 #pragma unroll
-    for (int j = 0; j < W; ++j) { ms[j] = (sa[j] == kNegInf) ? 0.f : sa[j]; sb[j] = 0.f; }
+    for (int j = 0; j < W; ++j) {
+      if (OP == OP_SOFTMAX) sa[j] *= kLog2e;
+      ms[j] = (sa[j] == kNegInf) ? 0.f : sa[j];
+      if (OP == OP_SOFTMAX) ms[j] = -ms[j];
+      sb[j] = 0.f;
+    }
 #pragma unroll
     for (int r = 0; r < R; ++r) {
       float v[W];
       A::unpack(raw[r], v);
 #pragma unroll
-      for (int j = 0; j < W; ++j) { v[j] = exp_diff(v[j], ms[j]); sb[j] += v[j]; }
+      for (int j = 0; j < W; ++j) {
+        v[j] = (OP == OP_SOFTMAX) ? ex2_approx(fmaf(v[j], kLog2e, ms[j])) : exp_diff(v[j], ms[j]);
+        sb[j] += v[j];
+      }
       if (KEEP) raw[r] = A::pack(v);
     }
   } else if (OP == OP_LAYERNORM) {
@@ -150,16 +237,19 @@ __device__ __forceinline__ void axis_reg_load(const T* px, long long xstep, bool
 
 // Phase 3 of a strip: normalise the rows held in registers with the columns' scalars
 // (cp, cq) and store them.  gp / bp point at gamma[wf] / beta[wf] (or are nullptr).
-template <int OP, typename T, bool VEC, int R, bool FULL>
+template <int OP, typename T, int MODE, int R, bool FULL>
 __device__ __forceinline__ void axis_reg_store(T* py, long long ystep, bool active, int nt, int nf,
                                                const T* gp, const T* bp,
-                                               const typename AxisRaw<T, VEC>::Raw (&raw)[R],
-                                               const float (&cp)[AxisRaw<T, VEC>::W],
-                                               const float (&cq)[AxisRaw<T, VEC>::W]) {
-  using A = AxisRaw<T, VEC>;
+                                               const typename AxisRaw<T, MODE>::Raw (&raw)[R],
+                                               const float (&cp)[AxisRaw<T, MODE>::W],
+                                               const float (&cq)[AxisRaw<T, MODE>::W]) {
+  using A = AxisRaw<T, MODE>;
   using E = Elem<T>;
   constexpr int W = A::W;
-  constexpr bool KEEP = (OP == OP_SOFTMAX) && (sizeof(T) == 4);
+  constexpr bool KEEP = (OP == OP_SOFTMAX) && A::kFloatRaw;
+  float ncp[W];                              // softmax from packed values: exp2(x log2e - C) / S
+#pragma unroll
+  for (int j = 0; j < W; ++j) ncp[j] = -cp[j];
 #pragma unroll
   for (int r = 0; r < R; ++r, py += ystep) {
     if (FULL || (active && r < nt)) {
@@ -172,7 +262,7 @@ __device__ __forceinline__ void axis_reg_store(T* py, long long ystep, bool acti
       A::unpack(raw[r], v);
 #pragma unroll
       for (int j = 0; j < W; ++j) {
-        if (OP == OP_SOFTMAX) v[j] = (KEEP ? v[j] : exp_diff(v[j], cp[j])) * cq[j];
+        if (OP == OP_SOFTMAX) v[j] = (KEEP ? v[j] : ex2_approx(fmaf(v[j], kLog2e, ncp[j]))) * cq[j];
         else if (OP == OP_LOG_SOFTMAX) v[j] = (v[j] - cp[j]) - cq[j];
         else if (OP == OP_LAYERNORM) v[j] = (v[j] - cp[j]) * cq[j] * g + be;
         else v[j] = v[j] * cq[j] * g;
@@ -183,12 +273,12 @@ __device__ __forceinline__ void axis_reg_store(T* py, long long ystep, bool acti
 }
 
 // nbase, nrem: reduce / nf and reduce % nf (warp-row i holds nbase + (i < nrem) rows).
-template <int OP, typename T, bool VEC, int R>
+template <int OP, typename T, int MODE, int R>
 __global__ void __launch_bounds__(32 * kAxisMaxWarps, 2)
 axis_reg_kernel(const AxisParams p, const unsigned strips_per_outer, const int nf, const int nc,
                 const int nbase, const int nrem) {
   pdl_prologue();
-  using A = AxisRaw<T, VEC>;
+  using A = AxisRaw<T, MODE>;
   using Raw = typename A::Raw;
   constexpr int W = A::W;
   constexpr int CW = 32 * W;                 // columns of one column block
@@ -196,7 +286,7 @@ axis_reg_kernel(const AxisParams p, const unsigned strips_per_outer, const int n
   constexpr int KS = (OP == OP_RMSNORM) ? 1 : 2;
   // fp32 softmax keeps exp(x - m_local) in the registers the values came in; bf16 cannot
   // (a second rounding), it evaluates the exponential again for the output
-  constexpr bool KEEP = (OP == OP_SOFTMAX) && (sizeof(T) == 4);
+  constexpr bool KEEP = (OP == OP_SOFTMAX) && A::kFloatRaw;
   extern __shared__ __align__(16) float axis_smem[];
 
   const int lane = threadIdx.x & 31;
@@ -224,8 +314,8 @@ axis_reg_kernel(const AxisParams p, const unsigned strips_per_outer, const int n
 
       Raw raw[R];
       float sa[W], sb[W];
-      if (full) axis_reg_load<OP, T, VEC, R, true>(xb, xstep, active, nt, raw, sa, sb);
-      else axis_reg_load<OP, T, VEC, R, false>(xb, xstep, active, nt, raw, sa, sb);
+      if (full) axis_reg_load<OP, T, MODE, R, true>(xb, xstep, active, nt, raw, sa, sb);
+      else axis_reg_load<OP, T, MODE, R, false>(xb, xstep, active, nt, raw, sa, sb);
 
       // ---- the two scalars of every column
       float cp[W], cq[W];
@@ -236,27 +326,10 @@ axis_reg_kernel(const AxisParams p, const unsigned strips_per_outer, const int n
           if (KS == 2) part1[warp * CW + lane * W + j] = sb[j];
         }
         __syncthreads();
-        const float* q0 = part0 + wc * nf * CW;
-        const float* q1 = part1 + wc * nf * CW;
         for (int c = wf * 32 + lane; c < CW; c += 32 * nf) {
-          float a = 0.f, bb = 0.f;
-          if (SM) {
-            a = kNegInf;
-            for (int i = 0; i < nf; ++i) a = fmaxf(a, q0[i * CW + c]);
-            const float ms = (a == kNegInf) ? 0.f : a;
-            for (int i = 0; i < nf; ++i) bb = fmaf(q1[i * CW + c], exp_diff(q0[i * CW + c], ms), bb);
-          } else if (OP == OP_LAYERNORM) {
-            for (int i = 0; i < nf; ++i) a = fmaf(static_cast<float>(nbase + (i < nrem ? 1 : 0)), q0[i * CW + c], a);
-            a *= inv_f;
-            for (int i = 0; i < nf; ++i) {
-              const float d = q0[i * CW + c] - a;
-              bb += fmaf(static_cast<float>(nbase + (i < nrem ? 1 : 0)) * d, d, q1[i * CW + c]);
-            }
-          } else {
-            for (int i = 0; i < nf; ++i) a += q0[i * CW + c];
-          }
           float sp, sq;
-          axis_scalars<OP>(a, bb, inv_f, p.eps, sp, sq);
+          axis_merge_column<OP, CW>(part0 + wc * nf * CW + c, part1 + wc * nf * CW + c, nf, nbase, nrem, inv_f, p.eps,
+                                    sp, sq);
           fin0[wc * CW + c] = sp;
           fin1[wc * CW + c] = sq;
         }
@@ -269,11 +342,11 @@ axis_reg_kernel(const AxisParams p, const unsigned strips_per_outer, const int n
       }
       if (KEEP) {
 #pragma unroll
-        for (int j = 0; j < W; ++j) cq[j] *= exp_diff(sa[j], cp[j]);     // exp(m_local - M) / S
+        for (int j = 0; j < W; ++j) cq[j] *= ex2_approx(sa[j] - cp[j]);  // exp2(c_local - C) / S
       }
 
-      if (full) axis_reg_store<OP, T, VEC, R, true>(yb, ystep, active, nt, nf, gp, bp, raw, cp, cq);
-      else axis_reg_store<OP, T, VEC, R, false>(yb, ystep, active, nt, nf, gp, bp, raw, cp, cq);
+      if (full) axis_reg_store<OP, T, MODE, R, true>(yb, ystep, active, nt, nf, gp, bp, raw, cp, cq);
+      else axis_reg_store<OP, T, MODE, R, false>(yb, ystep, active, nt, nf, gp, bp, raw, cp, cq);
     }
   }
 }

@@ -27,15 +27,20 @@ struct LaunchPlan {
 template <int OP>
 cudaError_t launch_op(const LaunchPlan& plan, int dtype, const RowParams& p, cudaStream_t stream);
 
-// Non-last-axis kernel (op_axis.cu).  vec: 16-byte vectors along the inner axis are usable.
-cudaError_t launch_axis(int op, int dtype, bool vec, const AxisParams& p, unsigned grid,
-                        long long strips_per_outer, int pdl, cudaStream_t stream);
+// Two-pass non-last-axis kernel (op_axis.cu), 256 threads.  vec: 16-byte vectors along the
+// inner axis are usable.  A warp lies 1 << lc_shift lanes along the columns and the rest along
+// rows; strips_per_outer counts strips of (1 << lc_shift) lanes; grid as for launch_axis_reg.
+cudaError_t launch_axis(int op, int dtype, bool vec, const AxisParams& p, dim3 grid, unsigned strips_per_outer,
+                        int lc_shift, int pdl, cudaStream_t stream);
 
 // Register-resident non-last-axis kernel (op_axis_reg.cu): a CTA of nf x nc warps, nf
 // along the reduced axis with r rows per thread (reduce <= nf * r, r in {2, 4, 8}), nc
-// column blocks of 32 vectors (or 32 elements when !vec); strips_per_outer counts strips of
-// nc * 32 vectors; grid = (strips of one outer index, outer indices), either may be smaller.
-cudaError_t launch_axis_reg(int op, int dtype, bool vec, int r, const AxisParams& p, dim3 grid,
+// column blocks of 32 lanes.  mode: what a lane holds of a row - 0 one element, 1 one 16-byte
+// vector, 2 (bf16) one 8-byte vector widened to floats; axis_reg_width gives its elements.
+// strips_per_outer counts strips of nc * 32 lanes; grid = (strips of one outer index, outer
+// indices), either may be smaller.
+int axis_reg_width(int dtype, int mode);
+cudaError_t launch_axis_reg(int op, int dtype, int mode, int r, const AxisParams& p, dim3 grid,
                             unsigned strips_per_outer, int nf, int nc, int pdl, cudaStream_t stream);
 
 extern template cudaError_t launch_op<OP_SOFTMAX>(const LaunchPlan&, int, const RowParams&, cudaStream_t);

@@ -85,6 +85,37 @@ def test_axis_strides_in_place_and_padding(op, dtype):
     check(op, dtype, x, g, None, got, eps, "axis misaligned base")
 
 
+@pytest.mark.parametrize("op", OPS)
+@pytest.mark.parametrize("dtype", [wl.F32, wl.BF16])
+def test_axis_every_kernel_shape(op, dtype):
+    """Each lane layout (16-byte vectors, widened 8-byte bf16 vectors, elements), each rows-per-
+    thread count, several column blocks per CTA, and the two-pass kernel, on ragged shapes."""
+    eps = 1e-5
+    shapes = [(2, 64, 512), (3, 37, 264), (2, 5, 1032), (1, 128, 96), (2, 19, 4100)]
+    settings = [dict(axis_mode=m, axis_r=r, axis_nc=nc)
+                for m in (1, 2, 3) for r, nc in ((8, 0), (4, 2), (2, 3), (0, 1))] + [dict(axis_r=-1)]
+    try:
+        for i, (outer, red, inner) in enumerate(shapes):
+            x, g, b = make(op, dtype, outer, red, inner, seed=90 + i)
+            xd = to_torch(x.reshape(outer * red, inner), dtype).view(outer, red, inner)
+            seen = set()
+            for st in settings:
+                for k in ("axis_mode", "axis_r", "axis_nc"):
+                    akg.set_tuning(k, st.get(k, 0))
+                out = binding.rowop_axis(op, xd, gamma=to_torch(g, dtype), beta=to_torch(b, dtype), eps=eps)
+                torch.cuda.synchronize()
+                name = akg.last_kernel()
+                if name in seen:
+                    continue
+                seen.add(name)
+                got = to_numpy(out.view(outer * red, inner)).reshape(outer, red, inner)
+                check(op, dtype, x, g, b, got, eps, f"axis {op} {outer}x{red}x{inner} [{name}]")
+            assert len(seen) >= 2
+    finally:
+        for k in ("axis_mode", "axis_r", "axis_nc"):
+            akg.set_tuning(k, 0)
+
+
 def test_axis_sketch_workload_and_special_columns():
     # the sketch's shape class: X[B, F, D1, D2] fp32, reduced over F
     B, F, D1, D2 = 4, 96, 16, 64
@@ -102,6 +133,23 @@ def test_axis_sketch_workload_and_special_columns():
         check(op, wl.F32, xs, None, None, got, 0.0, f"axis special {op}")
         if op == "softmax":
             assert (got[0, :, 1].view(np.uint32) == 0).all()
+
+
+@pytest.mark.parametrize("dtype", [wl.F32, wl.BF16])
+def test_axis_softmax_large_magnitudes(dtype):
+    """Logits of magnitude 1e3..1e4: the rounding of max * log2(e) must not reach the output."""
+    rng = np.random.default_rng(11)
+    for scale, shape in ((3.0e3, (2, 64, 512)), (2.0e4, (1, 24, 264)), (5.0e2, (2, 7, 40))):
+        x = (rng.normal(0.0, 1.0, size=shape) * scale + rng.normal(0.0, 2.0, size=shape)).astype(np.float32)
+        x[0, : shape[1] // 2, 3] = x[0, 0, 3]                      # ties at the maximum
+        if dtype == wl.BF16:
+            x = wl.f32_to_bf16_bits(x)
+        # (log-softmax is left out: its outputs are of the inputs' magnitude, where fp32 values
+        # are spaced 1e-3 apart and no kernel can meet an absolute 1e-5)
+        out = binding.rowop_axis("softmax", to_torch(x.reshape(-1, shape[2]), dtype).view(*shape))
+        torch.cuda.synchronize()
+        got = to_numpy(out.view(-1, shape[2])).reshape(shape)
+        check("softmax", dtype, x, None, None, got, 0.0, f"axis softmax scale {scale} [{akg.last_kernel()}]")
 
 
 def test_axis_argument_errors():
