@@ -7,8 +7,9 @@ A step is one launch of the headline operator (LayerNorm fp32 [4096, 4096], the
 second benchmark configuration) through the C ABI on inputs already resident in
 HBM; successive steps rotate over four buffer pairs so the working set (512 MiB)
 exceeds L2.  The one JSON line printed by rank 0 carries the headline number,
-the same figure for every configuration (`per_config`), the roofline fraction,
-the end-to-end figure with host buffers, and the fp64 CPU oracle's timing.
+the same figure for every configuration (`per_config`) and for the operators
+over a non-last axis (`axis_rows`), the roofline fraction, the end-to-end figure
+with host buffers, and the fp64 CPU oracle's timing.
 
 With N > 1 (launched by torch.distributed.run) every rank runs the same
 per-GPU workload on its own seed: rows are independent, there is no collective
@@ -153,8 +154,36 @@ class DeviceWorkload:
         return call.launch()
 
 
-def pairs_for(w: wl.Workload) -> int:
-    one = 2 * w.rows * w.cols * w.itemsize
+class AxisDeviceWorkload:
+    """A non-last-axis workload x[outer, reduce, inner] resident in HBM, rotating buffer pairs."""
+
+    def __init__(self, w: wl.AxisWorkload, pairs: int):
+        import torch
+        from paper_2512_23424_b200 import binding
+        self.w, self.binding, self.torch = w, binding, torch
+
+        def dev(a):
+            if a is None:
+                return None
+            if w.dtype == wl.F32:
+                return torch.from_numpy(a).cuda()
+            return torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
+
+        x0 = dev(w.x)
+        self.xs = [x0] + [x0.clone() for _ in range(pairs - 1)]
+        self.ys = [torch.empty_like(x0) for _ in range(pairs)]
+        self.gamma, self.beta = dev(w.gamma), dev(w.beta)
+        self.i = 0
+
+    def launch(self):
+        k = self.i % len(self.xs)
+        self.i += 1
+        return self.binding.rowop_axis(self.w.op, self.xs[k], out=self.ys[k], gamma=self.gamma, beta=self.beta,
+                                       eps=self.w.eps)
+
+
+def pairs_for(w) -> int:
+    one = w.algorithmic_bytes() if isinstance(w, wl.AxisWorkload) else 2 * w.rows * w.cols * w.itemsize
     if one >= 3 * L2_BYTES:
         return 1
     return max(2, int(np.ceil(4 * L2_BYTES / one)))
@@ -266,7 +295,7 @@ def oracle_baseline(w: wl.Workload, budget_s: float = 12.0):
     rows = int(min(w.rows, max(probe_rows, probe_rows * budget_s / max(t_probe, 1e-4))))
     # the sample is repeated until about budget_s of CPU time has been spent
     passes, secs, nbytes = 0, 0.0, 0
-    while passes == 0 or (secs < budget_s and passes < 200):
+    while passes == 0 or (secs < budget_s and passes < 5000):
         t, b = run(rows)
         secs, nbytes, passes = secs + t, nbytes + b, passes + 1
     return {"value": nbytes / secs / 1e9, "unit": "GB/s", "cores": oracle.last_threads(),
@@ -383,6 +412,20 @@ def run_ours(args):
             del dwk, wk
             torch.cuda.empty_cache()
         line["per_config"] = table
+        # the operators over a non-last axis (the layout of the paper's RMSNorm sketch)
+        axis = []
+        for name in wl.AXIS_CONFIGS:
+            wa = wl.make_axis(name)
+            dwa = AxisDeviceWorkload(wa, pairs_for(wa))
+            reps = max(10, min(100, 100 * args.steps // 1000))
+            sa = time_launches(dwa, reps, 5) / reps
+            ba = wa.algorithmic_bytes()
+            axis.append({"workload": name, "kernel": binding.last_kernel(), "us": sa * 1e6, "gbs": ba / sa / 1e9,
+                         "frac_measured": ba / sa / 1e9 / peak, "algorithmic_bytes": ba, "launches": reps,
+                         "traffic": profiled_traffic(name)})
+            del dwa, wa
+            torch.cuda.empty_cache()
+        line["axis_rows"] = axis
     if rank == 0 and world == 1:
         line["cpu_baseline"] = oracle_baseline(w)
     assert binding.device_status() == 0, "a device-side bounded wait expired"
@@ -437,6 +480,17 @@ def run_profile(args):
     import torch
     from paper_2512_23424_b200 import binding
     torch.cuda.set_device(0)
+    if args.profile_axis:
+        w = wl.make_axis(args.profile_axis, outer=args.profile_rows)
+        for item in filter(None, args.tune.split(",")):
+            key, _, val = item.partition("=")
+            binding.set_tuning(key, int(val))
+        dw = AxisDeviceWorkload(w, pairs_for(w) if args.profile_rows is None else 1)
+        secs = time_launches(dw, args.steps, args.warmup)
+        print(json.dumps({"profile": args.profile_axis, "shape": list(w.x.shape), "kernel": binding.last_kernel(),
+                          "us_per_launch": secs / args.steps * 1e6, "launches": args.steps + max(args.warmup, 3),
+                          "algorithmic_bytes": w.algorithmic_bytes()}))
+        return
     w = wl.make_config(args.profile, rows=args.profile_rows)
     if args.variant:
         binding.set_variant(args.variant)
@@ -460,11 +514,14 @@ def main():
                     help="skip the per-configuration table (the headline line is unchanged)")
     ap.add_argument("--profile", type=int, default=0, metavar="K",
                     help="only launch configuration K (1..5) warmup+steps times, for use under ncu")
-    ap.add_argument("--profile-rows", type=int, default=None, help="truncate the rows of --profile")
+    ap.add_argument("--profile-axis", default="", metavar="NAME",
+                    help="as --profile, for a non-last-axis configuration (workloads.AXIS_CONFIGS)")
+    ap.add_argument("--profile-rows", type=int, default=None,
+                    help="truncate the rows of --profile (the outer axis of --profile-axis)")
     ap.add_argument("--variant", default="", help="force a kernel family in --profile mode")
     ap.add_argument("--tune", default="", help="--profile mode: key=value[,key=value] launch-geometry overrides")
     args = ap.parse_args()
-    if args.profile:
+    if args.profile or args.profile_axis:
         run_profile(args)
     elif args.impl == "reference":
         run_reference(args)

@@ -166,3 +166,60 @@ def make_random(op: str, dtype: int, rows: int, cols: int, seed: int,
     return Workload(f"{op}_{'f32' if dtype == F32 else 'bf16'}_{rows}x{cols}", op, dtype,
                     rows, cols, x, eps=eps if op in ("layernorm", "rmsnorm") else 0.0,
                     gamma=gamma, beta=beta)
+
+
+# ---------------------------------------------------------------------------------------------
+# Operators over a non-last axis: x[outer, reduce, inner], inner contiguous.  The first shape is
+# the one of the paper's RMSNorm sketch (Unified Sketch figure: X[B, F, D1, D2] normalised over
+# the feature axis F) with B = 16, F = 64, D1 = D2 = 256; the long-axis shapes exercise the
+# two-pass kernel.
+# ---------------------------------------------------------------------------------------------
+AXIS_CONFIGS: Dict[str, tuple] = {
+    "axis_sketch_rmsnorm_f32_16x64x65536": ("rmsnorm", F32, 16, 64, 65536),
+    "axis_softmax_f32_16x64x65536": ("softmax", F32, 16, 64, 65536),
+    "axis_layernorm_f32_16x64x65536": ("layernorm", F32, 16, 64, 65536),
+    "axis_sketch_rmsnorm_bf16_16x64x65536": ("rmsnorm", BF16, 16, 64, 65536),
+    "axis_softmax_bf16_16x64x65536": ("softmax", BF16, 16, 64, 65536),
+    "axis_layernorm_bf16_16x64x65536": ("layernorm", BF16, 16, 64, 65536),
+    "axis_rmsnorm_f32_8x512x16384": ("rmsnorm", F32, 8, 512, 16384),
+    "axis_softmax_f32_2x1024x32768": ("softmax", F32, 2, 1024, 32768),
+}
+
+
+@dataclass
+class AxisWorkload:
+    name: str
+    op: str
+    dtype: int                         # F32 / BF16
+    x: np.ndarray                      # [outer, reduce, inner]; float32, or uint16 bf16 bits
+    eps: float = 0.0
+    gamma: Optional[np.ndarray] = None  # [reduce]
+    beta: Optional[np.ndarray] = None
+
+    @property
+    def itemsize(self) -> int:
+        return 4 if self.dtype == F32 else 2
+
+    def algorithmic_bytes(self) -> int:
+        """One read and one write of every element (gamma / beta are negligible)."""
+        return 2 * self.x.size * self.itemsize
+
+
+def make_axis(name: str, outer: Optional[int] = None, seed_offset: int = 0) -> AxisWorkload:
+    """Seeded input of a non-last-axis configuration; `outer` truncates the outer axis."""
+    op, dtype, o, f, d = AXIS_CONFIGS[name]
+    o = o if outer is None else min(o, outer)
+    seed = 100 + sorted(AXIS_CONFIGS).index(name) + 1000 * seed_offset
+    s_x, s_g, s_b = np.random.SeedSequence(seed).spawn(3)
+    rx, rg, rb = (np.random.Generator(np.random.PCG64(s)) for s in (s_x, s_g, s_b))
+    x = (_normal_f32(rx, o * f, d) * np.float32(1.5) + np.float32(0.25)).reshape(o, f, d)
+    gamma = beta = None
+    if op in ("layernorm", "rmsnorm"):
+        gamma = rg.uniform(0.5, 1.5, f).astype(np.float32)
+        if op == "layernorm":
+            beta = (rb.standard_normal(f) * 0.1).astype(np.float32)
+    if dtype == BF16:
+        x = f32_to_bf16_bits(x)
+        gamma = None if gamma is None else f32_to_bf16_bits(gamma)
+        beta = None if beta is None else f32_to_bf16_bits(beta)
+    return AxisWorkload(name, op, dtype, x, eps=1e-5 if gamma is not None else 0.0, gamma=gamma, beta=beta)
