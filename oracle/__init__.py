@@ -188,6 +188,30 @@ def rmsnorm(x, weight=None, eps: float = 1e-6, nthreads: int = 1):
     return out
 
 
+def add_norm(op: str, x, res, gamma=None, beta=None, eps: float = 1e-5, nthreads: int = 1):
+    """Fused residual add + LayerNorm / RMSNorm (a fused variant of Section 3.6):
+    returns (norm(x + res), x + res), both float64 [rows, cols]."""
+    x, rows, cols, xs = _as2d(x)
+    res, rrows, rcols, rs = _as2d(res)
+    if (rrows, rcols) != (rows, cols) or res.dtype != x.dtype:
+        raise ValueError("oracle: res must match x's shape and dtype")
+    out_y = np.empty((rows, cols), dtype=np.float64)
+    out_s = np.empty((rows, cols), dtype=np.float64)
+    g, gp = _vec(gamma, x, cols)
+    b, bp = _vec(beta, x, cols)
+    L = lib()
+    if not L.oracle_add_norm.argtypes:
+        i64, vp, ci, cd = ctypes.c_int64, ctypes.c_void_p, ctypes.c_int, ctypes.c_double
+        dp = ctypes.POINTER(ctypes.c_double)
+        L.oracle_add_norm.argtypes = [ci, vp, vp, ci, i64, i64, i64, i64, vp, vp, cd, dp, dp, ci]
+        L.oracle_add_norm.restype = ci
+    rc = L.oracle_add_norm({"layernorm": 2, "rmsnorm": 3}[op], x.ctypes.data, res.ctypes.data, _dtype_code(x),
+                           rows, cols, xs, rs, gp, bp, float(eps), _dptr(out_y), _dptr(out_s), int(nthreads))
+    if rc != 0:
+        raise ValueError("oracle_add_norm: malformed argument")
+    return out_y, out_s
+
+
 AXIS_OPS = {"softmax": 0, "log_softmax": 1, "layernorm": 2, "rmsnorm": 3}
 
 

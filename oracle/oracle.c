@@ -301,6 +301,34 @@ int oracle_rowop_axis(int op, const void* x, int dtype, int64_t outer, int64_t r
   return failed;
 }
 
+/* ---- fused residual add + normalisation (a "fused variant" of Section 3.6) ----------- */
+
+int oracle_add_norm(int op, const void* x, const void* res, int dtype, int64_t rows, int64_t cols,
+                    int64_t x_stride, int64_t res_stride, const void* gamma, const void* beta,
+                    double eps, double* out_y, double* out_sum, int nthreads) {
+  if (op != 2 && op != 3) return 1;
+  if (bad_shape(x, dtype, rows, cols, x_stride, out_y)) return 1;
+  if (rows > 0 && cols > 0 && (!res || !out_sum || res_stride < cols)) return 1;
+  if (!(eps >= 0.0)) return 1;
+  int t = use_threads(nthreads);
+  if (rows == 0 || cols == 0) return 0;
+  double* g = gamma ? widen_vector(gamma, dtype, cols) : NULL;
+  double* b = (beta && op == 2) ? widen_vector(beta, dtype, cols) : NULL;
+  int failed = (gamma && !g) || (beta && op == 2 && !b);
+#pragma omp parallel for schedule(static) num_threads(t)
+  for (int64_t i = 0; i < rows; ++i) {
+    if (failed) continue;
+    double* s = out_sum + i * cols;
+    /* the sum of two widened values is exact in double for fp32 / bf16 storage */
+    for (int64_t c = 0; c < cols; ++c) s[c] = widen(x, dtype, i * x_stride + c) + widen(res, dtype, i * res_stride + c);
+    if (op == 2) oracle_layernorm_row(s, cols, g, b, eps, out_y + i * cols);
+    else oracle_rmsnorm_row(s, cols, g, eps, out_y + i * cols);
+  }
+  free(g);
+  free(b);
+  return failed;
+}
+
 /* ---- the paper's verifier criterion (Section 3.2.3, Eq. 2-3) ------------------ */
 
 double oracle_verifier_fraction(const double* gen, const double* ref, int64_t n,

@@ -104,6 +104,17 @@ int oracle_rowop_axis(int op, const void* x, int dtype, int64_t outer, int64_t r
                       int64_t outer_stride, int64_t reduce_stride, const void* gamma, const void* beta,
                       double eps, double* out, int nthreads);
 
+/* Fused residual add + normalisation, one of the "fused variants" the paper's operator
+ * benchmark lists (Section 3.6): s = x + res element by element, out_sum = s, and
+ * out_y = LayerNorm(s) (op 2) or RMSNorm(s) (op 3) over the last axis, with the
+ * definitions of oracle_layernorm / oracle_rmsnorm (gamma doubles as the RMSNorm weight;
+ * beta is ignored by RMSNorm).  x and res share dtype and shape [rows, cols] with their own
+ * row strides; the normalisation sees the unrounded sum.  out_y, out_sum: rows x cols
+ * doubles, contiguous.  Returns 0, or 1 on a bad argument. */
+int oracle_add_norm(int op, const void* x, const void* res, int dtype, int64_t rows, int64_t cols,
+                    int64_t x_stride, int64_t res_stride, const void* gamma, const void* beta,
+                    double eps, double* out_y, double* out_sum, int nthreads);
+
 /* The paper's correctness criterion (Section 3.2.3, Eq. 2-3): element error is
  * |gen-ref|/|ref| when |ref| > eps_switch, else |gen-ref|; returns the fraction
  * of elements whose error exceeds tau (the kernel passes iff that fraction is
