@@ -154,15 +154,38 @@ size_t akg_host_workspace_bytes(int64_t rows, int64_t cols, akg_dtype dtype, int
  *   LayerNorm  y = (x - mean_f) / sqrt(var_f + eps) * gamma[f] + beta[f]
  *   softmax / log-softmax over f (no masks on this entry point)
  * gamma / beta: DEVICE vectors of `reduce` elements of x's dtype, indexed by f, or NULL
- * (1 / 0); ignored by the softmax pair.  One kernel, two passes over the data, the second
- * served by L2: HBM sees each element once in and once out.  16-byte aligned bases and
- * strides with inner a multiple of the vector width take 128-bit accesses, anything else
- * a scalar path with the same results.  In place (y == x, equal strides) is allowed.
+ * (1 / 0); ignored by the softmax pair.  One kernel: a reduced axis of up to 128 entries is
+ * held in registers, a longer one takes two passes, the second served by L2; either way HBM
+ * sees each element once in and once out.  16-byte aligned bases and strides with inner a
+ * multiple of the vector width take 128-bit accesses, anything else a scalar path with the
+ * same results.  In place (y == x, equal strides) is allowed.
  * Enqueues on `stream` and returns; errors as for the last-axis entry points. */
 akg_status akg_rowop_axis(akg_op op, const void* x, void* y, int64_t outer, int64_t reduce, int64_t inner,
                           int64_t x_outer_stride, int64_t x_reduce_stride, int64_t y_outer_stride,
                           int64_t y_reduce_stride, akg_dtype dtype, const void* gamma, const void* beta,
                           float eps, void* stream);
+
+/* Fused residual add + normalisation over the last axis (one of the "fused variants" of the
+ * paper's operator benchmark, Section 3.6; the paper gives no formula, this is the usual
+ * pre-norm residual step):
+ *   s = x + residual;   sum_out = s;   y = LayerNorm(s) or RMSNorm(s)
+ * op is AKG_OP_LAYERNORM or AKG_OP_RMSNORM, with the definitions, gamma / beta (beta ignored
+ * by RMSNorm) and eps of akg_layernorm / akg_rmsnorm.  x, residual, y, sum_out: DEVICE
+ * matrices [rows, cols] of `dtype`, each with its own row stride in elements (>= cols).
+ * The sum is formed in fp32 from the widened operands; the normalisation sees that fp32
+ * sum, sum_out receives it rounded once to `dtype`.  sum_out may be NULL (the sum is then
+ * not stored).  Aliasing: y and sum_out may each be exactly x or exactly residual (same base
+ * and stride - e.g. sum_out == residual updates the residual stream in place, y == x
+ * overwrites the branch input) or disjoint from them; y and sum_out must not overlap each
+ * other; x and residual may overlap freely.  Rows of a whole number of 16-byte vectors per
+ * thread (cols a multiple of 128 fp32 / 256 bf16 elements, up to 32768 / 65536, everything
+ * 16-byte aligned) move every byte once; other shapes take a scalar two-pass kernel with
+ * the same results.  Enqueues on `stream` and returns; errors as for akg_layernorm, plus
+ * AKG_ERR_INVALID_ARG for a NULL residual or a forbidden overlap. */
+akg_status akg_add_norm(akg_op op, const void* x, const void* residual, void* y, void* sum_out,
+                        int64_t rows, int64_t cols, int64_t x_row_stride, int64_t res_row_stride,
+                        int64_t y_row_stride, int64_t sum_row_stride, akg_dtype dtype,
+                        const void* gamma, const void* beta, float eps, void* stream);
 
 /* Size of the staging area built into the library (see akg_rowop_host_static). */
 #define AKG_STATIC_STAGING_BYTES (16u << 20)

@@ -286,6 +286,46 @@ def rowop_axis(op: str, x: torch.Tensor, out: Optional[torch.Tensor] = None, *,
     return out
 
 
+_NO_SUM = object()
+
+
+def add_norm(op: str, x: torch.Tensor, residual: torch.Tensor, *, gamma: Optional[torch.Tensor] = None,
+             beta: Optional[torch.Tensor] = None, eps: float = 1e-5, out: Optional[torch.Tensor] = None,
+             sum_out=_NO_SUM, stream=None):
+    """akg_add_norm: s = x + residual, returns (LayerNorm or RMSNorm of s, s) for 2-D CUDA tensors.
+    `out` / `sum_out` default to new tensors; pass sum_out=None to skip storing the sum (the second
+    result is then None); either may be `x` or `residual` themselves (in place)."""
+    if op not in ("layernorm", "rmsnorm"):
+        raise ValueError("op must be 'layernorm' or 'rmsnorm'")
+    rows, cols, xs = _matrix(x, "x")
+    rrows, rcols, rs = _matrix(residual, "residual")
+    if out is None:
+        out = torch.empty_like(x)
+    if sum_out is _NO_SUM:
+        sum_out = torch.empty_like(x)
+    orow, ocol, ys = _matrix(out, "out")
+    others = [(residual, rrows, rcols, "residual"), (out, orow, ocol, "out")]
+    ss = cols
+    if sum_out is not None:
+        srow, scol, ss = _matrix(sum_out, "sum_out")
+        others.append((sum_out, srow, scol, "sum_out"))
+    for t, r, c, what in others:
+        if (r, c) != (rows, cols) or t.dtype != x.dtype or t.device != x.device:
+            raise ValueError(f"{what} must match x in shape, dtype and device")
+    fn = lib().akg_add_norm
+    if not fn.argtypes:
+        vp, i64, ci = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int
+        fn.argtypes = [ci, vp, vp, vp, vp, i64, i64, i64, i64, i64, i64, ci, vp, vp, ctypes.c_float, vp]
+        fn.restype = ci
+    with torch.cuda.device(x.device):
+        st = fn(OPS[op], x.data_ptr(), residual.data_ptr(), out.data_ptr(),
+                None if sum_out is None else sum_out.data_ptr(), rows, cols, xs, rs, ys, ss, _dtype_code(x),
+                _vector(gamma, x, cols, "gamma"), _vector(beta, x, cols, "beta") if op == "layernorm" else None,
+                float(eps), _stream(stream))
+    _check(st, "akg_add_norm")
+    return out, sum_out
+
+
 STATIC_STAGING_BYTES = 16 << 20
 
 

@@ -779,6 +779,97 @@ extern "C" akg_status akg_rowop_axis(akg_op op, const void* x, void* y, int64_t 
   return AKG_OK;
 }
 
+// ---- fused residual add + LayerNorm / RMSNorm ----------------------------------------------
+extern "C" akg_status akg_add_norm(akg_op op, const void* x, const void* residual, void* y, void* sum_out,
+                                   int64_t rows, int64_t cols, int64_t x_row_stride, int64_t res_row_stride,
+                                   int64_t y_row_stride, int64_t sum_row_stride, akg_dtype dtype,
+                                   const void* gamma, const void* beta, float eps, void* stream) {
+  using namespace akg;
+  const char* name = "akg_add_norm";
+  t_error[0] = '\0';
+  if (op != AKG_OP_LAYERNORM && op != AKG_OP_RMSNORM)
+    return fail(AKG_ERR_INVALID_ARG, "%s: the operator must be LayerNorm or RMSNorm", name);
+  Call c;
+  c.op = static_cast<int>(op); c.x = x; c.y = y; c.rows = rows; c.cols = cols; c.xs = x_row_stride; c.ys = y_row_stride;
+  c.dtype = static_cast<int>(dtype); c.mask = nullptr; c.gamma = gamma;
+  c.beta = (op == AKG_OP_LAYERNORM) ? beta : nullptr; c.eps = eps; c.stream = stream;
+  const akg_status st = validate(c, name);
+  if (st != AKG_OK) return st;
+  if (rows == 0 || cols == 0) return AKG_OK;
+  if (residual == nullptr) return fail(AKG_ERR_INVALID_ARG, "%s: residual must not be NULL", name);
+  if (res_row_stride < cols || (sum_out != nullptr && sum_row_stride < cols))
+    return fail(AKG_ERR_INVALID_ARG, "%s: row stride smaller than cols", name);
+  const int64_t es = (dtype == AKG_F32) ? 4 : 2;
+  if (static_cast<long double>(rows) * res_row_stride * es > 9.0e18L ||
+      static_cast<long double>(rows) * sum_row_stride * es > 9.0e18L)
+    return fail(AKG_ERR_INVALID_ARG, "%s: rows * stride overflows", name);
+  // An output may be one of the inputs exactly (same base and stride: every element is read
+  // before it is written, by the same thread) or disjoint from it; the two outputs are disjoint.
+  struct Span { uintptr_t lo, hi; int64_t stride; };
+  auto span = [&](const void* ptr, int64_t stride) {
+    const uintptr_t lo = reinterpret_cast<uintptr_t>(ptr);
+    return Span{lo, lo + static_cast<uintptr_t>(((rows - 1) * stride + cols) * es), stride};
+  };
+  auto clash = [&](const Span& out, const Span& in) {
+    return out.lo < in.hi && in.lo < out.hi && !(out.lo == in.lo && (rows == 1 || out.stride == in.stride));
+  };
+  const Span sx = span(x, x_row_stride), sr = span(residual, res_row_stride), sy = span(y, y_row_stride);
+  if (clash(sy, sr)) return fail(AKG_ERR_INVALID_ARG, "%s: y overlaps residual without being the same matrix", name);
+  if (sum_out != nullptr) {
+    const Span ss = span(sum_out, sum_row_stride);
+    if (clash(ss, sx) || clash(ss, sr))
+      return fail(AKG_ERR_INVALID_ARG, "%s: sum_out overlaps an input without being the same matrix", name);
+    if (ss.lo < sy.hi && sy.lo < ss.hi) return fail(AKG_ERR_INVALID_ARG, "%s: sum_out overlaps y", name);
+  }
+
+  RowParams p;
+  std::memset(&p, 0, sizeof p);
+  p.x = x; p.y = y; p.rows = rows; p.cols = cols; p.xs = x_row_stride; p.ys = y_row_stride;
+  p.gamma = gamma; p.beta = c.beta; p.eps = eps; p.period = 1; p.add_rows = 1;
+  p.res = residual; p.rs = res_row_stride; p.sum = sum_out; p.ss = sum_row_stride;
+  const int pdl = g_tune_pdl.load() == 2 ? 0 : 1;
+  const int cap = g_tune_grid_cap.load();
+  unsigned grid = static_cast<unsigned>(rows > INT_MAX ? INT_MAX : rows);
+  if (cap > 0 && grid > static_cast<unsigned>(cap)) grid = static_cast<unsigned>(cap);
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+
+  const int64_t epv = 16 / es;
+  bool vec = vector_ok(c) && g_forced_variant.load() != V_STREAM && aligned16(residual) &&
+             (rows == 1 || (res_row_stride * es) % 16 == 0);
+  if (sum_out != nullptr) vec = vec && aligned16(sum_out) && (rows == 1 || (sum_row_stride * es) % 16 == 0);
+  int vpt = 0;
+  int64_t threads = 0;
+  if (vec) {
+    // a CTA per row, the row in registers: 2 * vpt loads in flight per thread, so four vectors
+    // per thread are preferred; at least 128 threads where the row allows
+    const int64_t nvec = cols / epv;
+    const int order[8] = {4, 3, 2, 1, 8, 7, 6, 5};
+    const int t_vpt = g_tune_reg_vpt.load();
+    for (int lo : {128, 32}) {
+      for (int v : order) {
+        if (vpt || (t_vpt > 0 && v != t_vpt) || nvec % v) continue;
+        const int64_t g = nvec / v;
+        if (g % 32 == 0 && g >= lo && g <= 1024) { vpt = v; threads = g; }
+      }
+    }
+  }
+  cudaError_t err;
+  if (vpt > 0) {
+    err = launch_add_norm(static_cast<int>(op), static_cast<int>(dtype), vpt, static_cast<int>(threads), p, grid, pdl, cs);
+    std::snprintf(t_kernel, sizeof t_kernel, "add_flex<%s,t%d,v%d>", dtype == AKG_F32 ? "f32" : "bf16",
+                  static_cast<int>(threads), vpt);
+  } else {
+    LaunchPlan plan;
+    std::memset(&plan, 0, sizeof plan);
+    plan_stream(c, &plan);
+    plan.pdl = pdl;
+    err = (op == AKG_OP_LAYERNORM) ? launch_op<OP_LAYERNORM>(plan, c.dtype, p, cs) : launch_op<OP_RMSNORM>(plan, c.dtype, p, cs);
+    std::snprintf(t_kernel, sizeof t_kernel, "add_stream<%s,t%d>", dtype == AKG_F32 ? "f32" : "bf16", plan.threads);
+  }
+  if (err != cudaSuccess) return cuda_fail(name, err);
+  return AKG_OK;
+}
+
 // ---- host buffers without any allocation ---------------------------------------------------
 // akg_rowop_host needs a device staging area from its caller.  Some callers have no way to
 // get one: a plug-in that is handed host buffers and a stream but no allocator, a service

@@ -30,6 +30,12 @@ struct RowParams {
   int interleave;           // 1: visit the rows of a causal period short/long alternately
   long long row_base;       // global index of row 0 (mask rules use row + row_base); 0 unless chunked
   int* status;              // device status word (bounded waits report here)
+  // fused residual add (normalisations only): the operator runs on x + res; the sum is also
+  // stored to `sum` unless that is nullptr.  res == nullptr: plain operator.
+  const void* res;
+  long long rs;             // row stride of res
+  void* sum;
+  long long ss;             // row stride of sum
 };
 
 // One call over a non-last axis: x[outer, reduce, inner], inner contiguous.

@@ -151,6 +151,8 @@ __global__ void __launch_bounds__(THREADS) reg_kernel(const RowParams p) {
 // stream_kernel: one CTA per row at a time, scalar accesses at any alignment.
 // Pass 1 keeps running statistics per thread (online max / rescaled sum, Welford, or
 // a sum of squares); pass 2 re-reads the row (served by L2 for all but huge rows).
+// With a residual (normalisations), both passes form x + res; the sum is stored in pass 2
+// only, element by element after its operands were read, so it may alias x or res.
 // ------------------------------------------------------------------------------------
 template <int OP, typename T, int THREADS>
 __global__ void __launch_bounds__(THREADS) stream_kernel(const RowParams p) {
@@ -168,10 +170,13 @@ __global__ void __launch_bounds__(THREADS) stream_kernel(const RowParams p) {
     const T* ar = (SM && p.add != nullptr)
                       ? reinterpret_cast<const T*>(p.add) + add_row(p, row) * p.add_stride
                       : nullptr;
+    const T* rr = (!SM && p.res != nullptr) ? reinterpret_cast<const T*>(p.res) + row * p.rs : nullptr;
+    T* sr = (!SM && p.res != nullptr && p.sum != nullptr) ? reinterpret_cast<T*>(p.sum) + row * p.ss : nullptr;
 
     Stat st = stat_identity<OP>();
     for (long long c = threadIdx.x; c < live; c += THREADS) {
       float z = E::load1(xr, c);
+      if (!SM && rr != nullptr) z += E::load1(rr, c);
       if (SM) {
         if (ar != nullptr) z += E::load1(ar, c);
         const float mn = fmaxf(st.a, z);
@@ -200,6 +205,10 @@ __global__ void __launch_bounds__(THREADS) stream_kernel(const RowParams p) {
           // exp(z - M) / S; a dead row (no live entry) has q = 0 and p = 0
           o = exp_diff(z, rs.p) * rs.q;
         } else {
+          if (!SM && rr != nullptr) {
+            z += E::load1(rr, c);
+            if (sr != nullptr) E::store1(sr, c, z);
+          }
           const float g = (!SM && p.gamma != nullptr) ? E::load1(p.gamma, c) : 1.f;
           const float b = (OP == OP_LAYERNORM && p.beta != nullptr) ? E::load1(p.beta, c) : 0.f;
           o = apply_one<OP>(z, rs, 0.f, g, b);

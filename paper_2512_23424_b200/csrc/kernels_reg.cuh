@@ -142,6 +142,55 @@ __device__ __forceinline__ void norm_row_full(const RowParams& p, long long row,
   }
 }
 
+// Row statistics of the flex scheme: every thread of the CTA holds N values of the row; NW
+// warps.  red: [2][32] floats of shared memory reserved for this row.  One barrier.
+template <int OP, int N>
+__device__ __forceinline__ void flex_row_stats(const float (&v)[N], float (*red)[32], int NW, float inv_warps,
+                                               float inv_cols, float eps, float& mean, float& rstd) {
+  mean = 0.f;
+  if (OP == OP_RMSNORM) {
+    float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+    for (int i = 0; i < N; i += 2) { s0 = fmaf(v[i], v[i], s0); s1 = fmaf(v[i + 1], v[i + 1], s1); }
+    float ss = warp_sum(s0 + s1);
+    if ((threadIdx.x & 31) == 0) red[0][threadIdx.x >> 5] = ss;
+    __syncthreads();
+    ss = 0.f;
+    for (int w = 0; w < NW; ++w) ss += red[0][w];
+    rstd = rsqrt_refined(fmaf(ss, inv_cols, eps));
+  } else {
+    float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+    for (int i = 0; i < N; i += 2) { s0 += v[i]; s1 += v[i + 1]; }
+    float mu = (s0 + s1) * (1.0f / N);
+    float q0 = 0.f, q1 = 0.f;
+#pragma unroll
+    for (int i = 0; i < N; i += 2) {
+      const float d0 = v[i] - mu, d1 = v[i + 1] - mu;
+      q0 = fmaf(d0, d0, q0); q1 = fmaf(d1, d1, q1);
+    }
+    float m2 = q0 + q1;
+    float half_c = 0.5f * N;
+#pragma unroll
+    for (int m = 1; m <= 16; m <<= 1) {                 // equal-count merges inside the warp
+      const float mb = __shfl_xor_sync(0xffffffffu, mu, m);
+      const float qb = __shfl_xor_sync(0xffffffffu, m2, m);
+      const float d = mb - mu;
+      mu = fmaf(0.5f, d, mu);
+      m2 = fmaf(d * d, half_c, m2 + qb);
+      half_c *= 2.f;
+    }
+    if ((threadIdx.x & 31) == 0) { red[0][threadIdx.x >> 5] = mu; red[1][threadIdx.x >> 5] = m2; }
+    __syncthreads();
+    float msum = 0.f, qsum = 0.f;
+    for (int w = 0; w < NW; ++w) { msum += red[0][w]; qsum += red[1][w]; }
+    mean = msum * inv_warps;
+    float dev = 0.f;
+    for (int w = 0; w < NW; ++w) { const float d = red[0][w] - mean; dev = fmaf(d, d, dev); }
+    rstd = rsqrt_refined(fmaf(fmaf(dev, 32.0f * N, qsum), inv_cols, eps));
+  }
+}
+
 // reg_norm_flex: the same predicate-free scheme for rows of exactly blockDim.x * VPT
 // vectors where blockDim.x is any multiple of 32 (hidden sizes such as 5120, 6144, 7168).
 // A CTA per row.  Every warp holds the same number of values, so the warps' (mean, M2)
@@ -174,48 +223,8 @@ __global__ void __launch_bounds__(1024, 1) reg_norm_flex(const RowParams p, cons
 #pragma unroll
       for (int j = 0; j < EPV; ++j) v[k * EPV + j] = f[j];
     }
-    float mean = 0.f, rstd;
-    if (OP == OP_RMSNORM) {
-      float s0 = 0.f, s1 = 0.f;
-#pragma unroll
-      for (int i = 0; i < N; i += 2) { s0 = fmaf(v[i], v[i], s0); s1 = fmaf(v[i + 1], v[i + 1], s1); }
-      float ss = warp_sum(s0 + s1);
-      if ((threadIdx.x & 31) == 0) red[parity][0][threadIdx.x >> 5] = ss;
-      __syncthreads();
-      ss = 0.f;
-      for (int w = 0; w < NW; ++w) ss += red[parity][0][w];
-      rstd = rsqrt_refined(fmaf(ss, inv_cols, p.eps));
-    } else {
-      float s0 = 0.f, s1 = 0.f;
-#pragma unroll
-      for (int i = 0; i < N; i += 2) { s0 += v[i]; s1 += v[i + 1]; }
-      float mu = (s0 + s1) * (1.0f / N);
-      float q0 = 0.f, q1 = 0.f;
-#pragma unroll
-      for (int i = 0; i < N; i += 2) {
-        const float d0 = v[i] - mu, d1 = v[i + 1] - mu;
-        q0 = fmaf(d0, d0, q0); q1 = fmaf(d1, d1, q1);
-      }
-      float m2 = q0 + q1;
-      float half_c = 0.5f * N;
-#pragma unroll
-      for (int m = 1; m <= 16; m <<= 1) {                 // equal-count merges inside the warp
-        const float mb = __shfl_xor_sync(0xffffffffu, mu, m);
-        const float qb = __shfl_xor_sync(0xffffffffu, m2, m);
-        const float d = mb - mu;
-        mu = fmaf(0.5f, d, mu);
-        m2 = fmaf(d * d, half_c, m2 + qb);
-        half_c *= 2.f;
-      }
-      if ((threadIdx.x & 31) == 0) { red[parity][0][threadIdx.x >> 5] = mu; red[parity][1][threadIdx.x >> 5] = m2; }
-      __syncthreads();
-      float msum = 0.f, qsum = 0.f;
-      for (int w = 0; w < NW; ++w) { msum += red[parity][0][w]; qsum += red[parity][1][w]; }
-      mean = msum * inv_warps;
-      float dev = 0.f;
-      for (int w = 0; w < NW; ++w) { const float d = red[parity][0][w] - mean; dev = fmaf(d, d, dev); }
-      rstd = rsqrt_refined(fmaf(fmaf(dev, 32.0f * N, qsum), inv_cols, p.eps));
-    }
+    float mean, rstd;
+    flex_row_stats<OP, N>(v, red[parity], NW, inv_warps, inv_cols, p.eps, mean, rstd);
     const T* gp = reinterpret_cast<const T*>(p.gamma) + tg * EPV;
     const T* bp = reinterpret_cast<const T*>(p.beta) + tg * EPV;
 #pragma unroll

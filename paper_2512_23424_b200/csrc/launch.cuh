@@ -43,6 +43,11 @@ int axis_reg_width(int dtype, int mode);
 cudaError_t launch_axis_reg(int op, int dtype, int mode, int r, const AxisParams& p, dim3 grid,
                             unsigned strips_per_outer, int nf, int nc, int pdl, cudaStream_t stream);
 
+// Fused residual add + LayerNorm / RMSNorm (op_fused.cu): a CTA of `threads` (a multiple of 32)
+// per row of exactly threads * vpt 16-byte vectors; p.res / p.sum carry the extra streams.
+cudaError_t launch_add_norm(int op, int dtype, int vpt, int threads, const RowParams& p, unsigned grid, int pdl,
+                            cudaStream_t stream);
+
 extern template cudaError_t launch_op<OP_SOFTMAX>(const LaunchPlan&, int, const RowParams&, cudaStream_t);
 extern template cudaError_t launch_op<OP_LOG_SOFTMAX>(const LaunchPlan&, int, const RowParams&, cudaStream_t);
 extern template cudaError_t launch_op<OP_LAYERNORM>(const LaunchPlan&, int, const RowParams&, cudaStream_t);
