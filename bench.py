@@ -8,7 +8,8 @@ second benchmark configuration) through the C ABI on inputs already resident in
 HBM; successive steps rotate over four buffer pairs so the working set (512 MiB)
 exceeds L2.  The one JSON line printed by rank 0 carries the headline number,
 the same figure for every configuration (`per_config`) and for the operators
-over a non-last axis (`axis_rows`), the roofline fraction, the end-to-end figure
+over a non-last axis (`axis_rows`) and the fused residual add + normalisation
+(`fused_rows`), the roofline fraction, the end-to-end figure
 with host buffers, and the fp64 CPU oracle's timing.
 
 With N > 1 (launched by torch.distributed.run) every rank runs the same
@@ -182,8 +183,39 @@ class AxisDeviceWorkload:
                                        eps=self.w.eps)
 
 
+class FusedDeviceWorkload:
+    """A fused residual add + normalisation workload resident in HBM, rotating buffer sets."""
+
+    def __init__(self, w: wl.FusedWorkload, sets: int):
+        import torch
+        from paper_2512_23424_b200 import binding
+        self.w, self.binding, self.torch = w, binding, torch
+
+        def dev(a):
+            if a is None:
+                return None
+            if w.dtype == wl.F32:
+                return torch.from_numpy(a).cuda()
+            return torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
+
+        x0, r0 = dev(w.x), dev(w.res)
+        self.xs = [x0] + [x0.clone() for _ in range(sets - 1)]
+        self.rs = [r0] + [r0.clone() for _ in range(sets - 1)]
+        self.ys = [torch.empty_like(x0) for _ in range(sets)]
+        self.ss = [torch.empty_like(x0) for _ in range(sets)]
+        self.gamma, self.beta = dev(w.gamma), dev(w.beta)
+        self.i = 0
+
+    def launch(self):
+        k = self.i % len(self.xs)
+        self.i += 1
+        return self.binding.add_norm(self.w.op, self.xs[k], self.rs[k], gamma=self.gamma, beta=self.beta,
+                                     eps=self.w.eps, out=self.ys[k], sum_out=self.ss[k])
+
+
 def pairs_for(w) -> int:
-    one = w.algorithmic_bytes() if isinstance(w, wl.AxisWorkload) else 2 * w.rows * w.cols * w.itemsize
+    one = (w.algorithmic_bytes() if isinstance(w, (wl.AxisWorkload, wl.FusedWorkload))
+           else 2 * w.rows * w.cols * w.itemsize)
     if one >= 3 * L2_BYTES:
         return 1
     return max(2, int(np.ceil(4 * L2_BYTES / one)))
@@ -426,6 +458,20 @@ def run_ours(args):
             del dwa, wa
             torch.cuda.empty_cache()
         line["axis_rows"] = axis
+        # fused residual add + normalisation (x and the residual in, y and the sum out)
+        fused = []
+        for name in wl.FUSED_CONFIGS:
+            wf = wl.make_fused(name)
+            dwf = FusedDeviceWorkload(wf, pairs_for(wf))
+            reps = max(10, min(100, 100 * args.steps // 1000))
+            sf = time_launches(dwf, reps, 5) / reps
+            bf = wf.algorithmic_bytes()
+            fused.append({"workload": name, "kernel": binding.last_kernel(), "us": sf * 1e6, "gbs": bf / sf / 1e9,
+                          "frac_measured": bf / sf / 1e9 / peak, "algorithmic_bytes": bf, "launches": reps,
+                          "rows_per_s": wf.x.shape[0] / sf, "traffic": profiled_traffic(name)})
+            del dwf, wf
+            torch.cuda.empty_cache()
+        line["fused_rows"] = fused
     if rank == 0 and world == 1:
         line["cpu_baseline"] = oracle_baseline(w)
     assert binding.device_status() == 0, "a device-side bounded wait expired"
@@ -480,6 +526,14 @@ def run_profile(args):
     import torch
     from paper_2512_23424_b200 import binding
     torch.cuda.set_device(0)
+    if args.profile_fused:
+        w = wl.make_fused(args.profile_fused, rows=args.profile_rows)
+        dw = FusedDeviceWorkload(w, pairs_for(w) if args.profile_rows is None else 1)
+        secs = time_launches(dw, args.steps, args.warmup)
+        print(json.dumps({"profile": args.profile_fused, "shape": list(w.x.shape), "kernel": binding.last_kernel(),
+                          "us_per_launch": secs / args.steps * 1e6, "launches": args.steps + max(args.warmup, 3),
+                          "algorithmic_bytes": w.algorithmic_bytes()}))
+        return
     if args.profile_axis:
         w = wl.make_axis(args.profile_axis, outer=args.profile_rows)
         for item in filter(None, args.tune.split(",")):
@@ -516,12 +570,14 @@ def main():
                     help="only launch configuration K (1..5) warmup+steps times, for use under ncu")
     ap.add_argument("--profile-axis", default="", metavar="NAME",
                     help="as --profile, for a non-last-axis configuration (workloads.AXIS_CONFIGS)")
+    ap.add_argument("--profile-fused", default="", metavar="NAME",
+                    help="as --profile, for a fused residual add + normalisation configuration (workloads.FUSED_CONFIGS)")
     ap.add_argument("--profile-rows", type=int, default=None,
                     help="truncate the rows of --profile (the outer axis of --profile-axis)")
     ap.add_argument("--variant", default="", help="force a kernel family in --profile mode")
     ap.add_argument("--tune", default="", help="--profile mode: key=value[,key=value] launch-geometry overrides")
     args = ap.parse_args()
-    if args.profile or args.profile_axis:
+    if args.profile or args.profile_axis or args.profile_fused:
         run_profile(args)
     elif args.impl == "reference":
         run_reference(args)

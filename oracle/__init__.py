@@ -212,6 +212,30 @@ def add_norm(op: str, x, res, gamma=None, beta=None, eps: float = 1e-5, nthreads
     return out_y, out_s
 
 
+ACTS = {"silu": 0, "gelu": 1, "gelu_tanh": 2}
+
+
+def act_mul(act: str, x, nthreads: int = 1):
+    """SiLU-and-Mul / GELU-and-Mul (named in Section 3.6): x is [rows, 2 d]; returns
+    act(x[:, :d]) * x[:, d:] as float64 [rows, d]."""
+    x, rows, cols, stride = _as2d(x)
+    if cols % 2:
+        raise ValueError("oracle: x must have an even number of columns")
+    d = cols // 2
+    out = np.empty((rows, d), dtype=np.float64)
+    L = lib()
+    if not L.oracle_act_mul.argtypes:
+        i64, vp, ci = ctypes.c_int64, ctypes.c_void_p, ctypes.c_int
+        L.oracle_act_mul.argtypes = [ci, vp, ci, i64, i64, i64, ctypes.POINTER(ctypes.c_double), ci]
+        L.oracle_act_mul.restype = ci
+        L.oracle_activation.argtypes = [ci, ctypes.c_double]
+        L.oracle_activation.restype = ctypes.c_double
+    rc = L.oracle_act_mul(ACTS[act], x.ctypes.data, _dtype_code(x), rows, d, stride, _dptr(out), int(nthreads))
+    if rc != 0:
+        raise ValueError("oracle_act_mul: malformed argument")
+    return out
+
+
 AXIS_OPS = {"softmax": 0, "log_softmax": 1, "layernorm": 2, "rmsnorm": 3}
 
 

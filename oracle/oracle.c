@@ -329,6 +329,30 @@ int oracle_add_norm(int op, const void* x, const void* res, int dtype, int64_t r
   return failed;
 }
 
+/* ---- gated activations: SiLU-and-Mul, GELU-and-Mul (named in Section 3.6) ---------- */
+
+double oracle_activation(int act, double a) {
+  if (act == 0) return a / (1.0 + exp(-a));                           /* SiLU: a * sigmoid(a) */
+  if (act == 1) return 0.5 * a * (1.0 + erf(a * 0.70710678118654752440)); /* GELU: a * Phi(a) */
+  /* GELU, tanh form: 0.5 a (1 + tanh(sqrt(2/pi) (a + 0.044715 a^3))) */
+  return 0.5 * a * (1.0 + tanh(0.79788456080286535588 * (a + 0.044715 * a * a * a)));
+}
+
+int oracle_act_mul(int act, const void* x, int dtype, int64_t rows, int64_t d, int64_t x_stride,
+                   double* out, int nthreads) {
+  if (act < 0 || act > 2) return 1;
+  if (rows < 0 || d < 0) return 1;
+  if (dtype != ORACLE_F32 && dtype != ORACLE_BF16 && dtype != ORACLE_F64) return 1;
+  int t = use_threads(nthreads);
+  if (rows == 0 || d == 0) return 0;
+  if (!x || !out || x_stride < 2 * d) return 1;
+#pragma omp parallel for schedule(static) num_threads(t)
+  for (int64_t i = 0; i < rows; ++i)
+    for (int64_t c = 0; c < d; ++c)
+      out[i * d + c] = oracle_activation(act, widen(x, dtype, i * x_stride + c)) * widen(x, dtype, i * x_stride + d + c);
+  return 0;
+}
+
 /* ---- the paper's verifier criterion (Section 3.2.3, Eq. 2-3) ------------------ */
 
 double oracle_verifier_fraction(const double* gen, const double* ref, int64_t n,

@@ -115,6 +115,18 @@ int oracle_add_norm(int op, const void* x, const void* res, int dtype, int64_t r
                     int64_t x_stride, int64_t res_stride, const void* gamma, const void* beta,
                     double eps, double* out_y, double* out_sum, int nthreads);
 
+/* Gated activations, "SiLU-and-Mul" and "GELU-and-Mul" of the paper's operator benchmark
+ * (Section 3.6 names them; the formulas are the textbook ones).  x is [rows, 2 d] with row
+ * stride x_stride >= 2 d: the first d columns are the gate a, the last d the factor b;
+ * out[i, c] = act(a[i, c]) * b[i, c], rows x d doubles, contiguous.
+ *   act 0: SiLU   a / (1 + e^-a)
+ *   act 1: GELU   a * Phi(a) = 0.5 a (1 + erf(a / sqrt 2))
+ *   act 2: GELU, tanh form   0.5 a (1 + tanh(sqrt(2 / pi) (a + 0.044715 a^3)))
+ * Returns 0, or 1 on a bad argument. */
+double oracle_activation(int act, double a);
+int oracle_act_mul(int act, const void* x, int dtype, int64_t rows, int64_t d, int64_t x_stride,
+                   double* out, int nthreads);
+
 /* The paper's correctness criterion (Section 3.2.3, Eq. 2-3): element error is
  * |gen-ref|/|ref| when |ref| > eps_switch, else |gen-ref|; returns the fraction
  * of elements whose error exceeds tau (the kernel passes iff that fraction is

@@ -223,3 +223,53 @@ def make_axis(name: str, outer: Optional[int] = None, seed_offset: int = 0) -> A
         gamma = None if gamma is None else f32_to_bf16_bits(gamma)
         beta = None if beta is None else f32_to_bf16_bits(beta)
     return AxisWorkload(name, op, dtype, x, eps=1e-5 if gamma is not None else 0.0, gamma=gamma, beta=beta)
+
+
+# ---------------------------------------------------------------------------------------------
+# Fused residual add + normalisation (a "fused variant" of the paper's operator benchmark,
+# Section 3.6): the pre-norm residual step of a transformer block at the hidden sizes of
+# configurations 2 and 3; x is the branch output, res the residual stream.
+# ---------------------------------------------------------------------------------------------
+FUSED_CONFIGS: Dict[str, tuple] = {
+    "add_rmsnorm_bf16_16384x8192": ("rmsnorm", BF16, 16384, 8192, 1e-6),
+    "add_layernorm_f32_4096x4096": ("layernorm", F32, 4096, 4096, 1e-5),
+    "add_rmsnorm_f32_8192x4096": ("rmsnorm", F32, 8192, 4096, 1e-6),
+    "add_layernorm_bf16_16384x4096": ("layernorm", BF16, 16384, 4096, 1e-5),
+}
+
+
+@dataclass
+class FusedWorkload:
+    name: str
+    op: str
+    dtype: int
+    x: np.ndarray                      # [rows, cols]; float32, or uint16 bf16 bits
+    res: np.ndarray                    # same shape and storage
+    eps: float
+    gamma: Optional[np.ndarray] = None
+    beta: Optional[np.ndarray] = None
+
+    @property
+    def itemsize(self) -> int:
+        return 4 if self.dtype == F32 else 2
+
+    def algorithmic_bytes(self) -> int:
+        """x and res read once, y and the sum written once, gamma / beta once."""
+        vec = sum(v.size for v in (self.gamma, self.beta) if v is not None)
+        return (4 * self.x.size + vec) * self.itemsize
+
+
+def make_fused(name: str, rows: Optional[int] = None, seed_offset: int = 0) -> FusedWorkload:
+    op, dtype, r, c, eps = FUSED_CONFIGS[name]
+    r = r if rows is None else min(r, rows)
+    seed = 200 + sorted(FUSED_CONFIGS).index(name) + 1000 * seed_offset
+    s_x, s_r, s_g, s_b = np.random.SeedSequence(seed).spawn(4)
+    rx, rr, rg, rb = (np.random.Generator(np.random.PCG64(s)) for s in (s_x, s_r, s_g, s_b))
+    x = _normal_f32(rx, r, c)                                        # branch output ~ N(0, 1)
+    res = _normal_f32(rr, r, c) * np.float32(2.0) + np.float32(0.5)  # residual stream: wider, offset
+    gamma = rg.uniform(0.5, 1.5, c).astype(np.float32)
+    beta = (rb.standard_normal(c) * 0.1).astype(np.float32) if op == "layernorm" else None
+    if dtype == BF16:
+        x, res, gamma = f32_to_bf16_bits(x), f32_to_bf16_bits(res), f32_to_bf16_bits(gamma)
+        beta = None if beta is None else f32_to_bf16_bits(beta)
+    return FusedWorkload(name, op, dtype, x, res, eps, gamma=gamma, beta=beta)
