@@ -187,6 +187,23 @@ akg_status akg_add_norm(akg_op op, const void* x, const void* residual, void* y,
                         int64_t y_row_stride, int64_t sum_row_stride, akg_dtype dtype,
                         const void* gamma, const void* beta, float eps, void* stream);
 
+/* Gated activations "SiLU-and-Mul" / "GELU-and-Mul" (named among the operators of the paper's
+ * benchmark, Section 3.6; textbook formulas).  x: DEVICE matrix [rows, 2 d] with row stride
+ * x_row_stride >= 2 d elements; the first d columns of a row are the gate a, the last d the
+ * factor b.  y: DEVICE matrix [rows, d], row stride y_row_stride >= d:
+ *   y[r, c] = act(a[r, c]) * b[r, c]
+ *   AKG_ACT_SILU       act(a) = a / (1 + e^-a)
+ *   AKG_ACT_GELU       act(a) = 0.5 a (1 + erf(a / sqrt 2))
+ *   AKG_ACT_GELU_TANH  act(a) = 0.5 a (1 + tanh(sqrt(2 / pi) (a + 0.044715 a^3)))
+ * fp32 arithmetic on the widened inputs, one rounding at the store.  y may be x itself with
+ * the same row stride (the result replaces the gate half); any other overlap is
+ * AKG_ERR_INVALID_ARG.  16-byte aligned bases and strides with d a multiple of the vector
+ * width take 128-bit accesses, anything else a scalar path with the same results.  Enqueues
+ * on `stream` and returns; errors as for the other entry points. */
+typedef enum akg_act { AKG_ACT_SILU = 0, AKG_ACT_GELU = 1, AKG_ACT_GELU_TANH = 2 } akg_act;
+akg_status akg_act_mul(akg_act act, const void* x, void* y, int64_t rows, int64_t d,
+                       int64_t x_row_stride, int64_t y_row_stride, akg_dtype dtype, void* stream);
+
 /* Size of the staging area built into the library (see akg_rowop_host_static). */
 #define AKG_STATIC_STAGING_BYTES (16u << 20)
 

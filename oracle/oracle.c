@@ -333,9 +333,13 @@ int oracle_add_norm(int op, const void* x, const void* res, int dtype, int64_t r
 
 double oracle_activation(int act, double a) {
   if (act == 0) return a / (1.0 + exp(-a));                           /* SiLU: a * sigmoid(a) */
-  if (act == 1) return 0.5 * a * (1.0 + erf(a * 0.70710678118654752440)); /* GELU: a * Phi(a) */
-  /* GELU, tanh form: 0.5 a (1 + tanh(sqrt(2/pi) (a + 0.044715 a^3))) */
-  return 0.5 * a * (1.0 + tanh(0.79788456080286535588 * (a + 0.044715 * a * a * a)));
+  /* GELU: a * Phi(a), Phi(a) = 0.5 (1 + erf(a / sqrt 2)) = 0.5 erfc(-a / sqrt 2); the second
+   * form is the same number without the cancellation of 1 + erf in the left tail */
+  if (act == 1) return 0.5 * a * erfc(-a * 0.70710678118654752440);
+  /* GELU, tanh form: 0.5 a (1 + tanh(u)), u = sqrt(2/pi) (a + 0.044715 a^3); by the identity
+   * 0.5 (1 + tanh u) = 1 / (1 + e^(-2u)) it is evaluated without the cancellation of 1 + tanh */
+  double u = 0.79788456080286535588 * (a + 0.044715 * a * a * a);
+  return a / (1.0 + exp(-2.0 * u));
 }
 
 int oracle_act_mul(int act, const void* x, int dtype, int64_t rows, int64_t d, int64_t x_stride,

@@ -326,6 +326,33 @@ def add_norm(op: str, x: torch.Tensor, residual: torch.Tensor, *, gamma: Optiona
     return out, sum_out
 
 
+ACTS = {"silu": 0, "gelu": 1, "gelu_tanh": 2}
+
+
+def act_mul(act: str, x: torch.Tensor, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """akg_act_mul: act(x[:, :d]) * x[:, d:] for a 2-D CUDA tensor [rows, 2 d]; act is "silu",
+    "gelu" or "gelu_tanh".  `out` ([rows, d]) defaults to a new tensor."""
+    rows, cols, xs = _matrix(x, "x")
+    if cols % 2:
+        raise ValueError("x must have an even number of columns (gate | factor)")
+    d = cols // 2
+    if out is None:
+        out = torch.empty((rows, d), dtype=x.dtype, device=x.device)
+    orow, ocol, ys = _matrix(out, "out")
+    if (orow, ocol) != (rows, d) or out.dtype != x.dtype or out.device != x.device:
+        raise ValueError("out must be [rows, d] of x's dtype on x's device")
+    fn = lib().akg_act_mul
+    if not fn.argtypes:
+        vp, i64, ci = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int
+        fn.argtypes = [ci, vp, vp, i64, i64, i64, i64, ci, vp]
+        fn.restype = ci
+    with torch.cuda.device(x.device):
+        st = fn(ACTS[act], x.data_ptr(), out.data_ptr(), rows, d, xs if rows > 1 else max(xs, 2 * d), ys,
+                _dtype_code(x), _stream(stream))
+    _check(st, "akg_act_mul")
+    return out
+
+
 STATIC_STAGING_BYTES = 16 << 20
 
 

@@ -870,6 +870,53 @@ extern "C" akg_status akg_add_norm(akg_op op, const void* x, const void* residua
   return AKG_OK;
 }
 
+// ---- gated activations: SiLU-and-Mul, GELU-and-Mul -----------------------------------------
+extern "C" akg_status akg_act_mul(akg_act act, const void* x, void* y, int64_t rows, int64_t d,
+                                  int64_t x_row_stride, int64_t y_row_stride, akg_dtype dtype, void* stream) {
+  using namespace akg;
+  const char* name = "akg_act_mul";
+  t_error[0] = '\0';
+  if (act < AKG_ACT_SILU || act > AKG_ACT_GELU_TANH) return fail(AKG_ERR_INVALID_ARG, "%s: unknown activation", name);
+  if (dtype != AKG_F32 && dtype != AKG_BF16) return fail(AKG_ERR_INVALID_ARG, "%s: unknown dtype", name);
+  if (rows < 0 || d < 0) return fail(AKG_ERR_INVALID_ARG, "%s: negative rows or d", name);
+  if (rows == 0 || d == 0) return AKG_OK;
+  if (x == nullptr || y == nullptr) return fail(AKG_ERR_INVALID_ARG, "%s: x and y must not be NULL", name);
+  if (d > (int64_t(1) << 40)) return fail(AKG_ERR_UNSUPPORTED, "%s: d above 2^40", name);
+  if (x_row_stride < 2 * d || y_row_stride < d) return fail(AKG_ERR_INVALID_ARG, "%s: row stride too small", name);
+  const int64_t es = (dtype == AKG_F32) ? 4 : 2;
+  if (static_cast<long double>(rows) * x_row_stride * es > 9.0e18L ||
+      static_cast<long double>(rows) * y_row_stride * es > 9.0e18L)
+    return fail(AKG_ERR_INVALID_ARG, "%s: rows * stride overflows", name);
+  // y may be x itself with the same row stride (the result then replaces the gate half: every
+  // element is read before the same thread writes it); any other overlap is refused
+  const uintptr_t x0 = reinterpret_cast<uintptr_t>(x), y0 = reinterpret_cast<uintptr_t>(y);
+  const uintptr_t x1 = x0 + static_cast<uintptr_t>(((rows - 1) * x_row_stride + 2 * d) * es);
+  const uintptr_t y1 = y0 + static_cast<uintptr_t>(((rows - 1) * y_row_stride + d) * es);
+  if (x0 < y1 && y0 < x1 && !(x0 == y0 && (rows == 1 || x_row_stride == y_row_stride)))
+    return fail(AKG_ERR_INVALID_ARG, "%s: x and y overlap without y being x", name);
+
+  ActParams p;
+  p.x = x; p.y = y; p.rows = rows; p.d = d; p.xs = x_row_stride; p.ys = y_row_stride;
+  const int64_t epv = 16 / es;
+  const bool vec = g_forced_variant.load() != V_STREAM && d % epv == 0 && aligned16(x) && aligned16(y) &&
+                   (rows == 1 || ((x_row_stride * es) % 16 == 0 && (y_row_stride * es) % 16 == 0));
+  const int64_t lanes = vec ? d / epv : d;
+  const int u = act_mul_unroll();
+  int threads = 32;
+  while (threads < 256 && static_cast<int64_t>(threads) * u < lanes) threads <<= 1;
+  const int64_t chunks = (lanes + static_cast<int64_t>(threads) * u - 1) / (static_cast<int64_t>(threads) * u);
+  const int cap = g_tune_grid_cap.load();
+  const dim3 grid(static_cast<unsigned>(std::min<int64_t>(chunks, cap > 0 ? cap : (int64_t(1) << 30))),
+                  static_cast<unsigned>(std::min<int64_t>(rows, 65535)));
+  const cudaError_t err = launch_act_mul(static_cast<int>(act), static_cast<int>(dtype), vec, p, grid, threads,
+                                         g_tune_pdl.load() == 2 ? 0 : 1, static_cast<cudaStream_t>(stream));
+  if (err != cudaSuccess) return cuda_fail(name, err);
+  std::snprintf(t_kernel, sizeof t_kernel, "act_mul<%s,%s,%s,t%d,grid%ux%u>",
+                act == AKG_ACT_SILU ? "silu" : (act == AKG_ACT_GELU ? "gelu" : "gelu_tanh"),
+                dtype == AKG_F32 ? "f32" : "bf16", vec ? "vec" : "scalar", threads, grid.x, grid.y);
+  return AKG_OK;
+}
+
 // ---- host buffers without any allocation ---------------------------------------------------
 // akg_rowop_host needs a device staging area from its caller.  Some callers have no way to
 // get one: a plug-in that is handed host buffers and a stream but no allocator, a service

@@ -49,6 +49,14 @@ struct AxisParams {
   float eps;
 };
 
+// One gated-activation call: x[rows, 2 d] (gate | factor), y[rows, d].
+struct ActParams {
+  const void* x;
+  void* y;
+  long long rows, d;                  // d: output columns
+  long long xs, ys;                   // row strides in elements
+};
+
 // Shared-memory ring kernels: limits and the size of the bookkeeping area that
 // precedes the ring buffers (mbarriers, CTA reduction slots, cluster exchange slots).
 constexpr int kMaxCluster = 16;

@@ -48,6 +48,12 @@ cudaError_t launch_axis_reg(int op, int dtype, int mode, int r, const AxisParams
 cudaError_t launch_add_norm(int op, int dtype, int vpt, int threads, const RowParams& p, unsigned grid, int pdl,
                             cudaStream_t stream);
 
+// Gated activations (op_act.cu).  act: 0 SiLU, 1 GELU, 2 GELU tanh form.  vec: 16-byte vectors.
+// grid = (chunks of act_mul_unroll() * threads lanes of one row, rows), either may be smaller.
+int act_mul_unroll();
+cudaError_t launch_act_mul(int act, int dtype, bool vec, const ActParams& p, dim3 grid, int threads, int pdl,
+                           cudaStream_t stream);
+
 extern template cudaError_t launch_op<OP_SOFTMAX>(const LaunchPlan&, int, const RowParams&, cudaStream_t);
 extern template cudaError_t launch_op<OP_LOG_SOFTMAX>(const LaunchPlan&, int, const RowParams&, cudaStream_t);
 extern template cudaError_t launch_op<OP_LAYERNORM>(const LaunchPlan&, int, const RowParams&, cudaStream_t);

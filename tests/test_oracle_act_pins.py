@@ -18,7 +18,7 @@ ACTS = ["silu", "gelu", "gelu_tanh"]
 
 
 def mp_act(act, a):
-    mp.dps = 40
+    mp.dps = 100                    # 1 + erf and 1 + tanh cancel up to 60 digits at the gates tested below
     a = mpf(float(a))
     if act == "silu":
         return a / (1 + mpexp(-a))
@@ -65,6 +65,17 @@ def test_identities_of_the_activations():
     t = oracle.act_mul("gelu_tanh", np.concatenate([a, one], axis=1))
     e = oracle.act_mul("gelu", np.concatenate([a, one], axis=1))
     assert 1e-6 < np.max(np.abs(t - e)) < 5e-4
+
+
+def test_left_tail_keeps_its_relative_accuracy():
+    """1 + erf and 1 + tanh cancel for very negative gates; the oracle must not (the GPU kernels
+    are checked against it to a relative tolerance there)."""
+    a = np.array([[-4.0, -6.0, -8.0, -10.0, -12.5, -7.625, 1.0, 1.0, 1.0, 1.0, 1.0, 1.0]])
+    for act in ACTS:
+        got = oracle.act_mul(act, a)[0]
+        want = np.array([float(mp_act(act, v)) for v in a[0, :6]])
+        assert np.all(want < 0) and np.all(got < 0)
+        assert np.max(np.abs(got - want) / np.abs(want)) < 1e-12
 
 
 def test_against_torch_float64():
