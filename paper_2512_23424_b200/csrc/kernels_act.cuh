@@ -15,11 +15,11 @@ namespace akg {
 
 enum Act : int { ACT_SILU = 0, ACT_GELU = 1, ACT_GELU_TANH = 2 };
 
-// 1 / (1 + e^-t): two special-function evaluations (about 1 ulp each); the reciprocal keeps
-// subnormal results, so the far left tail fades out instead of being cut to zero
+// 1 / (1 + e^-t): two special-function evaluations (about 1 ulp each), both flushing
+// subnormal results to zero: a sigmoid below 2^-126 (t < -87.3) is returned as 0
 __device__ __forceinline__ float sigmoid_f32(float t) {
   float r;
-  asm("rcp.approx.f32 %0, %1;" : "=f"(r) : "f"(1.0f + ex2_approx(-t * kLog2e)));
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(1.0f + ex2_approx(-t * kLog2e)));
   return r;
 }
 
@@ -38,7 +38,7 @@ template <int DEG> __device__ __forceinline__ float normal_cdf(float a) {
                            2.017114013e-01f, 8.792584389e-02f, -9.248869121e-02f};
   static_assert(DEG == 9 || DEG == 5, "fitted degrees");
   float t;
-  asm("rcp.approx.f32 %0, %1;" : "=f"(t) : "f"(fmaf(fabsf(a), 0.35355339059327376220f, 1.0f)));
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t) : "f"(fmaf(fabsf(a), 0.35355339059327376220f, 1.0f)));
   float h = (DEG == 9) ? c9[9] : c5[5];
 #pragma unroll
   for (int i = DEG - 1; i >= 0; --i) h = fmaf(h, t, (DEG == 9) ? c9[i] : c5[i]);

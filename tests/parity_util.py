@@ -141,8 +141,9 @@ def cancel_magnitude(w: wl.Workload, ref: np.ndarray, additive: Optional[np.ndar
 
 
 def compare(got_stored: np.ndarray, ref: np.ndarray, dtype: int, what: str = "",
-            cancel_mag: Optional[np.ndarray] = None) -> dict:
-    """Assert parity under the tolerances above; returns error statistics."""
+            cancel_mag: Optional[np.ndarray] = None, tiny: float = 2.0 ** -126) -> dict:
+    """Assert parity under the tolerances above; returns error statistics.  `tiny`: bf16 results
+    whose reference is below it in magnitude may be returned as a flushed zero."""
     got = widen(got_stored)
     assert got.shape == ref.shape, (what, got.shape, ref.shape)
     ref_nan, got_nan = np.isnan(ref), np.isnan(got)
@@ -163,7 +164,7 @@ def compare(got_stored: np.ndarray, ref: np.ndarray, dtype: int, what: str = "",
     else:
         ulp = bf16_ulp(ref[fin])
         ulps = err / ulp
-        tiny_ok = (np.abs(ref[fin]) < 2.0 ** -126) & (got[fin] == 0)
+        tiny_ok = (np.abs(ref[fin]) < tiny) & (got[fin] == 0)
         bad = (ulps > BF16_ULPS) & ~tiny_ok
         stats["max_ulp"] = float(ulps.max()) if ulps.size else 0.0
         assert not bad.any(), f"{what}: {bad.sum()} elements beyond {BF16_ULPS} bf16 ulps (max {stats['max_ulp']:.3f})"

@@ -22,7 +22,10 @@ def make(dtype, rows, d, seed, scale=1.5):
 
 def check(act, dtype, x, got, what):
     ref = oracle.act_mul(act, x, nthreads=8)
-    compare(got, ref, dtype, what)
+    # the kernels flush a sigmoid / distribution value below 2^-126 to zero before the two
+    # multiplications, so a product below 2^-126 * |gate * factor| (< 2^-110 for any input these
+    # tests draw) may come back as zero; everything else is held to the usual tolerance
+    compare(got, ref, dtype, what, tiny=2.0 ** -110)
     assert verifier_passes(got, ref, dtype)
 
 
