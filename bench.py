@@ -9,7 +9,7 @@ HBM; successive steps rotate over four buffer pairs so the working set (512 MiB)
 exceeds L2.  The one JSON line printed by rank 0 carries the headline number,
 the same figure for every configuration (`per_config`) and for the operators
 over a non-last axis (`axis_rows`) and the fused residual add + normalisation
-(`fused_rows`), the roofline fraction, the end-to-end figure
+(`fused_rows`) and the gated activations (`act_rows`), the roofline fraction, the end-to-end figure
 with host buffers, and the fp64 CPU oracle's timing.
 
 With N > 1 (launched by torch.distributed.run) every rank runs the same
@@ -213,8 +213,29 @@ class FusedDeviceWorkload:
                                      eps=self.w.eps, out=self.ys[k], sum_out=self.ss[k])
 
 
+class ActDeviceWorkload:
+    """A gated-activation workload x[rows, 2 d] resident in HBM, rotating buffer pairs."""
+
+    def __init__(self, w: wl.ActWorkload, pairs: int):
+        import torch
+        from paper_2512_23424_b200 import binding
+        self.w, self.binding, self.torch = w, binding, torch
+        if w.dtype == wl.F32:
+            x0 = torch.from_numpy(w.x).cuda()
+        else:
+            x0 = torch.from_numpy(w.x.view(np.int16)).cuda().view(torch.bfloat16)
+        self.xs = [x0] + [x0.clone() for _ in range(pairs - 1)]
+        self.ys = [torch.empty((x0.shape[0], x0.shape[1] // 2), dtype=x0.dtype, device="cuda") for _ in range(pairs)]
+        self.i = 0
+
+    def launch(self):
+        k = self.i % len(self.xs)
+        self.i += 1
+        return self.binding.act_mul(self.w.act, self.xs[k], out=self.ys[k])
+
+
 def pairs_for(w) -> int:
-    one = (w.algorithmic_bytes() if isinstance(w, (wl.AxisWorkload, wl.FusedWorkload))
+    one = (w.algorithmic_bytes() if isinstance(w, (wl.AxisWorkload, wl.FusedWorkload, wl.ActWorkload))
            else 2 * w.rows * w.cols * w.itemsize)
     if one >= 3 * L2_BYTES:
         return 1
@@ -472,6 +493,20 @@ def run_ours(args):
             del dwf, wf
             torch.cuda.empty_cache()
         line["fused_rows"] = fused
+        # gated activations (gate and factor in, product out)
+        acts = []
+        for name in wl.ACT_CONFIGS:
+            wa = wl.make_act(name)
+            dwa = ActDeviceWorkload(wa, pairs_for(wa))
+            reps = max(10, min(100, 100 * args.steps // 1000))
+            sa = time_launches(dwa, reps, 5) / reps
+            ba = wa.algorithmic_bytes()
+            acts.append({"workload": name, "kernel": binding.last_kernel(), "us": sa * 1e6, "gbs": ba / sa / 1e9,
+                         "frac_measured": ba / sa / 1e9 / peak, "algorithmic_bytes": ba, "launches": reps,
+                         "rows_per_s": wa.x.shape[0] / sa, "traffic": profiled_traffic(name)})
+            del dwa, wa
+            torch.cuda.empty_cache()
+        line["act_rows"] = acts
     if rank == 0 and world == 1:
         line["cpu_baseline"] = oracle_baseline(w)
     assert binding.device_status() == 0, "a device-side bounded wait expired"
@@ -526,6 +561,14 @@ def run_profile(args):
     import torch
     from paper_2512_23424_b200 import binding
     torch.cuda.set_device(0)
+    if args.profile_act:
+        w = wl.make_act(args.profile_act, rows=args.profile_rows)
+        dw = ActDeviceWorkload(w, pairs_for(w) if args.profile_rows is None else 1)
+        secs = time_launches(dw, args.steps, args.warmup)
+        print(json.dumps({"profile": args.profile_act, "shape": list(w.x.shape), "kernel": binding.last_kernel(),
+                          "us_per_launch": secs / args.steps * 1e6, "launches": args.steps + max(args.warmup, 3),
+                          "algorithmic_bytes": w.algorithmic_bytes()}))
+        return
     if args.profile_fused:
         w = wl.make_fused(args.profile_fused, rows=args.profile_rows)
         dw = FusedDeviceWorkload(w, pairs_for(w) if args.profile_rows is None else 1)
@@ -570,6 +613,8 @@ def main():
                     help="only launch configuration K (1..5) warmup+steps times, for use under ncu")
     ap.add_argument("--profile-axis", default="", metavar="NAME",
                     help="as --profile, for a non-last-axis configuration (workloads.AXIS_CONFIGS)")
+    ap.add_argument("--profile-act", default="", metavar="NAME",
+                    help="as --profile, for a gated-activation configuration (workloads.ACT_CONFIGS)")
     ap.add_argument("--profile-fused", default="", metavar="NAME",
                     help="as --profile, for a fused residual add + normalisation configuration (workloads.FUSED_CONFIGS)")
     ap.add_argument("--profile-rows", type=int, default=None,
@@ -577,7 +622,7 @@ def main():
     ap.add_argument("--variant", default="", help="force a kernel family in --profile mode")
     ap.add_argument("--tune", default="", help="--profile mode: key=value[,key=value] launch-geometry overrides")
     args = ap.parse_args()
-    if args.profile or args.profile_axis or args.profile_fused:
+    if args.profile or args.profile_axis or args.profile_fused or args.profile_act:
         run_profile(args)
     elif args.impl == "reference":
         run_reference(args)

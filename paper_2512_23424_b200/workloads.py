@@ -273,3 +273,43 @@ def make_fused(name: str, rows: Optional[int] = None, seed_offset: int = 0) -> F
         x, res, gamma = f32_to_bf16_bits(x), f32_to_bf16_bits(res), f32_to_bf16_bits(gamma)
         beta = None if beta is None else f32_to_bf16_bits(beta)
     return FusedWorkload(name, op, dtype, x, res, eps, gamma=gamma, beta=beta)
+
+
+# ---------------------------------------------------------------------------------------------
+# Gated activations (SiLU-and-Mul, GELU-and-Mul; named in Section 3.6): x = [gate | factor] of
+# a feed-forward block, [tokens, 2 d] with d the intermediate size.
+# ---------------------------------------------------------------------------------------------
+ACT_CONFIGS: Dict[str, tuple] = {
+    "silu_and_mul_bf16_8192x14336": ("silu", BF16, 8192, 14336),
+    "gelu_and_mul_bf16_8192x14336": ("gelu", BF16, 8192, 14336),
+    "gelu_tanh_and_mul_bf16_8192x14336": ("gelu_tanh", BF16, 8192, 14336),
+    "silu_and_mul_f32_4096x11008": ("silu", F32, 4096, 11008),
+    "gelu_and_mul_f32_4096x11008": ("gelu", F32, 4096, 11008),
+}
+
+
+@dataclass
+class ActWorkload:
+    name: str
+    act: str
+    dtype: int
+    x: np.ndarray                      # [rows, 2 d]; float32, or uint16 bf16 bits
+
+    @property
+    def itemsize(self) -> int:
+        return 4 if self.dtype == F32 else 2
+
+    def algorithmic_bytes(self) -> int:
+        """Gate and factor read once, the product written once."""
+        return (self.x.size + self.x.size // 2) * self.itemsize
+
+
+def make_act(name: str, rows: Optional[int] = None, seed_offset: int = 0) -> ActWorkload:
+    act, dtype, r, d = ACT_CONFIGS[name]
+    r = r if rows is None else min(r, rows)
+    seed = 300 + sorted(ACT_CONFIGS).index(name) + 1000 * seed_offset
+    rx = np.random.Generator(np.random.PCG64(np.random.SeedSequence(seed)))
+    x = _normal_f32(rx, r, 2 * d) * np.float32(1.5)                  # pre-activations ~ N(0, 1.5^2)
+    if dtype == BF16:
+        x = f32_to_bf16_bits(x)
+    return ActWorkload(name, act, dtype, x)
