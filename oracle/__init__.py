@@ -125,7 +125,7 @@ def _vec(v: Optional[np.ndarray], like: np.ndarray, cols: int):
     return v, v.ctypes.data
 
 
-def _softmax_like(fn_name, x, mask, row_ids, nthreads):
+def _softmax_like(fn_name, x, mask, row_ids, nthreads, scale=None, want_log=0):
     x, rows, cols, stride = _as2d(x)
     out = np.empty((rows, cols), dtype=np.float64)
     cm, keep = None, None
@@ -143,10 +143,21 @@ def _softmax_like(fn_name, x, mask, row_ids, nthreads):
         ids = np.ascontiguousarray(row_ids, dtype=np.int64)
         if ids.shape != (rows,):
             raise ValueError("oracle: row_ids must have one entry per row")
-    rc = getattr(lib(), fn_name)(
-        x.ctypes.data, _dtype_code(x), rows, cols, stride,
-        ids.ctypes.data if ids is not None else None,
-        ctypes.byref(cm) if cm is not None else None, _dptr(out), int(nthreads))
+    if scale is not None:
+        fn = lib().oracle_softmax_scaled
+        if not fn.argtypes:
+            i64, vp, ci = ctypes.c_int64, ctypes.c_void_p, ctypes.c_int
+            fn.argtypes = [vp, ci, i64, i64, i64, ctypes.c_double, vp, vp, ci, ctypes.POINTER(ctypes.c_double), ci]
+            fn.restype = ci
+        rc = fn(x.ctypes.data, _dtype_code(x), rows, cols, stride, float(scale),
+                ids.ctypes.data if ids is not None else None,
+                ctypes.cast(ctypes.byref(cm), ctypes.c_void_p) if cm is not None else None, int(want_log),
+                _dptr(out), int(nthreads))
+    else:
+        rc = getattr(lib(), fn_name)(
+            x.ctypes.data, _dtype_code(x), rows, cols, stride,
+            ids.ctypes.data if ids is not None else None,
+            ctypes.byref(cm) if cm is not None else None, _dptr(out), int(nthreads))
     if rc != 0:
         raise ValueError(f"{fn_name}: malformed argument")
     return out
@@ -158,6 +169,13 @@ def softmax(x, mask: Optional[Mask] = None, row_ids=None, nthreads: int = 1):
 
 def log_softmax(x, mask: Optional[Mask] = None, row_ids=None, nthreads: int = 1):
     return _softmax_like("oracle_log_softmax", x, mask, row_ids, nthreads)
+
+
+def softmax_scaled(x, scale: float, mask: Optional[Mask] = None, log: bool = False, row_ids=None,
+                   nthreads: int = 1):
+    """softmax (or log-softmax) of scale * x + additive mask under the causal rule: the fused
+    pre-scale variant.  The additive mask is not scaled."""
+    return _softmax_like("oracle_softmax_scaled", x, mask, row_ids, nthreads, scale=scale, want_log=1 if log else 0)
 
 
 def logsumexp_row(z: np.ndarray) -> float:

@@ -132,10 +132,11 @@ static int use_threads(int nthreads) {
   return t;
 }
 
-/* z for one row: widen, add the additive mask, apply the causal rule */
+/* z for one row: widen, scale (1.0 for the plain operators: exact), add the additive mask,
+ * apply the causal rule */
 static void masked_row(const void* x, int dtype, int64_t cols, int64_t x_off,
-                       int64_t grow, const oracle_mask* mask, double* z) {
-  for (int64_t c = 0; c < cols; ++c) z[c] = widen(x, dtype, x_off + c);
+                       int64_t grow, const oracle_mask* mask, double scale, double* z) {
+  for (int64_t c = 0; c < cols; ++c) z[c] = scale * widen(x, dtype, x_off + c);
   if (!mask) return;
   if (mask->additive) {
     int64_t mr = grow % mask->add_rows;
@@ -152,8 +153,9 @@ static void masked_row(const void* x, int dtype, int64_t cols, int64_t x_off,
 static int softmax_driver(const void* x, int dtype, int64_t rows, int64_t cols,
                           int64_t x_stride, const int64_t* row_ids,
                           const oracle_mask* mask, double* out, int nthreads,
-                          int want_log) {
+                          int want_log, double scale) {
   if (bad_shape(x, dtype, rows, cols, x_stride, out)) return 1;
+  if (!(scale > 0.0) || isinf(scale)) return 1;
   if (mask) {
     if (mask->additive && (mask->add_rows < 1 || mask->add_row_stride < cols)) return 1;
     if (mask->causal && mask->causal_period < 1) return 1;
@@ -172,7 +174,7 @@ static int softmax_driver(const void* x, int dtype, int64_t rows, int64_t cols,
     for (int64_t i = 0; i < rows; ++i) {
       if (!z) continue;
       int64_t grow = row_ids ? row_ids[i] : i;
-      masked_row(x, dtype, cols, i * x_stride, grow, mask, z);
+      masked_row(x, dtype, cols, i * x_stride, grow, mask, scale, z);
       if (want_log) oracle_log_softmax_row(z, cols, out + i * cols);
       else          oracle_softmax_row(z, cols, out + i * cols);
     }
@@ -184,13 +186,20 @@ static int softmax_driver(const void* x, int dtype, int64_t rows, int64_t cols,
 int oracle_softmax(const void* x, int dtype, int64_t rows, int64_t cols,
                    int64_t x_stride, const int64_t* row_ids,
                    const oracle_mask* mask, double* out, int nthreads) {
-  return softmax_driver(x, dtype, rows, cols, x_stride, row_ids, mask, out, nthreads, 0);
+  return softmax_driver(x, dtype, rows, cols, x_stride, row_ids, mask, out, nthreads, 0, 1.0);
 }
 
 int oracle_log_softmax(const void* x, int dtype, int64_t rows, int64_t cols,
                        int64_t x_stride, const int64_t* row_ids,
                        const oracle_mask* mask, double* out, int nthreads) {
-  return softmax_driver(x, dtype, rows, cols, x_stride, row_ids, mask, out, nthreads, 1);
+  return softmax_driver(x, dtype, rows, cols, x_stride, row_ids, mask, out, nthreads, 1, 1.0);
+}
+
+/* softmax / log-softmax of scale * x (+ additive mask, causal rule): the fused pre-scale */
+int oracle_softmax_scaled(const void* x, int dtype, int64_t rows, int64_t cols,
+                          int64_t x_stride, double scale, const int64_t* row_ids,
+                          const oracle_mask* mask, int want_log, double* out, int nthreads) {
+  return softmax_driver(x, dtype, rows, cols, x_stride, row_ids, mask, out, nthreads, want_log ? 1 : 0, scale);
 }
 
 static double* widen_vector(const void* v, int dtype, int64_t n) {

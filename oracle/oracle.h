@@ -84,6 +84,13 @@ int oracle_softmax(const void* x, int dtype, int64_t rows, int64_t cols,
 int oracle_log_softmax(const void* x, int dtype, int64_t rows, int64_t cols,
                        int64_t x_stride, const int64_t* row_ids,
                        const oracle_mask* mask, double* out, int nthreads);
+/* The same pair with a fused pre-scale (a "fused variant", Section 3.6; the attention form
+ * softmax(scale * scores + mask)): z = scale * x, then the additive mask (not scaled) and the
+ * causal rule as above, then softmax (want_log 0) or log-softmax (want_log 1) of z.
+ * scale must be finite and > 0. */
+int oracle_softmax_scaled(const void* x, int dtype, int64_t rows, int64_t cols,
+                          int64_t x_stride, double scale, const int64_t* row_ids,
+                          const oracle_mask* mask, int want_log, double* out, int nthreads);
 int oracle_layernorm(const void* x, int dtype, int64_t rows, int64_t cols,
                      int64_t x_stride, const void* gamma, const void* beta,
                      double eps, double* out, int nthreads);

@@ -12,7 +12,9 @@ from golden_io import _mat, _vec, read_records
 from paper_2512_23424_b200 import workloads as wl
 
 GOLDEN = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
-RECORDS = read_records(os.path.join(GOLDEN, "fused_examples.txt"))
+ALL_RECORDS = read_records(os.path.join(GOLDEN, "fused_examples.txt"))
+RECORDS = [r for r in ALL_RECORDS if "res" in r]
+SCALED = [r for r in ALL_RECORDS if "scale" in r]
 OPS = ["layernorm", "rmsnorm"]
 
 
@@ -146,3 +148,85 @@ def test_brute_force_mpmath(seed):
         want = np.array([[float(v) for v in row] for row in my])
         assert np.max(np.abs(y - want) / np.maximum(1.0, np.abs(want))) < 1e-13
         assert np.array_equal(s, np.array([[float(v) for v in row] for row in ms]))
+
+
+# ---- softmax with a fused pre-scale ---------------------------------------------------------
+
+def mp_scaled_softmax(x, scale, additive, log):
+    """softmax / log-softmax of scale * x + additive, written independently at 40 digits."""
+    from mpmath import exp as mpexp, log as mplog
+    mp.dps = 40
+    out = []
+    for i, row in enumerate(x):
+        z = [mpf(float(scale)) * mpf(float(v)) + (mpf(float(additive[i % len(additive)][c])) if additive is not None else 0)
+             for c, v in enumerate(row)]
+        m = max(z)
+        s = sum(mpexp(v - m) for v in z)
+        out.append([(v - m) - mplog(s) if log else mpexp(v - m) / s for v in z])
+    return out
+
+
+@pytest.mark.parametrize("rec", SCALED, ids=[r["name"] for r in SCALED])
+def test_scaled_softmax_worked_examples(rec):
+    x = np.array(_mat(rec["x"]))
+    add = np.array(_mat(rec["additive"])) if "additive" in rec else None
+    scale, log = float(rec["scale"]), rec["op"] == "log_softmax"
+    want = np.array(_mat(rec["expect"]))
+    mine = np.array([[float(v) for v in r] for r in mp_scaled_softmax(x, scale, add, log)])
+    assert np.max(np.abs(mine - want)) <= 4e-16
+    mask = oracle.Mask(additive=add) if add is not None else None
+    got = oracle.softmax_scaled(x, scale, mask=mask, log=log)
+    assert np.max(np.abs(got - want)) <= 1e-15
+
+
+def test_scaled_softmax_identities_and_torch():
+    rng = np.random.default_rng(8)
+    x = rng.normal(0, 2, (9, 37))
+    for s in (0.125, 1.0, 0.08838834764831845, 3.0):
+        p = oracle.softmax_scaled(x, s)
+        lp = oracle.softmax_scaled(x, s, log=True)
+        # a power-of-two scale commutes exactly with the rounding of the input
+        if s in (0.125, 1.0):
+            assert np.array_equal(p, oracle.softmax(x * s))
+        assert np.max(np.abs(p.sum(axis=1) - 1)) < 1e-14
+        # shifting x does not matter; scaling the scale is the same as scaling x
+        assert np.max(np.abs(oracle.softmax_scaled(x + 5.0, s) - p)) < 1e-13
+        assert np.max(np.abs(oracle.softmax_scaled(2.0 * x, s / 2.0) - p)) < 1e-14
+        # two entries: a logistic of scale * difference
+        two = oracle.softmax_scaled(x[:, :2], s)
+        assert np.max(np.abs(two[:, 1] - 1.0 / (1.0 + np.exp(-s * (x[:, 1] - x[:, 0]))))) < 1e-14
+        # library second opinion, with and without an (unscaled) additive mask
+        tx = torch.from_numpy(x)
+        assert np.max(np.abs(p - torch.softmax(s * tx, dim=1).numpy())) < 1e-14
+        assert np.max(np.abs(lp - torch.log_softmax(s * tx, dim=1).numpy())) < 1e-13
+        a = rng.normal(0, 1, (3, 37))
+        a[1, 5] = -np.inf
+        pa = oracle.softmax_scaled(x, s, mask=oracle.Mask(additive=a))
+        want = torch.softmax(s * tx + torch.from_numpy(a)[torch.arange(9) % 3], dim=1).numpy()
+        assert np.max(np.abs(pa - want)) < 1e-14
+        # causal rows are the scaled softmax of their prefix
+        pc = oracle.softmax_scaled(x, s, mask=oracle.Mask(causal=True, causal_period=4))
+        for r in range(9):
+            live = r % 4 + 1
+            assert np.max(np.abs(pc[r, :live] - oracle.softmax_scaled(x[r:r + 1, :live], s)[0])) < 1e-14
+            assert np.all(pc[r, live:] == 0)
+    # the limit of a small scale is the uniform row, of a large one the arg-max indicator
+    assert np.max(np.abs(oracle.softmax_scaled(x, 1e-12) - 1.0 / 37)) < 1e-12
+    hot = oracle.softmax_scaled(x, 1e6)
+    assert np.array_equal(hot.argmax(axis=1), x.argmax(axis=1)) and np.all(hot.max(axis=1) == 1.0)
+    for bad in (0.0, -1.0, np.inf, np.nan):
+        with pytest.raises(ValueError):
+            oracle.softmax_scaled(x, bad)
+
+
+@pytest.mark.parametrize("seed", range(3))
+def test_scaled_softmax_brute_force(seed):
+    rng = np.random.default_rng(500 + seed)
+    rows, cols = int(rng.integers(1, 4)), int(rng.integers(1, 8))
+    x = rng.normal(0, 3, (rows, cols))
+    a = rng.normal(0, 1, (2, cols))
+    s = float(rng.uniform(0.05, 4.0))
+    for log in (False, True):
+        got = oracle.softmax_scaled(x, s, mask=oracle.Mask(additive=a), log=log)
+        want = np.array([[float(v) for v in r] for r in mp_scaled_softmax(x, s, a, log)])
+        assert np.max(np.abs(got - want) / np.maximum(1.0, np.abs(want))) < 1e-13
