@@ -165,6 +165,18 @@ akg_status akg_rowop_axis(akg_op op, const void* x, void* y, int64_t outer, int6
                           int64_t y_reduce_stride, akg_dtype dtype, const void* gamma, const void* beta,
                           float eps, void* stream);
 
+/* Softmax / log-softmax with a fused pre-scale (a "fused variant", Section 3.6; the paper
+ * gives no formula: this is the attention form softmax(scale * scores + mask)):
+ *   z[r,c] = scale * x[r,c] + additive[...]  (the additive mask is NOT scaled), causal rule as
+ *   for akg_softmax; y = softmax(z) if log_output == 0, log-softmax(z) otherwise.
+ * scale must be finite and > 0 (AKG_ERR_INVALID_ARG otherwise).  Everything else - masks,
+ * special rows, strides, alignment, in place, errors - as for akg_softmax / akg_log_softmax;
+ * scale == 1 gives bit-identical results to them.  The scale costs no extra instruction:
+ * the kernels fold it into the constant of the exponential. */
+akg_status akg_softmax_scaled(const void* x, void* y, int64_t rows, int64_t cols, int64_t x_row_stride,
+                              int64_t y_row_stride, akg_dtype dtype, float scale, const akg_mask* mask,
+                              int log_output, void* stream);
+
 /* Fused residual add + normalisation over the last axis (one of the "fused variants" of the
  * paper's operator benchmark, Section 3.6; the paper gives no formula, this is the usual
  * pre-norm residual step):

@@ -420,6 +420,29 @@ def log_softmax(x: torch.Tensor, out: Optional[torch.Tensor] = None, mask: Optio
     return _softmax_like("akg_log_softmax", x, out, mask, stream)
 
 
+def softmax_scaled(x: torch.Tensor, scale: float, out: Optional[torch.Tensor] = None, mask: Optional[Mask] = None,
+                   log: bool = False, stream=None) -> torch.Tensor:
+    """akg_softmax_scaled: softmax (log=False) or log-softmax (log=True) of scale * x + additive
+    mask under the causal rule, over the last axis of a 2-D CUDA tensor; scale > 0."""
+    rows, cols, xs = _matrix(x, "x")
+    if out is None:
+        out = torch.empty_like(x)
+    orow, ocol, ys = _matrix(out, "out")
+    if (orow, ocol) != (rows, cols) or out.dtype != x.dtype or out.device != x.device:
+        raise ValueError("out must match x in shape, dtype and device")
+    fn = lib().akg_softmax_scaled
+    if not fn.argtypes:
+        vp, i64, ci = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int
+        fn.argtypes = [vp, vp, i64, i64, i64, i64, ci, ctypes.c_float, vp, ci, vp]
+        fn.restype = ci
+    with torch.cuda.device(x.device):
+        st = fn(x.data_ptr(), out.data_ptr(), rows, cols, xs, ys, _dtype_code(x), float(scale),
+                ctypes.cast(ctypes.byref(mask), ctypes.c_void_p) if mask is not None else None, 1 if log else 0,
+                _stream(stream))
+    _check(st, "akg_softmax_scaled")
+    return out
+
+
 def layernorm(x: torch.Tensor, gamma: Optional[torch.Tensor] = None, beta: Optional[torch.Tensor] = None,
               eps: float = 1e-5, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
     """akg_layernorm over the last axis of a 2-D CUDA tensor."""

@@ -54,6 +54,7 @@ struct Call {
   float eps;
   void* stream;
   int64_t row_base = 0;      // global index of row 0 (host-buffer chunks)
+  float scale = 1.f;         // fused pre-scale of the softmax pair
 };
 
 akg_status validate(const Call& c, const char* name) {
@@ -351,6 +352,7 @@ akg_status run(const Call& c, const char* name) {
     }
   }
   p.status = nullptr;
+  p.scale = c.scale; p.inv_scale = 1.0f / c.scale; p.l2e = kLog2e * c.scale;   // scale 1: exactly log2(e)
   p.row_base = c.row_base;
   if (c.row_base != 0) { p.interleave = 0; if (p.add_mode == 2) p.add_mode = 0; }
 
@@ -777,6 +779,24 @@ extern "C" akg_status akg_rowop_axis(akg_op op, const void* x, void* y, int64_t 
   std::snprintf(akg::t_kernel, sizeof akg::t_kernel, "axis<%s,%s,t256,lc%d,grid%ux%u>", dtype == AKG_F32 ? "f32" : "bf16",
                 vec ? "vec" : "scalar", 1 << lc_shift, grid.x, grid.y);
   return AKG_OK;
+}
+
+// ---- softmax pair with a fused pre-scale -----------------------------------------------------
+extern "C" akg_status akg_softmax_scaled(const void* x, void* y, int64_t rows, int64_t cols, int64_t x_row_stride,
+                                         int64_t y_row_stride, akg_dtype dtype, float scale, const akg_mask* mask,
+                                         int log_output, void* stream) {
+  using namespace akg;
+  const char* name = "akg_softmax_scaled";
+  if (!(scale > 0.f) || std::isinf(scale)) {
+    t_error[0] = '\0';
+    return fail(AKG_ERR_INVALID_ARG, "%s: scale must be finite and > 0", name);
+  }
+  Call c;
+  c.op = log_output ? OP_LOG_SOFTMAX : OP_SOFTMAX;
+  c.x = x; c.y = y; c.rows = rows; c.cols = cols; c.xs = x_row_stride; c.ys = y_row_stride;
+  c.dtype = static_cast<int>(dtype); c.mask = mask; c.gamma = nullptr; c.beta = nullptr; c.eps = 0.f;
+  c.stream = stream; c.scale = scale;
+  return run(c, name);
 }
 
 // ---- fused residual add + LayerNorm / RMSNorm ----------------------------------------------

@@ -36,6 +36,11 @@ struct RowParams {
   long long rs;             // row stride of res
   void* sum;
   long long ss;             // row stride of sum
+  // fused pre-scale of the softmax pair: the operator runs on scale * x (+ additive mask).
+  // The kernels keep x unscaled (for scale > 0 the maximum sits at the same place) and fold the
+  // scale into the constant of the exponential: l2e = scale * log2(e).  The additive mask is
+  // taken as add * inv_scale; log-softmax multiplies its difference by scale at the end.
+  float l2e, scale, inv_scale;
 };
 
 // One call over a non-last axis: x[outer, reduce, inner], inner contiguous.
@@ -87,6 +92,8 @@ __device__ __forceinline__ float ex2_approx(float x) {
 }
 // e^(a - b) for a <= b (or NaN / inf operands, which propagate as IEEE says)
 __device__ __forceinline__ float exp_diff(float a, float b) { return ex2_approx((a - b) * kLog2e); }
+// e^(scale (a - b)) with l2e = scale * log2(e)
+__device__ __forceinline__ float exp_diff(float a, float b, float l2e) { return ex2_approx((a - b) * l2e); }
 
 // 128-bit streaming accesses: the row data is touched once, keep it out of L1.
 __device__ __forceinline__ uint4 ld_stream(const void* p) {
@@ -195,14 +202,14 @@ template <int OP> __device__ __forceinline__ Stat stat_identity() {
   return Stat{0.f, 0.f, 0.f};
 }
 
-template <int OP> __device__ __forceinline__ Stat stat_merge(const Stat& x, const Stat& y) {
+template <int OP> __device__ __forceinline__ Stat stat_merge(const Stat& x, const Stat& y, float l2e = kLog2e) {
   Stat r;
   if (OpTraits<OP>::kSoftmaxLike) {
     // (m, s) (+) (m', s') = (M, s e^(m-M) + s' e^(m'-M)); equal maxima (also both
     // -inf, or both +inf) take factor 1 so that no inf - inf is formed here.
     const float M = fmaxf(x.a, y.a);
-    const float fx = (x.a == M) ? 1.f : exp_diff(x.a, M);
-    const float fy = (y.a == M) ? 1.f : exp_diff(y.a, M);
+    const float fx = (x.a == M) ? 1.f : exp_diff(x.a, M, l2e);
+    const float fy = (y.a == M) ? 1.f : exp_diff(y.a, M, l2e);
     r.a = M; r.b = x.b * fx + y.b * fy; r.c = 0.f;
   } else if (OP == OP_LAYERNORM) {
     // Chan's pairwise update of (count, mean, M2)
@@ -224,9 +231,9 @@ template <int OP> __device__ __forceinline__ Stat stat_shfl_xor(const Stat& s, i
   return r;
 }
 
-template <int OP> __device__ __forceinline__ Stat warp_reduce(Stat s) {
+template <int OP> __device__ __forceinline__ Stat warp_reduce(Stat s, float l2e = kLog2e) {
 #pragma unroll
-  for (int m = 16; m >= 1; m >>= 1) s = stat_merge<OP>(s, stat_shfl_xor<OP>(s, m));
+  for (int m = 16; m >= 1; m >>= 1) s = stat_merge<OP>(s, stat_shfl_xor<OP>(s, m), l2e);
   return s;
 }
 
@@ -234,14 +241,14 @@ template <int OP> __device__ __forceinline__ Stat warp_reduce(Stat s) {
 // memory reserved for this call; callers alternate between two slot sets on
 // successive rows so one barrier per row is enough.  Every thread gets the result,
 // combined in the same order, hence bit-identical across the CTA.
-template <int OP, int NW> __device__ __forceinline__ Stat cta_reduce(Stat s, Stat* slots) {
-  s = warp_reduce<OP>(s);
+template <int OP, int NW> __device__ __forceinline__ Stat cta_reduce(Stat s, Stat* slots, float l2e = kLog2e) {
+  s = warp_reduce<OP>(s, l2e);
   if (NW == 1) return s;
   if ((threadIdx.x & 31) == 0) slots[threadIdx.x >> 5] = s;
   __syncthreads();
   Stat r = slots[0];
 #pragma unroll
-  for (int w = 1; w < NW; ++w) r = stat_merge<OP>(r, slots[w]);
+  for (int w = 1; w < NW; ++w) r = stat_merge<OP>(r, slots[w], l2e);
   return r;
 }
 
@@ -277,7 +284,7 @@ template <int OP> __device__ __forceinline__ RowScalars finalize(const Stat& s, 
 // For softmax the values are replaced by exp(z - m_local) so that the exponential
 // is evaluated once per element; the caller later scales by exp(m_local - M) / S.
 template <int OP, int N>
-__device__ __forceinline__ Stat tile_stats(float (&v)[N], int n_valid, float& m_local) {
+__device__ __forceinline__ Stat tile_stats(float (&v)[N], int n_valid, float& m_local, float l2e = kLog2e) {
   Stat s = stat_identity<OP>();
   m_local = 0.f;
   if (OpTraits<OP>::kSoftmaxLike) {
@@ -288,7 +295,7 @@ __device__ __forceinline__ Stat tile_stats(float (&v)[N], int n_valid, float& m_
     float acc = 0.f;
 #pragma unroll
     for (int i = 0; i < N; ++i) {
-      const float e = exp_diff(v[i], ms);
+      const float e = exp_diff(v[i], ms, l2e);
       acc += e;
       if (OP == OP_SOFTMAX) v[i] = e;
     }

@@ -12,9 +12,10 @@ namespace akg {
 
 // Apply the row scalars to one element (z already masked).
 template <int OP>
-__device__ __forceinline__ float apply_one(float z, const RowScalars& rs, float scale, float g, float b) {
+__device__ __forceinline__ float apply_one(float z, const RowScalars& rs, float scale, float g, float b,
+                                           float pre = 1.f) {
   if (OP == OP_SOFTMAX) return z * scale;                      // z holds exp(z - m_local)
-  if (OP == OP_LOG_SOFTMAX) return rs.dead ? kNegInf : (z - rs.p) - rs.q;
+  if (OP == OP_LOG_SOFTMAX) return rs.dead ? kNegInf : fmaf(z - rs.p, pre, -rs.q);   // pre: the fused pre-scale
   if (OP == OP_LAYERNORM) return (z - rs.p) * rs.q * g + b;
   return z * rs.q * g;
 }
@@ -90,7 +91,7 @@ __global__ void __launch_bounds__(THREADS) reg_kernel(const RowParams p) {
             float a[EPV];
             E::unpack(ld_stream(ar + static_cast<long long>(idx) * EPV), a);
 #pragma unroll
-            for (int j = 0; j < EPV; ++j) v[k * EPV + j] += a[j];
+            for (int j = 0; j < EPV; ++j) v[k * EPV + j] = fmaf(a[j], p.inv_scale, v[k * EPV + j]);
           }
         }
       }
@@ -109,11 +110,11 @@ __global__ void __launch_bounds__(THREADS) reg_kernel(const RowParams p) {
 
     // ---- statistics: thread tile -> warp -> CTA
     float m_local;
-    Stat st = tile_stats<OP, N>(v, n_valid, m_local);
-    st = (NW > 1) ? cta_reduce<OP, (NW > 1 ? NW : 1)>(st, red[parity]) : warp_reduce<OP>(st);
+    Stat st = tile_stats<OP, N>(v, n_valid, m_local, p.l2e);
+    st = (NW > 1) ? cta_reduce<OP, (NW > 1 ? NW : 1)>(st, red[parity], p.l2e) : warp_reduce<OP>(st, p.l2e);
     const RowScalars rs = finalize<OP>(st, p.cols, p.eps);
     float scale = 0.f;
-    if (OP == OP_SOFTMAX) scale = (m_local == st.a) ? rs.q : exp_diff(m_local, st.a) * rs.q;
+    if (OP == OP_SOFTMAX) scale = (m_local == st.a) ? rs.q : exp_diff(m_local, st.a, p.l2e) * rs.q;
 
     // ---- normalise and store
     const float fill = SM ? masked_fill<OP>(rs) : 0.f;
@@ -135,7 +136,7 @@ __global__ void __launch_bounds__(THREADS) reg_kernel(const RowParams p) {
 #pragma unroll
           for (int j = 0; j < EPV; ++j) {
             const bool masked = SM && (idx * EPV + j >= live);
-            o[j] = masked ? fill : apply_one<OP>(v[k * EPV + j], rs, scale, g[j], b[j]);
+            o[j] = masked ? fill : apply_one<OP>(v[k * EPV + j], rs, scale, g[j], b[j], p.scale);
           }
         } else {
 #pragma unroll
@@ -178,10 +179,10 @@ __global__ void __launch_bounds__(THREADS) stream_kernel(const RowParams p) {
       float z = E::load1(xr, c);
       if (!SM && rr != nullptr) z += E::load1(rr, c);
       if (SM) {
-        if (ar != nullptr) z += E::load1(ar, c);
+        if (ar != nullptr) z = fmaf(E::load1(ar, c), p.inv_scale, z);
         const float mn = fmaxf(st.a, z);
         const float ms = (mn == kNegInf) ? 0.f : mn;
-        st.b = st.b * exp_diff(st.a, ms) + exp_diff(z, ms);
+        st.b = st.b * exp_diff(st.a, ms, p.l2e) + exp_diff(z, ms, p.l2e);
         st.a = mn;
       } else if (OP == OP_LAYERNORM) {
         st.a += 1.f;
@@ -192,7 +193,7 @@ __global__ void __launch_bounds__(THREADS) stream_kernel(const RowParams p) {
         st.a += z * z;
       }
     }
-    st = cta_reduce<OP, NW>(st, red[parity]);
+    st = cta_reduce<OP, NW>(st, red[parity], p.l2e);
     const RowScalars rs = finalize<OP>(st, p.cols, p.eps);
     const float fill = SM ? masked_fill<OP>(rs) : 0.f;
 
@@ -200,10 +201,10 @@ __global__ void __launch_bounds__(THREADS) stream_kernel(const RowParams p) {
       float o;
       if (c < live) {
         float z = E::load1(xr, c);
-        if (SM && ar != nullptr) z += E::load1(ar, c);
+        if (SM && ar != nullptr) z = fmaf(E::load1(ar, c), p.inv_scale, z);
         if (OP == OP_SOFTMAX) {
           // exp(z - M) / S; a dead row (no live entry) has q = 0 and p = 0
-          o = exp_diff(z, rs.p) * rs.q;
+          o = exp_diff(z, rs.p, p.l2e) * rs.q;
         } else {
           if (!SM && rr != nullptr) {
             z += E::load1(rr, c);
@@ -211,7 +212,7 @@ __global__ void __launch_bounds__(THREADS) stream_kernel(const RowParams p) {
           }
           const float g = (!SM && p.gamma != nullptr) ? E::load1(p.gamma, c) : 1.f;
           const float b = (OP == OP_LAYERNORM && p.beta != nullptr) ? E::load1(p.beta, c) : 0.f;
-          o = apply_one<OP>(z, rs, 0.f, g, b);
+          o = apply_one<OP>(z, rs, 0.f, g, b, p.scale);
         }
       } else {
         o = fill;

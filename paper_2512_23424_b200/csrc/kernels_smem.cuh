@@ -21,16 +21,16 @@ namespace akg {
 
 // Fold one vector of EPV (masked) values into the running thread statistics.
 template <int OP, int EPV>
-__device__ __forceinline__ void fold_vector(Stat& st, const float (&z)[EPV]) {
+__device__ __forceinline__ void fold_vector(Stat& st, const float (&z)[EPV], float l2e = kLog2e) {
   if (OpTraits<OP>::kSoftmaxLike) {
     float mv = z[0];
 #pragma unroll
     for (int j = 1; j < EPV; ++j) mv = fmaxf(mv, z[j]);
     const float mn = fmaxf(st.a, mv);
     const float ms = (mn == kNegInf) ? 0.f : mn;
-    float acc = st.b * exp_diff(st.a, ms);
+    float acc = st.b * exp_diff(st.a, ms, l2e);
 #pragma unroll
-    for (int j = 0; j < EPV; ++j) acc += exp_diff(z[j], ms);
+    for (int j = 0; j < EPV; ++j) acc += exp_diff(z[j], ms, l2e);
     st.a = mn; st.b = acc;
   } else if (OP == OP_LAYERNORM) {
     float sum = 0.f;
@@ -50,7 +50,7 @@ __device__ __forceinline__ void fold_vector(Stat& st, const float (&z)[EPV]) {
 // Fold a block of four vectors: one running-maximum update and one rescale for the block
 // (softmax pair); the normalisations fold the vectors one after the other.
 template <int OP, int EPV>
-__device__ __forceinline__ void fold_block(Stat& st, const float (&z)[4][EPV]) {
+__device__ __forceinline__ void fold_block(Stat& st, const float (&z)[4][EPV], float l2e = kLog2e) {
   if (OpTraits<OP>::kSoftmaxLike) {
     float mv = z[0][0];
 #pragma unroll
@@ -59,15 +59,15 @@ __device__ __forceinline__ void fold_block(Stat& st, const float (&z)[4][EPV]) {
       for (int j = 0; j < EPV; ++j) mv = fmaxf(mv, z[u][j]);
     const float mn = fmaxf(st.a, mv);
     const float ms = (mn == kNegInf) ? 0.f : mn;
-    float acc[4] = {st.b * exp_diff(st.a, ms), 0.f, 0.f, 0.f};
+    float acc[4] = {st.b * exp_diff(st.a, ms, l2e), 0.f, 0.f, 0.f};
 #pragma unroll
     for (int u = 0; u < 4; ++u)
 #pragma unroll
-      for (int j = 0; j < EPV; ++j) acc[u] += exp_diff(z[u][j], ms);
+      for (int j = 0; j < EPV; ++j) acc[u] += exp_diff(z[u][j], ms, l2e);
     st.a = mn; st.b = (acc[0] + acc[1]) + (acc[2] + acc[3]);
   } else {
 #pragma unroll
-    for (int u = 0; u < 4; ++u) fold_vector<OP, EPV>(st, z[u]);
+    for (int u = 0; u < 4; ++u) fold_vector<OP, EPV>(st, z[u], l2e);
   }
 }
 
@@ -163,7 +163,7 @@ __global__ void __launch_bounds__(THREADS) smem_kernel(const RowParams p, const 
         float z[4][EPV];
 #pragma unroll
         for (int u = 0; u < 4; ++u) E::unpack(lds128(buf + static_cast<uint32_t>(v + u * THREADS) * 16u), z[u]);
-        fold_block<OP, EPV>(st, z);
+        fold_block<OP, EPV>(st, z, p.l2e);
       }
     }
     for (; v < lv; v += THREADS) {
@@ -175,16 +175,16 @@ __global__ void __launch_bounds__(THREADS) smem_kernel(const RowParams p, const 
           float a[EPV];
           E::unpack(ld_stream(ar + c0), a);
 #pragma unroll
-          for (int j = 0; j < EPV; ++j) z[j] += a[j];
+          for (int j = 0; j < EPV; ++j) z[j] = fmaf(a[j], p.inv_scale, z[j]);
         }
         if (c0 + EPV > live) {
 #pragma unroll
           for (int j = 0; j < EPV; ++j) if (c0 + j >= live) z[j] = kNegInf;
         }
       }
-      fold_vector<OP, EPV>(st, z);
+      fold_vector<OP, EPV>(st, z, p.l2e);
     }
-    st = cta_reduce<OP, NW>(st, red + par * NW);
+    st = cta_reduce<OP, NW>(st, red + par * NW, p.l2e);
 
     // ---- combine across the cluster through distributed shared memory
     if (cs > 1) {
@@ -197,7 +197,7 @@ __global__ void __launch_bounds__(THREADS) smem_kernel(const RowParams p, const 
       cluster_arrive();
       cluster_wait();
       Stat r = peers[par * kMaxCluster];
-      for (uint32_t k = 1; k < cs; ++k) r = stat_merge<OP>(r, peers[par * kMaxCluster + k]);
+      for (uint32_t k = 1; k < cs; ++k) r = stat_merge<OP>(r, peers[par * kMaxCluster + k], p.l2e);
       st = r;
     }
     const RowScalars rs = finalize<OP>(st, p.cols, p.eps);
@@ -224,8 +224,8 @@ __global__ void __launch_bounds__(THREADS) smem_kernel(const RowParams p, const 
           }
 #pragma unroll
           for (int j = 0; j < EPV; ++j) {
-            if (OP == OP_SOFTMAX) o[j] = exp_diff(z[u][j], rs.p) * rs.q;
-            else o[j] = apply_one<OP>(z[u][j], rs, 0.f, ga[j], be[j]);
+            if (OP == OP_SOFTMAX) o[j] = exp_diff(z[u][j], rs.p, p.l2e) * rs.q;
+            else o[j] = apply_one<OP>(z[u][j], rs, 0.f, ga[j], be[j], p.scale);
           }
           st_stream(yr + static_cast<long long>(v + u * THREADS) * EPV, E::pack(o));
         }
@@ -245,7 +245,7 @@ __global__ void __launch_bounds__(THREADS) smem_kernel(const RowParams p, const 
             float a[EPV];
             E::unpack(ld_stream(ar + c0), a);
 #pragma unroll
-            for (int j = 0; j < EPV; ++j) z[j] += a[j];
+            for (int j = 0; j < EPV; ++j) z[j] = fmaf(a[j], p.inv_scale, z[j]);
           }
         } else {
           if (p.gamma != nullptr) E::unpack(ld_cached(reinterpret_cast<const T*>(p.gamma) + c0), ga);
@@ -255,8 +255,8 @@ __global__ void __launch_bounds__(THREADS) smem_kernel(const RowParams p, const 
 #pragma unroll
         for (int j = 0; j < EPV; ++j) {
           if (SM && c0 + j >= live) o[j] = fill;
-          else if (OP == OP_SOFTMAX) o[j] = exp_diff(z[j], rs.p) * rs.q;
-          else o[j] = apply_one<OP>(z[j], rs, 0.f, ga[j], be[j]);
+          else if (OP == OP_SOFTMAX) o[j] = exp_diff(z[j], rs.p, p.l2e) * rs.q;
+          else o[j] = apply_one<OP>(z[j], rs, 0.f, ga[j], be[j], p.scale);
         }
       } else {
 #pragma unroll

@@ -57,7 +57,7 @@ __device__ __forceinline__ void softmax_row(const RowParams& p, long long row, i
         float a[EPV];
         E::unpack(ld_stream(ar + k * G * EPV), a);
 #pragma unroll
-        for (int j = 0; j < EPV; ++j) v[k][j] += a[j];
+        for (int j = 0; j < EPV; ++j) v[k][j] = fmaf(a[j], p.inv_scale, v[k][j]);
       }
       if (k == NK - 1 && ragged && tg + k * G == live_vecs - 1) {
 #pragma unroll
@@ -77,12 +77,13 @@ __device__ __forceinline__ void softmax_row(const RowParams& p, long long row, i
   // bf16 storage: one fused multiply-add forms the exponent (its rounding, below 1e-5
   // relative, is far inside the 2^-9 of the bf16 result); fp32 keeps the exact difference
   constexpr bool kFusedExponent = (sizeof(T) == 2);
-  const float neg_m_l2 = -m_ws * kLog2e;
+  const float l2e = p.l2e;                                  // scale * log2(e): the pre-scale costs nothing
+  const float neg_m_l2 = -m_ws * l2e;
 #pragma unroll
   for (int k = 0; k < NK; ++k) {
 #pragma unroll
     for (int j = 0; j < EPV; ++j) {
-      const float e = kFusedExponent ? ex2_approx(fmaf(v[k][j], kLog2e, neg_m_l2)) : exp_diff(v[k][j], m_ws);
+      const float e = kFusedExponent ? ex2_approx(fmaf(v[k][j], l2e, neg_m_l2)) : exp_diff(v[k][j], m_ws, l2e);
       s_t += e;
       if (OP == OP_SOFTMAX) v[k][j] = e;
     }
@@ -103,10 +104,10 @@ __device__ __forceinline__ void softmax_row(const RowParams& p, long long row, i
 #pragma unroll
     for (int m = 1; m < NW && m < 32; m <<= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, m));
     const float Ms = (M == kNegInf) ? 0.f : M;
-    S = sw * ((mw == M) ? 1.f : exp_diff(mw, Ms));          // equal maxima (also +-inf): factor 1
+    S = sw * ((mw == M) ? 1.f : exp_diff(mw, Ms, l2e));          // equal maxima (also +-inf): factor 1
 #pragma unroll
     for (int m = 1; m < NW && m < 32; m <<= 1) S += __shfl_xor_sync(0xffffffffu, S, m);
-    my_factor = (m_w == M) ? 1.f : exp_diff(m_w, Ms);
+    my_factor = (m_w == M) ? 1.f : exp_diff(m_w, Ms, l2e);
   }
 
   const bool dead = (M == kNegInf) && !(S != S);   // only NaN / -inf entries: a NaN row, not a dead one
@@ -137,7 +138,7 @@ __device__ __forceinline__ void softmax_row(const RowParams& p, long long row, i
 #pragma unroll
       for (int j = 0; j < EPV; ++j) {
         if (OP == OP_SOFTMAX) o[j] = v[k < NK ? k : 0][j] * scale;
-        else o[j] = dead ? kNegInf : (v[k < NK ? k : 0][j] - M) - lse_l;
+        else o[j] = dead ? kNegInf : fmaf(v[k < NK ? k : 0][j] - M, p.scale, -lse_l);
       }
       if (k == NK - 1 && ragged && idx == live_vecs - 1) {
 #pragma unroll

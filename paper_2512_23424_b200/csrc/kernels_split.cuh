@@ -86,7 +86,7 @@ split_kernel(const RowParams p, const int slice_vecs) {
           float z[4][EPV];
 #pragma unroll
           for (int u = 0; u < 4; ++u) E::unpack(raw[4 * h + u], z[u]);
-          fold_block<OP, EPV>(st, z);
+          fold_block<OP, EPV>(st, z, p.l2e);
         }
       }
       for (; v + 3 * THREADS < lv; v += 4 * THREADS, px += 4 * THREADS) {
@@ -96,7 +96,7 @@ split_kernel(const RowParams p, const int slice_vecs) {
         float z[4][EPV];
 #pragma unroll
         for (int u = 0; u < 4; ++u) E::unpack(raw[u], z[u]);
-        fold_block<OP, EPV>(st, z);
+        fold_block<OP, EPV>(st, z, p.l2e);
       }
     }
     for (; v < lv; v += THREADS) {
@@ -108,16 +108,16 @@ split_kernel(const RowParams p, const int slice_vecs) {
           float a[EPV];
           E::unpack(ld_hint(ar + static_cast<long long>(v) * EPV, keep), a);
 #pragma unroll
-          for (int j = 0; j < EPV; ++j) z[j] += a[j];
+          for (int j = 0; j < EPV; ++j) z[j] = fmaf(a[j], p.inv_scale, z[j]);
         }
         if (c0 + EPV > live) {
 #pragma unroll
           for (int j = 0; j < EPV; ++j) if (c0 + j >= live) z[j] = kNegInf;
         }
       }
-      fold_vector<OP, EPV>(st, z);
+      fold_vector<OP, EPV>(st, z, p.l2e);
     }
-    st = cta_reduce<OP, NW>(st, red[par]);
+    st = cta_reduce<OP, NW>(st, red[par], p.l2e);
 
     if (cs > 1) {
       if (threadIdx.x < cs) {
@@ -129,7 +129,7 @@ split_kernel(const RowParams p, const int slice_vecs) {
       cluster_arrive();
       cluster_wait();
       Stat r = peers[par][0];
-      for (uint32_t k = 1; k < cs; ++k) r = stat_merge<OP>(r, peers[par][k]);
+      for (uint32_t k = 1; k < cs; ++k) r = stat_merge<OP>(r, peers[par][k], p.l2e);
       st = r;
     }
     const RowScalars rs = finalize<OP>(st, p.cols, p.eps);
@@ -158,8 +158,8 @@ split_kernel(const RowParams p, const int slice_vecs) {
           }
 #pragma unroll
           for (int j = 0; j < EPV; ++j) {
-            if (OP == OP_SOFTMAX) o[j] = exp_diff(z[j], rs.p) * rs.q;
-            else o[j] = apply_one<OP>(z[j], rs, 0.f, ga[j], be[j]);
+            if (OP == OP_SOFTMAX) o[j] = exp_diff(z[j], rs.p, p.l2e) * rs.q;
+            else o[j] = apply_one<OP>(z[j], rs, 0.f, ga[j], be[j], p.scale);
           }
           st_stream(py + u * THREADS, E::pack(o));
         }
@@ -179,7 +179,7 @@ split_kernel(const RowParams p, const int slice_vecs) {
             float a[EPV];
             E::unpack(ld_hint(ar + static_cast<long long>(v) * EPV, drop), a);
 #pragma unroll
-            for (int j = 0; j < EPV; ++j) z[j] += a[j];
+            for (int j = 0; j < EPV; ++j) z[j] = fmaf(a[j], p.inv_scale, z[j]);
           }
         } else {
           if (p.gamma != nullptr) E::unpack(ld_cached(reinterpret_cast<const T*>(p.gamma) + c0), ga);
@@ -189,8 +189,8 @@ split_kernel(const RowParams p, const int slice_vecs) {
 #pragma unroll
         for (int j = 0; j < EPV; ++j) {
           if (SM && c0 + j >= live) o[j] = fill;
-          else if (OP == OP_SOFTMAX) o[j] = exp_diff(z[j], rs.p) * rs.q;
-          else o[j] = apply_one<OP>(z[j], rs, 0.f, ga[j], be[j]);
+          else if (OP == OP_SOFTMAX) o[j] = exp_diff(z[j], rs.p, p.l2e) * rs.q;
+          else o[j] = apply_one<OP>(z[j], rs, 0.f, ga[j], be[j], p.scale);
         }
       } else {
 #pragma unroll
