@@ -313,3 +313,17 @@ def make_act(name: str, rows: Optional[int] = None, seed_offset: int = 0) -> Act
     if dtype == BF16:
         x = f32_to_bf16_bits(x)
     return ActWorkload(name, act, dtype, x)
+
+
+def make_scaled_causal(rows: Optional[int] = None, seed_offset: int = 0) -> Workload:
+    """Configuration 5 with its 1/sqrt(128) moved out of the input and into the call: x holds
+    the unscaled bf16 scores N(0, 1); `extra["scale"]` is the pre-scale to pass to the fused
+    softmax (same seed, shape and causal period as configuration 5)."""
+    k = 5
+    op, dtype, r, c = _SHAPES[k]
+    name = "scaled_causal_softmax_bf16_32x4096x4096"
+    r = r if rows is None else min(r, rows)
+    s_x = np.random.SeedSequence(k - 1 + 1000 * seed_offset).spawn(4)[0]
+    x = _normal_f32(np.random.Generator(np.random.PCG64(s_x)), r, c)
+    return Workload(name, op, dtype, r, c, f32_to_bf16_bits(x), causal_period=4096,
+                    extra={"scale": float(np.float32(1.0 / np.sqrt(128.0)))})
