@@ -254,6 +254,39 @@ def act_mul(act: str, x, nthreads: int = 1):
     return out
 
 
+def argreduce(op: str, x, nthreads: int = 1) -> np.ndarray:
+    """"argmax" / "argmin" over the last axis (Section 3.6): int64 [rows]; first index on ties,
+    NaN counts as the extreme."""
+    x, rows, cols, stride = _as2d(x)
+    out = np.empty((rows,), dtype=np.int64)
+    L = lib()
+    if not L.oracle_argreduce.argtypes:
+        i64, vp, ci = ctypes.c_int64, ctypes.c_void_p, ctypes.c_int
+        L.oracle_argreduce.argtypes = [ci, vp, ci, i64, i64, i64, vp, ci]
+        L.oracle_argreduce.restype = ci
+    rc = L.oracle_argreduce({"argmax": 0, "argmin": 1}[op], x.ctypes.data, _dtype_code(x), rows, cols, stride,
+                            out.ctypes.data, int(nthreads))
+    if rc != 0:
+        raise ValueError("oracle_argreduce: malformed argument")
+    return out
+
+
+def cumulative(op: str, x, nthreads: int = 1) -> np.ndarray:
+    """"cumsum" / "cumprod" along the last axis (Section 3.6), inclusive: float64 [rows, cols]."""
+    x, rows, cols, stride = _as2d(x)
+    out = np.empty((rows, cols), dtype=np.float64)
+    L = lib()
+    if not L.oracle_cumulative.argtypes:
+        i64, vp, ci = ctypes.c_int64, ctypes.c_void_p, ctypes.c_int
+        L.oracle_cumulative.argtypes = [ci, vp, ci, i64, i64, i64, ctypes.POINTER(ctypes.c_double), ci]
+        L.oracle_cumulative.restype = ci
+    rc = L.oracle_cumulative({"cumsum": 0, "cumprod": 1}[op], x.ctypes.data, _dtype_code(x), rows, cols, stride,
+                             _dptr(out), int(nthreads))
+    if rc != 0:
+        raise ValueError("oracle_cumulative: malformed argument")
+    return out
+
+
 AXIS_OPS = {"softmax": 0, "log_softmax": 1, "layernorm": 2, "rmsnorm": 3}
 
 

@@ -366,6 +366,60 @@ int oracle_act_mul(int act, const void* x, int dtype, int64_t rows, int64_t d, i
   return 0;
 }
 
+/* ---- other reduction-category operators of Section 3.6: arg-max / arg-min, cumulative --- */
+
+/* Does a beat b as the arg-max (want_min 0) or arg-min (want_min 1) candidate?  NaN beats every
+ * number (and another NaN does not beat it); equal values (-0 == +0 included) do not beat. */
+static int arg_beats(double a, double b, int want_min) {
+  if (isnan(b)) return 0;
+  if (isnan(a)) return 1;
+  return want_min ? (a < b) : (a > b);
+}
+
+int oracle_argreduce(int want_min, const void* x, int dtype, int64_t rows, int64_t cols, int64_t x_stride,
+                     int64_t* out, int nthreads) {
+  if (rows < 0 || cols < 0) return 1;
+  if (dtype != ORACLE_F32 && dtype != ORACLE_BF16 && dtype != ORACLE_F64) return 1;
+  int t = use_threads(nthreads);
+  if (rows == 0) return 0;
+  if (cols == 0 || !x || !out || x_stride < cols) return 1;      /* an empty row has no arg-max */
+#pragma omp parallel for schedule(static) num_threads(t)
+  for (int64_t i = 0; i < rows; ++i) {
+    int64_t best = 0;
+    double bv = widen(x, dtype, i * x_stride);
+    for (int64_t c = 1; c < cols; ++c) {
+      double v = widen(x, dtype, i * x_stride + c);
+      if (arg_beats(v, bv, want_min)) { bv = v; best = c; }     /* strict: the first of equals stays */
+    }
+    out[i] = best;
+  }
+  return 0;
+}
+
+int oracle_cumulative(int want_prod, const void* x, int dtype, int64_t rows, int64_t cols, int64_t x_stride,
+                      double* out, int nthreads) {
+  if (bad_shape(x, dtype, rows, cols, x_stride, out)) return 1;
+  int t = use_threads(nthreads);
+  if (rows == 0 || cols == 0) return 0;
+#pragma omp parallel for schedule(static) num_threads(t)
+  for (int64_t i = 0; i < rows; ++i) {
+    if (want_prod) {
+      double p = 1.0;
+      for (int64_t c = 0; c < cols; ++c) { p *= widen(x, dtype, i * x_stride + c); out[i * cols + c] = p; }
+    } else {
+      nsum s = {0.0, 0.0};                                      /* compensated running sum */
+      double plain = 0.0;                                       /* carries inf / NaN as the arithmetic says */
+      for (int64_t c = 0; c < cols; ++c) {
+        double v = widen(x, dtype, i * x_stride + c);
+        nsum_add(&s, v);
+        plain += v;
+        out[i * cols + c] = isfinite(plain) ? nsum_get(&s) : plain;
+      }
+    }
+  }
+  return 0;
+}
+
 /* ---- the paper's verifier criterion (Section 3.2.3, Eq. 2-3) ------------------ */
 
 double oracle_verifier_fraction(const double* gen, const double* ref, int64_t n,

@@ -134,6 +134,20 @@ double oracle_activation(int act, double a);
 int oracle_act_mul(int act, const void* x, int dtype, int64_t rows, int64_t d, int64_t x_stride,
                    double* out, int nthreads);
 
+/* Arg-max / arg-min over the last axis ("argmax/argmin" of the reduction category, Section
+ * 3.6).  out[i] = the smallest column index at which row i attains its maximum (want_min 0) or
+ * minimum (want_min 1).  Comparisons are made on the stored values, exactly: -0 and +0 are
+ * equal; a NaN counts as the extreme for both (the first NaN of a row wins), as in numpy and
+ * torch.  cols == 0 with rows > 0 is an error (no index exists).  Returns 0, or 1. */
+int oracle_argreduce(int want_min, const void* x, int dtype, int64_t rows, int64_t cols, int64_t x_stride,
+                     int64_t* out, int nthreads);
+
+/* Cumulative sum (want_prod 0) or product (want_prod 1) along the last axis ("cumulative
+ * operations", Section 3.6): out[i, c] = x[i, 0] (+ or *) ... (+ or *) x[i, c], inclusive,
+ * in double (the sum compensated).  out: rows x cols doubles, contiguous.  Returns 0, or 1. */
+int oracle_cumulative(int want_prod, const void* x, int dtype, int64_t rows, int64_t cols, int64_t x_stride,
+                      double* out, int nthreads);
+
 /* The paper's correctness criterion (Section 3.2.3, Eq. 2-3): element error is
  * |gen-ref|/|ref| when |ref| > eps_switch, else |gen-ref|; returns the fraction
  * of elements whose error exceeds tau (the kernel passes iff that fraction is
