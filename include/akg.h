@@ -216,6 +216,26 @@ typedef enum akg_act { AKG_ACT_SILU = 0, AKG_ACT_GELU = 1, AKG_ACT_GELU_TANH = 2
 akg_status akg_act_mul(akg_act act, const void* x, void* y, int64_t rows, int64_t d,
                        int64_t x_row_stride, int64_t y_row_stride, akg_dtype dtype, void* stream);
 
+/* Arg-max (want_min == 0) or arg-min (want_min == 1) over the last axis ("argmax/argmin" of the
+ * reduction category, Section 3.6).  x: DEVICE matrix [rows, cols] of `dtype`; index_out: DEVICE
+ * vector of `rows` int64.  index_out[r] = the smallest column at which row r attains its maximum
+ * (minimum).  Values are compared exactly as stored: -0 equals +0, and a NaN counts as the extreme
+ * for both operators (the first NaN of a row wins), as in numpy and torch.  cols == 0 with
+ * rows > 0 is AKG_ERR_INVALID_ARG.  Reads every element once; any alignment. */
+akg_status akg_argreduce(int want_min, const void* x, int64_t* index_out, int64_t rows, int64_t cols,
+                         int64_t x_row_stride, akg_dtype dtype, void* stream);
+
+/* Cumulative sum (want_prod == 0) or product (want_prod == 1) along the last axis ("cumulative
+ * operations" of the reduction category, Section 3.6), inclusive:
+ *   y[r, c] = x[r, 0] (+ or *) ... (+ or *) x[r, c].
+ * One pass (each element read once, written once), fp32 arithmetic, one rounding at the store.
+ * The partial results are combined as a tree (vector, warp, CTA, chunk), not left to right: the
+ * rounding differs from a sequential loop by the usual O(log cols) ulps of the running magnitude,
+ * and a product whose sequential partials stay finite may overflow in a tree partial.  In place
+ * (y == x, equal strides) is allowed; any alignment. */
+akg_status akg_cumulative(int want_prod, const void* x, void* y, int64_t rows, int64_t cols,
+                          int64_t x_row_stride, int64_t y_row_stride, akg_dtype dtype, void* stream);
+
 /* Size of the staging area built into the library (see akg_rowop_host_static). */
 #define AKG_STATIC_STAGING_BYTES (16u << 20)
 

@@ -353,6 +353,61 @@ def act_mul(act: str, x: torch.Tensor, out: Optional[torch.Tensor] = None, strea
     return out
 
 
+def _argreduce(want_min: int, x: torch.Tensor, out, stream):
+    rows, cols, xs = _matrix(x, "x")
+    if out is None:
+        out = torch.empty((rows,), dtype=torch.int64, device=x.device)
+    if out.shape != (rows,) or out.dtype != torch.int64 or out.device != x.device or not out.is_contiguous():
+        raise ValueError("out must be a contiguous int64 vector of `rows` entries on x's device")
+    fn = lib().akg_argreduce
+    if not fn.argtypes:
+        vp, i64, ci = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int
+        fn.argtypes = [ci, vp, vp, i64, i64, i64, ci, vp]
+        fn.restype = ci
+    with torch.cuda.device(x.device):
+        st = fn(want_min, x.data_ptr(), out.data_ptr(), rows, cols, xs, _dtype_code(x), _stream(stream))
+    _check(st, "akg_argreduce")
+    return out
+
+
+def argmax(x: torch.Tensor, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """akg_argreduce(0): first index of the row maximum (NaN counts as the maximum), int64 [rows]."""
+    return _argreduce(0, x, out, stream)
+
+
+def argmin(x: torch.Tensor, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """akg_argreduce(1): first index of the row minimum (NaN counts as the minimum), int64 [rows]."""
+    return _argreduce(1, x, out, stream)
+
+
+def _cumulative(want_prod: int, x: torch.Tensor, out, stream):
+    rows, cols, xs = _matrix(x, "x")
+    if out is None:
+        out = torch.empty_like(x)
+    orow, ocol, ys = _matrix(out, "out")
+    if (orow, ocol) != (rows, cols) or out.dtype != x.dtype or out.device != x.device:
+        raise ValueError("out must match x in shape, dtype and device")
+    fn = lib().akg_cumulative
+    if not fn.argtypes:
+        vp, i64, ci = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int
+        fn.argtypes = [ci, vp, vp, i64, i64, i64, i64, ci, vp]
+        fn.restype = ci
+    with torch.cuda.device(x.device):
+        st = fn(want_prod, x.data_ptr(), out.data_ptr(), rows, cols, xs, ys, _dtype_code(x), _stream(stream))
+    _check(st, "akg_cumulative")
+    return out
+
+
+def cumsum(x: torch.Tensor, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """akg_cumulative(0): inclusive running sum along the last axis of a 2-D CUDA tensor."""
+    return _cumulative(0, x, out, stream)
+
+
+def cumprod(x: torch.Tensor, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """akg_cumulative(1): inclusive running product along the last axis of a 2-D CUDA tensor."""
+    return _cumulative(1, x, out, stream)
+
+
 STATIC_STAGING_BYTES = 16 << 20
 
 

@@ -937,6 +937,67 @@ extern "C" akg_status akg_act_mul(akg_act act, const void* x, void* y, int64_t r
   return AKG_OK;
 }
 
+// ---- arg-max / arg-min and cumulative sum / product over the last axis -------------------------
+extern "C" akg_status akg_argreduce(int want_min, const void* x, int64_t* index_out, int64_t rows, int64_t cols,
+                                    int64_t x_row_stride, akg_dtype dtype, void* stream) {
+  using namespace akg;
+  const char* name = "akg_argreduce";
+  t_error[0] = '\0';
+  if (want_min != 0 && want_min != 1) return fail(AKG_ERR_INVALID_ARG, "%s: want_min must be 0 or 1", name);
+  if (dtype != AKG_F32 && dtype != AKG_BF16) return fail(AKG_ERR_INVALID_ARG, "%s: unknown dtype", name);
+  if (rows < 0 || cols < 0) return fail(AKG_ERR_INVALID_ARG, "%s: negative rows or cols", name);
+  if (rows == 0) return AKG_OK;
+  if (cols == 0) return fail(AKG_ERR_INVALID_ARG, "%s: an empty row has no arg-max", name);
+  if (x == nullptr || index_out == nullptr) return fail(AKG_ERR_INVALID_ARG, "%s: x and index_out must not be NULL", name);
+  if (x_row_stride < cols) return fail(AKG_ERR_INVALID_ARG, "%s: row stride smaller than cols", name);
+  if (cols > INT_MAX / 2) return fail(AKG_ERR_UNSUPPORTED, "%s: cols above 2^30 - 1", name);
+  const int64_t es = (dtype == AKG_F32) ? 4 : 2;
+  if (static_cast<long double>(rows) * x_row_stride * es > 9.0e18L)
+    return fail(AKG_ERR_INVALID_ARG, "%s: rows * stride overflows", name);
+  const bool vec = g_forced_variant.load() != V_STREAM && cols % (16 / es) == 0 && aligned16(x) &&
+                   (rows == 1 || (x_row_stride * es) % 16 == 0);
+  const bool warp_rows = cols * es <= 4096;
+  const int64_t ctas = warp_rows ? (rows + 7) / 8 : rows;
+  const int cap = g_tune_grid_cap.load();
+  const unsigned grid = static_cast<unsigned>(std::min<int64_t>(ctas, cap > 0 ? cap : INT_MAX));
+  const cudaError_t err = launch_argreduce(want_min == 1, static_cast<int>(dtype), vec, warp_rows, x,
+                                           reinterpret_cast<long long*>(index_out), rows, cols, x_row_stride, grid,
+                                           g_tune_pdl.load() == 2 ? 0 : 1, static_cast<cudaStream_t>(stream));
+  if (err != cudaSuccess) return cuda_fail(name, err);
+  std::snprintf(t_kernel, sizeof t_kernel, "arg<%s,%s,%s,g%d,t256,grid%u>", want_min ? "min" : "max",
+                dtype == AKG_F32 ? "f32" : "bf16", vec ? "vec" : "scalar", warp_rows ? 32 : 256, grid);
+  return AKG_OK;
+}
+
+extern "C" akg_status akg_cumulative(int want_prod, const void* x, void* y, int64_t rows, int64_t cols,
+                                     int64_t x_row_stride, int64_t y_row_stride, akg_dtype dtype, void* stream) {
+  using namespace akg;
+  const char* name = "akg_cumulative";
+  t_error[0] = '\0';
+  if (want_prod != 0 && want_prod != 1) return fail(AKG_ERR_INVALID_ARG, "%s: want_prod must be 0 or 1", name);
+  Call c;
+  c.op = OP_SOFTMAX; c.x = x; c.y = y; c.rows = rows; c.cols = cols; c.xs = x_row_stride; c.ys = y_row_stride;
+  c.dtype = static_cast<int>(dtype); c.mask = nullptr; c.gamma = nullptr; c.beta = nullptr; c.eps = 0.f; c.stream = stream;
+  const akg_status st = validate(c, name);                  // shapes, strides, NULLs, overlap (in place allowed)
+  if (st != AKG_OK) return st;
+  if (rows == 0 || cols == 0) return AKG_OK;
+  const int64_t es = (dtype == AKG_F32) ? 4 : 2;
+  const bool vec = g_forced_variant.load() != V_STREAM && vector_ok(c);
+  const int64_t nvec = vec ? cols / (16 / es) : cols;
+  const int u = scan_unroll();
+  int threads = 32;
+  while (threads < 256 && static_cast<int64_t>(threads) * u < nvec) threads <<= 1;
+  const int cap = g_tune_grid_cap.load();
+  const unsigned grid = static_cast<unsigned>(std::min<int64_t>(rows, cap > 0 ? cap : INT_MAX));
+  const cudaError_t err = launch_cumulative(want_prod == 1, static_cast<int>(dtype), vec, x, y, rows, cols, x_row_stride,
+                                            y_row_stride, grid, threads, g_tune_pdl.load() == 2 ? 0 : 1,
+                                            static_cast<cudaStream_t>(stream));
+  if (err != cudaSuccess) return cuda_fail(name, err);
+  std::snprintf(t_kernel, sizeof t_kernel, "scan<%s,%s,%s,t%d,grid%u>", want_prod ? "prod" : "sum",
+                dtype == AKG_F32 ? "f32" : "bf16", vec ? "vec" : "scalar", threads, grid);
+  return AKG_OK;
+}
+
 // ---- host buffers without any allocation ---------------------------------------------------
 // akg_rowop_host needs a device staging area from its caller.  Some callers have no way to
 // get one: a plug-in that is handed host buffers and a stream but no allocator, a service

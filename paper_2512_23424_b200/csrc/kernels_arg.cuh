@@ -1,0 +1,142 @@
+// Arg-max / arg-min over the last axis ("argmax/argmin" of the reduction category, Section 3.6).
+// out[r] = the smallest column index at which row r attains its maximum (minimum); values are
+// compared exactly as stored (-0 == +0); a NaN counts as the extreme for both, the first NaN wins.
+//
+// Read-only and HBM-bound, so the loop does as little as it can per element and never branches: a
+// NaN-propagating max (min) over the 8 or 4 values of a vector, and a select that keeps the
+// better of that and the thread's best so far together with the vector's index.  The position
+// inside the winning vector is looked up once per thread and row.  Threads merge through a 64-bit key (order-preserving image of
+// the value in the high word, inverted index in the low word), whose maximum is the winner with
+// the lowest index.  G threads own a row: a warp (short rows, several rows per CTA) or the CTA.
+#pragma once
+
+#include "common.cuh"
+
+namespace akg {
+
+struct ArgParams {
+  const void* x;
+  long long* out;
+  long long rows, cols, xs;
+};
+
+template <bool MIN> __device__ __forceinline__ float nan_ext(float a, float b) {
+  float r;
+  if (MIN) asm("min.NaN.f32 %0, %1, %2;" : "=f"(r) : "f"(a), "f"(b));
+  else asm("max.NaN.f32 %0, %1, %2;" : "=f"(r) : "f"(a), "f"(b));
+  return r;
+}
+
+// does v beat the best so far?  (NaN beats every number; nothing beats a NaN; equals do not beat)
+template <bool MIN> __device__ __forceinline__ bool arg_beats(float v, float best) {
+  if (best != best) return false;
+  if (v != v) return true;
+  return MIN ? (v < best) : (v > best);
+}
+
+// order-preserving 32-bit image: larger = better candidate; NaN is the largest; -0 maps like +0
+template <bool MIN> __device__ __forceinline__ uint32_t arg_key(float v) {
+  if (v != v) return 0xffffffffu;
+  uint32_t b = __float_as_uint(v + 0.0f);
+  b = (b & 0x80000000u) ? ~b : (b | 0x80000000u);            // ascending with the value
+  return MIN ? ~b : b;
+}
+
+template <bool MIN, typename T, int G, int THREADS, bool VEC>
+__global__ void __launch_bounds__(THREADS) arg_kernel(const ArgParams p) {
+  pdl_prologue();
+  using E = Elem<T>;
+  constexpr int EPV = VEC ? E::EPV : 1;
+  constexpr int RPC = THREADS / G;
+  constexpr int NW = G / 32;
+  constexpr int U = 4;
+  __shared__ unsigned long long red[THREADS / 32];
+  const int tg = threadIdx.x % G;
+  const int grp = threadIdx.x / G;
+  const long long nvec = p.cols / EPV;                          // VEC: cols is a multiple of EPV
+
+  for (long long rb = static_cast<long long>(blockIdx.x) * RPC; rb < p.rows; rb += static_cast<long long>(gridDim.x) * RPC) {
+    const long long row = rb + grp;
+    const bool have = row < p.rows;
+    const T* xr = reinterpret_cast<const T*>(p.x) + (have ? row : 0) * p.xs;
+    // the extreme of nothing: every first value beats it, and it loses every merge
+    float best = MIN ? __int_as_float(0x7f800000) : kNegInf;
+    long long bvec = -1;                                        // vector (element when !VEC) holding it
+    bool seen = false;
+
+    // per vector: its extreme (NaN-propagating), and a branch-free "take it if it improves"
+    auto visit = [&](const float (&v)[EPV], long long vec_index) {
+      float ext = v[0];
+#pragma unroll
+      for (int j = 1; j < EPV; ++j) ext = nan_ext<MIN>(ext, v[j]);
+      const bool take = !seen || arg_beats<MIN>(ext, best);
+      best = take ? ext : best;
+      bvec = take ? vec_index : bvec;
+      seen = true;
+    };
+
+    if (have) {
+      long long i = tg;
+      if (VEC) {
+        for (; i + (U - 1) * G < nvec; i += U * G) {
+          uint4 raw[U];
+#pragma unroll
+          for (int u = 0; u < U; ++u) raw[u] = ld_stream(xr + (i + u * G) * EPV);
+#pragma unroll
+          for (int u = 0; u < U; ++u) {
+            float v[E::EPV];
+            E::unpack(raw[u], v);
+            float w[EPV];
+#pragma unroll
+            for (int j = 0; j < EPV; ++j) w[j] = v[j];
+            visit(w, i + u * G);
+          }
+        }
+      }
+      for (; i < nvec; i += G) {
+        float w[EPV];
+        if (VEC) {
+          float v[E::EPV];
+          E::unpack(ld_stream(xr + i * EPV), v);
+#pragma unroll
+          for (int j = 0; j < EPV; ++j) w[j] = v[j];
+        } else {
+          w[0] = E::load1(xr, i);
+        }
+        visit(w, i);
+      }
+    }
+    // the position inside the winning vector: its first element equal to the extreme (first NaN
+    // if the extreme is NaN); one more load per thread and row, served by L2
+    long long bidx = bvec * EPV;
+    if (VEC && seen) {
+      float v[E::EPV];
+      E::unpack(ld_stream(xr + bvec * EPV), v);
+      int pos = EPV - 1;
+#pragma unroll
+      for (int j = EPV - 1; j >= 0; --j)
+        if ((best != best) ? (v[j] != v[j]) : (v[j] == best)) pos = j;
+      bidx += pos;
+    }
+    // merge: the largest (key, inverted index) pair is the winner with the lowest index
+    unsigned long long key = 0ull;
+    if (seen) key = (static_cast<unsigned long long>(arg_key<MIN>(best)) << 32) |
+                    (0xffffffffull - static_cast<unsigned long long>(bidx));
+#pragma unroll
+    for (int m = 16; m >= 1; m >>= 1) {
+      const unsigned long long o = __shfl_xor_sync(0xffffffffu, key, m);
+      key = o > key ? o : key;
+    }
+    if (NW > 1) {
+      __syncthreads();                                          // red is reused by the next row
+      if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = key;
+      __syncthreads();
+      key = red[0];
+#pragma unroll
+      for (int w = 1; w < NW; ++w) key = red[w] > key ? red[w] : key;
+    }
+    if (have && tg == 0) p.out[row] = static_cast<long long>(0xffffffffull - (key & 0xffffffffull));
+  }
+}
+
+}  // namespace akg

@@ -54,6 +54,17 @@ int act_mul_unroll();
 cudaError_t launch_act_mul(int act, int dtype, bool vec, const ActParams& p, dim3 grid, int threads, int pdl,
                            cudaStream_t stream);
 
+// Arg-max / arg-min and cumulative sum / product over the last axis (op_scan.cu).
+// warp_rows: a warp per row (eight rows per CTA of 256), else a CTA per row.  Cumulative: a CTA of
+// `threads` (a multiple of 32, at most 256) per row, chunks of scan_unroll() * threads vectors.
+int scan_unroll();
+cudaError_t launch_argreduce(bool want_min, int dtype, bool vec, bool warp_rows, const void* x, long long* out,
+                             long long rows, long long cols, long long xs, unsigned grid, int pdl,
+                             cudaStream_t stream);
+cudaError_t launch_cumulative(bool want_prod, int dtype, bool vec, const void* x, void* y, long long rows,
+                              long long cols, long long xs, long long ys, unsigned grid, int threads, int pdl,
+                              cudaStream_t stream);
+
 extern template cudaError_t launch_op<OP_SOFTMAX>(const LaunchPlan&, int, const RowParams&, cudaStream_t);
 extern template cudaError_t launch_op<OP_LOG_SOFTMAX>(const LaunchPlan&, int, const RowParams&, cudaStream_t);
 extern template cudaError_t launch_op<OP_LAYERNORM>(const LaunchPlan&, int, const RowParams&, cudaStream_t);

@@ -1,0 +1,67 @@
+// Arg-max / arg-min and cumulative sum / product over the last axis: kernels and launchers.
+#include "kernels_arg.cuh"
+#include "kernels_scan.cuh"
+#include "launch.cuh"
+
+namespace akg {
+namespace {
+
+template <typename K, typename P>
+cudaError_t launch_1d(K kernel, const P& p, unsigned grid, int threads, int pdl, cudaStream_t s) {
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(threads);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = s;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, p);
+}
+
+template <bool MIN, typename T>
+cudaError_t launch_arg_t(bool vec, bool warp_rows, const ArgParams& p, unsigned grid, int pdl, cudaStream_t s) {
+  if (vec) return warp_rows ? launch_1d(arg_kernel<MIN, T, 32, 256, true>, p, grid, 256, pdl, s)
+                            : launch_1d(arg_kernel<MIN, T, 256, 256, true>, p, grid, 256, pdl, s);
+  return warp_rows ? launch_1d(arg_kernel<MIN, T, 32, 256, false>, p, grid, 256, pdl, s)
+                   : launch_1d(arg_kernel<MIN, T, 256, 256, false>, p, grid, 256, pdl, s);
+}
+
+template <bool PROD, typename T>
+cudaError_t launch_scan_t(bool vec, const ScanParams& p, unsigned grid, int threads, int pdl, cudaStream_t s) {
+  return vec ? launch_1d(scan_kernel<PROD, T, true>, p, grid, threads, pdl, s)
+             : launch_1d(scan_kernel<PROD, T, false>, p, grid, threads, pdl, s);
+}
+
+}  // namespace
+
+int scan_unroll() { return kScanU; }
+
+cudaError_t launch_argreduce(bool want_min, int dtype, bool vec, bool warp_rows, const void* x, long long* out,
+                             long long rows, long long cols, long long xs, unsigned grid, int pdl,
+                             cudaStream_t stream) {
+  ArgParams p;
+  p.x = x; p.out = out; p.rows = rows; p.cols = cols; p.xs = xs;
+  if (dtype == DT_F32)
+    return want_min ? launch_arg_t<true, float>(vec, warp_rows, p, grid, pdl, stream)
+                    : launch_arg_t<false, float>(vec, warp_rows, p, grid, pdl, stream);
+  return want_min ? launch_arg_t<true, __nv_bfloat16>(vec, warp_rows, p, grid, pdl, stream)
+                  : launch_arg_t<false, __nv_bfloat16>(vec, warp_rows, p, grid, pdl, stream);
+}
+
+cudaError_t launch_cumulative(bool want_prod, int dtype, bool vec, const void* x, void* y, long long rows,
+                              long long cols, long long xs, long long ys, unsigned grid, int threads, int pdl,
+                              cudaStream_t stream) {
+  if (threads < 32 || threads > 32 * kScanMaxWarps || threads % 32) return cudaErrorInvalidValue;
+  ScanParams p;
+  p.x = x; p.y = y; p.rows = rows; p.cols = cols; p.xs = xs; p.ys = ys;
+  if (dtype == DT_F32)
+    return want_prod ? launch_scan_t<true, float>(vec, p, grid, threads, pdl, stream)
+                     : launch_scan_t<false, float>(vec, p, grid, threads, pdl, stream);
+  return want_prod ? launch_scan_t<true, __nv_bfloat16>(vec, p, grid, threads, pdl, stream)
+                   : launch_scan_t<false, __nv_bfloat16>(vec, p, grid, threads, pdl, stream);
+}
+
+}  // namespace akg
