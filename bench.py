@@ -9,7 +9,8 @@ HBM; successive steps rotate over four buffer pairs so the working set (512 MiB)
 exceeds L2.  The one JSON line printed by rank 0 carries the headline number,
 the same figure for every configuration (`per_config`) and for the operators
 over a non-last axis (`axis_rows`) and the fused residual add + normalisation
-(`fused_rows`) and the gated activations (`act_rows`), the roofline fraction, the end-to-end figure
+(`fused_rows`), the gated activations (`act_rows`) and arg-max / cumulative operators
+(`reduction_rows`), the roofline fraction, the end-to-end figure
 with host buffers, and the fp64 CPU oracle's timing.
 
 With N > 1 (launched by torch.distributed.run) every rank runs the same
@@ -235,7 +236,7 @@ class ActDeviceWorkload:
 
 
 def pairs_for(w) -> int:
-    one = (w.algorithmic_bytes() if isinstance(w, (wl.AxisWorkload, wl.FusedWorkload, wl.ActWorkload))
+    one = (w.algorithmic_bytes() if isinstance(w, (wl.AxisWorkload, wl.FusedWorkload, wl.ActWorkload, wl.ReductionWorkload))
            else 2 * w.rows * w.cols * w.itemsize)
     if one >= 3 * L2_BYTES:
         return 1
@@ -526,6 +527,37 @@ def run_ours(args):
             del dwa, wa
             torch.cuda.empty_cache()
         line["act_rows"] = acts
+        # arg-max / arg-min and cumulative sum / product over the last axis
+        reds = []
+        for name in wl.REDUCTION_CONFIGS:
+            wr = wl.make_reduction(name)
+            fn = getattr(binding, wr.op)
+            n_buf = pairs_for(wr)
+            if wr.dtype == wl.F32:
+                x0 = torch.from_numpy(wr.x).cuda()
+            else:
+                x0 = torch.from_numpy(wr.x.view(np.int16)).cuda().view(torch.bfloat16)
+            rxs = [x0] + [x0.clone() for _ in range(n_buf - 1)]
+            routs = [fn(x) for x in rxs]
+
+            class _Red:
+                i = 0
+
+                def launch(self):
+                    k = self.i % len(rxs)
+                    self.i += 1
+                    return fn(rxs[k], out=routs[k])
+
+            _Red.torch = torch
+            reps = max(10, min(100, 100 * args.steps // 1000))
+            sr = time_launches(_Red(), reps, 5) / reps
+            br = wr.algorithmic_bytes()
+            reds.append({"workload": name, "kernel": binding.last_kernel(), "us": sr * 1e6, "gbs": br / sr / 1e9,
+                         "frac_measured": br / sr / 1e9 / peak, "algorithmic_bytes": br, "launches": reps,
+                         "rows_per_s": wr.x.shape[0] / sr, "traffic": profiled_traffic(name)})
+            del rxs, routs, x0, wr
+            torch.cuda.empty_cache()
+        line["reduction_rows"] = reds
     if rank == 0 and world == 1:
         line["cpu_baseline"] = oracle_baseline(w)
     assert binding.device_status() == 0, "a device-side bounded wait expired"

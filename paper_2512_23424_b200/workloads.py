@@ -327,3 +327,48 @@ def make_scaled_causal(rows: Optional[int] = None, seed_offset: int = 0) -> Work
     x = _normal_f32(np.random.Generator(np.random.PCG64(s_x)), r, c)
     return Workload(name, op, dtype, r, c, f32_to_bf16_bits(x), causal_period=4096,
                     extra={"scale": float(np.float32(1.0 / np.sqrt(128.0)))})
+
+
+# ---------------------------------------------------------------------------------------------
+# Other reduction-category operators of Section 3.6 (arg-max / arg-min, cumulative sum /
+# product) on the shapes of configurations 2 and 3 and on a vocabulary-like axis.
+# ---------------------------------------------------------------------------------------------
+REDUCTION_CONFIGS: Dict[str, tuple] = {
+    "argmax_f32_16384x8192": ("argmax", F32, 16384, 8192),
+    "argmax_bf16_16384x8192": ("argmax", BF16, 16384, 8192),
+    "argmin_f32_1024x131072": ("argmin", F32, 1024, 131072),
+    "cumsum_f32_16384x8192": ("cumsum", F32, 16384, 8192),
+    "cumsum_bf16_16384x8192": ("cumsum", BF16, 16384, 8192),
+    "cumprod_f32_16384x8192": ("cumprod", F32, 16384, 8192),
+}
+
+
+@dataclass
+class ReductionWorkload:
+    name: str
+    op: str                            # argmax | argmin | cumsum | cumprod
+    dtype: int
+    x: np.ndarray                      # [rows, cols]; float32, or uint16 bf16 bits
+
+    @property
+    def itemsize(self) -> int:
+        return 4 if self.dtype == F32 else 2
+
+    def algorithmic_bytes(self) -> int:
+        """Every element read once; an int64 index per row, or every element written once."""
+        if self.op in ("argmax", "argmin"):
+            return self.x.size * self.itemsize + self.x.shape[0] * 8
+        return 2 * self.x.size * self.itemsize
+
+
+def make_reduction(name: str, rows: Optional[int] = None, seed_offset: int = 0) -> ReductionWorkload:
+    op, dtype, r, c = REDUCTION_CONFIGS[name]
+    r = r if rows is None else min(r, rows)
+    seed = 400 + sorted(REDUCTION_CONFIGS).index(name) + 1000 * seed_offset
+    rx = np.random.Generator(np.random.PCG64(np.random.SeedSequence(seed)))
+    x = _normal_f32(rx, r, c)
+    if op == "cumprod":                                 # factors near one keep the product in range
+        x = np.float32(1.0) + np.float32(0.002) * x
+    if dtype == BF16:
+        x = f32_to_bf16_bits(x)
+    return ReductionWorkload(name, op, dtype, x)
