@@ -45,7 +45,10 @@ typedef enum akg_status {
   AKG_ERR_DEVICE_TIMEOUT = 4
 } akg_status;
 
-typedef enum akg_dtype { AKG_F32 = 0, AKG_BF16 = 1 } akg_dtype;
+/* Storage types.  AKG_F16 (IEEE half, the paper's float16 regime of Section 4.1) behaves like
+ * AKG_BF16 everywhere: widened once, fp32 arithmetic, one round-to-nearest-even at the store
+ * (a result beyond 65504 becomes an infinity, as the conversion says). */
+typedef enum akg_dtype { AKG_F32 = 0, AKG_BF16 = 1, AKG_F16 = 2 } akg_dtype;
 
 /* Kernel families (for akg_set_variant; AKG_VARIANT_AUTO lets the library choose).
  *   STREAM  scalar loads, any alignment, statistics pass + second read of the row

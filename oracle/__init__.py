@@ -24,7 +24,7 @@ _SRC = os.path.join(_HERE, "oracle.c")
 _HDR = os.path.join(_HERE, "oracle.h")
 _LIB = os.path.join(_HERE, "liboracle.so")
 
-F32, BF16, F64 = 0, 1, 2
+F32, BF16, F64, F16 = 0, 1, 2, 3
 
 
 def build(force: bool = False) -> str:
@@ -97,6 +97,8 @@ def _dtype_code(a: np.ndarray) -> int:
         return BF16
     if a.dtype == np.float64:
         return F64
+    if a.dtype == np.float16:
+        return F16
     raise TypeError(f"oracle: unsupported storage dtype {a.dtype}")
 
 
@@ -329,6 +331,18 @@ def verifier_fraction(gen, ref, eps_switch: float = 1e-8, tau: float = 1e-3) -> 
         raise ValueError("verifier_fraction: size mismatch")
     return float(lib().oracle_verifier_fraction(_dptr(g), _dptr(r), g.size,
                                                 float(eps_switch), float(tau)))
+
+
+def widen(a: np.ndarray) -> np.ndarray:
+    """The exact values of a stored array (float32, float16, float64, or uint16 bf16 bits)."""
+    a = np.ascontiguousarray(a)
+    out = np.empty(a.shape, dtype=np.float64)
+    L = lib()
+    L.oracle_widen.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.POINTER(ctypes.c_double)]
+    L.oracle_widen.restype = ctypes.c_int
+    if L.oracle_widen(a.ctypes.data, _dtype_code(a), a.size, _dptr(out)) != 0:
+        raise ValueError("oracle_widen: malformed argument")
+    return out
 
 
 def last_threads() -> int:

@@ -32,11 +32,31 @@ static double nsum_get(const nsum* a) { return a->s + a->c; }
 static double widen(const void* base, int dtype, int64_t idx) {
   if (dtype == ORACLE_F32) return (double)((const float*)base)[idx];
   if (dtype == ORACLE_F64) return ((const double*)base)[idx];
+  if (dtype == ORACLE_F16) {
+    /* IEEE binary16: 1 sign, 5 exponent (bias 15), 10 fraction bits */
+    uint16_t h = ((const uint16_t*)base)[idx];
+    int e = (h >> 10) & 31, m = h & 1023;
+    double v;
+    if (e == 0) v = ldexp((double)m, -24);                       /* zero and subnormals */
+    else if (e == 31) v = m ? NAN : INFINITY;
+    else v = ldexp(1.0 + (double)m / 1024.0, e - 15);
+    return (h & 0x8000) ? -v : v;
+  }
   /* bf16: the 16 stored bits are the high half of an IEEE binary32 */
   uint32_t bits = (uint32_t)((const uint16_t*)base)[idx] << 16;
   float f;
   memcpy(&f, &bits, sizeof f);
   return (double)f;
+}
+
+static int bad_dtype(int dtype) {
+  return dtype != ORACLE_F32 && dtype != ORACLE_BF16 && dtype != ORACLE_F64 && dtype != ORACLE_F16;
+}
+
+int oracle_widen(const void* base, int dtype, int64_t n, double* out) {
+  if (bad_dtype(dtype) || n < 0 || (n > 0 && (!base || !out))) return 1;
+  for (int64_t i = 0; i < n; ++i) out[i] = widen(base, dtype, i);
+  return 0;
 }
 
 /* ---- softmax family --------------------------------------------------------- */
@@ -118,7 +138,7 @@ static int bad_shape(const void* x, int dtype, int64_t rows, int64_t cols,
   if (rows == 0 || cols == 0) return 0;
   if (!x || !out) return 1;
   if (stride < cols) return 1;
-  if (dtype != ORACLE_F32 && dtype != ORACLE_BF16 && dtype != ORACLE_F64) return 1;
+  if (bad_dtype(dtype)) return 1;
   return 0;
 }
 
@@ -273,7 +293,7 @@ int oracle_rowop_axis(int op, const void* x, int dtype, int64_t outer, int64_t r
                       double eps, double* out, int nthreads) {
   if (op < 0 || op > 3) return 1;
   if (outer < 0 || reduce < 0 || inner < 0) return 1;
-  if (dtype != ORACLE_F32 && dtype != ORACLE_BF16 && dtype != ORACLE_F64) return 1;
+  if (bad_dtype(dtype)) return 1;
   if ((op == 2 || op == 3) && !(eps >= 0.0)) return 1;
   int t = use_threads(nthreads);
   if (outer == 0 || reduce == 0 || inner == 0) return 0;
@@ -355,7 +375,7 @@ int oracle_act_mul(int act, const void* x, int dtype, int64_t rows, int64_t d, i
                    double* out, int nthreads) {
   if (act < 0 || act > 2) return 1;
   if (rows < 0 || d < 0) return 1;
-  if (dtype != ORACLE_F32 && dtype != ORACLE_BF16 && dtype != ORACLE_F64) return 1;
+  if (bad_dtype(dtype)) return 1;
   int t = use_threads(nthreads);
   if (rows == 0 || d == 0) return 0;
   if (!x || !out || x_stride < 2 * d) return 1;
@@ -379,7 +399,7 @@ static int arg_beats(double a, double b, int want_min) {
 int oracle_argreduce(int want_min, const void* x, int dtype, int64_t rows, int64_t cols, int64_t x_stride,
                      int64_t* out, int nthreads) {
   if (rows < 0 || cols < 0) return 1;
-  if (dtype != ORACLE_F32 && dtype != ORACLE_BF16 && dtype != ORACLE_F64) return 1;
+  if (bad_dtype(dtype)) return 1;
   int t = use_threads(nthreads);
   if (rows == 0) return 0;
   if (cols == 0 || !x || !out || x_stride < cols) return 1;      /* an empty row has no arg-max */

@@ -29,7 +29,7 @@ extern "C" {
 #endif
 
 /* storage types of the input arrays */
-enum { ORACLE_F32 = 0, ORACLE_BF16 = 1, ORACLE_F64 = 2 };
+enum { ORACLE_F32 = 0, ORACLE_BF16 = 1, ORACLE_F64 = 2, ORACLE_F16 = 3 };  /* F16: IEEE binary16 */
 
 /* Mask descriptor (NULL pointer = no mask).
  *   z[r,c] = x[r,c] + additive[(r % add_rows) * add_row_stride + c]   (if additive != NULL)
@@ -147,6 +147,9 @@ int oracle_argreduce(int want_min, const void* x, int dtype, int64_t rows, int64
  * in double (the sum compensated).  out: rows x cols doubles, contiguous.  Returns 0, or 1. */
 int oracle_cumulative(int want_prod, const void* x, int dtype, int64_t rows, int64_t cols, int64_t x_stride,
                       double* out, int nthreads);
+
+/* The exact value of n stored elements as doubles (how every driver reads its input). */
+int oracle_widen(const void* base, int dtype, int64_t n, double* out);
 
 /* The paper's correctness criterion (Section 3.2.3, Eq. 2-3): element error is
  * |gen-ref|/|ref| when |ref| > eps_switch, else |gen-ref|; returns the fraction

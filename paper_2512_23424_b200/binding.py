@@ -15,7 +15,7 @@ import torch
 from . import build as _build
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_DEVICE_TIMEOUT = range(5)
-F32, BF16 = 0, 1
+F32, BF16, F16 = 0, 1, 2
 VARIANT_AUTO, VARIANT_STREAM, VARIANT_REG, VARIANT_TMA, VARIANT_CLUSTER = range(5)
 VARIANTS = {"auto": 0, "stream": 1, "reg": 2, "tma": 3, "cluster": 4}
 
@@ -117,7 +117,9 @@ def _dtype_code(t: torch.Tensor) -> int:
         return F32
     if t.dtype == torch.bfloat16:
         return BF16
-    raise TypeError(f"unsupported dtype {t.dtype}: the library handles float32 and bfloat16")
+    if t.dtype == torch.float16:
+        return F16
+    raise TypeError(f"unsupported dtype {t.dtype}: the library handles float32, bfloat16 and float16")
 
 
 def _matrix(t: torch.Tensor, what: str):

@@ -44,6 +44,9 @@ akg_status fail(akg_status st, const char* fmt, const char* a = "", long long b 
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+bool valid_dtype(int dtype) { return dtype == AKG_F32 || dtype == AKG_BF16 || dtype == AKG_F16; }
+const char* dtype_name(int dtype) { return dtype == AKG_F32 ? "f32" : (dtype == AKG_F16 ? "f16" : "bf16"); }
+
 struct Call {
   int op;
   const void* x; void* y;
@@ -58,7 +61,7 @@ struct Call {
 };
 
 akg_status validate(const Call& c, const char* name) {
-  if (c.dtype != AKG_F32 && c.dtype != AKG_BF16) return fail(AKG_ERR_INVALID_ARG, "%s: unknown dtype", name);
+  if (!valid_dtype(c.dtype)) return fail(AKG_ERR_INVALID_ARG, "%s: unknown dtype", name);
   if (c.rows < 0 || c.cols < 0) return fail(AKG_ERR_INVALID_ARG, "%s: negative rows or cols", name);
   const bool norm = (c.op == OP_LAYERNORM || c.op == OP_RMSNORM);
   if (norm && !(c.eps >= 0.f)) return fail(AKG_ERR_INVALID_ARG, "%s: eps must be >= 0 and not NaN", name);
@@ -368,7 +371,7 @@ akg_status run(const Call& c, const char* name) {
   //   every other row that fits a CTA's registers -> register kernel
   //   longer aligned rows -> two-pass split cluster kernel (second pass from L2)
   //   anything unaligned -> scalar stream kernel
-  if (forced == V_AUTO && vec && c.dtype == AKG_BF16 && c.op == OP_RMSNORM &&
+  if (forced == V_AUTO && vec && c.dtype != AKG_F32 && c.op == OP_RMSNORM &&
       c.rows >= 2048 && c.cols >= 2048 && g_tune_tma_mode.load() != 2) {
     planned = plan_ring(c, &plan);
     if (planned) {
@@ -408,7 +411,7 @@ akg_status run(const Call& c, const char* name) {
     std::snprintf(t_error, sizeof t_error, "%s: launch failed: %s", name, cudaGetErrorString(err));
     return AKG_ERR_CUDA;
   }
-  const char* dt = (c.dtype == AKG_F32) ? "f32" : "bf16";
+  const char* dt = dtype_name(c.dtype);
   if (plan.variant == V_REG)
     std::snprintf(t_kernel, sizeof t_kernel, "reg<%s,g%d,t%d,v%d%s>", dt, plan.group, plan.threads, plan.vpt,
                   plan.mode == 2 ? ",flex"
@@ -585,7 +588,7 @@ akg_status akg_rowop_host(akg_op op, const void* x_host, void* y_host, int64_t r
 }
 
 size_t akg_host_workspace_bytes(int64_t rows, int64_t cols, akg_dtype dtype, int has_gamma, int has_beta) {
-  if (rows <= 0 || cols <= 0 || (dtype != AKG_F32 && dtype != AKG_BF16)) return 0;
+  if (rows <= 0 || cols <= 0 || !valid_dtype(dtype)) return 0;
   const size_t row_bytes = static_cast<size_t>(cols) * ((dtype == AKG_F32) ? 4 : 2);
   size_t chunk_rows = (static_cast<size_t>(rows) + 11) / 12;
   const size_t min_rows = ((size_t(4) << 20) + row_bytes - 1) / row_bytes;
@@ -668,7 +671,7 @@ extern "C" akg_status akg_rowop_axis(akg_op op, const void* x, void* y, int64_t 
   const char* name = "akg_rowop_axis";
   akg::t_error[0] = '\0';
   if (op < AKG_OP_SOFTMAX || op > AKG_OP_RMSNORM) return akg::fail(AKG_ERR_INVALID_ARG, "%s: unknown operator", name);
-  if (dtype != AKG_F32 && dtype != AKG_BF16) return akg::fail(AKG_ERR_INVALID_ARG, "%s: unknown dtype", name);
+  if (!valid_dtype(dtype)) return akg::fail(AKG_ERR_INVALID_ARG, "%s: unknown dtype", name);
   if (outer < 0 || reduce < 0 || inner < 0) return akg::fail(AKG_ERR_INVALID_ARG, "%s: negative size", name);
   const bool norm = (op == AKG_OP_LAYERNORM || op == AKG_OP_RMSNORM);
   if (norm && (!(eps >= 0.f) || std::isinf(eps)))
@@ -750,7 +753,7 @@ extern "C" akg_status akg_rowop_axis(akg_op op, const void* x, void* y, int64_t 
                                                  static_cast<cudaStream_t>(stream));
     if (err != cudaSuccess) return akg::cuda_fail(name, err);
     std::snprintf(akg::t_kernel, sizeof akg::t_kernel, "axis_reg<%s,%s,r%d,nf%d,nc%d,grid%ux%u>",
-                  dtype == AKG_F32 ? "f32" : "bf16", mode == 1 ? "vec" : (mode == 2 ? "wide8" : "scalar"), r_best,
+                  dtype_name(dtype), mode == 1 ? "vec" : (mode == 2 ? "wide8" : "scalar"), r_best,
                   nf_best, static_cast<int>(nc), grid.x, grid.y);
     return AKG_OK;
   }
@@ -776,7 +779,7 @@ extern "C" akg_status akg_rowop_axis(akg_op op, const void* x, void* y, int64_t 
   const cudaError_t err = akg::launch_axis(static_cast<int>(op), static_cast<int>(dtype), vec, p, grid,
                                           static_cast<unsigned>(spo), lc_shift, pdl, static_cast<cudaStream_t>(stream));
   if (err != cudaSuccess) return akg::cuda_fail(name, err);
-  std::snprintf(akg::t_kernel, sizeof akg::t_kernel, "axis<%s,%s,t256,lc%d,grid%ux%u>", dtype == AKG_F32 ? "f32" : "bf16",
+  std::snprintf(akg::t_kernel, sizeof akg::t_kernel, "axis<%s,%s,t256,lc%d,grid%ux%u>", dtype_name(dtype),
                 vec ? "vec" : "scalar", 1 << lc_shift, grid.x, grid.y);
   return AKG_OK;
 }
@@ -876,7 +879,7 @@ extern "C" akg_status akg_add_norm(akg_op op, const void* x, const void* residua
   cudaError_t err;
   if (vpt > 0) {
     err = launch_add_norm(static_cast<int>(op), static_cast<int>(dtype), vpt, static_cast<int>(threads), p, grid, pdl, cs);
-    std::snprintf(t_kernel, sizeof t_kernel, "add_flex<%s,t%d,v%d>", dtype == AKG_F32 ? "f32" : "bf16",
+    std::snprintf(t_kernel, sizeof t_kernel, "add_flex<%s,t%d,v%d>", dtype_name(dtype),
                   static_cast<int>(threads), vpt);
   } else {
     LaunchPlan plan;
@@ -884,7 +887,7 @@ extern "C" akg_status akg_add_norm(akg_op op, const void* x, const void* residua
     plan_stream(c, &plan);
     plan.pdl = pdl;
     err = (op == AKG_OP_LAYERNORM) ? launch_op<OP_LAYERNORM>(plan, c.dtype, p, cs) : launch_op<OP_RMSNORM>(plan, c.dtype, p, cs);
-    std::snprintf(t_kernel, sizeof t_kernel, "add_stream<%s,t%d>", dtype == AKG_F32 ? "f32" : "bf16", plan.threads);
+    std::snprintf(t_kernel, sizeof t_kernel, "add_stream<%s,t%d>", dtype_name(dtype), plan.threads);
   }
   if (err != cudaSuccess) return cuda_fail(name, err);
   return AKG_OK;
@@ -897,7 +900,7 @@ extern "C" akg_status akg_act_mul(akg_act act, const void* x, void* y, int64_t r
   const char* name = "akg_act_mul";
   t_error[0] = '\0';
   if (act < AKG_ACT_SILU || act > AKG_ACT_GELU_TANH) return fail(AKG_ERR_INVALID_ARG, "%s: unknown activation", name);
-  if (dtype != AKG_F32 && dtype != AKG_BF16) return fail(AKG_ERR_INVALID_ARG, "%s: unknown dtype", name);
+  if (!valid_dtype(dtype)) return fail(AKG_ERR_INVALID_ARG, "%s: unknown dtype", name);
   if (rows < 0 || d < 0) return fail(AKG_ERR_INVALID_ARG, "%s: negative rows or d", name);
   if (rows == 0 || d == 0) return AKG_OK;
   if (x == nullptr || y == nullptr) return fail(AKG_ERR_INVALID_ARG, "%s: x and y must not be NULL", name);
@@ -933,7 +936,7 @@ extern "C" akg_status akg_act_mul(akg_act act, const void* x, void* y, int64_t r
   if (err != cudaSuccess) return cuda_fail(name, err);
   std::snprintf(t_kernel, sizeof t_kernel, "act_mul<%s,%s,%s,t%d,grid%ux%u>",
                 act == AKG_ACT_SILU ? "silu" : (act == AKG_ACT_GELU ? "gelu" : "gelu_tanh"),
-                dtype == AKG_F32 ? "f32" : "bf16", vec ? "vec" : "scalar", threads, grid.x, grid.y);
+                dtype_name(dtype), vec ? "vec" : "scalar", threads, grid.x, grid.y);
   return AKG_OK;
 }
 
@@ -944,7 +947,7 @@ extern "C" akg_status akg_argreduce(int want_min, const void* x, int64_t* index_
   const char* name = "akg_argreduce";
   t_error[0] = '\0';
   if (want_min != 0 && want_min != 1) return fail(AKG_ERR_INVALID_ARG, "%s: want_min must be 0 or 1", name);
-  if (dtype != AKG_F32 && dtype != AKG_BF16) return fail(AKG_ERR_INVALID_ARG, "%s: unknown dtype", name);
+  if (!valid_dtype(dtype)) return fail(AKG_ERR_INVALID_ARG, "%s: unknown dtype", name);
   if (rows < 0 || cols < 0) return fail(AKG_ERR_INVALID_ARG, "%s: negative rows or cols", name);
   if (rows == 0) return AKG_OK;
   if (cols == 0) return fail(AKG_ERR_INVALID_ARG, "%s: an empty row has no arg-max", name);
@@ -965,7 +968,7 @@ extern "C" akg_status akg_argreduce(int want_min, const void* x, int64_t* index_
                                            g_tune_pdl.load() == 2 ? 0 : 1, static_cast<cudaStream_t>(stream));
   if (err != cudaSuccess) return cuda_fail(name, err);
   std::snprintf(t_kernel, sizeof t_kernel, "arg<%s,%s,%s,g%d,t256,grid%u>", want_min ? "min" : "max",
-                dtype == AKG_F32 ? "f32" : "bf16", vec ? "vec" : "scalar", warp_rows ? 32 : 256, grid);
+                dtype_name(dtype), vec ? "vec" : "scalar", warp_rows ? 32 : 256, grid);
   return AKG_OK;
 }
 
@@ -994,7 +997,7 @@ extern "C" akg_status akg_cumulative(int want_prod, const void* x, void* y, int6
                                             static_cast<cudaStream_t>(stream));
   if (err != cudaSuccess) return cuda_fail(name, err);
   std::snprintf(t_kernel, sizeof t_kernel, "scan<%s,%s,%s,t%d,grid%u>", want_prod ? "prod" : "sum",
-                dtype == AKG_F32 ? "f32" : "bf16", vec ? "vec" : "scalar", threads, grid);
+                dtype_name(dtype), vec ? "vec" : "scalar", threads, grid);
   return AKG_OK;
 }
 

@@ -5,13 +5,14 @@
 #pragma once
 
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
 namespace akg {
 
 enum Op : int { OP_SOFTMAX = 0, OP_LOG_SOFTMAX = 1, OP_LAYERNORM = 2, OP_RMSNORM = 3 };
-enum DType : int { DT_F32 = 0, DT_BF16 = 1 };
+enum DType : int { DT_F32 = 0, DT_BF16 = 1, DT_F16 = 2 };
 
 // One operator call.  Strides in elements.  gamma doubles as the RMSNorm weight.
 struct RowParams {
@@ -130,6 +131,8 @@ template <> struct Elem<float> {
   static __device__ __forceinline__ void store1(void* base, long long i, float v) {
     reinterpret_cast<float*>(base)[i] = v;
   }
+  // the stored bits of v, replicated to fill a 32-bit word (for constant fills)
+  static __device__ __forceinline__ uint32_t fill_word(float v) { return __float_as_uint(v); }
 };
 
 template <> struct Elem<__nv_bfloat16> {
@@ -156,6 +159,37 @@ template <> struct Elem<__nv_bfloat16> {
   static __device__ __forceinline__ void store1(void* base, long long i, float v) {
     reinterpret_cast<__nv_bfloat16*>(base)[i] = __float2bfloat16_rn(v);
   }
+  static __device__ __forceinline__ uint32_t fill_word(float v) { return pack2(v, v); }
+};
+
+// IEEE half (the paper's float16 regime, Section 4.1): same vector shape as bf16, hardware
+// conversions in both directions, one rounding (nearest-even) at the store.
+template <> struct Elem<__half> {
+  static constexpr int EPV = 8;
+  static constexpr int DT = DT_F16;
+  static __device__ __forceinline__ void unpack(const uint4& u, float (&f)[8]) {
+    const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float2 p = __half22float2(*reinterpret_cast<const __half2*>(&w[i]));
+      f[2 * i] = p.x;
+      f[2 * i + 1] = p.y;
+    }
+  }
+  static __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
+    __half2 h = __floats2half2_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&h);
+  }
+  static __device__ __forceinline__ uint4 pack(const float (&f)[8]) {
+    return make_uint4(pack2(f[0], f[1]), pack2(f[2], f[3]), pack2(f[4], f[5]), pack2(f[6], f[7]));
+  }
+  static __device__ __forceinline__ float load1(const void* base, long long i) {
+    return __half2float(reinterpret_cast<const __half*>(base)[i]);
+  }
+  static __device__ __forceinline__ void store1(void* base, long long i, float v) {
+    reinterpret_cast<__half*>(base)[i] = __float2half_rn(v);
+  }
+  static __device__ __forceinline__ uint32_t fill_word(float v) { return pack2(v, v); }
 };
 
 template <int OP> struct OpTraits {

@@ -121,8 +121,7 @@ __device__ __forceinline__ void softmax_row(const RowParams& p, long long row, i
     fill = (S != S) ? nan : kNegInf;
   }
   // the fill value as stored bits: +0, -inf or quiet NaN in the element type
-  uint32_t fill_word = __float_as_uint(fill);
-  if (sizeof(T) == 2) fill_word = (fill_word >> 16) | (fill_word & 0xffff0000u);
+  const uint32_t fill_word = E::fill_word(fill);
   const uint4 fill_vec = make_uint4(fill_word, fill_word, fill_word, fill_word);
 
 #pragma unroll

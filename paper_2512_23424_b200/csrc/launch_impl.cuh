@@ -275,6 +275,7 @@ cudaError_t launch_typed(const LaunchPlan& plan, const RowParams& p, cudaStream_
 template <int OP>
 cudaError_t launch_op(const LaunchPlan& plan, int dtype, const RowParams& p, cudaStream_t stream) {
   if (dtype == DT_F32) return launch_typed<OP, float>(plan, p, stream);
+  if (dtype == DT_F16) return launch_typed<OP, __half>(plan, p, stream);
   return launch_typed<OP, __nv_bfloat16>(plan, p, stream);
 }
 

@@ -27,6 +27,9 @@ cudaError_t launch_act_a(int dtype, bool vec, const ActParams& p, dim3 grid, int
   if (dtype == DT_F32)
     return vec ? launch_act_typed<ACT, float, true>(p, grid, threads, pdl, s)
                : launch_act_typed<ACT, float, false>(p, grid, threads, pdl, s);
+  if (dtype == DT_F16)
+    return vec ? launch_act_typed<ACT, __half, true>(p, grid, threads, pdl, s)
+               : launch_act_typed<ACT, __half, false>(p, grid, threads, pdl, s);
   return vec ? launch_act_typed<ACT, __nv_bfloat16, true>(p, grid, threads, pdl, s)
              : launch_act_typed<ACT, __nv_bfloat16, false>(p, grid, threads, pdl, s);
 }

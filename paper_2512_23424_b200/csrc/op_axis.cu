@@ -29,6 +29,9 @@ cudaError_t launch_axis_op(int dtype, bool vec, const AxisParams& p, dim3 grid, 
   if (dtype == DT_F32)
     return vec ? launch_axis_typed<OP, float, 1>(p, grid, spo, lc_shift, pdl, s)
                : launch_axis_typed<OP, float, 0>(p, grid, spo, lc_shift, pdl, s);
+  if (dtype == DT_F16)
+    return vec ? launch_axis_typed<OP, __half, 1>(p, grid, spo, lc_shift, pdl, s)
+               : launch_axis_typed<OP, __half, 0>(p, grid, spo, lc_shift, pdl, s);
   return vec ? launch_axis_typed<OP, __nv_bfloat16, 1>(p, grid, spo, lc_shift, pdl, s)
              : launch_axis_typed<OP, __nv_bfloat16, 0>(p, grid, spo, lc_shift, pdl, s);
 }

@@ -41,6 +41,11 @@ cudaError_t launch_axis_reg_op(int dtype, int mode, int r, const AxisParams& p, 
     if (mode == 0) return launch_axis_reg_m<OP, float, 0>(r, p, grid, spo, nf, nc, pdl, s);
     return cudaErrorInvalidValue;
   }
+  if (dtype == DT_F16) {
+    if (mode == 1) return launch_axis_reg_m<OP, __half, 1>(r, p, grid, spo, nf, nc, pdl, s);
+    if (mode == 0) return launch_axis_reg_m<OP, __half, 0>(r, p, grid, spo, nf, nc, pdl, s);
+    return cudaErrorInvalidValue;
+  }
   if (mode == 2) return launch_axis_reg_m<OP, __nv_bfloat16, 2>(r, p, grid, spo, nf, nc, pdl, s);
   if (mode == 1) return launch_axis_reg_m<OP, __nv_bfloat16, 1>(r, p, grid, spo, nf, nc, pdl, s);
   return launch_axis_reg_m<OP, __nv_bfloat16, 0>(r, p, grid, spo, nf, nc, pdl, s);

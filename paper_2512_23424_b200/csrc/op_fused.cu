@@ -42,10 +42,12 @@ cudaError_t launch_add_norm(int op, int dtype, int vpt, int threads, const RowPa
   if (threads < 32 || threads > 1024 || threads % 32) return cudaErrorInvalidValue;
   if (op == OP_LAYERNORM)
     return dtype == DT_F32 ? launch_add_norm_t<OP_LAYERNORM, float>(vpt, p, grid, threads, pdl, stream)
-                           : launch_add_norm_t<OP_LAYERNORM, __nv_bfloat16>(vpt, p, grid, threads, pdl, stream);
+           : dtype == DT_F16 ? launch_add_norm_t<OP_LAYERNORM, __half>(vpt, p, grid, threads, pdl, stream)
+                             : launch_add_norm_t<OP_LAYERNORM, __nv_bfloat16>(vpt, p, grid, threads, pdl, stream);
   if (op == OP_RMSNORM)
     return dtype == DT_F32 ? launch_add_norm_t<OP_RMSNORM, float>(vpt, p, grid, threads, pdl, stream)
-                           : launch_add_norm_t<OP_RMSNORM, __nv_bfloat16>(vpt, p, grid, threads, pdl, stream);
+           : dtype == DT_F16 ? launch_add_norm_t<OP_RMSNORM, __half>(vpt, p, grid, threads, pdl, stream)
+                             : launch_add_norm_t<OP_RMSNORM, __nv_bfloat16>(vpt, p, grid, threads, pdl, stream);
   return cudaErrorInvalidValue;
 }
 

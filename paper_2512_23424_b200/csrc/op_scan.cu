@@ -47,6 +47,9 @@ cudaError_t launch_argreduce(bool want_min, int dtype, bool vec, bool warp_rows,
   if (dtype == DT_F32)
     return want_min ? launch_arg_t<true, float>(vec, warp_rows, p, grid, pdl, stream)
                     : launch_arg_t<false, float>(vec, warp_rows, p, grid, pdl, stream);
+  if (dtype == DT_F16)
+    return want_min ? launch_arg_t<true, __half>(vec, warp_rows, p, grid, pdl, stream)
+                    : launch_arg_t<false, __half>(vec, warp_rows, p, grid, pdl, stream);
   return want_min ? launch_arg_t<true, __nv_bfloat16>(vec, warp_rows, p, grid, pdl, stream)
                   : launch_arg_t<false, __nv_bfloat16>(vec, warp_rows, p, grid, pdl, stream);
 }
@@ -60,6 +63,9 @@ cudaError_t launch_cumulative(bool want_prod, int dtype, bool vec, const void* x
   if (dtype == DT_F32)
     return want_prod ? launch_scan_t<true, float>(vec, p, grid, threads, pdl, stream)
                      : launch_scan_t<false, float>(vec, p, grid, threads, pdl, stream);
+  if (dtype == DT_F16)
+    return want_prod ? launch_scan_t<true, __half>(vec, p, grid, threads, pdl, stream)
+                     : launch_scan_t<false, __half>(vec, p, grid, threads, pdl, stream);
   return want_prod ? launch_scan_t<true, __nv_bfloat16>(vec, p, grid, threads, pdl, stream)
                    : launch_scan_t<false, __nv_bfloat16>(vec, p, grid, threads, pdl, stream);
 }

@@ -20,7 +20,7 @@ from typing import Dict, Optional
 
 import numpy as np
 
-F32, BF16 = 0, 1
+F32, BF16, F16 = 0, 1, 2      # F16 arrays are numpy float16
 
 
 def f32_to_bf16_bits(a: np.ndarray) -> np.ndarray:
@@ -163,7 +163,11 @@ def make_random(op: str, dtype: int, rows: int, cols: int, seed: int,
         x = f32_to_bf16_bits(x)
         gamma = None if gamma is None else f32_to_bf16_bits(gamma)
         beta = None if beta is None else f32_to_bf16_bits(beta)
-    return Workload(f"{op}_{'f32' if dtype == F32 else 'bf16'}_{rows}x{cols}", op, dtype,
+    if dtype == F16:
+        x = x.astype(np.float16)
+        gamma = None if gamma is None else gamma.astype(np.float16)
+        beta = None if beta is None else beta.astype(np.float16)
+    return Workload(f"{op}_{ {F32: 'f32', BF16: 'bf16', F16: 'f16'}[dtype]}_{rows}x{cols}", op, dtype,
                     rows, cols, x, eps=eps if op in ("layernorm", "rmsnorm") else 0.0,
                     gamma=gamma, beta=beta)
 

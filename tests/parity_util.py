@@ -34,6 +34,8 @@ def to_torch(a: Optional[np.ndarray], dtype: int, device="cuda") -> Optional[tor
         return None
     if dtype == wl.F32:
         return torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).to(device)
+    if dtype == wl.F16:
+        return torch.from_numpy(np.ascontiguousarray(a, dtype=np.float16)).to(device)
     t = torch.from_numpy(np.ascontiguousarray(a, dtype=np.uint16).view(np.int16)).to(device)
     return t.view(torch.bfloat16)
 
@@ -58,7 +60,7 @@ def strided_device_matrix(host: np.ndarray, dtype: int, stride: int, offset_elem
     """Place `host` [rows, cols] in a device buffer with the given row stride and a
     leading element offset; padding holds the sentinel.  Returns (buffer, view)."""
     rows, cols = host.shape
-    tdt = torch.float32 if dtype == wl.F32 else torch.bfloat16
+    tdt = {wl.F32: torch.float32, wl.BF16: torch.bfloat16, wl.F16: torch.float16}[dtype]
     buf = torch.full((offset_elems + rows * stride + 8,), sentinel, dtype=tdt, device="cuda")
     view = torch.as_strided(buf, (rows, cols), (stride, 1), storage_offset=offset_elems)
     view.copy_(to_torch(host, dtype))
@@ -101,6 +103,14 @@ def run_oracle(w: wl.Workload, rows: Optional[Sequence[int]] = None,
     return oracle.rmsnorm(x, w.gamma, eps=eps, nthreads=nthreads)
 
 
+def f16_ulp(ref: np.ndarray) -> np.ndarray:
+    """Spacing of IEEE half at |ref|: 2^(max(floor(log2 |ref|), -14) - 10) (2^-24 in the subnormal range)."""
+    a = np.abs(ref)
+    e = np.floor(np.log2(np.where(a > 0, a, 1.0)))
+    e = np.where(a > 0, e, -14.0)
+    return np.exp2(np.maximum(e, -14.0) - 10.0)
+
+
 def bf16_ulp(ref: np.ndarray) -> np.ndarray:
     a = np.abs(ref)
     e = np.floor(np.log2(np.where(a > 0, a, 1.0)))
@@ -125,11 +135,11 @@ def cancel_magnitude(w: wl.Workload, ref: np.ndarray, additive: Optional[np.ndar
         rstd = 1.0 / np.sqrt(x.var(axis=1, keepdims=True) + eps)
         gamma = 1.0 if w.gamma is None else np.abs(widen(w.gamma))[None, :]
         slack = 2.0 ** -23 * np.abs(x).max(axis=1, keepdims=True) * rstd * gamma * np.ones_like(ref)
-        if w.dtype == wl.BF16:
+        if w.dtype != wl.F32:
             beta = 0.0 if w.beta is None else widen(w.beta)[None, :]
             slack = slack + 2.0 ** -20 * (np.abs(ref - beta) + np.abs(beta))
         return slack
-    if w.op == "log_softmax" and w.dtype == wl.BF16:
+    if w.op == "log_softmax" and w.dtype != wl.F32:
         z = widen(w.x)
         if additive is not None:
             a = widen(additive)
@@ -162,12 +172,13 @@ def compare(got_stored: np.ndarray, ref: np.ndarray, dtype: int, what: str = "",
         worst = float(err.max()) if err.size else 0.0
         assert worst <= FP32_ATOL, f"{what}: max abs error {stats['max_abs']:.3e} > {FP32_ATOL}"
     else:
-        ulp = bf16_ulp(ref[fin])
+        # fp16 I/O: the same rule with the spacing of IEEE half (2 ulps; no flush below its range)
+        ulp = f16_ulp(ref[fin]) if dtype == wl.F16 else bf16_ulp(ref[fin])
         ulps = err / ulp
-        tiny_ok = (np.abs(ref[fin]) < tiny) & (got[fin] == 0)
+        tiny_ok = (np.abs(ref[fin]) < (0.0 if dtype == wl.F16 else tiny)) & (got[fin] == 0)
         bad = (ulps > BF16_ULPS) & ~tiny_ok
         stats["max_ulp"] = float(ulps.max()) if ulps.size else 0.0
-        assert not bad.any(), f"{what}: {bad.sum()} elements beyond {BF16_ULPS} bf16 ulps (max {stats['max_ulp']:.3f})"
+        assert not bad.any(), f"{what}: {bad.sum()} elements beyond {BF16_ULPS} ulps of the storage type (max {stats['max_ulp']:.3f})"
     return stats
 
 
@@ -180,5 +191,5 @@ def assert_positive_zero(stored: np.ndarray, where: np.ndarray, what: str = ""):
 def verifier_passes(got_stored: np.ndarray, ref: np.ndarray, dtype: int) -> bool:
     """The paper's own criterion (Section 3.2.3, Eq. 2-3): tau = 1e-3 for fp32; the
     paper's float16 threshold 4e-3 is borrowed for bf16 (it gives none)."""
-    tau = 1e-3 if dtype == wl.F32 else 4e-3
+    tau = 1e-3 if dtype == wl.F32 else 4e-3          # 4e-3 is the paper's own float16 threshold (Section 4.1)
     return oracle.verifier_fraction(widen(got_stored), ref, eps_switch=1e-8, tau=tau) <= tau

@@ -396,3 +396,22 @@ def test_config2_and_config5_statistics():
         assert y[r, :r + 1].sum() == pytest.approx(1.0, abs=1e-14)
         assert (y[r, r + 1:] == 0).all()
     assert w5.algorithmic_bytes() == (sum(range(1, 65)) + 64 * 4096) * 2
+
+
+def test_half_and_bf16_widening_is_exact_for_every_bit_pattern():
+    """All 65536 patterns of both 16-bit storage types against numpy's own conversions."""
+    bits = np.arange(65536, dtype=np.uint16)
+    half = bits.view(np.float16)
+    got, want = oracle.widen(half), half.astype(np.float64)
+    nan = np.isnan(want)
+    assert np.array_equal(np.isnan(got), nan)
+    assert np.array_equal(got[~nan], want[~nan]) and np.array_equal(np.signbit(got[~nan]), np.signbit(want[~nan]))
+    got = oracle.widen(bits)                                   # uint16 = bf16 bits
+    want = (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    nan = np.isnan(want)
+    assert np.array_equal(np.isnan(got), nan)
+    assert np.array_equal(got[~nan], want[~nan]) and np.array_equal(np.signbit(got[~nan]), np.signbit(want[~nan]))
+    # the drivers read half through the same conversion
+    x = np.random.default_rng(0).normal(0, 2, (5, 33)).astype(np.float16)
+    assert np.array_equal(oracle.softmax(x), oracle.softmax(x.astype(np.float64)))
+    assert np.array_equal(oracle.rmsnorm(x, x[0], eps=1e-6), oracle.rmsnorm(x.astype(np.float64), x[0].astype(np.float64), eps=1e-6))
