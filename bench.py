@@ -131,12 +131,12 @@ class DeviceWorkload:
         import torch
         from paper_2512_23424_b200 import binding
         self.w, self.binding, self.torch = w, binding, torch
-        tdt = torch.float32 if w.dtype == wl.F32 else torch.bfloat16
+        tdt = {wl.F32: torch.float32, wl.BF16: torch.bfloat16, wl.F16: torch.float16}[w.dtype]
 
         def dev(a):
             if a is None:
                 return None
-            if w.dtype == wl.F32:
+            if w.dtype in (wl.F32, wl.F16):
                 return torch.from_numpy(a).cuda()
             return torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
 
@@ -466,6 +466,20 @@ def run_ours(args):
             del dwk, wk
             torch.cuda.empty_cache()
         line["per_config"] = table
+        # configurations 3 and 5 stored as IEEE half (the paper's float16 regime)
+        halves = []
+        for k in (3, 5):
+            wk = wl.as_f16(wl.make_config(k))
+            dwk = DeviceWorkload(wk, pairs_for(wk))
+            reps = max(10, min(100, 100 * args.steps // 1000))
+            sk = time_launches(dwk, reps, 5) / reps
+            bk = wk.algorithmic_bytes()
+            halves.append({"workload": wk.name, "kernel": binding.last_kernel(), "us": sk * 1e6, "gbs": bk / sk / 1e9,
+                           "frac_measured": bk / sk / 1e9 / peak, "algorithmic_bytes": bk, "launches": reps,
+                           "rows_per_s": wk.rows / sk})
+            del dwk, wk
+            torch.cuda.empty_cache()
+        line["fp16_rows"] = halves
         # the operators over a non-last axis (the layout of the paper's RMSNorm sketch)
         axis = []
         for name in wl.AXIS_CONFIGS:

@@ -376,3 +376,16 @@ def make_reduction(name: str, rows: Optional[int] = None, seed_offset: int = 0) 
     if dtype == BF16:
         x = f32_to_bf16_bits(x)
     return ReductionWorkload(name, op, dtype, x)
+
+
+def as_f16(w: Workload) -> Workload:
+    """The same workload stored as IEEE half (the paper's float16 regime, Section 4.1): every
+    array is converted from its stored values with numpy's round-to-nearest-even."""
+    def conv(a):
+        if a is None:
+            return None
+        f = bf16_bits_to_f32(a) if a.dtype == np.uint16 else a
+        return f.astype(np.float16)
+    name = w.name.replace("bf16", "f16").replace("f32", "f16")
+    return Workload(name, w.op, F16, w.rows, w.cols, conv(w.x), eps=w.eps, gamma=conv(w.gamma), beta=conv(w.beta),
+                    causal_period=w.causal_period, extra=dict(w.extra))
