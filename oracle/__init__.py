@@ -289,6 +289,26 @@ def cumulative(op: str, x, nthreads: int = 1) -> np.ndarray:
     return out
 
 
+def colnorm(x, gamma=None, beta=None, eps: float = 1e-5, nthreads: int = 1):
+    """BatchNorm-style normalisation of every column of x[rows, cols] with its own mean and
+    biased variance over the rows; returns (y, mean, var) as float64."""
+    x, rows, cols, stride = _as2d(x)
+    y = np.empty((rows, cols), dtype=np.float64)
+    mean, var = np.empty(cols, dtype=np.float64), np.empty(cols, dtype=np.float64)
+    g, gp = _vec(gamma, x, cols)
+    b, bp = _vec(beta, x, cols)
+    L = lib()
+    if not L.oracle_colnorm.argtypes:
+        i64, vp, ci, dp = ctypes.c_int64, ctypes.c_void_p, ctypes.c_int, ctypes.POINTER(ctypes.c_double)
+        L.oracle_colnorm.argtypes = [vp, ci, i64, i64, i64, vp, vp, ctypes.c_double, dp, dp, dp, ci]
+        L.oracle_colnorm.restype = ci
+    rc = L.oracle_colnorm(x.ctypes.data, _dtype_code(x), rows, cols, stride, gp, bp, float(eps), _dptr(y),
+                          _dptr(mean), _dptr(var), int(nthreads))
+    if rc != 0:
+        raise ValueError("oracle_colnorm: malformed argument")
+    return y, mean, var
+
+
 AXIS_OPS = {"softmax": 0, "log_softmax": 1, "layernorm": 2, "rmsnorm": 3}
 
 

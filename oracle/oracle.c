@@ -440,6 +440,38 @@ int oracle_cumulative(int want_prod, const void* x, int dtype, int64_t rows, int
   return 0;
 }
 
+/* ---- BatchNorm-style column statistics (BatchNorm is listed in Section 3.6) ----------- */
+
+int oracle_colnorm(const void* x, int dtype, int64_t rows, int64_t cols, int64_t x_stride,
+                   const void* gamma, const void* beta, double eps, double* out_y, double* out_mean,
+                   double* out_var, int nthreads) {
+  if (bad_shape(x, dtype, rows, cols, x_stride, out_y)) return 1;
+  if (!(eps >= 0.0)) return 1;
+  int t = use_threads(nthreads);
+  if (rows == 0 || cols == 0) return 0;
+  double* g = gamma ? widen_vector(gamma, dtype, cols) : NULL;
+  double* b = beta ? widen_vector(beta, dtype, cols) : NULL;
+  int failed = (gamma && !g) || (beta && !b);
+#pragma omp parallel for schedule(static) num_threads(t)
+  for (int64_t c = 0; c < cols; ++c) {
+    if (failed) continue;
+    nsum s = {0.0, 0.0};
+    for (int64_t r = 0; r < rows; ++r) nsum_add(&s, widen(x, dtype, r * x_stride + c));
+    double mean = nsum_get(&s) / (double)rows;
+    nsum q = {0.0, 0.0};
+    for (int64_t r = 0; r < rows; ++r) { double d = widen(x, dtype, r * x_stride + c) - mean; nsum_add(&q, d * d); }
+    double var = nsum_get(&q) / (double)rows;                    /* biased, as in the forward pass */
+    double rstd = 1.0 / sqrt(var + eps);
+    double gc = g ? g[c] : 1.0, bc = b ? b[c] : 0.0;
+    for (int64_t r = 0; r < rows; ++r) out_y[r * cols + c] = (widen(x, dtype, r * x_stride + c) - mean) * rstd * gc + bc;
+    if (out_mean) out_mean[c] = mean;
+    if (out_var) out_var[c] = var;
+  }
+  free(g);
+  free(b);
+  return failed;
+}
+
 /* ---- the paper's verifier criterion (Section 3.2.3, Eq. 2-3) ------------------ */
 
 double oracle_verifier_fraction(const double* gen, const double* ref, int64_t n,

@@ -148,6 +148,15 @@ int oracle_argreduce(int want_min, const void* x, int dtype, int64_t rows, int64
 int oracle_cumulative(int want_prod, const void* x, int dtype, int64_t rows, int64_t cols, int64_t x_stride,
                       double* out, int nthreads);
 
+/* BatchNorm-style column statistics (BatchNorm is among the operators Section 3.6 lists; the
+ * formula is the textbook training-mode forward): for every column c of x[rows, cols]
+ *   mean_c = sum_r x[r,c] / rows,  var_c = sum_r (x[r,c] - mean_c)^2 / rows  (biased),
+ *   y[r,c] = (x[r,c] - mean_c) / sqrt(var_c + eps) * gamma_c + beta_c   (NULL: 1 / 0).
+ * out_y: rows x cols doubles; out_mean / out_var: cols doubles each or NULL.  Returns 0 or 1. */
+int oracle_colnorm(const void* x, int dtype, int64_t rows, int64_t cols, int64_t x_stride,
+                   const void* gamma, const void* beta, double eps, double* out_y, double* out_mean,
+                   double* out_var, int nthreads);
+
 /* The exact value of n stored elements as doubles (how every driver reads its input). */
 int oracle_widen(const void* base, int dtype, int64_t n, double* out);
 

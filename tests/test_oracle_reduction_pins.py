@@ -15,7 +15,8 @@ GOLDEN = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
 RECORDS = read_records(os.path.join(GOLDEN, "reduction_examples.txt"))
 
 
-@pytest.mark.parametrize("rec", RECORDS, ids=[r["name"] for r in RECORDS])
+@pytest.mark.parametrize("rec", [r for r in RECORDS if r["op"] != "colnorm"],
+                         ids=[r["name"] for r in RECORDS if r["op"] != "colnorm"])
 def test_worked_examples_and_their_derivation(rec):
     x = np.array(_mat(rec["x"]))
     op = rec["op"]
@@ -140,3 +141,64 @@ def test_brute_force_exact_rationals(seed):
             assert abs(cp[i, c] - float(acc_p)) <= 1e-14 * abs(float(acc_p))
         assert oracle.argreduce("argmax", x)[i] == max(range(cols), key=lambda c: (x[i, c], -c))
         assert oracle.argreduce("argmin", x)[i] == min(range(cols), key=lambda c: (x[i, c], c))
+
+
+# ---- BatchNorm-style column statistics ---------------------------------------------------------
+
+def test_colnorm_worked_example_and_identities():
+    from mpmath import mp, mpf, sqrt as mpsqrt
+    mp.dps = 40
+    rec = [r for r in RECORDS if r["name"] == "colnorm_3x2"][0]
+    want0 = np.array([float(v) for v in rec["expect"].split(";")])
+    # the file against the closed form at 40 digits
+    root = mpsqrt(mpf(3) / 2)
+    assert np.max(np.abs(want0 - np.array([float(-root * 2 + mpf("0.5")), 0.5, float(root * 2 + mpf("0.5"))]))) < 4e-16
+    x = np.array(_mat(rec["x"]))
+    g, b = np.array([2.0, 3.0]), np.array([0.5, -1.0])
+    y, mean, var = oracle.colnorm(x, g, b, eps=1e-9)
+    assert np.array_equal(mean, [2.0, 10.0]) and abs(var[0] - 2.0 / 3.0) < 1e-16 and var[1] == 0.0
+    assert np.max(np.abs(y[:, 0] - want0)) < 1e-8                  # eps = 1e-9 against the eps = 0 closed form
+    assert np.array_equal(y[:, 1], [-1.0, -1.0, -1.0])             # a constant column returns beta
+    rng = np.random.default_rng(9)
+    x = rng.normal(3.0, 2.0, (257, 37))
+    g, b = rng.uniform(0.5, 1.5, 37), rng.normal(0, 0.3, 37)
+    y, mean, var = oracle.colnorm(x, g, b, eps=1e-5)
+    # it is LayerNorm of the transpose with the affine moved to the other side
+    yt = oracle.layernorm(np.ascontiguousarray(x.T), eps=1e-5).T * g[None, :] + b[None, :]
+    assert np.max(np.abs(y - yt)) < 1e-13
+    assert np.max(np.abs(mean - x.mean(axis=0))) < 1e-14 and np.max(np.abs(var - x.var(axis=0))) < 1e-14
+    # column moments of the normalised values; a permutation of the rows permutes the output
+    z, _, _ = oracle.colnorm(x, eps=1e-5)
+    assert np.max(np.abs(z.mean(axis=0))) < 1e-14
+    assert np.max(np.abs((z * z).mean(axis=0) - var / (var + 1e-5))) < 1e-13
+    perm = rng.permutation(257)
+    assert np.max(np.abs(oracle.colnorm(x[perm], g, b, eps=1e-5)[0] - y[perm])) < 1e-13
+    # shifting and scaling a column by a positive factor leaves it unchanged at eps = 0
+    y0 = oracle.colnorm(x, eps=0.0)[0]
+    assert np.max(np.abs(oracle.colnorm(x * 3.0 + 7.0, eps=0.0)[0] - y0)) < 1e-12
+    # library second opinion: training-mode batch norm in double
+    t = torch.nn.functional.batch_norm(torch.from_numpy(x), None, None, torch.from_numpy(g), torch.from_numpy(b),
+                                       training=True, eps=1e-5).numpy()
+    assert np.max(np.abs(y - t)) < 1e-12
+    # large offset: no cancellation
+    off = oracle.colnorm(x + 1e8, eps=0.0)[0]
+    assert np.max(np.abs(off - y0)) < 1e-6
+    # storage types, strides, threads
+    xf = x.astype(np.float32)
+    a = oracle.colnorm(xf, g.astype(np.float32), b.astype(np.float32), eps=1e-5)
+    c = oracle.colnorm(xf.astype(np.float64), g.astype(np.float32).astype(np.float64), b.astype(np.float32).astype(np.float64), eps=1e-5)
+    assert all(np.array_equal(p, q) for p, q in zip(a, c))
+    big = np.zeros((257, 50), dtype=np.float32)
+    big[:, :37] = xf
+    d = oracle.colnorm(big[:, :37], g.astype(np.float32), b.astype(np.float32), eps=1e-5, nthreads=4)
+    assert all(np.array_equal(p, q) for p, q in zip(a, d))
+    # brute force at 40 digits on a tiny case
+    xs = rng.normal(0, 1, (5, 3))
+    ys, ms, vs = oracle.colnorm(xs, eps=1e-3)
+    for cidx in range(3):
+        col = [mpf(float(v)) for v in xs[:, cidx]]
+        m = sum(col) / 5
+        v = sum((e - m) ** 2 for e in col) / 5
+        assert abs(ms[cidx] - float(m)) < 1e-15 and abs(vs[cidx] - float(v)) < 1e-15
+        for r in range(5):
+            assert abs(ys[r, cidx] - float((col[r] - m) / mpsqrt(v + mpf("0.001")))) < 1e-14
