@@ -572,6 +572,44 @@ def run_ours(args):
             del rxs, routs, x0, wr
             torch.cuda.empty_cache()
         line["reduction_rows"] = reds
+        # BatchNorm-style column normalisation (two kernels; x is read twice, the second time from
+        # L2 while it fits: `gbs` counts one read and one write, `gbs_three_streams` all three)
+        colrows = []
+        for name in wl.COLNORM_CONFIGS:
+            wc = wl.make_colnorm(name)
+            cdt = torch.float32 if wc.dtype == wl.F32 else torch.bfloat16
+
+            def cdev(a):
+                if wc.dtype == wl.F32:
+                    return torch.from_numpy(a).cuda()
+                return torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
+
+            cx0 = cdev(wc.x)
+            n_buf = 2 if 2 * cx0.numel() * cx0.element_size() >= 2 * L2_BYTES else 3
+            cxs = [cx0] + [cx0.clone() for _ in range(n_buf - 1)]
+            cys = [torch.empty_like(cx0) for _ in range(n_buf)]
+            cg, cb = cdev(wc.gamma), cdev(wc.beta)
+            cws = torch.empty(binding.colnorm_workspace_bytes(wc.rows, wc.cols) or 8, dtype=torch.uint8, device="cuda")
+
+            class _Col:
+                i = 0
+
+                def launch(self):
+                    k = self.i % len(cxs)
+                    self.i += 1
+                    return binding.colnorm(cxs[k], cg, cb, eps=wc.eps, out=cys[k], workspace=cws)
+
+            _Col.torch = torch
+            binding.colnorm(cxs[0], cg, cb, eps=wc.eps, out=cys[0], workspace=cws)      # sets the ctypes signatures
+            reps = max(10, min(100, 100 * args.steps // 1000))
+            sc = time_launches(_Col(), reps, 5) / reps
+            bc = 2 * wc.rows * wc.cols * wc.itemsize
+            colrows.append({"workload": name, "kernel": binding.last_kernel(), "us": sc * 1e6, "gbs": bc / sc / 1e9,
+                            "frac_measured": bc / sc / 1e9 / peak, "gbs_three_streams": 1.5 * bc / sc / 1e9,
+                            "algorithmic_bytes": bc, "launches": 2 * reps, "rows_per_s": wc.rows / sc})
+            del cxs, cys, cx0, wc
+            torch.cuda.empty_cache()
+        line["colnorm_rows"] = colrows
     if rank == 0 and world == 1:
         line["cpu_baseline"] = oracle_baseline(w)
     assert binding.device_status() == 0, "a device-side bounded wait expired"

@@ -239,6 +239,25 @@ akg_status akg_argreduce(int want_min, const void* x, int64_t* index_out, int64_
 akg_status akg_cumulative(int want_prod, const void* x, void* y, int64_t rows, int64_t cols,
                           int64_t x_row_stride, int64_t y_row_stride, akg_dtype dtype, void* stream);
 
+/* BatchNorm-style column normalisation (BatchNorm is among the operators the paper's benchmark
+ * lists, Section 3.6; the training-mode forward with batch statistics): for every column c of the
+ * DEVICE matrix x[rows, cols]
+ *   mean_c = sum_r x[r,c] / rows,   var_c = sum_r (x[r,c] - mean_c)^2 / rows   (biased),
+ *   y[r,c] = (x[r,c] - mean_c) / sqrt(var_c + eps) * gamma_c + beta_c.
+ * gamma / beta: DEVICE vectors of cols elements of `dtype`, or NULL (1 / 0).  mean_out / var_out:
+ * DEVICE vectors of cols floats that receive the statistics, or NULL.  workspace: DEVICE memory,
+ * 8-byte aligned, owned by the caller, not read before it is written; the size returned by
+ * akg_colnorm_workspace_bytes (blocks * cols * 8 bytes with at most 256 blocks: about 1 MiB for a
+ * thousand columns) lets the rows be cut into enough blocks to fill the GPU, a smaller one (at
+ * least cols * 8 bytes) into fewer.  Two kernels are enqueued on `stream` (statistics per row block, then merge
+ * and normalise); x is read twice, the second time from L2 while the matrix fits there.  In place
+ * (y == x, equal strides) is allowed; any alignment; errors as for akg_layernorm, plus
+ * AKG_ERR_INVALID_ARG for a NULL, misaligned or too small workspace. */
+akg_status akg_colnorm(const void* x, void* y, int64_t rows, int64_t cols, int64_t x_row_stride,
+                       int64_t y_row_stride, akg_dtype dtype, const void* gamma, const void* beta, float eps,
+                       float* mean_out, float* var_out, void* workspace, size_t workspace_bytes, void* stream);
+size_t akg_colnorm_workspace_bytes(int64_t rows, int64_t cols);
+
 /* Size of the staging area built into the library (see akg_rowop_host_static). */
 #define AKG_STATIC_STAGING_BYTES (16u << 20)
 

@@ -6,6 +6,6 @@ The operators live in ``libakg.so`` (hand-written sm_100a CUDA behind the C ABI 
 generates the seeded benchmark inputs.  There is no CPU implementation here.
 """
 from . import workloads  # noqa: F401
-from .binding import (AkgError, Mask, act_mul, add_norm, argmax, argmin, cumprod, cumsum, device_status, last_error, last_kernel, layernorm,  # noqa: F401
+from .binding import (AkgError, Mask, act_mul, add_norm, argmax, argmin, colnorm, cumprod, cumsum, device_status, last_error, last_kernel, layernorm,  # noqa: F401
                       lib, log_softmax, make_mask, rmsnorm, rowop_axis, set_tuning, set_variant, softmax, softmax_scaled,
                       status_string)

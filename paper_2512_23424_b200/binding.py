@@ -410,6 +410,44 @@ def cumprod(x: torch.Tensor, out: Optional[torch.Tensor] = None, stream=None) ->
     return _cumulative(1, x, out, stream)
 
 
+def colnorm_workspace_bytes(rows: int, cols: int) -> int:
+    """akg_colnorm_workspace_bytes: the workspace with which akg_colnorm fills the GPU."""
+    fn = lib().akg_colnorm_workspace_bytes
+    fn.argtypes = [ctypes.c_int64, ctypes.c_int64]
+    fn.restype = ctypes.c_size_t
+    return int(fn(rows, cols))
+
+
+def colnorm(x: torch.Tensor, gamma: Optional[torch.Tensor] = None, beta: Optional[torch.Tensor] = None,
+            eps: float = 1e-5, out: Optional[torch.Tensor] = None, want_stats: bool = False,
+            workspace: Optional[torch.Tensor] = None, stream=None):
+    """akg_colnorm: every column of a 2-D CUDA tensor normalised with its own mean and biased variance
+    over the rows (BatchNorm-style), per-column gamma / beta.  Returns y, or (y, mean, var) with
+    float32 statistics when want_stats.  `workspace` (a CUDA byte tensor) defaults to a new one."""
+    rows, cols, xs = _matrix(x, "x")
+    if out is None:
+        out = torch.empty_like(x)
+    orow, ocol, ys = _matrix(out, "out")
+    if (orow, ocol) != (rows, cols) or out.dtype != x.dtype or out.device != x.device:
+        raise ValueError("out must match x in shape, dtype and device")
+    L = lib()
+    fn = L.akg_colnorm
+    if not fn.argtypes:
+        vp, i64, ci = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int
+        fn.argtypes = [vp, vp, i64, i64, i64, i64, ci, vp, vp, ctypes.c_float, vp, vp, vp, ctypes.c_size_t, vp]
+        fn.restype = ci
+    if workspace is None:
+        workspace = torch.empty(max(colnorm_workspace_bytes(rows, cols), 8), dtype=torch.uint8, device=x.device)
+    mean = torch.empty(cols, dtype=torch.float32, device=x.device) if want_stats else None
+    var = torch.empty(cols, dtype=torch.float32, device=x.device) if want_stats else None
+    with torch.cuda.device(x.device):
+        st = fn(x.data_ptr(), out.data_ptr(), rows, cols, xs, ys, _dtype_code(x), _vector(gamma, x, cols, "gamma"),
+                _vector(beta, x, cols, "beta"), float(eps), mean.data_ptr() if want_stats else None,
+                var.data_ptr() if want_stats else None, workspace.data_ptr(), workspace.numel(), _stream(stream))
+    _check(st, "akg_colnorm")
+    return (out, mean, var) if want_stats else out
+
+
 STATIC_STAGING_BYTES = 16 << 20
 
 

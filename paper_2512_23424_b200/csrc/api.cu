@@ -1001,6 +1001,81 @@ extern "C" akg_status akg_cumulative(int want_prod, const void* x, void* y, int6
   return AKG_OK;
 }
 
+// ---- BatchNorm-style column normalisation ------------------------------------------------------
+namespace akg {
+constexpr int kColMaxBlocks = 256;
+// row blocks that fill the GPU (up to eight CTAs per SM) when the strips are a full warp of 16-byte vectors wide
+int64_t colnorm_blocks(int64_t cols, int64_t es) {
+  const int64_t strips = (cols * es + 511) / 512;
+  return std::max<int64_t>(1, std::min<int64_t>(kColMaxBlocks, (int64_t(sm_count()) * 8 + strips - 1) / strips));
+}
+}
+
+extern "C" size_t akg_colnorm_workspace_bytes(int64_t rows, int64_t cols) {
+  if (rows <= 0 || cols <= 0) return 0;
+  return static_cast<size_t>(akg::colnorm_blocks(cols, 2)) * static_cast<size_t>(cols) * sizeof(float2);
+}
+
+extern "C" akg_status akg_colnorm(const void* x, void* y, int64_t rows, int64_t cols, int64_t x_row_stride,
+                                  int64_t y_row_stride, akg_dtype dtype, const void* gamma, const void* beta,
+                                  float eps, float* mean_out, float* var_out, void* workspace,
+                                  size_t workspace_bytes, void* stream) {
+  using namespace akg;
+  const char* name = "akg_colnorm";
+  t_error[0] = '\0';
+  Call c;
+  c.op = OP_LAYERNORM; c.x = x; c.y = y; c.rows = rows; c.cols = cols; c.xs = x_row_stride; c.ys = y_row_stride;
+  c.dtype = static_cast<int>(dtype); c.mask = nullptr; c.gamma = gamma; c.beta = beta; c.eps = eps; c.stream = stream;
+  const akg_status st = validate(c, name);
+  if (st != AKG_OK) return st;
+  if (rows == 0 || cols == 0) return AKG_OK;
+  const int64_t es = (dtype == AKG_F32) ? 4 : 2;
+  if (workspace == nullptr || (reinterpret_cast<uintptr_t>(workspace) & 7u) != 0 ||
+      workspace_bytes < static_cast<size_t>(cols) * sizeof(float2))
+    return fail(AKG_ERR_INVALID_ARG, "%s: workspace must be 8-byte aligned and hold at least cols * 8 bytes", name);
+  const bool vec = g_forced_variant.load() != V_STREAM && cols % (16 / es) == 0 && aligned16(x) && aligned16(y) &&
+                   (rows == 1 || ((x_row_stride * es) % 16 == 0 && (y_row_stride * es) % 16 == 0));
+  const int64_t w = vec ? 16 / es : 1;
+  // Row blocks the workspace and the matrix allow, then the lanes of a warp along the columns: 32
+  // (512-byte row segments) unless narrower strips are needed to give every SM its CTAs.
+  const int64_t ws_blocks = static_cast<int64_t>(workspace_bytes / (static_cast<size_t>(cols) * sizeof(float2)));
+  int64_t max_rb = std::min<int64_t>(kColMaxBlocks, ws_blocks);
+  const int t_rb = g_tune_grid_cap.load();
+  if (t_rb > 0) max_rb = std::min<int64_t>(max_rb, t_rb);
+  const int64_t want = static_cast<int64_t>(sm_count()) * 4;
+  int lc_shift = 5;
+  while (lc_shift > 3 && ((int64_t(1) << lc_shift) * w > cols ||
+                          ((cols + (int64_t(1) << lc_shift) * w - 1) / ((int64_t(1) << lc_shift) * w)) * max_rb < want))
+    --lc_shift;
+  const int t_lc = g_tune_axis_lc.load();
+  if (t_lc > 0) lc_shift = std::min(5, std::max(0, t_lc - 1));
+  const int64_t cw = (int64_t(1) << lc_shift) * w;
+  const int64_t strips = (cols + cw - 1) / cw;
+  if (strips > INT_MAX) return fail(AKG_ERR_UNSUPPORTED, "%s: too many columns", name);
+  const int64_t slots = colnorm_row_slots(lc_shift);
+  // Four CTAs are resident per SM, so strips * blocks is aimed at one full wave of them, or at two
+  // where that still leaves blocks of 512 rows or more; a partial second wave measured 10 - 20 %
+  // slower than either (16384 x 8192: 64 x 10 blocks 76 %, 64 x 18 blocks 95 % of the three-stream rate).
+  const int64_t one = std::max<int64_t>(1, want / strips), two = std::max<int64_t>(1, 2 * want / strips);
+  int64_t rb = (two <= max_rb && rows / two >= 512) ? two : std::min<int64_t>(one, max_rb);
+  rb = std::max<int64_t>(1, std::min<int64_t>(rb, (rows + slots - 1) / slots));
+  int64_t rpb = (rows + rb - 1) / rb;
+  rpb = (rpb + slots - 1) / slots * slots;
+  rb = (rows + rpb - 1) / rpb;
+
+  ColParams p;
+  p.x = x; p.y = y; p.rows = rows; p.cols = cols; p.xs = x_row_stride; p.ys = y_row_stride;
+  p.gamma = gamma; p.beta = beta; p.eps = eps; p.partial = static_cast<float2*>(workspace);
+  p.mean_out = mean_out; p.var_out = var_out; p.rows_per_block = rpb; p.lc_shift = lc_shift;
+  const dim3 grid(static_cast<unsigned>(strips), static_cast<unsigned>(rb));
+  const cudaError_t err = launch_colnorm(static_cast<int>(dtype), vec, p, grid, g_tune_pdl.load() == 2 ? 0 : 1,
+                                         static_cast<cudaStream_t>(stream));
+  if (err != cudaSuccess) return cuda_fail(name, err);
+  std::snprintf(t_kernel, sizeof t_kernel, "colnorm<%s,%s,lc%d,grid%ux%u>", dtype_name(dtype), vec ? "vec" : "scalar",
+                1 << lc_shift, grid.x, grid.y);
+  return AKG_OK;
+}
+
 // ---- host buffers without any allocation ---------------------------------------------------
 // akg_rowop_host needs a device staging area from its caller.  Some callers have no way to
 // get one: a plug-in that is handed host buffers and a stream but no allocator, a service

@@ -63,6 +63,21 @@ struct ActParams {
   long long xs, ys;                   // row strides in elements
 };
 
+// One BatchNorm-style column normalisation: x, y [rows, cols]; per-column gamma / beta.
+struct ColParams {
+  const void* x;
+  void* y;
+  long long rows, cols, xs, ys;
+  const void* gamma;
+  const void* beta;
+  float eps;
+  float2* partial;                    // workspace [row blocks][cols]: (mean, M2) of each block
+  float* mean_out;                    // [cols] or nullptr
+  float* var_out;                     // [cols] or nullptr
+  long long rows_per_block;           // a multiple of the CTA's row slots
+  int lc_shift;                       // log2 of the lanes of a warp that lie along the columns
+};
+
 // Shared-memory ring kernels: limits and the size of the bookkeeping area that
 // precedes the ring buffers (mbarriers, CTA reduction slots, cluster exchange slots).
 constexpr int kMaxCluster = 16;

@@ -1,0 +1,167 @@
+// BatchNorm-style column normalisation (BatchNorm is among the operators of Section 3.6): every
+// column of x[rows, cols] is normalised with its own mean and biased variance over the rows and
+// a per-column affine.  The reduction runs across rows, so a column's statistics come from every
+// part of the matrix: two kernels on one stream, with a small workspace between them.
+//   col_stat_kernel   grid (column strips, row blocks): per-column (mean, M2) of the block's rows,
+//                     written to workspace[block][column]
+//   col_apply_kernel  same grid: merges the blocks' pairs of its columns (Chan's formula, counts
+//                     known from the geometry), derives mean and 1 / std once per column, then
+//                     normalises its block of rows
+// x is read twice; the second read is served by L2 while the matrix fits there.  Threads own
+// columns (a warp lies 1 << lc_shift lanes along the columns and the rest along rows), as in the
+// non-last-axis kernels, whose loaders and running statistics are reused.
+#pragma once
+
+#include "kernels_axis.cuh"
+
+namespace akg {
+
+constexpr int kColUB = 4;
+
+template <typename T, int MODE>
+__global__ void __launch_bounds__(kAxisThreads, 4) col_stat_kernel(const ColParams p) {
+  pdl_prologue();
+  using A = AxisRaw<T, MODE>;
+  using Raw = typename A::Raw;
+  constexpr int W = A::W;
+  constexpr int UB = kColUB;
+  __shared__ __align__(16) float part[2][kAxisThreads * W];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int lc = 1 << p.lc_shift;
+  const int lcol = lane & (lc - 1);
+  const int slot = warp * (32 >> p.lc_shift) + (lane >> p.lc_shift);
+  const int ns = kAxisThreads >> p.lc_shift;
+  const int cw = lc * W;
+  const long long col0 = static_cast<long long>(blockIdx.x) * cw + lcol * W;
+  const bool active = col0 < p.cols;
+  const long long r0 = static_cast<long long>(blockIdx.y) * p.rows_per_block;
+  const long long r1 = min(p.rows, r0 + p.rows_per_block);
+  const long long xstep = p.xs * ns;
+
+  AxisRun<OP_LAYERNORM, W> run;
+  run.init();
+  if (active) {
+    const T* px = reinterpret_cast<const T*>(p.x) + (r0 + slot) * p.xs + col0;
+    long long f = r0 + slot;
+    for (; f + (UB - 1) * ns < r1; f += UB * ns) {
+      Raw raw[UB];
+#pragma unroll
+      for (int u = 0; u < UB; ++u, px += xstep) raw[u] = A::load(px);
+      float v[UB][W];
+#pragma unroll
+      for (int u = 0; u < UB; ++u) A::unpack(raw[u], v[u]);
+      run.template fold<UB, true>(v, UB);
+    }
+    if (f < r1) {
+      const int cnt = static_cast<int>((r1 - f + ns - 1) / ns);
+      float v[UB][W];
+#pragma unroll
+      for (int u = 0; u < UB; ++u, px += xstep) {
+        if (u < cnt) A::unpack(A::load(px), v[u]);
+        else A::unpack(A::fill(0.f), v[u]);
+      }
+      run.template fold<UB, false>(v, cnt);
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < W; ++j) {
+    part[0][slot * cw + lcol * W + j] = run.a[j];
+    part[1][slot * cw + lcol * W + j] = run.b[j];
+  }
+  __syncthreads();
+  // one thread per column merges the row slots (slot i holds nbase + (i < nrem) rows of the block)
+  const long long c = static_cast<long long>(blockIdx.x) * cw + threadIdx.x;
+  if (static_cast<int>(threadIdx.x) < cw && c < p.cols) {
+    const long long n = r1 - r0;
+    const int nbase = static_cast<int>(n / ns), nrem = static_cast<int>(n % ns);
+    float mean = 0.f;
+    for (int i = 0; i < ns; ++i) mean = fmaf(static_cast<float>(nbase + (i < nrem ? 1 : 0)), part[0][i * cw + threadIdx.x], mean);
+    mean *= 1.0f / static_cast<float>(n);
+    float m2 = 0.f;
+    for (int i = 0; i < ns; ++i) {
+      const float d = part[0][i * cw + threadIdx.x] - mean;
+      m2 += fmaf(static_cast<float>(nbase + (i < nrem ? 1 : 0)) * d, d, part[1][i * cw + threadIdx.x]);
+    }
+    p.partial[static_cast<long long>(blockIdx.y) * p.cols + c] = make_float2(mean, m2);
+  }
+}
+
+template <typename T, int MODE>
+__global__ void __launch_bounds__(kAxisThreads, 4) col_apply_kernel(const ColParams p) {
+  pdl_prologue();                              // the statistics kernel has completed when this returns
+  using A = AxisRaw<T, MODE>;
+  using E = Elem<T>;
+  using Raw = typename A::Raw;
+  constexpr int W = A::W;
+  constexpr int UB = kColUB;
+  __shared__ float fin[2][32 * W];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int lc = 1 << p.lc_shift;
+  const int lcol = lane & (lc - 1);
+  const int slot = warp * (32 >> p.lc_shift) + (lane >> p.lc_shift);
+  const int ns = kAxisThreads >> p.lc_shift;
+  const int cw = lc * W;
+  const long long r0 = static_cast<long long>(blockIdx.y) * p.rows_per_block;
+  const long long r1 = min(p.rows, r0 + p.rows_per_block);
+
+  // ---- column statistics over all row blocks, once per column of this strip
+  const long long c = static_cast<long long>(blockIdx.x) * cw + threadIdx.x;
+  if (static_cast<int>(threadIdx.x) < cw && c < p.cols) {
+    const int nblk = static_cast<int>(gridDim.y);
+    const float inv_rows = 1.0f / static_cast<float>(p.rows);
+    float mean = 0.f;
+    for (int b = 0; b < nblk; ++b) {
+      const float nb = static_cast<float>(min(p.rows, (b + 1) * p.rows_per_block) - b * p.rows_per_block);
+      mean = fmaf(nb, p.partial[static_cast<long long>(b) * p.cols + c].x, mean);
+    }
+    mean *= inv_rows;
+    float m2 = 0.f;
+    for (int b = 0; b < nblk; ++b) {
+      const float nb = static_cast<float>(min(p.rows, (b + 1) * p.rows_per_block) - b * p.rows_per_block);
+      const float2 pb = p.partial[static_cast<long long>(b) * p.cols + c];
+      const float d = pb.x - mean;
+      m2 += fmaf(nb * d, d, pb.y);
+    }
+    const float var = m2 * inv_rows;
+    fin[0][threadIdx.x] = mean;
+    fin[1][threadIdx.x] = rsqrt_refined(var + p.eps);
+    if (blockIdx.y == 0) {
+      if (p.mean_out != nullptr) p.mean_out[c] = mean;
+      if (p.var_out != nullptr) p.var_out[c] = var;
+    }
+  }
+  __syncthreads();
+
+  const long long col0 = static_cast<long long>(blockIdx.x) * cw + lcol * W;
+  if (col0 >= p.cols) return;
+  float mean[W], scale[W], shift[W];
+#pragma unroll
+  for (int j = 0; j < W; ++j) {
+    mean[j] = fin[0][lcol * W + j];
+    const float g = (p.gamma != nullptr) ? E::load1(p.gamma, col0 + j) : 1.f;
+    shift[j] = (p.beta != nullptr) ? E::load1(p.beta, col0 + j) : 0.f;
+    scale[j] = fin[1][lcol * W + j] * g;
+  }
+  const long long xstep = p.xs * ns, ystep = p.ys * ns;
+  const T* px = reinterpret_cast<const T*>(p.x) + (r0 + slot) * p.xs + col0;
+  T* py = reinterpret_cast<T*>(p.y) + (r0 + slot) * p.ys + col0;
+  for (long long f = r0 + slot; f < r1; f += static_cast<long long>(UB) * ns) {
+    const bool whole = f + (UB - 1) * ns < r1;
+    Raw raw[UB];
+#pragma unroll
+    for (int u = 0; u < UB; ++u, px += xstep)
+      if (whole || f + u * ns < r1) raw[u] = A::load(px);
+#pragma unroll
+    for (int u = 0; u < UB; ++u, py += ystep) {
+      if (whole || f + u * ns < r1) {
+        float v[W];
+        A::unpack(raw[u], v);
+#pragma unroll
+        for (int j = 0; j < W; ++j) v[j] = fmaf(v[j] - mean[j], scale[j], shift[j]);
+        A::store(py, A::pack(v));
+      }
+    }
+  }
+}
+
+}  // namespace akg

@@ -65,6 +65,11 @@ cudaError_t launch_cumulative(bool want_prod, int dtype, bool vec, const void* x
                               long long cols, long long xs, long long ys, unsigned grid, int threads, int pdl,
                               cudaStream_t stream);
 
+// BatchNorm-style column normalisation (op_colnorm.cu): two kernels, grid (column strips of
+// (1 << lc_shift) lanes, row blocks of p.rows_per_block rows).  colnorm_row_slots: rows a CTA walks at once.
+int colnorm_row_slots(int lc_shift);
+cudaError_t launch_colnorm(int dtype, bool vec, const ColParams& p, dim3 grid, int pdl, cudaStream_t stream);
+
 extern template cudaError_t launch_op<OP_SOFTMAX>(const LaunchPlan&, int, const RowParams&, cudaStream_t);
 extern template cudaError_t launch_op<OP_LOG_SOFTMAX>(const LaunchPlan&, int, const RowParams&, cudaStream_t);
 extern template cudaError_t launch_op<OP_LAYERNORM>(const LaunchPlan&, int, const RowParams&, cudaStream_t);

@@ -389,3 +389,29 @@ def as_f16(w: Workload) -> Workload:
     name = w.name.replace("bf16", "f16").replace("f32", "f16")
     return Workload(name, w.op, F16, w.rows, w.cols, conv(w.x), eps=w.eps, gamma=conv(w.gamma), beta=conv(w.beta),
                     causal_period=w.causal_period, extra=dict(w.extra))
+
+
+# ---------------------------------------------------------------------------------------------
+# BatchNorm-style column normalisation (BatchNorm is listed in Section 3.6): activations
+# [N * H * W, C] in channels-last layout, statistics per channel over all rows.
+# ---------------------------------------------------------------------------------------------
+COLNORM_CONFIGS: Dict[str, tuple] = {
+    "colnorm_f32_16384x8192": (F32, 16384, 8192),
+    "colnorm_bf16_65536x1024": (BF16, 65536, 1024),
+    "colnorm_f32_1048576x64": (F32, 1048576, 64),
+}
+
+
+def make_colnorm(name: str, rows: Optional[int] = None, seed_offset: int = 0) -> Workload:
+    """x ~ N(1, 2^2), gamma ~ U(0.5, 1.5), beta ~ N(0, 0.1^2), eps 1e-5; `op` is "colnorm"."""
+    dtype, r, c = COLNORM_CONFIGS[name]
+    r = r if rows is None else min(r, rows)
+    seed = 500 + sorted(COLNORM_CONFIGS).index(name) + 1000 * seed_offset
+    s_x, s_g, s_b = np.random.SeedSequence(seed).spawn(3)
+    rx, rg, rb = (np.random.Generator(np.random.PCG64(s)) for s in (s_x, s_g, s_b))
+    x = _normal_f32(rx, r, c) * np.float32(2.0) + np.float32(1.0)
+    gamma = rg.uniform(0.5, 1.5, c).astype(np.float32)
+    beta = (rb.standard_normal(c) * 0.1).astype(np.float32)
+    if dtype == BF16:
+        x, gamma, beta = f32_to_bf16_bits(x), f32_to_bf16_bits(gamma), f32_to_bf16_bits(beta)
+    return Workload(name, "colnorm", dtype, r, c, x, eps=1e-5, gamma=gamma, beta=beta)
