@@ -135,7 +135,12 @@ bool plan_reg(const Call& c, LaunchPlan* plan) {
   const int t_group = g_tune_reg_group.load(), t_threads = g_tune_reg_threads.load(), t_vpt = g_tune_reg_vpt.load();
   const bool many_rows = c.rows >= 4096;
   const bool want_warp = (t_group == 32) || (t_group == 0 && nvec <= 256 && many_rows);
-  if (want_warp && nvec <= 256) {
+  if (want_warp && t_group == 0 && c.dtype != AKG_F32 && nvec > 128 && (c.op == OP_LAYERNORM || c.op == OP_RMSNORM)) {
+    // 16-bit normalisation rows of 1025 .. 2048 columns: a warp per row would hold 64 values per
+    // thread and spills (LayerNorm 58 % of the copy rate); a CTA of 128 threads per row measured
+    // 70 - 75 % (RMSNorm 91 - 93 %); two warps per row and a packed-register variant were no better
+    group = threads = 128; vpt = 2;
+  } else if (want_warp && nvec <= 256) {
     group = 32; threads = 128;
     vpt = pow2_ceil(static_cast<int>((nvec + 31) / 32));
   } else if (t_threads > 0 && t_vpt > 0) {

@@ -132,7 +132,7 @@ def test_add_norm_argument_errors():
     assert call(op=0) == 1 and call(op=1) == 1 and call(op=7) == 1
     assert call(rp=None) == 1
     assert call(rs=255) == 1 and call(ss=100) == 1 and call(xs=1) == 1
-    assert call(dt=2) == 1 and call(eps=-1.0) == 1 and call(rows=-1) == 1
+    assert call(dt=3) == 1 and call(eps=-1.0) == 1 and call(rows=-1) == 1
     assert call(sp=None) == 0
     assert call(sp=P(y)) == 1                                   # the two outputs overlap
     assert call(sp=P(y) + 64, rows=1) == 1
