@@ -968,12 +968,26 @@ extern "C" akg_status akg_argreduce(int want_min, const void* x, int64_t* index_
   const int64_t ctas = warp_rows ? (rows + 7) / 8 : rows;
   const int cap = g_tune_grid_cap.load();
   const unsigned grid = static_cast<unsigned>(std::min<int64_t>(ctas, cap > 0 ? cap : INT_MAX));
+  // few, long rows (a batch of vocabulary-sized rows): cut every row into segments so that about
+  // four CTAs per SM are busy, each with at least 4096 lanes of work
+  const int64_t lanes = vec ? cols / (16 / es) : cols;
+  int64_t segments = 1;
+  if (!warp_rows && rows < 2 * static_cast<int64_t>(sm_count()) && g_tune_reg_general.load() == 0) {
+    segments = std::min<int64_t>((4 * static_cast<int64_t>(sm_count()) + rows - 1) / rows, lanes / 4096);
+    segments = std::max<int64_t>(1, std::min<int64_t>(segments, 1024));
+  }
+  const int64_t seg_vecs = (lanes + segments - 1) / segments;
   const cudaError_t err = launch_argreduce(want_min == 1, static_cast<int>(dtype), vec, warp_rows, x,
                                            reinterpret_cast<long long*>(index_out), rows, cols, x_row_stride, grid,
+                                           static_cast<unsigned>(segments), seg_vecs,
                                            g_tune_pdl.load() == 2 ? 0 : 1, static_cast<cudaStream_t>(stream));
   if (err != cudaSuccess) return cuda_fail(name, err);
-  std::snprintf(t_kernel, sizeof t_kernel, "arg<%s,%s,%s,g%d,t256,grid%u>", want_min ? "min" : "max",
-                dtype_name(dtype), vec ? "vec" : "scalar", warp_rows ? 32 : 256, grid);
+  if (segments > 1)
+    std::snprintf(t_kernel, sizeof t_kernel, "arg_split<%s,%s,%s,t256,seg%u>", want_min ? "min" : "max",
+                  dtype_name(dtype), vec ? "vec" : "scalar", static_cast<unsigned>(segments));
+  else
+    std::snprintf(t_kernel, sizeof t_kernel, "arg<%s,%s,%s,g%d,t256,grid%u>", want_min ? "min" : "max",
+                  dtype_name(dtype), vec ? "vec" : "scalar", warp_rows ? 32 : 256, grid);
   return AKG_OK;
 }
 

@@ -58,9 +58,11 @@ cudaError_t launch_act_mul(int act, int dtype, bool vec, const ActParams& p, dim
 // warp_rows: a warp per row (eight rows per CTA of 256), else a CTA per row.  Cumulative: a CTA of
 // `threads` (a multiple of 32, at most 256) per row, chunks of scan_unroll() * threads vectors.
 int scan_unroll();
+// segments > 1: every row is cut into that many pieces of seg_vecs vectors (elements when !vec), one
+// CTA each, merged by an atomic maximum on the output word (three launches).
 cudaError_t launch_argreduce(bool want_min, int dtype, bool vec, bool warp_rows, const void* x, long long* out,
-                             long long rows, long long cols, long long xs, unsigned grid, int pdl,
-                             cudaStream_t stream);
+                             long long rows, long long cols, long long xs, unsigned grid, unsigned segments,
+                             long long seg_vecs, int pdl, cudaStream_t stream);
 cudaError_t launch_cumulative(bool want_prod, int dtype, bool vec, const void* x, void* y, long long rows,
                               long long cols, long long xs, long long ys, unsigned grid, int threads, int pdl,
                               cudaStream_t stream);

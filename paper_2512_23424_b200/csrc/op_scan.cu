@@ -6,6 +6,21 @@
 namespace akg {
 namespace {
 
+template <typename K, typename... Args>
+cudaError_t launch_grid(K kernel, dim3 grid, int threads, int pdl, cudaStream_t s, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(threads);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = s;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
 template <typename K, typename P>
 cudaError_t launch_1d(K kernel, const P& p, unsigned grid, int threads, int pdl, cudaStream_t s) {
   cudaLaunchConfig_t cfg = {};
@@ -29,6 +44,20 @@ cudaError_t launch_arg_t(bool vec, bool warp_rows, const ArgParams& p, unsigned 
                    : launch_1d(arg_kernel<MIN, T, 256, 256, false>, p, grid, 256, pdl, s);
 }
 
+// rows cut into `segments` pieces of seg_vecs vectors: clear, per-segment maxima, finish
+template <bool MIN, typename T>
+cudaError_t launch_arg_split_t(bool vec, const ArgParams& p, unsigned segments, long long seg_vecs, int pdl,
+                               cudaStream_t s) {
+  const unsigned small = static_cast<unsigned>(p.rows < 65536 ? (p.rows + 255) / 256 : 256);
+  cudaError_t e = launch_grid(arg_clear_kernel, dim3(small), 256, pdl, s, p);
+  if (e != cudaSuccess) return e;
+  const dim3 grid(segments, static_cast<unsigned>(p.rows < 65535 ? p.rows : 65535));
+  e = vec ? launch_grid(arg_split_kernel<MIN, T, true>, grid, 256, pdl, s, p, seg_vecs)
+          : launch_grid(arg_split_kernel<MIN, T, false>, grid, 256, pdl, s, p, seg_vecs);
+  if (e != cudaSuccess) return e;
+  return launch_grid(arg_finish_kernel, dim3(small), 256, pdl, s, p);
+}
+
 template <bool PROD, typename T>
 cudaError_t launch_scan_t(bool vec, const ScanParams& p, unsigned grid, int threads, int pdl, cudaStream_t s) {
   return vec ? launch_1d(scan_kernel<PROD, T, true>, p, grid, threads, pdl, s)
@@ -40,10 +69,20 @@ cudaError_t launch_scan_t(bool vec, const ScanParams& p, unsigned grid, int thre
 int scan_unroll() { return kScanU; }
 
 cudaError_t launch_argreduce(bool want_min, int dtype, bool vec, bool warp_rows, const void* x, long long* out,
-                             long long rows, long long cols, long long xs, unsigned grid, int pdl,
-                             cudaStream_t stream) {
+                             long long rows, long long cols, long long xs, unsigned grid, unsigned segments,
+                             long long seg_vecs, int pdl, cudaStream_t stream) {
   ArgParams p;
   p.x = x; p.out = out; p.rows = rows; p.cols = cols; p.xs = xs;
+  if (segments > 1) {
+    if (dtype == DT_F32)
+      return want_min ? launch_arg_split_t<true, float>(vec, p, segments, seg_vecs, pdl, stream)
+                      : launch_arg_split_t<false, float>(vec, p, segments, seg_vecs, pdl, stream);
+    if (dtype == DT_F16)
+      return want_min ? launch_arg_split_t<true, __half>(vec, p, segments, seg_vecs, pdl, stream)
+                      : launch_arg_split_t<false, __half>(vec, p, segments, seg_vecs, pdl, stream);
+    return want_min ? launch_arg_split_t<true, __nv_bfloat16>(vec, p, segments, seg_vecs, pdl, stream)
+                    : launch_arg_split_t<false, __nv_bfloat16>(vec, p, segments, seg_vecs, pdl, stream);
+  }
   if (dtype == DT_F32)
     return want_min ? launch_arg_t<true, float>(vec, warp_rows, p, grid, pdl, stream)
                     : launch_arg_t<false, float>(vec, warp_rows, p, grid, pdl, stream);

@@ -58,7 +58,19 @@ def test_argreduce_shapes_ties_and_special_values(dtype):
             elif k == 4:
                 s[r, :] = -np.inf if r % 2 else np.inf
         check_arg(store(s, dtype), dtype, f"special {rows}x{cols}")
-    assert len(kernels) >= 3, kernels
+    assert len(kernels) >= 3 and any(k.startswith("arg_split") for k in kernels), kernels
+    # few long rows with and without the split into segments: same indices, ties and NaN across segments
+    x = np.round(rng.normal(0, 1, (3, 200000)) * 4).astype(np.float32) / 4
+    x[1, 150000] = np.nan
+    x[1, 70000] = np.nan
+    x[2, :] = 0.5
+    try:
+        for general in (0, 1):
+            akg.set_tuning("reg_general", general)
+            check_arg(store(x, dtype), dtype, f"long rows, split {1 - general}")
+            assert akg.last_kernel().startswith("arg_split") == (general == 0)
+    finally:
+        akg.set_tuning("reg_general", 0)
 
 
 @pytest.mark.parametrize("dtype", DTYPES)
