@@ -33,6 +33,8 @@ std::atomic<int> g_tune_reg_flex{0};      // 2 = never the runtime-thread-count 
 std::atomic<int> g_tune_axis_r{0};        // non-last axis: rows per thread (2 / 4 / 8), -1 = two-pass kernel only
 std::atomic<int> g_tune_axis_nc{0};       //   column blocks per CTA
 std::atomic<int> g_tune_axis_lc{0};       //   two-pass kernel: 1 + log2 of the lanes along the columns
+std::atomic<int> g_tune_host_chunks{0};   // host-buffer pipeline: chunks per call (0 = default)
+std::atomic<int> g_tune_host_min_kib{0};  //   smallest chunk in KiB (0 = default)
 std::atomic<int> g_tune_axis_mode{0};     //   1 = 16-byte vectors, 2 = bf16 8-byte vectors widened, 3 = elements
 
 __device__ int g_status_word = 0;
@@ -475,8 +477,10 @@ akg_status run_host(const Call& hc, const char* name, void* workspace, size_t ws
   const size_t slot_bytes = ((ws_bytes - vec_bytes) / kHostSlots) & ~static_cast<size_t>(255);
   int64_t chunk_rows = static_cast<int64_t>(slot_bytes / row_bytes);
   // about a dozen chunks so the pipeline fills, but no chunk under 4 MiB (copy efficiency)
-  int64_t want = (hc.rows + 11) / 12;
-  const int64_t min_rows = static_cast<int64_t>(((size_t(4) << 20) + row_bytes - 1) / row_bytes);
+  const int64_t nchunks = g_tune_host_chunks.load() > 0 ? g_tune_host_chunks.load() : 12;
+  const size_t min_bytes = g_tune_host_min_kib.load() > 0 ? (size_t(g_tune_host_min_kib.load()) << 10) : (size_t(4) << 20);
+  int64_t want = (hc.rows + nchunks - 1) / nchunks;
+  const int64_t min_rows = static_cast<int64_t>((min_bytes + row_bytes - 1) / row_bytes);
   if (want < min_rows) want = min_rows;
   if (chunk_rows > want) chunk_rows = want;
   if (chunk_rows < 1) chunk_rows = 1;
@@ -524,16 +528,24 @@ akg_status run_host(const Call& hc, const char* name, void* workspace, size_t ws
     const int k = static_cast<int>(chunk % kHostSlots);
     const int64_t n = (hc.rows - r0 < chunk_rows) ? hc.rows - r0 : chunk_rows;
     unsigned char* slot = ws + vec_bytes + static_cast<size_t>(k) * slot_bytes;
-    err = cudaMemcpy2DAsync(slot, row_bytes, hx + static_cast<size_t>(r0) * hc.xs * es, static_cast<size_t>(hc.xs) * es,
-                            row_bytes, static_cast<size_t>(n), cudaMemcpyHostToDevice, pipe.s[k]);
+    if (hc.xs == hc.cols)
+      err = cudaMemcpyAsync(slot, hx + static_cast<size_t>(r0) * row_bytes, static_cast<size_t>(n) * row_bytes,
+                            cudaMemcpyHostToDevice, pipe.s[k]);
+    else
+      err = cudaMemcpy2DAsync(slot, row_bytes, hx + static_cast<size_t>(r0) * hc.xs * es, static_cast<size_t>(hc.xs) * es,
+                              row_bytes, static_cast<size_t>(n), cudaMemcpyHostToDevice, pipe.s[k]);
     if (err != cudaSuccess) return cuda_fail(name, err);
     Call dc = hc;
     dc.x = slot; dc.y = slot; dc.rows = n; dc.xs = hc.cols; dc.ys = hc.cols;
     dc.gamma = d_gamma; dc.beta = d_beta; dc.stream = pipe.s[k]; dc.row_base = r0;
     st = run(dc, name);
     if (st != AKG_OK) return st;
-    err = cudaMemcpy2DAsync(hy + static_cast<size_t>(r0) * hc.ys * es, static_cast<size_t>(hc.ys) * es, slot, row_bytes,
-                            row_bytes, static_cast<size_t>(n), cudaMemcpyDeviceToHost, pipe.s[k]);
+    if (hc.ys == hc.cols)
+      err = cudaMemcpyAsync(hy + static_cast<size_t>(r0) * row_bytes, slot, static_cast<size_t>(n) * row_bytes,
+                            cudaMemcpyDeviceToHost, pipe.s[k]);
+    else
+      err = cudaMemcpy2DAsync(hy + static_cast<size_t>(r0) * hc.ys * es, static_cast<size_t>(hc.ys) * es, slot, row_bytes,
+                              row_bytes, static_cast<size_t>(n), cudaMemcpyDeviceToHost, pipe.s[k]);
     if (err != cudaSuccess) return cuda_fail(name, err);
   }
   for (int k = 0; k < kHostSlots; ++k) {
@@ -641,6 +653,8 @@ akg_status akg_set_tuning(const char* key, int value) {
   else if (!std::strcmp(key, "interleave")) g_tune_interleave.store(value);
   else if (!std::strcmp(key, "pdl")) g_tune_pdl.store(value);
   else if (!std::strcmp(key, "reg_flex")) g_tune_reg_flex.store(value);
+  else if (!std::strcmp(key, "host_chunks")) g_tune_host_chunks.store(value);
+  else if (!std::strcmp(key, "host_min_kib")) g_tune_host_min_kib.store(value);
   else if (!std::strcmp(key, "axis_r")) g_tune_axis_r.store(value);
   else if (!std::strcmp(key, "axis_nc")) g_tune_axis_nc.store(value);
   else if (!std::strcmp(key, "axis_mode")) g_tune_axis_mode.store(value);
