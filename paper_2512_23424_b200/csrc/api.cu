@@ -165,8 +165,12 @@ bool plan_reg(const Call& c, LaunchPlan* plan) {
   int cap = g_tune_grid_cap.load();
   // the softmax pair runs persistent (two resident waves of CTAs, grid-stride over rows):
   // measured a little faster than one CTA per row, most under a causal mask
-  if (cap == 0 && group == threads && (c.op == OP_SOFTMAX || c.op == OP_LOG_SOFTMAX))
-    cap = sm_count() * (2048 / threads);
+  // (the cap has to be a multiple of the CTAs resident at once, 1024 / threads per SM, fewer
+  // where the kernel trades occupancy for registers: 2.67 waves measured 4 % slower than 2 or 4)
+  if (cap == 0 && group == threads && (c.op == OP_SOFTMAX || c.op == OP_LOG_SOFTMAX)) {
+    const int resident = (vpt == 4 && threads == 128) ? 6 : (vpt == 4 && threads == 256) ? 3 : 1024 / threads;
+    cap = sm_count() * 2 * resident;
+  }
   if (cap > 0 && grid > cap) grid = cap;
   if (grid > INT_MAX) grid = INT_MAX;
   plan->variant = V_REG; plan->threads = threads; plan->group = group; plan->vpt = vpt;
