@@ -45,9 +45,12 @@ template <bool MIN> __device__ __forceinline__ uint32_t arg_key(float v) {
 // The 64-bit key of the best candidate among vectors v_begin + tg, v_begin + tg + G, ... < v_end of
 // the row at xr (elements when !VEC); 0 if the thread saw nothing.  Larger key = better candidate,
 // ties resolved towards the lower index.
-template <bool MIN, typename T, bool VEC>
+// PRE: the caller may already hold the thread's first four vectors (v_begin + tg + u * G, u < 4)
+// in `first` (use_first says whether it does), loaded while it worked on the row before.
+template <bool MIN, typename T, bool VEC, bool PRE = false>
 __device__ __forceinline__ unsigned long long arg_thread_key(const T* xr, long long v_begin, long long v_end,
-                                                             int tg, int G) {
+                                                             int tg, int G, const uint4* first = nullptr,
+                                                             bool use_first = false) {
   using E = Elem<T>;
   constexpr int EPV = VEC ? E::EPV : 1;
   constexpr int U = 4;
@@ -69,6 +72,18 @@ __device__ __forceinline__ unsigned long long arg_thread_key(const T* xr, long l
 
   long long i = v_begin + tg;
   if (VEC) {
+    if (PRE && use_first) {
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        float v[E::EPV];
+        E::unpack(first[u], v);
+        float w[EPV];
+#pragma unroll
+        for (int j = 0; j < EPV; ++j) w[j] = v[j];
+        visit(w, i + u * G);
+      }
+      i += U * G;
+    }
     for (; i + (U - 1) * G < v_end; i += U * G) {
       uint4 raw[U];
 #pragma unroll
@@ -132,6 +147,42 @@ __global__ void __launch_bounds__(THREADS) arg_kernel(const ArgParams p) {
   const int tg = threadIdx.x % G;
   const int grp = threadIdx.x / G;
   const long long nvec = p.cols / EPV;                          // VEC: cols is a multiple of EPV
+
+  if constexpr (VEC && G == THREADS) {
+    // a CTA per row, grid-stride: the first four vectors of the CTA's next row are loaded before
+    // the current row is searched, so that their latency hides behind it
+    const bool can_pre = nvec >= 4 * G;
+    long long row = blockIdx.x;
+    if (row >= p.rows) return;
+    uint4 pre[4];
+    if (can_pre) {
+      const T* xr = reinterpret_cast<const T*>(p.x) + row * p.xs;
+#pragma unroll
+      for (int u = 0; u < 4; ++u) pre[u] = ld_stream(xr + (static_cast<long long>(tg) + u * G) * EPV);
+    }
+    for (; row < p.rows; row += gridDim.x) {
+      uint4 cur[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) cur[u] = pre[u];
+      const long long nrow = row + gridDim.x;
+      if (can_pre && nrow < p.rows) {
+        const T* xn = reinterpret_cast<const T*>(p.x) + nrow * p.xs;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) pre[u] = ld_stream(xn + (static_cast<long long>(tg) + u * G) * EPV);
+      }
+      unsigned long long key = arg_thread_key<MIN, T, VEC, true>(reinterpret_cast<const T*>(p.x) + row * p.xs, 0, nvec,
+                                                                 tg, G, cur, can_pre);
+      key = warp_max_key(key);
+      __syncthreads();                                          // red is reused by the next row
+      if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = key;
+      __syncthreads();
+      key = red[0];
+#pragma unroll
+      for (int w = 1; w < NW; ++w) key = red[w] > key ? red[w] : key;
+      if (tg == 0) p.out[row] = static_cast<long long>(0xffffffffull - (key & 0xffffffffull));
+    }
+    return;
+  }
 
   for (long long rb = static_cast<long long>(blockIdx.x) * RPC; rb < p.rows; rb += static_cast<long long>(gridDim.x) * RPC) {
     const long long row = rb + grp;
