@@ -1017,6 +1017,11 @@ extern "C" akg_status akg_argreduce(int want_min, const void* x, int64_t* index_
   return AKG_OK;
 }
 
+// Rows up to this many bytes take a warp each (measured against a CTA per row: fp32 512 columns 107 %
+// of the copy rate against 61 %, 1024 - 2048 columns level, 8192 columns 98 % against 105 %; bf16
+// 1024 columns 96 % against 60 %, 8192 columns 95 % against 80 %, 16384 columns 91 % against 87 %).
+namespace akg { constexpr int64_t scan_warp_row_bytes(int64_t es) { return es == 2 ? 32768 : 2048; } }
+
 extern "C" akg_status akg_cumulative(int want_prod, const void* x, void* y, int64_t rows, int64_t cols,
                                      int64_t x_row_stride, int64_t y_row_stride, akg_dtype dtype, void* stream) {
   using namespace akg;
@@ -1036,13 +1041,17 @@ extern "C" akg_status akg_cumulative(int want_prod, const void* x, void* y, int6
   int threads = 32;
   while (threads < 256 && static_cast<int64_t>(threads) * u < nvec) threads <<= 1;
   const int cap = g_tune_grid_cap.load();
-  const unsigned grid = static_cast<unsigned>(std::min<int64_t>(rows, cap > 0 ? cap : INT_MAX));
+  const int t_group = g_tune_reg_group.load();
+  // short rows: a warp per row, eight rows per CTA (no CTA barrier, no one- or two-warp CTAs)
+  const bool warp_rows = vec && (t_group == 32 || (t_group == 0 && cols * es <= scan_warp_row_bytes(es)));
+  const int64_t ctas = warp_rows ? (rows + 7) / 8 : rows;
+  const unsigned grid = static_cast<unsigned>(std::min<int64_t>(ctas, cap > 0 ? cap : INT_MAX));
   const cudaError_t err = launch_cumulative(want_prod == 1, static_cast<int>(dtype), vec, x, y, rows, cols, x_row_stride,
-                                            y_row_stride, grid, threads, g_tune_pdl.load() == 2 ? 0 : 1,
+                                            y_row_stride, grid, threads, warp_rows, g_tune_pdl.load() == 2 ? 0 : 1,
                                             static_cast<cudaStream_t>(stream));
   if (err != cudaSuccess) return cuda_fail(name, err);
-  std::snprintf(t_kernel, sizeof t_kernel, "scan<%s,%s,%s,t%d,grid%u>", want_prod ? "prod" : "sum",
-                dtype_name(dtype), vec ? "vec" : "scalar", threads, grid);
+  std::snprintf(t_kernel, sizeof t_kernel, "scan<%s,%s,%s,%s%d,grid%u>", want_prod ? "prod" : "sum",
+                dtype_name(dtype), vec ? "vec" : "scalar", warp_rows ? "g32,t" : "t", warp_rows ? 256 : threads, grid);
   return AKG_OK;
 }
 

@@ -27,21 +27,40 @@ template <bool PROD> __device__ __forceinline__ float scan_identity() { return P
 constexpr int kScanU = 4;
 constexpr int kScanMaxWarps = 8;
 
-template <bool PROD, typename T, bool VEC>
+// WARP = true: every warp of the CTA owns rows of its own (short rows: no shared memory and no
+// CTA barrier, the warp's total comes from lane 31 by shuffle); WARP = false: the CTA owns a row.
+template <bool PROD, typename T, bool VEC, bool WARP = false>
 __global__ void __launch_bounds__(32 * kScanMaxWarps, 4) scan_kernel(const ScanParams p) {
   pdl_prologue();
   using E = Elem<T>;
   constexpr int EPV = VEC ? E::EPV : 1;
   constexpr int U = kScanU;
   __shared__ float wtot[2][U][kScanMaxWarps];
-  const int T_ = blockDim.x;
-  const int NW = T_ >> 5;
   const int lane = threadIdx.x & 31;
-  const int warp = threadIdx.x >> 5;
+  const int T_ = WARP ? 32 : static_cast<int>(blockDim.x);      // threads per row
+  const int tid = WARP ? lane : static_cast<int>(threadIdx.x);  // position among them
+  const int NW = T_ >> 5;
+  const int warp = WARP ? 0 : static_cast<int>(threadIdx.x >> 5);
+  const long long row0 = WARP ? static_cast<long long>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5)
+                              : static_cast<long long>(blockIdx.x);
+  const long long row_step = WARP ? static_cast<long long>(gridDim.x) * (blockDim.x >> 5)
+                                  : static_cast<long long>(gridDim.x);
   const long long nvec = (p.cols + EPV - 1) / EPV;              // VEC: cols is a multiple of EPV
   const float id = scan_identity<PROD>();
 
-  for (long long row = blockIdx.x; row < p.rows; row += gridDim.x) {
+  // the 16-byte vectors of a chunk are loaded one chunk ahead (the row's next chunk, or the first
+  // chunk of the CTA's next row), so that their latency hides behind the scan of the current one
+  uint4 ahead[U];
+  auto load_chunk = [&](const T* xr, long long base) {
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const long long i = base + static_cast<long long>(u) * T_ + tid;
+      if (i < nvec) ahead[u] = ld_stream(xr + i * EPV);
+    }
+  };
+  if (VEC && row0 < p.rows) load_chunk(reinterpret_cast<const T*>(p.x) + row0 * p.xs, 0);
+
+  for (long long row = row0; row < p.rows; row += row_step) {
     const T* xr = reinterpret_cast<const T*>(p.x) + row * p.xs;
     T* yr = reinterpret_cast<T*>(p.y) + row * p.ys;
     float carry = id;
@@ -52,13 +71,13 @@ __global__ void __launch_bounds__(32 * kScanMaxWarps, 4) scan_kernel(const ScanP
       if (VEC) {
         uint4 raw[U];
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-          const long long i = base + static_cast<long long>(u) * T_ + threadIdx.x;
-          if (i < nvec) raw[u] = ld_stream(xr + i * EPV);
-        }
+        for (int u = 0; u < U; ++u) raw[u] = ahead[u];
+        const long long nbase = base + static_cast<long long>(U) * T_;
+        if (nbase < nvec) load_chunk(xr, nbase);
+        else if (row + row_step < p.rows) load_chunk(xr + row_step * p.xs, 0);
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-          const long long i = base + static_cast<long long>(u) * T_ + threadIdx.x;
+          const long long i = base + static_cast<long long>(u) * T_ + tid;
           float f[E::EPV];
           if (i < nvec) E::unpack(raw[u], f);
 #pragma unroll
@@ -67,7 +86,7 @@ __global__ void __launch_bounds__(32 * kScanMaxWarps, 4) scan_kernel(const ScanP
       } else {
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-          const long long i = base + static_cast<long long>(u) * T_ + threadIdx.x;
+          const long long i = base + static_cast<long long>(u) * T_ + tid;
           v[u][0] = (i < nvec) ? E::load1(xr, i) : id;
         }
       }
@@ -87,11 +106,13 @@ __global__ void __launch_bounds__(32 * kScanMaxWarps, 4) scan_kernel(const ScanP
           if (lane >= d) incl[u] = scan_op<PROD>(o, incl[u]);
         }
       }
-      if (lane == 31) {
+      if (!WARP) {
+        if (lane == 31) {
 #pragma unroll
-        for (int u = 0; u < U; ++u) wtot[par][u][warp] = incl[u];
+          for (int u = 0; u < U; ++u) wtot[par][u][warp] = incl[u];
+        }
+        __syncthreads();
       }
-      __syncthreads();
       // ---- what precedes this thread's vector u: carry, earlier u, earlier warps, earlier lanes
       float before = carry;
 #pragma unroll
@@ -99,16 +120,20 @@ __global__ void __launch_bounds__(32 * kScanMaxWarps, 4) scan_kernel(const ScanP
         // the warps' totals of this u are combined on their own, so that the carry picks up one
         // operation per u (its rounding error grows with the number of chunks, not of warps)
         float pre = id, tot = id;
-        for (int w = 0; w < NW; ++w) {
-          const float t = wtot[par][u][w];
-          if (w < warp) pre = scan_op<PROD>(pre, t);
-          tot = scan_op<PROD>(tot, t);
+        if (WARP) {
+          tot = __shfl_sync(0xffffffffu, incl[u], 31);
+        } else {
+          for (int w = 0; w < NW; ++w) {
+            const float t = wtot[par][u][w];
+            if (w < warp) pre = scan_op<PROD>(pre, t);
+            tot = scan_op<PROD>(tot, t);
+          }
         }
         float mine = scan_op<PROD>(before, pre);                // carry, all of the earlier u, earlier warps
         before = scan_op<PROD>(before, tot);
         const float excl = __shfl_up_sync(0xffffffffu, incl[u], 1);
         if (lane > 0) mine = scan_op<PROD>(mine, excl);
-        const long long i = base + static_cast<long long>(u) * T_ + threadIdx.x;
+        const long long i = base + static_cast<long long>(u) * T_ + tid;
         if (i < nvec) {
           float o[EPV];
 #pragma unroll
@@ -125,7 +150,7 @@ __global__ void __launch_bounds__(32 * kScanMaxWarps, 4) scan_kernel(const ScanP
       }
       carry = before;
     }
-    __syncthreads();                                            // wtot[par] of the next row
+    if (!WARP) __syncthreads();                                 // wtot[par] of the next row
   }
 }
 

@@ -64,8 +64,8 @@ cudaError_t launch_argreduce(bool want_min, int dtype, bool vec, bool warp_rows,
                              long long rows, long long cols, long long xs, unsigned grid, unsigned segments,
                              long long seg_vecs, int pdl, cudaStream_t stream);
 cudaError_t launch_cumulative(bool want_prod, int dtype, bool vec, const void* x, void* y, long long rows,
-                              long long cols, long long xs, long long ys, unsigned grid, int threads, int pdl,
-                              cudaStream_t stream);
+                              long long cols, long long xs, long long ys, unsigned grid, int threads, bool warp_rows,
+                              int pdl, cudaStream_t stream);
 
 // BatchNorm-style column normalisation (op_colnorm.cu): two kernels, grid (column strips of
 // (1 << lc_shift) lanes, row blocks of p.rows_per_block rows).  colnorm_row_slots: rows a CTA walks at once.
