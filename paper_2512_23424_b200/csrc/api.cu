@@ -300,13 +300,25 @@ bool plan_split(const Call& c, LaunchPlan* plan) {
   const int64_t epv = (c.dtype == AKG_F32) ? 4 : 8;
   const int64_t nvec = c.cols / epv;
   const int t_cs = g_tune_cluster_size.load(), t_threads = g_tune_smem_threads.load();
-  int cs = t_cs > 0 ? t_cs : 16;
-  if (cs < 1 || cs > kMaxCluster || (cs & (cs - 1))) return false;
   const int threads = t_threads > 0 ? t_threads : 256;
   if (threads != 256 && threads != 512 && threads != 1024) return false;
+  int cs = t_cs;
+  if (cs == 0) {
+    // slices of about 4096 vectors (16 per thread) measured best at every row length (65536 fp32
+    // columns: 4 CTAs 82 %, 16 CTAs 45 % of the copy rate; 131072: 8 CTAs 84 %, 16 CTAs 64 %);
+    // few rows take larger clusters so that there are about two CTAs per SM
+    int by_len = 1, by_fill = 1;
+    while (by_len < kMaxCluster && nvec / (2 * by_len) >= 3072) by_len *= 2;
+    while (by_fill < kMaxCluster && c.rows * by_fill < 2 * static_cast<int64_t>(sm_count())) by_fill *= 2;
+    cs = std::max(by_len, by_fill);
+  }
+  if (cs < 1 || cs > kMaxCluster || (cs & (cs - 1))) return false;
   while (cs > 1 && nvec / cs < threads) cs /= 2;          // keep at least one vector per thread
   plan->variant = V_CLUSTER; plan->threads = threads; plan->group = threads;
-  plan->vpt = static_cast<int>((nvec + cs - 1) / cs);
+  // slices are whole unrolled steps (4 vectors per thread) except the row's last one
+  int64_t slice = (nvec + cs - 1) / cs;
+  if (slice >= 4 * threads) slice = (slice + 4 * threads - 1) / (4 * threads) * (4 * threads);
+  plan->vpt = static_cast<int>(slice);
   plan->cluster = cs; plan->stages = 0; plan->smem = 0;
   const int cap = g_tune_grid_cap.load();
   plan->grid = cap > 0 ? static_cast<unsigned>((cap / cs > 0 ? cap / cs : 1) * cs) : 0u;
@@ -400,7 +412,23 @@ akg_status run(const Call& c, const char* name) {
       p.status = status_word_ptr();
     }
   }
-  if (!planned && (forced == V_AUTO || forced == V_REG) && vec) planned = plan_reg(c, &plan);
+  // rows beyond 2048 vectors in the 16-bit types (beyond 4096 for the fp32 softmax pair) measured
+  // faster in the two-pass kernel than in one CTA of 640 - 1024 threads: bf16 32768 columns 77 - 79 %
+  // against 63 %, fp32 softmax 32768 columns 81 % against 77 % (fp32 normalisations: 82 % against 93 %, kept)
+  const int64_t row_vecs = c.cols / ((c.dtype == AKG_F32) ? 4 : 8);
+  const bool long_row = forced == V_AUTO && g_tune_cluster_mode.load() != 1 &&
+                        ((c.dtype != AKG_F32 && row_vecs > 2048) ||
+                         (c.dtype == AKG_F32 && row_vecs > 4096 && (c.op == OP_SOFTMAX || c.op == OP_LOG_SOFTMAX)));
+  if (!planned && (forced == V_AUTO || forced == V_REG) && vec && !long_row) {
+    planned = plan_reg(c, &plan);
+    // fp32 normalisation rows beyond 4096 vectors stay in registers only as an exact fit (the ragged
+    // 1024-thread form measured 49 % on 32000 columns)
+    if (planned && forced == V_AUTO && g_tune_cluster_mode.load() != 1 && c.dtype == AKG_F32 && row_vecs > 4096 &&
+        plan.mode != 2 && plan.stages != 1) {
+      planned = false;
+      plan = LaunchPlan{};
+    }
+  }
   if (!planned && vec) {
     if (forced == V_AUTO) planned = (g_tune_cluster_mode.load() == 1) ? plan_smem(c, 1, kMaxCluster, &plan)
                                                                       : plan_split(c, &plan);
