@@ -137,7 +137,16 @@ bool plan_reg(const Call& c, LaunchPlan* plan) {
   const int t_group = g_tune_reg_group.load(), t_threads = g_tune_reg_threads.load(), t_vpt = g_tune_reg_vpt.load();
   const bool many_rows = c.rows >= 4096;
   const bool want_warp = (t_group == 32) || (t_group == 0 && nvec <= 256 && many_rows);
-  if (want_warp && t_group == 0 && c.dtype != AKG_F32 && nvec > 128 && (c.op == OP_LAYERNORM || c.op == OP_RMSNORM)) {
+  const bool norm_op = (c.op == OP_LAYERNORM || c.op == OP_RMSNORM);
+  // normalisation rows of exactly 32 x (3, 5, 6, 7) vectors: a warp per row, predicate-free (fp32
+  // 768 columns, 16-bit 768 and 1280 columns; more than 40 values per thread would spill)
+  const int64_t per_lane = (nvec % 32 == 0) ? nvec / 32 : 0;
+  const bool odd_warp_fit = want_warp && t_group == 0 && norm_op && g_tune_reg_general.load() == 0 &&
+                            (per_lane == 3 || per_lane == 5 || per_lane == 6 || per_lane == 7) &&
+                            (per_lane * epv <= 40 || per_lane == 7);   // 7: the alternative is 224 x 1
+  if (odd_warp_fit) {
+    group = 32; threads = 128; vpt = static_cast<int>(per_lane);
+  } else if (want_warp && t_group == 0 && c.dtype != AKG_F32 && nvec > 128 && (c.op == OP_LAYERNORM || c.op == OP_RMSNORM)) {
     // 16-bit normalisation rows of 1025 .. 2048 columns: a warp per row would hold 64 values per
     // thread and spills (LayerNorm 58 % of the copy rate); a CTA of 128 threads per row measured
     // 70 - 75 % (RMSNorm 91 - 93 %); two warps per row and a packed-register variant were no better
@@ -193,7 +202,7 @@ bool plan_reg(const Call& c, LaunchPlan* plan) {
     // fewer, fatter threads measured best (the per-row reduction is paid per thread): take
     // the largest vectors-per-thread that leaves at least 128 threads, else whatever fits
     // (one vector per thread only as a last resort: 1536 16-bit columns ran at 38 - 44 % as 192 x 1)
-    for (int v = max_vpt; v >= 2 && best_vpt == 0; --v) {
+    for (int v = max_vpt; v >= 3 && best_vpt == 0; --v) {
       if (nvec % v) continue;
       const int64_t g = nvec / v;
       if (g % 32 == 0 && g >= 128 && g <= 1024) { best_vpt = v; best_g = g; }

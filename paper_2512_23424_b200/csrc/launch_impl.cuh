@@ -241,6 +241,19 @@ cudaError_t launch_typed(const LaunchPlan& plan, const RowParams& p, cudaStream_
   }
     AKG_REG_SHAPES(AKG_REG_CASE)
 #undef AKG_REG_CASE
+    // a warp per row with an odd number of vectors per lane (768, 1280, 1536 ... columns): exact
+    // fits of the normalisation kernel only
+    if constexpr (!OpTraits<OP>::kSoftmaxLike) {
+      if (plan.stages == 1 && plan.group == 32 && plan.threads == 128) {
+        switch (plan.vpt) {
+          case 3: return launch_plain(reg_norm_full<OP, T, 32, 3, 128>, plan, plan.grid, 128, 0, s, p);
+          case 5: return launch_plain(reg_norm_full<OP, T, 32, 5, 128>, plan, plan.grid, 128, 0, s, p);
+          case 6: return launch_plain(reg_norm_full<OP, T, 32, 6, 128>, plan, plan.grid, 128, 0, s, p);
+          case 7: return launch_plain(reg_norm_full<OP, T, 32, 7, 128>, plan, plan.grid, 128, 0, s, p);
+          default: break;
+        }
+      }
+    }
     return cudaErrorInvalidConfiguration;
   }
   if (plan.variant == V_TMA && plan.mode == 1) {             // ring-fed register kernels
