@@ -704,6 +704,50 @@ def run_profile(args):
                       "algorithmic_bytes": w.algorithmic_bytes()}))
 
 
+SWEEP_COLS = (256, 512, 768, 1024, 1280, 1536, 2048, 2560, 3072, 4096, 5120, 6144, 7168, 8192, 12288, 16384,
+              20480, 32000, 32768, 50304, 65536, 128256, 131072, 151936, 262144)
+
+
+def run_sweep(args):
+    """Width sweep of the four operators (fp32 and bf16; 2^26 elements per call, rows = 2^26 / cols;
+    seeded normal inputs, unit gamma / beta): fraction of the measured copy peak and the kernel the
+    planner chose, one JSON line per (dtype, cols).  Not part of the bench line."""
+    import torch
+    from paper_2512_23424_b200 import binding
+    torch.cuda.set_device(0)
+    peak = measured_peak()[0]
+    gen = torch.Generator(device="cuda").manual_seed(2512)
+    for tdt, dname in ((torch.float32, "f32"), (torch.bfloat16, "bf16")):
+        for cols in SWEEP_COLS:
+            rows = (1 << 26) // cols
+            sets = max(2, (1 << 30) // (rows * cols * 4))              # rotate over > L2 worth of buffers
+            xs = [torch.randn((rows, cols), device="cuda", dtype=torch.float32, generator=gen).to(tdt)
+                  for _ in range(sets)]
+            ys = [torch.empty_like(x) for x in xs]
+            g = torch.ones(cols, device="cuda", dtype=tdt)
+            b = torch.zeros(cols, device="cuda", dtype=tdt)
+            calls = {"softmax": lambda i: binding.softmax(xs[i], out=ys[i]),
+                     "log_softmax": lambda i: binding.log_softmax(xs[i], out=ys[i]),
+                     "layernorm": lambda i: binding.layernorm(xs[i], g, b, out=ys[i]),
+                     "rmsnorm": lambda i: binding.rmsnorm(xs[i], g, out=ys[i])}
+            line = {"dtype": dname, "rows": rows, "cols": cols}
+            for op, call in calls.items():
+                for i in range(sets):
+                    call(i)
+                torch.cuda.synchronize()
+                start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                start.record()
+                for k in range(args.steps):
+                    call(k % sets)
+                stop.record()
+                torch.cuda.synchronize()
+                secs = start.elapsed_time(stop) * 1e-3 / args.steps
+                gbs = 2 * rows * cols * xs[0].element_size() / secs / 1e9
+                line[op] = {"frac": round(gbs / peak, 3), "us": round(secs * 1e6, 1), "kernel": binding.last_kernel()}
+            print(json.dumps(line), flush=True)
+            del xs, ys
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -724,7 +768,14 @@ def main():
                     help="truncate the rows of --profile (the outer axis of --profile-axis)")
     ap.add_argument("--variant", default="", help="force a kernel family in --profile mode")
     ap.add_argument("--tune", default="", help="--profile mode: key=value[,key=value] launch-geometry overrides")
+    ap.add_argument("--sweep", action="store_true",
+                    help="width sweep of the four operators (one JSON line per dtype and width) instead of the bench line")
     args = ap.parse_args()
+    if args.sweep:
+        if args.steps == 1000:
+            args.steps = 20
+        run_sweep(args)
+        return
     if args.profile or args.profile_axis or args.profile_fused or args.profile_act:
         run_profile(args)
     elif args.impl == "reference":

@@ -1,6 +1,6 @@
 #!/usr/bin/env python3
 """Generates the polynomial coefficients of the normal distribution function used by the
-GELU-and-Mul kernel (kernels_act.cuh: phi_lower).
+GELU-and-Mul kernel (kernels_act.cuh: normal_cdf).
 
 For x >= 0 the scaled complementary error function erfcx(x) = exp(x^2) erfc(x) behaves like
 1 / (x sqrt(pi)) at infinity, so with t = 1 / (1 + x / 2) in (0, 1] the ratio

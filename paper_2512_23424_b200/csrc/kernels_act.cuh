@@ -28,8 +28,9 @@ __device__ __forceinline__ float sigmoid_f32(float t) {
 // h(t) (coefficients and their measured error: gen_phi_coeffs.py), so
 //   Phi(-|a|) = 0.5 exp(-a^2 / 2) t h(t)
 // holds its RELATIVE accuracy in the far left tail, where 1 + erf(.) cancels: degree 9 is
-// 4e-7 near the centre (fp32 output), degree 5 is 7e-5 (enough for a bf16 output).  One
-// reciprocal, one exponential, DEG multiply-adds.
+// 4e-7 near the centre (fp32 output), degree 5 is 7e-5 (enough for a 16-bit output; degree 4,
+// 3.9e-4, failed the parity test on bf16).  One reciprocal, one exponential, DEG multiply-adds;
+// the factor 0.5 is folded into the coefficients at compile time.
 template <int DEG> __device__ __forceinline__ float normal_cdf(float a) {
   constexpr float c9[10] = {2.820947468e-01f, 2.821037173e-01f, 2.465246618e-01f, 1.803003252e-01f,
                             5.878400058e-02f, 7.814583927e-02f, -1.966046691e-01f, 2.911409736e-02f,
@@ -39,16 +40,19 @@ template <int DEG> __device__ __forceinline__ float normal_cdf(float a) {
   static_assert(DEG == 9 || DEG == 5, "fitted degrees");
   float t;
   asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t) : "f"(fmaf(fabsf(a), 0.35355339059327376220f, 1.0f)));
-  float h = (DEG == 9) ? c9[9] : c5[5];
+  float h = 0.5f * ((DEG == 9) ? c9[9] : c5[5]);
 #pragma unroll
-  for (int i = DEG - 1; i >= 0; --i) h = fmaf(h, t, (DEG == 9) ? c9[i] : c5[i]);
-  const float q = 0.5f * t * h * ex2_approx(a * a * (-0.5f * kLog2e));      // Phi(-|a|)
+  for (int i = DEG - 1; i >= 0; --i) h = fmaf(h, t, 0.5f * ((DEG == 9) ? c9[i] : c5[i]));
+  const float q = t * h * ex2_approx(a * a * (-0.5f * kLog2e));             // Phi(-|a|)
   return a > 0.f ? 1.0f - q : q;
 }
 
+// degree of the fit by storage type: fp32 9, 16-bit 5
+template <typename T> constexpr int kPhiDegree = (sizeof(T) == 4) ? 9 : 5;
+
 template <int ACT, typename T> __device__ __forceinline__ float act_gate(float a) {
   if (ACT == ACT_SILU) return a * sigmoid_f32(a);
-  if (ACT == ACT_GELU) return a * normal_cdf<sizeof(T) == 4 ? 9 : 5>(a);
+  if (ACT == ACT_GELU) return a * normal_cdf<kPhiDegree<T>>(a);
   const float u2 = 1.5957691216057307117f * fmaf(0.044715f * a * a, a, a);      // 2 u
   return a * sigmoid_f32(u2);
 }

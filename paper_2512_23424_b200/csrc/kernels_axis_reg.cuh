@@ -200,6 +200,32 @@ __device__ __forceinline__ void axis_reg_load(const T* px, long long xstep, bool
       }
       if (KEEP) raw[r] = A::pack(v);
     }
+  } else if (OP == OP_LAYERNORM && sizeof(T) == 2) {
+    // 16-bit storage: one sweep of sums shifted by the thread's first row, k = x[0]:
+    //   mean = k + S1 / n,  M2 = S2 - S1^2 / n  with S1 = sum (x - k), S2 = sum (x - k)^2.
+    // k lies among the data, so S2 exceeds M2 by n (mean - k)^2 only and the subtraction costs a
+    // few of fp32's bits, far inside the 2^-9 of the stored result; it saves an unpack and an
+    // operation per element against the exact two sweeps that fp32 storage keeps.
+    float k[W];
+    A::unpack(raw[0], k);
+#pragma unroll
+    for (int j = 0; j < W; ++j) { sa[j] = 0.f; sb[j] = 0.f; }
+#pragma unroll
+    for (int r = 1; r < R; ++r) {
+      if (FULL || r < nt) {
+        float v[W];
+        A::unpack(raw[r], v);
+#pragma unroll
+        for (int j = 0; j < W; ++j) { const float d = v[j] - k[j]; sa[j] += d; sb[j] = fmaf(d, d, sb[j]); }
+      }
+    }
+    const float inv_nt = FULL ? (1.0f / R) : ((nt > 0) ? __frcp_rn(static_cast<float>(nt)) : 0.f);
+#pragma unroll
+    for (int j = 0; j < W; ++j) {
+      const float m = sa[j] * inv_nt;                         // mean - k
+      sb[j] = fmaxf(fmaf(-sa[j], m, sb[j]), 0.f);
+      sa[j] = (FULL || nt > 0) ? k[j] + m : 0.f;
+    }
   } else if (OP == OP_LAYERNORM) {
 #pragma unroll
     for (int j = 0; j < W; ++j) { sa[j] = 0.f; sb[j] = 0.f; }
@@ -247,9 +273,12 @@ __device__ __forceinline__ void axis_reg_store(T* py, long long ystep, bool acti
   using E = Elem<T>;
   constexpr int W = A::W;
   constexpr bool KEEP = (OP == OP_SOFTMAX) && A::kFloatRaw;
-  float ncp[W];                              // softmax from packed values: exp2(x log2e - C) / S
+  // softmax from packed values: exp2(x log2e - C) / S with ncp = -C; 16-bit LayerNorm: (x - mean) rstd as
+  // one fused multiply-add with ncp = -mean rstd (rounding 2^-24 |mean| rstd, far inside the stored 2^-9)
+  constexpr bool kFusedCentre = (OP == OP_LAYERNORM) && (sizeof(T) == 2);
+  float ncp[W];
 #pragma unroll
-  for (int j = 0; j < W; ++j) ncp[j] = -cp[j];
+  for (int j = 0; j < W; ++j) ncp[j] = kFusedCentre ? -cp[j] * cq[j] : -cp[j];
 #pragma unroll
   for (int r = 0; r < R; ++r, py += ystep) {
     if (FULL || (active && r < nt)) {
@@ -264,7 +293,8 @@ __device__ __forceinline__ void axis_reg_store(T* py, long long ystep, bool acti
       for (int j = 0; j < W; ++j) {
         if (OP == OP_SOFTMAX) v[j] = (KEEP ? v[j] : ex2_approx(fmaf(v[j], kLog2e, ncp[j]))) * cq[j];
         else if (OP == OP_LOG_SOFTMAX) v[j] = (v[j] - cp[j]) - cq[j];
-        else if (OP == OP_LAYERNORM) v[j] = (v[j] - cp[j]) * cq[j] * g + be;
+        else if (OP == OP_LAYERNORM) v[j] = kFusedCentre ? fmaf(fmaf(v[j], cq[j], ncp[j]), g, be)
+                                                         : (v[j] - cp[j]) * cq[j] * g + be;
         else v[j] = v[j] * cq[j] * g;
       }
       A::store(py, A::pack(v));

@@ -124,6 +124,11 @@ __device__ __forceinline__ void norm_row_full(const RowParams& p, long long row,
     rstd = rsqrt_refined(fmaf(m2, inv_cols, p.eps));
   }
 
+  // 16-bit storage: (x - mean) * rstd as one fused multiply-add with the row constant -mean * rstd
+  // (its rounding, 2^-24 |mean| rstd, is far inside the 2^-9 of the stored result); fp32 keeps
+  // the exact difference
+  constexpr bool kFusedCentre = (sizeof(T) == 2);
+  const float neg_mean_rstd = -mean * rstd;
   const T* gp = reinterpret_cast<const T*>(p.gamma) + tg * EPV;
   const T* bp = reinterpret_cast<const T*>(p.beta) + tg * EPV;
 #pragma unroll
@@ -135,7 +140,8 @@ __device__ __forceinline__ void norm_row_full(const RowParams& p, long long row,
     if (OP == OP_LAYERNORM && p.beta != nullptr) E::unpack(ld_cached(bp + k * G * EPV), b);
 #pragma unroll
     for (int j = 0; j < EPV; ++j) {
-      if (OP == OP_LAYERNORM) o[j] = fmaf((v[k * EPV + j] - mean) * rstd, g[j], b[j]);
+      if (OP == OP_LAYERNORM) o[j] = kFusedCentre ? fmaf(fmaf(v[k * EPV + j], rstd, neg_mean_rstd), g[j], b[j])
+                                                  : fmaf((v[k * EPV + j] - mean) * rstd, g[j], b[j]);
       else o[j] = v[k * EPV + j] * rstd * g[j];
     }
     st_stream(yr + k * G * EPV, E::pack(o));
@@ -225,6 +231,8 @@ __global__ void __launch_bounds__(1024, 1) reg_norm_flex(const RowParams p, cons
     }
     float mean, rstd;
     flex_row_stats<OP, N>(v, red[parity], NW, inv_warps, inv_cols, p.eps, mean, rstd);
+    constexpr bool kFusedCentre = (sizeof(T) == 2);        // as in norm_row_full
+    const float neg_mean_rstd = -mean * rstd;
     const T* gp = reinterpret_cast<const T*>(p.gamma) + tg * EPV;
     const T* bp = reinterpret_cast<const T*>(p.beta) + tg * EPV;
 #pragma unroll
@@ -236,7 +244,8 @@ __global__ void __launch_bounds__(1024, 1) reg_norm_flex(const RowParams p, cons
       if (OP == OP_LAYERNORM && p.beta != nullptr) E::unpack(ld_cached(bp + static_cast<long long>(k) * G * EPV), b);
 #pragma unroll
       for (int j = 0; j < EPV; ++j) {
-        if (OP == OP_LAYERNORM) o[j] = fmaf((v[k * EPV + j] - mean) * rstd, g[j], b[j]);
+        if (OP == OP_LAYERNORM) o[j] = kFusedCentre ? fmaf(fmaf(v[k * EPV + j], rstd, neg_mean_rstd), g[j], b[j])
+                                                    : fmaf((v[k * EPV + j] - mean) * rstd, g[j], b[j]);
         else o[j] = v[k * EPV + j] * rstd * g[j];
       }
       st_stream(yr + static_cast<long long>(k) * G * EPV, E::pack(o));
