@@ -153,6 +153,10 @@ bool plan_reg(const Call& c, LaunchPlan* plan) {
     group = threads = 128; vpt = 2;
     // LayerNorm: grid-stride over 64 CTAs per SM measured 82 % against 71 % with a CTA per row
     if (c.op == OP_LAYERNORM) persist = sm_count() * 64;
+  } else if (want_warp && t_group == 0 && c.dtype != AKG_F32 && nvec > 192 && !norm_op) {
+    // the 16-bit softmax pair at 1544 .. 2048 columns: eight vectors per lane spill in the warp form
+    // (2048 columns: 69 % softmax, 73 % log-softmax against 86 % and 80 % with a CTA of 128 per row)
+    group = threads = 128; vpt = 2;
   } else if (want_warp && nvec <= 256) {
     group = 32; threads = 128;
     vpt = pow2_ceil(static_cast<int>((nvec + 31) / 32));
