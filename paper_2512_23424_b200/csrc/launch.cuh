@@ -67,6 +67,12 @@ cudaError_t launch_cumulative(bool want_prod, int dtype, bool vec, const void* x
                               long long cols, long long xs, long long ys, unsigned grid, int threads, bool warp_rows,
                               int pdl, cudaStream_t stream);
 
+// Short unmasked rows, 32 / lanes rows per warp (op_short.cu): lanes in {4, 8, 16, 32}, rows of
+// up to short_max_vectors(lanes) vectors.
+int short_rows_per_cta(int lanes);
+int short_max_vectors(int lanes);
+cudaError_t launch_short(int op, int dtype, int lanes, const RowParams& p, unsigned grid, int pdl, cudaStream_t stream);
+
 // BatchNorm-style column normalisation (op_colnorm.cu): two kernels, grid (column strips of
 // (1 << lc_shift) lanes, row blocks of p.rows_per_block rows).  colnorm_row_slots: rows a CTA walks at once.
 int colnorm_row_slots(int lc_shift);

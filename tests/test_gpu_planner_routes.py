@@ -212,3 +212,41 @@ def test_cumulative_routes(dtype):
             compare(got, ref, dtype, f"cumsum capped {cols}", tree_slack(cols, np.cumsum(np.abs(widen(x)), axis=1)))
     finally:
         akg.set_tuning("grid_cap", 0)
+
+
+# ---- short rows: several rows per warp ----------------------------------------------------------------
+
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("op", ["softmax", "log_softmax", "layernorm", "rmsnorm"])
+def test_short_rows_share_a_warp(op, dtype):
+    epv = 4 if dtype == wl.F32 else 8
+    norm = op in ("layernorm", "rmsnorm")
+    # vectors per row -> lanes per row: 1..16 -> 4, ..32 -> 8, ..64 -> 16, ..128 -> 32
+    for nv, lanes in ((1, 4), (3, 4), (16, 4), (17, 8), (32, 8), (33, 16), (50, 16), (64, 16), (80, 32), (112, 32)):
+        if nv > 64 and not norm and dtype == wl.F32 and nv > 96:
+            continue
+        for rows in (1, 37, 1031):                       # rows that do not fill the last warp or CTA
+            w = wl.make_random(op, dtype, rows, nv * epv, seed=390 + nv, loc=0.3, scale=1.7)
+            check(w, ("short<", f"l{lanes},"))
+    # non-finite rows keep the semantics of the other kernels: NaN rows, +inf rows, rows of -inf
+    w = wl.make_random(op, dtype, 8, 16 * epv, seed=399)
+    x = widen(w.x).copy()
+    x[1, 3] = np.nan
+    x[4, :] = 0.0
+    if not norm:                                         # infinities: pinned for the softmax pair only
+        x[2, 5] = np.inf
+        x[3, :] = -np.inf
+        x[5, 7] = -np.inf
+    w = dataclasses.replace(w, x=store(x.astype(np.float32), dtype))
+    check(w, ("short<",))
+    # strided rows and a grid smaller than the work
+    try:
+        akg.set_tuning("grid_cap", 2)
+        w = wl.make_random(op, dtype, 700, 24 * epv, seed=398)
+        check(w, ("short<", "grid2>"))
+    finally:
+        akg.set_tuning("grid_cap", 0)
+    # a mask sends the call back to the masked kernels
+    if not norm:
+        w = dataclasses.replace(wl.make_random(op, dtype, 64, 16 * epv, seed=397), causal_period=16)
+        got, name = check(w, ("reg<",))
