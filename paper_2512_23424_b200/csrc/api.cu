@@ -404,15 +404,18 @@ akg_status run(const Call& c, const char* name) {
 
   const int forced = g_forced_variant.load();
   const bool vec = vector_ok(c);
-  // Short unmasked rows (up to 64 vectors; normalisation rows below 128 vectors that are not a
+  // Short rows without an additive mask (up to 64 vectors; normalisation rows below 128 vectors that are not a
   // multiple of a warp): several rows per warp and four vectors per lane, see kernels_short.cuh.
-  if (forced == V_AUTO && vec && p.add == nullptr && !p.causal && g_tune_reg_general.load() == 0 &&
+  if (forced == V_AUTO && vec && p.add == nullptr && g_tune_reg_general.load() == 0 &&
       g_tune_reg_group.load() == 0) {
     const int64_t nv = c.cols / ((c.dtype == AKG_F32) ? 4 : 8);
     const bool norm = (c.op == OP_LAYERNORM || c.op == OP_RMSNORM);
     // (the softmax pair also up to 128 vectors in the 16-bit types, 96 in fp32: bf16 1024 columns 96 %
     // of the copy rate against 72 % with a warp per row, fp32 320 columns 94 % against 87 %)
-    if (nv <= 64 || (norm && nv < 128 && nv % 32 != 0) || (!norm && nv <= (c.dtype == AKG_F32 ? 96 : 128))) {
+    // under the causal rule only up to 64 vectors: beyond, the warp-per-row kernel's skipping of
+    // masked iterations is level or ahead (bf16 1024 columns: 67 % against 58 - 65 %)
+    if (nv <= 64 || (norm && nv < 128 && nv % 32 != 0) ||
+        (!norm && !p.causal && nv <= (c.dtype == AKG_F32 ? 96 : 128))) {
       int lanes = 4;
       while (lanes < 32 && short_max_vectors(lanes) < nv) lanes *= 2;
       const int64_t rpc = short_rows_per_cta(lanes);

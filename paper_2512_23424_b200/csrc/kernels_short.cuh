@@ -1,4 +1,4 @@
-// short_rows_kernel: rows of up to 128 vectors without a mask, several rows per warp.
+// short_rows_kernel: rows of up to 128 vectors, plain or under the causal rule, several rows per warp.
 //
 // A warp per row leaves most of a warp waiting when the row is one or two vectors per lane (a
 // bf16 row of 256 columns is 32 vectors): the row's latency chain (load, two reductions, store)
@@ -6,7 +6,9 @@
 // each (vector l, l + L, ...), so a warp works on 32 / L rows at once: four loads in flight
 // per lane whatever the row length, and reductions of log2 L shuffle steps.  Control flow is
 // uniform over the warp (lanes without a row or a vector compute on neutral values and skip
-// the store), so the shuffles always name the full warp.
+// the store), so the shuffles always name the full warp.  Under a causal mask a row's vectors
+// beyond its live prefix are not read, the masked part of the boundary vector counts as -inf and
+// masked outputs get the fill value (+0, -inf, or NaN for a NaN row), as in the register kernels.
 //
 // The arithmetic is that of the register kernels: softmax against the row maximum with one
 // exponential per element, log-softmax as scale (x - max) - ln S, LayerNorm with the exact two
@@ -32,7 +34,8 @@ template <int L> __device__ __forceinline__ float group_max(float v) {
 constexpr int kShortThreads = 128;
 constexpr int kShortVecs = 4;                 // vectors per lane
 
-template <int OP, typename T, int L>
+// CAUSAL: compiled with the causal rule (softmax pair only); the plain form carries none of its bookkeeping.
+template <int OP, typename T, int L, bool CAUSAL>
 __global__ void __launch_bounds__(kShortThreads, 8) short_rows_kernel(const RowParams p) {
   pdl_prologue();
   using E = Elem<T>;
@@ -57,15 +60,25 @@ __global__ void __launch_bounds__(kShortThreads, 8) short_rows_kernel(const RowP
     const bool have = row < p.rows;
     const T* xr = reinterpret_cast<const T*>(p.x) + row * p.xs + sub * EPV;
     T* yr = reinterpret_cast<T*>(p.y) + row * p.ys + sub * EPV;
+    static_assert(!CAUSAL || SM, "the causal rule belongs to the softmax pair");
+    const int live = (CAUSAL && have) ? static_cast<int>(live_cols(p, row)) : static_cast<int>(p.cols);
+    const bool masked = CAUSAL && live < static_cast<int>(p.cols);
+    bool in[K];                                    // vector k holds live data
+#pragma unroll
+    for (int k = 0; k < K; ++k) in[k] = have && ok[k] && (!CAUSAL || (sub + k * L) * EPV < live);
     uint4 raw[K];
 #pragma unroll
     for (int k = 0; k < K; ++k)
-      if (have && ok[k]) raw[k] = ld_stream(xr + k * L * EPV);
+      if (in[k]) raw[k] = ld_stream(xr + k * L * EPV);
     float v[K][EPV];
 #pragma unroll
     for (int k = 0; k < K; ++k) {
-      if (have && ok[k]) {
+      if (in[k]) {
         E::unpack(raw[k], v[k]);
+        if (masked) {
+#pragma unroll
+          for (int j = 0; j < EPV; ++j) if ((sub + k * L) * EPV + j >= live) v[k][j] = kNegInf;
+        }
       } else {
 #pragma unroll
         for (int j = 0; j < EPV; ++j) v[k][j] = SM ? kNegInf : 0.f;
@@ -94,6 +107,7 @@ __global__ void __launch_bounds__(kShortThreads, 8) short_rows_kernel(const RowP
       const bool dead = (M == kNegInf) && !(S != S);         // only -inf entries (a NaN row is not dead)
       const float scale = dead ? 0.f : __frcp_rn(S);
       const float lse = logf(S);
+      const float fill = (S != S) ? __int_as_float(0x7fc00000) : (OP == OP_SOFTMAX ? 0.f : kNegInf);
 #pragma unroll
       for (int k = 0; k < K; ++k) {
         float o[EPV];
@@ -101,6 +115,10 @@ __global__ void __launch_bounds__(kShortThreads, 8) short_rows_kernel(const RowP
         for (int j = 0; j < EPV; ++j) {
           if (OP == OP_SOFTMAX) o[j] = v[k][j] * scale;
           else o[j] = dead ? kNegInf : fmaf(v[k][j] - M, p.scale, -lse);
+        }
+        if (masked) {
+#pragma unroll
+          for (int j = 0; j < EPV; ++j) if ((sub + k * L) * EPV + j >= live) o[j] = fill;
         }
         if (have && ok[k]) st_stream(yr + k * L * EPV, E::pack(o));
       }

@@ -20,22 +20,30 @@ cudaError_t launch_short_k(K kernel, const RowParams& p, unsigned grid, int pdl,
   return cudaLaunchKernelEx(&cfg, kernel, p);
 }
 
-template <int OP, typename T>
+template <int OP, typename T, bool CAUSAL>
 cudaError_t launch_short_l(int lanes, const RowParams& p, unsigned grid, int pdl, cudaStream_t s) {
   switch (lanes) {
-    case 4: return launch_short_k(short_rows_kernel<OP, T, 4>, p, grid, pdl, s);
-    case 8: return launch_short_k(short_rows_kernel<OP, T, 8>, p, grid, pdl, s);
-    case 16: return launch_short_k(short_rows_kernel<OP, T, 16>, p, grid, pdl, s);
-    case 32: return launch_short_k(short_rows_kernel<OP, T, 32>, p, grid, pdl, s);
+    case 4: return launch_short_k(short_rows_kernel<OP, T, 4, CAUSAL>, p, grid, pdl, s);
+    case 8: return launch_short_k(short_rows_kernel<OP, T, 8, CAUSAL>, p, grid, pdl, s);
+    case 16: return launch_short_k(short_rows_kernel<OP, T, 16, CAUSAL>, p, grid, pdl, s);
+    case 32: return launch_short_k(short_rows_kernel<OP, T, 32, CAUSAL>, p, grid, pdl, s);
     default: return cudaErrorInvalidValue;
   }
 }
 
+template <int OP, typename T>
+cudaError_t launch_short_c(int lanes, const RowParams& p, unsigned grid, int pdl, cudaStream_t s) {
+  if constexpr (OpTraits<OP>::kSoftmaxLike) {
+    if (p.causal) return launch_short_l<OP, T, true>(lanes, p, grid, pdl, s);
+  }
+  return launch_short_l<OP, T, false>(lanes, p, grid, pdl, s);
+}
+
 template <int OP>
 cudaError_t launch_short_t(int dtype, int lanes, const RowParams& p, unsigned grid, int pdl, cudaStream_t s) {
-  if (dtype == DT_F32) return launch_short_l<OP, float>(lanes, p, grid, pdl, s);
-  if (dtype == DT_F16) return launch_short_l<OP, __half>(lanes, p, grid, pdl, s);
-  return launch_short_l<OP, __nv_bfloat16>(lanes, p, grid, pdl, s);
+  if (dtype == DT_F32) return launch_short_c<OP, float>(lanes, p, grid, pdl, s);
+  if (dtype == DT_F16) return launch_short_c<OP, __half>(lanes, p, grid, pdl, s);
+  return launch_short_c<OP, __nv_bfloat16>(lanes, p, grid, pdl, s);
 }
 
 }  // namespace

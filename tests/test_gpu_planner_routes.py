@@ -246,7 +246,21 @@ def test_short_rows_share_a_warp(op, dtype):
         check(w, ("short<", "grid2>"))
     finally:
         akg.set_tuning("grid_cap", 0)
-    # a mask sends the call back to the masked kernels
+    # the causal rule: live prefixes of every length, masked inputs poisoned, masked outputs exact
     if not norm:
-        w = dataclasses.replace(wl.make_random(op, dtype, 64, 16 * epv, seed=397), causal_period=16)
-        got, name = check(w, ("reg<",))
+        for nv, period in ((16, 16 * epv), (50, 37), (64, 1000)):
+            cols = nv * epv
+            rows = 3 * period + 5
+            w = dataclasses.replace(wl.make_random(op, dtype, rows, cols, seed=397 + nv), causal_period=period)
+            x = w.x.copy()
+            bad = np.float32(np.nan) if dtype == wl.F32 else (np.uint16(0x7FC0) if dtype == wl.BF16 else np.float16(np.nan))
+            live = np.minimum(np.arange(rows) % period + 1, cols)
+            for r in range(rows):
+                x[r, live[r]:] = bad
+            w = dataclasses.replace(w, x=x)
+            got, name = check(w, ("short<",))
+            dead = np.arange(cols)[None, :] >= live[:, None]
+            if op == "softmax":
+                assert_positive_zero(got, dead, name)
+            else:
+                assert np.all(np.isneginf(widen(got)[dead]))
