@@ -193,8 +193,8 @@ __device__ __forceinline__ void softmax_row_dispatch(const RowParams& p, long lo
 // the causal bf16 workload); wider CTAs keep the 64-register form without prefetch.
 template <int THREADS, int VPT> constexpr bool kSoftmaxPref = (VPT <= 2) || (VPT == 4 && THREADS <= 256);
 template <int G, int THREADS, int VPT> constexpr int kSoftmaxMinBlocks =
-    (G == THREADS && VPT == 4 && THREADS == 128) ? 6 : (G == THREADS && VPT == 4 && THREADS == 256) ? 3
-                                                                                                  : kRegMinBlocks<THREADS>;
+    (G == THREADS && VPT == 4 && THREADS == 128) ? 6
+    : (G == THREADS && (VPT == 4 || VPT == 8) && THREADS == 256) ? 3 : kRegMinBlocks<THREADS>;
 
 template <int OP, typename T, int G, int VPT, int THREADS>
 __global__ void __launch_bounds__(THREADS, kSoftmaxMinBlocks<G, THREADS, VPT>) reg_softmax(const RowParams p) {

@@ -20,7 +20,7 @@ namespace akg {
 #define AKG_REG_SHAPES(X) \
   X(32, 1, 128) X(32, 2, 128) X(32, 4, 128) X(32, 8, 128) \
   X(128, 1, 128) X(128, 2, 128) X(128, 4, 128) \
-  X(256, 1, 256) X(256, 2, 256) X(256, 4, 256) \
+  X(256, 1, 256) X(256, 2, 256) X(256, 4, 256) X(256, 8, 256) \
   X(512, 1, 512) X(512, 2, 512) X(512, 4, 512) X(512, 8, 512) \
   X(1024, 1, 1024) X(1024, 2, 1024) X(1024, 4, 1024) X(1024, 8, 1024)
 
