@@ -107,6 +107,8 @@ __global__ void __launch_bounds__(kShortThreads, 8) short_rows_kernel(const RowP
       const bool dead = (M == kNegInf) && !(S != S);         // only -inf entries (a NaN row is not dead)
       const float scale = dead ? 0.f : __frcp_rn(S);
       const float lse = logf(S);
+      const float m_out = dead ? 0.f : M, lse_out = dead ? 0.f : lse;   // a dead row comes out as -inf by itself
+      const float neg_shift = -fmaf(m_out, p.scale, lse_out);           // 16-bit log-softmax: one multiply-add per element
       const float fill = (S != S) ? __int_as_float(0x7fc00000) : (OP == OP_SOFTMAX ? 0.f : kNegInf);
 #pragma unroll
       for (int k = 0; k < K; ++k) {
@@ -114,7 +116,7 @@ __global__ void __launch_bounds__(kShortThreads, 8) short_rows_kernel(const RowP
 #pragma unroll
         for (int j = 0; j < EPV; ++j) {
           if (OP == OP_SOFTMAX) o[j] = v[k][j] * scale;
-          else o[j] = dead ? kNegInf : fmaf(v[k][j] - M, p.scale, -lse);
+          else o[j] = kFused ? fmaf(v[k][j], p.scale, neg_shift) : fmaf(v[k][j] - m_out, p.scale, -lse_out);
         }
         if (masked) {
 #pragma unroll

@@ -133,6 +133,13 @@ __device__ __forceinline__ void softmax_row(const RowParams& p, long long row, i
     lse_l = logf(S);
     fill = (S != S) ? nan : kNegInf;
   }
+  // 16-bit log-softmax: scale x - (scale M + ln S) as one fused multiply-add per element (the
+  // rounding of the bracket, 2^-24 of its magnitude, is inside the cancellation allowance of a
+  // 16-bit result); fp32 keeps the exact difference x - M
+  // a dead row (every entry -inf) must come out as -inf: with the row constants zeroed each
+  // element does that by itself (scale (-inf) - 0), and no element needs a select
+  const float m_out = dead ? 0.f : M, lse_out = dead ? 0.f : lse_l;
+  const float neg_shift = -fmaf(m_out, p.scale, lse_out);
   // the fill value as stored bits: +0, -inf or quiet NaN in the element type
   const uint32_t fill_word = E::fill_word(fill);
   const uint4 fill_vec = make_uint4(fill_word, fill_word, fill_word, fill_word);
@@ -150,7 +157,8 @@ __device__ __forceinline__ void softmax_row(const RowParams& p, long long row, i
 #pragma unroll
       for (int j = 0; j < EPV; ++j) {
         if (OP == OP_SOFTMAX) o[j] = v[k < NK ? k : 0][j] * scale;
-        else o[j] = dead ? kNegInf : fmaf(v[k < NK ? k : 0][j] - M, p.scale, -lse_l);
+        else o[j] = kFusedExponent ? fmaf(v[k < NK ? k : 0][j], p.scale, neg_shift)
+                                   : fmaf(v[k < NK ? k : 0][j] - m_out, p.scale, -lse_out);
       }
       if (k == NK - 1 && ragged && idx == live_vecs - 1) {
 #pragma unroll
