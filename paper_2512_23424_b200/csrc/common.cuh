@@ -303,7 +303,7 @@ template <int OP, int NW> __device__ __forceinline__ Stat cta_reduce(Stat s, Sta
 
 // Row scalars derived from the reduced statistics.
 //   softmax     : p = M (row max, or 0 if no live entry), q = 1 / S (0 if no live entry)
-//   log-softmax : p = M, q = ln S; dead = no live entry
+//   log-softmax : p = M, q = ln S (both 0 if no live entry); dead = no live entry
 //   LayerNorm   : p = mean, q = 1 / sqrt(var + eps)
 //   RMSNorm     : q = 1 / sqrt(mean square + eps)
 struct RowScalars { float p, q; bool dead; };
@@ -317,8 +317,8 @@ template <int OP> __device__ __forceinline__ RowScalars finalize(const Stat& s, 
     r.q = r.dead ? 0.f : 1.0f / s.b;
   } else if (OP == OP_LOG_SOFTMAX) {
     r.dead = (s.a == kNegInf) && !(s.b != s.b);   // a row of only NaN / -inf is a NaN row
-    r.p = s.a;
-    r.q = logf(s.b);
+    r.p = r.dead ? 0.f : s.a;                     // zeroed for a dead row: pre (-inf - 0) - 0 = -inf without a select
+    r.q = r.dead ? 0.f : logf(s.b);
   } else if (OP == OP_LAYERNORM) {
     r.p = s.b;
     r.q = 1.0f / sqrtf(s.c / static_cast<float>(cols) + eps);

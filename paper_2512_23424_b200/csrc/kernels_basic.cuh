@@ -15,7 +15,8 @@ template <int OP>
 __device__ __forceinline__ float apply_one(float z, const RowScalars& rs, float scale, float g, float b,
                                            float pre = 1.f) {
   if (OP == OP_SOFTMAX) return z * scale;                      // z holds exp(z - m_local)
-  if (OP == OP_LOG_SOFTMAX) return rs.dead ? kNegInf : fmaf(z - rs.p, pre, -rs.q);   // pre: the fused pre-scale
+  // pre: the fused pre-scale.  A dead row has p = q = 0 (see finalize), so its -inf entries come out as -inf
+  if (OP == OP_LOG_SOFTMAX) return fmaf(z - rs.p, pre, -rs.q);
   if (OP == OP_LAYERNORM) return (z - rs.p) * rs.q * g + b;
   return z * rs.q * g;
 }
