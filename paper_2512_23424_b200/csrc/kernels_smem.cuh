@@ -29,8 +29,12 @@ __device__ __forceinline__ void fold_vector(Stat& st, const float (&z)[EPV], flo
     const float mn = fmaxf(st.a, mv);
     const float ms = (mn == kNegInf) ? 0.f : mn;
     float acc = st.b * exp_diff(st.a, ms, l2e);
+    // vectors of eight are 16-bit storage: the exponent as one fused multiply-add (its rounding,
+    // below 1e-5 relative, is far inside the 2^-9 of the stored result); fp32 keeps the exact difference
+    constexpr bool kFused = (EPV == 8);
+    const float nms = -ms * l2e;
 #pragma unroll
-    for (int j = 0; j < EPV; ++j) acc += exp_diff(z[j], ms, l2e);
+    for (int j = 0; j < EPV; ++j) acc += kFused ? ex2_approx(fmaf(z[j], l2e, nms)) : exp_diff(z[j], ms, l2e);
     st.a = mn; st.b = acc;
   } else if (OP == OP_LAYERNORM) {
     float sum = 0.f;
@@ -60,10 +64,13 @@ __device__ __forceinline__ void fold_block(Stat& st, const float (&z)[4][EPV], f
     const float mn = fmaxf(st.a, mv);
     const float ms = (mn == kNegInf) ? 0.f : mn;
     float acc[4] = {st.b * exp_diff(st.a, ms, l2e), 0.f, 0.f, 0.f};
+    constexpr bool kFused = (EPV == 8);                    // as in fold_vector
+    const float nms = -ms * l2e;
 #pragma unroll
     for (int u = 0; u < 4; ++u)
 #pragma unroll
-      for (int j = 0; j < EPV; ++j) acc[u] += exp_diff(z[u][j], ms, l2e);
+      for (int j = 0; j < EPV; ++j)
+        acc[u] += kFused ? ex2_approx(fmaf(z[u][j], l2e, nms)) : exp_diff(z[u][j], ms, l2e);
     st.a = mn; st.b = (acc[0] + acc[1]) + (acc[2] + acc[3]);
   } else {
 #pragma unroll

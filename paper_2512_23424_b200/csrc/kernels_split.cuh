@@ -128,9 +128,11 @@ __device__ __forceinline__ uint4 split_apply_plain(const RowParams& p, const Row
     if (p.gamma != nullptr) E::unpack(ld_cached(reinterpret_cast<const T*>(p.gamma) + c0), ga);
     if (OP == OP_LAYERNORM && p.beta != nullptr) E::unpack(ld_cached(reinterpret_cast<const T*>(p.beta) + c0), be);
   }
+  constexpr bool kFused = (sizeof(T) == 2);               // 16-bit storage: exponent as one multiply-add
+  const float nml = -rs.p * p.l2e;
 #pragma unroll
   for (int j = 0; j < EPV; ++j) {
-    if (OP == OP_SOFTMAX) o[j] = exp_diff(z[j], rs.p, p.l2e) * rs.q;
+    if (OP == OP_SOFTMAX) o[j] = (kFused ? ex2_approx(fmaf(z[j], p.l2e, nml)) : exp_diff(z[j], rs.p, p.l2e)) * rs.q;
     else o[j] = apply_one<OP>(z[j], rs, 0.f, ga[j], be[j], p.scale);
   }
   return E::pack(o);
