@@ -72,6 +72,20 @@ __device__ __forceinline__ void fold_block(Stat& st, const float (&z)[4][EPV], f
       for (int j = 0; j < EPV; ++j)
         acc[u] += kFused ? ex2_approx(fmaf(z[u][j], l2e, nms)) : exp_diff(z[u][j], ms, l2e);
     st.a = mn; st.b = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+  } else if (OP == OP_LAYERNORM) {
+    // exact two sweeps over the 4 * EPV values of the block, then one merge with the running
+    // statistics (a merge per vector cost a division for every EPV values)
+    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+    for (int j = 0; j < EPV; ++j) { s0 += z[0][j]; s1 += z[1][j]; s2 += z[2][j]; s3 += z[3][j]; }
+    const float mean = ((s0 + s1) + (s2 + s3)) * (1.0f / (4 * EPV));
+    float q0 = 0.f, q1 = 0.f, q2 = 0.f, q3 = 0.f;
+#pragma unroll
+    for (int j = 0; j < EPV; ++j) {
+      const float d0 = z[0][j] - mean, d1 = z[1][j] - mean, d2 = z[2][j] - mean, d3 = z[3][j] - mean;
+      q0 = fmaf(d0, d0, q0); q1 = fmaf(d1, d1, q1); q2 = fmaf(d2, d2, q2); q3 = fmaf(d3, d3, q3);
+    }
+    st = stat_merge<OP>(st, Stat{static_cast<float>(4 * EPV), mean, (q0 + q1) + (q2 + q3)});
   } else {
 #pragma unroll
     for (int u = 0; u < 4; ++u) fold_vector<OP, EPV>(st, z[u], l2e);
