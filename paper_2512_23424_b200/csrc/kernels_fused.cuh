@@ -58,16 +58,27 @@ __global__ void __launch_bounds__(1024, 1) add_norm_flex(const RowParams p, cons
     flex_row_stats<OP, N>(v, red[parity], NW, inv_warps, inv_cols, p.eps, mean, rstd);
     const T* gp = reinterpret_cast<const T*>(p.gamma) + tg * EPV;
     const T* bp = reinterpret_cast<const T*>(p.beta) + tg * EPV;
+    // every affine vector present: no defaults to materialise per element (as in norm_row_full);
+    // 16-bit storage: the centring as one fused multiply-add with the row constant -mean * rstd
+    const bool affine_all = p.gamma != nullptr && (OP != OP_LAYERNORM || p.beta != nullptr);
+    constexpr bool kFusedCentre = (sizeof(T) == 2);
+    const float neg_mean_rstd = -mean * rstd;
 #pragma unroll
     for (int k = 0; k < VPT; ++k) {
       float g[EPV], b[EPV], o[EPV];
+      if (affine_all) {
+        E::unpack(ld_cached(gp + k * step), g);
+        if (OP == OP_LAYERNORM) E::unpack(ld_cached(bp + k * step), b);
+      } else {
 #pragma unroll
-      for (int j = 0; j < EPV; ++j) { g[j] = 1.f; b[j] = 0.f; }
-      if (p.gamma != nullptr) E::unpack(ld_cached(gp + k * step), g);
-      if (OP == OP_LAYERNORM && p.beta != nullptr) E::unpack(ld_cached(bp + k * step), b);
+        for (int j = 0; j < EPV; ++j) { g[j] = 1.f; b[j] = 0.f; }
+        if (p.gamma != nullptr) E::unpack(ld_cached(gp + k * step), g);
+        if (OP == OP_LAYERNORM && p.beta != nullptr) E::unpack(ld_cached(bp + k * step), b);
+      }
 #pragma unroll
       for (int j = 0; j < EPV; ++j) {
-        if (OP == OP_LAYERNORM) o[j] = fmaf((v[k * EPV + j] - mean) * rstd, g[j], b[j]);
+        if (OP == OP_LAYERNORM) o[j] = kFusedCentre ? fmaf(fmaf(v[k * EPV + j], rstd, neg_mean_rstd), g[j], b[j])
+                                                    : fmaf((v[k * EPV + j] - mean) * rstd, g[j], b[j]);
         else o[j] = v[k * EPV + j] * rstd * g[j];
       }
       st_stream(yr + k * step, E::pack(o));

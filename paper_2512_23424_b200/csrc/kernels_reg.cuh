@@ -131,13 +131,22 @@ __device__ __forceinline__ void norm_row_full(const RowParams& p, long long row,
   const float neg_mean_rstd = -mean * rstd;
   const T* gp = reinterpret_cast<const T*>(p.gamma) + tg * EPV;
   const T* bp = reinterpret_cast<const T*>(p.beta) + tg * EPV;
+  // every affine vector present (the usual call): unpack straight into the arithmetic; otherwise
+  // defaults are materialised per element first (two instructions per element that the usual call
+  // would pay for nothing: measured 1.75 of 16 instructions per bf16 LayerNorm element)
+  const bool affine_all = p.gamma != nullptr && (OP != OP_LAYERNORM || p.beta != nullptr);
 #pragma unroll
   for (int k = 0; k < VPT; ++k) {
     float g[EPV], b[EPV], o[EPV];
+    if (affine_all) {
+      E::unpack(ld_cached(gp + k * G * EPV), g);
+      if (OP == OP_LAYERNORM) E::unpack(ld_cached(bp + k * G * EPV), b);
+    } else {
 #pragma unroll
-    for (int j = 0; j < EPV; ++j) { g[j] = 1.f; b[j] = 0.f; }
-    if (p.gamma != nullptr) E::unpack(ld_cached(gp + k * G * EPV), g);
-    if (OP == OP_LAYERNORM && p.beta != nullptr) E::unpack(ld_cached(bp + k * G * EPV), b);
+      for (int j = 0; j < EPV; ++j) { g[j] = 1.f; b[j] = 0.f; }
+      if (p.gamma != nullptr) E::unpack(ld_cached(gp + k * G * EPV), g);
+      if (OP == OP_LAYERNORM && p.beta != nullptr) E::unpack(ld_cached(bp + k * G * EPV), b);
+    }
 #pragma unroll
     for (int j = 0; j < EPV; ++j) {
       if (OP == OP_LAYERNORM) o[j] = kFusedCentre ? fmaf(fmaf(v[k * EPV + j], rstd, neg_mean_rstd), g[j], b[j])
@@ -235,13 +244,19 @@ __global__ void __launch_bounds__(1024, 1) reg_norm_flex(const RowParams p, cons
     const float neg_mean_rstd = -mean * rstd;
     const T* gp = reinterpret_cast<const T*>(p.gamma) + tg * EPV;
     const T* bp = reinterpret_cast<const T*>(p.beta) + tg * EPV;
+    const bool affine_all = p.gamma != nullptr && (OP != OP_LAYERNORM || p.beta != nullptr);   // as in norm_row_full
 #pragma unroll
     for (int k = 0; k < VPT; ++k) {
       float g[EPV], b[EPV], o[EPV];
+      if (affine_all) {
+        E::unpack(ld_cached(gp + static_cast<long long>(k) * G * EPV), g);
+        if (OP == OP_LAYERNORM) E::unpack(ld_cached(bp + static_cast<long long>(k) * G * EPV), b);
+      } else {
 #pragma unroll
-      for (int j = 0; j < EPV; ++j) { g[j] = 1.f; b[j] = 0.f; }
-      if (p.gamma != nullptr) E::unpack(ld_cached(gp + static_cast<long long>(k) * G * EPV), g);
-      if (OP == OP_LAYERNORM && p.beta != nullptr) E::unpack(ld_cached(bp + static_cast<long long>(k) * G * EPV), b);
+        for (int j = 0; j < EPV; ++j) { g[j] = 1.f; b[j] = 0.f; }
+        if (p.gamma != nullptr) E::unpack(ld_cached(gp + static_cast<long long>(k) * G * EPV), g);
+        if (OP == OP_LAYERNORM && p.beta != nullptr) E::unpack(ld_cached(bp + static_cast<long long>(k) * G * EPV), b);
+      }
 #pragma unroll
       for (int j = 0; j < EPV; ++j) {
         if (OP == OP_LAYERNORM) o[j] = kFusedCentre ? fmaf(fmaf(v[k * EPV + j], rstd, neg_mean_rstd), g[j], b[j])
