@@ -156,20 +156,14 @@ __global__ void __launch_bounds__(kShortThreads, 8) short_rows_kernel(const RowP
       const float neg_mean_rstd = -mean * rstd;
       const T* gp = reinterpret_cast<const T*>(p.gamma) + sub * EPV;
       const T* bp = reinterpret_cast<const T*>(p.beta) + sub * EPV;
-      const bool affine_all = p.gamma != nullptr && (OP != OP_LAYERNORM || p.beta != nullptr);
 #pragma unroll
       for (int k = 0; k < K; ++k) {
         if (have && ok[k]) {
           float g[EPV], b[EPV], o[EPV];
-          if (affine_all) {                                  // no defaults to materialise per element
-            E::unpack(ld_cached(gp + k * L * EPV), g);
-            if (OP == OP_LAYERNORM) E::unpack(ld_cached(bp + k * L * EPV), b);
-          } else {
 #pragma unroll
-            for (int j = 0; j < EPV; ++j) { g[j] = 1.f; b[j] = 0.f; }
-            if (p.gamma != nullptr) E::unpack(ld_cached(gp + k * L * EPV), g);
-            if (OP == OP_LAYERNORM && p.beta != nullptr) E::unpack(ld_cached(bp + k * L * EPV), b);
-          }
+          for (int j = 0; j < EPV; ++j) { g[j] = 1.f; b[j] = 0.f; }
+          if (p.gamma != nullptr) E::unpack(ld_cached(gp + k * L * EPV), g);
+          if (OP == OP_LAYERNORM && p.beta != nullptr) E::unpack(ld_cached(bp + k * L * EPV), b);
 #pragma unroll
           for (int j = 0; j < EPV; ++j) {
             if (OP == OP_LAYERNORM) o[j] = kFused ? fmaf(fmaf(v[k][j], rstd, neg_mean_rstd), g[j], b[j])
