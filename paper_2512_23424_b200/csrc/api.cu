@@ -1024,7 +1024,9 @@ extern "C" akg_status akg_act_mul(akg_act act, const void* x, void* y, int64_t r
   ActParams p;
   p.x = x; p.y = y; p.rows = rows; p.d = d; p.xs = x_row_stride; p.ys = y_row_stride;
   const int64_t epv = 16 / es;
+  // (the vector kernel indexes a row's vectors with 32 bits)
   const bool vec = g_forced_variant.load() != V_STREAM && d % epv == 0 && aligned16(x) && aligned16(y) &&
+                   d / epv <= (int64_t(1) << 29) &&
                    (rows == 1 || ((x_row_stride * es) % 16 == 0 && (y_row_stride * es) % 16 == 0));
   const int64_t lanes = vec ? d / epv : d;
   const int u = act_mul_unroll();
