@@ -204,6 +204,13 @@ bool plan_reg(const Call& c, LaunchPlan* plan) {
     const int max_vpt = (c.dtype == AKG_F32) ? 8 : 4;
     int best_vpt = 0;
     int64_t best_g = 0;
+    // 16-bit rows of 9216 .. 16384 columns: eight vectors per thread in a CTA of up to 256 fat threads
+    // (128 registers) instead of 288 .. 512 threads of four
+    // (RMSNorm: 12288 columns 69 -> 77 %, 14336: 72 -> 82 %, 16384: 82 % with the ring -> 86 %; LayerNorm level, not taken)
+    if (c.dtype != AKG_F32 && c.op == OP_RMSNORM && g_tune_reg_flex.load() != 4 && nvec > 1024 && nvec % 8 == 0 &&
+        (nvec / 8) % 32 == 0 && nvec / 8 <= 256) {
+      best_vpt = 8; best_g = nvec / 8;
+    }
     // fewer, fatter threads measured best (the per-row reduction is paid per thread): take
     // the largest vectors-per-thread that leaves at least 128 threads, else whatever fits
     // (one vector per thread only as a last resort: 1536 16-bit columns ran at 38 - 44 % as 192 x 1)
@@ -447,7 +454,7 @@ akg_status run(const Call& c, const char* name) {
   //   longer aligned rows -> two-pass split cluster kernel (second pass from L2)
   //   anything unaligned -> scalar stream kernel
   if (forced == V_AUTO && vec && c.dtype != AKG_F32 && c.op == OP_RMSNORM &&
-      c.rows >= 2048 && c.cols >= 2048 && g_tune_tma_mode.load() != 2) {
+      c.rows >= 2048 && c.cols >= 2048 && c.cols <= 8192 && g_tune_tma_mode.load() != 2) {   // beyond: fat threads (plan_reg)
     planned = plan_ring(c, &plan);
     if (planned) {
       if (g_tune_smem_nbuf.load() == 0) {                  // one buffer per CTA measured best

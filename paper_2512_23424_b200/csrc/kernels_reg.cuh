@@ -211,8 +211,11 @@ __device__ __forceinline__ void flex_row_stats(const float (&v)[N], float (*red)
 // A CTA per row.  Every warp holds the same number of values, so the warps' (mean, M2)
 // pairs combine without divisions:  mean = avg(mean_w),  M2 = sum(M2_w) + c * sum((mean_w - mean)^2)
 // with c = values per warp; every thread reads the NW pairs from shared memory.
+// (64 values per thread, i.e. eight 16-bit vectors, are only launched with up to 256 threads and get
+// 128 registers; everything else keeps the 64-register bound of a full-size CTA)
 template <int OP, typename T, int VPT>
-__global__ void __launch_bounds__(1024, 1) reg_norm_flex(const RowParams p, const float inv_warps) {
+__global__ void __launch_bounds__((VPT * Elem<T>::EPV >= 64) ? 256 : 1024, (VPT * Elem<T>::EPV >= 64) ? 2 : 1)
+reg_norm_flex(const RowParams p, const float inv_warps) {
   pdl_prologue();
   using E = Elem<T>;
   constexpr int EPV = E::EPV;
