@@ -3,15 +3,21 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
-A step is one launch of the headline operator (LayerNorm fp32 [4096, 4096], the
-second benchmark configuration) through the C ABI on inputs already resident in
-HBM; successive steps rotate over four buffer pairs so the working set (512 MiB)
-exceeds L2.  The one JSON line printed by rank 0 carries the headline number,
-the same figure for every configuration (`per_config`) and for the operators
-over a non-last axis (`axis_rows`) and the fused residual add + normalisation
-(`fused_rows`), the gated activations (`act_rows`) and arg-max / cumulative operators
-(`reduction_rows`), the roofline fraction, the end-to-end figure
-with host buffers, and the fp64 CPU oracle's timing.
+A step is one launch of the headline operator - the causally masked bf16 softmax
+[32 x 4096, 4096], the largest of the five benchmark configurations - through the
+C ABI on inputs already resident in HBM (its 2 GiB working set exceeds L2 many
+times over).  The one JSON line printed by rank 0 carries the headline number and,
+inside `roofline`, one row per benchmark configuration (`per_config`) and per
+widened operator (`next_rows`: non-last axis, fused residual add + normalisation,
+gated activations, arg-max / cumulative operators, column normalisation, fp16
+storage).  Every row is timed three ways over at least 50 launches whatever
+--steps is: each launch inside its own CUDA event pair (`us_median`, `us_min`:
+the latency of one kernel), all launches back to back inside one event pair
+(`us_pipelined`: consecutive launches overlap through programmatic dependent
+launch, so this is a throughput), and a few launches each preceded by a 256 MiB
+fill that empties L2 (`us_cold_median`).  `frac` is algorithmic bytes / us_median /
+the measured copy peak.  Beside them the line carries the end-to-end figure with
+host buffers and the fp64 CPU oracle's timing.
 
 With N > 1 (launched by torch.distributed.run) every rank runs the same
 per-GPU workload on its own seed: rows are independent, there is no collective
@@ -35,7 +41,9 @@ if ROOT not in sys.path:
 from paper_2512_23424_b200 import workloads as wl  # noqa: E402
 
 METRIC = "achieved HBM GB/s (fraction of B200 peak) and rows/s per op and shape"
-HEADLINE = 2
+HEADLINE = 5
+HEADLINE_DTYPE = "bf16 I/O, fp32 accumulate"
+MIN_LAUNCHES = 50
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 L2_BYTES = 126 * 1000 * 1000
@@ -263,6 +271,63 @@ def time_launches(dw: DeviceWorkload, steps: int, warmup: int, barrier=None):
     return start.elapsed_time(stop) * 1e-3          # seconds
 
 
+def measure_row(obj, nbytes: int, peak: float, launches: int = MIN_LAUNCHES, warmup: int = 20, cold: int = 8):
+    """Three timings of `obj.launch()` (see the module docstring), as one table row."""
+    torch = obj.torch
+    launches = max(launches, MIN_LAUNCHES)
+    pipelined = time_launches(obj, launches, warmup) / launches
+    pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(launches)]
+    for a, b in pairs:                                   # one event pair per launch: no overlap between launches
+        a.record()
+        obj.launch()
+        b.record()
+    torch.cuda.synchronize()
+    each = np.array([a.elapsed_time(b) for a, b in pairs]) * 1e3
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    cold_pairs = pairs[:cold]
+    for a, b in cold_pairs:
+        flush.fill_(1)                                    # 256 MiB of stores: nothing of the inputs stays in L2
+        a.record()
+        obj.launch()
+        b.record()
+    torch.cuda.synchronize()
+    cold_us = np.array([a.elapsed_time(b) for a, b in cold_pairs]) * 1e3
+    del flush
+    us = float(np.median(each))
+    return {"us_median": us, "us_min": float(each.min()), "us_pipelined": pipelined * 1e6,
+            "us_cold_median": float(np.median(cold_us)), "launches": launches,
+            "gbs": nbytes / us / 1e3, "frac": nbytes / us / 1e3 / peak,
+            "frac_nominal": nbytes / us / 1e3 / NOMINAL_HBM_GBS,
+            "frac_pipelined": nbytes / pipelined / 1e9 / peak, "algorithmic_bytes": nbytes}
+
+
+def launch_floor_us(launches: int = 256, replays: int = 20) -> float:
+    """Device time per launch of the library's smallest call (one 4-element row) inside a CUDA
+    graph: what any launch costs on this stream before it moves a byte."""
+    import torch
+    from paper_2512_23424_b200 import binding
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        x = torch.zeros((1, 4), device="cuda")
+        call = binding.prepare("rmsnorm", x, torch.empty_like(x), eps=1e-6)
+        for _ in range(3):
+            call.launch()
+        stream.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            for _ in range(launches):
+                call.launch()
+        graph.replay()
+        stream.synchronize()
+        start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        start.record(stream)
+        for _ in range(replays):
+            graph.replay()
+        stop.record(stream)
+        stream.synchronize()
+    return start.elapsed_time(stop) * 1e3 / (launches * replays)
+
+
 def e2e_steps(w: wl.Workload, steps: int, warmup: int):
     """Same operator through the C ABI's host-buffer entry point: every step uploads the
     inputs from pinned host memory, runs the kernels and downloads the result, all inside
@@ -270,6 +335,7 @@ def e2e_steps(w: wl.Workload, steps: int, warmup: int):
     import torch
     from paper_2512_23424_b200 import binding
     tdt = torch.float32 if w.dtype == wl.F32 else torch.bfloat16
+    assert w.dtype in (wl.F32, wl.BF16)
 
     def host(a):
         if a is None:
@@ -347,6 +413,8 @@ def oracle_baseline(w: wl.Workload, budget_s: float = 12.0):
     run(probe_rows)                                           # page-in / thread start-up
     t_probe, _ = run(probe_rows)
     rows = int(min(w.rows, max(probe_rows, probe_rows * budget_s / max(t_probe, 1e-4))))
+    if w.causal_period > 0:                                   # whole causal periods: every live length equally often
+        rows = min(w.rows, max(w.causal_period, rows // w.causal_period * w.causal_period))
     # the sample is repeated until about budget_s of CPU time has been spent
     passes, secs, nbytes = 0, 0.0, 0
     while passes == 0 or (secs < budget_s and passes < 5000):
@@ -371,6 +439,101 @@ def slowest_rank(seconds: float, world: int, device: str) -> float:
 def whole_job_value(bytes_per_rank: int, world: int, seconds: float) -> float:
     """GB/s of the whole job: every rank moves bytes_per_rank in `seconds` (weak scaling)."""
     return bytes_per_rank * world / seconds / 1e9
+
+
+def _dev(a, dtype):
+    """Host array (float32 / float16, or uint16 bf16 bits) -> device tensor of the same bits."""
+    import torch
+    if a is None:
+        return None
+    if dtype in (wl.F32, wl.F16):
+        return torch.from_numpy(a).cuda()
+    return torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
+
+
+class _Rotating:
+    """`launch()` calls fn(k) for k cycling over n buffer sets."""
+
+    def __init__(self, torch, n, fn):
+        self.torch, self.n, self.fn, self.i = torch, n, fn, 0
+
+    def launch(self):
+        k = self.i % self.n
+        self.i += 1
+        return self.fn(k)
+
+
+def next_rows_table(peak: float):
+    """One row per widened operator (the "next" rows): same three timings as the five configurations."""
+    import torch
+    from paper_2512_23424_b200 import binding
+    rows = []
+
+    def add(name, obj, nbytes, **more):
+        row = {"workload": name}
+        row.update(measure_row(obj, nbytes, peak))
+        row["kernel"] = binding.last_kernel()
+        row["traffic"] = profiled_traffic(name)
+        row.update(more)
+        rows.append(row)
+        torch.cuda.empty_cache()
+
+    # configurations 3 and 5 stored as IEEE half (the paper's float16 regime)
+    for k in (3, 5):
+        wk = wl.as_f16(wl.make_config(k))
+        add(wk.name, DeviceWorkload(wk, pairs_for(wk)), wk.algorithmic_bytes())
+        del wk
+    # the operators over a non-last axis (the layout of the paper's RMSNorm sketch)
+    for name in wl.AXIS_CONFIGS:
+        wa = wl.make_axis(name)
+        add(name, AxisDeviceWorkload(wa, pairs_for(wa)), wa.algorithmic_bytes())
+        del wa
+    # fused residual add + normalisation (x and the residual in, y and the sum out)
+    for name in wl.FUSED_CONFIGS:
+        wf = wl.make_fused(name)
+        add(name, FusedDeviceWorkload(wf, pairs_for(wf)), wf.algorithmic_bytes())
+        del wf
+    # configuration 5 with its 1/sqrt(128) given to the call instead of baked into the input
+    ws = wl.make_scaled_causal()
+    xs0 = _dev(ws.x, ws.dtype)
+    ys0 = torch.empty_like(xs0)
+    mask = binding.make_mask(xs0, causal=True, causal_period=ws.causal_period)
+    scale = ws.extra["scale"]
+    add(ws.name, _Rotating(torch, 1, lambda k: binding.softmax_scaled(xs0, scale, out=ys0, mask=mask)),
+        ws.algorithmic_bytes(), scale=scale)
+    del xs0, ys0, ws
+    # gated activations (gate and factor in, product out)
+    for name in wl.ACT_CONFIGS:
+        wa = wl.make_act(name)
+        add(name, ActDeviceWorkload(wa, pairs_for(wa)), wa.algorithmic_bytes())
+        del wa
+    # arg-max / arg-min and cumulative sum / product over the last axis
+    for name in wl.REDUCTION_CONFIGS:
+        wr = wl.make_reduction(name)
+        fn = getattr(binding, wr.op)
+        x0 = _dev(wr.x, wr.dtype)
+        rxs = [x0] + [x0.clone() for _ in range(pairs_for(wr) - 1)]
+        routs = [fn(x) for x in rxs]
+        add(name, _Rotating(torch, len(rxs), lambda k: fn(rxs[k], out=routs[k])), wr.algorithmic_bytes())
+        del rxs, routs, x0, wr
+    # BatchNorm-style column normalisation: two kernels, x is read twice (the second time from L2
+    # while it fits), so the bound is three streams and `frac` counts three; `frac_two_streams`
+    # counts one read and one write
+    for name in wl.COLNORM_CONFIGS:
+        wc = wl.make_colnorm(name)
+        cx0 = _dev(wc.x, wc.dtype)
+        n_buf = 2 if 2 * cx0.numel() * cx0.element_size() >= 2 * L2_BYTES else 3
+        cxs = [cx0] + [cx0.clone() for _ in range(n_buf - 1)]
+        cys = [torch.empty_like(cx0) for _ in range(n_buf)]
+        cg, cb = _dev(wc.gamma, wc.dtype), _dev(wc.beta, wc.dtype)
+        cws = torch.empty(binding.colnorm_workspace_bytes(wc.rows, wc.cols) or 8, dtype=torch.uint8, device="cuda")
+        eps = wc.eps
+        two = 2 * wc.rows * wc.cols * wc.itemsize
+        add(name, _Rotating(torch, n_buf, lambda k: binding.colnorm(cxs[k], cg, cb, eps=eps, out=cys[k], workspace=cws)),
+            two * 3 // 2, bound="hbm, three streams (x read twice)", kernels_per_call=2)
+        rows[-1]["frac_two_streams"] = rows[-1]["frac"] * 2 / 3
+        del cxs, cys, cx0, wc
+    return rows
 
 
 def run_ours(args):
@@ -416,201 +579,68 @@ def run_ours(args):
     nbytes = w.algorithmic_bytes()
     gbs_one = nbytes / per_step / 1e9
     value = whole_job_value(nbytes, world, per_step)
+    working_set = len(dw.xs) * 2 * w.rows * w.cols * w.itemsize
 
     line = {
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": per_step * 1e3, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "scaling": "weak", "vs_baseline": None, "dtype": HEADLINE_DTYPE, "data": "synthetic",
         "config": {"workload": wl.CONFIG_NAMES[HEADLINE], "op": w.op, "rows": w.rows, "cols": w.cols,
-                   "io_dtype": "f32", "rows_per_s": w.rows * world / per_step, "kernel": kernel,
-                   "l2": f"rotating {len(dw.xs)} buffer pairs ({len(dw.xs) * 2 * w.rows * w.cols * w.itemsize >> 20} MiB > L2)",
+                   "io_dtype": "bf16", "causal_period": w.causal_period,
+                   "rows_per_s": w.rows * world / per_step, "kernel": kernel,
+                   "l2": f"{len(dw.xs)} buffer pair(s), working set {working_set >> 20} MiB > L2",
+                   "timing": "steps launched back to back (consecutive launches overlap through programmatic "
+                             "dependent launch); per-launch figures in roofline.per_config",
                    "parallelism": f"replicas x{world}, no collective"},
         "gpu_launches": args.steps,
         "clocks": sampler.summary(note),
     }
-    if rank == 0 and world == 1:
+    detail = rank == 0 and world == 1
+    if detail:
         line["roofline"] = {"bound": "hbm", "achieved": gbs_one, "peak": peak, "unit": "GB/s",
                             "frac": gbs_one / peak, "frac_nominal": gbs_one / NOMINAL_HBM_GBS,
                             "peak_kind": peak_kind, "traffic": profiled_traffic(wl.CONFIG_NAMES[HEADLINE]),
-                            "algorithmic_bytes": nbytes, "kernel": kernel}
+                            "algorithmic_bytes": nbytes, "kernel": kernel,
+                            "note": "achieved / frac: the timed region (pipelined launches); per_config[*].frac: "
+                                    "median of single launches, each in its own event pair"}
     # end to end with host buffers
     e2e_k = max(3, min(args.steps, 20))
     t_e2e, h2d, d2h = e2e_steps(w, e2e_k, args.warmup)
     t_e2e = max_over_ranks(t_e2e)
     line["e2e"] = {"value": nbytes * world / t_e2e / 1e9, "unit": "GB/s", "h2d_bytes_per_step": h2d,
-                   "d2h_bytes_per_step": d2h, "ms_per_step": t_e2e * 1e3, "steps": e2e_k}
+                   "d2h_bytes_per_step": d2h, "ms_per_step": t_e2e * 1e3, "steps": e2e_k,
+                   "copied_gbs": (h2d + d2h) * world / t_e2e / 1e9,
+                   "note": "value counts the algorithmic bytes (live reads + writes); copied_gbs counts the bytes "
+                           "that crossed PCIe (the whole input matrix is uploaded)"}
     del dw
     torch.cuda.empty_cache()
 
-    if rank == 0 and world == 1 and not args.headline_only:
+    if detail and not args.headline_only:
         table = []
         for k in (1, 2, 3, 4, 5):
             wk = w if k == HEADLINE else wl.make_config(k)
             dwk = DeviceWorkload(wk, pairs_for(wk))
-            # launches per configuration at the default --steps 1000; fewer steps scale them down
-            full = {1: 2000, 2: 1000, 3: 300, 4: 300, 5: 100}[k]
-            reps = max(10, min(full, full * args.steps // 1000))
-            sk = time_launches(dwk, reps, 10) / reps
-            bk = wk.algorithmic_bytes()
-            row = {"workload": wl.CONFIG_NAMES[k], "kernel": binding.last_kernel(), "us": sk * 1e6,
-                   "rows_per_s": wk.rows / sk, "launches": reps}
+            row = {"workload": wl.CONFIG_NAMES[k]}
+            row.update(measure_row(dwk, wk.algorithmic_bytes(), peak, launches=200 if k <= 2 else MIN_LAUNCHES))
+            row.update({"kernel": binding.last_kernel(), "rows_per_s": wk.rows / (row["us_median"] * 1e-6),
+                        "traffic": profiled_traffic(wl.CONFIG_NAMES[k])})
             if k == 1:
-                row["note"] = ("latency-bound (0.5 MiB, L2-resident); GB/s not meaningful; 'us' is paced by the "
-                               "host's launch rate, 'graph_us' is one launch inside a CUDA graph of 256")
-                row["graph_us"] = graph_launch_us(wk, replays=max(2, min(20, args.steps // 50)))
-            else:
-                row.update({"gbs": bk / sk / 1e9, "frac_measured": bk / sk / 1e9 / peak,
-                            "frac_nominal": bk / sk / 1e9 / NOMINAL_HBM_GBS, "algorithmic_bytes": bk,
-                            "traffic": profiled_traffic(wl.CONFIG_NAMES[k])})
+                for key in ("gbs", "frac", "frac_nominal", "frac_pipelined"):
+                    row.pop(key)
+                row["graph_us"] = graph_launch_us(wk, replays=10)
+                row["launch_floor_graph_us"] = launch_floor_us(replays=10)
+                row["note"] = ("latency-bound (0.5 MiB, L2-resident): no bandwidth figure; 'us_pipelined' is paced by "
+                               "the host's launch rate, 'graph_us' is one launch inside a CUDA graph of 256, "
+                               "'launch_floor_graph_us' the same for a one-vector call of this library")
             table.append(row)
             del dwk, wk
             torch.cuda.empty_cache()
-        line["per_config"] = table
-        # configurations 3 and 5 stored as IEEE half (the paper's float16 regime)
-        halves = []
-        for k in (3, 5):
-            wk = wl.as_f16(wl.make_config(k))
-            dwk = DeviceWorkload(wk, pairs_for(wk))
-            reps = max(10, min(100, 100 * args.steps // 1000))
-            sk = time_launches(dwk, reps, 5) / reps
-            bk = wk.algorithmic_bytes()
-            halves.append({"workload": wk.name, "kernel": binding.last_kernel(), "us": sk * 1e6, "gbs": bk / sk / 1e9,
-                           "frac_measured": bk / sk / 1e9 / peak, "algorithmic_bytes": bk, "launches": reps,
-                           "rows_per_s": wk.rows / sk})
-            del dwk, wk
-            torch.cuda.empty_cache()
-        line["fp16_rows"] = halves
-        # the operators over a non-last axis (the layout of the paper's RMSNorm sketch)
-        axis = []
-        for name in wl.AXIS_CONFIGS:
-            wa = wl.make_axis(name)
-            dwa = AxisDeviceWorkload(wa, pairs_for(wa))
-            reps = max(10, min(100, 100 * args.steps // 1000))
-            sa = time_launches(dwa, reps, 5) / reps
-            ba = wa.algorithmic_bytes()
-            axis.append({"workload": name, "kernel": binding.last_kernel(), "us": sa * 1e6, "gbs": ba / sa / 1e9,
-                         "frac_measured": ba / sa / 1e9 / peak, "algorithmic_bytes": ba, "launches": reps,
-                         "traffic": profiled_traffic(name)})
-            del dwa, wa
-            torch.cuda.empty_cache()
-        line["axis_rows"] = axis
-        # fused residual add + normalisation (x and the residual in, y and the sum out)
-        fused = []
-        for name in wl.FUSED_CONFIGS:
-            wf = wl.make_fused(name)
-            dwf = FusedDeviceWorkload(wf, pairs_for(wf))
-            reps = max(10, min(100, 100 * args.steps // 1000))
-            sf = time_launches(dwf, reps, 5) / reps
-            bf = wf.algorithmic_bytes()
-            fused.append({"workload": name, "kernel": binding.last_kernel(), "us": sf * 1e6, "gbs": bf / sf / 1e9,
-                          "frac_measured": bf / sf / 1e9 / peak, "algorithmic_bytes": bf, "launches": reps,
-                          "rows_per_s": wf.x.shape[0] / sf, "traffic": profiled_traffic(name)})
-            del dwf, wf
-            torch.cuda.empty_cache()
-        # configuration 5 with its 1/sqrt(128) given to the call instead of baked into the input
-        ws = wl.make_scaled_causal()
-        xs0 = torch.from_numpy(ws.x.view(np.int16)).cuda().view(torch.bfloat16)
-        ys0 = torch.empty_like(xs0)
-        mask = binding.make_mask(xs0, causal=True, causal_period=ws.causal_period)
-
-        class _Scaled:
-            def launch(self):
-                return binding.softmax_scaled(xs0, ws.extra["scale"], out=ys0, mask=mask)
-
-        _Scaled.torch = torch
-        reps = max(10, min(100, 100 * args.steps // 1000))
-        ss_ = time_launches(_Scaled(), reps, 5) / reps
-        bs_ = ws.algorithmic_bytes()
-        fused.append({"workload": ws.name, "kernel": binding.last_kernel(), "us": ss_ * 1e6, "gbs": bs_ / ss_ / 1e9,
-                      "frac_measured": bs_ / ss_ / 1e9 / peak, "algorithmic_bytes": bs_, "launches": reps,
-                      "rows_per_s": ws.rows / ss_, "scale": ws.extra["scale"], "traffic": None})
-        del xs0, ys0, ws
-        torch.cuda.empty_cache()
-        line["fused_rows"] = fused
-        # gated activations (gate and factor in, product out)
-        acts = []
-        for name in wl.ACT_CONFIGS:
-            wa = wl.make_act(name)
-            dwa = ActDeviceWorkload(wa, pairs_for(wa))
-            reps = max(10, min(100, 100 * args.steps // 1000))
-            sa = time_launches(dwa, reps, 5) / reps
-            ba = wa.algorithmic_bytes()
-            acts.append({"workload": name, "kernel": binding.last_kernel(), "us": sa * 1e6, "gbs": ba / sa / 1e9,
-                         "frac_measured": ba / sa / 1e9 / peak, "algorithmic_bytes": ba, "launches": reps,
-                         "rows_per_s": wa.x.shape[0] / sa, "traffic": profiled_traffic(name)})
-            del dwa, wa
-            torch.cuda.empty_cache()
-        line["act_rows"] = acts
-        # arg-max / arg-min and cumulative sum / product over the last axis
-        reds = []
-        for name in wl.REDUCTION_CONFIGS:
-            wr = wl.make_reduction(name)
-            fn = getattr(binding, wr.op)
-            n_buf = pairs_for(wr)
-            if wr.dtype == wl.F32:
-                x0 = torch.from_numpy(wr.x).cuda()
-            else:
-                x0 = torch.from_numpy(wr.x.view(np.int16)).cuda().view(torch.bfloat16)
-            rxs = [x0] + [x0.clone() for _ in range(n_buf - 1)]
-            routs = [fn(x) for x in rxs]
-
-            class _Red:
-                i = 0
-
-                def launch(self):
-                    k = self.i % len(rxs)
-                    self.i += 1
-                    return fn(rxs[k], out=routs[k])
-
-            _Red.torch = torch
-            reps = max(10, min(100, 100 * args.steps // 1000))
-            sr = time_launches(_Red(), reps, 5) / reps
-            br = wr.algorithmic_bytes()
-            reds.append({"workload": name, "kernel": binding.last_kernel(), "us": sr * 1e6, "gbs": br / sr / 1e9,
-                         "frac_measured": br / sr / 1e9 / peak, "algorithmic_bytes": br, "launches": reps,
-                         "rows_per_s": wr.x.shape[0] / sr, "traffic": profiled_traffic(name)})
-            del rxs, routs, x0, wr
-            torch.cuda.empty_cache()
-        line["reduction_rows"] = reds
-        # BatchNorm-style column normalisation (two kernels; x is read twice, the second time from
-        # L2 while it fits: `gbs` counts one read and one write, `gbs_three_streams` all three)
-        colrows = []
-        for name in wl.COLNORM_CONFIGS:
-            wc = wl.make_colnorm(name)
-            cdt = torch.float32 if wc.dtype == wl.F32 else torch.bfloat16
-
-            def cdev(a):
-                if wc.dtype == wl.F32:
-                    return torch.from_numpy(a).cuda()
-                return torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
-
-            cx0 = cdev(wc.x)
-            n_buf = 2 if 2 * cx0.numel() * cx0.element_size() >= 2 * L2_BYTES else 3
-            cxs = [cx0] + [cx0.clone() for _ in range(n_buf - 1)]
-            cys = [torch.empty_like(cx0) for _ in range(n_buf)]
-            cg, cb = cdev(wc.gamma), cdev(wc.beta)
-            cws = torch.empty(binding.colnorm_workspace_bytes(wc.rows, wc.cols) or 8, dtype=torch.uint8, device="cuda")
-
-            class _Col:
-                i = 0
-
-                def launch(self):
-                    k = self.i % len(cxs)
-                    self.i += 1
-                    return binding.colnorm(cxs[k], cg, cb, eps=wc.eps, out=cys[k], workspace=cws)
-
-            _Col.torch = torch
-            binding.colnorm(cxs[0], cg, cb, eps=wc.eps, out=cys[0], workspace=cws)      # sets the ctypes signatures
-            reps = max(10, min(100, 100 * args.steps // 1000))
-            sc = time_launches(_Col(), reps, 5) / reps
-            bc = 2 * wc.rows * wc.cols * wc.itemsize
-            colrows.append({"workload": name, "kernel": binding.last_kernel(), "us": sc * 1e6, "gbs": bc / sc / 1e9,
-                            "frac_measured": bc / sc / 1e9 / peak, "gbs_three_streams": 1.5 * bc / sc / 1e9,
-                            "algorithmic_bytes": bc, "launches": 2 * reps, "rows_per_s": wc.rows / sc})
-            del cxs, cys, cx0, wc
-            torch.cuda.empty_cache()
-        line["colnorm_rows"] = colrows
-    if rank == 0 and world == 1:
+        line["roofline"]["per_config"] = table
+        large = [r for r in table if "frac" in r]
+        line["roofline"]["min_frac"] = min(r["frac"] for r in large)
+        line["roofline"]["min_frac_workload"] = min(large, key=lambda r: r["frac"])["workload"]
+        line["roofline"]["next_rows"] = next_rows_table(peak)
+    if detail:
         line["cpu_baseline"] = oracle_baseline(w)
     assert binding.device_status() == 0, "a device-side bounded wait expired"
     if rank == 0:
@@ -629,12 +659,13 @@ def run_reference(args):
     if rank != 0:
         return
     import oracle
-    w = wl.make_config(HEADLINE, rows=256)                   # bounded sample of the workload per step
+    full = wl.config_shape(HEADLINE)[0]
+    w = wl.make_config(HEADLINE, rows=4096)                  # one whole causal period (one head) per step
     cores = os.cpu_count() or 1
-    eps = float(np.float32(w.eps))
+    mask = oracle.Mask(causal=True, causal_period=w.causal_period)
 
     def step():
-        oracle.layernorm(w.x, w.gamma, w.beta, eps=eps, nthreads=cores)
+        oracle.softmax(w.x, mask=mask, nthreads=cores)
 
     for _ in range(max(args.warmup, 1)):
         step()
@@ -643,14 +674,15 @@ def run_reference(args):
         step()
     per_step = (time.perf_counter() - t0) / args.steps
     gbs = w.algorithmic_bytes() / per_step / 1e9
-    sample = f"first 256 of 4096 rows of {wl.CONFIG_NAMES[HEADLINE]} per step, OpenMP over rows"
+    sample = (f"first {w.rows} of {full} rows (one whole causal period) of {wl.CONFIG_NAMES[HEADLINE]} per step, "
+              "OpenMP over rows")
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_step * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
         "data": "synthetic",
         "config": {"workload": wl.CONFIG_NAMES[HEADLINE], "op": w.op, "rows": w.rows, "cols": w.cols,
-                   "io_dtype": "f32", "sample": sample},
+                   "io_dtype": "bf16", "causal_period": w.causal_period, "sample": sample},
         "gpu_launches": 0,
         "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": oracle.last_threads(), "kind": "oracle",
                          "sample": sample},
@@ -691,7 +723,14 @@ def run_profile(args):
                           "us_per_launch": secs / args.steps * 1e6, "launches": args.steps + max(args.warmup, 3),
                           "algorithmic_bytes": w.algorithmic_bytes()}))
         return
-    w = wl.make_config(args.profile, rows=args.profile_rows)
+    if args.profile_shape:
+        op, dname, rows, cols = args.profile_shape.split(":")
+        dtype = {"f32": wl.F32, "bf16": wl.BF16, "f16": wl.F16}[dname]
+        w = wl.make_random(op, dtype, int(rows), int(cols), seed=2512, loc=0.5, eps=1e-5)
+        name = w.name
+    else:
+        w = wl.make_config(args.profile, rows=args.profile_rows)
+        name = wl.CONFIG_NAMES[args.profile]
     if args.variant:
         binding.set_variant(args.variant)
     for item in filter(None, args.tune.split(",")):
@@ -699,7 +738,8 @@ def run_profile(args):
         binding.set_tuning(key, int(val))
     dw = DeviceWorkload(w, pairs_for(w) if args.profile_rows is None else 1)
     secs = time_launches(dw, args.steps, args.warmup)
-    print(json.dumps({"profile": wl.CONFIG_NAMES[args.profile], "rows": w.rows, "kernel": binding.last_kernel(),
+    print(json.dumps({"profile": name, "rows": w.rows, "kernel": binding.last_kernel(),
+                      "frac_of_copy_peak": w.algorithmic_bytes() / (secs / args.steps) / 1e9 / measured_peak()[0],
                       "us_per_launch": secs / args.steps * 1e6, "launches": args.steps + max(args.warmup, 3),
                       "algorithmic_bytes": w.algorithmic_bytes()}))
 
@@ -764,6 +804,8 @@ def main():
                     help="as --profile, for a gated-activation configuration (workloads.ACT_CONFIGS)")
     ap.add_argument("--profile-fused", default="", metavar="NAME",
                     help="as --profile, for a fused residual add + normalisation configuration (workloads.FUSED_CONFIGS)")
+    ap.add_argument("--profile-shape", default="", metavar="OP:DTYPE:ROWS:COLS",
+                    help="as --profile, for a seeded random matrix, e.g. layernorm:bf16:512:131072")
     ap.add_argument("--profile-rows", type=int, default=None,
                     help="truncate the rows of --profile (the outer axis of --profile-axis)")
     ap.add_argument("--variant", default="", help="force a kernel family in --profile mode")
@@ -776,7 +818,7 @@ def main():
             args.steps = 20
         run_sweep(args)
         return
-    if args.profile or args.profile_axis or args.profile_fused or args.profile_act:
+    if args.profile or args.profile_axis or args.profile_fused or args.profile_act or args.profile_shape:
         run_profile(args)
     elif args.impl == "reference":
         run_reference(args)

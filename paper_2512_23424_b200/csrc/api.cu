@@ -35,6 +35,8 @@ std::atomic<int> g_tune_axis_nc{0};       //   column blocks per CTA
 std::atomic<int> g_tune_axis_lc{0};       //   two-pass kernel: 1 + log2 of the lanes along the columns
 std::atomic<int> g_tune_host_chunks{0};   // host-buffer pipeline: chunks per call (0 = default)
 std::atomic<int> g_tune_host_min_kib{0};  //   smallest chunk in KiB (0 = default)
+std::atomic<int> g_tune_split_exchange{0};  // two-pass split kernel: 1 = cluster barrier per row instead of st.async + mbarrier
+std::atomic<int> g_tune_split_l2{0};        //   L2 priority scheme (see split_kernel)
 std::atomic<int> g_tune_axis_mode{0};     //   1 = 16-byte vectors, 2 = bf16 8-byte vectors widened, 3 = elements
 
 __device__ int g_status_word = 0;
@@ -336,11 +338,17 @@ bool plan_split(const Call& c, LaunchPlan* plan) {
   if (cs < 1 || cs > kMaxCluster || (cs & (cs - 1))) return false;
   while (cs > 1 && nvec / cs < threads) cs /= 2;          // keep at least one vector per thread
   plan->variant = V_CLUSTER; plan->threads = threads; plan->group = threads;
-  // slices are whole unrolled steps (4 vectors per thread) except the row's last one
+  // slices of one vector per thread more or less (a slice's ragged last step is predicated, so the
+  // CTAs of a cluster get equal work: rounding to whole unrolled steps of four vectors per thread
+  // gave 50304 fp32 columns slices of 4096 / 4096 / 4096 / 288 vectors)
   int64_t slice = (nvec + cs - 1) / cs;
-  if (slice >= 4 * threads) slice = (slice + 4 * threads - 1) / (4 * threads) * (4 * threads);
+  slice = (slice + threads - 1) / threads * threads;
   plan->vpt = static_cast<int>(slice);
   plan->cluster = cs; plan->stages = 0; plan->smem = 0;
+  // mode 1: the partials are exchanged under a cluster barrier per row (the first version); otherwise
+  // st.async + mbarrier
+  plan->mode = g_tune_split_exchange.load() == 1 ? 1 : 0;
+  plan->split_l2 = g_tune_split_l2.load();
   const int cap = g_tune_grid_cap.load();
   plan->grid = cap > 0 ? static_cast<unsigned>((cap / cs > 0 ? cap / cs : 1) * cs) : 0u;
   if (cap == 0) {
@@ -516,7 +524,8 @@ akg_status run(const Call& c, const char* name) {
                                  : ((plan.stages == 1 && (c.op == OP_LAYERNORM || c.op == OP_RMSNORM)) ? ",full" : ""));
   else if (plan.variant == V_TMA || plan.variant == V_CLUSTER)
     std::snprintf(t_kernel, sizeof t_kernel, "%s<%s,t%d,cs%d,nbuf%d,slice%d>",
-                  plan.variant == V_TMA ? (plan.mode == 1 ? "ring" : "tma") : (plan.stages == 0 ? "split" : "cluster"),
+                  plan.variant == V_TMA ? (plan.mode == 1 ? "ring" : "tma")
+                  : (plan.stages != 0 ? "cluster" : "split"),
                   dt, plan.threads,
                   plan.cluster, plan.stages, plan.vpt);
   else
@@ -750,6 +759,8 @@ akg_status akg_set_tuning(const char* key, int value) {
   else if (!std::strcmp(key, "axis_nc")) g_tune_axis_nc.store(value);
   else if (!std::strcmp(key, "axis_mode")) g_tune_axis_mode.store(value);
   else if (!std::strcmp(key, "axis_lc")) g_tune_axis_lc.store(value);
+  else if (!std::strcmp(key, "split_exchange")) g_tune_split_exchange.store(value);
+  else if (!std::strcmp(key, "split_l2")) g_tune_split_l2.store(value);
   else return fail(AKG_ERR_INVALID_ARG, "akg_set_tuning: unknown key %s", key);
   return AKG_OK;
 }

@@ -24,6 +24,15 @@ __device__ __forceinline__ uint64_t l2_policy_keep() {
   asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
   return pol;
 }
+__device__ __forceinline__ uint64_t l2_policy_normal() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+// Back to normal priority for the 128-byte line at p (which a "keep" load marked evict_last).
+__device__ __forceinline__ void l2_demote_line(const void* p) {
+  asm volatile("applypriority.global.L2::evict_normal [%0], 128;" :: "l"(p) : "memory");
+}
 __device__ __forceinline__ uint64_t l2_policy_drop() {
   uint64_t pol;
   asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
@@ -93,6 +102,20 @@ __device__ __forceinline__ void split_pass1(const RowParams& p, const SplitRow<T
       for (int u = 0; u < 4; ++u) E::unpack(raw[u], z[u]);
       fold_block<OP, EPV>(st, z, p.l2e);
     }
+    if (v < r.lv) {                     // the ragged last step: up to three loads, in flight together
+      uint4 raw[3];
+#pragma unroll
+      for (int u = 0; u < 3; ++u)
+        if (v + u * THREADS < r.lv) raw[u] = ld_hint(px + u * THREADS, keep);
+#pragma unroll
+      for (int u = 0; u < 3; ++u)
+        if (v + u * THREADS < r.lv) {
+          float z[EPV];
+          E::unpack(raw[u], z);
+          fold_vector<OP, EPV>(st, z, p.l2e);
+        }
+    }
+    return;
   }
   for (; v < r.lv; v += THREADS) {
     float z[EPV];
@@ -157,6 +180,17 @@ __device__ __forceinline__ void split_pass2(const RowParams& p, const SplitRow<T
       for (int u = 0; u < 4; ++u)
         st_stream(py + u * THREADS, split_apply_plain<OP, T>(p, rs, raw[u], (v0 + v + u * THREADS) * EPV));
     }
+    if (v < my_vecs) {                  // the ragged last step
+      uint4 raw[3];
+#pragma unroll
+      for (int u = 0; u < 3; ++u)
+        if (v + u * THREADS < my_vecs) raw[u] = ld_hint(px + u * THREADS, drop);
+#pragma unroll
+      for (int u = 0; u < 3; ++u)
+        if (v + u * THREADS < my_vecs)
+          st_stream(py + u * THREADS, split_apply_plain<OP, T>(p, rs, raw[u], (v0 + v + u * THREADS) * EPV));
+    }
+    return;
   }
   for (; v < my_vecs; v += THREADS) {
     float o[EPV];
@@ -194,19 +228,121 @@ __device__ __forceinline__ void split_pass2(const RowParams& p, const SplitRow<T
 }
 
 
+// LayerNorm with 16-bit storage folds the next row in ONE sweep: every thread accumulates
+// s1 = sum(x - K) and s2 = sum((x - K)^2) about a shift K of its own, the first element it owns in
+// the slice, and turns them into (count, mean, M2) once per row.  K being one of the thread's values,
+// (mean_t - K)^2 <= M2_t, hence s2 <= (n_t + 1) M2_t and the cancellation in M2_t = s2 - s1^2 / n_t
+// costs at most a relative (n_t + 1) 2^-24 (n_t is a few hundred: 1e-5), far inside the 2^-9 of a
+// 16-bit result; fp32 storage keeps the exact two sweeps per block of four vectors.  What is saved
+// is registers: the two sweeps hold 32 widened values at once and spilled 280 bytes.
+template <int OP, typename T> constexpr bool kShiftedStats = (OP == OP_LAYERNORM && sizeof(T) == 2);
+
+// (K, s1, s2) over n values -> (count, mean, M2)
+__device__ __forceinline__ Stat shifted_finish(const Stat& acc, int n) {
+  if (n <= 0) return Stat{0.f, 0.f, 0.f};
+  const float inv = 1.0f / static_cast<float>(n);
+  const float m = acc.b * inv;
+  return Stat{static_cast<float>(n), acc.a + m, fmaxf(acc.c - acc.b * m, 0.f)};
+}
+
+// One unrolled step of the merged loop on vectors v, v + THREADS, ... (four per thread) of two
+// unmasked rows: the loads of the cluster's next row (xn: HBM, "keep") and of the current row (xc:
+// L2, "drop") are issued by split_step_load; split_step_use normalises and stores the current row
+// and folds the next one.  PRED: the step is the slice's last, ragged one, and vector u takes part
+// only if v + u * THREADS < my_vecs.
+template <int THREADS, bool PRED>
+__device__ __forceinline__ void split_step_load(const uint4* xn, const uint4* xc, int v, int my_vecs, uint64_t keep,
+                                                uint64_t drop, uint4 (&rn)[4], uint4 (&rc)[4]) {
+#pragma unroll
+  for (int u = 0; u < 4; ++u)
+    if (!PRED || v + u * THREADS < my_vecs) rn[u] = ld_hint(xn + v + u * THREADS, keep);
+#pragma unroll
+  for (int u = 0; u < 4; ++u)
+    if (!PRED || v + u * THREADS < my_vecs) rc[u] = ld_hint(xc + v + u * THREADS, drop);
+}
+
+template <int OP, typename T, int THREADS, bool PRED>
+__device__ __forceinline__ void split_step_use(const RowParams& p, uint4* yc, const RowScalars& rs, int v0, int v,
+                                               int my_vecs, const uint4 (&rn)[4], const uint4 (&rc)[4], Stat& stn,
+                                               const uint4* demote = nullptr) {
+  using E = Elem<T>;
+  constexpr int EPV = E::EPV;
+  if (!PRED && demote != nullptr && (threadIdx.x & 7) == 0) {
+#pragma unroll
+    for (int u = 0; u < 4; ++u) l2_demote_line(demote + v + u * THREADS);
+  }
+#pragma unroll
+  for (int u = 0; u < 4; ++u)
+    if (!PRED || v + u * THREADS < my_vecs)
+      st_stream(yc + v + u * THREADS, split_apply_plain<OP, T>(p, rs, rc[u], (v0 + v + u * THREADS) * EPV));
+  if (kShiftedStats<OP, T>) {
+    // 16-bit LayerNorm: one sweep of sums about the thread's shift stn.a (see shifted_finish)
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      if (!PRED || v + u * THREADS < my_vecs) {
+        float z[EPV];
+        E::unpack(rn[u], z);
+#pragma unroll
+        for (int j = 0; j < EPV; ++j) {
+          const float d = z[j] - stn.a;
+          stn.b += d;
+          stn.c = fmaf(d, d, stn.c);
+        }
+      }
+  } else if (!PRED) {
+    float z[4][EPV];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) E::unpack(rn[u], z[u]);
+    fold_block<OP, EPV>(stn, z, p.l2e);
+  } else {
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      if (v + u * THREADS < my_vecs) {
+        float z[EPV];
+        E::unpack(rn[u], z);
+        fold_vector<OP, EPV>(stn, z, p.l2e);
+      }
+  }
+}
+
 // The row loop is software-pipelined: while a CTA writes row r (pass 2: L2 reads, HBM
 // writes) it already folds its slice of the cluster's next row (pass 1: HBM reads), four
 // vectors of each per thread and step, so that every warp keeps DRAM reads and writes in
 // flight at once and a row costs one trip through the slice instead of two.
+//
+// Exchange of the slices' partial statistics (xmode 1, the default): every CTA owns two
+// mbarriers (rows alternate between them).  After the CTA reduction, thread k < CS sends the
+// CTA's partial to CTA k with one 16-byte st.async, which lands in slot [parity][sender] of the
+// receiver's shared memory and counts 16 bytes on the receiver's mbarrier; a CTA waits on its
+// own mbarrier for CS x 16 bytes.  Nothing waits for the CTA's global stores (a cluster barrier's
+// release does: the profile showed it as membar stalls), and the first loads of the next step
+// are already in flight while a thread waits for the partials.  Reuse of a slot and of a phase
+// two rows later is ordered by the exchange itself: a peer can send row r + 2 only after it has
+// received this CTA's partial of row r + 1, which this CTA sends after all its threads have read
+// the slots of row r (the CTA reduction's barrier lies in between).
+// xmode 0 keeps the first version: plain remote stores and a cluster barrier per row.
+//
+// L2 priorities (l2mode 0, the default): pass 1 loads mark their lines "evict last", pass 2 loads
+// "evict first", and pass 2 also puts each 128-byte line it has consumed back to normal priority
+// (applypriority): in a run of back-to-back calls the lines marked by earlier calls otherwise stay
+// privileged and take the room of the rows in flight (config 4: 97.3 us without, 95.3 us with the
+// demotion).  l2mode 1: pass 1 with normal priority (97.4 us); l2mode 2: marks, no demotion.
+//
+// Waits are bounded (two seconds of the global timer).  A CTA whose wait runs out sets the status
+// word, stops storing and leaves the row loop; its peers run into the same limit one after the
+// other.  All CTAs of a cluster meet at a cluster barrier before they exit, so no partial is ever
+// sent to a CTA that has left.
 template <int OP, typename T, int THREADS>
 __global__ void __launch_bounds__(THREADS, (1024 / THREADS) > 0 ? (1024 / THREADS) : 1)
-split_kernel(const RowParams p, const int slice_vecs) {
+split_kernel(const RowParams p, const int slice_vecs, const int xmode, const int l2mode) {
   pdl_prologue();
   using E = Elem<T>;
   constexpr int EPV = E::EPV;
   constexpr int NW = THREADS / 32;
   __shared__ Stat red[2][NW];
   __shared__ Stat peers[2][kMaxCluster];
+  __shared__ __align__(16) float4 inbox[2][kMaxCluster];
+  __shared__ __align__(8) uint64_t xbar[2];
 
   const uint32_t cs = cluster_size();
   const uint32_t rank = cluster_rank();
@@ -214,19 +350,32 @@ split_kernel(const RowParams p, const int slice_vecs) {
   const int nvec = static_cast<int>(p.cols / EPV);
   const int v0 = static_cast<int>(rank) * slice_vecs;
   const int my_vecs = max(0, min(slice_vecs, nvec - v0));
-  const uint64_t keep = l2_policy_keep();
+  const uint64_t keep = (l2mode == 1) ? l2_policy_normal() : l2_policy_keep();   // see split_kernel's comment
   const uint64_t drop = l2_policy_drop();
+  const bool async_x = (xmode != 0) && cs > 1;
 
-  if (cs > 1) {            // every CTA of the cluster is running before any remote store
+  if (cs > 1) {            // every CTA of the cluster is running (mbarriers set up) before any remote store
+    if (threadIdx.x == 0) {
+      mbar_init(smem_addr(&xbar[0]), 1);
+      mbar_init(smem_addr(&xbar[1]), 1);
+      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
     cluster_arrive();
     cluster_wait();
   }
 
   int par = 0;
-  // thread statistics of a slice -> statistics of the whole row, in every CTA of the cluster
-  auto row_stats = [&](Stat st) -> Stat {
+  uint32_t phases = 0;        // bit k: parity of the phase of xbar[k] that the next wait is for
+  bool failed = false;
+  // thread statistics of a slice -> this CTA's partial, sent to every CTA of the cluster
+  auto send_stats = [&](Stat st) -> Stat {
     st = cta_reduce<OP, NW>(st, red[par], p.l2e);
-    if (cs > 1) {
+    if (async_x) {
+      if (threadIdx.x == 0) mbar_expect_tx(smem_addr(&xbar[par]), cs * 16u);
+      if (threadIdx.x < cs)
+        st_async_f32x4(smem_addr(&inbox[par][rank]), smem_addr(&xbar[par]), threadIdx.x, st.a, st.b, st.c, 0.f);
+    } else if (cs > 1) {
       if (threadIdx.x < cs) {
         const uint32_t slot = smem_addr(&peers[par][rank]);
         st_remote_f32(slot, threadIdx.x, st.a);
@@ -234,6 +383,22 @@ split_kernel(const RowParams p, const int slice_vecs) {
         st_remote_f32(slot + 8, threadIdx.x, st.c);
       }
       cluster_arrive();
+    }
+    return st;
+  };
+  // ... and the statistics of the whole row, in every CTA of the cluster
+  auto recv_stats = [&](Stat st) -> Stat {
+    if (async_x) {
+      if (!mbar_wait_timed<true>(smem_addr(&xbar[par]), (phases >> par) & 1u, p.status)) failed = true;
+      phases ^= 1u << par;
+      const float4 f = inbox[par][0];
+      Stat r{f.x, f.y, f.z};
+      for (uint32_t k = 1; k < cs; ++k) {
+        const float4 g = inbox[par][k];
+        r = stat_merge<OP>(r, Stat{g.x, g.y, g.z}, p.l2e);
+      }
+      st = r;
+    } else if (cs > 1) {
       cluster_wait();
       Stat r = peers[par][0];
       for (uint32_t k = 1; k < cs; ++k) r = stat_merge<OP>(r, peers[par][k], p.l2e);
@@ -244,49 +409,94 @@ split_kernel(const RowParams p, const int slice_vecs) {
   };
 
   long long row = cluster_id();
-  if (row >= p.rows) return;
-  SplitRow<T> cur = split_row<OP, T>(p, row, v0, my_vecs);
-  Stat st = stat_identity<OP>();
-  split_pass1<OP, T, THREADS>(p, cur, v0, threadIdx.x, st, keep);
-  st = row_stats(st);
-
-  for (;;) {
-    const RowScalars rs = finalize<OP>(st, p.cols, p.eps);
-    const long long next_row = row + row_step;
-    const bool has_next = next_row < p.rows;
-    int v = threadIdx.x;
-    if (!has_next) {
-      split_pass2<OP, T, THREADS>(p, cur, rs, v0, my_vecs, v, drop);
-      break;
+  constexpr bool SM = OpTraits<OP>::kSoftmaxLike;
+  if (row < p.rows && (!SM || (p.add == nullptr && !p.causal))) {
+    // ---- no mask anywhere: every slice is whole, and a row's pointers follow from the previous row's
+    const long long dx = row_step * p.xs * static_cast<long long>(sizeof(T)) / 16;   // in vectors
+    const long long dy = row_step * p.ys * static_cast<long long>(sizeof(T)) / 16;
+    const uint4* xc = reinterpret_cast<const uint4*>(reinterpret_cast<const T*>(p.x) + row * p.xs) + v0;
+    uint4* yc = reinterpret_cast<uint4*>(reinterpret_cast<T*>(p.y) + row * p.ys) + v0;
+    Stat st = stat_identity<OP>();
+    {
+      SplitRow<T> first;
+      first.xr = reinterpret_cast<const T*>(xc); first.yr = reinterpret_cast<T*>(yc); first.ar = nullptr;
+      first.live = static_cast<int>(p.cols); first.lv = my_vecs; first.plain = true;
+      split_pass1<OP, T, THREADS>(p, first, v0, threadIdx.x, st, keep);
     }
-    const SplitRow<T> nxt = split_row<OP, T>(p, next_row, v0, my_vecs);
-    Stat stn = stat_identity<OP>();
-    if (cur.plain && nxt.plain && cur.lv == my_vecs && nxt.lv == my_vecs) {
-      const uint4* pn = reinterpret_cast<const uint4*>(nxt.xr) + v;
-      const uint4* px = reinterpret_cast<const uint4*>(cur.xr) + v;
-      uint4* py = reinterpret_cast<uint4*>(cur.yr) + v;
-      for (; v + 3 * THREADS < my_vecs; v += 4 * THREADS, pn += 4 * THREADS, px += 4 * THREADS, py += 4 * THREADS) {
-        uint4 rn[4], rc[4];
+    st = send_stats(st);
+    for (;; row += row_step, xc += dx, yc += dy) {
+      const bool has_next = row + row_step < p.rows;
+      const uint4* xn = xc + dx;
+      int v = threadIdx.x;
+      uint4 rn[4], rc[4];
+      const bool first_full = has_next && v + 3 * THREADS < my_vecs;
+      if (first_full) {                              // in flight while this thread waits for the partials
 #pragma unroll
-        for (int u = 0; u < 4; ++u) rn[u] = ld_hint(pn + u * THREADS, keep);
-#pragma unroll
-        for (int u = 0; u < 4; ++u) rc[u] = ld_hint(px + u * THREADS, drop);
-#pragma unroll
-        for (int u = 0; u < 4; ++u)
-          st_stream(py + u * THREADS, split_apply_plain<OP, T>(p, rs, rc[u], (v0 + v + u * THREADS) * EPV));
-        float z[4][EPV];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) E::unpack(rn[u], z[u]);
-        fold_block<OP, EPV>(stn, z, p.l2e);
+        for (int u = 0; u < 4; ++u) rn[u] = ld_hint(xn + v + u * THREADS, keep);
       }
+      st = recv_stats(st);
+      if (failed) break;
+      const RowScalars rs = finalize<OP>(st, p.cols, p.eps);
+      if (!has_next) {
+        SplitRow<T> last;
+        last.xr = reinterpret_cast<const T*>(xc); last.yr = reinterpret_cast<T*>(yc); last.ar = nullptr;
+        last.live = static_cast<int>(p.cols); last.lv = my_vecs; last.plain = true;
+        split_pass2<OP, T, THREADS>(p, last, rs, v0, my_vecs, v, drop);
+        break;
+      }
+      Stat stn = stat_identity<OP>();
+      if (kShiftedStats<OP, T> && v < my_vecs)       // the shift: the first element this thread owns
+        stn.a = Elem<T>::load1(xn + v, 0);
+      if (first_full) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) rc[u] = ld_hint(xc + v + u * THREADS, drop);
+        const uint4* demote = (l2mode == 0 && ((reinterpret_cast<uintptr_t>(xc) & 127u) == 0)) ? xc : nullptr;
+        split_step_use<OP, T, THREADS, false>(p, yc, rs, v0, v, my_vecs, rn, rc, stn, demote);
+        v += 4 * THREADS;
+        for (; v + 3 * THREADS < my_vecs; v += 4 * THREADS) {
+          split_step_load<THREADS, false>(xn, xc, v, my_vecs, keep, drop, rn, rc);
+          split_step_use<OP, T, THREADS, false>(p, yc, rs, v0, v, my_vecs, rn, rc, stn, demote);
+        }
+      }
+      if (v < my_vecs) {                             // the ragged last step: its loads in flight together
+        split_step_load<THREADS, true>(xn, xc, v, my_vecs, keep, drop, rn, rc);
+        split_step_use<OP, T, THREADS, true>(p, yc, rs, v0, v, my_vecs, rn, rc, stn);
+      }
+      if (kShiftedStats<OP, T>) {
+        const int t = static_cast<int>(threadIdx.x);
+        stn = shifted_finish(stn, t < my_vecs ? ((my_vecs - 1 - t) / THREADS + 1) * Elem<T>::EPV : 0);
+      }
+      st = send_stats(stn);
     }
-    // whatever the merged loop left (all of both passes when it did not run)
-    split_pass2<OP, T, THREADS>(p, cur, rs, v0, my_vecs, v, drop);
-    split_pass1<OP, T, THREADS>(p, nxt, v0, v, stn, keep);
-    st = row_stats(stn);
-    cur = nxt;
-    row = next_row;
+  } else if (row < p.rows) {
+    // ---- masked rows: slices may be cut short by the causal rule or carry an additive mask
+    SplitRow<T> cur = split_row<OP, T>(p, row, v0, my_vecs);
+    Stat st = stat_identity<OP>();
+    split_pass1<OP, T, THREADS>(p, cur, v0, threadIdx.x, st, keep);
+    st = send_stats(st);
+    for (;;) {
+      st = recv_stats(st);
+      if (failed) break;
+      const RowScalars rs = finalize<OP>(st, p.cols, p.eps);
+      const long long next_row = row + row_step;
+      if (next_row >= p.rows) {
+        split_pass2<OP, T, THREADS>(p, cur, rs, v0, my_vecs, threadIdx.x, drop);
+        break;
+      }
+      const SplitRow<T> nxt = split_row<OP, T>(p, next_row, v0, my_vecs);
+      Stat stn = stat_identity<OP>();
+      split_pass2<OP, T, THREADS>(p, cur, rs, v0, my_vecs, threadIdx.x, drop);
+      split_pass1<OP, T, THREADS>(p, nxt, v0, threadIdx.x, stn, keep);
+      st = send_stats(stn);
+      cur = nxt;
+      row = next_row;
+    }
+  }
+  if (cs > 1) {            // nobody leaves while a peer may still send to it
+    cluster_arrive();
+    cluster_wait();
   }
 }
+
 
 }  // namespace akg

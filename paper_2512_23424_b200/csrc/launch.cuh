@@ -22,6 +22,7 @@ struct LaunchPlan {
   size_t smem;        // dynamic shared memory per CTA
   int mode;           // V_TMA: 1 = register kernels fed by a ring, 0 = shared-memory-resident kernel
   int pdl;            // 1 = launch with programmatic stream serialisation (see pdl_prologue)
+  int split_l2;       // two-pass split kernel: L2 priority scheme (0 = default, see split_kernel)
 };
 
 template <int OP>

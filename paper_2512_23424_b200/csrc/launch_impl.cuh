@@ -204,7 +204,7 @@ cudaError_t launch_split(const LaunchPlan& plan, const RowParams& p, cudaStream_
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.numAttrs = 2;
   }
-  return cudaLaunchKernelEx(&cfg, kernel, p, plan.vpt);
+  return cudaLaunchKernelEx(&cfg, kernel, p, plan.vpt, plan.mode == 1 ? 0 : 1, plan.split_l2);
 }
 
 template <int OP, typename T>

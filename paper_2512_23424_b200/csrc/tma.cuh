@@ -35,6 +35,48 @@ __device__ __forceinline__ void mbar_wait_bounded(uint32_t bar, uint32_t parity,
     if (mbar_try_wait(bar, parity)) return;
   if (status != nullptr) atomicExch(status, kStatusTimeout);
 }
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Wait for a phase, at most kWaitNs of the global timer.  False on expiry, with the status word set.
+// CLUSTER: acquire at cluster scope (the data was written by another CTA of the cluster); otherwise
+// the default, CTA scope (data written by this CTA's bulk copies).
+constexpr unsigned long long kWaitNs = 2000000000ull;
+template <bool CLUSTER>
+__device__ __forceinline__ bool mbar_try_wait_scope(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  if (CLUSTER)
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+                 "selp.u32 %0, 1, 0, p;\n\t}" : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  else
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                 "selp.u32 %0, 1, 0, p;\n\t}" : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+template <bool CLUSTER = false>
+__device__ __forceinline__ bool mbar_wait_timed(uint32_t bar, uint32_t parity, int* status,
+                                                unsigned long long limit_ns = kWaitNs) {
+  if (mbar_try_wait_scope<CLUSTER>(bar, parity)) return true;
+  const unsigned long long t0 = global_timer_ns();
+  for (;;) {
+    if (mbar_try_wait_scope<CLUSTER>(bar, parity)) return true;
+    if (global_timer_ns() - t0 > limit_ns) break;
+  }
+  if (status != nullptr) atomicExch(status, kStatusTimeout);
+  return false;
+}
+// Four floats into the shared memory of CTA `rank` of the cluster, counted as 16 bytes on that
+// CTA's mbarrier (both addresses are this CTA's own; mapa translates them to the target's).
+__device__ __forceinline__ void st_async_f32x4(uint32_t local_dst, uint32_t local_bar, uint32_t rank, float a,
+                                               float b, float c, float d) {
+  uint32_t dst, bar;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(dst) : "r"(local_dst), "r"(rank));
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(bar) : "r"(local_bar), "r"(rank));
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.f32 [%0], {%1, %2, %3, %4}, [%5];"
+               :: "r"(dst), "f"(a), "f"(b), "f"(c), "f"(d), "r"(bar) : "memory");
+}
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                :: "r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");

@@ -96,6 +96,11 @@ CONFIG_NAMES = {
 }
 
 
+def config_shape(k: int):
+    """(rows, cols) of configuration k at full size."""
+    return _SHAPES[k][2], _SHAPES[k][3]
+
+
 def _normal_f32(rng: np.random.Generator, rows: int, cols: int) -> np.ndarray:
     out = np.empty((rows, cols), dtype=np.float32)
     block = max(1, (1 << 24) // max(cols, 1))

@@ -9,12 +9,14 @@ Tolerances (the build contract's):
              accepted when |y_ref| < 2^-126.  LayerNorm (+ beta) and log-softmax
              (- logsumexp) end in an addition that can cancel, so "output magnitude"
              is read there as the magnitude of the two addends: the bound gains
-             2^-20 * (|addend 1| + |addend 2|), i.e. 16 fp32 ulps of the terms that
-             the fp32 arithmetic actually rounds (nothing for softmax / RMSNorm)
+             2^-22 * (|addend 1| + |addend 2|), i.e. 4 fp32 ulps of the terms that
+             the fp32 arithmetic actually rounds (nothing for softmax / RMSNorm).
+             compare() counts the elements that need it (stats["rescued"])
   masked softmax entries and rows with no live entry: +0, bit for bit
 """
 from __future__ import annotations
 
+import os
 from typing import Optional, Sequence
 
 import numpy as np
@@ -26,6 +28,8 @@ from paper_2512_23424_b200 import workloads as wl
 
 FP32_ATOL = 1e-5
 BF16_ULPS = 2.0
+#: 16-bit LayerNorm / log-softmax: slack per unit of |addend 1| + |addend 2| (four fp32 ulps)
+CANCEL_16BIT = 2.0 ** -22
 
 
 def to_torch(a: Optional[np.ndarray], dtype: int, device="cuda") -> Optional[torch.Tensor]:
@@ -86,11 +90,12 @@ def run_gpu(w: wl.Workload, *, x_dev: Optional[torch.Tensor] = None, out: Option
 
 def run_oracle(w: wl.Workload, rows: Optional[Sequence[int]] = None,
                additive: Optional[np.ndarray] = None, causal_offset: int = 0,
-               nthreads: int = 8) -> np.ndarray:
+               nthreads: int = 0) -> np.ndarray:
     """fp64 reference for all rows, or for the listed global row indices."""
     x = w.x if rows is None else np.ascontiguousarray(w.x[np.asarray(rows)])
     ids = None if rows is None else np.asarray(rows, dtype=np.int64)
     eps = float(np.float32(w.eps))          # the library takes eps as a float
+    nthreads = nthreads or min(32, os.cpu_count() or 1)
     if w.op in ("softmax", "log_softmax"):
         mask = None
         if additive is not None or w.causal_period > 0:
@@ -121,7 +126,7 @@ def bf16_ulp(ref: np.ndarray) -> np.ndarray:
 def cancel_magnitude(w: wl.Workload, ref: np.ndarray, additive: Optional[np.ndarray] = None):
     """Absolute slack added to the tolerance, per element (None = none).
 
-    bf16 LayerNorm / log-softmax: 2^-20 * (|addend 1| + |addend 2|) of the final
+    bf16 LayerNorm / log-softmax: CANCEL_16BIT * (|addend 1| + |addend 2|) of the final
     addition (see the module docstring).
     LayerNorm, both dtypes: 2^-23 * max|x_row| * rstd_row * |gamma_c|.  The row mean is
     a real number that fp32 holds to half an ulp of |mean| <= max|x_row| at best; that
@@ -137,7 +142,7 @@ def cancel_magnitude(w: wl.Workload, ref: np.ndarray, additive: Optional[np.ndar
         slack = 2.0 ** -23 * np.abs(x).max(axis=1, keepdims=True) * rstd * gamma * np.ones_like(ref)
         if w.dtype != wl.F32:
             beta = 0.0 if w.beta is None else widen(w.beta)[None, :]
-            slack = slack + 2.0 ** -20 * (np.abs(ref - beta) + np.abs(beta))
+            slack = slack + CANCEL_16BIT * (np.abs(ref - beta) + np.abs(beta))
         return slack
     if w.op == "log_softmax" and w.dtype != wl.F32:
         z = widen(w.x)
@@ -146,14 +151,23 @@ def cancel_magnitude(w: wl.Workload, ref: np.ndarray, additive: Optional[np.ndar
             z = z + a[np.arange(w.rows) % a.shape[0], :w.cols]
         with np.errstate(invalid="ignore"):
             mag = np.abs(z) + np.abs(z - ref)
-        return 2.0 ** -20 * np.where(np.isfinite(mag), mag, 0.0)
+        return CANCEL_16BIT * np.where(np.isfinite(mag), mag, 0.0)
     return None
 
 
+#: one entry per comparison that was given a slack: (what, elements, rescued) where `rescued`
+#: counts the elements beyond the strict bound that only the slack lets pass.  Written to the
+#: file named by AKG_PARITY_LOG at the end of the session (see conftest.py).
+RESCUE_LOG = []
+
+
 def compare(got_stored: np.ndarray, ref: np.ndarray, dtype: int, what: str = "",
-            cancel_mag: Optional[np.ndarray] = None, tiny: float = 2.0 ** -126) -> dict:
+            cancel_mag: Optional[np.ndarray] = None, tiny: float = 2.0 ** -126,
+            max_rescued: Optional[int] = None) -> dict:
     """Assert parity under the tolerances above; returns error statistics.  `tiny`: bf16 results
-    whose reference is below it in magnitude may be returned as a flushed zero."""
+    whose reference is below it in magnitude may be returned as a flushed zero.  `cancel_mag`
+    widens the bound per element; stats["rescued"] counts the elements that needed it and
+    `max_rescued` (where given) limits that count."""
     got = widen(got_stored)
     assert got.shape == ref.shape, (what, got.shape, ref.shape)
     ref_nan, got_nan = np.isnan(ref), np.isnan(got)
@@ -164,21 +178,31 @@ def compare(got_stored: np.ndarray, ref: np.ndarray, dtype: int, what: str = "",
         assert np.array_equal(np.sign(ref[ref_inf]), np.sign(got[ref_inf])), f"{what}: infinity signs differ"
     fin = ~(ref_nan | ref_inf)
     err = np.abs(got[fin] - ref[fin])
-    stats = {"max_abs": float(err.max()) if err.size else 0.0, "n": int(fin.sum())}
-    if cancel_mag is not None:
-        err = np.maximum(err - cancel_mag[fin], 0.0)
-        stats["max_abs_after_slack"] = float(err.max()) if err.size else 0.0
+    stats = {"max_abs": float(err.max()) if err.size else 0.0, "n": int(fin.sum()), "rescued": 0}
     if dtype == wl.F32:
-        worst = float(err.max()) if err.size else 0.0
-        assert worst <= FP32_ATOL, f"{what}: max abs error {stats['max_abs']:.3e} > {FP32_ATOL}"
+        bound = np.full(err.shape, FP32_ATOL)
+        excused = np.zeros(err.shape, dtype=bool)
     else:
         # fp16 I/O: the same rule with the spacing of IEEE half (2 ulps; no flush below its range)
         ulp = f16_ulp(ref[fin]) if dtype == wl.F16 else bf16_ulp(ref[fin])
-        ulps = err / ulp
-        tiny_ok = (np.abs(ref[fin]) < (0.0 if dtype == wl.F16 else tiny)) & (got[fin] == 0)
-        bad = (ulps > BF16_ULPS) & ~tiny_ok
-        stats["max_ulp"] = float(ulps.max()) if ulps.size else 0.0
-        assert not bad.any(), f"{what}: {bad.sum()} elements beyond {BF16_ULPS} ulps of the storage type (max {stats['max_ulp']:.3f})"
+        bound = BF16_ULPS * ulp
+        excused = (np.abs(ref[fin]) < (0.0 if dtype == wl.F16 else tiny)) & (got[fin] == 0)
+        stats["max_ulp"] = float((err / ulp).max()) if err.size else 0.0
+    strict_bad = (err > bound) & ~excused
+    bad = strict_bad
+    if cancel_mag is not None:
+        bad = (err > bound + cancel_mag[fin]) & ~excused
+        stats["rescued"] = int(strict_bad.sum() - bad.sum())
+        stats["max_abs_after_slack"] = float(np.maximum(err - cancel_mag[fin], 0.0).max()) if err.size else 0.0
+        RESCUE_LOG.append((what, stats["n"], stats["rescued"]))
+    if dtype == wl.F32:
+        assert not bad.any(), f"{what}: max abs error {stats['max_abs']:.3e} > {FP32_ATOL}"
+    else:
+        assert not bad.any(), (f"{what}: {bad.sum()} elements beyond {BF16_ULPS} ulps of the storage type "
+                               f"(max {stats['max_ulp']:.3f})")
+    if max_rescued is not None:
+        assert stats["rescued"] <= max_rescued, (f"{what}: {stats['rescued']} elements pass only with the "
+                                                 f"cancellation slack (allowed: {max_rescued})")
     return stats
 
 

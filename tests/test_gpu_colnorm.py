@@ -8,7 +8,7 @@ import oracle
 import paper_2512_23424_b200 as akg
 from paper_2512_23424_b200 import binding
 from paper_2512_23424_b200 import workloads as wl
-from parity_util import compare, to_numpy, to_torch, widen
+from parity_util import CANCEL_16BIT, compare, to_numpy, to_torch, widen
 
 pytestmark = pytest.mark.gpu
 DTYPES = [wl.F32, wl.BF16, wl.F16]
@@ -31,7 +31,7 @@ def check(x, g, b, dtype, eps, got_y, got_mean, got_var, what):
     slack = 2.0 ** -23 * np.abs(xv).max(axis=0)[None, :] * (rstd * gam)[None, :] * np.ones_like(ref_y)
     if dtype != wl.F32:
         beta = np.zeros(x.shape[1]) if b is None else widen(b)
-        slack = slack + 2.0 ** -20 * (np.abs(ref_y - beta[None, :]) + np.abs(beta)[None, :])
+        slack = slack + CANCEL_16BIT * (np.abs(ref_y - beta[None, :]) + np.abs(beta)[None, :])
     compare(got_y, ref_y, dtype, what, slack)
     if got_mean is not None:
         scale = np.abs(xv).max(axis=0) + 1e-30

@@ -9,7 +9,7 @@ import oracle
 import paper_2512_23424_b200 as akg
 from paper_2512_23424_b200 import binding
 from paper_2512_23424_b200 import workloads as wl
-from parity_util import (assert_positive_zero, cancel_magnitude, compare, run_gpu, run_oracle, to_numpy, to_torch,
+from parity_util import (CANCEL_16BIT, assert_positive_zero, cancel_magnitude, compare, run_gpu, run_oracle, to_numpy, to_torch,
                          verifier_passes, widen)
 
 pytestmark = pytest.mark.gpu
@@ -82,7 +82,7 @@ def test_masks_and_prescale():
                         z = z + widen(add)[np.arange(rows) % 3, :]
                     with np.errstate(invalid="ignore"):
                         m = np.abs(z) + np.abs(z - ref)
-                    mag = 2.0 ** -20 * np.where(np.isfinite(m), m, 0.0)
+                    mag = CANCEL_16BIT * np.where(np.isfinite(m), m, 0.0)
                 mask = akg.make_mask(xd, additive=to_torch(add, F16) if add is not None else None, causal=per > 0,
                                      causal_period=max(per, 1))
                 got = to_numpy(binding.softmax_scaled(xd, scale, mask=mask, log=log))

@@ -115,7 +115,10 @@ SWEEP_COLS = [1, 2, 3, 4, 5, 7, 8, 9, 31, 32, 33, 127, 128, 129, 1000, 1023, 102
               4097, 8191, 8192, 32768 + 8,
               # hidden sizes that are (a multiple of 32 threads) x (1..8 vectors), not a power of two
               1536, 2560, 5120, 6144, 7168, 12288, 20480]
-SWEEP_ROWS = [1, 2, 3, 63, 65, 149]
+SWEEP_ROWS = [1, 2, 3, 63, 65, 148, 149]
+# long rows around the sizes a tile size would divide (two or three rows each): odd, a multiple of
+# one fp32 vector only, of one 16-bit vector only, and a row of a million columns
+SWEEP_LONG_COLS = [262144 - 1, 262144 + 4, 262144 + 8, 1048576 + 12]
 
 
 @pytest.mark.parametrize("op", ["softmax", "log_softmax", "layernorm", "rmsnorm"])
@@ -130,6 +133,13 @@ def test_shape_sweep(op, dtype):
             else:
                 w = wl.make_random(op, dtype, rows, cols, seed, loc=1.0, scale=1.5, eps=1e-5)
             check_workload(w)
+    for i, cols in enumerate(SWEEP_LONG_COLS):
+        rows = 2 + i % 2
+        if op in ("softmax", "log_softmax"):
+            w = wl.make_random(op, dtype, rows, cols, 900 + i, scale=2.0)
+        else:
+            w = wl.make_random(op, dtype, rows, cols, 900 + i, loc=1.0, scale=1.5, eps=1e-5)
+        check_workload(w)
 
 
 @pytest.mark.parametrize("op", ["softmax", "log_softmax", "layernorm", "rmsnorm"])

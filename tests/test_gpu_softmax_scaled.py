@@ -8,7 +8,7 @@ import oracle
 import paper_2512_23424_b200 as akg
 from paper_2512_23424_b200 import binding
 from paper_2512_23424_b200 import workloads as wl
-from parity_util import assert_positive_zero, compare, to_numpy, to_torch, verifier_passes, widen
+from parity_util import CANCEL_16BIT, assert_positive_zero, compare, to_numpy, to_torch, verifier_passes, widen
 
 pytestmark = pytest.mark.gpu
 VARIANTS = ["auto", "stream", "reg", "tma", "tma_smem", "cluster", "split"]
@@ -51,7 +51,7 @@ def check_all(x, dtype, scale, log, additive=None, causal_period=0, variants=VAR
             z = z + widen(additive)[np.arange(rows) % additive.shape[0], :cols]
         with np.errstate(invalid="ignore"):
             m = np.abs(z) + np.abs(z - ref)
-        mag = 2.0 ** -20 * np.where(np.isfinite(m), m, 0.0)
+        mag = CANCEL_16BIT * np.where(np.isfinite(m), m, 0.0)
     ran = []
     for v in variants:
         xd = to_torch(x, dtype)

@@ -66,4 +66,4 @@ def test_reference_arm_prints_one_line_on_rank0_only():
     line = json.loads(out.stdout.strip().splitlines()[-1])
     assert line["impl"] == "reference" and line["unit"] == "GB/s" and line["value"] > 0
     assert line["cpu_baseline"]["kind"] == "oracle" and line["e2e"]["h2d_bytes_per_step"] == 0
-    assert line["config"]["workload"] == wl.CONFIG_NAMES[2]
+    assert line["config"]["workload"] == wl.CONFIG_NAMES[bench.HEADLINE]

@@ -5,8 +5,10 @@ Who needs it: code that gets host buffers and a stream but cannot obtain device 
 its own - a plug-in that may not touch its host application's memory pool, a service that
 must not allocate once it is running.  Such a caller cannot give akg_rowop_host the staging
 workspace it asks for, so the library carries a fixed 16 MiB staging area instead.  The
-area is shared by all calls and keeps the previous call's bytes, hence the test runs two
-different problems back to back and checks that neither sees the other's leftovers.
+area is shared by all calls and keeps the previous call's bytes, hence the test runs
+different problems back to back and checks that neither sees the other's leftovers.  Every
+result is also compared with the fp64 oracle at the parity tests' strict tolerance, so an
+error common to both entry points cannot hide.
 
 This file is named so that pytest collects it last.
 """
@@ -17,7 +19,7 @@ import torch
 import paper_2512_23424_b200 as akg
 from paper_2512_23424_b200 import binding
 from paper_2512_23424_b200 import workloads as wl
-from parity_util import BF16_ULPS, FP32_ATOL, bf16_ulp, to_numpy, widen
+from parity_util import BF16_ULPS, FP32_ATOL, bf16_ulp, compare, run_oracle, to_numpy, widen
 
 pytestmark = pytest.mark.gpu
 
@@ -64,6 +66,7 @@ def test_static_entry_matches_workspace_entry_twice_in_a_row():
     got_first = got.copy()
     assert not np.isnan(widen(got)).any()
     assert_same(want, got, w1.dtype, "first call (layernorm f32)")
+    compare(got, run_oracle(w1), w1.dtype, "first call against the oracle")
     # second call, straight after: a smaller causal bf16 softmax; leftovers of call one in
     # the staging area must not show (masked entries are exactly +0, live ones match)
     w2 = wl.make_random("softmax", wl.BF16, 700, 1024, seed=12)
@@ -72,10 +75,21 @@ def test_static_entry_matches_workspace_entry_twice_in_a_row():
     assert_same(want, got, w2.dtype, "second call (causal softmax bf16)")
     dead = np.arange(1024)[None, :] > (np.arange(700)[:, None] % 256)
     assert (got[dead] == 0).all()
+    compare(got, run_oracle(w2), w2.dtype, "second call against the oracle")
+    # third call: a causal softmax larger than the staging area (3000 x 4096 bf16 = 23 MiB), so the
+    # rows go through it in chunks of 2048 and the second chunk starts in the middle of a causal
+    # period (1500 rows, not a power of two): the rule has to see global row numbers
+    w3 = wl.make_random("softmax", wl.BF16, 3000, 4096, seed=13)
+    w3.causal_period = 1500
+    want, got = run_both(w3)
+    assert_same(want, got, w3.dtype, "third call (causal softmax bf16, chunked)")
+    compare(got, run_oracle(w3), w3.dtype, "third call against the oracle")
+    dead = np.arange(4096)[None, :] > (np.arange(3000)[:, None] % 1500)
+    assert (got[dead] == 0).all()
     # and the first problem again gives the first answer again
     want1, got1 = run_both(w1)
     assert np.array_equal(got1.view(np.uint32), got_first.view(np.uint32))
-    assert_same(want1, got1, w1.dtype, "third call (layernorm f32 again)")
+    assert_same(want1, got1, w1.dtype, "fourth call (layernorm f32 again)")
     assert akg.device_status() == 0
 
 
