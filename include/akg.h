@@ -5,7 +5,7 @@
  * X[rows, cols]: softmax, log-softmax, LayerNorm, RMSNorm, with optional
  * additive and/or causal masking for the softmax pair.  One fused kernel per
  * call: every live input element is read from HBM once and every output
- * element written once.  fp32 or bf16 storage; all arithmetic in fp32; a bf16
+ * element written once.  fp32, bf16 or fp16 storage; all arithmetic in fp32; a bf16
  * result is rounded once (nearest-even) at the store.
  *
  * General rules for every entry point
@@ -21,8 +21,10 @@
  *   - rows == 0 or cols == 0 is AKG_OK with nothing launched.  Any alignment of
  *     pointers and strides is accepted: 16-byte aligned rows select vectorised
  *     kernels, anything else a scalar kernel with the same results.
- *   - In place (y == x with equal strides) is allowed; any other overlap of the
- *     x and y ranges is AKG_ERR_INVALID_ARG.
+ *   - In place (y == x with equal strides) is allowed, and so are two column
+ *     windows of one buffer that share no element (x = buf[:, :cols], y = buf[:, cols:]
+ *     with the same row stride); any other overlap of x and y is
+ *     AKG_ERR_INVALID_ARG.
  *   - On AKG_ERR_INVALID_ARG / AKG_ERR_UNSUPPORTED nothing has been launched.
  *     AKG_ERR_CUDA reports a failed launch (the CUDA error is consumed; its
  *     text is available from akg_last_error_string on the same thread).
@@ -95,8 +97,8 @@ akg_status akg_log_softmax(const void* x, void* y, int64_t rows, int64_t cols,
                            int64_t x_row_stride, int64_t y_row_stride, akg_dtype dtype,
                            const akg_mask* mask, void* stream);
 
-/* LayerNorm over the last axis ("LayerNorm ... mean, variance, and normalization
- * steps" fused into one kernel, Section 4.3):
+/* LayerNorm over the last axis (the operator whose statistics and normalisation
+ * the paper's Section 4.3 describes as fused into one kernel):
  *   mu = mean(x), var = mean((x - mu)^2) (biased),
  *   y_c = (x_c - mu) / sqrt(var + eps) * gamma_c + beta_c.
  * gamma == NULL means 1, beta == NULL means 0.  eps >= 0 (NaN is rejected). */
@@ -314,7 +316,14 @@ akg_status akg_set_variant(akg_variant variant);
  * sized for), "tma_mode" (1 = ring-fed register kernels, 2 = shared-memory passes),
  * "cluster_mode" (1 = row resident in the cluster's shared memory, 2 = two streaming
  * passes with the second served by L2), "reg_general" (1 = never the predicate-free
- * normalisation kernel), "interleave" (1 = visit causal rows short/long alternately).
+ * normalisation kernel), "interleave" (1 = visit causal rows short/long alternately),
+ * "split_exchange" (two-pass cluster kernel: 1 = partial statistics exchanged under a
+ * cluster barrier per row instead of st.async + mbarrier), "split_l2" (its L2 priority
+ * scheme: 1 = no "keep" marks, 2 = marks without demotion).  Two keys exist for the test
+ * of the failure path only: "test_wait_us" (limit of the kernels' bounded waits in
+ * microseconds; 0 = two seconds) and "test_no_copies" (1 = the ring kernels issue no
+ * bulk copy, so that every wait on one runs out and the call reports
+ * AKG_ERR_DEVICE_TIMEOUT through akg_device_status).
  * A geometry the library was not
  * built for makes the next call return AKG_ERR_CUDA.  Unknown key:
  * AKG_ERR_INVALID_ARG. */
@@ -325,9 +334,14 @@ akg_status akg_set_tuning(const char* key, int value);
 const char* akg_last_kernel_name(void);
 
 /* Reads the device-side status word of the current device (synchronises with
- * the device).  0 = clean; non-zero = a bounded wait on a bulk copy expired in
- * some kernel since the last call (the word is reset to 0 by this call).
- * Returns AKG_OK, AKG_ERR_DEVICE_TIMEOUT, or AKG_ERR_CUDA. */
+ * the device).  0 = clean; non-zero = a bounded wait (on a bulk copy, or on the
+ * partial statistics of a cluster peer) ran out in some kernel since the last
+ * call; the word is reset to 0 by this call.  Every such wait is limited to two
+ * seconds of the device's global timer.  A CTA whose wait ran out stores nothing
+ * from then on, issues no further copy and still takes part in its barriers, so the
+ * kernel ends by itself and the context stays usable; the output of that call is
+ * undefined (partly written).  Returns AKG_OK, AKG_ERR_DEVICE_TIMEOUT, or
+ * AKG_ERR_CUDA. */
 akg_status akg_device_status(int* word_out);
 
 #ifdef __cplusplus

@@ -37,6 +37,8 @@ std::atomic<int> g_tune_host_chunks{0};   // host-buffer pipeline: chunks per ca
 std::atomic<int> g_tune_host_min_kib{0};  //   smallest chunk in KiB (0 = default)
 std::atomic<int> g_tune_split_exchange{0};  // two-pass split kernel: 1 = cluster barrier per row instead of st.async + mbarrier
 std::atomic<int> g_tune_split_l2{0};        //   L2 priority scheme (see split_kernel)
+std::atomic<int> g_tune_test_wait_us{0};    // test only: limit of the kernels' bounded waits in microseconds (0 = two seconds)
+std::atomic<int> g_tune_test_no_copies{0};  // test only: 1 = the ring kernels issue no bulk copy, so that their waits run out
 std::atomic<int> g_tune_axis_mode{0};     //   1 = 16-byte vectors, 2 = bf16 8-byte vectors widened, 3 = elements
 
 __device__ int g_status_word = 0;
@@ -90,8 +92,19 @@ akg_status validate(const Call& c, const char* name) {
   const uintptr_t x1 = x0 + static_cast<uintptr_t>(((c.rows - 1) * c.xs + c.cols) * es);
   const uintptr_t y1 = y0 + static_cast<uintptr_t>(((c.rows - 1) * c.ys + c.cols) * es);
   const bool overlap = x0 < y1 && y0 < x1;
-  if (overlap && !(x0 == y0 && c.xs == c.ys))
-    return fail(AKG_ERR_INVALID_ARG, "%s: x and y overlap without being the same matrix", name);
+  if (overlap && !(x0 == y0 && c.xs == c.ys)) {
+    // Two column windows of one buffer (x = buf[:, :cols], y = buf[:, cols:], equal strides, as in a
+    // fused gate / up or q / k / v layout) interleave without sharing an element: with d the distance of
+    // the bases modulo the row pitch, the windows are disjoint iff cols <= d and d + cols <= pitch.
+    bool disjoint_windows = false;
+    if (c.xs == c.ys) {
+      const uintptr_t pitch = static_cast<uintptr_t>(c.xs * es), width = static_cast<uintptr_t>(c.cols * es);
+      const uintptr_t d = (x0 > y0 ? x0 - y0 : y0 - x0) % pitch;
+      disjoint_windows = d >= width && d + width <= pitch;
+    }
+    if (!disjoint_windows)
+      return fail(AKG_ERR_INVALID_ARG, "%s: x and y overlap without being the same matrix", name);
+  }
   return AKG_OK;
 }
 
@@ -173,7 +186,7 @@ bool plan_reg(const Call& c, LaunchPlan* plan) {
     else if (nvec <= 1024) { threads = 256; vpt = 4; }
     else if (nvec <= 2048 && c.dtype == AKG_F32 && !norm_op) { threads = 256; vpt = 8; }   // fp32 softmax pair: fat threads (5120 columns: 80 % against 71 % as 512 x 4)
     else if (nvec <= 2048) { threads = 512; vpt = 4; }
-    else if (nvec <= 4096) { threads = (c.dtype == AKG_F32) ? 512 : 1024; vpt = (c.dtype == AKG_F32) ? 8 : 4; }
+    else if (nvec <= 4096 && c.dtype == AKG_F32) { threads = 512; vpt = 8; }   // (16-bit rows beyond 2048 vectors: other families)
     else if (nvec <= 8192 && c.dtype == AKG_F32) { threads = 1024; vpt = 8; }
     else return false;
     group = threads;
@@ -242,11 +255,12 @@ bool plan_reg(const Call& c, LaunchPlan* plan) {
 // Shared-memory ring plan with a cluster of cs CTAs per row, cs_min <= cs <= cs_max
 // (cs = 1 is the plain TMA ring).  Picks the smallest cluster whose slice leaves room
 // for at least two ring buffers, else the smallest with one.  False if nothing fits.
-bool plan_smem(const Call& c, int cs_min, int cs_max, LaunchPlan* plan) {
+bool plan_smem(const Call& c, int cs_min, int cs_max, LaunchPlan* plan, int want_threads = 0, int want_ctas = 0) {
   const int64_t epv = (c.dtype == AKG_F32) ? 4 : 8;
   const int64_t nvec = c.cols / epv;
   const int t_cs = g_tune_cluster_size.load(), t_nbuf = g_tune_smem_nbuf.load();
-  const int t_threads = g_tune_smem_threads.load(), t_ctas = g_tune_smem_ctas.load();
+  const int t_threads = g_tune_smem_threads.load() > 0 ? g_tune_smem_threads.load() : want_threads;
+  const int t_ctas = g_tune_smem_ctas.load() > 0 ? g_tune_smem_ctas.load() : want_ctas;
   if (t_cs > 0) {
     if (t_cs < cs_min || t_cs > cs_max) return false;
     cs_min = cs_max = t_cs;
@@ -414,6 +428,8 @@ akg_status run(const Call& c, const char* name) {
     }
   }
   p.status = nullptr;
+  p.wait_us = g_tune_test_wait_us.load() > 0 ? static_cast<unsigned>(g_tune_test_wait_us.load()) : 0u;
+  p.no_copies = g_tune_test_no_copies.load() == 1 ? 1 : 0;
   p.scale = c.scale; p.inv_scale = 1.0f / c.scale; p.l2e = kLog2e * c.scale;   // scale 1: exactly log2(e)
   p.row_base = c.row_base;
   if (c.row_base != 0) { p.interleave = 0; if (p.add_mode == 2) p.add_mode = 0; }
@@ -471,6 +487,20 @@ akg_status run(const Call& c, const char* name) {
       }
       p.status = status_word_ptr();
     }
+  }
+  // 16-bit rows of 16 - 64 KB without a mask, where a CTA's registers no longer hold the row comfortably:
+  // the row resident in shared memory (bulk-copied in, two sweeps over shared memory), several CTAs per SM
+  // so that one row's sweeps overlap the others' copies.  Measured against the register and two-pass
+  // kernels (bf16, fraction of the copy rate): log-softmax 12288 / 16384 / 20480 columns 0.69 / 0.85 / 0.81
+  // against 0.65 / 0.69 / 0.78 with three CTAs of 256 threads per SM; RMSNorm 20480 / 32768 columns
+  // 0.89 / 0.84 against 0.87 / 0.78 with two CTAs of 512.  (Softmax and LayerNorm were level or behind.)
+  if (!planned && forced == V_AUTO && vec && c.dtype != AKG_F32 && c.rows >= 2 * static_cast<int64_t>(sm_count()) &&
+      (c.mask == nullptr || (c.mask->additive == nullptr && !c.mask->causal)) && g_tune_tma_mode.load() == 0 &&
+      g_tune_cluster_mode.load() == 0) {
+    const int64_t nv16 = c.cols / 8;
+    if (c.op == OP_LOG_SOFTMAX && nv16 > 1024 && nv16 <= 3072) planned = plan_smem(c, 1, 1, &plan, 256, 3);
+    else if (c.op == OP_RMSNORM && nv16 > 2048 && nv16 <= 4096) planned = plan_smem(c, 1, 1, &plan, 512, 2);
+    if (planned) p.status = status_word_ptr();
   }
   // rows beyond 2048 vectors in the 16-bit types (beyond 4096 for the fp32 softmax pair) measured
   // faster in the two-pass kernel than in one CTA of 640 - 1024 threads: bf16 32768 columns 77 - 79 %
@@ -761,6 +791,8 @@ akg_status akg_set_tuning(const char* key, int value) {
   else if (!std::strcmp(key, "axis_lc")) g_tune_axis_lc.store(value);
   else if (!std::strcmp(key, "split_exchange")) g_tune_split_exchange.store(value);
   else if (!std::strcmp(key, "split_l2")) g_tune_split_l2.store(value);
+  else if (!std::strcmp(key, "test_wait_us")) g_tune_test_wait_us.store(value);
+  else if (!std::strcmp(key, "test_no_copies")) g_tune_test_no_copies.store(value);
   else return fail(AKG_ERR_INVALID_ARG, "akg_set_tuning: unknown key %s", key);
   return AKG_OK;
 }
@@ -1146,6 +1178,36 @@ extern "C" akg_status akg_cumulative(int want_prod, const void* x, void* y, int6
   const bool warp_rows = vec && (t_group == 32 || (t_group == 0 && cols * es <= scan_warp_row_bytes(es)));
   const int64_t ctas = warp_rows ? (rows + 7) / 8 : rows;
   const unsigned grid = static_cast<unsigned>(std::min<int64_t>(ctas, cap > 0 ? cap : INT_MAX));
+  // Few, long rows (at least 8192 vectors each; fewer rows than SMs in fp32, than two per SM in the 16-bit
+  // types): a cluster per row, every CTA a slice of about 4096 vectors, the carry of a slice from the cluster's
+  // totals (scan_split_kernel).  Measured against a CTA per row, fraction of the copy rate: [64, 2^20] fp32 0.54
+  // against 0.30, bf16 0.64 against 0.22; [256, 262144] bf16 0.74 against 0.65, fp32 0.75 against 0.83 (hence the
+  // fp32 limit); [148, 131072] level in fp32, bf16 0.53 against 0.46.
+  const int t_cs = g_tune_cluster_size.load();
+  if (vec && !warp_rows && g_tune_reg_general.load() == 0 &&
+      (t_cs > 1 || (t_cs == 0 && rows < (es == 4 ? 1 : 2) * static_cast<int64_t>(sm_count()) && nvec >= 8192))) {
+    int cs = t_cs;
+    if (cs == 0) {
+      cs = 2;
+      while (cs < kMaxCluster && (nvec / (2 * cs) >= 3072 || rows * cs < 2 * static_cast<int64_t>(sm_count()))) cs *= 2;
+    }
+    if (cs >= 2 && cs <= kMaxCluster && (cs & (cs - 1)) == 0 && nvec / cs >= 256 && nvec <= INT_MAX / 2) {
+      int64_t slice = (nvec + cs - 1) / cs;
+      slice = (slice + 255) / 256 * 256;
+      // rows in flight stay in L2 between the two phases: at most 64 MB of them
+      int64_t clusters = (int64_t(64) << 20) / (cols * es);
+      if (clusters < (160 + cs - 1) / cs) clusters = (160 + cs - 1) / cs;
+      if (cap > 0) clusters = std::max(1, cap / cs);
+      const cudaError_t e2 = launch_cumulative_split(want_prod == 1, static_cast<int>(dtype), x, y, rows, cols, x_row_stride,
+                                                     y_row_stride, cs, static_cast<int>(slice), clusters, status_word_ptr(),
+                                                     g_tune_test_wait_us.load() > 0 ? static_cast<unsigned>(g_tune_test_wait_us.load()) : 0u,
+                                                     static_cast<cudaStream_t>(stream));
+      if (e2 != cudaSuccess) return cuda_fail(name, e2);
+      std::snprintf(t_kernel, sizeof t_kernel, "scan_split<%s,%s,t256,cs%d,slice%d>", want_prod ? "prod" : "sum",
+                    dtype_name(dtype), cs, static_cast<int>(slice));
+      return AKG_OK;
+    }
+  }
   const cudaError_t err = launch_cumulative(want_prod == 1, static_cast<int>(dtype), vec, x, y, rows, cols, x_row_stride,
                                             y_row_stride, grid, threads, warp_rows, g_tune_pdl.load() == 2 ? 0 : 1,
                                             static_cast<cudaStream_t>(stream));

@@ -31,6 +31,8 @@ struct RowParams {
   int interleave;           // 1: visit the rows of a causal period short/long alternately
   long long row_base;       // global index of row 0 (mask rules use row + row_base); 0 unless chunked
   int* status;              // device status word (bounded waits report here)
+  unsigned wait_us;         // limit of a bounded wait in microseconds; 0 = two seconds
+  int no_copies;            // test only: the ring kernels issue no bulk copy, so every wait runs out
   // fused residual add (normalisations only): the operator runs on x + res; the sum is also
   // stored to `sum` unless that is nullptr.  res == nullptr: plain operator.
   const void* res;
@@ -175,7 +177,24 @@ template <> struct Elem<__nv_bfloat16> {
     reinterpret_cast<__nv_bfloat16*>(base)[i] = __float2bfloat16_rn(v);
   }
   static __device__ __forceinline__ uint32_t fill_word(float v) { return pack2(v, v); }
+  // Mixed-precision arithmetic of sm_100: a 16-bit operand is widened inside the instruction, which
+  // runs on the FMA pipe, so the value never has to be unpacked by a shift / mask on the ALU pipe.
+  // `h` is one stored element (either half of a packed word, see halves()).
+  static __device__ __forceinline__ float sub_wide(unsigned short h, float c) {            // h - c
+    float d; asm("sub.rn.f32.bf16 %0, %1, %2;" : "=f"(d) : "h"(h), "f"(c)); return d;
+  }
+  static __device__ __forceinline__ float add_wide(unsigned short h, float c) {            // h + c
+    float d; asm("add.rn.f32.bf16 %0, %1, %2;" : "=f"(d) : "h"(h), "f"(c)); return d;
+  }
+  static __device__ __forceinline__ float fma_wide(unsigned short a, unsigned short b, float c) {   // a * b + c
+    float d; asm("fma.rn.f32.bf16 %0, %1, %2, %3;" : "=f"(d) : "h"(a), "h"(b), "f"(c)); return d;
+  }
 };
+
+// the two 16-bit halves of a packed word (low half = even element)
+__device__ __forceinline__ void halves(uint32_t w, unsigned short& lo, unsigned short& hi) {
+  asm("mov.b32 {%0, %1}, %2;" : "=h"(lo), "=h"(hi) : "r"(w));
+}
 
 // IEEE half (the paper's float16 regime, Section 4.1): same vector shape as bf16, hardware
 // conversions in both directions, one rounding (nearest-even) at the store.
@@ -205,6 +224,15 @@ template <> struct Elem<__half> {
     reinterpret_cast<__half*>(base)[i] = __float2half_rn(v);
   }
   static __device__ __forceinline__ uint32_t fill_word(float v) { return pack2(v, v); }
+  static __device__ __forceinline__ float sub_wide(unsigned short h, float c) {
+    float d; asm("sub.rn.f32.f16 %0, %1, %2;" : "=f"(d) : "h"(h), "f"(c)); return d;
+  }
+  static __device__ __forceinline__ float add_wide(unsigned short h, float c) {
+    float d; asm("add.rn.f32.f16 %0, %1, %2;" : "=f"(d) : "h"(h), "f"(c)); return d;
+  }
+  static __device__ __forceinline__ float fma_wide(unsigned short a, unsigned short b, float c) {
+    float d; asm("fma.rn.f32.f16 %0, %1, %2, %3;" : "=f"(d) : "h"(a), "h"(b), "f"(c)); return d;
+  }
 };
 
 template <int OP> struct OpTraits {

@@ -42,7 +42,7 @@ __device__ __forceinline__ float warp_max(float v) {
 template <int OP, typename T, int G, int VPT, int THREADS, bool RING = false>
 __device__ __forceinline__ void norm_row_full(const RowParams& p, long long row, int tg,
                                               float (*red)[(G / 32) > 1 ? (G / 32) : 1],
-                                              uint32_t ring_buf = 0) {
+                                              uint32_t ring_buf = 0, bool dead = false) {
   using E = Elem<T>;
   constexpr int EPV = E::EPV;
   constexpr int N = VPT * EPV;
@@ -124,6 +124,9 @@ __device__ __forceinline__ void norm_row_full(const RowParams& p, long long row,
     rstd = rsqrt_refined(fmaf(m2, inv_cols, p.eps));
   }
 
+  // (ring kernels: a thread whose wait for the row ran out took part in the reduction above, for its
+  // CTA's barrier, and stores nothing)
+  if (RING && dead) return;
   // 16-bit storage: (x - mean) * rstd as one fused multiply-add with the row constant -mean * rstd
   // (its rounding, 2^-24 |mean| rstd, is far inside the 2^-9 of the stored result); fp32 keeps
   // the exact difference

@@ -41,8 +41,16 @@ struct RowRing {
     for (uint32_t off = 0; off < bytes; off += kChunk)
       bulk_load(buf(b) + off, reinterpret_cast<const unsigned char*>(src) + off, min(kChunk, bytes - off), bar);
   }
-  __device__ __forceinline__ void wait(int b, uint32_t phase, int* status) const {
-    mbar_wait_bounded(bars + 8u * b, phase, status);
+  __device__ __forceinline__ bool wait(int b, uint32_t phase, const RowParams& p) const {
+    return mbar_wait_timed(bars + 8u * b, phase, p.status, p.wait_us);
+  }
+  // thread 0, before a CTA that gave up leaves: no copy may still be on its way into the CTA's shared
+  // memory; `pending` buffers starting at b (phase of the first) have one
+  __device__ __forceinline__ void drain(int b, uint32_t phase, int pending, const RowParams& p) const {
+    for (; pending > 0; --pending) {
+      (void)mbar_wait_timed(bars + 8u * b, phase, nullptr, p.wait_us);
+      if (++b == nbuf) { b = 0; phase ^= 1u; }
+    }
   }
 };
 
@@ -57,23 +65,37 @@ __global__ void __launch_bounds__(THREADS, kRegMinBlocks<THREADS>) ring_norm_ful
   RowRing ring;
   ring.init(ring_smem, kRowBytes, nbuf);
 
+  // A wait that runs out (see mbar_wait_timed) makes its thread "dead": it stores nothing any more and
+  // waits for nothing, but still runs the row bodies, whose barriers its CTA needs.  The flag in shared
+  // memory spreads the state to the whole CTA at the next row (the row body's barrier lies in between),
+  // so that a lost copy costs one wait, not one per remaining row.
+  __shared__ int cta_dead;
+  if (threadIdx.x == 0) cta_dead = 0;
+  __syncthreads();
   const long long step = gridDim.x;
   const T* x = reinterpret_cast<const T*>(p.x);
-  if (threadIdx.x == 0) {
+  int in_flight = 0;                                   // thread 0: copies issued and not yet waited for
+  if (threadIdx.x == 0 && !p.no_copies) {
     long long r = blockIdx.x;
-    for (int b = 0; b < nbuf && r < p.rows; ++b, r += step) ring.issue(x + r * p.xs, kRowBytes, b);
+    for (int b = 0; b < nbuf && r < p.rows; ++b, r += step) { ring.issue(x + r * p.xs, kRowBytes, b); ++in_flight; }
   }
   int b = 0, parity = 0;
   uint32_t phase = 0;
+  bool dead = false;
   for (long long row = blockIdx.x; row < p.rows; row += step, parity ^= 1) {
-    ring.wait(b, phase, p.status);
-    norm_row_full<OP, T, THREADS, VPT, THREADS, true>(p, row, threadIdx.x, red[parity], ring.buf(b));
-    if (threadIdx.x == 0) {
-      const long long next = row + step * nbuf;
-      if (next < p.rows) ring.issue(x + next * p.xs, kRowBytes, b);
+    if (!dead && *reinterpret_cast<volatile int*>(&cta_dead)) dead = true;
+    if (!dead) {
+      if (ring.wait(b, phase, p)) { if (threadIdx.x == 0) --in_flight; }
+      else { dead = true; cta_dead = 1; }
     }
-    if (++b == nbuf) { b = 0; phase ^= 1u; }
+    norm_row_full<OP, T, THREADS, VPT, THREADS, true>(p, row, threadIdx.x, red[parity], ring.buf(b), dead);
+    if (threadIdx.x == 0 && !dead && !p.no_copies) {
+      const long long next = row + step * nbuf;
+      if (next < p.rows) { ring.issue(x + next * p.xs, kRowBytes, b); ++in_flight; }
+    }
+    if (!dead && ++b == nbuf) { b = 0; phase ^= 1u; }
   }
+  if (threadIdx.x == 0 && dead) ring.drain(b, phase, in_flight, p);
   (void)EPV;
 }
 
@@ -95,29 +117,37 @@ __global__ void __launch_bounds__(THREADS, kRegMinBlocks<THREADS>) ring_softmax(
     const int live = static_cast<int>(live_cols(p, r));
     return static_cast<uint32_t>((live + EPV - 1) / EPV) * 16u;
   };
-  if (threadIdx.x == 0) {
+  int in_flight = 0;                                   // thread 0: copies issued and not yet waited for
+  if (threadIdx.x == 0 && !p.no_copies) {
     long long r = blockIdx.x;
     for (int b = 0; b < nbuf && r < p.rows; ++b, r += step) {
       const long long mr = balanced_row(p, r);
       ring.issue(x + mr * p.xs, live_bytes(mr), b);
+      ++in_flight;
     }
   }
   int b = 0, parity = 0;
   uint32_t phase = 0;
+  bool dead = false;
   for (long long item = blockIdx.x; item < p.rows; item += step, parity ^= 1) {
     const long long row = balanced_row(p, item);
-    ring.wait(b, phase, p.status);
+    // (only forced launches reach this kernel: the CTA-wide vote costs it a barrier per row)
+    if (__syncthreads_or(ring.wait(b, phase, p) ? 0 : 1)) { dead = true; break; }
+    if (threadIdx.x == 0) --in_flight;
     softmax_row_dispatch<OP, T, THREADS, VPT, VPT, THREADS, true>(p, row, threadIdx.x, nvec, red[parity],
                                                                   ring.buf(b));
-    if (threadIdx.x == 0) {
+    if (threadIdx.x == 0 && !p.no_copies) {
       const long long next = item + step * nbuf;
       if (next < p.rows) {
         const long long mr = balanced_row(p, next);
         ring.issue(x + mr * p.xs, live_bytes(mr), b);
+        ++in_flight;
       }
     }
     if (++b == nbuf) { b = 0; phase ^= 1u; }
   }
+  // a CTA that gave up stores nothing more; the copy it waited for in vain is still counted
+  if (threadIdx.x == 0 && dead) ring.drain(b, phase, in_flight, p);
 }
 
 }  // namespace akg

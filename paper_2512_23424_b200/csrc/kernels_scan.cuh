@@ -11,7 +11,7 @@
 // of the earlier warps of its own u.  fp32 arithmetic throughout; one rounding at the store.
 #pragma once
 
-#include "common.cuh"
+#include "tma.cuh"
 
 namespace akg {
 
@@ -152,6 +152,187 @@ __global__ void __launch_bounds__(32 * kScanMaxWarps, 4) scan_kernel(const ScanP
     }
     if (!WARP) __syncthreads();                                 // wtot[par] of the next row
   }
+}
+
+
+// ------------------------------------------------------------------------------------------------
+// scan_split_kernel: few, long rows (a CTA per row would leave most SMs idle and walk a megabyte on
+// its own).  A cluster of CS CTAs owns a row at a time and CTA k its slice k of slice_vecs vectors:
+//   phase 1  the slice's total: streaming loads marked "keep in L2", eight per thread in flight,
+//            thread -> warp -> CTA reduction
+//   exchange every CTA sends its total to every CTA of the cluster (one 16-byte st.async into the
+//            receiver's shared memory, counted on the receiver's mbarrier: the scheme of
+//            split_kernel); a CTA's carry-in is the combination, in slice order, of the totals of
+//            the slices before its own - a look-back that never leaves the cluster: no flag in
+//            global memory, nothing to spin on but the CTA's own mbarrier, and that wait is bounded
+//   phase 2  the chunked scan of scan_kernel over the slice, starting from the carry-in; the slice
+//            is read again, now from L2 ("evict first"), and stored
+// HBM sees one read and one write per element.  Vectorised rows only.
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint4 scan_ld_hint(const void* p, uint64_t pol) {
+  uint4 v;
+  asm volatile("ld.global.L1::no_allocate.L2::cache_hint.v4.u32 {%0, %1, %2, %3}, [%4], %5;"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p), "l"(pol) : "memory");
+  return v;
+}
+
+template <bool PROD, typename T>
+__global__ void __launch_bounds__(256, 4) scan_split_kernel(const ScanParams p, const int slice_vecs,
+                                                           int* status, const unsigned wait_us) {
+  pdl_prologue();
+  using E = Elem<T>;
+  constexpr int EPV = E::EPV;
+  constexpr int U = kScanU;
+  constexpr int T_ = 256, NW = T_ / 32;
+  __shared__ float wtot[2][U][NW];
+  __shared__ float red[NW];
+  __shared__ __align__(16) float4 inbox[2][kMaxCluster];
+  __shared__ __align__(8) uint64_t xbar[2];
+  __shared__ int cta_failed;
+  const int tid = static_cast<int>(threadIdx.x), lane = tid & 31, warp = tid >> 5;
+  const uint32_t cs = cluster_size(), rank = cluster_rank();
+  const long long row_step = cluster_count();
+  const int nvec = static_cast<int>(p.cols / EPV);
+  const int v0 = static_cast<int>(rank) * slice_vecs;
+  const int my_vecs = max(0, min(slice_vecs, nvec - v0));
+  const float id = scan_identity<PROD>();
+  uint64_t keep, drop;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(keep));
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(drop));
+
+  if (tid == 0) {
+    cta_failed = 0;
+    mbar_init(smem_addr(&xbar[0]), 1);
+    mbar_init(smem_addr(&xbar[1]), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if (cs > 1) { cluster_arrive(); cluster_wait(); }
+
+  int par = 0;
+  uint32_t phases = 0;
+  int mv = my_vecs;                        // -1 once a wait ran out: nothing is loaded or stored any more
+  for (long long row = cluster_id(); row < p.rows; row += row_step, par ^= 1) {
+    if (*reinterpret_cast<volatile int*>(&cta_failed)) mv = -1;
+    const uint4* xs = reinterpret_cast<const uint4*>(reinterpret_cast<const T*>(p.x) + row * p.xs) + v0;
+    uint4* ys = reinterpret_cast<uint4*>(reinterpret_cast<T*>(p.y) + row * p.ys) + v0;
+
+    // ---- phase 1: total of the slice
+    float t0 = id, t1 = id;
+    int v = tid;
+    for (; v + 7 * T_ < mv; v += 8 * T_) {
+      uint4 raw[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) raw[u] = scan_ld_hint(xs + v + u * T_, keep);
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        float f[EPV];
+        E::unpack(raw[u], f);
+#pragma unroll
+        for (int j = 0; j < EPV; j += 2) { t0 = scan_op<PROD>(t0, f[j]); t1 = scan_op<PROD>(t1, f[j + 1]); }
+      }
+    }
+    for (; v < mv; v += T_) {
+      float f[EPV];
+      E::unpack(scan_ld_hint(xs + v, keep), f);
+#pragma unroll
+      for (int j = 0; j < EPV; j += 2) { t0 = scan_op<PROD>(t0, f[j]); t1 = scan_op<PROD>(t1, f[j + 1]); }
+    }
+    float tot = scan_op<PROD>(t0, t1);
+#pragma unroll
+    for (int m = 16; m >= 1; m >>= 1) tot = scan_op<PROD>(tot, __shfl_xor_sync(0xffffffffu, tot, m));
+    if (lane == 0) red[warp] = tot;
+    __syncthreads();
+    tot = red[0];
+#pragma unroll
+    for (int w = 1; w < NW; ++w) tot = scan_op<PROD>(tot, red[w]);
+
+    // ---- exchange; carry-in = totals of the slices before mine, in slice order
+    float carry = id;
+    if (cs > 1) {
+      if (tid == 0) mbar_expect_tx(smem_addr(&xbar[par]), cs * 16u);
+      if (tid < static_cast<int>(cs))
+        st_async_f32x4(smem_addr(&inbox[par][rank]), smem_addr(&xbar[par]), static_cast<uint32_t>(tid), tot, 0.f, 0.f, 0.f);
+      if (mv >= 0 && !mbar_wait_timed<true>(smem_addr(&xbar[par]), (phases >> par) & 1u, status, wait_us)) {
+        mv = -1;
+        cta_failed = 1;
+      }
+      phases ^= 1u << par;
+      for (uint32_t k = 0; k < rank; ++k) carry = scan_op<PROD>(carry, inbox[par][k].x);
+    }
+
+    // ---- phase 2: scan of the slice from the carry-in (chunks of U * T_ vectors, as scan_kernel)
+    int cpar = 0;
+    uint4 ahead[U];                        // a chunk's vectors are loaded one chunk ahead
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int i = u * T_ + tid;
+      if (i < mv) ahead[u] = scan_ld_hint(xs + i, drop);
+    }
+    for (int base = 0; base < my_vecs; base += U * T_, cpar ^= 1) {     // (every thread: the chunks have a barrier)
+      float val[U][EPV];
+      uint4 raw[U];
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        raw[u] = ahead[u];
+        const int i = base + (U + u) * T_ + tid;
+        if (i < mv) ahead[u] = scan_ld_hint(xs + i, drop);
+      }
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const int i = base + u * T_ + tid;
+        float f[EPV];
+        if (i < mv) E::unpack(raw[u], f);
+#pragma unroll
+        for (int j = 0; j < EPV; ++j) val[u][j] = (i < mv) ? f[j] : id;
+      }
+      float incl[U];
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+#pragma unroll
+        for (int j = 1; j < EPV; ++j) val[u][j] = scan_op<PROD>(val[u][j - 1], val[u][j]);
+        incl[u] = val[u][EPV - 1];
+      }
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+          const float o = __shfl_up_sync(0xffffffffu, incl[u], d);
+          if (lane >= d) incl[u] = scan_op<PROD>(o, incl[u]);
+        }
+      }
+      if (lane == 31) {
+#pragma unroll
+        for (int u = 0; u < U; ++u) wtot[cpar][u][warp] = incl[u];
+      }
+      __syncthreads();
+      float before = carry;
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        float pre = id, tot_u = id;
+#pragma unroll
+        for (int w = 0; w < NW; ++w) {
+          const float t = wtot[cpar][u][w];
+          if (w < warp) pre = scan_op<PROD>(pre, t);
+          tot_u = scan_op<PROD>(tot_u, t);
+        }
+        float mine = scan_op<PROD>(before, pre);
+        before = scan_op<PROD>(before, tot_u);
+        const float excl = __shfl_up_sync(0xffffffffu, incl[u], 1);
+        if (lane > 0) mine = scan_op<PROD>(mine, excl);
+        const int i = base + u * T_ + tid;
+        if (i < mv) {
+          float o[EPV];
+#pragma unroll
+          for (int j = 0; j < EPV; ++j) o[j] = scan_op<PROD>(mine, val[u][j]);
+          st_stream(ys + i, E::pack(o));
+        }
+      }
+      carry = before;
+    }
+    __syncthreads();                       // red[] and wtot[] of the next row
+  }
+  if (cs > 1) { cluster_arrive(); cluster_wait(); }   // nobody leaves while a peer may still send to it
 }
 
 }  // namespace akg

@@ -156,12 +156,17 @@ __global__ void __launch_bounds__(THREADS) smem_kernel(const RowParams p, const 
     }
   };
 
-  if (threadIdx.x == 0) {
+  int in_flight = 0;                 // thread 0: slices issued and not yet waited for
+  if (threadIdx.x == 0 && !p.no_copies) {
     long long r = first_row;
-    for (int b = 0; b < g.nbuf && r < p.rows; ++b, r += row_step) issue(r, b);
+    for (int b = 0; b < g.nbuf && r < p.rows; ++b, r += row_step) { issue(r, b); ++in_flight; }
   }
 
-  long long it = 0;
+  // A wait that runs out makes the whole CTA "dead" (the vote below): it reads and stores nothing any
+  // more and issues no copy, but goes on through its rows for the sake of the cluster exchange, so that
+  // no peer waits at a cluster barrier for a CTA that has left.
+  bool dead = false;
+  long long it = 0, dead_it = 0;     // dead_it: the iteration whose wait ran out
   for (long long row = first_row; row < p.rows; row += row_step, ++it) {
     const int b = static_cast<int>(it % g.nbuf);
     const uint32_t phase = static_cast<uint32_t>((it / g.nbuf) & 1);
@@ -172,13 +177,20 @@ __global__ void __launch_bounds__(THREADS) smem_kernel(const RowParams p, const 
     const T* ar = (SM && p.add != nullptr)
                       ? reinterpret_cast<const T*>(p.add) + add_row(p, row) * p.add_stride
                       : nullptr;
-    mbar_wait_bounded(smem_addr(&bars[b]), phase, p.status);
+    if (!dead) {
+      if (__syncthreads_or(mbar_wait_timed(smem_addr(&bars[b]), phase, p.status, p.wait_us) ? 0 : 1)) {
+        dead = true;
+        dead_it = it;
+      } else if (threadIdx.x == 0) {
+        --in_flight;
+      }
+    }
 
     // ---- pass 1: thread-local statistics over my slice.  `plain` = no element of the
     // slice is masked: four vectors per step, loads first, one rescale per block.
     Stat st = stat_identity<OP>();
     const bool plain = !SM || (ar == nullptr && (v0 + lv) * EPV <= live);
-    int v = threadIdx.x;
+    int v = dead ? lv : static_cast<int>(threadIdx.x);          // a dead CTA folds nothing
     if (plain) {
       for (; v + 3 * THREADS < lv; v += 4 * THREADS) {
         float z[4][EPV];
@@ -226,7 +238,7 @@ __global__ void __launch_bounds__(THREADS) smem_kernel(const RowParams p, const 
 
     // ---- pass 2: normalise from shared memory, 128-bit stores
     T* yr = reinterpret_cast<T*>(p.y) + row * p.ys + static_cast<long long>(v0) * EPV;
-    v = threadIdx.x;
+    v = dead ? my_vecs : static_cast<int>(threadIdx.x);         // ... and stores nothing
     if (plain && lv == my_vecs) {
       for (; v + 3 * THREADS < my_vecs; v += 4 * THREADS) {
         float z[4][EPV];
@@ -288,14 +300,19 @@ __global__ void __launch_bounds__(THREADS) smem_kernel(const RowParams p, const 
 
     // ---- the buffer is free once every thread has read it: refill for row it + nbuf
     __syncthreads();
-    if (threadIdx.x == 0) {
+    if (threadIdx.x == 0 && !dead && !p.no_copies) {
       const long long next = row + row_step * g.nbuf;
-      if (next < p.rows) issue(next, b);
+      if (next < p.rows) { issue(next, b); ++in_flight; }
     }
+  }
+  // no copy may still be on its way into this CTA's shared memory when it leaves
+  if (threadIdx.x == 0 && dead) {
+    for (long long k = dead_it; in_flight > 0; --in_flight, ++k)
+      (void)mbar_wait_timed(smem_addr(&bars[k % g.nbuf]), static_cast<uint32_t>((k / g.nbuf) & 1), nullptr, p.wait_us);
   }
   // Peers write into this CTA's shared memory only before the cluster barrier of a row
   // this CTA also takes part in, so leaving after the last row is safe; every bulk copy
-  // issued was waited for above (each issued row is consumed by the loop).
+  // issued was waited for above (each issued row is consumed by the loop, or drained).
 }
 
 }  // namespace akg

@@ -143,6 +143,40 @@ __device__ __forceinline__ uint4 split_apply_plain(const RowParams& p, const Row
   using E = Elem<T>;
   constexpr int EPV = E::EPV;
   constexpr bool SM = OpTraits<OP>::kSoftmaxLike;
+  if constexpr (!SM && sizeof(T) == 2) {
+    // 16-bit normalisations with every affine vector present (the usual call): the stored values go
+    // into the arithmetic as they are (see Elem::fma_wide), only gamma is unpacked for LayerNorm
+    //   RMSNorm   (x * w) * rstd            the product of two 16-bit values is exact in fp32
+    //   LayerNorm beta + ((x - mean) * rstd) * gamma
+    if (p.gamma != nullptr && (OP != OP_LAYERNORM || p.beta != nullptr)) {
+      const uint4 gw = ld_cached(reinterpret_cast<const T*>(p.gamma) + c0);
+      const uint32_t xs[4] = {raw.x, raw.y, raw.z, raw.w}, gs[4] = {gw.x, gw.y, gw.z, gw.w};
+      uint32_t out[4];
+      if constexpr (OP == OP_RMSNORM) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          unsigned short x0, x1, g0, g1;
+          halves(xs[i], x0, x1);
+          halves(gs[i], g0, g1);
+          out[i] = E::pack2(E::fma_wide(x0, g0, 0.f) * rs.q, E::fma_wide(x1, g1, 0.f) * rs.q);
+        }
+      } else {
+        const uint4 bw = ld_cached(reinterpret_cast<const T*>(p.beta) + c0);
+        const uint32_t bs[4] = {bw.x, bw.y, bw.z, bw.w};
+        float ga[EPV];
+        E::unpack(gw, ga);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          unsigned short x0, x1, b0, b1;
+          halves(xs[i], x0, x1);
+          halves(bs[i], b0, b1);
+          out[i] = E::pack2(E::add_wide(b0, E::sub_wide(x0, rs.p) * rs.q * ga[2 * i]),
+                            E::add_wide(b1, E::sub_wide(x1, rs.p) * rs.q * ga[2 * i + 1]));
+        }
+      }
+      return make_uint4(out[0], out[1], out[2], out[3]);
+    }
+  }
   float z[EPV], ga[EPV], be[EPV], o[EPV];
   E::unpack(raw, z);
 #pragma unroll
@@ -275,20 +309,38 @@ __device__ __forceinline__ void split_step_use(const RowParams& p, uint4* yc, co
   for (int u = 0; u < 4; ++u)
     if (!PRED || v + u * THREADS < my_vecs)
       st_stream(yc + v + u * THREADS, split_apply_plain<OP, T>(p, rs, rc[u], (v0 + v + u * THREADS) * EPV));
-  if (kShiftedStats<OP, T>) {
-    // 16-bit LayerNorm: one sweep of sums about the thread's shift stn.a (see shifted_finish)
+  if constexpr (kShiftedStats<OP, T>) {
+    // 16-bit LayerNorm: one sweep of sums about the thread's shift stn.a (see shifted_finish); the
+    // stored values enter the subtraction as they are (Elem::sub_wide)
 #pragma unroll
     for (int u = 0; u < 4; ++u)
       if (!PRED || v + u * THREADS < my_vecs) {
-        float z[EPV];
-        E::unpack(rn[u], z);
+        const uint32_t ws[4] = {rn[u].x, rn[u].y, rn[u].z, rn[u].w};
 #pragma unroll
-        for (int j = 0; j < EPV; ++j) {
-          const float d = z[j] - stn.a;
-          stn.b += d;
-          stn.c = fmaf(d, d, stn.c);
+        for (int i = 0; i < 4; ++i) {
+          unsigned short h0, h1;
+          halves(ws[i], h0, h1);
+          const float d0 = E::sub_wide(h0, stn.a), d1 = E::sub_wide(h1, stn.a);
+          stn.b += d0 + d1;
+          stn.c = fmaf(d1, d1, fmaf(d0, d0, stn.c));
         }
       }
+  } else if constexpr (OP == OP_RMSNORM && sizeof(T) == 2) {
+    // 16-bit RMSNorm: x * x + acc in one instruction per element (Elem::fma_wide), two chains
+    float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      if (!PRED || v + u * THREADS < my_vecs) {
+        const uint32_t ws[4] = {rn[u].x, rn[u].y, rn[u].z, rn[u].w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          unsigned short h0, h1;
+          halves(ws[i], h0, h1);
+          s0 = E::fma_wide(h0, h0, s0);
+          s1 = E::fma_wide(h1, h1, s1);
+        }
+      }
+    stn.a += s0 + s1;
   } else if (!PRED) {
     float z[4][EPV];
 #pragma unroll
@@ -367,7 +419,16 @@ split_kernel(const RowParams p, const int slice_vecs, const int xmode, const int
 
   int par = 0;
   uint32_t phases = 0;        // bit k: parity of the phase of xbar[k] that the next wait is for
-  bool failed = false;
+  // A thread whose wait ran out has mv = -1 vectors to work on from then on (mv is my_vecs otherwise): it
+  // loads and stores nothing, waits for nothing, and still passes every barrier and sends its CTA's
+  // partials, so that neither its CTA nor its cluster waits for it.  The flag in shared memory takes the
+  // rest of the CTA along at the next row.
+  __shared__ int cta_failed;
+  if (threadIdx.x == 0) cta_failed = 0;
+  int mv = my_vecs;
+  auto give_up_with_the_cta = [&]() {
+    if (*reinterpret_cast<volatile int*>(&cta_failed)) mv = -1;
+  };
   // thread statistics of a slice -> this CTA's partial, sent to every CTA of the cluster
   auto send_stats = [&](Stat st) -> Stat {
     st = cta_reduce<OP, NW>(st, red[par], p.l2e);
@@ -389,7 +450,10 @@ split_kernel(const RowParams p, const int slice_vecs, const int xmode, const int
   // ... and the statistics of the whole row, in every CTA of the cluster
   auto recv_stats = [&](Stat st) -> Stat {
     if (async_x) {
-      if (!mbar_wait_timed<true>(smem_addr(&xbar[par]), (phases >> par) & 1u, p.status)) failed = true;
+      if (mv >= 0 && !mbar_wait_timed<true>(smem_addr(&xbar[par]), (phases >> par) & 1u, p.status, p.wait_us)) {
+        mv = -1;
+        cta_failed = 1;
+      }
       phases ^= 1u << par;
       const float4 f = inbox[par][0];
       Stat r{f.x, f.y, f.z};
@@ -420,72 +484,73 @@ split_kernel(const RowParams p, const int slice_vecs, const int xmode, const int
     {
       SplitRow<T> first;
       first.xr = reinterpret_cast<const T*>(xc); first.yr = reinterpret_cast<T*>(yc); first.ar = nullptr;
-      first.live = static_cast<int>(p.cols); first.lv = my_vecs; first.plain = true;
+      first.live = static_cast<int>(p.cols); first.lv = mv; first.plain = true;
       split_pass1<OP, T, THREADS>(p, first, v0, threadIdx.x, st, keep);
     }
     st = send_stats(st);
     for (;; row += row_step, xc += dx, yc += dy) {
+      give_up_with_the_cta();
       const bool has_next = row + row_step < p.rows;
       const uint4* xn = xc + dx;
       int v = threadIdx.x;
       uint4 rn[4], rc[4];
-      const bool first_full = has_next && v + 3 * THREADS < my_vecs;
+      const bool first_full = has_next && v + 3 * THREADS < mv;
       if (first_full) {                              // in flight while this thread waits for the partials
 #pragma unroll
         for (int u = 0; u < 4; ++u) rn[u] = ld_hint(xn + v + u * THREADS, keep);
       }
       st = recv_stats(st);
-      if (failed) break;
       const RowScalars rs = finalize<OP>(st, p.cols, p.eps);
       if (!has_next) {
         SplitRow<T> last;
         last.xr = reinterpret_cast<const T*>(xc); last.yr = reinterpret_cast<T*>(yc); last.ar = nullptr;
-        last.live = static_cast<int>(p.cols); last.lv = my_vecs; last.plain = true;
-        split_pass2<OP, T, THREADS>(p, last, rs, v0, my_vecs, v, drop);
+        last.live = static_cast<int>(p.cols); last.lv = mv; last.plain = true;
+        split_pass2<OP, T, THREADS>(p, last, rs, v0, mv, v, drop);
         break;
       }
       Stat stn = stat_identity<OP>();
-      if (kShiftedStats<OP, T> && v < my_vecs)       // the shift: the first element this thread owns
+      if (kShiftedStats<OP, T> && v < mv)       // the shift: the first element this thread owns
         stn.a = Elem<T>::load1(xn + v, 0);
-      if (first_full) {
+      if (first_full && mv >= 0) {
 #pragma unroll
         for (int u = 0; u < 4; ++u) rc[u] = ld_hint(xc + v + u * THREADS, drop);
         const uint4* demote = (l2mode == 0 && ((reinterpret_cast<uintptr_t>(xc) & 127u) == 0)) ? xc : nullptr;
-        split_step_use<OP, T, THREADS, false>(p, yc, rs, v0, v, my_vecs, rn, rc, stn, demote);
+        split_step_use<OP, T, THREADS, false>(p, yc, rs, v0, v, mv, rn, rc, stn, demote);
         v += 4 * THREADS;
-        for (; v + 3 * THREADS < my_vecs; v += 4 * THREADS) {
-          split_step_load<THREADS, false>(xn, xc, v, my_vecs, keep, drop, rn, rc);
-          split_step_use<OP, T, THREADS, false>(p, yc, rs, v0, v, my_vecs, rn, rc, stn, demote);
+        for (; v + 3 * THREADS < mv; v += 4 * THREADS) {
+          split_step_load<THREADS, false>(xn, xc, v, mv, keep, drop, rn, rc);
+          split_step_use<OP, T, THREADS, false>(p, yc, rs, v0, v, mv, rn, rc, stn, demote);
         }
       }
-      if (v < my_vecs) {                             // the ragged last step: its loads in flight together
-        split_step_load<THREADS, true>(xn, xc, v, my_vecs, keep, drop, rn, rc);
-        split_step_use<OP, T, THREADS, true>(p, yc, rs, v0, v, my_vecs, rn, rc, stn);
+      if (v < mv) {                             // the ragged last step: its loads in flight together
+        split_step_load<THREADS, true>(xn, xc, v, mv, keep, drop, rn, rc);
+        split_step_use<OP, T, THREADS, true>(p, yc, rs, v0, v, mv, rn, rc, stn);
       }
       if (kShiftedStats<OP, T>) {
         const int t = static_cast<int>(threadIdx.x);
-        stn = shifted_finish(stn, t < my_vecs ? ((my_vecs - 1 - t) / THREADS + 1) * Elem<T>::EPV : 0);
+        stn = shifted_finish(stn, t < mv ? ((mv - 1 - t) / THREADS + 1) * Elem<T>::EPV : 0);
       }
       st = send_stats(stn);
     }
   } else if (row < p.rows) {
     // ---- masked rows: slices may be cut short by the causal rule or carry an additive mask
-    SplitRow<T> cur = split_row<OP, T>(p, row, v0, my_vecs);
+    SplitRow<T> cur = split_row<OP, T>(p, row, v0, mv);
     Stat st = stat_identity<OP>();
     split_pass1<OP, T, THREADS>(p, cur, v0, threadIdx.x, st, keep);
     st = send_stats(st);
     for (;;) {
+      give_up_with_the_cta();
       st = recv_stats(st);
-      if (failed) break;
+      if (mv < 0) { cur.lv = 0; cur.plain = false; }
       const RowScalars rs = finalize<OP>(st, p.cols, p.eps);
       const long long next_row = row + row_step;
       if (next_row >= p.rows) {
-        split_pass2<OP, T, THREADS>(p, cur, rs, v0, my_vecs, threadIdx.x, drop);
+        split_pass2<OP, T, THREADS>(p, cur, rs, v0, mv, threadIdx.x, drop);
         break;
       }
-      const SplitRow<T> nxt = split_row<OP, T>(p, next_row, v0, my_vecs);
+      const SplitRow<T> nxt = split_row<OP, T>(p, next_row, v0, mv);
       Stat stn = stat_identity<OP>();
-      split_pass2<OP, T, THREADS>(p, cur, rs, v0, my_vecs, threadIdx.x, drop);
+      split_pass2<OP, T, THREADS>(p, cur, rs, v0, mv, threadIdx.x, drop);
       split_pass1<OP, T, THREADS>(p, nxt, v0, threadIdx.x, stn, keep);
       st = send_stats(stn);
       cur = nxt;

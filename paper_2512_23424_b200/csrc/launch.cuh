@@ -68,6 +68,12 @@ cudaError_t launch_cumulative(bool want_prod, int dtype, bool vec, const void* x
                               long long cols, long long xs, long long ys, unsigned grid, int threads, bool warp_rows,
                               int pdl, cudaStream_t stream);
 
+// Few, long rows: a cluster of `cluster` CTAs (256 threads) per row, slices of slice_vecs vectors, the carry
+// of a slice from its cluster peers (scan_split_kernel); vectorised rows only.  clusters = 0: one resident wave.
+cudaError_t launch_cumulative_split(bool want_prod, int dtype, const void* x, void* y, long long rows, long long cols,
+                                    long long xs, long long ys, int cluster, int slice_vecs, long long clusters,
+                                    int* status, unsigned wait_us, cudaStream_t stream);
+
 // Short unmasked rows, 32 / lanes rows per warp (op_short.cu): lanes in {4, 8, 16, 32}, rows of
 // up to short_max_vectors(lanes) vectors.
 int short_rows_per_cta(int lanes);

@@ -24,6 +24,12 @@ namespace akg {
   X(512, 1, 512) X(512, 2, 512) X(512, 4, 512) X(512, 8, 512) \
   X(1024, 1, 1024) X(1024, 2, 1024) X(1024, 4, 1024) X(1024, 8, 1024)
 
+// Shapes that are compiled for element type T.  The 16-bit types never get a CTA of 1024 threads or eight
+// vectors per thread in a CTA of 256 and more from the planner (rows beyond 2048 vectors leave the register
+// family, and the fat-thread normalisation is reg_norm_flex); those bodies spilled 0.2 - 1 KB per thread.
+template <typename T, int G_, int V_, int T_>
+constexpr bool kRegShapeBuilt = sizeof(T) == 4 || !((T_) >= 1024 || ((V_) == 8 && (T_) >= 256));
+
 // Fill the launch attributes: programmatic stream serialisation when the plan asks for
 // it, a cluster dimension when cluster > 1.  Returns the number of attributes set.
 inline unsigned launch_attrs(cudaLaunchAttribute* attr, const LaunchPlan& plan, int cluster) {
@@ -231,7 +237,9 @@ cudaError_t launch_typed(const LaunchPlan& plan, const RowParams& p, cudaStream_
     // normalisation kernel); the softmax pair always takes its own lean kernel.
 #define AKG_REG_CASE(G_, V_, T_)                                              \
   if (plan.group == (G_) && plan.vpt == (V_) && plan.threads == (T_)) {       \
-    if constexpr (OpTraits<OP>::kSoftmaxLike) {                               \
+    if constexpr (!kRegShapeBuilt<T, G_, V_, T_>) {                           \
+      return cudaErrorInvalidConfiguration;                                   \
+    } else if constexpr (OpTraits<OP>::kSoftmaxLike) {                        \
       return launch_plain(reg_softmax<OP, T, G_, V_, T_>, plan, plan.grid, T_, 0, s, p);      \
     } else {                                                                  \
       if (plan.stages == 1)                                                   \

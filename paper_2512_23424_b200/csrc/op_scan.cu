@@ -1,4 +1,7 @@
 // Arg-max / arg-min and cumulative sum / product over the last axis: kernels and launchers.
+#include <map>
+#include <mutex>
+
 #include "kernels_arg.cuh"
 #include "kernels_scan.cuh"
 #include "launch.cuh"
@@ -66,9 +69,74 @@ cudaError_t launch_scan_t(bool vec, bool warp_rows, const ScanParams& p, unsigne
              : launch_1d(scan_kernel<PROD, T, false>, p, grid, threads, pdl, s);
 }
 
+// scan_split_kernel: a cluster of `cluster` CTAs per row; clusters = 0 asks for one resident wave
+template <bool PROD, typename T>
+cudaError_t launch_scan_split_t(const ScanParams& p, int cluster, int slice_vecs, long long clusters, int* status,
+                                unsigned wait_us, cudaStream_t s) {
+  auto kernel = scan_split_kernel<PROD, T>;
+  static std::mutex mu;
+  static std::map<std::pair<int, int>, int> resident;   // (device, cluster) -> co-resident clusters
+  static std::map<int, bool> prepared;
+  int dev = 0;
+  cudaError_t err = cudaGetDevice(&dev);
+  if (err != cudaSuccess) return err;
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = static_cast<unsigned>(cluster);
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.blockDim = dim3(256);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = s;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  int max_clusters = 0;
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    if (!prepared[dev]) {
+      err = cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+      if (err != cudaSuccess) return err;
+      prepared[dev] = true;
+    }
+    auto key = std::make_pair(dev, cluster);
+    auto it = resident.find(key);
+    if (it == resident.end()) {
+      cfg.gridDim = dim3(static_cast<unsigned>(cluster) * 1024u);
+      int n = 0;
+      err = cudaOccupancyMaxActiveClusters(&n, kernel, &cfg);
+      if (err != cudaSuccess) return err;
+      it = resident.emplace(key, n).first;
+    }
+    max_clusters = it->second;
+  }
+  if (max_clusters < 1) return cudaErrorLaunchOutOfResources;
+  long long n = max_clusters;
+  if (clusters > 0 && clusters < n) n = clusters;
+  if (n > p.rows) n = p.rows;
+  if (n < 1) n = 1;
+  cfg.gridDim = dim3(static_cast<unsigned>(n * cluster));
+  return cudaLaunchKernelEx(&cfg, kernel, p, slice_vecs, status, wait_us);
+}
+
 }  // namespace
 
 int scan_unroll() { return kScanU; }
+
+cudaError_t launch_cumulative_split(bool want_prod, int dtype, const void* x, void* y, long long rows, long long cols,
+                                    long long xs, long long ys, int cluster, int slice_vecs, long long clusters,
+                                    int* status, unsigned wait_us, cudaStream_t stream) {
+  ScanParams p;
+  p.x = x; p.y = y; p.rows = rows; p.cols = cols; p.xs = xs; p.ys = ys;
+  if (dtype == DT_F32)
+    return want_prod ? launch_scan_split_t<true, float>(p, cluster, slice_vecs, clusters, status, wait_us, stream)
+                     : launch_scan_split_t<false, float>(p, cluster, slice_vecs, clusters, status, wait_us, stream);
+  if (dtype == DT_F16)
+    return want_prod ? launch_scan_split_t<true, __half>(p, cluster, slice_vecs, clusters, status, wait_us, stream)
+                     : launch_scan_split_t<false, __half>(p, cluster, slice_vecs, clusters, status, wait_us, stream);
+  return want_prod ? launch_scan_split_t<true, __nv_bfloat16>(p, cluster, slice_vecs, clusters, status, wait_us, stream)
+                   : launch_scan_split_t<false, __nv_bfloat16>(p, cluster, slice_vecs, clusters, status, wait_us, stream);
+}
 
 cudaError_t launch_argreduce(bool want_min, int dtype, bool vec, bool warp_rows, const void* x, long long* out,
                              long long rows, long long cols, long long xs, unsigned grid, unsigned segments,

@@ -1,5 +1,5 @@
 // Thin wrappers over the PTX used by the shared-memory ring and cluster kernels:
-// mbarrier (with bounded waits), untiled bulk copies global -> shared (TMA, never
+// mbarrier (with waits bounded by the global timer), untiled bulk copies global -> shared (TMA, never
 // multicast), cluster identity / barrier, and distributed-shared-memory stores.
 #pragma once
 
@@ -7,7 +7,6 @@
 
 namespace akg {
 
-constexpr uint32_t kWaitLimit = 1u << 22;     // bounded mbarrier wait (each try blocks for a while)
 constexpr int kStatusTimeout = 1;
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) {
@@ -28,19 +27,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
                "selp.u32 %0, 1, 0, p;\n\t}" : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-// Wait for a phase with an iteration limit; on expiry the status word is set and the
-// caller carries on (its output for that row is then undefined, never out of bounds).
-__device__ __forceinline__ void mbar_wait_bounded(uint32_t bar, uint32_t parity, int* status) {
-  for (uint32_t i = 0; i < kWaitLimit; ++i)
-    if (mbar_try_wait(bar, parity)) return;
-  if (status != nullptr) atomicExch(status, kStatusTimeout);
-}
 __device__ __forceinline__ unsigned long long global_timer_ns() {
   unsigned long long t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
-// Wait for a phase, at most kWaitNs of the global timer.  False on expiry, with the status word set.
+// Wait for a phase, at most limit_ns of the global timer (two seconds unless the call says otherwise:
+// RowParams::wait_us).  False on expiry, with the status word set; what a kernel does then is written
+// at its waits: it stops storing, issues no further copy, keeps taking part in its CTA's and cluster's
+// barriers, and waits (bounded again) for the copies it still has in flight before it leaves.
 // CLUSTER: acquire at cluster scope (the data was written by another CTA of the cluster); otherwise
 // the default, CTA scope (data written by this CTA's bulk copies).
 constexpr unsigned long long kWaitNs = 2000000000ull;
@@ -56,9 +51,9 @@ __device__ __forceinline__ bool mbar_try_wait_scope(uint32_t bar, uint32_t parit
   return ok != 0;
 }
 template <bool CLUSTER = false>
-__device__ __forceinline__ bool mbar_wait_timed(uint32_t bar, uint32_t parity, int* status,
-                                                unsigned long long limit_ns = kWaitNs) {
+__device__ __forceinline__ bool mbar_wait_timed(uint32_t bar, uint32_t parity, int* status, unsigned wait_us = 0) {
   if (mbar_try_wait_scope<CLUSTER>(bar, parity)) return true;
+  const unsigned long long limit_ns = wait_us ? wait_us * 1000ull : kWaitNs;    // (off the fast path)
   const unsigned long long t0 = global_timer_ns();
   for (;;) {
     if (mbar_try_wait_scope<CLUSTER>(bar, parity)) return true;

@@ -349,6 +349,8 @@ REDUCTION_CONFIGS: Dict[str, tuple] = {
     "cumsum_f32_16384x8192": ("cumsum", F32, 16384, 8192),
     "cumsum_bf16_16384x8192": ("cumsum", BF16, 16384, 8192),
     "cumprod_f32_16384x8192": ("cumprod", F32, 16384, 8192),
+    "cumsum_f32_256x262144": ("cumsum", F32, 256, 262144),
+    "cumsum_bf16_256x262144": ("cumsum", BF16, 256, 262144),
 }
 
 

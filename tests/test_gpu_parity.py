@@ -266,6 +266,26 @@ def test_in_place(op, dtype):
             compare(to_numpy(x), ref, dtype, f"in-place {w.name}[{v}]", cancel_magnitude(w, ref))
 
 
+def test_interleaved_column_windows_of_one_buffer():
+    """x = buf[:, :cols] and y = buf[:, cols:] share rows of one buffer but no element: accepted."""
+    for dtype in (wl.F32, wl.BF16):
+        w = wl.make_random("rmsnorm", dtype, 48, 512, seed=77, eps=1e-6)
+        tdt = torch.float32 if dtype == wl.F32 else torch.bfloat16
+        buf = torch.zeros((w.rows, 2 * w.cols), dtype=tdt, device="cuda")
+        buf[:, :w.cols] = to_torch(w.x, dtype)
+        before = buf[:, :w.cols].clone()
+        run_gpu(w, x_dev=buf[:, :w.cols], out=buf[:, w.cols:])
+        torch.cuda.synchronize()
+        compare(to_numpy(buf[:, w.cols:]), run_oracle(w), dtype, "interleaved windows")
+        assert torch.equal(buf[:, :w.cols], before)
+    # windows that do share elements are still refused
+    L = akg.lib()
+    f = torch.zeros(4 * 24, device="cuda")
+    assert L.akg_softmax(f.data_ptr(), f.data_ptr() + 4 * 4, 4, 8, 24, 24, 0, None, None) == 1
+    assert L.akg_softmax(f.data_ptr(), f.data_ptr() + 4 * 20, 4, 8, 24, 24, 0, None, None) == 1
+    assert L.akg_softmax(f.data_ptr(), f.data_ptr() + 4 * 8, 3, 8, 24, 24, 0, None, None) == 0
+
+
 def test_empty_and_invalid_arguments():
     x = torch.zeros((4, 8), device="cuda")
     y = torch.empty_like(x)

@@ -116,7 +116,15 @@ def test_long_causal_rows_mix_merged_and_plain_steps(dtype):
 def test_sixteen_bit_rows_beyond_2048_vectors_leave_the_register_form(dtype):
     for op in ("softmax", "layernorm", "rmsnorm"):
         check(wl.make_random(op, dtype, 200, 20480, seed=350), ("split", "cs2,"))
-        check(wl.make_random(op, dtype, 600, 20480, seed=351), ("split", "cs1,"))
+        if op != "rmsnorm":
+            check(wl.make_random(op, dtype, 600, 20480, seed=351), ("split", "cs1,"))
+    # with rows for every SM, unmasked 16-bit log-softmax rows of 16 - 48 KB and RMSNorm rows of 32 - 64 KB
+    # take the kernel that keeps the row in shared memory (three CTAs of 256 / two of 512 per SM)
+    check(wl.make_random("rmsnorm", dtype, 600, 20480, seed=351), ("tma<", "t512,"))
+    check(wl.make_random("rmsnorm", dtype, 310, 32768, seed=355), ("tma<", "t512,"))
+    check(wl.make_random("log_softmax", dtype, 600, 12288, seed=356, scale=2.0), ("tma<", "t256,"))
+    check(wl.make_random("log_softmax", dtype, 333, 20480 + 8, seed=357, scale=2.0), ("tma<", "t256,"))
+    check(wl.make_random("log_softmax", dtype, 100, 16384, seed=358, scale=2.0), ("reg<",))
     # the fp32 normalisations stay in registers while the row is an exact fit, ragged rows do not
     check(wl.make_random("rmsnorm", wl.F32, 300, 32768, seed=352), ("reg", "flex"))
     check(wl.make_random("layernorm", wl.F32, 300, 32000, seed=353), ("split",))

@@ -134,6 +134,43 @@ def test_cumulative_shapes(dtype):
 
 
 @pytest.mark.parametrize("dtype", DTYPES)
+def test_cumulative_long_rows_split_over_a_cluster(dtype):
+    """Few, long rows: a cluster per row, a slice per CTA, the carry of a slice from the peers' totals."""
+    rng = np.random.default_rng(25)
+    epv = 4 if dtype == wl.F32 else 8
+    try:
+        for rows, cols, cs in [(3, 65536 * epv // 4, 0), (2, 262144 + 8, 0), (5, 100000, 4), (7, 40960, 2),
+                               (2, 70000 * epv // 4 + epv, 16), (300, 9000 * epv, 8), (1, 4096 * epv, 8)]:
+            akg.set_tuning("cluster_size", cs)
+            x = rng.normal(0.05, 1, (rows, cols)).astype(np.float32)
+            check_cum("cumsum", store(x, dtype), dtype, f"{rows}x{cols} cs{cs}")
+            assert akg.last_kernel().startswith("scan_split<"), akg.last_kernel()
+            if cs:
+                assert f"cs{cs}," in akg.last_kernel()
+            f = (1.0 + 0.002 * rng.normal(0, 1, (rows, cols))).astype(np.float32)
+            f[rng.random((rows, cols)) < 0.01] *= -1
+            check_cum("cumprod", store(f, dtype), dtype, f"{rows}x{cols} cs{cs}")
+            assert akg.last_kernel().startswith("scan_split<")
+        # exact arithmetic across slices: small integers, and in place with padded rows
+        akg.set_tuning("cluster_size", 4)
+        x = rng.integers(-2, 3, (3, 24576)).astype(np.float32)
+        ref = oracle.cumulative("cumsum", x)
+        tdt = torch.float32 if dtype == wl.F32 else torch.bfloat16
+        big = torch.full((3, 24576 + 8 * epv), 7.0, dtype=tdt, device="cuda")
+        big[:, :24576].copy_(to_torch(store(x, dtype), dtype))
+        binding.cumsum(big[:, :24576], out=big[:, :24576])
+        torch.cuda.synchronize()
+        assert akg.last_kernel().startswith("scan_split<")
+        got = widen(to_numpy(big[:, :24576].contiguous()))
+        exact = np.abs(ref) < (2 ** 24 if dtype == wl.F32 else 256)
+        assert np.array_equal(got[exact], ref[exact])
+        assert torch.all(big[:, 24576:] == 7.0)
+    finally:
+        akg.set_tuning("cluster_size", 0)
+    assert akg.device_status() == 0
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
 def test_cumulative_exact_cases_in_place_and_strides(dtype):
     tdt = torch.float32 if dtype == wl.F32 else torch.bfloat16
     # small integers: every partial sum is exact in fp32 (and in bf16 while below 256)
