@@ -723,6 +723,32 @@ def run_profile(args):
                           "us_per_launch": secs / args.steps * 1e6, "launches": args.steps + max(args.warmup, 3),
                           "algorithmic_bytes": w.algorithmic_bytes()}))
         return
+    if args.profile_next:
+        # one of the arg-max / cumulative / column-normalisation rows (workloads.REDUCTION_CONFIGS, COLNORM_CONFIGS)
+        name = args.profile_next
+        if name in wl.REDUCTION_CONFIGS:
+            wr = wl.make_reduction(name, rows=args.profile_rows)
+            fn = getattr(binding, wr.op)
+            x0 = _dev(wr.x, wr.dtype)
+            rxs = [x0] + [x0.clone() for _ in range(pairs_for(wr) - 1)]
+            routs = [fn(x) for x in rxs]
+            obj = _Rotating(torch, len(rxs), lambda k: fn(rxs[k], out=routs[k]))
+            nbytes, shape = wr.algorithmic_bytes(), list(wr.x.shape)
+        else:
+            wc = wl.make_colnorm(name, rows=args.profile_rows)
+            cx0 = _dev(wc.x, wc.dtype)
+            cxs = [cx0, cx0.clone()]
+            cys = [torch.empty_like(cx0) for _ in cxs]
+            cg, cb = _dev(wc.gamma, wc.dtype), _dev(wc.beta, wc.dtype)
+            cws = torch.empty(binding.colnorm_workspace_bytes(wc.rows, wc.cols) or 8, dtype=torch.uint8, device="cuda")
+            obj = _Rotating(torch, 2, lambda k: binding.colnorm(cxs[k], cg, cb, eps=wc.eps, out=cys[k], workspace=cws))
+            nbytes, shape = 3 * wc.rows * wc.cols * wc.itemsize, [wc.rows, wc.cols]
+        secs = time_launches(obj, args.steps, args.warmup)
+        print(json.dumps({"profile": name, "shape": shape, "kernel": binding.last_kernel(),
+                          "us_per_launch": secs / args.steps * 1e6, "launches": args.steps + max(args.warmup, 3),
+                          "algorithmic_bytes": nbytes,
+                          "frac_of_copy_peak": nbytes / (secs / args.steps) / 1e9 / measured_peak()[0]}))
+        return
     if args.profile_shape:
         op, dname, rows, cols = args.profile_shape.split(":")
         dtype = {"f32": wl.F32, "bf16": wl.BF16, "f16": wl.F16}[dname]
@@ -804,6 +830,9 @@ def main():
                     help="as --profile, for a gated-activation configuration (workloads.ACT_CONFIGS)")
     ap.add_argument("--profile-fused", default="", metavar="NAME",
                     help="as --profile, for a fused residual add + normalisation configuration (workloads.FUSED_CONFIGS)")
+    ap.add_argument("--profile-next", default="", metavar="NAME",
+                    help="as --profile, for an arg-max / cumulative / column-normalisation row of the bench "
+                         "(workloads.REDUCTION_CONFIGS, COLNORM_CONFIGS)")
     ap.add_argument("--profile-shape", default="", metavar="OP:DTYPE:ROWS:COLS",
                     help="as --profile, for a seeded random matrix, e.g. layernorm:bf16:512:131072")
     ap.add_argument("--profile-rows", type=int, default=None,
@@ -818,7 +847,7 @@ def main():
             args.steps = 20
         run_sweep(args)
         return
-    if args.profile or args.profile_axis or args.profile_fused or args.profile_act or args.profile_shape:
+    if args.profile or args.profile_axis or args.profile_fused or args.profile_act or args.profile_shape or args.profile_next:
         run_profile(args)
     elif args.impl == "reference":
         run_reference(args)

@@ -288,6 +288,7 @@ bool plan_smem(const Call& c, int cs_min, int cs_max, LaunchPlan* plan, int want
   if (best_cs == 0) return false;
   const int64_t buf = (best_slice * 16 + 127) & ~int64_t(127);
   plan->variant = (best_cs == 1) ? V_TMA : V_CLUSTER;
+  plan->mode = (best_cs > 1 && g_tune_split_exchange.load() == 1) ? 1 : 0;   // clusters, 1: partials exchanged under a cluster barrier
   plan->threads = best_threads; plan->group = best_threads; plan->vpt = static_cast<int>(best_slice);
   plan->cluster = best_cs; plan->stages = best_nbuf;
   plan->smem = smem_header_bytes(best_threads) + static_cast<size_t>(best_nbuf) * buf;
@@ -1283,6 +1284,9 @@ extern "C" akg_status akg_colnorm(const void* x, void* y, int64_t rows, int64_t 
   p.x = x; p.y = y; p.rows = rows; p.cols = cols; p.xs = x_row_stride; p.ys = y_row_stride;
   p.gamma = gamma; p.beta = beta; p.eps = eps; p.partial = static_cast<float2*>(workspace);
   p.mean_out = mean_out; p.var_out = var_out; p.rows_per_block = rpb; p.lc_shift = lc_shift;
+  // L2 priorities ("keep" while the statistics are taken, "drop" when the rows are read again) while the
+  // matrix is at most about twice the size of L2
+  p.l2_keep = (static_cast<long double>(rows) * cols * es <= 288.0L * 1048576.0L) ? 1 : 0;
   const dim3 grid(static_cast<unsigned>(strips), static_cast<unsigned>(rb));
   const cudaError_t err = launch_colnorm(static_cast<int>(dtype), vec, p, grid, g_tune_pdl.load() == 2 ? 0 : 1,
                                          static_cast<cudaStream_t>(stream));

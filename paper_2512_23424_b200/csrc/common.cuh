@@ -78,6 +78,7 @@ struct ColParams {
   float* var_out;                     // [cols] or nullptr
   long long rows_per_block;           // a multiple of the CTA's row slots
   int lc_shift;                       // log2 of the lanes of a warp that lie along the columns
+  int l2_keep;                        // 1: the matrix is small enough for L2 priorities to pay (see kernels_colnorm.cuh)
 };
 
 // Shared-memory ring kernels: limits and the size of the bookkeeping area that
@@ -85,8 +86,10 @@ struct ColParams {
 constexpr int kMaxCluster = 16;
 constexpr int kMaxBuf = 16;
 constexpr unsigned kMaxDynSmem = 232448;      // 227 KiB opt-in limit per CTA
+// layout: ring mbarriers [kMaxBuf] | exchange mbarriers [4] | inbox of the st.async exchange
+// [4][kMaxCluster] x 16 bytes | CTA reduction slots [2][warps] | remote-store slots [2][kMaxCluster]
 __host__ __device__ constexpr unsigned smem_header_bytes(int threads) {
-  return (kMaxBuf * 8u + (2u * (threads / 32) + 2u * kMaxCluster) * 12u + 127u) & ~127u;
+  return (kMaxBuf * 8u + 4u * 8u + 4u * kMaxCluster * 16u + (2u * (threads / 32) + 2u * kMaxCluster) * 12u + 127u) & ~127u;
 }
 
 // Programmatic dependent launch.  Every kernel starts with this: it waits until the
@@ -314,6 +317,19 @@ template <int OP> __device__ __forceinline__ Stat warp_reduce(Stat s, float l2e 
   return s;
 }
 
+// Merge n statistics (n a power of two, at most 32) held one per lane, lane l holding entry l mod n, by a
+// butterfly of log2 n steps.  Both partners of a step merge (entry of the lower lane, entry of the higher
+// lane) in that order, so every lane ends with the same bits; a serial merge of 16 entries is a chain of 15
+// dependent merges (two exponentials each for the softmax pair), this one of four.
+template <int OP> __device__ __forceinline__ Stat butterfly_merge(Stat s, int n, float l2e = kLog2e) {
+  const int lane = threadIdx.x & 31;
+  for (int k = 1; k < n; k <<= 1) {
+    const Stat o = stat_shfl_xor<OP>(s, k);
+    s = (lane & k) ? stat_merge<OP>(o, s, l2e) : stat_merge<OP>(s, o, l2e);
+  }
+  return s;
+}
+
 // Reduce over a whole CTA of NW warps.  `slots` points at NW Stat entries of shared
 // memory reserved for this call; callers alternate between two slot sets on
 // successive rows so one barrier per row is enough.  Every thread gets the result,
@@ -323,10 +339,14 @@ template <int OP, int NW> __device__ __forceinline__ Stat cta_reduce(Stat s, Sta
   if (NW == 1) return s;
   if ((threadIdx.x & 31) == 0) slots[threadIdx.x >> 5] = s;
   __syncthreads();
-  Stat r = slots[0];
+  if constexpr ((NW & (NW - 1)) == 0 && NW <= 32) {
+    return butterfly_merge<OP>(slots[threadIdx.x & (NW - 1)], NW, l2e);
+  } else {
+    Stat r = slots[0];
 #pragma unroll
-  for (int w = 1; w < NW; ++w) r = stat_merge<OP>(r, slots[w], l2e);
-  return r;
+    for (int w = 1; w < NW; ++w) r = stat_merge<OP>(r, slots[w], l2e);
+    return r;
+  }
 }
 
 // Row scalars derived from the reduced statistics.

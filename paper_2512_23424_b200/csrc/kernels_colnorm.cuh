@@ -2,12 +2,16 @@
 // column of x[rows, cols] is normalised with its own mean and biased variance over the rows and
 // a per-column affine.  The reduction runs across rows, so a column's statistics come from every
 // part of the matrix: two kernels on one stream, with a small workspace between them.
-//   col_stat_kernel   grid (column strips, row blocks): per-column (mean, M2) of the block's rows,
-//                     written to workspace[block][column]
-//   col_apply_kernel  same grid: merges the blocks' pairs of its columns (Chan's formula, counts
-//                     known from the geometry), derives mean and 1 / std once per column, then
-//                     normalises its block of rows
-// x is read twice; the second read is served by L2 while the matrix fits there.  Threads own
+//   col_stat_kernel    grid (column strips, row blocks): per-column (mean, M2) of the block's rows,
+//                      written to workspace[block][column]; its loads mark their lines "keep in L2"
+//   col_finish_kernel  a warp per column merges the blocks' pairs (counts known from the geometry) and
+//                      leaves (mean, 1 / std) in workspace[0][column]: once per column, not once per CTA
+//                      of the third kernel (147 row blocks x 4 strips each merged all 147 pairs of their
+//                      256 columns before: 40 M warp instructions against 16 M of the statistics kernel)
+//   col_apply_kernel   the first kernel's grid, walked in REVERSE block order: the blocks the statistics
+//                      kernel read last are the ones still in L2, so a matrix somewhat larger than L2 is
+//                      still re-read from there for the most part; normalises its block of rows
+// x is read twice; the second read is served by L2 as far as the matrix fits there.  Threads own
 // columns (a warp lies 1 << lc_shift lanes along the columns and the rest along rows), as in the
 // non-last-axis kernels, whose loaders and running statistics are reused.
 #pragma once
@@ -40,13 +44,15 @@ __global__ void __launch_bounds__(kAxisThreads, 4) col_stat_kernel(const ColPara
 
   AxisRun<OP_LAYERNORM, W> run;
   run.init();
+  // (a matrix far beyond L2 gains nothing from the marks and measured 8 % slower with them: plain priority then)
+  const uint64_t keep = p.l2_keep ? l2_policy_keep() : l2_policy_normal();
   if (active) {
     const T* px = reinterpret_cast<const T*>(p.x) + (r0 + slot) * p.xs + col0;
     long long f = r0 + slot;
     for (; f + (UB - 1) * ns < r1; f += UB * ns) {
       Raw raw[UB];
 #pragma unroll
-      for (int u = 0; u < UB; ++u, px += xstep) raw[u] = A::load(px);
+      for (int u = 0; u < UB; ++u, px += xstep) raw[u] = A::load_hint(px, keep);
       float v[UB][W];
 #pragma unroll
       for (int u = 0; u < UB; ++u) A::unpack(raw[u], v[u]);
@@ -86,62 +92,65 @@ __global__ void __launch_bounds__(kAxisThreads, 4) col_stat_kernel(const ColPara
   }
 }
 
+// A warp per column: lane l takes row blocks l, l + 32, ...; two sweeps (mean of the block means weighted by
+// their counts, then the M2 of the blocks about it), each finished by a shuffle sum.
+__global__ void __launch_bounds__(256) col_finish_kernel(const ColParams p, const int nblk) {
+  pdl_prologue();                              // the statistics kernel has completed when this returns
+  const int lane = threadIdx.x & 31;
+  const long long c = static_cast<long long>(blockIdx.x) * 8 + (threadIdx.x >> 5);
+  if (c >= p.cols) return;
+  const float inv_rows = 1.0f / static_cast<float>(p.rows);
+  auto count = [&](int b) {
+    return static_cast<float>(min(p.rows, (b + 1) * p.rows_per_block) - b * p.rows_per_block);
+  };
+  float mean = 0.f;
+  for (int b = lane; b < nblk; b += 32) mean = fmaf(count(b), p.partial[static_cast<long long>(b) * p.cols + c].x, mean);
+  mean = warp_sum(mean) * inv_rows;
+  float m2 = 0.f;
+  for (int b = lane; b < nblk; b += 32) {
+    const float2 pb = p.partial[static_cast<long long>(b) * p.cols + c];
+    const float d = pb.x - mean;
+    m2 += fmaf(count(b) * d, d, pb.y);
+  }
+  const float var = warp_sum(m2) * inv_rows;
+  __syncwarp();                                // every lane has read the column's pairs
+  if (lane == 0) {
+    p.partial[c] = make_float2(mean, rsqrt_refined(var + p.eps));
+    if (p.mean_out != nullptr) p.mean_out[c] = mean;
+    if (p.var_out != nullptr) p.var_out[c] = var;
+  }
+}
+
+
 template <typename T, int MODE>
 __global__ void __launch_bounds__(kAxisThreads, 4) col_apply_kernel(const ColParams p) {
-  pdl_prologue();                              // the statistics kernel has completed when this returns
+  pdl_prologue();                              // the merge kernel has completed when this returns
   using A = AxisRaw<T, MODE>;
   using E = Elem<T>;
   using Raw = typename A::Raw;
   constexpr int W = A::W;
   constexpr int UB = kColUB;
-  __shared__ float fin[2][32 * W];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int lc = 1 << p.lc_shift;
   const int lcol = lane & (lc - 1);
   const int slot = warp * (32 >> p.lc_shift) + (lane >> p.lc_shift);
   const int ns = kAxisThreads >> p.lc_shift;
   const int cw = lc * W;
-  const long long r0 = static_cast<long long>(blockIdx.y) * p.rows_per_block;
+  const long long blk = static_cast<long long>(gridDim.y) - 1 - blockIdx.y;     // last read, first re-read
+  const long long r0 = blk * p.rows_per_block;
   const long long r1 = min(p.rows, r0 + p.rows_per_block);
-
-  // ---- column statistics over all row blocks, once per column of this strip
-  const long long c = static_cast<long long>(blockIdx.x) * cw + threadIdx.x;
-  if (static_cast<int>(threadIdx.x) < cw && c < p.cols) {
-    const int nblk = static_cast<int>(gridDim.y);
-    const float inv_rows = 1.0f / static_cast<float>(p.rows);
-    float mean = 0.f;
-    for (int b = 0; b < nblk; ++b) {
-      const float nb = static_cast<float>(min(p.rows, (b + 1) * p.rows_per_block) - b * p.rows_per_block);
-      mean = fmaf(nb, p.partial[static_cast<long long>(b) * p.cols + c].x, mean);
-    }
-    mean *= inv_rows;
-    float m2 = 0.f;
-    for (int b = 0; b < nblk; ++b) {
-      const float nb = static_cast<float>(min(p.rows, (b + 1) * p.rows_per_block) - b * p.rows_per_block);
-      const float2 pb = p.partial[static_cast<long long>(b) * p.cols + c];
-      const float d = pb.x - mean;
-      m2 += fmaf(nb * d, d, pb.y);
-    }
-    const float var = m2 * inv_rows;
-    fin[0][threadIdx.x] = mean;
-    fin[1][threadIdx.x] = rsqrt_refined(var + p.eps);
-    if (blockIdx.y == 0) {
-      if (p.mean_out != nullptr) p.mean_out[c] = mean;
-      if (p.var_out != nullptr) p.var_out[c] = var;
-    }
-  }
-  __syncthreads();
-
   const long long col0 = static_cast<long long>(blockIdx.x) * cw + lcol * W;
   if (col0 >= p.cols) return;
   float mean[W], scale[W], shift[W];
 #pragma unroll
   for (int j = 0; j < W; ++j) {
-    mean[j] = fin[0][lcol * W + j];
-    const float g = (p.gamma != nullptr) ? E::load1(p.gamma, col0 + j) : 1.f;
-    shift[j] = (p.beta != nullptr) ? E::load1(p.beta, col0 + j) : 0.f;
-    scale[j] = fin[1][lcol * W + j] * g;
+    const float2 ms = (col0 + j < p.cols) ? p.partial[col0 + j] : make_float2(0.f, 0.f);
+    mean[j] = ms.x;
+    const float g = (p.gamma != nullptr && col0 + j < p.cols) ? E::load1(p.gamma, col0 + j) : 1.f;
+    shift[j] = (p.beta != nullptr && col0 + j < p.cols) ? E::load1(p.beta, col0 + j) : 0.f;
+    scale[j] = ms.y * g;
   }
+  const uint64_t drop = p.l2_keep ? l2_policy_drop() : l2_policy_normal();
   const long long xstep = p.xs * ns, ystep = p.ys * ns;
   const T* px = reinterpret_cast<const T*>(p.x) + (r0 + slot) * p.xs + col0;
   T* py = reinterpret_cast<T*>(p.y) + (r0 + slot) * p.ys + col0;
@@ -150,7 +159,7 @@ __global__ void __launch_bounds__(kAxisThreads, 4) col_apply_kernel(const ColPar
     Raw raw[UB];
 #pragma unroll
     for (int u = 0; u < UB; ++u, px += xstep)
-      if (whole || f + u * ns < r1) raw[u] = A::load(px);
+      if (whole || f + u * ns < r1) raw[u] = A::load_hint(px, drop);
 #pragma unroll
     for (int u = 0; u < UB; ++u, py += ystep) {
       if (whole || f + u * ns < r1) {

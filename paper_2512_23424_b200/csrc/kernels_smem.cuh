@@ -98,8 +98,10 @@ struct SmemGeom {
   unsigned buf_bytes;     // bytes reserved per ring buffer (multiple of 128)
 };
 
+constexpr int kXSlots = 4;          // exchange slots of smem_kernel (see its comment)
+
 template <int OP, typename T, int THREADS>
-__global__ void __launch_bounds__(THREADS) smem_kernel(const RowParams p, const SmemGeom g) {
+__global__ void __launch_bounds__(THREADS) smem_kernel(const RowParams p, const SmemGeom g, const int xmode) {
   pdl_prologue();
   using E = Elem<T>;
   constexpr int EPV = E::EPV;
@@ -108,7 +110,10 @@ __global__ void __launch_bounds__(THREADS) smem_kernel(const RowParams p, const 
 
   extern __shared__ __align__(128) unsigned char smem_raw[];
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem_raw);                       // [kMaxBuf]
-  Stat* red = reinterpret_cast<Stat*>(smem_raw + kMaxBuf * sizeof(uint64_t));    // [2][NW]
+  uint64_t* xbar = bars + kMaxBuf;                                               // [kXSlots]
+  float4 (*inbox)[kMaxCluster] =
+      reinterpret_cast<float4 (*)[kMaxCluster]>(smem_raw + kMaxBuf * 8 + kXSlots * 8);       // [kXSlots][kMaxCluster]
+  Stat* red = reinterpret_cast<Stat*>(smem_raw + kMaxBuf * 8 + kXSlots * 8 + kXSlots * kMaxCluster * 16);   // [2][NW]
   Stat* peers = red + 2 * NW;                                                     // [2][kMaxCluster]
   constexpr unsigned kHeader = smem_header_bytes(THREADS);
   unsigned char* bufs = smem_raw + kHeader;
@@ -121,8 +126,21 @@ __global__ void __launch_bounds__(THREADS) smem_kernel(const RowParams p, const 
   const int v0 = static_cast<int>(rank) * g.slice_vecs;                          // my first vector
   const int my_vecs = max(0, min(g.slice_vecs, nvec - v0));
 
+  // Exchange of the slices' partial statistics.
+  // xmode 1 (default): as in split_kernel, one 16-byte st.async per peer that counts on the receiver's
+  // mbarrier, so that no cluster barrier (whose release waits for the CTA's global stores of the row
+  // before) stands between two rows.  With a ring of two and more buffers the row loop is also software-
+  // pipelined: the first sweep of row r + 1 and the sending of its partials come BEFORE the wait for the
+  // partials of row r, whose latency then hides behind that sweep (one CTA per SM has nothing else to hide
+  // it behind).  A CTA can therefore be up to two rows ahead of a peer's reads, hence four exchange slots
+  // (row r uses slot r mod 4): a peer sends row r + 4 only after it has received every CTA's partial of
+  // row r + 2, and a CTA sends that after it has read the slot of row r.
+  // xmode 0: plain remote stores and a cluster barrier per row, no pipelining (the first version).
+  const bool async_x = xmode != 0 && cs > 1;
+  const bool pipelined = (xmode != 0 || cs == 1) && g.nbuf >= 2;
   if (threadIdx.x == 0) {
     for (int b = 0; b < g.nbuf; ++b) mbar_init(smem_addr(&bars[b]), 1);
+    for (int k = 0; k < kXSlots; ++k) mbar_init(smem_addr(&xbar[k]), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
@@ -162,12 +180,16 @@ __global__ void __launch_bounds__(THREADS) smem_kernel(const RowParams p, const 
     for (int b = 0; b < g.nbuf && r < p.rows; ++b, r += row_step) { issue(r, b); ++in_flight; }
   }
 
-  // A wait that runs out makes the whole CTA "dead" (the vote below): it reads and stores nothing any
+  // A wait that runs out makes the whole CTA "dead" (the vote in sweep1): it reads and stores nothing any
   // more and issues no copy, but goes on through its rows for the sake of the cluster exchange, so that
-  // no peer waits at a cluster barrier for a CTA that has left.
-  bool dead = false;
-  long long it = 0, dead_it = 0;     // dead_it: the iteration whose wait ran out
-  for (long long row = first_row; row < p.rows; row += row_step, ++it) {
+  // no peer waits for a CTA that has left.
+  bool dead = false, xfail = false;  // xfail: this thread's wait for the cluster's partials ran out
+  long long dead_it = 0;             // the iteration whose wait ran out
+  uint32_t xphases = 0;              // bit k: parity of the phase of xbar[k] that the next wait is for
+
+  // ---- first sweep of iteration `it` (row `row`): wait for the slice, thread statistics, CTA reduction,
+  // and the CTA's partial on its way to the peers
+  auto sweep1 = [&](long long row, long long it) -> Stat {
     const int b = static_cast<int>(it % g.nbuf);
     const uint32_t phase = static_cast<uint32_t>((it / g.nbuf) & 1);
     const int par = static_cast<int>(it & 1);
@@ -178,16 +200,14 @@ __global__ void __launch_bounds__(THREADS) smem_kernel(const RowParams p, const 
                       ? reinterpret_cast<const T*>(p.add) + add_row(p, row) * p.add_stride
                       : nullptr;
     if (!dead) {
-      if (__syncthreads_or(mbar_wait_timed(smem_addr(&bars[b]), phase, p.status, p.wait_us) ? 0 : 1)) {
+      if (__syncthreads_or((xfail || !mbar_wait_timed(smem_addr(&bars[b]), phase, p.status, p.wait_us)) ? 1 : 0)) {
         dead = true;
         dead_it = it;
       } else if (threadIdx.x == 0) {
         --in_flight;
       }
     }
-
-    // ---- pass 1: thread-local statistics over my slice.  `plain` = no element of the
-    // slice is masked: four vectors per step, loads first, one rescale per block.
+    // `plain` = no element of the slice is masked: four vectors per step, loads first, one rescale per block
     Stat st = stat_identity<OP>();
     const bool plain = !SM || (ar == nullptr && (v0 + lv) * EPV <= live);
     int v = dead ? lv : static_cast<int>(threadIdx.x);          // a dead CTA folds nothing
@@ -218,9 +238,12 @@ __global__ void __launch_bounds__(THREADS) smem_kernel(const RowParams p, const 
       fold_vector<OP, EPV>(st, z, p.l2e);
     }
     st = cta_reduce<OP, NW>(st, red + par * NW, p.l2e);
-
-    // ---- combine across the cluster through distributed shared memory
-    if (cs > 1) {
+    if (async_x) {
+      const int slot = static_cast<int>(it % kXSlots);
+      if (threadIdx.x == 0) mbar_expect_tx(smem_addr(&xbar[slot]), cs * 16u);
+      if (threadIdx.x < cs)
+        st_async_f32x4(smem_addr(&inbox[slot][rank]), smem_addr(&xbar[slot]), threadIdx.x, st.a, st.b, st.c, 0.f);
+    } else if (cs > 1) {
       if (threadIdx.x < cs) {
         const uint32_t slot = smem_addr(&peers[par * kMaxCluster + rank]);
         st_remote_f32(slot, threadIdx.x, st.a);
@@ -228,6 +251,31 @@ __global__ void __launch_bounds__(THREADS) smem_kernel(const RowParams p, const 
         st_remote_f32(slot + 8, threadIdx.x, st.c);
       }
       cluster_arrive();
+    }
+    return st;
+  };
+
+  // ---- the row's statistics from the cluster, second sweep (normalise from shared memory, 128-bit
+  // stores), and the buffer handed back to the copy engine
+  auto sweep2 = [&](long long row, long long it, Stat st) {
+    const int b = static_cast<int>(it % g.nbuf);
+    const int par = static_cast<int>(it & 1);
+    int live;
+    const int lv = live_in_slice(row, live);
+    const uint32_t buf = smem_addr(bufs + static_cast<size_t>(b) * g.buf_bytes);
+    const T* ar = (SM && p.add != nullptr)
+                      ? reinterpret_cast<const T*>(p.add) + add_row(p, row) * p.add_stride
+                      : nullptr;
+    const bool plain = !SM || (ar == nullptr && (v0 + lv) * EPV <= live);
+    if (async_x) {
+      const int slot = static_cast<int>(it % kXSlots);
+      // (a dead CTA does not wait; a wait that runs out here makes the CTA dead at the vote of its next sweep1)
+      if (!dead && !mbar_wait_timed<true>(smem_addr(&xbar[slot]), (xphases >> slot) & 1u, p.status, p.wait_us))
+        xfail = true;
+      xphases ^= 1u << slot;
+      const float4 f = inbox[slot][threadIdx.x & (cs - 1)];          // cs is a power of two
+      st = butterfly_merge<OP>(Stat{f.x, f.y, f.z}, static_cast<int>(cs), p.l2e);
+    } else if (cs > 1) {
       cluster_wait();
       Stat r = peers[par * kMaxCluster];
       for (uint32_t k = 1; k < cs; ++k) r = stat_merge<OP>(r, peers[par * kMaxCluster + k], p.l2e);
@@ -236,9 +284,8 @@ __global__ void __launch_bounds__(THREADS) smem_kernel(const RowParams p, const 
     const RowScalars rs = finalize<OP>(st, p.cols, p.eps);
     const float fill = SM ? masked_fill<OP>(rs) : 0.f;
 
-    // ---- pass 2: normalise from shared memory, 128-bit stores
     T* yr = reinterpret_cast<T*>(p.y) + row * p.ys + static_cast<long long>(v0) * EPV;
-    v = dead ? my_vecs : static_cast<int>(threadIdx.x);         // ... and stores nothing
+    int v = (dead || xfail) ? my_vecs : static_cast<int>(threadIdx.x);      // a dead CTA stores nothing
     if (plain && lv == my_vecs) {
       for (; v + 3 * THREADS < my_vecs; v += 4 * THREADS) {
         float z[4][EPV];
@@ -298,11 +345,30 @@ __global__ void __launch_bounds__(THREADS) smem_kernel(const RowParams p, const 
       st_stream(yr + static_cast<long long>(v) * EPV, E::pack(o));
     }
 
-    // ---- the buffer is free once every thread has read it: refill for row it + nbuf
+    // the buffer is free once every thread has read it: refill for row it + nbuf
     __syncthreads();
     if (threadIdx.x == 0 && !dead && !p.no_copies) {
       const long long next = row + row_step * g.nbuf;
       if (next < p.rows) { issue(next, b); ++in_flight; }
+    }
+  };
+
+  long long it = 0;
+  if (first_row < p.rows) {
+    if (pipelined) {
+      Stat st = sweep1(first_row, 0);
+      for (long long row = first_row; row < p.rows; row += row_step, ++it) {
+        const long long next = row + row_step;
+        Stat stn = st;
+        if (next < p.rows) stn = sweep1(next, it + 1);      // (its partials are on their way while ...)
+        sweep2(row, it, st);                                 // (... this row waits for its own)
+        st = stn;
+      }
+    } else {
+      for (long long row = first_row; row < p.rows; row += row_step, ++it) {
+        const Stat st = sweep1(row, it);
+        sweep2(row, it, st);
+      }
     }
   }
   // no copy may still be on its way into this CTA's shared memory when it leaves
@@ -310,9 +376,10 @@ __global__ void __launch_bounds__(THREADS) smem_kernel(const RowParams p, const 
     for (long long k = dead_it; in_flight > 0; --in_flight, ++k)
       (void)mbar_wait_timed(smem_addr(&bars[k % g.nbuf]), static_cast<uint32_t>((k / g.nbuf) & 1), nullptr, p.wait_us);
   }
-  // Peers write into this CTA's shared memory only before the cluster barrier of a row
-  // this CTA also takes part in, so leaving after the last row is safe; every bulk copy
-  // issued was waited for above (each issued row is consumed by the loop, or drained).
+  if (cs > 1) {            // nobody leaves while a peer may still send to it
+    cluster_arrive();
+    cluster_wait();
+  }
 }
 
 }  // namespace akg

@@ -455,13 +455,8 @@ split_kernel(const RowParams p, const int slice_vecs, const int xmode, const int
         cta_failed = 1;
       }
       phases ^= 1u << par;
-      const float4 f = inbox[par][0];
-      Stat r{f.x, f.y, f.z};
-      for (uint32_t k = 1; k < cs; ++k) {
-        const float4 g = inbox[par][k];
-        r = stat_merge<OP>(r, Stat{g.x, g.y, g.z}, p.l2e);
-      }
-      st = r;
+      const float4 f = inbox[par][threadIdx.x & (cs - 1)];           // cs is a power of two
+      st = butterfly_merge<OP>(Stat{f.x, f.y, f.z}, static_cast<int>(cs), p.l2e);
     } else if (cs > 1) {
       cluster_wait();
       Stat r = peers[par][0];

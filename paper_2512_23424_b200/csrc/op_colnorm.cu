@@ -22,8 +22,21 @@ cudaError_t launch_col(K kernel, const ColParams& p, dim3 grid, int pdl, cudaStr
 
 template <typename T, int MODE>
 cudaError_t launch_colnorm_t(const ColParams& p, dim3 grid, int pdl, cudaStream_t s) {
-  const cudaError_t e = launch_col(col_stat_kernel<T, MODE>, p, grid, pdl, s);
+  cudaError_t e = launch_col(col_stat_kernel<T, MODE>, p, grid, pdl, s);
   if (e != cudaSuccess) return e;
+  {
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.gridDim = dim3(static_cast<unsigned>((p.cols + 7) / 8));
+    cfg.blockDim = dim3(256);
+    cfg.stream = s;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    e = cudaLaunchKernelEx(&cfg, col_finish_kernel, p, static_cast<int>(grid.y));
+    if (e != cudaSuccess) return e;
+  }
   return launch_col(col_apply_kernel<T, MODE>, p, grid, pdl, s);
 }
 
