@@ -317,6 +317,8 @@ akg_status akg_set_variant(akg_variant variant);
  * "cluster_mode" (1 = row resident in the cluster's shared memory, 2 = two streaming
  * passes with the second served by L2), "reg_general" (1 = never the predicate-free
  * normalisation kernel), "interleave" (1 = visit causal rows short/long alternately),
+ * "host_chunks", "host_min_kib" (host-buffer entry point: chunks per call, smallest chunk),
+ * "host_full_upload" (1 = upload the masked columns of causal rows too),
  * "split_exchange" (two-pass cluster kernel: 1 = partial statistics exchanged under a
  * cluster barrier per row instead of st.async + mbarrier), "split_l2" (its L2 priority
  * scheme: 1 = no "keep" marks, 2 = marks without demotion).  Two keys exist for the test
@@ -332,6 +334,13 @@ akg_status akg_set_tuning(const char* key, int value);
 /* Name of the kernel family and geometry the last successful call on this thread
  * launched, e.g. "reg<f32,t256,v4>" (static/thread-local storage). */
 const char* akg_last_kernel_name(void);
+
+/* Bytes that the last akg_rowop_host call on this thread copied from host to device and from
+ * device to host (either pointer may be NULL).  The upload is smaller than the matrix under a
+ * causal mask: the masked columns of a row are never read by the kernels, so they are not sent
+ * either (chunks lie inside a causal period and carry the columns up to their last row's live
+ * length).  Always returns AKG_OK. */
+akg_status akg_last_host_copy_bytes(size_t* h2d_bytes, size_t* d2h_bytes);
 
 /* Reads the device-side status word of the current device (synchronises with
  * the device).  0 = clean; non-zero = a bounded wait (on a bulk copy, or on the

@@ -90,6 +90,16 @@ def last_kernel() -> str:
     return lib().akg_last_kernel_name().decode()
 
 
+def last_host_copy_bytes():
+    """(host -> device, device -> host) bytes copied by the last rowop_host call of this thread."""
+    up, down = ctypes.c_size_t(0), ctypes.c_size_t(0)
+    fn = lib().akg_last_host_copy_bytes
+    fn.restype = ctypes.c_int
+    fn.argtypes = [ctypes.POINTER(ctypes.c_size_t), ctypes.POINTER(ctypes.c_size_t)]
+    fn(ctypes.byref(up), ctypes.byref(down))
+    return up.value, down.value
+
+
 def set_variant(variant) -> None:
     code = VARIANTS[variant] if isinstance(variant, str) else int(variant)
     _check(lib().akg_set_variant(code), "akg_set_variant")

@@ -73,6 +73,42 @@ def test_host_entry_causal_chunks_keep_global_rows(dtype):
     assert (bits[dead] == 0).all()
 
 
+@pytest.mark.parametrize("dtype", [wl.F32, wl.BF16])
+def test_host_entry_uploads_only_live_columns_and_ramps_its_chunks(dtype):
+    """Under a causal mask the masked columns of a chunk are not uploaded (the kernels never read them):
+    NaN in the masked part of the host matrix does not show, the byte counter reports the smaller upload,
+    and the result is the oracle's.  Without a mask the first and last chunks are smaller than the rest;
+    the counter then reports the whole matrix."""
+    es = 4 if dtype == wl.F32 else 2
+    rows, cols, period = 6144, 2048, 2048
+    w = wl.make_random("softmax", dtype, rows, cols, seed=5)
+    w.causal_period = period
+    ref = run_oracle(w)
+    dead = np.arange(cols)[None, :] > (np.arange(rows)[:, None] % period)
+    x = w.x.copy()
+    x[dead] = np.float32(np.nan) if dtype == wl.F32 else np.uint16(0x7FC0)
+    wp = wl.Workload(w.name, w.op, dtype, rows, cols, x, causal_period=period)
+    got = run_host(wp)
+    compare(got, ref, dtype, "host causal, poisoned masked columns")
+    up, down = binding.last_host_copy_bytes()
+    assert down == rows * cols * es
+    # chunks of a quarter period: 1/4, 2/4, 3/4, 4/4 of the columns -> 62.5 % of the matrix (chunks of at
+    # least 4 MiB: 512 rows of 8 KiB for fp32, 1024 rows of 4 KiB otherwise, i.e. a quarter / a half period)
+    assert up < 0.80 * rows * cols * es and up >= 0.5 * rows * cols * es, (up, rows * cols * es)
+    try:
+        akg.set_tuning("host_full_upload", 1)
+        got2 = run_host(w)
+        assert binding.last_host_copy_bytes()[0] == rows * cols * es
+        assert np.array_equal(got2, got)
+    finally:
+        akg.set_tuning("host_full_upload", 0)
+    # no mask: ramped chunks (1/8, 1/8, 1/4, 1/2, 1, ... of a chunk), every row exactly once
+    wn = wl.make_random("rmsnorm", dtype, 40000, 1024, seed=6, eps=1e-6)
+    gotn = run_host(wn)
+    compare(gotn, run_oracle(wn), dtype, "host ramped chunks")
+    assert binding.last_host_copy_bytes() == (40000 * 1024 * es + 1024 * es, 40000 * 1024 * es)
+
+
 def test_host_entry_argument_errors():
     L = akg.lib()
     x = torch.zeros((4, 8)).pin_memory()
