@@ -1227,6 +1227,22 @@ extern "C" akg_status akg_cumulative(int want_prod, const void* x, void* y, int6
   const bool warp_rows = vec && (t_group == 32 || (t_group == 0 && cols * es <= scan_warp_row_bytes(es)));
   const int64_t ctas = warp_rows ? (rows + 7) / 8 : rows;
   const unsigned grid = static_cast<unsigned>(std::min<int64_t>(ctas, cap > 0 ? cap : INT_MAX));
+  // Rows of at most 64 vectors (a kilobyte): 4, 8 or 16 lanes per row, several rows per warp (scan_short_kernel)
+  if (vec && nvec <= 64 && t_group == 0 && g_tune_reg_general.load() == 0) {
+    int lanes = 4;
+    while (4 * lanes < nvec) lanes *= 2;
+    const int64_t rows_per_cta = 8 * (32 / lanes);
+    int64_t sctas = (rows + rows_per_cta - 1) / rows_per_cta;
+    const int64_t scap = cap > 0 ? cap : static_cast<int64_t>(sm_count()) * 32;     // grid-stride beyond four waves
+    if (sctas > scap) sctas = scap;
+    const cudaError_t e1 = launch_cumulative_short(want_prod == 1, static_cast<int>(dtype), lanes, x, y, rows, cols,
+                                                   x_row_stride, y_row_stride, static_cast<unsigned>(sctas),
+                                                   g_tune_pdl.load() == 2 ? 0 : 1, static_cast<cudaStream_t>(stream));
+    if (e1 != cudaSuccess) return cuda_fail(name, e1);
+    std::snprintf(t_kernel, sizeof t_kernel, "scan_short<%s,%s,l%d,grid%u>", want_prod ? "prod" : "sum", dtype_name(dtype),
+                  lanes, static_cast<unsigned>(sctas));
+    return AKG_OK;
+  }
   // Few, long rows (at least 8192 vectors each; fewer rows than SMs in fp32, than two per SM in the 16-bit
   // types): a cluster per row, every CTA a slice of about 4096 vectors, the carry of a slice from the cluster's
   // totals (scan_split_kernel).  Measured against a CTA per row, fraction of the copy rate: [64, 2^20] fp32 0.54

@@ -156,6 +156,90 @@ __global__ void __launch_bounds__(32 * kScanMaxWarps, 4) scan_kernel(const ScanP
 
 
 // ------------------------------------------------------------------------------------------------
+// scan_short_kernel: rows of at most 4 * L vectors (L = 4, 8 or 16 lanes per row, so up to 64 vectors: a
+// kilobyte).  A warp per row leaves most lanes without a vector on such rows (bf16 rows of 256 columns
+// are 32 vectors: one per lane, three quarters of the chunk empty, and the row's chain of load, scan
+// and store is paid for 512 bytes: 0.35 - 0.45 of the copy rate).  Here L lanes own a row and hold up to
+// four of its vectors each (lane l of the group: vectors l, l + L, ...), so a warp works on 32 / L rows
+// at once with four loads in flight per lane, shuffle scans of log2 L steps inside the group, and the
+// next rows of the warp loaded while the current ones are scanned.  No shared memory, no barrier.
+// ------------------------------------------------------------------------------------------------
+template <bool PROD, typename T, int L>
+__global__ void __launch_bounds__(256, 4) scan_short_kernel(const ScanParams p) {
+  pdl_prologue();
+  using E = Elem<T>;
+  constexpr int EPV = E::EPV;
+  constexpr int U = kScanU;
+  constexpr int RPW = 32 / L;                                   // rows per warp
+  const int lane = threadIdx.x & 31;
+  const int gl = lane & (L - 1);                                // lane inside the row's group
+  const int nvec = static_cast<int>(p.cols / EPV);
+  const float id = scan_identity<PROD>();
+  const long long warps = static_cast<long long>(gridDim.x) * (blockDim.x >> 5);
+  long long row = (static_cast<long long>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5)) * RPW + lane / L;
+  const long long row_step = warps * RPW;
+
+  uint4 ahead[U];
+  auto load_row = [&](long long r) {
+    if (r < p.rows) {
+      const T* xr = reinterpret_cast<const T*>(p.x) + r * p.xs;
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const int i = u * L + gl;
+        if (i < nvec) ahead[u] = ld_stream(xr + static_cast<long long>(i) * EPV);
+      }
+    }
+  };
+  load_row(row);
+  // (the loop bound is the warp's first row, so that every lane of a warp takes part in the shuffles)
+  for (long long base = row - lane / L; base < p.rows; base += row_step, row += row_step) {
+    float v[U][EPV];
+    const bool active = row < p.rows;
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int i = u * L + gl;
+      float f[EPV];
+      if (active && i < nvec) E::unpack(ahead[u], f);
+#pragma unroll
+      for (int j = 0; j < EPV; ++j) v[u][j] = (active && i < nvec) ? f[j] : id;
+    }
+    load_row(row + row_step);
+    float incl[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+#pragma unroll
+      for (int j = 1; j < EPV; ++j) v[u][j] = scan_op<PROD>(v[u][j - 1], v[u][j]);
+      incl[u] = v[u][EPV - 1];
+    }
+#pragma unroll
+    for (int d = 1; d < L; d <<= 1) {
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const float o = __shfl_up_sync(0xffffffffu, incl[u], d, L);
+        if (gl >= d) incl[u] = scan_op<PROD>(o, incl[u]);
+      }
+    }
+    float before = id;
+    T* yr = reinterpret_cast<T*>(p.y) + row * p.ys;
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const float tot = __shfl_sync(0xffffffffu, incl[u], L - 1, L);
+      const float excl = __shfl_up_sync(0xffffffffu, incl[u], 1, L);
+      float mine = before;
+      if (gl > 0) mine = scan_op<PROD>(mine, excl);
+      before = scan_op<PROD>(before, tot);
+      const int i = u * L + gl;
+      if (active && i < nvec) {
+        float o[EPV];
+#pragma unroll
+        for (int j = 0; j < EPV; ++j) o[j] = scan_op<PROD>(mine, v[u][j]);
+        st_stream(yr + static_cast<long long>(i) * EPV, E::pack(o));
+      }
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
 // scan_split_kernel: few, long rows (a CTA per row would leave most SMs idle and walk a megabyte on
 // its own).  A cluster of CS CTAs owns a row at a time and CTA k its slice k of slice_vecs vectors:
 //   phase 1  the slice's total: streaming loads marked "keep in L2", eight per thread in flight,

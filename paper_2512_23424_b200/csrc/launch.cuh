@@ -68,6 +68,10 @@ cudaError_t launch_cumulative(bool want_prod, int dtype, bool vec, const void* x
                               long long cols, long long xs, long long ys, unsigned grid, int threads, bool warp_rows,
                               int pdl, cudaStream_t stream);
 
+// Short vectorised rows (at most 4 * lanes vectors, lanes in {4, 8, 16}): 32 / lanes rows per warp, CTAs of 256.
+cudaError_t launch_cumulative_short(bool want_prod, int dtype, int lanes, const void* x, void* y, long long rows,
+                                    long long cols, long long xs, long long ys, unsigned grid, int pdl, cudaStream_t stream);
+
 // Few, long rows: a cluster of `cluster` CTAs (256 threads) per row, slices of slice_vecs vectors, the carry
 // of a slice from its cluster peers (scan_split_kernel); vectorised rows only.  clusters = 0: one resident wave.
 cudaError_t launch_cumulative_split(bool want_prod, int dtype, const void* x, void* y, long long rows, long long cols,

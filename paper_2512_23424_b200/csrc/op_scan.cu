@@ -69,6 +69,14 @@ cudaError_t launch_scan_t(bool vec, bool warp_rows, const ScanParams& p, unsigne
              : launch_1d(scan_kernel<PROD, T, false>, p, grid, threads, pdl, s);
 }
 
+template <bool PROD, typename T>
+cudaError_t launch_scan_short_t(int lanes, const ScanParams& p, unsigned grid, int pdl, cudaStream_t s) {
+  if (lanes == 4) return launch_1d(scan_short_kernel<PROD, T, 4>, p, grid, 256, pdl, s);
+  if (lanes == 8) return launch_1d(scan_short_kernel<PROD, T, 8>, p, grid, 256, pdl, s);
+  if (lanes == 16) return launch_1d(scan_short_kernel<PROD, T, 16>, p, grid, 256, pdl, s);
+  return cudaErrorInvalidValue;
+}
+
 // scan_split_kernel: a cluster of `cluster` CTAs per row; clusters = 0 asks for one resident wave
 template <bool PROD, typename T>
 cudaError_t launch_scan_split_t(const ScanParams& p, int cluster, int slice_vecs, long long clusters, int* status,
@@ -122,6 +130,20 @@ cudaError_t launch_scan_split_t(const ScanParams& p, int cluster, int slice_vecs
 }  // namespace
 
 int scan_unroll() { return kScanU; }
+
+cudaError_t launch_cumulative_short(bool want_prod, int dtype, int lanes, const void* x, void* y, long long rows,
+                                    long long cols, long long xs, long long ys, unsigned grid, int pdl, cudaStream_t stream) {
+  ScanParams p;
+  p.x = x; p.y = y; p.rows = rows; p.cols = cols; p.xs = xs; p.ys = ys;
+  if (dtype == DT_F32)
+    return want_prod ? launch_scan_short_t<true, float>(lanes, p, grid, pdl, stream)
+                     : launch_scan_short_t<false, float>(lanes, p, grid, pdl, stream);
+  if (dtype == DT_F16)
+    return want_prod ? launch_scan_short_t<true, __half>(lanes, p, grid, pdl, stream)
+                     : launch_scan_short_t<false, __half>(lanes, p, grid, pdl, stream);
+  return want_prod ? launch_scan_short_t<true, __nv_bfloat16>(lanes, p, grid, pdl, stream)
+                   : launch_scan_short_t<false, __nv_bfloat16>(lanes, p, grid, pdl, stream);
+}
 
 cudaError_t launch_cumulative_split(bool want_prod, int dtype, const void* x, void* y, long long rows, long long cols,
                                     long long xs, long long ys, int cluster, int slice_vecs, long long clusters,

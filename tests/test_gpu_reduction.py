@@ -134,6 +134,43 @@ def test_cumulative_shapes(dtype):
 
 
 @pytest.mark.parametrize("dtype", DTYPES)
+def test_cumulative_short_rows_several_per_warp(dtype):
+    """Rows of at most 64 vectors: 4, 8 or 16 lanes per row (every group size, ragged row counts, rows that
+    do not fill their lanes, more rows than the grid holds warps)."""
+    rng = np.random.default_rng(26)
+    epv = 4 if dtype == wl.F32 else 8
+    seen = set()
+    try:
+        for rows, nvec, cap in [(1, 1, 0), (7, 3, 0), (1000, 8, 0), (37, 16, 0), (999, 17, 0), (5000, 32, 0), (130, 33, 0),
+                                (3001, 64, 0), (20000, 32, 5), (8, 64, 0), (65, 12, 1)]:
+            akg.set_tuning("grid_cap", cap)
+            cols = nvec * epv
+            x = rng.normal(0.05, 1, (rows, cols)).astype(np.float32)
+            check_cum("cumsum", store(x, dtype), dtype, f"{rows}x{cols}")
+            assert akg.last_kernel().startswith("scan_short<"), akg.last_kernel()
+            seen.add(akg.last_kernel().split(",")[2])
+            f = (1.0 + 0.01 * rng.normal(0, 1, (rows, cols))).astype(np.float32)
+            check_cum("cumprod", store(f, dtype), dtype, f"{rows}x{cols}")
+        assert seen == {"l4", "l8", "l16"}, seen
+        # exact arithmetic and padded rows in place
+        akg.set_tuning("grid_cap", 0)
+        x = rng.integers(-3, 4, (77, 24 * epv)).astype(np.float32)
+        tdt = torch.float32 if dtype == wl.F32 else torch.bfloat16
+        big = torch.full((77, 24 * epv + 2 * epv), 9.0, dtype=tdt, device="cuda")
+        big[:, :24 * epv].copy_(to_torch(store(x, dtype), dtype))
+        binding.cumsum(big[:, :24 * epv], out=big[:, :24 * epv])
+        torch.cuda.synchronize()
+        assert akg.last_kernel().startswith("scan_short<")
+        ref = oracle.cumulative("cumsum", x)
+        got = widen(to_numpy(big[:, :24 * epv].contiguous()))
+        exact = np.abs(ref) < (2 ** 24 if dtype == wl.F32 else 256)
+        assert np.array_equal(got[exact], ref[exact])
+        assert torch.all(big[:, 24 * epv:] == 9.0)
+    finally:
+        akg.set_tuning("grid_cap", 0)
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
 def test_cumulative_long_rows_split_over_a_cluster(dtype):
     """Few, long rows: a cluster per row, a slice per CTA, the carry of a slice from the peers' totals."""
     rng = np.random.default_rng(25)
