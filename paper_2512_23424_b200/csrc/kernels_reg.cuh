@@ -200,11 +200,14 @@ __device__ __forceinline__ void flex_row_stats(const float (&v)[N], float (*red)
     }
     if ((threadIdx.x & 31) == 0) { red[0][threadIdx.x >> 5] = mu; red[1][threadIdx.x >> 5] = m2; }
     __syncthreads();
-    float msum = 0.f, qsum = 0.f;
-    for (int w = 0; w < NW; ++w) { msum += red[0][w]; qsum += red[1][w]; }
-    mean = msum * inv_warps;
-    float dev = 0.f;
-    for (int w = 0; w < NW; ++w) { const float d = red[0][w] - mean; dev = fmaf(d, d, dev); }
+    // lane l takes warp l's pair (nothing beyond the CTA's warps): three shuffle sums instead of three
+    // shared loads and a dependent chain per warp of the CTA
+    const bool mine = static_cast<int>(threadIdx.x & 31) < NW;
+    const float mw = mine ? red[0][threadIdx.x & 31] : 0.f;
+    const float qsum = warp_sum(mine ? red[1][threadIdx.x & 31] : 0.f);
+    mean = warp_sum(mw) * inv_warps;
+    const float d = mine ? mw - mean : 0.f;
+    const float dev = warp_sum(d * d);
     rstd = rsqrt_refined(fmaf(fmaf(dev, 32.0f * N, qsum), inv_cols, eps));
   }
 }
