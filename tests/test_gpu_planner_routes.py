@@ -199,7 +199,7 @@ def test_cumulative_routes(dtype):
     es = 4 if dtype == wl.F32 else 2
     warp_cols = (2048 if dtype == wl.F32 else 32768) // es
     for rows, cols, expect in ((270, warp_cols, "g32"), (270, warp_cols + 64, "vec,t"), (1000, 256, "scan_short"),
-                               (1000, 512, "g32"), (9, 40000, ",t256")):
+                               (1000, 128 * 16 // es, "g32"), (9, 40000, ",t256")):
         x = store(rng.normal(0.05, 1, (rows, cols)).astype(np.float32), dtype)
         ref = oracle.cumulative("cumsum", x, nthreads=8)
         got = to_numpy(binding.cumsum(to_torch(x, dtype)))
