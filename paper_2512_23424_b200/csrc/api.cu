@@ -30,7 +30,8 @@ std::atomic<int> g_tune_cluster_mode{0};  // 0 = planner's choice, 1 = row resid
 std::atomic<int> g_tune_tma_mode{0};      // 0 = planner's choice, 1 = ring-fed register kernel, 2 = shared-memory passes
 std::atomic<int> g_tune_interleave{0};    // 1 = visit causal rows short/long alternately (default: storage order)
 std::atomic<int> g_tune_pdl{0};           // 2 = launch without programmatic stream serialisation
-std::atomic<int> g_tune_reg_flex{0};      // 2 = never the runtime-thread-count normalisation kernel
+std::atomic<int> g_tune_reg_flex{0};      // 2 = never the runtime-thread-count normalisation kernel, 5 = never its packed 16-bit form
+std::atomic<int> g_tune_packed_vpt{0};    // packed 16-bit form: vectors per thread (0 = planner's choice)
 std::atomic<int> g_tune_axis_r{0};        // non-last axis: rows per thread (2 / 4 / 8), -1 = two-pass kernel only
 std::atomic<int> g_tune_axis_nc{0};       //   column blocks per CTA
 std::atomic<int> g_tune_axis_lc{0};       //   two-pass kernel: 1 + log2 of the lanes along the columns
@@ -249,6 +250,33 @@ bool plan_reg(const Call& c, LaunchPlan* plan) {
       const unsigned flex_cap = g_tune_grid_cap.load() > 0 ? static_cast<unsigned>(g_tune_grid_cap.load())
                                 : (c.dtype != AKG_F32 ? static_cast<unsigned>(sm_count()) * 64u : 0u);
       if (flex_cap > 0 && plan->grid > flex_cap) plan->grid = flex_cap;
+    }
+  }
+  // 16-bit normalisation rows with a CTA per row: the packed form of the runtime-thread-count kernel
+  // (reg_norm_packed: the row stays packed in registers, eight vectors per thread fit 64 registers).  Measured
+  // on bf16 rows of 2048 .. 16384 columns against everything above (fraction of the copy rate): LayerNorm
+  // 0.73 - 0.95 -> 0.93 - 0.99, RMSNorm 0.79 - 0.98 (ring-fed: 0.91) -> 0.96 - 1.01.  Vectors per thread:
+  // LayerNorm the most that leaves 64 threads (8192 columns: eight 0.95, four 0.88); RMSNorm four while that
+  // keeps the CTA at 384 threads or fewer (8192 columns: four 1.01, eight 0.98), else the most (16384: eight
+  // 0.97, four 0.89).
+  if (norm && c.dtype != AKG_F32 && group == threads && g_tune_reg_general.load() == 0 &&
+      !(t_threads > 0 && t_vpt > 0) && g_tune_reg_flex.load() != 2 && g_tune_reg_flex.load() != 5) {
+    const int want = g_tune_packed_vpt.load();
+    int pv = 0;
+    auto fits = [&](int v) {
+      if (nvec % v) return false;
+      const int64_t g = nvec / v;
+      return g % 32 == 0 && g >= 64 && g <= 1024;
+    };
+    if (want > 0) { if (want >= 2 && want <= 8 && fits(want)) pv = want; }
+    else if (c.op == OP_RMSNORM && fits(4) && nvec / 4 <= 384) pv = 4;
+    else { for (int v = 8; v >= 2 && pv == 0; --v) if (fits(v)) pv = v; }
+    if (pv > 0) {
+      plan->mode = 3; plan->stages = 0; plan->vpt = pv; plan->threads = static_cast<int>(nvec / pv); plan->group = plan->threads;
+      plan->grid = static_cast<unsigned>(c.rows > INT_MAX ? INT_MAX : c.rows);
+      const unsigned pcap = g_tune_grid_cap.load() > 0 ? static_cast<unsigned>(g_tune_grid_cap.load())
+                                                       : static_cast<unsigned>(sm_count()) * 64u;
+      if (plan->grid > pcap) plan->grid = pcap;
     }
   }
   return true;
@@ -474,23 +502,14 @@ akg_status run(const Call& c, const char* name) {
   std::memset(&plan, 0, sizeof plan);
   bool planned = false;
   // Automatic choice (each rule is a measured preference on B200, see the profiles):
-  //   bf16 RMSNorm rows of exactly threads * vpt vectors, many rows -> ring-fed register
-  //     kernel (the load latency is hidden by the copy ring, not by occupancy; bf16
-  //     LayerNorm, heavier per element, measured faster without the ring)
-  //   every other row that fits a CTA's registers -> register kernel
+  //   every row that fits a CTA's registers -> register kernels (plan_reg; 16-bit normalisation rows in
+  //     their packed form)
+  //   16-bit log-softmax rows of 16 - 48 KB and RMSNorm rows of 32 - 64 KB -> row resident in shared memory
   //   longer aligned rows -> two-pass split cluster kernel (second pass from L2)
   //   anything unaligned -> scalar stream kernel
-  if (forced == V_AUTO && vec && c.dtype != AKG_F32 && c.op == OP_RMSNORM &&
-      c.rows >= 2048 && c.cols >= 2048 && c.cols <= 8192 && g_tune_tma_mode.load() != 2) {   // beyond: fat threads (plan_reg)
-    planned = plan_ring(c, &plan);
-    if (planned) {
-      if (g_tune_smem_nbuf.load() == 0) {                  // one buffer per CTA measured best
-        plan.smem -= static_cast<size_t>(plan.stages - 1) * ((plan.smem - 128) / plan.stages);
-        plan.stages = 1;
-      }
-      p.status = status_word_ptr();
-    }
-  }
+  // (the ring-fed register kernels are no automatic choice any more: bf16 RMSNorm with many rows, their one
+  // case, runs at 0.91 - 0.96 of the copy rate through the ring and at 0.98 - 1.01 in the packed register
+  // kernel; forcing the TMA family still reaches them)
   // 16-bit rows of 16 - 64 KB without a mask, where a CTA's registers no longer hold the row comfortably:
   // the row resident in shared memory (bulk-copied in, two sweeps over shared memory), several CTAs per SM
   // so that one row's sweeps overlap the others' copies.  Measured against the register and two-pass
@@ -553,7 +572,7 @@ akg_status run(const Call& c, const char* name) {
   const char* dt = dtype_name(c.dtype);
   if (plan.variant == V_REG)
     std::snprintf(t_kernel, sizeof t_kernel, "reg<%s,g%d,t%d,v%d%s>", dt, plan.group, plan.threads, plan.vpt,
-                  plan.mode == 2 ? ",flex"
+                  plan.mode == 3 ? ",packed" : plan.mode == 2 ? ",flex"
                                  : ((plan.stages == 1 && (c.op == OP_LAYERNORM || c.op == OP_RMSNORM)) ? ",full" : ""));
   else if (plan.variant == V_TMA || plan.variant == V_CLUSTER)
     std::snprintf(t_kernel, sizeof t_kernel, "%s<%s,t%d,cs%d,nbuf%d,slice%d>",
@@ -825,6 +844,7 @@ akg_status akg_set_tuning(const char* key, int value) {
   else if (!std::strcmp(key, "interleave")) g_tune_interleave.store(value);
   else if (!std::strcmp(key, "pdl")) g_tune_pdl.store(value);
   else if (!std::strcmp(key, "reg_flex")) g_tune_reg_flex.store(value);
+  else if (!std::strcmp(key, "packed_vpt")) g_tune_packed_vpt.store(value);
   else if (!std::strcmp(key, "host_chunks")) g_tune_host_chunks.store(value);
   else if (!std::strcmp(key, "host_min_kib")) g_tune_host_min_kib.store(value);
   else if (!std::strcmp(key, "host_full_upload")) g_tune_host_full_upload.store(value);

@@ -212,6 +212,170 @@ __device__ __forceinline__ void flex_row_stats(const float (&v)[N], float (*red)
   }
 }
 
+// The cross-thread part of flex_row_stats on its own: every thread brings the statistics of its own n
+// values - LayerNorm: (mu, m2) = their mean and sum of squared deviations; RMSNorm: mu = their sum of squares.
+template <int OP>
+__device__ __forceinline__ void flex_merge(float mu, float m2, int n, float (*red)[32], int NW, float inv_warps,
+                                           float inv_cols, float eps, float& mean, float& rstd) {
+  mean = 0.f;
+  if (OP == OP_RMSNORM) {
+    float ss = warp_sum(mu);
+    if ((threadIdx.x & 31) == 0) red[0][threadIdx.x >> 5] = ss;
+    __syncthreads();
+    ss = 0.f;
+    for (int w = 0; w < NW; ++w) ss += red[0][w];
+    rstd = rsqrt_refined(fmaf(ss, inv_cols, eps));
+  } else {
+    float half_c = 0.5f * static_cast<float>(n);
+#pragma unroll
+    for (int m = 1; m <= 16; m <<= 1) {                 // equal-count merges inside the warp
+      const float mb = __shfl_xor_sync(0xffffffffu, mu, m);
+      const float qb = __shfl_xor_sync(0xffffffffu, m2, m);
+      const float d = mb - mu;
+      mu = fmaf(0.5f, d, mu);
+      m2 = fmaf(d * d, half_c, m2 + qb);
+      half_c *= 2.f;
+    }
+    if ((threadIdx.x & 31) == 0) { red[0][threadIdx.x >> 5] = mu; red[1][threadIdx.x >> 5] = m2; }
+    __syncthreads();
+    const bool mine = static_cast<int>(threadIdx.x & 31) < NW;
+    const float mw = mine ? red[0][threadIdx.x & 31] : 0.f;
+    const float qsum = warp_sum(mine ? red[1][threadIdx.x & 31] : 0.f);
+    mean = warp_sum(mw) * inv_warps;
+    const float d = mine ? mw - mean : 0.f;
+    const float dev = warp_sum(d * d);
+    rstd = rsqrt_refined(fmaf(fmaf(dev, 32.0f * static_cast<float>(n), qsum), inv_cols, eps));
+  }
+}
+
+// reg_norm_packed: reg_norm_flex for the 16-bit types with the row kept PACKED in registers (four
+// registers per vector instead of eight) and the stored values fed to the arithmetic as they are
+// (Elem::add_wide / sub_wide / fma_wide: widened inside the instruction, on the FMA pipe).  Eight vectors
+// per thread then fit 64 registers, so a row needs half the threads of the widened form: the per-row
+// work that every thread pays (shuffle merges, barrier, the warps' pairs) is spread over twice the
+// elements, eight loads per thread are in flight, and four CTAs of 256 share an SM.
+//   RMSNorm   sum x^2 with one fma_wide per element; y = (x * w) * rstd, the product of two 16-bit values
+//             being exact in fp32
+//   LayerNorm exact two sweeps over the thread's values (sum with add_wide, deviations with sub_wide),
+//             equal-count merges as in reg_norm_flex; y = beta + ((x - mean) * rstd) * gamma
+template <int OP, typename T, int VPT>
+__global__ void __launch_bounds__(1024, 1) reg_norm_packed(const RowParams p, const float inv_warps) {
+  pdl_prologue();
+  using E = Elem<T>;
+  static_assert(sizeof(T) == 2, "16-bit storage only");
+  static_assert(OP == OP_LAYERNORM || OP == OP_RMSNORM, "normalisations only");
+  constexpr int EPV = E::EPV;
+  constexpr int N = VPT * EPV;
+  __shared__ float red[2][2][32];
+  const int G = blockDim.x;
+  const int NW = G >> 5;
+  const int tg = threadIdx.x;
+  const float inv_cols = 1.0f / static_cast<float>(p.cols);
+  const bool affine_all = p.gamma != nullptr && (OP != OP_LAYERNORM || p.beta != nullptr);
+  int parity = 0;
+  for (long long row = blockIdx.x; row < p.rows; row += gridDim.x, parity ^= 1) {
+    const T* xr = reinterpret_cast<const T*>(p.x) + row * p.xs + tg * EPV;
+    T* yr = reinterpret_cast<T*>(p.y) + row * p.ys + tg * EPV;
+    uint4 raw[VPT];
+#pragma unroll
+    for (int k = 0; k < VPT; ++k) raw[k] = ld_stream(xr + static_cast<long long>(k) * G * EPV);
+    float mu, m2 = 0.f;
+    if (OP == OP_RMSNORM) {
+      float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+      for (int k = 0; k < VPT; ++k) {
+        const uint32_t w[4] = {raw[k].x, raw[k].y, raw[k].z, raw[k].w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          unsigned short h0, h1;
+          halves(w[i], h0, h1);
+          s0 = E::fma_wide(h0, h0, s0);
+          s1 = E::fma_wide(h1, h1, s1);
+        }
+      }
+      mu = s0 + s1;
+    } else {
+      float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+      for (int k = 0; k < VPT; ++k) {
+        const uint32_t w[4] = {raw[k].x, raw[k].y, raw[k].z, raw[k].w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          unsigned short h0, h1;
+          halves(w[i], h0, h1);
+          s0 = E::add_wide(h0, s0);
+          s1 = E::add_wide(h1, s1);
+        }
+      }
+      mu = (s0 + s1) * (1.0f / N);
+      float q0 = 0.f, q1 = 0.f;
+#pragma unroll
+      for (int k = 0; k < VPT; ++k) {
+        const uint32_t w[4] = {raw[k].x, raw[k].y, raw[k].z, raw[k].w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          unsigned short h0, h1;
+          halves(w[i], h0, h1);
+          const float d0 = E::sub_wide(h0, mu), d1 = E::sub_wide(h1, mu);
+          q0 = fmaf(d0, d0, q0);
+          q1 = fmaf(d1, d1, q1);
+        }
+      }
+      m2 = q0 + q1;
+    }
+    float mean, rstd;
+    flex_merge<OP>(mu, m2, N, red[parity], NW, inv_warps, inv_cols, p.eps, mean, rstd);
+
+    const T* gp = reinterpret_cast<const T*>(p.gamma) + tg * EPV;
+    const T* bp = reinterpret_cast<const T*>(p.beta) + tg * EPV;
+#pragma unroll
+    for (int k = 0; k < VPT; ++k) {
+      const uint32_t xw[4] = {raw[k].x, raw[k].y, raw[k].z, raw[k].w};
+      uint32_t out[4];
+      if (affine_all) {
+        const uint4 gv = ld_cached(gp + static_cast<long long>(k) * G * EPV);
+        const uint32_t gw[4] = {gv.x, gv.y, gv.z, gv.w};
+        if (OP == OP_RMSNORM) {
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            unsigned short x0, x1, g0, g1;
+            halves(xw[i], x0, x1);
+            halves(gw[i], g0, g1);
+            out[i] = E::pack2(E::fma_wide(x0, g0, 0.f) * rstd, E::fma_wide(x1, g1, 0.f) * rstd);
+          }
+        } else {
+          const uint4 bv = ld_cached(bp + static_cast<long long>(k) * G * EPV);
+          const uint32_t bw[4] = {bv.x, bv.y, bv.z, bv.w};
+          float ga[EPV];
+          E::unpack(gv, ga);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            unsigned short x0, x1, b0, b1;
+            halves(xw[i], x0, x1);
+            halves(bw[i], b0, b1);
+            out[i] = E::pack2(E::add_wide(b0, E::sub_wide(x0, mean) * rstd * ga[2 * i]),
+                              E::add_wide(b1, E::sub_wide(x1, mean) * rstd * ga[2 * i + 1]));
+          }
+        }
+      } else {
+        // an absent gamma or beta (1 / 0): the plain formula on unpacked values
+        float v[EPV], g[EPV], b[EPV], o[EPV];
+        E::unpack(raw[k], v);
+#pragma unroll
+        for (int j = 0; j < EPV; ++j) { g[j] = 1.f; b[j] = 0.f; }
+        if (p.gamma != nullptr) E::unpack(ld_cached(gp + static_cast<long long>(k) * G * EPV), g);
+        if (OP == OP_LAYERNORM && p.beta != nullptr) E::unpack(ld_cached(bp + static_cast<long long>(k) * G * EPV), b);
+#pragma unroll
+        for (int j = 0; j < EPV; ++j)
+          o[j] = (OP == OP_LAYERNORM) ? fmaf((v[j] - mean) * rstd, g[j], b[j]) : v[j] * rstd * g[j];
+        const uint4 ov = E::pack(o);
+        out[0] = ov.x; out[1] = ov.y; out[2] = ov.z; out[3] = ov.w;
+      }
+      st_stream(yr + static_cast<long long>(k) * G * EPV, make_uint4(out[0], out[1], out[2], out[3]));
+    }
+  }
+}
+
 // reg_norm_flex: the same predicate-free scheme for rows of exactly blockDim.x * VPT
 // vectors where blockDim.x is any multiple of 32 (hidden sizes such as 5120, 6144, 7168).
 // A CTA per row.  Every warp holds the same number of values, so the warps' (mean, M2)

@@ -218,6 +218,20 @@ cudaError_t launch_typed(const LaunchPlan& plan, const RowParams& p, cudaStream_
   if (plan.variant == V_STREAM) {
     return launch_plain(stream_kernel<OP, T, 256>, plan, plan.grid, 256, 0, s, p);
   }
+  if (plan.variant == V_REG && plan.mode == 3) {            // runtime thread count, exact fit, 16-bit row kept packed
+    if constexpr (!OpTraits<OP>::kSoftmaxLike && sizeof(T) == 2) {
+      const float inv_warps = 1.0f / static_cast<float>(plan.threads / 32);
+      switch (plan.vpt) {
+#define AKG_PACKED_CASE(V_) \
+  case V_: return launch_plain(reg_norm_packed<OP, T, V_>, plan, plan.grid, plan.threads, 0, s, p, inv_warps);
+        AKG_PACKED_CASE(2) AKG_PACKED_CASE(3) AKG_PACKED_CASE(4) AKG_PACKED_CASE(5)
+        AKG_PACKED_CASE(6) AKG_PACKED_CASE(7) AKG_PACKED_CASE(8)
+#undef AKG_PACKED_CASE
+        default: break;
+      }
+    }
+    return cudaErrorInvalidConfiguration;
+  }
   if (plan.variant == V_REG && plan.mode == 2) {            // runtime thread count, exact fit
     if constexpr (!OpTraits<OP>::kSoftmaxLike) {
       const float inv_warps = 1.0f / static_cast<float>(plan.threads / 32);
