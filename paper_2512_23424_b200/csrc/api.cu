@@ -191,6 +191,10 @@ bool plan_reg(const Call& c, LaunchPlan* plan) {
     else if (nvec <= 2048) { threads = 512; vpt = 4; }
     else if (nvec <= 4096 && c.dtype == AKG_F32) { threads = 512; vpt = 8; }   // (16-bit rows beyond 2048 vectors: other families)
     else if (nvec <= 8192 && c.dtype == AKG_F32) { threads = 1024; vpt = 8; }
+    else if (nvec <= 8192 && c.dtype != AKG_F32 && norm_op && nvec % 8 == 0 && (nvec / 8) % 32 == 0 &&
+             g_tune_reg_general.load() == 0 && g_tune_reg_flex.load() != 2 && g_tune_reg_flex.load() != 5) {
+      threads = static_cast<int>(nvec / 8); vpt = 8;     // only as the packed kernel, chosen below
+    }
     else return false;
     group = threads;
   }
@@ -318,7 +322,8 @@ bool plan_smem(const Call& c, int cs_min, int cs_max, LaunchPlan* plan, int want
   if (best_cs == 0) return false;
   const int64_t buf = (best_slice * 16 + 127) & ~int64_t(127);
   plan->variant = (best_cs == 1) ? V_TMA : V_CLUSTER;
-  plan->mode = (best_cs > 1 && g_tune_split_exchange.load() == 1) ? 1 : 0;   // clusters, 1: partials exchanged under a cluster barrier
+  // clusters, 1: partials exchanged under a cluster barrier; 2 (any cluster size): pipelined row loop
+  plan->mode = (best_cs > 1 && g_tune_split_exchange.load() == 1) ? 1 : (g_tune_split_exchange.load() == 2 ? 2 : 0);
   plan->threads = best_threads; plan->group = best_threads; plan->vpt = static_cast<int>(best_slice);
   plan->cluster = best_cs; plan->stages = best_nbuf;
   plan->smem = smem_header_bytes(best_threads) + static_cast<size_t>(best_nbuf) * buf;
@@ -510,25 +515,32 @@ akg_status run(const Call& c, const char* name) {
   // (the ring-fed register kernels are no automatic choice any more: bf16 RMSNorm with many rows, their one
   // case, runs at 0.91 - 0.96 of the copy rate through the ring and at 0.98 - 1.01 in the packed register
   // kernel; forcing the TMA family still reaches them)
-  // 16-bit rows of 16 - 64 KB without a mask, where a CTA's registers no longer hold the row comfortably:
-  // the row resident in shared memory (bulk-copied in, two sweeps over shared memory), several CTAs per SM
-  // so that one row's sweeps overlap the others' copies.  Measured against the register and two-pass
-  // kernels (bf16, fraction of the copy rate): log-softmax 12288 / 16384 / 20480 columns 0.69 / 0.85 / 0.81
-  // against 0.65 / 0.69 / 0.78 with three CTAs of 256 threads per SM; RMSNorm 20480 / 32768 columns
-  // 0.89 / 0.84 against 0.87 / 0.78 with two CTAs of 512.  (Softmax and LayerNorm were level or behind.)
+  // 16-bit log-softmax rows of 24 - 48 KB without a mask, where a CTA's registers no longer hold the row
+  // comfortably: the row resident in shared memory (bulk-copied in, two sweeps over shared memory), three CTAs
+  // of 256 threads per SM so that one row's sweeps overlap the others' copies.  Measured against the register
+  // and two-pass kernels (bf16, fraction of the copy rate): 16384 / 20480 columns 0.79 - 0.85 / 0.81 against
+  // 0.69 / 0.78.  (Softmax was level or behind; the normalisations take the packed register kernel.)
   if (!planned && forced == V_AUTO && vec && c.dtype != AKG_F32 && c.rows >= 2 * static_cast<int64_t>(sm_count()) &&
       (c.mask == nullptr || (c.mask->additive == nullptr && !c.mask->causal)) && g_tune_tma_mode.load() == 0 &&
       g_tune_cluster_mode.load() == 0) {
     const int64_t nv16 = c.cols / 8;
-    if (c.op == OP_LOG_SOFTMAX && nv16 > 1024 && nv16 <= 3072) planned = plan_smem(c, 1, 1, &plan, 256, 3);
-    else if (c.op == OP_RMSNORM && nv16 > 2048 && nv16 <= 4096) planned = plan_smem(c, 1, 1, &plan, 512, 2);
+    if (c.op == OP_LOG_SOFTMAX && nv16 > 1536 && nv16 <= 3072) planned = plan_smem(c, 1, 1, &plan, 256, 3);
     if (planned) p.status = status_word_ptr();
   }
   // rows beyond 2048 vectors in the 16-bit types (beyond 4096 for the fp32 softmax pair) measured
   // faster in the two-pass kernel than in one CTA of 640 - 1024 threads: bf16 32768 columns 77 - 79 %
   // against 63 %, fp32 softmax 32768 columns 81 % against 77 % (fp32 normalisations: 82 % against 93 %, kept)
   const int64_t row_vecs = c.cols / ((c.dtype == AKG_F32) ? 4 : 8);
-  const bool long_row = forced == V_AUTO && g_tune_cluster_mode.load() != 1 &&
+  // (16-bit normalisation rows stay in registers up to 8192 vectors where the packed kernel fits them: bf16
+  // 20480 - 32768 columns LayerNorm 0.86 - 0.92 against 0.74 - 0.77 in the two-pass kernel, RMSNorm 0.94 - 0.96
+  // against 0.64 - 0.85 with the row in shared memory; 65536 columns 0.71 / 0.85 against 0.69 / 0.75)
+  const bool packed_fits = c.dtype != AKG_F32 && (c.op == OP_LAYERNORM || c.op == OP_RMSNORM) && row_vecs <= 8192 &&
+                           row_vecs % 8 == 0 && (row_vecs / 8) % 32 == 0 && g_tune_reg_general.load() == 0 &&
+                           g_tune_reg_flex.load() != 2 && g_tune_reg_flex.load() != 5 &&
+                           // a CTA per row needs rows for about a full wave of threads; fewer rows are cut into
+                           // slices by the two-pass cluster kernel
+                           c.rows * (row_vecs / 8) >= static_cast<int64_t>(sm_count()) * 1024;
+  const bool long_row = forced == V_AUTO && g_tune_cluster_mode.load() != 1 && !packed_fits &&
                         ((c.dtype != AKG_F32 && row_vecs > 2048) ||
                          (c.dtype == AKG_F32 && row_vecs > 4096 && (c.op == OP_SOFTMAX || c.op == OP_LOG_SOFTMAX)));
   if (!planned && (forced == V_AUTO || forced == V_REG) && vec && !long_row) {

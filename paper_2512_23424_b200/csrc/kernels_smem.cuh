@@ -101,7 +101,8 @@ struct SmemGeom {
 constexpr int kXSlots = 4;          // exchange slots of smem_kernel (see its comment)
 
 template <int OP, typename T, int THREADS>
-__global__ void __launch_bounds__(THREADS) smem_kernel(const RowParams p, const SmemGeom g, const int xmode) {
+__global__ void __launch_bounds__(THREADS, THREADS == 256 ? 3 : 1)      // 256 threads: three CTAs per SM, 85 registers
+smem_kernel(const RowParams p, const SmemGeom g, const int xmode) {
   pdl_prologue();
   using E = Elem<T>;
   constexpr int EPV = E::EPV;
@@ -129,15 +130,19 @@ __global__ void __launch_bounds__(THREADS) smem_kernel(const RowParams p, const 
   // Exchange of the slices' partial statistics.
   // xmode 1 (default): as in split_kernel, one 16-byte st.async per peer that counts on the receiver's
   // mbarrier, so that no cluster barrier (whose release waits for the CTA's global stores of the row
-  // before) stands between two rows.  With a ring of two and more buffers the row loop is also software-
-  // pipelined: the first sweep of row r + 1 and the sending of its partials come BEFORE the wait for the
-  // partials of row r, whose latency then hides behind that sweep (one CTA per SM has nothing else to hide
-  // it behind).  A CTA can therefore be up to two rows ahead of a peer's reads, hence four exchange slots
+  // before) stands between two rows.  xmode 2 also software-pipelines the row loop over a ring of two and
+  // more buffers: the first sweep of row r + 1 and the sending of its partials come BEFORE the wait for the
+  // partials of row r, whose latency then hides behind that sweep.
+  // A CTA can therefore be up to two rows ahead of a peer's reads, hence four exchange slots
   // (row r uses slot r mod 4): a peer sends row r + 4 only after it has received every CTA's partial of
   // row r + 2, and a CTA sends that after it has read the slot of row r.
   // xmode 0: plain remote stores and a cluster barrier per row, no pipelining (the first version).
   const bool async_x = xmode != 0 && cs > 1;
-  const bool pipelined = (xmode != 0 || cs == 1) && g.nbuf >= 2;
+  // (measured: no gain for one CTA per SM - 166 us against 165 us on configuration 4 - and a loss where several
+  // CTAs share an SM and hide each other's waits anyway - bf16 log-softmax 16384 columns 0.66 against 0.85 of
+  // the copy rate, because the wait for the NEXT row's copy then delays the stores and the refill of the
+  // current one; the order is kept for experiments only)
+  const bool pipelined = xmode == 2 && g.nbuf >= 2;
   if (threadIdx.x == 0) {
     for (int b = 0; b < g.nbuf; ++b) mbar_init(smem_addr(&bars[b]), 1);
     for (int k = 0; k < kXSlots; ++k) mbar_init(smem_addr(&xbar[k]), 1);

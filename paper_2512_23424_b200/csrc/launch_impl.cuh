@@ -123,7 +123,7 @@ cudaError_t launch_smem(const LaunchPlan& plan, const RowParams& p, cudaStream_t
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.numAttrs = 2;
   }
-  return cudaLaunchKernelEx(&cfg, kernel, p, g, plan.mode == 1 ? 0 : 1);
+  return cudaLaunchKernelEx(&cfg, kernel, p, g, plan.variant == V_CLUSTER ? (plan.mode == 1 ? 0 : (plan.mode == 2 ? 2 : 1)) : (plan.mode == 2 ? 2 : 1));
 }
 
 // Launch a ring-fed register kernel (persistent; plan.grid == 0 asks for one full wave).
