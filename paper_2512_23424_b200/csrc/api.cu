@@ -191,7 +191,8 @@ bool plan_reg(const Call& c, LaunchPlan* plan) {
     else if (nvec <= 2048) { threads = 512; vpt = 4; }
     else if (nvec <= 4096 && c.dtype == AKG_F32) { threads = 512; vpt = 8; }   // (16-bit rows beyond 2048 vectors: other families)
     else if (nvec <= 8192 && c.dtype == AKG_F32) { threads = 1024; vpt = 8; }
-    else if (nvec <= 8192 && c.dtype != AKG_F32 && norm_op && nvec % 8 == 0 && (nvec / 8) % 32 == 0 &&
+    else if (nvec <= 8192 && c.dtype != AKG_F32 && nvec % 8 == 0 && (nvec / 8) % 32 == 0 &&
+             (norm_op || c.mask == nullptr || (c.mask->additive == nullptr && !c.mask->causal)) &&
              g_tune_reg_general.load() == 0 && g_tune_reg_flex.load() != 2 && g_tune_reg_flex.load() != 5) {
       threads = static_cast<int>(nvec / 8); vpt = 8;     // only as the packed kernel, chosen below
     }
@@ -263,7 +264,9 @@ bool plan_reg(const Call& c, LaunchPlan* plan) {
   // LayerNorm the most that leaves 64 threads (8192 columns: eight 0.95, four 0.88); RMSNorm four while that
   // keeps the CTA at 384 threads or fewer (8192 columns: four 1.01, eight 0.98), else the most (16384: eight
   // 0.97, four 0.89).
-  if (norm && c.dtype != AKG_F32 && group == threads && g_tune_reg_general.load() == 0 &&
+  // The unmasked softmax pair has a packed form too (reg_softmax_packed).
+  const bool unmasked = c.mask == nullptr || (c.mask->additive == nullptr && !c.mask->causal);
+  if ((norm || unmasked) && c.dtype != AKG_F32 && group == threads && g_tune_reg_general.load() == 0 &&
       !(t_threads > 0 && t_vpt > 0) && g_tune_reg_flex.load() != 2 && g_tune_reg_flex.load() != 5) {
     const int want = g_tune_packed_vpt.load();
     int pv = 0;
@@ -283,6 +286,8 @@ bool plan_reg(const Call& c, LaunchPlan* plan) {
       if (plan->grid > pcap) plan->grid = pcap;
     }
   }
+  // (16-bit rows beyond 2048 vectors are in this family only in their packed form)
+  if (c.dtype != AKG_F32 && nvec > 2048 && plan->mode != 3) return false;
   return true;
 }
 
@@ -507,34 +512,27 @@ akg_status run(const Call& c, const char* name) {
   std::memset(&plan, 0, sizeof plan);
   bool planned = false;
   // Automatic choice (each rule is a measured preference on B200, see the profiles):
-  //   every row that fits a CTA's registers -> register kernels (plan_reg; 16-bit normalisation rows in
-  //     their packed form)
-  //   16-bit log-softmax rows of 16 - 48 KB and RMSNorm rows of 32 - 64 KB -> row resident in shared memory
+  //   every row that fits a CTA's registers -> register kernels (plan_reg; 16-bit rows without a mask in
+  //     their packed form, up to 8192 vectors)
   //   longer aligned rows -> two-pass split cluster kernel (second pass from L2)
   //   anything unaligned -> scalar stream kernel
   // (the ring-fed register kernels are no automatic choice any more: bf16 RMSNorm with many rows, their one
   // case, runs at 0.91 - 0.96 of the copy rate through the ring and at 0.98 - 1.01 in the packed register
   // kernel; forcing the TMA family still reaches them)
-  // 16-bit log-softmax rows of 24 - 48 KB without a mask, where a CTA's registers no longer hold the row
-  // comfortably: the row resident in shared memory (bulk-copied in, two sweeps over shared memory), three CTAs
-  // of 256 threads per SM so that one row's sweeps overlap the others' copies.  Measured against the register
-  // and two-pass kernels (bf16, fraction of the copy rate): 16384 / 20480 columns 0.79 - 0.85 / 0.81 against
-  // 0.69 / 0.78.  (Softmax was level or behind; the normalisations take the packed register kernel.)
-  if (!planned && forced == V_AUTO && vec && c.dtype != AKG_F32 && c.rows >= 2 * static_cast<int64_t>(sm_count()) &&
-      (c.mask == nullptr || (c.mask->additive == nullptr && !c.mask->causal)) && g_tune_tma_mode.load() == 0 &&
-      g_tune_cluster_mode.load() == 0) {
-    const int64_t nv16 = c.cols / 8;
-    if (c.op == OP_LOG_SOFTMAX && nv16 > 1536 && nv16 <= 3072) planned = plan_smem(c, 1, 1, &plan, 256, 3);
-    if (planned) p.status = status_word_ptr();
-  }
+  // (the kernel that keeps a row in shared memory is no automatic choice either: its best case, 16-bit
+  // log-softmax rows of 32 - 40 KB with three CTAs of 256 threads per SM, measured 0.79 - 0.85 of the copy rate
+  // against 0.69 - 0.78 in the widened register / two-pass kernels, and 0.96 - 1.0 in the packed register kernel)
   // rows beyond 2048 vectors in the 16-bit types (beyond 4096 for the fp32 softmax pair) measured
   // faster in the two-pass kernel than in one CTA of 640 - 1024 threads: bf16 32768 columns 77 - 79 %
   // against 63 %, fp32 softmax 32768 columns 81 % against 77 % (fp32 normalisations: 82 % against 93 %, kept)
   const int64_t row_vecs = c.cols / ((c.dtype == AKG_F32) ? 4 : 8);
-  // (16-bit normalisation rows stay in registers up to 8192 vectors where the packed kernel fits them: bf16
+  // (unmasked 16-bit rows stay in registers up to 8192 vectors where the packed kernels fit them: bf16
   // 20480 - 32768 columns LayerNorm 0.86 - 0.92 against 0.74 - 0.77 in the two-pass kernel, RMSNorm 0.94 - 0.96
-  // against 0.64 - 0.85 with the row in shared memory; 65536 columns 0.71 / 0.85 against 0.69 / 0.75)
-  const bool packed_fits = c.dtype != AKG_F32 && (c.op == OP_LAYERNORM || c.op == OP_RMSNORM) && row_vecs <= 8192 &&
+  // against 0.64 - 0.85 with the row in shared memory, softmax 0.95 - 0.99 against 0.70, log-softmax 0.96
+  // against 0.72; 65536 columns 0.71 / 0.85 / 0.70 / 0.72 against 0.69 / 0.75 / 0.69 / 0.71)
+  const bool packed_fits = c.dtype != AKG_F32 && row_vecs <= 8192 &&
+                           (c.op == OP_LAYERNORM || c.op == OP_RMSNORM || c.mask == nullptr ||
+                            (c.mask->additive == nullptr && !c.mask->causal)) &&
                            row_vecs % 8 == 0 && (row_vecs / 8) % 32 == 0 && g_tune_reg_general.load() == 0 &&
                            g_tune_reg_flex.load() != 2 && g_tune_reg_flex.load() != 5 &&
                            // a CTA per row needs rows for about a full wave of threads; fewer rows are cut into

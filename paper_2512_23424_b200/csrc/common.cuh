@@ -194,6 +194,14 @@ template <> struct Elem<__nv_bfloat16> {
   }
 };
 
+// element-wise maximum of two packed pairs (a NaN operand is ignored, as fmaxf does)
+__device__ __forceinline__ uint32_t max_pair(const __nv_bfloat16*, uint32_t a, uint32_t b) {
+  uint32_t d; asm("max.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b)); return d;
+}
+__device__ __forceinline__ uint32_t max_pair(const __half*, uint32_t a, uint32_t b) {
+  uint32_t d; asm("max.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b)); return d;
+}
+
 // the two 16-bit halves of a packed word (low half = even element)
 __device__ __forceinline__ void halves(uint32_t w, unsigned short& lo, unsigned short& hi) {
   asm("mov.b32 {%0, %1}, %2;" : "=h"(lo), "=h"(hi) : "r"(w));

@@ -263,4 +263,110 @@ __global__ void __launch_bounds__(THREADS, kSoftmaxMinBlocks<G, THREADS, VPT>) r
   }
 }
 
+
+// ------------------------------------------------------------------------------------------------
+// reg_softmax_packed: the softmax pair on unmasked 16-bit rows of exactly blockDim.x * VPT vectors, the
+// row kept PACKED in registers (as reg_norm_packed: four registers per vector, eight vectors per thread in
+// 64 registers, half the threads per row of the widened form, eight loads per thread in flight).
+//   maximum   packed two-lane maxima over the words (one instruction per two elements)
+//   sum       e^(x - m_warp) with the stored value widened inside the subtraction (Elem::sub_wide), against
+//             the warp's own maximum, so that one barrier serves both reductions
+//   output    softmax: the exponential again, against the row maximum, times 1 / S (the widened form keeps
+//             the first exponential instead: a second one here costs less than the registers for it);
+//             log-softmax: scale (x - M) - ln S
+// A CTA per row, grid-stride.  No mask: the planner sends masked calls to the kernels above.
+// ------------------------------------------------------------------------------------------------
+template <int OP, typename T, int VPT>
+__global__ void __launch_bounds__(1024, 1) reg_softmax_packed(const RowParams p) {
+  pdl_prologue();
+  using E = Elem<T>;
+  static_assert(sizeof(T) == 2, "16-bit storage only");
+  static_assert(OP == OP_SOFTMAX || OP == OP_LOG_SOFTMAX, "softmax pair only");
+  constexpr int EPV = E::EPV;
+  __shared__ float red[2][2][32];
+  const int G = blockDim.x;
+  const int NW = G >> 5;
+  const int tg = threadIdx.x;
+  const int lane = tg & 31;
+  const float l2e = p.l2e;
+  int parity = 0;
+  for (long long row = blockIdx.x; row < p.rows; row += gridDim.x, parity ^= 1) {
+    const T* xr = reinterpret_cast<const T*>(p.x) + row * p.xs + tg * EPV;
+    T* yr = reinterpret_cast<T*>(p.y) + row * p.ys + tg * EPV;
+    uint4 raw[VPT];
+#pragma unroll
+    for (int k = 0; k < VPT; ++k) raw[k] = ld_stream(xr + static_cast<long long>(k) * G * EPV);
+    // ---- maximum
+    uint32_t mp = max_pair(static_cast<const T*>(nullptr), raw[0].x, raw[0].y);
+    mp = max_pair(static_cast<const T*>(nullptr), mp, max_pair(static_cast<const T*>(nullptr), raw[0].z, raw[0].w));
+#pragma unroll
+    for (int k = 1; k < VPT; ++k) {
+      const uint32_t a = max_pair(static_cast<const T*>(nullptr), raw[k].x, raw[k].y);
+      const uint32_t b = max_pair(static_cast<const T*>(nullptr), raw[k].z, raw[k].w);
+      mp = max_pair(static_cast<const T*>(nullptr), mp, max_pair(static_cast<const T*>(nullptr), a, b));
+    }
+    unsigned short m0, m1;
+    halves(mp, m0, m1);
+    const float m_w = warp_max(fmaxf(E::add_wide(m0, 0.f), E::add_wide(m1, 0.f)));
+    const float m_ws = (m_w == kNegInf) ? 0.f : m_w;        // keeps -inf - -inf out of the exponent
+    // ---- sum of exponentials against the warp's maximum (a NaN element makes the sum NaN)
+    float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+    for (int k = 0; k < VPT; ++k) {
+      const uint32_t w[4] = {raw[k].x, raw[k].y, raw[k].z, raw[k].w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        unsigned short h0, h1;
+        halves(w[i], h0, h1);
+        s0 += ex2_approx(E::sub_wide(h0, m_ws) * l2e);
+        s1 += ex2_approx(E::sub_wide(h1, m_ws) * l2e);
+      }
+    }
+    const float s_w = warp_sum(s0 + s1);
+    // ---- the warps' pairs: lane l takes warp l's (nothing beyond the CTA's warps)
+    float M = m_w, S = s_w;
+    if (NW > 1) {
+      if (lane == 0) { red[parity][0][tg >> 5] = m_w; red[parity][1][tg >> 5] = s_w; }
+      __syncthreads();
+      const float mw = lane < NW ? red[parity][0][lane] : kNegInf;
+      const float sw = lane < NW ? red[parity][1][lane] : 0.f;
+      M = warp_max(mw);
+      const float Ms = (M == kNegInf) ? 0.f : M;
+      S = warp_sum(sw * ((mw == M) ? 1.f : exp_diff(mw, Ms, l2e)));      // equal maxima (also +-inf): factor 1
+    }
+    const bool dead = (M == kNegInf) && !(S != S);        // only NaN / -inf entries: a NaN row, not a dead one
+    const float Mo = (M == kNegInf) ? 0.f : M;
+    if (OP == OP_SOFTMAX) {
+      const float inv = dead ? 0.f : __frcp_rn(S);
+#pragma unroll
+      for (int k = 0; k < VPT; ++k) {
+        const uint32_t w[4] = {raw[k].x, raw[k].y, raw[k].z, raw[k].w};
+        uint32_t o[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          unsigned short h0, h1;
+          halves(w[i], h0, h1);
+          o[i] = E::pack2(ex2_approx(E::sub_wide(h0, Mo) * l2e) * inv, ex2_approx(E::sub_wide(h1, Mo) * l2e) * inv);
+        }
+        st_stream(yr + static_cast<long long>(k) * G * EPV, make_uint4(o[0], o[1], o[2], o[3]));
+      }
+    } else {
+      // a dead row: M and ln S are taken as 0, and scale (-inf - 0) - 0 = -inf for every element by itself
+      const float neg_lse = dead ? 0.f : -logf(S);
+#pragma unroll
+      for (int k = 0; k < VPT; ++k) {
+        const uint32_t w[4] = {raw[k].x, raw[k].y, raw[k].z, raw[k].w};
+        uint32_t o[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          unsigned short h0, h1;
+          halves(w[i], h0, h1);
+          o[i] = E::pack2(fmaf(E::sub_wide(h0, Mo), p.scale, neg_lse), fmaf(E::sub_wide(h1, Mo), p.scale, neg_lse));
+        }
+        st_stream(yr + static_cast<long long>(k) * G * EPV, make_uint4(o[0], o[1], o[2], o[3]));
+      }
+    }
+  }
+}
+
 }  // namespace akg

@@ -219,6 +219,16 @@ cudaError_t launch_typed(const LaunchPlan& plan, const RowParams& p, cudaStream_
     return launch_plain(stream_kernel<OP, T, 256>, plan, plan.grid, 256, 0, s, p);
   }
   if (plan.variant == V_REG && plan.mode == 3) {            // runtime thread count, exact fit, 16-bit row kept packed
+    if constexpr (OpTraits<OP>::kSoftmaxLike && sizeof(T) == 2) {
+      switch (plan.vpt) {
+#define AKG_PACKED_SM_CASE(V_) \
+  case V_: return launch_plain(reg_softmax_packed<OP, T, V_>, plan, plan.grid, plan.threads, 0, s, p);
+        AKG_PACKED_SM_CASE(2) AKG_PACKED_SM_CASE(3) AKG_PACKED_SM_CASE(4) AKG_PACKED_SM_CASE(5)
+        AKG_PACKED_SM_CASE(6) AKG_PACKED_SM_CASE(7) AKG_PACKED_SM_CASE(8)
+#undef AKG_PACKED_SM_CASE
+        default: break;
+      }
+    }
     if constexpr (!OpTraits<OP>::kSoftmaxLike && sizeof(T) == 2) {
       const float inv_warps = 1.0f / static_cast<float>(plan.threads / 32);
       switch (plan.vpt) {
