@@ -191,8 +191,9 @@ bool plan_reg(const Call& c, LaunchPlan* plan) {
     else if (nvec <= 2048) { threads = 512; vpt = 4; }
     else if (nvec <= 4096 && c.dtype == AKG_F32) { threads = 512; vpt = 8; }   // (16-bit rows beyond 2048 vectors: other families)
     else if (nvec <= 8192 && c.dtype == AKG_F32) { threads = 1024; vpt = 8; }
-    else if (nvec <= 8192 && c.dtype != AKG_F32 && nvec % 8 == 0 && (nvec / 8) % 32 == 0 &&
-             (norm_op || c.mask == nullptr || (c.mask->additive == nullptr && !c.mask->causal)) &&
+    else if (nvec <= 8192 && nvec % 8 == 0 && (nvec / 8) % 32 == 0 &&
+             ((norm_op && c.dtype != AKG_F32) ||
+              (!norm_op && (c.mask == nullptr || (c.mask->additive == nullptr && !c.mask->causal)))) &&
              g_tune_reg_general.load() == 0 && g_tune_reg_flex.load() != 2 && g_tune_reg_flex.load() != 5) {
       threads = static_cast<int>(nvec / 8); vpt = 8;     // only as the packed kernel, chosen below
     }
@@ -266,7 +267,8 @@ bool plan_reg(const Call& c, LaunchPlan* plan) {
   // 0.97, four 0.89).
   // The unmasked softmax pair has a packed form too (reg_softmax_packed).
   const bool unmasked = c.mask == nullptr || (c.mask->additive == nullptr && !c.mask->causal);
-  if ((norm || unmasked) && c.dtype != AKG_F32 && group == threads && g_tune_reg_general.load() == 0 &&
+  // ... and so has the unmasked fp32 softmax pair its runtime-thread-count form (reg_softmax_flex).
+  if (((norm && c.dtype != AKG_F32) || (!norm && unmasked)) && group == threads && g_tune_reg_general.load() == 0 &&
       !(t_threads > 0 && t_vpt > 0) && g_tune_reg_flex.load() != 2 && g_tune_reg_flex.load() != 5) {
     const int want = g_tune_packed_vpt.load();
     int pv = 0;
@@ -286,8 +288,8 @@ bool plan_reg(const Call& c, LaunchPlan* plan) {
       if (plan->grid > pcap) plan->grid = pcap;
     }
   }
-  // (16-bit rows beyond 2048 vectors are in this family only in their packed form)
-  if (c.dtype != AKG_F32 && nvec > 2048 && plan->mode != 3) return false;
+  // (16-bit rows beyond 2048 vectors, and fp32 softmax rows beyond 4096, are in this family only in that form)
+  if (plan->mode != 3 && ((c.dtype != AKG_F32 && nvec > 2048) || (c.dtype == AKG_F32 && !norm && nvec > 4096))) return false;
   return true;
 }
 
@@ -530,9 +532,10 @@ akg_status run(const Call& c, const char* name) {
   // 20480 - 32768 columns LayerNorm 0.86 - 0.92 against 0.74 - 0.77 in the two-pass kernel, RMSNorm 0.94 - 0.96
   // against 0.64 - 0.85 with the row in shared memory, softmax 0.95 - 0.99 against 0.70, log-softmax 0.96
   // against 0.72; 65536 columns 0.71 / 0.85 / 0.70 / 0.72 against 0.69 / 0.75 / 0.69 / 0.71)
-  const bool packed_fits = c.dtype != AKG_F32 && row_vecs <= 8192 &&
-                           (c.op == OP_LAYERNORM || c.op == OP_RMSNORM || c.mask == nullptr ||
-                            (c.mask->additive == nullptr && !c.mask->causal)) &&
+  const bool norm_call = c.op == OP_LAYERNORM || c.op == OP_RMSNORM;
+  const bool packed_fits = row_vecs <= 8192 &&
+                           ((norm_call && c.dtype != AKG_F32) ||
+                            (!norm_call && (c.mask == nullptr || (c.mask->additive == nullptr && !c.mask->causal)))) &&
                            row_vecs % 8 == 0 && (row_vecs / 8) % 32 == 0 && g_tune_reg_general.load() == 0 &&
                            g_tune_reg_flex.load() != 2 && g_tune_reg_flex.load() != 5 &&
                            // a CTA per row needs rows for about a full wave of threads; fewer rows are cut into
@@ -546,7 +549,7 @@ akg_status run(const Call& c, const char* name) {
     // fp32 normalisation rows beyond 4096 vectors stay in registers only as an exact fit (the ragged
     // 1024-thread form measured 49 % on 32000 columns)
     if (planned && forced == V_AUTO && g_tune_cluster_mode.load() != 1 && c.dtype == AKG_F32 && row_vecs > 4096 &&
-        plan.mode != 2 && plan.stages != 1) {
+        plan.mode != 2 && plan.mode != 3 && plan.stages != 1) {
       planned = false;
       plan = LaunchPlan{};
     }
@@ -582,7 +585,7 @@ akg_status run(const Call& c, const char* name) {
   const char* dt = dtype_name(c.dtype);
   if (plan.variant == V_REG)
     std::snprintf(t_kernel, sizeof t_kernel, "reg<%s,g%d,t%d,v%d%s>", dt, plan.group, plan.threads, plan.vpt,
-                  plan.mode == 3 ? ",packed" : plan.mode == 2 ? ",flex"
+                  plan.mode == 3 ? (c.dtype == AKG_F32 ? ",flex" : ",packed") : plan.mode == 2 ? ",flex"
                                  : ((plan.stages == 1 && (c.op == OP_LAYERNORM || c.op == OP_RMSNORM)) ? ",full" : ""));
   else if (plan.variant == V_TMA || plan.variant == V_CLUSTER)
     std::snprintf(t_kernel, sizeof t_kernel, "%s<%s,t%d,cs%d,nbuf%d,slice%d>",

@@ -369,4 +369,86 @@ __global__ void __launch_bounds__(1024, 1) reg_softmax_packed(const RowParams p)
   }
 }
 
+
+// ------------------------------------------------------------------------------------------------
+// reg_softmax_flex: the fp32 counterpart of reg_softmax_packed - the softmax pair on unmasked fp32 rows of
+// exactly blockDim.x * VPT vectors, blockDim.x any multiple of 32, so that a row takes the fewest threads
+// that hold it with up to eight vectors each (12288 columns: 384 threads of eight instead of a ragged CTA of
+// 512).  Values in registers, one exponential per element (softmax keeps it for the output), one barrier.
+// ------------------------------------------------------------------------------------------------
+template <int OP, int VPT>
+__global__ void __launch_bounds__(1024, 1) reg_softmax_flex(const RowParams p) {
+  pdl_prologue();
+  using E = Elem<float>;
+  static_assert(OP == OP_SOFTMAX || OP == OP_LOG_SOFTMAX, "softmax pair only");
+  constexpr int EPV = E::EPV;
+  constexpr int N = VPT * EPV;
+  __shared__ float red[2][2][32];
+  const int G = blockDim.x;
+  const int NW = G >> 5;
+  const int tg = threadIdx.x;
+  const int lane = tg & 31;
+  const float l2e = p.l2e;
+  int parity = 0;
+  for (long long row = blockIdx.x; row < p.rows; row += gridDim.x, parity ^= 1) {
+    const float* xr = reinterpret_cast<const float*>(p.x) + row * p.xs + tg * EPV;
+    float* yr = reinterpret_cast<float*>(p.y) + row * p.ys + tg * EPV;
+    uint4 raw[VPT];
+#pragma unroll
+    for (int k = 0; k < VPT; ++k) raw[k] = ld_stream(xr + static_cast<long long>(k) * G * EPV);
+    float v[N];
+    float m_t = kNegInf;
+#pragma unroll
+    for (int k = 0; k < VPT; ++k) {
+      float f[EPV];
+      E::unpack(raw[k], f);
+#pragma unroll
+      for (int j = 0; j < EPV; ++j) { v[k * EPV + j] = f[j]; m_t = fmaxf(m_t, f[j]); }
+    }
+    const float m_w = warp_max(m_t);
+    const float m_ws = (m_w == kNegInf) ? 0.f : m_w;        // keeps -inf - -inf out of the exponent
+    float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+    for (int i = 0; i < N; i += 2) {
+      const float e0 = exp_diff(v[i], m_ws, l2e), e1 = exp_diff(v[i + 1], m_ws, l2e);
+      s0 += e0;
+      s1 += e1;
+      if (OP == OP_SOFTMAX) { v[i] = e0; v[i + 1] = e1; }
+    }
+    const float s_w = warp_sum(s0 + s1);
+    float M = m_w, S = s_w, my_factor = 1.f;
+    if (NW > 1) {
+      if (lane == 0) { red[parity][0][tg >> 5] = m_w; red[parity][1][tg >> 5] = s_w; }
+      __syncthreads();
+      const float mw = lane < NW ? red[parity][0][lane] : kNegInf;
+      const float sw = lane < NW ? red[parity][1][lane] : 0.f;
+      M = warp_max(mw);
+      const float Ms = (M == kNegInf) ? 0.f : M;
+      S = warp_sum(sw * ((mw == M) ? 1.f : exp_diff(mw, Ms, l2e)));      // equal maxima (also +-inf): factor 1
+      my_factor = (m_w == M) ? 1.f : exp_diff(m_w, Ms, l2e);
+    }
+    const bool dead = (M == kNegInf) && !(S != S);        // only NaN / -inf entries: a NaN row, not a dead one
+    if (OP == OP_SOFTMAX) {
+      const float scale = dead ? 0.f : my_factor * __frcp_rn(S);
+#pragma unroll
+      for (int k = 0; k < VPT; ++k) {
+        float o[EPV];
+#pragma unroll
+        for (int j = 0; j < EPV; ++j) o[j] = v[k * EPV + j] * scale;
+        st_stream(yr + static_cast<long long>(k) * G * EPV, E::pack(o));
+      }
+    } else {
+      // a dead row: M and ln S are taken as 0, and scale (-inf - 0) - 0 = -inf for every element by itself
+      const float Mo = dead ? 0.f : M, neg_lse = dead ? 0.f : -logf(S);
+#pragma unroll
+      for (int k = 0; k < VPT; ++k) {
+        float o[EPV];
+#pragma unroll
+        for (int j = 0; j < EPV; ++j) o[j] = fmaf(v[k * EPV + j] - Mo, p.scale, neg_lse);
+        st_stream(yr + static_cast<long long>(k) * G * EPV, E::pack(o));
+      }
+    }
+  }
+}
+
 }  // namespace akg

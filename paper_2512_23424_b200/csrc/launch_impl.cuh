@@ -229,6 +229,16 @@ cudaError_t launch_typed(const LaunchPlan& plan, const RowParams& p, cudaStream_
         default: break;
       }
     }
+    if constexpr (OpTraits<OP>::kSoftmaxLike && sizeof(T) == 4) {    // fp32: the same scheme on widened values
+      switch (plan.vpt) {
+#define AKG_FLEX_SM_CASE(V_) \
+  case V_: return launch_plain(reg_softmax_flex<OP, V_>, plan, plan.grid, plan.threads, 0, s, p);
+        AKG_FLEX_SM_CASE(2) AKG_FLEX_SM_CASE(3) AKG_FLEX_SM_CASE(4) AKG_FLEX_SM_CASE(5)
+        AKG_FLEX_SM_CASE(6) AKG_FLEX_SM_CASE(7) AKG_FLEX_SM_CASE(8)
+#undef AKG_FLEX_SM_CASE
+        default: break;
+      }
+    }
     if constexpr (!OpTraits<OP>::kSoftmaxLike && sizeof(T) == 2) {
       const float inv_warps = 1.0f / static_cast<float>(plan.threads / 32);
       switch (plan.vpt) {

@@ -132,7 +132,9 @@ def test_sixteen_bit_rows_beyond_2048_vectors_leave_the_register_form(dtype):
     # the fp32 normalisations stay in registers while the row is an exact fit, ragged rows do not
     check(wl.make_random("rmsnorm", wl.F32, 300, 32768, seed=352), ("reg", "flex"))
     check(wl.make_random("layernorm", wl.F32, 300, 32000, seed=353), ("split",))
-    check(wl.make_random("softmax", wl.F32, 300, 32768, seed=354), ("split", "cs2,"))
+    # the unmasked fp32 softmax pair stays in registers up to 8192 vectors as well; a mask sends it to the cluster
+    check(wl.make_random("softmax", wl.F32, 300, 32768, seed=354), ("reg<", "t1024,v8,flex"))
+    check(dataclasses.replace(wl.make_random("softmax", wl.F32, 300, 32768, seed=354), causal_period=77), ("split", "cs2,"))
 
 
 # ---- softmax, a CTA per row: the next row is loaded ahead -------------------------------------------
@@ -143,7 +145,7 @@ def test_softmax_prefetch_over_persistent_grid(dtype):
     rows, cols = sms * 12 + 301, 4096            # more rows than CTAs: each CTA prefetches its next row
     for op in ("softmax", "log_softmax"):
         w = wl.make_random(op, dtype, rows, cols, seed=360, scale=3.0)
-        w = dataclasses.replace(w, causal_period=4096 if dtype != wl.F32 else 0)
+        w = dataclasses.replace(w, causal_period=4096)     # (unmasked rows take the packed / flex kernels)
         if w.causal_period:
             x = w.x.copy()
             bad = np.float32(np.nan) if dtype == wl.F32 else (np.uint16(0x7FC0) if dtype == wl.BF16 else np.float16(np.nan))
