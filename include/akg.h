@@ -315,7 +315,8 @@ akg_status akg_set_variant(akg_variant variant);
  * limit), "smem_threads" (256, 512, 1024), "smem_ctas" (CTAs per SM the ring is
  * sized for), "tma_mode" (1 = ring-fed register kernels, 2 = shared-memory passes),
  * "cluster_mode" (1 = row resident in the cluster's shared memory, 2 = two streaming
- * passes with the second served by L2), "reg_general" (1 = never the predicate-free
+ * passes with the second served by L2, 3 = unmasked softmax rows resident in the cluster's
+ * registers), "reg_general" (1 = never the predicate-free
  * normalisation kernel), "interleave" (1 = visit causal rows short/long alternately),
  * "host_chunks", "host_min_kib" (host-buffer entry point: chunks per call, smallest chunk),
  * "host_full_upload" (1 = upload the masked columns of causal rows too),

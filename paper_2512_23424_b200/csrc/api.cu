@@ -293,6 +293,36 @@ bool plan_reg(const Call& c, LaunchPlan* plan) {
   return true;
 }
 
+// Register-resident cluster plan for the unmasked softmax pair: a cluster of cs CTAs per row, CTA k holding
+// slice k of the row in registers (eight vectors per thread), the (maximum, sum) pairs exchanged through
+// distributed shared memory.  Rows of exactly cs * threads * 8 vectors, threads a multiple of 32.  Among the
+// cluster sizes that fit, the smallest whose CTAs have at most 512 threads (two CTAs per SM) and that gives
+// the GPU two CTAs per SM; false if none fits.
+bool plan_cluster_reg(const Call& c, LaunchPlan* plan) {
+  if (c.op != OP_SOFTMAX && c.op != OP_LOG_SOFTMAX) return false;
+  if (c.mask != nullptr && (c.mask->additive != nullptr || c.mask->causal)) return false;
+  if (g_tune_reg_general.load() != 0 || g_tune_reg_flex.load() == 2 || g_tune_reg_flex.load() == 5) return false;
+  const int64_t epv = (c.dtype == AKG_F32) ? 4 : 8;
+  const int64_t nvec = c.cols / epv;
+  const int t_cs = g_tune_cluster_size.load();
+  int best = 0;
+  for (int cs = 2; cs <= kMaxCluster; cs *= 2) {
+    if (t_cs > 0 && cs != t_cs) continue;
+    if (nvec % (cs * 8)) continue;
+    const int64_t g = nvec / (cs * 8);
+    if (g % 32 || g < 64 || g > 1024) continue;
+    if (best == 0) best = cs;                               // the smallest that fits at all
+    if (g <= 512 && (c.rows * cs >= 2 * static_cast<int64_t>(sm_count()) || cs == kMaxCluster)) { best = cs; break; }
+    if (g <= 512) best = cs;
+  }
+  if (best == 0) return false;
+  const int64_t clusters = std::min<int64_t>(c.rows, INT_MAX / best);
+  plan->variant = V_REG; plan->mode = 3; plan->stages = 0; plan->vpt = 8; plan->cluster = best;
+  plan->threads = static_cast<int>(nvec / (best * 8)); plan->group = plan->threads;
+  plan->grid = static_cast<unsigned>(clusters * best); plan->smem = 0;
+  return true;
+}
+
 // Shared-memory ring plan with a cluster of cs CTAs per row, cs_min <= cs <= cs_max
 // (cs = 1 is the plain TMA ring).  Picks the smallest cluster whose slice leaves room
 // for at least two ring buffers, else the smallest with one.  False if nothing fits.
@@ -554,6 +584,14 @@ akg_status run(const Call& c, const char* name) {
       plan = LaunchPlan{};
     }
   }
+  // Unmasked softmax rows too long for one CTA's registers, held in the registers of a cluster instead
+  // (cluster_mode 3).  Not an automatic choice: one row at a time per CTA leaves the exchange of the pairs
+  // exposed (configuration 4: 150 us with 16 CTAs of 512 threads against 95 us in the two-pass kernel, which
+  // overlaps the second pass of a row with the first pass of the next; 131072 fp32 columns 0.65 against 0.78).
+  if (!planned && vec && forced == V_AUTO && g_tune_cluster_mode.load() == 3) {
+    planned = plan_cluster_reg(c, &plan);
+    if (planned) p.status = status_word_ptr();
+  }
   if (!planned && vec) {
     if (forced == V_AUTO) planned = (g_tune_cluster_mode.load() == 1) ? plan_smem(c, 1, kMaxCluster, &plan)
                                                                       : plan_split(c, &plan);
@@ -569,7 +607,7 @@ akg_status run(const Call& c, const char* name) {
   cudaStream_t stream = static_cast<cudaStream_t>(c.stream);
   // programmatic dependent launch hides the launch gap of back-to-back calls; cluster
   // launches measured slower with it (dependent clusters take SMs from the tail), so not there
-  plan.pdl = (g_tune_pdl.load() == 2 || (plan.variant == V_CLUSTER && g_tune_pdl.load() != 1)) ? 0 : 1;
+  plan.pdl = (g_tune_pdl.load() == 2 || ((plan.variant == V_CLUSTER || plan.cluster > 1) && g_tune_pdl.load() != 1)) ? 0 : 1;
   cudaError_t err;
   switch (c.op) {
     case OP_SOFTMAX: err = launch_op<OP_SOFTMAX>(plan, c.dtype, p, stream); break;
@@ -584,7 +622,8 @@ akg_status run(const Call& c, const char* name) {
   }
   const char* dt = dtype_name(c.dtype);
   if (plan.variant == V_REG)
-    std::snprintf(t_kernel, sizeof t_kernel, "reg<%s,g%d,t%d,v%d%s>", dt, plan.group, plan.threads, plan.vpt,
+    std::snprintf(t_kernel, sizeof t_kernel, "reg<%s,g%d,t%d,v%d%s%s>", dt, plan.group, plan.threads, plan.vpt,
+                  plan.cluster == 16 ? ",cs16" : plan.cluster == 8 ? ",cs8" : plan.cluster == 4 ? ",cs4" : plan.cluster == 2 ? ",cs2" : "",
                   plan.mode == 3 ? (c.dtype == AKG_F32 ? ",flex" : ",packed") : plan.mode == 2 ? ",flex"
                                  : ((plan.stages == 1 && (c.op == OP_LAYERNORM || c.op == OP_RMSNORM)) ? ",full" : ""));
   else if (plan.variant == V_TMA || plan.variant == V_CLUSTER)

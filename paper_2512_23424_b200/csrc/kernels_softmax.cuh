@@ -264,6 +264,45 @@ __global__ void __launch_bounds__(THREADS, kSoftmaxMinBlocks<G, THREADS, VPT>) r
 }
 
 
+// The (maximum, rescaled sum) pairs of the CTAs of a cluster -> the pair of the whole row, in every CTA:
+// each CTA sends its pair to every peer with one 16-byte st.async that counts on the receiver's mbarrier
+// (the scheme of split_kernel; slot and barrier alternate between two sets from row to row), waits for the
+// cluster's pairs with a bounded wait and merges them by a butterfly.  False if the wait ran out.
+struct ClusterPairs {
+  float4 (*inbox)[kMaxCluster];      // [2][kMaxCluster] in shared memory
+  uint64_t* xbar;                    // [2]
+  uint32_t cs, rank, phases;
+  __device__ __forceinline__ void init(float4 (*ib)[kMaxCluster], uint64_t* xb) {
+    inbox = ib; xbar = xb; phases = 0;
+    cs = cluster_size(); rank = cluster_rank();
+    if (cs > 1) {
+      if (threadIdx.x == 0) {
+        mbar_init(smem_addr(&xbar[0]), 1);
+        mbar_init(smem_addr(&xbar[1]), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+      }
+      __syncthreads();
+      cluster_arrive();            // every CTA of the cluster is running before any remote store
+      cluster_wait();
+    }
+  }
+  // every thread of the CTA calls this with the CTA's pair (M, S)
+  __device__ __forceinline__ bool merge(float& M, float& S, int par, float l2e, int* status, unsigned wait_us) {
+    if (threadIdx.x == 0) mbar_expect_tx(smem_addr(&xbar[par]), cs * 16u);
+    if (threadIdx.x < cs) st_async_f32x4(smem_addr(&inbox[par][rank]), smem_addr(&xbar[par]), threadIdx.x, M, S, 0.f, 0.f);
+    const bool ok = mbar_wait_timed<true>(smem_addr(&xbar[par]), (phases >> par) & 1u, status, wait_us);
+    phases ^= 1u << par;
+    const float4 f = inbox[par][threadIdx.x & (cs - 1)];
+    const Stat r = butterfly_merge<OP_SOFTMAX>(Stat{f.x, f.y, 0.f}, static_cast<int>(cs), l2e);
+    M = r.a; S = r.b;
+    return ok;
+  }
+  __device__ __forceinline__ void finish() const {
+    if (cs > 1) { cluster_arrive(); cluster_wait(); }   // nobody leaves while a peer may still send to it
+  }
+};
+
+
 // ------------------------------------------------------------------------------------------------
 // reg_softmax_packed: the softmax pair on unmasked 16-bit rows of exactly blockDim.x * VPT vectors, the
 // row kept PACKED in registers (as reg_norm_packed: four registers per vector, eight vectors per thread in
@@ -284,15 +323,23 @@ __global__ void __launch_bounds__(1024, 1) reg_softmax_packed(const RowParams p)
   static_assert(OP == OP_SOFTMAX || OP == OP_LOG_SOFTMAX, "softmax pair only");
   constexpr int EPV = E::EPV;
   __shared__ float red[2][2][32];
+  __shared__ __align__(16) float4 inbox[2][kMaxCluster];
+  __shared__ __align__(8) uint64_t xbar[2];
   const int G = blockDim.x;
   const int NW = G >> 5;
   const int tg = threadIdx.x;
   const int lane = tg & 31;
   const float l2e = p.l2e;
+  // launched with a cluster of CS CTAs, CTA k holds vectors [k, k + 1) * G * VPT of the row (rows too long
+  // for one CTA's registers: every element is still read from HBM once and never leaves the registers)
+  ClusterPairs cl;
+  cl.init(inbox, xbar);
+  const long long slice = static_cast<long long>(cl.rank) * G * VPT * EPV;
+  bool gave_up = false;
   int parity = 0;
-  for (long long row = blockIdx.x; row < p.rows; row += gridDim.x, parity ^= 1) {
-    const T* xr = reinterpret_cast<const T*>(p.x) + row * p.xs + tg * EPV;
-    T* yr = reinterpret_cast<T*>(p.y) + row * p.ys + tg * EPV;
+  for (long long row = cluster_id(); row < p.rows; row += cluster_count(), parity ^= 1) {
+    const T* xr = reinterpret_cast<const T*>(p.x) + row * p.xs + slice + tg * EPV;
+    T* yr = reinterpret_cast<T*>(p.y) + row * p.ys + slice + tg * EPV;
     uint4 raw[VPT];
 #pragma unroll
     for (int k = 0; k < VPT; ++k) raw[k] = ld_stream(xr + static_cast<long long>(k) * G * EPV);
@@ -334,6 +381,8 @@ __global__ void __launch_bounds__(1024, 1) reg_softmax_packed(const RowParams p)
       const float Ms = (M == kNegInf) ? 0.f : M;
       S = warp_sum(sw * ((mw == M) ? 1.f : exp_diff(mw, Ms, l2e)));      // equal maxima (also +-inf): factor 1
     }
+    if (cl.cs > 1 && !gave_up && !cl.merge(M, S, parity, l2e, p.status, p.wait_us)) gave_up = true;
+    if (gave_up) continue;                                // (no CTA barrier follows in this row: see below)
     const bool dead = (M == kNegInf) && !(S != S);        // only NaN / -inf entries: a NaN row, not a dead one
     const float Mo = (M == kNegInf) ? 0.f : M;
     if (OP == OP_SOFTMAX) {
@@ -367,8 +416,8 @@ __global__ void __launch_bounds__(1024, 1) reg_softmax_packed(const RowParams p)
       }
     }
   }
+  cl.finish();
 }
-
 
 // ------------------------------------------------------------------------------------------------
 // reg_softmax_flex: the fp32 counterpart of reg_softmax_packed - the softmax pair on unmasked fp32 rows of
@@ -384,15 +433,21 @@ __global__ void __launch_bounds__(1024, 1) reg_softmax_flex(const RowParams p) {
   constexpr int EPV = E::EPV;
   constexpr int N = VPT * EPV;
   __shared__ float red[2][2][32];
+  __shared__ __align__(16) float4 inbox[2][kMaxCluster];
+  __shared__ __align__(8) uint64_t xbar[2];
   const int G = blockDim.x;
   const int NW = G >> 5;
   const int tg = threadIdx.x;
   const int lane = tg & 31;
   const float l2e = p.l2e;
+  ClusterPairs cl;                    // a cluster of CS CTAs per row, as in reg_softmax_packed
+  cl.init(inbox, xbar);
+  const long long slice = static_cast<long long>(cl.rank) * G * VPT * EPV;
+  bool gave_up = false;
   int parity = 0;
-  for (long long row = blockIdx.x; row < p.rows; row += gridDim.x, parity ^= 1) {
-    const float* xr = reinterpret_cast<const float*>(p.x) + row * p.xs + tg * EPV;
-    float* yr = reinterpret_cast<float*>(p.y) + row * p.ys + tg * EPV;
+  for (long long row = cluster_id(); row < p.rows; row += cluster_count(), parity ^= 1) {
+    const float* xr = reinterpret_cast<const float*>(p.x) + row * p.xs + slice + tg * EPV;
+    float* yr = reinterpret_cast<float*>(p.y) + row * p.ys + slice + tg * EPV;
     uint4 raw[VPT];
 #pragma unroll
     for (int k = 0; k < VPT; ++k) raw[k] = ld_stream(xr + static_cast<long long>(k) * G * EPV);
@@ -427,6 +482,11 @@ __global__ void __launch_bounds__(1024, 1) reg_softmax_flex(const RowParams p) {
       S = warp_sum(sw * ((mw == M) ? 1.f : exp_diff(mw, Ms, l2e)));      // equal maxima (also +-inf): factor 1
       my_factor = (m_w == M) ? 1.f : exp_diff(m_w, Ms, l2e);
     }
+    if (cl.cs > 1) {
+      if (!gave_up && !cl.merge(M, S, parity, l2e, p.status, p.wait_us)) gave_up = true;
+      my_factor = (m_w == M) ? 1.f : exp_diff(m_w, (M == kNegInf) ? 0.f : M, l2e);
+    }
+    if (gave_up) continue;
     const bool dead = (M == kNegInf) && !(S != S);        // only NaN / -inf entries: a NaN row, not a dead one
     if (OP == OP_SOFTMAX) {
       const float scale = dead ? 0.f : my_factor * __frcp_rn(S);
@@ -449,6 +509,7 @@ __global__ void __launch_bounds__(1024, 1) reg_softmax_flex(const RowParams p) {
       }
     }
   }
+  cl.finish();
 }
 
 }  // namespace akg

@@ -64,6 +64,39 @@ cudaError_t launch_plain(void (*kernel)(KArgs...), const LaunchPlan& plan, unsig
   return cudaLaunchKernelEx(&cfg, kernel, args...);
 }
 
+// A launch of one of the packed / runtime-thread-count register kernels with a cluster of plan.cluster CTAs
+// per row (plan.grid counts CTAs, a multiple of the cluster size).
+template <typename... KArgs, typename... Args>
+cudaError_t launch_reg_cluster(void (*kernel)(KArgs...), const LaunchPlan& plan, cudaStream_t s, Args... args) {
+  static std::mutex mu;
+  static std::map<std::pair<const void*, int>, bool> prepared;     // (kernel, device) -> non-portable sizes allowed
+  int dev = 0;
+  cudaError_t err = cudaGetDevice(&dev);
+  if (err != cudaSuccess) return err;
+  if (plan.cluster > 8) {
+    std::lock_guard<std::mutex> lock(mu);
+    auto key = std::make_pair(reinterpret_cast<const void*>(kernel), dev);
+    if (!prepared[key]) {
+      err = cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+      if (err != cudaSuccess) return err;
+      prepared[key] = true;
+    }
+  }
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = static_cast<unsigned>(plan.cluster);
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.gridDim = dim3(plan.grid);
+  cfg.blockDim = dim3(static_cast<unsigned>(plan.threads));
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = s;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
 // Launch smem_kernel (TMA ring, optionally clustered).  plan.grid == 0 asks for as many
 // clusters as can be co-resident (capped by the number of rows).
 template <int OP, typename T, int THREADS>
@@ -221,8 +254,10 @@ cudaError_t launch_typed(const LaunchPlan& plan, const RowParams& p, cudaStream_
   if (plan.variant == V_REG && plan.mode == 3) {            // runtime thread count, exact fit, 16-bit row kept packed
     if constexpr (OpTraits<OP>::kSoftmaxLike && sizeof(T) == 2) {
       switch (plan.vpt) {
-#define AKG_PACKED_SM_CASE(V_) \
-  case V_: return launch_plain(reg_softmax_packed<OP, T, V_>, plan, plan.grid, plan.threads, 0, s, p);
+#define AKG_PACKED_SM_CASE(V_)                                                                              \
+  case V_:                                                                                                  \
+    if (plan.cluster > 1) return launch_reg_cluster(reg_softmax_packed<OP, T, V_>, plan, s, p);             \
+    return launch_plain(reg_softmax_packed<OP, T, V_>, plan, plan.grid, plan.threads, 0, s, p);
         AKG_PACKED_SM_CASE(2) AKG_PACKED_SM_CASE(3) AKG_PACKED_SM_CASE(4) AKG_PACKED_SM_CASE(5)
         AKG_PACKED_SM_CASE(6) AKG_PACKED_SM_CASE(7) AKG_PACKED_SM_CASE(8)
 #undef AKG_PACKED_SM_CASE
@@ -231,8 +266,10 @@ cudaError_t launch_typed(const LaunchPlan& plan, const RowParams& p, cudaStream_
     }
     if constexpr (OpTraits<OP>::kSoftmaxLike && sizeof(T) == 4) {    // fp32: the same scheme on widened values
       switch (plan.vpt) {
-#define AKG_FLEX_SM_CASE(V_) \
-  case V_: return launch_plain(reg_softmax_flex<OP, V_>, plan, plan.grid, plan.threads, 0, s, p);
+#define AKG_FLEX_SM_CASE(V_)                                                                                \
+  case V_:                                                                                                  \
+    if (plan.cluster > 1) return launch_reg_cluster(reg_softmax_flex<OP, V_>, plan, s, p);                  \
+    return launch_plain(reg_softmax_flex<OP, V_>, plan, plan.grid, plan.threads, 0, s, p);
         AKG_FLEX_SM_CASE(2) AKG_FLEX_SM_CASE(3) AKG_FLEX_SM_CASE(4) AKG_FLEX_SM_CASE(5)
         AKG_FLEX_SM_CASE(6) AKG_FLEX_SM_CASE(7) AKG_FLEX_SM_CASE(8)
 #undef AKG_FLEX_SM_CASE

@@ -137,6 +137,27 @@ def test_sixteen_bit_rows_beyond_2048_vectors_leave_the_register_form(dtype):
     check(dataclasses.replace(wl.make_random("softmax", wl.F32, 300, 32768, seed=354), causal_period=77), ("split", "cs2,"))
 
 
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_softmax_rows_in_the_registers_of_a_cluster(dtype):
+    """cluster_mode 3: an unmasked softmax row held in the registers of a cluster of CTAs (no automatic choice)."""
+    epv = 4 if dtype == wl.F32 else 8
+    try:
+        akg.set_tuning("cluster_mode", 3)
+        for rows, nvec, cs in ((9, 16 * 512 * 8, 16), (70, 4 * 1024 * 8, 4), (5, 2 * 1024 * 8, 2), (300, 8 * 160 * 8, 8)):
+            akg.set_tuning("cluster_size", cs)
+            for op in ("softmax", "log_softmax"):
+                w = wl.make_random(op, dtype, rows, nvec * epv, seed=370 + cs, scale=2.5)
+                x = w.x.copy()
+                if rows > 4:                       # a row without a live entry, and infinities in another
+                    x[1, :] = np.float32(-np.inf) if dtype == wl.F32 else np.uint16(0xFF80)
+                    x[2, 5] = np.float32(-np.inf) if dtype == wl.F32 else np.uint16(0xFF80)
+                check(dataclasses.replace(w, x=x), ("reg<", f"cs{cs},"))
+    finally:
+        akg.set_tuning("cluster_mode", 0)
+        akg.set_tuning("cluster_size", 0)
+    assert akg.device_status() == 0
+
+
 # ---- softmax, a CTA per row: the next row is loaded ahead -------------------------------------------
 
 @pytest.mark.parametrize("dtype", DTYPES)
