@@ -11,12 +11,15 @@ inside `roofline`, one row per benchmark configuration (`per_config`) and per
 widened operator (`next_rows`: non-last axis, fused residual add + normalisation,
 gated activations, arg-max / cumulative operators, column normalisation, fp16
 storage).  Every row is timed three ways over at least 50 launches whatever
---steps is: each launch inside its own CUDA event pair (`us_median`, `us_min`:
-the latency of one kernel), all launches back to back inside one event pair
-(`us_pipelined`: consecutive launches overlap through programmatic dependent
-launch, so this is a throughput), and a few launches each preceded by a 256 MiB
-fill that empties L2 (`us_cold_median`).  `frac` is algorithmic bytes / us_median /
-the measured copy peak.  Beside them the line carries the end-to-end figure with
+--steps is: all launches back to back inside one event pair (`us`, the average
+duration of a launch over a timed region, the protocol of the headline number;
+consecutive launches overlap their ramp-up and drain through programmatic
+dependent launch, so it is a steady-state figure), each launch inside its own CUDA
+event pair (`us_median`, `us_min`: one isolated launch, which includes what the
+event pair itself costs, `event_pair_floor_us`, measured on a one-vector call), and
+a few launches each preceded by a 256 MiB fill that empties L2 (`us_cold_median`).
+`frac` is algorithmic bytes / us / the measured copy peak; `frac_single_launch` the
+same from us_median.  Beside them the line carries the end-to-end figure with
 host buffers and the fp64 CPU oracle's timing.
 
 With N > 1 (launched by torch.distributed.run) every rank runs the same
@@ -293,12 +296,30 @@ def measure_row(obj, nbytes: int, peak: float, launches: int = MIN_LAUNCHES, war
     torch.cuda.synchronize()
     cold_us = np.array([a.elapsed_time(b) for a, b in cold_pairs]) * 1e3
     del flush
-    us = float(np.median(each))
-    return {"us_median": us, "us_min": float(each.min()), "us_pipelined": pipelined * 1e6,
-            "us_cold_median": float(np.median(cold_us)), "launches": launches,
-            "gbs": nbytes / us / 1e3, "frac": nbytes / us / 1e3 / peak,
+    single = float(np.median(each))
+    us = pipelined * 1e6
+    return {"us": us, "gbs": nbytes / us / 1e3, "frac": nbytes / us / 1e3 / peak,
             "frac_nominal": nbytes / us / 1e3 / NOMINAL_HBM_GBS,
-            "frac_pipelined": nbytes / pipelined / 1e9 / peak, "algorithmic_bytes": nbytes}
+            "us_median": single, "us_min": float(each.min()), "frac_single_launch": nbytes / single / 1e3 / peak,
+            "us_cold_median": float(np.median(cold_us)), "launches": launches, "algorithmic_bytes": nbytes}
+
+
+def event_pair_floor_us(launches: int = 200) -> float:
+    """Median time of an event pair around the library's smallest call (one 4-element row): what the
+    per-launch figures (`us_median`) contain besides the kernel's own duration."""
+    import torch
+    from paper_2512_23424_b200 import binding
+    x = torch.zeros((1, 4), device="cuda")
+    call = binding.prepare("rmsnorm", x, torch.empty_like(x), eps=1e-6)
+    for _ in range(10):
+        call.launch()
+    pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(launches)]
+    for a, b in pairs:
+        a.record()
+        call.launch()
+        b.record()
+    torch.cuda.synchronize()
+    return float(np.median([a.elapsed_time(b) for a, b in pairs])) * 1e3
 
 
 def launch_floor_us(launches: int = 256, replays: int = 20) -> float:
@@ -529,7 +550,7 @@ def next_rows_table(peak: float):
         eps = wc.eps
         two = 2 * wc.rows * wc.cols * wc.itemsize
         add(name, _Rotating(torch, n_buf, lambda k: binding.colnorm(cxs[k], cg, cb, eps=eps, out=cys[k], workspace=cws)),
-            two * 3 // 2, bound="hbm, three streams (x read twice)", kernels_per_call=2)
+            two * 3 // 2, bound="hbm, three streams (x read twice)", kernels_per_call=3)
         rows[-1]["frac_two_streams"] = rows[-1]["frac"] * 2 / 3
         del cxs, cys, cx0, wc
     return rows
@@ -600,8 +621,10 @@ def run_ours(args):
                             "frac": gbs_one / peak, "frac_nominal": gbs_one / NOMINAL_HBM_GBS,
                             "peak_kind": peak_kind, "traffic": profiled_traffic(wl.CONFIG_NAMES[HEADLINE]),
                             "algorithmic_bytes": nbytes, "kernel": kernel,
-                            "note": "achieved / frac: the timed region (pipelined launches); per_config[*].frac: "
-                                    "median of single launches, each in its own event pair"}
+                            "note": "achieved / frac: algorithmic bytes / average launch duration over the timed "
+                                    "region (launches back to back), here and in per_config / next_rows; "
+                                    "frac_single_launch: from the median of isolated launches, each in its own "
+                                    "event pair, which costs event_pair_floor_us by itself"}
     # end to end with host buffers
     e2e_k = max(3, min(args.steps, 20))
     t_e2e, h2d, d2h = e2e_steps(w, e2e_k, args.warmup)
@@ -622,20 +645,21 @@ def run_ours(args):
             dwk = DeviceWorkload(wk, pairs_for(wk))
             row = {"workload": wl.CONFIG_NAMES[k]}
             row.update(measure_row(dwk, wk.algorithmic_bytes(), peak, launches=200 if k <= 2 else MIN_LAUNCHES))
-            row.update({"kernel": binding.last_kernel(), "rows_per_s": wk.rows / (row["us_median"] * 1e-6),
+            row.update({"kernel": binding.last_kernel(), "rows_per_s": wk.rows / (row["us"] * 1e-6),
                         "traffic": profiled_traffic(wl.CONFIG_NAMES[k])})
             if k == 1:
-                for key in ("gbs", "frac", "frac_nominal", "frac_pipelined"):
+                for key in ("gbs", "frac", "frac_nominal", "frac_single_launch"):
                     row.pop(key)
                 row["graph_us"] = graph_launch_us(wk, replays=10)
                 row["launch_floor_graph_us"] = launch_floor_us(replays=10)
-                row["note"] = ("latency-bound (0.5 MiB, L2-resident): no bandwidth figure; 'us_pipelined' is paced by "
+                row["note"] = ("latency-bound (0.5 MiB, L2-resident): no bandwidth figure; 'us' is paced by "
                                "the host's launch rate, 'graph_us' is one launch inside a CUDA graph of 256, "
                                "'launch_floor_graph_us' the same for a one-vector call of this library")
             table.append(row)
             del dwk, wk
             torch.cuda.empty_cache()
         line["roofline"]["per_config"] = table
+        line["roofline"]["event_pair_floor_us"] = event_pair_floor_us()
         large = [r for r in table if "frac" in r]
         line["roofline"]["min_frac"] = min(r["frac"] for r in large)
         line["roofline"]["min_frac_workload"] = min(large, key=lambda r: r["frac"])["workload"]

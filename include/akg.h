@@ -322,7 +322,13 @@ akg_status akg_set_variant(akg_variant variant);
  * "host_full_upload" (1 = upload the masked columns of causal rows too),
  * "split_exchange" (two-pass cluster kernel: 1 = partial statistics exchanged under a
  * cluster barrier per row instead of st.async + mbarrier), "split_l2" (its L2 priority
- * scheme: 1 = no "keep" marks, 2 = marks without demotion).  Two keys exist for the test
+ * scheme: 1 = no "keep" marks, 2 = marks without demotion), "reg_flex" (register family:
+ * 1 = the runtime-thread-count normalisation kernel also where a fixed shape fits, 2 = never
+ * a runtime-thread-count kernel, 4 = no eight-vector threads for 16-bit RMSNorm, 5 = never
+ * the packed 16-bit / fp32 runtime-thread-count kernels), "packed_vpt" (vectors per thread of
+ * those kernels, 2 .. 8), "pdl" (1 = programmatic dependent launch also for cluster launches,
+ * 2 = never), "axis_r", "axis_nc", "axis_mode", "axis_lc" (non-last-axis kernels: rows per
+ * thread, column blocks per CTA, lane layout, lanes along the columns).  Two keys exist for the test
  * of the failure path only: "test_wait_us" (limit of the kernels' bounded waits in
  * microseconds; 0 = two seconds) and "test_no_copies" (1 = the ring kernels issue no
  * bulk copy, so that every wait on one runs out and the call reports

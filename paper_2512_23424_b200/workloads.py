@@ -351,6 +351,7 @@ REDUCTION_CONFIGS: Dict[str, tuple] = {
     "cumprod_f32_16384x8192": ("cumprod", F32, 16384, 8192),
     "cumsum_f32_256x262144": ("cumsum", F32, 256, 262144),
     "cumsum_bf16_256x262144": ("cumsum", BF16, 256, 262144),
+    "cumsum_bf16_1048576x256": ("cumsum", BF16, 1048576, 256),
 }
 
 
