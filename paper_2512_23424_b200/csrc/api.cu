@@ -175,7 +175,12 @@ bool plan_reg(const Call& c, LaunchPlan* plan) {
     // the 16-bit softmax pair at 1544 .. 2048 columns: eight vectors per lane spill in the warp form
     // (2048 columns: 69 % softmax, 73 % log-softmax against 86 % and 80 % with a CTA of 128 per row)
     group = threads = 128; vpt = 2;
-  } else if (want_warp && nvec <= 256) {
+  } else if (want_warp && nvec <= 256 &&
+             !(nvec == 192 && !norm_op && c.dtype != AKG_F32 && t_group == 0 && g_tune_reg_general.load() == 0 &&
+               g_tune_reg_flex.load() != 2 && g_tune_reg_flex.load() != 5 &&
+               (c.mask == nullptr || (c.mask->additive == nullptr && !c.mask->causal)))) {
+    // (the unmasked 16-bit softmax pair at 1536 columns goes on to the packed kernel, 64 threads of three vectors:
+    // log-softmax 0.82 -> 0.88, softmax 0.86 -> 0.86 against eight widened vectors per lane here)
     group = 32; threads = 128;
     vpt = pow2_ceil(static_cast<int>((nvec + 31) / 32));
   } else if (t_threads > 0 && t_vpt > 0) {
@@ -417,8 +422,19 @@ bool plan_split(const Call& c, LaunchPlan* plan) {
     // slices of about 4096 vectors (16 per thread) measured best at every row length (65536 fp32
     // columns: 4 CTAs 82 %, 16 CTAs 45 % of the copy rate; 131072: 8 CTAs 84 %, 16 CTAs 64 %);
     // few rows take larger clusters so that there are about two CTAs per SM
+    // (fp32 softmax pair and RMSNorm: slices of 1664 .. 3328 vectors instead.  Measured on 2^26 elements, fraction
+    // of the copy rate with slices of 4000 - 5120 vectors against 2000 - 2560: 32000 columns 0.76 -> 0.89 - 0.92,
+    // 40960: 0.73 -> 0.89 - 0.91, 65536: 0.76 -> 0.88 - 0.93, 81920: 0.75 -> 0.88 - 0.90; 98304 columns, where the
+    // old rule already gave 3072, 0.89 - 0.91.  fp32 LayerNorm and the 16-bit types measured the other way round:
+    // LayerNorm 65536 columns 0.79 with 4096, 0.76 with 2048; bf16 131072 columns 0.67 against 0.60.
+    // What the large slices cost is L2 room: a resident CTA keeps its slice of the current row and of the next
+    // one in L2 between the passes, 592 CTAs x 64 KB x 2 = 76 MB, and the second pass starts to miss (ncu, 65536
+    // columns: L2 hit rate 20 % and 310 MB read from DRAM with 4096-vector slices, 42 % and 269 MB with 2048;
+    // capping the grid at 448 CTAs brought the large slices from 0.77 to 0.85).)
+    const bool small_slices = c.dtype == AKG_F32 && c.op != OP_LAYERNORM;
+    const int64_t min_next = small_slices ? 1664 : 3072;
     int by_len = 1, by_fill = 1;
-    while (by_len < kMaxCluster && nvec / (2 * by_len) >= 3072) by_len *= 2;
+    while (by_len < kMaxCluster && nvec / (2 * by_len) >= min_next) by_len *= 2;
     while (by_fill < kMaxCluster && c.rows * by_fill < 2 * static_cast<int64_t>(sm_count())) by_fill *= 2;
     cs = std::max(by_len, by_fill);
   }

@@ -384,8 +384,14 @@ __device__ __forceinline__ void split_step_use(const RowParams& p, uint4* yc, co
 // word, stops storing and leaves the row loop; its peers run into the same limit one after the
 // other.  All CTAs of a cluster meet at a cluster barrier before they exit, so no partial is ever
 // sent to a CTA that has left.
+#ifndef AKG_SPLIT_MINB16
+#define AKG_SPLIT_MINB16 4
+#endif
+template <typename T, int THREADS> constexpr int kSplitMinBlocks =
+    (sizeof(T) == 2 && THREADS == 256) ? AKG_SPLIT_MINB16 : ((1024 / THREADS) > 0 ? (1024 / THREADS) : 1);
+
 template <int OP, typename T, int THREADS>
-__global__ void __launch_bounds__(THREADS, (1024 / THREADS) > 0 ? (1024 / THREADS) : 1)
+__global__ void __launch_bounds__(THREADS, kSplitMinBlocks<T, THREADS>)
 split_kernel(const RowParams p, const int slice_vecs, const int xmode, const int l2mode) {
   pdl_prologue();
   using E = Elem<T>;
