@@ -311,6 +311,46 @@ template <int OP> __device__ __forceinline__ Stat stat_merge(const Stat& x, cons
   return r;
 }
 
+// 1 / sqrt(a): hardware approximation plus one Newton step (about 1 ulp).
+__device__ __forceinline__ float rsqrt_refined(float a) {
+  float r = rsqrtf(a);
+  if (a > 0.f && a < __int_as_float(0x7f800000)) r = r * (1.5f - 0.5f * a * r * r);
+  return r;
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int m = 16; m >= 1; m >>= 1) v += __shfl_xor_sync(0xffffffffu, v, m);
+  return v;
+}
+
+// Sum of n values (n a power of two, at most 32) held one per lane, lane l holding entry l mod n; every
+// lane gets the same bits (an xor butterfly adds the same pairs in every lane).
+__device__ __forceinline__ float lanes_sum(float v, int n) {
+  for (int m = 1; m < n; m <<= 1) v += __shfl_xor_sync(0xffffffffu, v, m);
+  return v;
+}
+
+// (count, mean, M2) of n partial statistics held one per lane (as lanes_sum), all at once instead of by
+// pairwise Chan merges: N = sum n_i, mean = ref + sum n_i (mean_i - ref) / N, M2 = sum (M2_i + n_i (mean_i - mean)^2),
+// ref being the first entry's mean: the sums run over differences of means, so the error of the merged mean
+// scales with the spread of the partial means, not with their magnitude (as in the pairwise update).
+// Three butterflies of sums replace log2 n merges with a division each; the per-row reductions of the
+// two-pass cluster kernel were 590 warp instructions per warp and row-slice with pairwise merges, two fifths
+// of all its LayerNorm instructions (fp32, 65536 columns).
+template <int FULL_WARP> __device__ __forceinline__ Stat layernorm_merge_lanes(const Stat& s, int n) {
+  const int first = FULL_WARP ? 0 : static_cast<int>(threadIdx.x & 31u & ~static_cast<unsigned>(n - 1));
+  const float ref = __shfl_sync(0xffffffffu, s.b, first);
+  const float w = s.a * (s.b - ref);
+  const float cnt = FULL_WARP ? warp_sum(s.a) : lanes_sum(s.a, n);
+  const float sum = FULL_WARP ? warp_sum(w) : lanes_sum(w, n);
+  // correctly rounded division: an error of the mean is an error of every output
+  const float mean = (cnt > 0.f) ? ref + __fdiv_rn(sum, cnt) : 0.f;
+  const float d = s.b - mean;
+  const float m2 = fmaf(s.a * d, d, s.c);
+  return Stat{cnt, mean, FULL_WARP ? warp_sum(m2) : lanes_sum(m2, n)};
+}
+
 template <int OP> __device__ __forceinline__ Stat stat_shfl_xor(const Stat& s, int lane_mask) {
   Stat r;
   r.a = __shfl_xor_sync(0xffffffffu, s.a, lane_mask);
@@ -320,6 +360,8 @@ template <int OP> __device__ __forceinline__ Stat stat_shfl_xor(const Stat& s, i
 }
 
 template <int OP> __device__ __forceinline__ Stat warp_reduce(Stat s, float l2e = kLog2e) {
+  if constexpr (OP == OP_LAYERNORM) return layernorm_merge_lanes<1>(s, 32);
+  if constexpr (OP == OP_RMSNORM) return Stat{warp_sum(s.a), 0.f, 0.f};
 #pragma unroll
   for (int m = 16; m >= 1; m >>= 1) s = stat_merge<OP>(s, stat_shfl_xor<OP>(s, m), l2e);
   return s;
@@ -330,10 +372,14 @@ template <int OP> __device__ __forceinline__ Stat warp_reduce(Stat s, float l2e 
 // lane) in that order, so every lane ends with the same bits; a serial merge of 16 entries is a chain of 15
 // dependent merges (two exponentials each for the softmax pair), this one of four.
 template <int OP> __device__ __forceinline__ Stat butterfly_merge(Stat s, int n, float l2e = kLog2e) {
+  if constexpr (OP == OP_LAYERNORM) return layernorm_merge_lanes<0>(s, n);
+  if constexpr (OP == OP_RMSNORM) return Stat{lanes_sum(s.a, n), 0.f, 0.f};
   const int lane = threadIdx.x & 31;
   for (int k = 1; k < n; k <<= 1) {
     const Stat o = stat_shfl_xor<OP>(s, k);
-    s = (lane & k) ? stat_merge<OP>(o, s, l2e) : stat_merge<OP>(s, o, l2e);
+    const bool upper = (lane & k) != 0;                    // the operands are ordered, the merge is evaluated once
+    const Stat lo{upper ? o.a : s.a, upper ? o.b : s.b, 0.f}, hi{upper ? s.a : o.a, upper ? s.b : o.b, 0.f};
+    s = stat_merge<OP>(lo, hi, l2e);
   }
   return s;
 }
@@ -377,10 +423,10 @@ template <int OP> __device__ __forceinline__ RowScalars finalize(const Stat& s, 
     r.q = r.dead ? 0.f : logf(s.b);
   } else if (OP == OP_LAYERNORM) {
     r.p = s.b;
-    r.q = 1.0f / sqrtf(s.c / static_cast<float>(cols) + eps);
+    r.q = rsqrt_refined(fmaf(s.c, __frcp_rn(static_cast<float>(cols)), eps));
   } else {
     r.p = 0.f;
-    r.q = 1.0f / sqrtf(s.a / static_cast<float>(cols) + eps);
+    r.q = rsqrt_refined(fmaf(s.a, __frcp_rn(static_cast<float>(cols)), eps));
   }
   return r;
 }

@@ -20,18 +20,6 @@ namespace akg {
 // at most 64 registers per thread (occupancy, not instruction count, bounds them next).
 template <int THREADS> constexpr int kRegMinBlocks = (1024 / THREADS) > 0 ? (1024 / THREADS) : 1;
 
-// 1 / sqrt(a): hardware approximation plus one Newton step (about 1 ulp).
-__device__ __forceinline__ float rsqrt_refined(float a) {
-  float r = rsqrtf(a);
-  if (a > 0.f && a < __int_as_float(0x7f800000)) r = r * (1.5f - 0.5f * a * r * r);
-  return r;
-}
-
-__device__ __forceinline__ float warp_sum(float v) {
-#pragma unroll
-  for (int m = 16; m >= 1; m >>= 1) v += __shfl_xor_sync(0xffffffffu, v, m);
-  return v;
-}
 __device__ __forceinline__ float warp_max(float v) {
 #pragma unroll
   for (int m = 16; m >= 1; m >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, m));
