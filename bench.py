@@ -15,8 +15,8 @@ storage).  Every row is timed three ways over at least 50 launches whatever
 duration of a launch over a timed region, the protocol of the headline number;
 consecutive launches overlap their ramp-up and drain through programmatic
 dependent launch, so it is a steady-state figure), each launch inside its own CUDA
-event pair (`us_median`, `us_min`: one isolated launch, which includes what the
-event pair itself costs, `event_pair_floor_us`, measured on a one-vector call), and
+event pair (`us_median`, `us_min`: one isolated launch with its ramp-up and drain
+exposed), and
 a few launches each preceded by a 256 MiB fill that empties L2 (`us_cold_median`).
 `frac` is algorithmic bytes / us / the measured copy peak; `frac_single_launch` the
 same from us_median.  Beside them the line carries the end-to-end figure with
@@ -302,24 +302,6 @@ def measure_row(obj, nbytes: int, peak: float, launches: int = MIN_LAUNCHES, war
             "frac_nominal": nbytes / us / 1e3 / NOMINAL_HBM_GBS,
             "us_median": single, "us_min": float(each.min()), "frac_single_launch": nbytes / single / 1e3 / peak,
             "us_cold_median": float(np.median(cold_us)), "launches": launches, "algorithmic_bytes": nbytes}
-
-
-def event_pair_floor_us(launches: int = 200) -> float:
-    """Median time of an event pair around the library's smallest call (one 4-element row): what the
-    per-launch figures (`us_median`) contain besides the kernel's own duration."""
-    import torch
-    from paper_2512_23424_b200 import binding
-    x = torch.zeros((1, 4), device="cuda")
-    call = binding.prepare("rmsnorm", x, torch.empty_like(x), eps=1e-6)
-    for _ in range(10):
-        call.launch()
-    pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(launches)]
-    for a, b in pairs:
-        a.record()
-        call.launch()
-        b.record()
-    torch.cuda.synchronize()
-    return float(np.median([a.elapsed_time(b) for a, b in pairs])) * 1e3
 
 
 def launch_floor_us(launches: int = 256, replays: int = 20) -> float:
@@ -624,7 +606,7 @@ def run_ours(args):
                             "note": "achieved / frac: algorithmic bytes / average launch duration over the timed "
                                     "region (launches back to back), here and in per_config / next_rows; "
                                     "frac_single_launch: from the median of isolated launches, each in its own "
-                                    "event pair, which costs event_pair_floor_us by itself"}
+                                    "event pair (ramp-up and drain of the grid exposed)"}
     # end to end with host buffers
     e2e_k = max(3, min(args.steps, 20))
     t_e2e, h2d, d2h = e2e_steps(w, e2e_k, args.warmup)
@@ -659,7 +641,6 @@ def run_ours(args):
             del dwk, wk
             torch.cuda.empty_cache()
         line["roofline"]["per_config"] = table
-        line["roofline"]["event_pair_floor_us"] = event_pair_floor_us()
         large = [r for r in table if "frac" in r]
         line["roofline"]["min_frac"] = min(r["frac"] for r in large)
         line["roofline"]["min_frac_workload"] = min(large, key=lambda r: r["frac"])["workload"]
