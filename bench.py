@@ -731,6 +731,9 @@ def run_profile(args):
     if args.profile_next:
         # one of the arg-max / cumulative / column-normalisation rows (workloads.REDUCTION_CONFIGS, COLNORM_CONFIGS)
         name = args.profile_next
+        for item in filter(None, args.tune.split(",")):
+            key, _, val = item.partition("=")
+            binding.set_tuning(key, int(val))
         if name in wl.REDUCTION_CONFIGS:
             wr = wl.make_reduction(name, rows=args.profile_rows)
             fn = getattr(binding, wr.op)

@@ -432,7 +432,10 @@ bool plan_split(const Call& c, LaunchPlan* plan) {
     // columns: L2 hit rate 20 % and 310 MB read from DRAM with 4096-vector slices, 42 % and 269 MB with 2048;
     // capping the grid at 448 CTAs brought the large slices from 0.77 to 0.85).)
     const bool small_slices = c.dtype == AKG_F32 && c.op != OP_LAYERNORM;
-    const int64_t min_next = small_slices ? 1664 : 3072;
+    // (16-bit log-softmax and normalisations: 2300 .. 4600, which moves 81920 and 151936 columns to half the slice:
+    // bf16 81920 columns log-softmax 0.69 -> 0.73, LayerNorm 0.63 -> 0.71, RMSNorm 0.69 -> 0.80; 151936: 0.67 -> 0.71,
+    // 0.59 -> 0.66, 0.65 -> 0.73; the 16-bit softmax measured level or worse with the smaller slices)
+    const int64_t min_next = small_slices ? 1664 : ((c.dtype != AKG_F32 && c.op != OP_SOFTMAX) ? 2300 : 3072);
     int by_len = 1, by_fill = 1;
     while (by_len < kMaxCluster && nvec / (2 * by_len) >= min_next) by_len *= 2;
     while (by_fill < kMaxCluster && c.rows * by_fill < 2 * static_cast<int64_t>(sm_count())) by_fill *= 2;

@@ -123,9 +123,20 @@ __device__ __forceinline__ uint4 ld_stream(const void* p) {
                : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
   return v;
 }
+#ifndef AKG_ST_MODE
+#define AKG_ST_MODE 0
+#endif
 __device__ __forceinline__ void st_stream(void* p, const uint4& v) {
+#if AKG_ST_MODE == 1
+  asm volatile("st.global.v4.u32 [%0], {%1, %2, %3, %4};"
+               :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+#elif AKG_ST_MODE == 2
+  asm volatile("st.global.cg.v4.u32 [%0], {%1, %2, %3, %4};"
+               :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+#else
   asm volatile("st.global.cs.v4.u32 [%0], {%1, %2, %3, %4};"
                :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+#endif
 }
 // read-only, cached (gamma / beta / weight are reused by every row)
 __device__ __forceinline__ uint4 ld_cached(const void* p) {
