@@ -586,14 +586,16 @@ akg_status run(const Call& c, const char* name) {
                            ((norm_call && c.dtype != AKG_F32) ||
                             (!norm_call && (c.mask == nullptr || (c.mask->additive == nullptr && !c.mask->causal)))) &&
                            row_vecs % 8 == 0 && (row_vecs / 8) % 32 == 0 && g_tune_reg_general.load() == 0 &&
-                           !(c.dtype == AKG_F32 && row_vecs > 4096 && row_vecs < 6144) &&     // see long_row
+                           !(c.dtype == AKG_F32 && row_vecs > 4096) &&                        // see long_row
                            g_tune_reg_flex.load() != 2 && g_tune_reg_flex.load() != 5 &&
                            // a CTA per row needs rows for about a full wave of threads; fewer rows are cut into
                            // slices by the two-pass cluster kernel
                            c.rows * (row_vecs / 8) >= static_cast<int64_t>(sm_count()) * 1024;
   // (fp32 rows of 4097 .. 6143 vectors would take one CTA of 544 .. 736 fat threads per SM: 20480 columns measured
   // 0.81 - 0.83 there and 0.91 - 0.93 in the two-pass kernel for the softmax pair and RMSNorm; LayerNorm 0.82 against
-  // 0.79 and stays; from 6144 vectors on the register kernels are level or ahead)
+  // 0.79 and stays; from 6144 vectors on RMSNorm is level in both; the fp32 softmax pair, with its slices sized
+  // for L2, is level at 24576 columns and ahead beyond - 28672: 0.91 against 0.90, 32768: 0.95 against 0.92 - so
+  // every fp32 softmax row beyond 4096 vectors takes the two-pass kernel)
   const bool thin_cta = c.dtype == AKG_F32 && row_vecs > 4096 && row_vecs < 6144 && c.op != OP_LAYERNORM &&
                         g_tune_reg_flex.load() != 1;
   const bool long_row = forced == V_AUTO && g_tune_cluster_mode.load() != 1 && !packed_fits &&
