@@ -438,6 +438,7 @@ bool plan_split(const Call& c, LaunchPlan* plan) {
     const int64_t min_next = small_slices ? 1664 : ((c.dtype != AKG_F32 && c.op != OP_SOFTMAX) ? 2300 : 3072);
     int by_len = 1, by_fill = 1;
     while (by_len < kMaxCluster && nvec / (2 * by_len) >= min_next) by_len *= 2;
+    if (c.dtype == AKG_F32 && c.op == OP_LAYERNORM && nvec > 4096 && nvec <= 8192) by_len = 2;   // see run()
     while (by_fill < kMaxCluster && c.rows * by_fill < 2 * static_cast<int64_t>(sm_count())) by_fill *= 2;
     cs = std::max(by_len, by_fill);
   }
@@ -598,8 +599,13 @@ akg_status run(const Call& c, const char* name) {
   // every fp32 softmax row beyond 4096 vectors takes the two-pass kernel)
   const bool thin_cta = c.dtype == AKG_F32 && row_vecs > 4096 && row_vecs < 6144 && c.op != OP_LAYERNORM &&
                         g_tune_reg_flex.load() != 1;
+  // (fp32 LayerNorm rows of 4097 .. 8192 vectors, given rows enough to matter: two CTAs of a cluster per row
+  // measured 0.83 - 0.87 against 0.79 - 0.83 in one CTA of 576 - 1024 threads; with a few hundred rows the
+  // register kernel stays ahead, 0.49 - 0.51 against 0.41 - 0.50)
+  const bool ln_two_ctas = c.dtype == AKG_F32 && c.op == OP_LAYERNORM && row_vecs > 4096 && row_vecs <= 8192 &&
+                           c.rows >= 1024 && g_tune_reg_flex.load() != 1;
   const bool long_row = forced == V_AUTO && g_tune_cluster_mode.load() != 1 && !packed_fits &&
-                        ((c.dtype != AKG_F32 && row_vecs > 2048) || thin_cta ||
+                        ((c.dtype != AKG_F32 && row_vecs > 2048) || thin_cta || ln_two_ctas ||
                          (c.dtype == AKG_F32 && row_vecs > 4096 && (c.op == OP_SOFTMAX || c.op == OP_LOG_SOFTMAX)));
   if (!planned && (forced == V_AUTO || forced == V_REG) && vec && !long_row) {
     planned = plan_reg(c, &plan);

@@ -134,6 +134,12 @@ def test_sixteen_bit_rows_beyond_2048_vectors_leave_the_register_form(dtype):
     # the fp32 normalisations stay in registers while the row is an exact fit, ragged rows do not
     check(wl.make_random("rmsnorm", wl.F32, 300, 32768, seed=352), ("reg", "flex"))
     check(wl.make_random("layernorm", wl.F32, 300, 32000, seed=353), ("split",))
+    # ... and, with a thousand rows or more, leave one CTA of 576 - 1024 threads for a cluster of two
+    check(wl.make_random("layernorm", wl.F32, 1100, 20480, seed=359, loc=0.5), ("split", "cs2,"), rows=list(range(0, 1100, 37)))
+    check(wl.make_random("layernorm", wl.F32, 300, 20480, seed=359, loc=0.5), ("reg", "flex"))
+    # fp32 softmax pair and RMSNorm rows of 4097 .. 6143 vectors: no thin CTA
+    check(wl.make_random("rmsnorm", wl.F32, 300, 20480, seed=360), ("split", "cs2,"))
+    check(wl.make_random("rmsnorm", wl.F32, 300, 24576, seed=360), ("reg", "flex"))
     # the fp32 softmax pair leaves the registers beyond 4096 vectors, masked or not (slices of about 2048 vectors)
     check(wl.make_random("softmax", wl.F32, 300, 32768, seed=354), ("split", "cs4,"))
     check(wl.make_random("log_softmax", wl.F32, 300, 16384, seed=357), ("reg<", "t512,v8,flex"))
