@@ -607,6 +607,16 @@ akg_status run(const Call& c, const char* name) {
   const bool long_row = forced == V_AUTO && g_tune_cluster_mode.load() != 1 && !packed_fits &&
                         ((c.dtype != AKG_F32 && row_vecs > 2048) || thin_cta || ln_two_ctas ||
                          (c.dtype == AKG_F32 && row_vecs > 4096 && (c.op == OP_SOFTMAX || c.op == OP_LOG_SOFTMAX)));
+  // Unmasked softmax rows too long for one CTA's registers, held in the registers of a cluster instead
+  // (cluster_mode 3).  Not an automatic choice: one row at a time per CTA leaves the exchange of the pairs
+  // exposed (configuration 4: 150 us with 16 CTAs of 512 threads against 95 us in the two-pass kernel, which
+  // overlaps the second pass of a row with the first pass of the next; 131072 fp32 columns 0.65 against 0.78).
+  // (asked for with a forced cluster size, it also takes rows that one CTA could hold)
+  if (!planned && vec && forced == V_AUTO && g_tune_cluster_mode.load() == 3 &&
+      (g_tune_cluster_size.load() > 1 || long_row || row_vecs > 8192)) {
+    planned = plan_cluster_reg(c, &plan);
+    if (planned) p.status = status_word_ptr();
+  }
   if (!planned && (forced == V_AUTO || forced == V_REG) && vec && !long_row) {
     planned = plan_reg(c, &plan);
     // fp32 normalisation rows beyond 4096 vectors stay in registers only as an exact fit (the ragged
@@ -616,14 +626,6 @@ akg_status run(const Call& c, const char* name) {
       planned = false;
       plan = LaunchPlan{};
     }
-  }
-  // Unmasked softmax rows too long for one CTA's registers, held in the registers of a cluster instead
-  // (cluster_mode 3).  Not an automatic choice: one row at a time per CTA leaves the exchange of the pairs
-  // exposed (configuration 4: 150 us with 16 CTAs of 512 threads against 95 us in the two-pass kernel, which
-  // overlaps the second pass of a row with the first pass of the next; 131072 fp32 columns 0.65 against 0.78).
-  if (!planned && vec && forced == V_AUTO && g_tune_cluster_mode.load() == 3) {
-    planned = plan_cluster_reg(c, &plan);
-    if (planned) p.status = status_word_ptr();
   }
   if (!planned && vec) {
     if (forced == V_AUTO) planned = (g_tune_cluster_mode.load() == 1) ? plan_smem(c, 1, kMaxCluster, &plan)
