@@ -177,6 +177,19 @@ __device__ __forceinline__ uint4 split_apply_plain(const RowParams& p, const Row
       return make_uint4(out[0], out[1], out[2], out[3]);
     }
   }
+  if constexpr (OP == OP_RMSNORM && sizeof(T) == 4) {
+    // fp32 RMSNorm with its weight present: no defaults to set up and overwrite (the generic form below spends
+    // about two instructions per element on them; 65536 columns 0.93 -> 0.96 of the copy rate).  The same
+    // shortcut made fp32 LayerNorm slower (0.82 -> 0.72: its gamma and beta loads then sit between the streaming
+    // stores, which the compiler may not move them across), so LayerNorm keeps the generic form.
+    if (p.gamma != nullptr) {
+      const uint4 gw = ld_cached(reinterpret_cast<const T*>(p.gamma) + c0);
+      return make_uint4(__float_as_uint(__uint_as_float(raw.x) * rs.q * __uint_as_float(gw.x)),
+                        __float_as_uint(__uint_as_float(raw.y) * rs.q * __uint_as_float(gw.y)),
+                        __float_as_uint(__uint_as_float(raw.z) * rs.q * __uint_as_float(gw.z)),
+                        __float_as_uint(__uint_as_float(raw.w) * rs.q * __uint_as_float(gw.w)));
+    }
+  }
   float z[EPV], ga[EPV], be[EPV], o[EPV];
   E::unpack(raw, z);
 #pragma unroll
