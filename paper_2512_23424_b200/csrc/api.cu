@@ -435,9 +435,17 @@ bool plan_split(const Call& c, LaunchPlan* plan) {
     // (16-bit log-softmax and normalisations: 2300 .. 4600, which moves 81920 and 151936 columns to half the slice:
     // bf16 81920 columns log-softmax 0.69 -> 0.73, LayerNorm 0.63 -> 0.71, RMSNorm 0.69 -> 0.80; 151936: 0.67 -> 0.71,
     // 0.59 -> 0.66, 0.65 -> 0.73; the 16-bit softmax measured level or worse with the smaller slices)
-    const int64_t min_next = small_slices ? 1664 : ((c.dtype != AKG_F32 && c.op != OP_SOFTMAX) ? 2300 : 3072);
+    // 16-bit RMSNorm and log-softmax take the small slices as well (bf16 131072 columns: RMSNorm 0.75 -> 0.80,
+    // log-softmax 0.71 -> 0.74; 32000 columns log-softmax 0.73 -> 0.76), but no 16-bit operator gains from a
+    // cluster of 16 with slices below 3072 vectors (only 31 such clusters fit the GPU, 496 of its 592 CTA slots:
+    // bf16 262144 columns log-softmax 0.66 with 16 CTAs of 2048 vectors against 0.71 with 8 of 4096).
+    const bool sixteen = c.dtype != AKG_F32;
+    const int64_t min_next = (small_slices || (sixteen && (c.op == OP_RMSNORM || c.op == OP_LOG_SOFTMAX))) ? 1664
+                             : ((sixteen && c.op == OP_LAYERNORM) ? 2300 : 3072);
     int by_len = 1, by_fill = 1;
-    while (by_len < kMaxCluster && nvec / (2 * by_len) >= min_next) by_len *= 2;
+    while (by_len < kMaxCluster &&
+           nvec / (2 * by_len) >= ((sixteen && 2 * by_len == kMaxCluster) ? std::max<int64_t>(min_next, 3072) : min_next))
+      by_len *= 2;
     if (c.dtype == AKG_F32 && c.op == OP_LAYERNORM && nvec > 4096 && nvec <= 8192) by_len = 2;   // see run()
     while (by_fill < kMaxCluster && c.rows * by_fill < 2 * static_cast<int64_t>(sm_count())) by_fill *= 2;
     cs = std::max(by_len, by_fill);

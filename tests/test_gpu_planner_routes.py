@@ -89,8 +89,10 @@ def test_long_rows_cluster_size_follows_length(dtype):
         for op in ("softmax", "log_softmax", "layernorm", "rmsnorm"):
             if dtype == wl.F32 and cols // epv <= 8192 and op in ("layernorm", "rmsnorm"):
                 continue                       # exact fits of fp32 normalisations stay in registers
-            # the fp32 softmax pair and RMSNorm take slices of about 2048 vectors: twice the CTAs by length
-            by_length = rows >= 300 and dtype == wl.F32 and op != "layernorm"
+            # the fp32 softmax pair and RMSNorm take slices of about 2048 vectors: twice the CTAs by length;
+            # so do the 16-bit RMSNorm and log-softmax
+            by_length = rows >= 300 and ((dtype == wl.F32 and op != "layernorm") or
+                                         (dtype != wl.F32 and op in ("rmsnorm", "log_softmax")))
             w = wl.make_random(op, dtype, rows, cols, seed=330 + cs, scale=2.0)
             check(w, ("split", f"cs{2 * cs if by_length else cs},"))
 
