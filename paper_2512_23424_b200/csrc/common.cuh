@@ -334,6 +334,30 @@ __device__ __forceinline__ float lanes_sum(float v, int n) {
   return v;
 }
 
+__device__ __forceinline__ float lanes_max(float v, int n) {
+  for (int m = 1; m < n; m <<= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, m));
+  return v;
+}
+
+// (maximum, rescaled sum) of n softmax partials held one per lane: the maximum first, then every partial
+// rescaled once, then the sum - two butterflies and one exponential per lane instead of log2 n ordered merges
+// with two exponentials each (those merges were 0.4 special-function and 2.3 instructions in all per element of
+// the two-pass kernel on configuration 4, on the path between a row's two passes).  Equal maxima (also both
+// -inf, or both +inf) take factor 1, so that no inf - inf is formed; a NaN maximum cannot occur (fmaxf drops
+// NaN), a NaN partial sum makes the row NaN.
+template <int FULL_WARP> __device__ __forceinline__ Stat softmax_merge_lanes(const Stat& s, int n, float l2e) {
+  float M = s.a;
+  if (FULL_WARP) {
+#pragma unroll
+    for (int m = 16; m >= 1; m >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, m));
+  } else {
+    M = lanes_max(M, n);
+  }
+  const float Ms = (M == kNegInf) ? 0.f : M;
+  const float w = s.b * ((s.a == M) ? 1.f : exp_diff(s.a, Ms, l2e));
+  return Stat{M, FULL_WARP ? warp_sum(w) : lanes_sum(w, n), 0.f};
+}
+
 // (count, mean, M2) of n partial statistics held one per lane (as lanes_sum), all at once instead of by
 // pairwise Chan merges: N = sum n_i, mean = ref + sum n_i (mean_i - ref) / N, M2 = sum (M2_i + n_i (mean_i - mean)^2),
 // ref being the first entry's mean: the sums run over differences of means, so the error of the merged mean
@@ -366,6 +390,7 @@ template <int OP> __device__ __forceinline__ Stat stat_shfl_xor(const Stat& s, i
 template <int OP> __device__ __forceinline__ Stat warp_reduce(Stat s, float l2e = kLog2e) {
   if constexpr (OP == OP_LAYERNORM) return layernorm_merge_lanes<1>(s, 32);
   if constexpr (OP == OP_RMSNORM) return Stat{warp_sum(s.a), 0.f, 0.f};
+  if constexpr (OpTraits<OP>::kSoftmaxLike) return softmax_merge_lanes<1>(s, 32, l2e);
 #pragma unroll
   for (int m = 16; m >= 1; m >>= 1) s = stat_merge<OP>(s, stat_shfl_xor<OP>(s, m), l2e);
   return s;
@@ -378,6 +403,7 @@ template <int OP> __device__ __forceinline__ Stat warp_reduce(Stat s, float l2e 
 template <int OP> __device__ __forceinline__ Stat butterfly_merge(Stat s, int n, float l2e = kLog2e) {
   if constexpr (OP == OP_LAYERNORM) return layernorm_merge_lanes<0>(s, n);
   if constexpr (OP == OP_RMSNORM) return Stat{lanes_sum(s.a, n), 0.f, 0.f};
+  if constexpr (OpTraits<OP>::kSoftmaxLike) return softmax_merge_lanes<0>(s, n, l2e);
   const int lane = threadIdx.x & 31;
   for (int k = 1; k < n; k <<= 1) {
     const Stat o = stat_shfl_xor<OP>(s, k);
