@@ -82,8 +82,9 @@ template <typename T> struct AxisRaw<T, 0> {
 constexpr int kAxisMaxWarps = 16;
 
 // Shared memory of one CTA in floats: partials [KS][nf * nc][32 W], then scalars [2][nc][32 W].
+constexpr int kAxisAffineFloats = 2 * kAxisMaxWarps * 8;     // gamma and beta of up to 16 warp-rows x 8 rows
 __host__ __device__ constexpr unsigned axis_reg_smem_floats(int ks, int nf, int nc, int w) {
-  return nf > 1 ? static_cast<unsigned>((ks * nf * nc + 2 * nc) * 32 * w) : 0u;
+  return nf > 1 ? static_cast<unsigned>((ks * nf * nc + 2 * nc) * 32 * w + kAxisAffineFloats) : 0u;
 }
 
 // The two scalars of a column from its merged statistics:
@@ -213,10 +214,23 @@ __device__ __forceinline__ void axis_reg_load(const T* px, long long xstep, bool
 #pragma unroll
     for (int r = 1; r < R; ++r) {
       if (FULL || r < nt) {
-        float v[W];
-        A::unpack(raw[r], v);
+        if constexpr (MODE == 1 && sizeof(T) == 2) {
+          // packed row: the stored values enter the subtraction as they are (Elem::sub_wide), no unpack
+          const uint32_t ws[4] = {raw[r].x, raw[r].y, raw[r].z, raw[r].w};
 #pragma unroll
-        for (int j = 0; j < W; ++j) { const float d = v[j] - k[j]; sa[j] += d; sb[j] = fmaf(d, d, sb[j]); }
+          for (int i = 0; i < 4; ++i) {
+            unsigned short h0, h1;
+            halves(ws[i], h0, h1);
+            const float d0 = Elem<T>::sub_wide(h0, k[2 * i]), d1 = Elem<T>::sub_wide(h1, k[2 * i + 1]);
+            sa[2 * i] += d0; sb[2 * i] = fmaf(d0, d0, sb[2 * i]);
+            sa[2 * i + 1] += d1; sb[2 * i + 1] = fmaf(d1, d1, sb[2 * i + 1]);
+          }
+        } else {
+          float v[W];
+          A::unpack(raw[r], v);
+#pragma unroll
+          for (int j = 0; j < W; ++j) { const float d = v[j] - k[j]; sa[j] += d; sb[j] = fmaf(d, d, sb[j]); }
+        }
       }
     }
     const float inv_nt = FULL ? (1.0f / R) : ((nt > 0) ? __frcp_rn(static_cast<float>(nt)) : 0.f);
@@ -265,7 +279,7 @@ __device__ __forceinline__ void axis_reg_load(const T* px, long long xstep, bool
 // (cp, cq) and store them.  gp / bp point at gamma[wf] / beta[wf] (or are nullptr).
 template <int OP, typename T, int MODE, int R, bool FULL>
 __device__ __forceinline__ void axis_reg_store(T* py, long long ystep, bool active, int nt, int nf,
-                                               const T* gp, const T* bp,
+                                               const T* gp, const T* bp, const float* gs, const float* bs,
                                                const typename AxisRaw<T, MODE>::Raw (&raw)[R],
                                                const float (&cp)[AxisRaw<T, MODE>::W],
                                                const float (&cq)[AxisRaw<T, MODE>::W]) {
@@ -284,8 +298,13 @@ __device__ __forceinline__ void axis_reg_store(T* py, long long ystep, bool acti
     if (FULL || (active && r < nt)) {
       float g = 1.f, be = 0.f;
       if (!OpTraits<OP>::kSoftmaxLike) {
-        if (gp != nullptr) g = E::load1(gp, r * nf);
-        if (OP == OP_LAYERNORM && bp != nullptr) be = E::load1(bp, r * nf);
+        if (gs != nullptr) {                               // staged once per CTA: one shared load, constant offset
+          g = gs[r];
+          if (OP == OP_LAYERNORM) be = bs[r];
+        } else {
+          if (gp != nullptr) g = E::load1(gp, r * nf);
+          if (OP == OP_LAYERNORM && bp != nullptr) be = E::load1(bp, r * nf);
+        }
       }
       float v[W];
       A::unpack(raw[r], v);
@@ -333,6 +352,23 @@ axis_reg_kernel(const AxisParams p, const unsigned strips_per_outer, const int n
   const long long xstep = p.xsf * nf, ystep = p.ysf * nf;
   const T* gp = (!SM && p.gamma != nullptr) ? reinterpret_cast<const T*>(p.gamma) + wf : nullptr;
   const T* bp = (OP == OP_LAYERNORM && p.beta != nullptr) ? reinterpret_cast<const T*>(p.beta) + wf : nullptr;
+  // The affine scalars of the reduced axis are the same for every strip: with several warp-rows they are staged
+  // once per CTA in shared memory as floats, [warp-row][row], so that the store phase reads them with one shared
+  // load at a constant offset (a 16-bit global load with a 64-bit index each cost five instructions per row and
+  // scalar: one instruction per element of the 16-bit LayerNorm).  The strip loop's first barrier orders them.
+  float* aff = fin1 + nc * CW;                              // [2][nf * R]
+  const float* gs = nullptr;
+  const float* bs = nullptr;
+  if (!SM && nf > 1 && nf * R <= kAxisAffineFloats / 2) {
+    for (int i = threadIdx.x; i < nf * R; i += blockDim.x) {
+      const int w = i / R, r = i - w * R;
+      const long long f = w + static_cast<long long>(r) * nf;
+      aff[i] = (p.gamma != nullptr && f < p.reduce) ? Elem<T>::load1(p.gamma, f) : 1.f;
+      if (OP == OP_LAYERNORM) aff[nf * R + i] = (p.beta != nullptr && f < p.reduce) ? Elem<T>::load1(p.beta, f) : 0.f;
+    }
+    gs = aff + wf * R;
+    bs = aff + nf * R + wf * R;
+  }
 
   for (long long b = blockIdx.y; b < p.outer; b += gridDim.y) {
     for (unsigned sc = blockIdx.x; sc < strips_per_outer; sc += gridDim.x) {
@@ -375,8 +411,8 @@ axis_reg_kernel(const AxisParams p, const unsigned strips_per_outer, const int n
         for (int j = 0; j < W; ++j) cq[j] *= ex2_approx(sa[j] - cp[j]);  // exp2(c_local - C) / S
       }
 
-      if (full) axis_reg_store<OP, T, MODE, R, true>(yb, ystep, active, nt, nf, gp, bp, raw, cp, cq);
-      else axis_reg_store<OP, T, MODE, R, false>(yb, ystep, active, nt, nf, gp, bp, raw, cp, cq);
+      if (full) axis_reg_store<OP, T, MODE, R, true>(yb, ystep, active, nt, nf, gp, bp, gs, bs, raw, cp, cq);
+      else axis_reg_store<OP, T, MODE, R, false>(yb, ystep, active, nt, nf, gp, bp, gs, bs, raw, cp, cq);
     }
   }
 }
