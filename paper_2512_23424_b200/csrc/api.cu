@@ -1358,14 +1358,14 @@ extern "C" akg_status akg_cumulative(int want_prod, const void* x, void* y, int6
                   lanes, static_cast<unsigned>(sctas));
     return AKG_OK;
   }
-  // Few, long rows (at least 8192 vectors each; fewer rows than SMs in fp32, than two per SM in the 16-bit
-  // types): a cluster per row, every CTA a slice of about 4096 vectors, the carry of a slice from the cluster's
-  // totals (scan_split_kernel).  Measured against a CTA per row, fraction of the copy rate: [64, 2^20] fp32 0.54
-  // against 0.30, bf16 0.64 against 0.22; [256, 262144] bf16 0.74 against 0.65, fp32 0.75 against 0.83 (hence the
-  // fp32 limit); [148, 131072] level in fp32, bf16 0.53 against 0.46.
+  // Few, long rows (at least 8192 vectors each, fewer rows than SMs): a cluster per row, every CTA a slice of
+  // about 4096 vectors, the carry of a slice from the cluster's totals (scan_split_kernel).  Measured against a
+  // CTA per row, fraction of the copy rate: [64, 2^20] fp32 0.54 against 0.30, bf16 0.64 against 0.22;
+  // [100, 262144] fp32 0.66 against 0.49, bf16 0.57 against 0.45; from one row per SM on a CTA per row is ahead
+  // ([256, 262144] fp32 0.85 against 0.75; bf16, with its loads three chunks ahead, 0.80 against 0.74).
   const int t_cs = g_tune_cluster_size.load();
   if (vec && !warp_rows && g_tune_reg_general.load() == 0 &&
-      (t_cs > 1 || (t_cs == 0 && rows < (es == 4 ? 1 : 2) * static_cast<int64_t>(sm_count()) && nvec >= 8192))) {
+      (t_cs > 1 || (t_cs == 0 && rows < static_cast<int64_t>(sm_count()) && nvec >= 8192))) {
     int cs = t_cs;
     if (cs == 0) {
       cs = 2;
@@ -1388,12 +1388,21 @@ extern "C" akg_status akg_cumulative(int want_prod, const void* x, void* y, int6
       return AKG_OK;
     }
   }
+  // 16-bit rows, a CTA per row with fewer CTAs than two per SM and rows of several chunks: the loads run three
+  // chunks ahead (bf16 [256, 262144] 0.67 -> 0.80 of the copy rate, [148, 131072] 0.48 -> 0.57; fp32 measured level
+  // or a little slower with them, 0.85 / 0.85 and 0.82 / 0.84, and keeps one chunk)
+  const int t_depth = g_tune_reg_vpt.load();                   // (tuning: reg_vpt 1 / 3 forces the depth)
+  const int depth = (vec && !warp_rows && threads == 256 &&
+                     (t_depth == 3 || (t_depth == 0 && es == 2 && ctas <= 2 * static_cast<int64_t>(sm_count()) &&
+                                       nvec >= 4 * 1024)))
+                        ? 3 : 1;
   const cudaError_t err = launch_cumulative(want_prod == 1, static_cast<int>(dtype), vec, x, y, rows, cols, x_row_stride,
                                             y_row_stride, grid, threads, warp_rows, g_tune_pdl.load() == 2 ? 0 : 1,
-                                            static_cast<cudaStream_t>(stream));
+                                            static_cast<cudaStream_t>(stream), depth);
   if (err != cudaSuccess) return cuda_fail(name, err);
-  std::snprintf(t_kernel, sizeof t_kernel, "scan<%s,%s,%s,%s%d,grid%u>", want_prod ? "prod" : "sum",
-                dtype_name(dtype), vec ? "vec" : "scalar", warp_rows ? "g32,t" : "t", warp_rows ? 256 : threads, grid);
+  std::snprintf(t_kernel, sizeof t_kernel, "scan<%s,%s,%s,%s%d,grid%u%s>", want_prod ? "prod" : "sum",
+                dtype_name(dtype), vec ? "vec" : "scalar", warp_rows ? "g32,t" : "t", warp_rows ? 256 : threads, grid,
+                depth > 1 ? ",ahead3" : "");
   return AKG_OK;
 }
 

@@ -155,6 +155,161 @@ __global__ void __launch_bounds__(32 * kScanMaxWarps, 4) scan_kernel(const ScanP
 }
 
 
+// scan_flat_kernel: the vectorised CTA-per-row form of scan_kernel (below) with its two loops - rows, chunks of a row -
+// flattened into one walk through the CTA's chunks: the loads keep running ahead across row ends, the two buffers of
+// warp totals alternate from chunk to chunk across rows as well (no extra barrier at a row's end), and the loads can
+// run more than one chunk ahead.  (A warp per row measured slower in this form, 0.82 against 0.94 on bf16
+// [16384, 8192], and keeps scan_kernel.)
+// DEPTH: how many chunks ahead of the one being scanned the vector loads run.  One is enough while four CTAs per SM
+// keep the memory system busy.  A few long rows (fewer CTAs than two per SM) are bound by the load latency instead:
+// a chunk's loads were issued only one chunk earlier, a chunk is scanned in a fraction of a microsecond, so every
+// chunk waited for most of a memory round trip ([256, 262144] fp32: 64 chunks per row at about 1.5 us each).  With
+// DEPTH 3 the loads are three chunks ahead (48 KB in flight per CTA, two CTAs per SM).  The chunk loop is unrolled
+// DEPTH times so that every buffer of the ring is a fixed set of registers: shifting the ring by register moves
+// made each iteration wait for loads still in flight and gained nothing.
+template <bool PROD, typename T, int DEPTH>
+__global__ void __launch_bounds__(32 * kScanMaxWarps, DEPTH > 1 ? 2 : 4) scan_flat_kernel(const ScanParams p) {
+  constexpr bool VEC = true;
+  constexpr bool WARP = false;
+  pdl_prologue();
+  using E = Elem<T>;
+  constexpr int EPV = VEC ? E::EPV : 1;
+  constexpr int U = kScanU;
+  __shared__ float wtot[2][U][kScanMaxWarps];
+  const int lane = threadIdx.x & 31;
+  const int T_ = WARP ? 32 : static_cast<int>(blockDim.x);      // threads per row
+  const int tid = WARP ? lane : static_cast<int>(threadIdx.x);  // position among them
+  const int NW = T_ >> 5;
+  const int warp = WARP ? 0 : static_cast<int>(threadIdx.x >> 5);
+  const long long row0 = WARP ? static_cast<long long>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5)
+                              : static_cast<long long>(blockIdx.x);
+  const long long row_step = WARP ? static_cast<long long>(gridDim.x) * (blockDim.x >> 5)
+                                  : static_cast<long long>(gridDim.x);
+  const long long nvec = (p.cols + EPV - 1) / EPV;              // VEC: cols is a multiple of EPV
+  const long long chunk = static_cast<long long>(U) * T_;
+  const float id = scan_identity<PROD>();
+
+  // the 16-byte vectors of a chunk are loaded DEPTH chunks ahead (the row's later chunks, or the first chunks of
+  // the CTA's next rows): the loads follow a cursor of their own through the chunks this CTA (or warp) will scan
+  uint4 ahead[DEPTH][U];
+  long long frow = row0, fbase = 0;
+  auto load_next = [&](uint4 (&dst)[U]) {
+    if (frow < p.rows) {
+      const T* xf = reinterpret_cast<const T*>(p.x) + frow * p.xs;
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const long long i = fbase + static_cast<long long>(u) * T_ + tid;
+        if (i < nvec) dst[u] = ld_stream(xf + i * EPV);
+      }
+      fbase += chunk;
+      if (fbase >= nvec) { fbase = 0; frow += row_step; }
+    }
+  };
+  if (VEC) {
+#pragma unroll
+    for (int d = 0; d < DEPTH; ++d) load_next(ahead[d]);
+  }
+
+  long long row = row0, base = 0;
+  float carry = id;
+  int par = 0;
+  while (row < p.rows) {
+#pragma unroll
+    for (int d = 0; d < DEPTH; ++d) {
+      if (row >= p.rows) break;                                 // the same for every thread that shares a barrier
+      const T* xr = reinterpret_cast<const T*>(p.x) + row * p.xs;
+      T* yr = reinterpret_cast<T*>(p.y) + row * p.ys;
+      float v[U][EPV];
+      // ---- the chunk's values (vectors beyond the row hold the identity)
+      if (VEC) {
+        uint4 raw[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) raw[u] = ahead[d][u];
+        load_next(ahead[d]);
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+          const long long i = base + static_cast<long long>(u) * T_ + tid;
+          float f[E::EPV];
+          if (i < nvec) E::unpack(raw[u], f);
+#pragma unroll
+          for (int j = 0; j < EPV; ++j) v[u][j] = (i < nvec) ? f[j] : id;
+        }
+      } else {
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+          const long long i = base + static_cast<long long>(u) * T_ + tid;
+          v[u][0] = (i < nvec) ? E::load1(xr, i) : id;
+        }
+      }
+      // ---- scan inside each vector, then the vector totals across the warp
+      float incl[U];                                            // inclusive scan of the totals over lanes
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+#pragma unroll
+        for (int j = 1; j < EPV; ++j) v[u][j] = scan_op<PROD>(v[u][j - 1], v[u][j]);
+        incl[u] = v[u][EPV - 1];
+      }
+#pragma unroll
+      for (int s = 1; s < 32; s <<= 1) {
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+          const float o = __shfl_up_sync(0xffffffffu, incl[u], s);
+          if (lane >= s) incl[u] = scan_op<PROD>(o, incl[u]);
+        }
+      }
+      if (!WARP) {
+        // (two buffers alternate from chunk to chunk, across rows as well: a thread can write the buffer of
+        // chunk k + 2 only after the barrier of chunk k + 1, which every thread reaches after reading chunk k's)
+        if (lane == 31) {
+#pragma unroll
+          for (int u = 0; u < U; ++u) wtot[par][u][warp] = incl[u];
+        }
+        __syncthreads();
+      }
+      // ---- what precedes this thread's vector u: carry, earlier u, earlier warps, earlier lanes
+      float before = carry;
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        // the warps' totals of this u are combined on their own, so that the carry picks up one
+        // operation per u (its rounding error grows with the number of chunks, not of warps)
+        float pre = id, tot = id;
+        if (WARP) {
+          tot = __shfl_sync(0xffffffffu, incl[u], 31);
+        } else {
+          for (int w = 0; w < NW; ++w) {
+            const float t = wtot[par][u][w];
+            if (w < warp) pre = scan_op<PROD>(pre, t);
+            tot = scan_op<PROD>(tot, t);
+          }
+        }
+        float mine = scan_op<PROD>(before, pre);                // carry, all of the earlier u, earlier warps
+        before = scan_op<PROD>(before, tot);
+        const float excl = __shfl_up_sync(0xffffffffu, incl[u], 1);
+        if (lane > 0) mine = scan_op<PROD>(mine, excl);
+        const long long i = base + static_cast<long long>(u) * T_ + tid;
+        if (i < nvec) {
+          float o[EPV];
+#pragma unroll
+          for (int j = 0; j < EPV; ++j) o[j] = scan_op<PROD>(mine, v[u][j]);
+          if (VEC) {
+            float f[E::EPV];
+#pragma unroll
+            for (int j = 0; j < EPV; ++j) f[j] = o[j];
+            st_stream(yr + i * EPV, E::pack(f));
+          } else {
+            E::store1(yr, i, o[0]);
+          }
+        }
+      }
+      carry = before;
+      par ^= 1;
+      base += chunk;
+      if (base >= nvec) { base = 0; row += row_step; carry = id; }
+    }
+  }
+}
+
+
 // ------------------------------------------------------------------------------------------------
 // scan_short_kernel: rows of at most 4 * L vectors (L = 4, 8 or 16 lanes per row, so up to 64 vectors: a
 // kilobyte).  A warp per row leaves most lanes without a vector on such rows (bf16 rows of 256 columns

@@ -66,7 +66,7 @@ cudaError_t launch_argreduce(bool want_min, int dtype, bool vec, bool warp_rows,
                              long long seg_vecs, int pdl, cudaStream_t stream);
 cudaError_t launch_cumulative(bool want_prod, int dtype, bool vec, const void* x, void* y, long long rows,
                               long long cols, long long xs, long long ys, unsigned grid, int threads, bool warp_rows,
-                              int pdl, cudaStream_t stream);
+                              int pdl, cudaStream_t stream, int depth = 1);   // depth: chunks loaded ahead (1 or 3)
 
 // Short vectorised rows (at most 4 * lanes vectors, lanes in {4, 8, 16}): 32 / lanes rows per warp, CTAs of 256.
 cudaError_t launch_cumulative_short(bool want_prod, int dtype, int lanes, const void* x, void* y, long long rows,

@@ -63,9 +63,10 @@ cudaError_t launch_arg_split_t(bool vec, const ArgParams& p, unsigned segments, 
 
 template <bool PROD, typename T>
 cudaError_t launch_scan_t(bool vec, bool warp_rows, const ScanParams& p, unsigned grid, int threads, int pdl,
-                          cudaStream_t s) {
+                          cudaStream_t s, int depth) {
   if (vec && warp_rows) return launch_1d(scan_kernel<PROD, T, true, true>, p, grid, 32 * kScanMaxWarps, pdl, s);
-  return vec ? launch_1d(scan_kernel<PROD, T, true>, p, grid, threads, pdl, s)
+  if (vec && depth > 1) return launch_1d(scan_flat_kernel<PROD, T, 3>, p, grid, threads, pdl, s);
+  return vec ? launch_1d(scan_flat_kernel<PROD, T, 1>, p, grid, threads, pdl, s)
              : launch_1d(scan_kernel<PROD, T, false>, p, grid, threads, pdl, s);
 }
 
@@ -187,18 +188,18 @@ cudaError_t launch_argreduce(bool want_min, int dtype, bool vec, bool warp_rows,
 
 cudaError_t launch_cumulative(bool want_prod, int dtype, bool vec, const void* x, void* y, long long rows,
                               long long cols, long long xs, long long ys, unsigned grid, int threads, bool warp_rows,
-                              int pdl, cudaStream_t stream) {
+                              int pdl, cudaStream_t stream, int depth) {
   if (threads < 32 || threads > 32 * kScanMaxWarps || threads % 32) return cudaErrorInvalidValue;
   ScanParams p;
   p.x = x; p.y = y; p.rows = rows; p.cols = cols; p.xs = xs; p.ys = ys;
   if (dtype == DT_F32)
-    return want_prod ? launch_scan_t<true, float>(vec, warp_rows, p, grid, threads, pdl, stream)
-                     : launch_scan_t<false, float>(vec, warp_rows, p, grid, threads, pdl, stream);
+    return want_prod ? launch_scan_t<true, float>(vec, warp_rows, p, grid, threads, pdl, stream, depth)
+                     : launch_scan_t<false, float>(vec, warp_rows, p, grid, threads, pdl, stream, depth);
   if (dtype == DT_F16)
-    return want_prod ? launch_scan_t<true, __half>(vec, warp_rows, p, grid, threads, pdl, stream)
-                     : launch_scan_t<false, __half>(vec, warp_rows, p, grid, threads, pdl, stream);
-  return want_prod ? launch_scan_t<true, __nv_bfloat16>(vec, warp_rows, p, grid, threads, pdl, stream)
-                   : launch_scan_t<false, __nv_bfloat16>(vec, warp_rows, p, grid, threads, pdl, stream);
+    return want_prod ? launch_scan_t<true, __half>(vec, warp_rows, p, grid, threads, pdl, stream, depth)
+                     : launch_scan_t<false, __half>(vec, warp_rows, p, grid, threads, pdl, stream, depth);
+  return want_prod ? launch_scan_t<true, __nv_bfloat16>(vec, warp_rows, p, grid, threads, pdl, stream, depth)
+                   : launch_scan_t<false, __nv_bfloat16>(vec, warp_rows, p, grid, threads, pdl, stream, depth);
 }
 
 }  // namespace akg

@@ -208,6 +208,41 @@ def test_cumulative_long_rows_split_over_a_cluster(dtype):
 
 
 @pytest.mark.parametrize("dtype", DTYPES)
+def test_cumulative_few_long_rows_load_three_chunks_ahead(dtype):
+    """A CTA per row with few CTAs: the loads run three chunks ahead of the scan, across row ends as well."""
+    rng = np.random.default_rng(26)
+    epv = 4 if dtype == wl.F32 else 8
+    try:
+        # (ragged last chunks, rows of exactly three and of four chunks, one chunk only, more rows than CTAs)
+        for rows, cols, cap in [(37, 5000 * epv, 0), (200, 4096 * epv, 0), (9, 3072 * epv + epv, 0), (50, 7777 * epv, 7),
+                                (11, 1024 * epv, 3), (5, 300 * epv, 2)]:
+            akg.set_tuning("reg_vpt", 3)
+            akg.set_tuning("cluster_size", 1)
+            akg.set_tuning("grid_cap", cap)
+            x = rng.normal(0.05, 1, (rows, cols)).astype(np.float32)
+            check_cum("cumsum", store(x, dtype), dtype, f"{rows}x{cols} ahead3")
+            if ",t256," in akg.last_kernel() and "g32" not in akg.last_kernel():     # a CTA of 256 threads per row
+                assert "ahead3" in akg.last_kernel(), akg.last_kernel()
+            f = (1.0 + 0.002 * rng.normal(0, 1, (rows, cols))).astype(np.float32)
+            check_cum("cumprod", store(f, dtype), dtype, f"{rows}x{cols} ahead3")
+        akg.set_tuning("reg_vpt", 0)
+        akg.set_tuning("grid_cap", 0)
+        akg.set_tuning("cluster_size", 0)
+        # the automatic choice (16-bit only): fewer CTAs than two per SM, rows of at least four chunks, no cluster
+        x = rng.integers(-2, 3, (200, 5120 * epv)).astype(np.float32)
+        ref = oracle.cumulative("cumsum", x)
+        got = widen(to_numpy(binding.cumsum(to_torch(store(x, dtype), dtype))))
+        assert akg.last_kernel().startswith("scan<") and ("ahead3" in akg.last_kernel()) == (dtype != wl.F32), \
+            akg.last_kernel()
+        exact = np.abs(ref) < (2 ** 24 if dtype == wl.F32 else 256)
+        assert np.array_equal(got[exact], ref[exact])
+    finally:
+        akg.set_tuning("reg_vpt", 0)
+        akg.set_tuning("grid_cap", 0)
+        akg.set_tuning("cluster_size", 0)
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
 def test_cumulative_exact_cases_in_place_and_strides(dtype):
     tdt = torch.float32 if dtype == wl.F32 else torch.bfloat16
     # small integers: every partial sum is exact in fp32 (and in bf16 while below 256)
