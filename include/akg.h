@@ -309,6 +309,7 @@ akg_status akg_set_variant(akg_variant variant);
 /* Override one launch-geometry choice for subsequent calls (benchmarking aid; 0
  * restores the library's own choice).  Keys: "reg_threads", "reg_vpt" (CTA size and
  * 16-byte vectors per thread of the register-resident family; both must be set),
+ * for akg_cumulative "reg_vpt" 1 / 3 is how many chunks ahead of the scan a CTA per row loads),
  * "reg_group" (32 = a warp per row, 1 = a CTA per row), "grid_cap" (maximum CTAs;
  * rows beyond it are taken in a grid-stride loop); for the shared-memory ring
  * families "cluster_size" (CTAs per row: 1, 2, 4, 8, 16), "smem_nbuf" (ring depth
