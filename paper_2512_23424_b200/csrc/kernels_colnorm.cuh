@@ -92,8 +92,12 @@ __global__ void __launch_bounds__(kAxisThreads, 4) col_stat_kernel(const ColPara
   }
 }
 
-// A warp per column: lane l takes row blocks l, l + 32, ...; two sweeps (mean of the block means weighted by
-// their counts, then the M2 of the blocks about it), each finished by a shuffle sum.
+// A warp per column: lane l takes row blocks l, l + 32, ...  One sweep over the blocks' pairs, with sums taken
+// about the first block's mean (ref): S1 = sum n_b (m_b - ref), S2 = sum (M2_b + n_b (m_b - ref)^2), then
+// mean = ref + S1 / N and M2 = S2 - N (mean - ref)^2.  The block means differ from the column mean by about
+// sigma / sqrt(rows per block), so the term subtracted at the end is a small fraction of M2 and the subtraction
+// costs no accuracy that matters; two sweeps (the mean first) read the pairs twice, one dependent trip to L2 more
+// in a kernel that is nothing but latency.
 __global__ void __launch_bounds__(256) col_finish_kernel(const ColParams p, const int nblk) {
   pdl_prologue();                              // the statistics kernel has completed when this returns
   const int lane = threadIdx.x & 31;
@@ -103,16 +107,19 @@ __global__ void __launch_bounds__(256) col_finish_kernel(const ColParams p, cons
   auto count = [&](int b) {
     return static_cast<float>(min(p.rows, (b + 1) * p.rows_per_block) - b * p.rows_per_block);
   };
-  float mean = 0.f;
-  for (int b = lane; b < nblk; b += 32) mean = fmaf(count(b), p.partial[static_cast<long long>(b) * p.cols + c].x, mean);
-  mean = warp_sum(mean) * inv_rows;
-  float m2 = 0.f;
+  const float ref = p.partial[c].x;            // block 0 always has rows
+  float s1 = 0.f, s2 = 0.f;
   for (int b = lane; b < nblk; b += 32) {
     const float2 pb = p.partial[static_cast<long long>(b) * p.cols + c];
-    const float d = pb.x - mean;
-    m2 += fmaf(count(b) * d, d, pb.y);
+    const float n = count(b), d = pb.x - ref;
+    s1 = fmaf(n, d, s1);
+    s2 += fmaf(n * d, d, pb.y);
   }
-  const float var = warp_sum(m2) * inv_rows;
+  s1 = warp_sum(s1);
+  s2 = warp_sum(s2);
+  const float dm = s1 * inv_rows;              // mean - ref
+  const float mean = ref + dm;
+  const float var = fmaxf(fmaf(-s1, dm, s2), 0.f) * inv_rows;
   __syncwarp();                                // every lane has read the column's pairs
   if (lane == 0) {
     p.partial[c] = make_float2(mean, rsqrt_refined(var + p.eps));
