@@ -46,7 +46,49 @@ __global__ void __launch_bounds__(kAxisThreads, 4) col_stat_kernel(const ColPara
   run.init();
   // (a matrix far beyond L2 gains nothing from the marks and measured 8 % slower with them: plain priority then)
   const uint64_t keep = p.l2_keep ? l2_policy_keep() : l2_policy_normal();
-  if (active) {
+  if constexpr (sizeof(T) == 2 && MODE == 1) {
+    // 16-bit storage: one sweep of sums about the thread's first row of the block, K = x[first]: S1 = sum (x - K),
+    // S2 = sum (x - K)^2, mean = K + S1 / n, M2 = S2 - S1^2 / n.  K lies among the data, so the subtraction at the
+    // end costs a relative (n + 1) 2^-24 at most (n is a few dozen rows), far inside the 2^-9 of a 16-bit result;
+    // the stored values enter the subtraction as they are (Elem::sub_wide).  Three instructions per element instead
+    // of the block-wise means, deviations and merges of the fp32 form.
+    if (active && r0 + slot < r1) {
+      using E = Elem<T>;
+      const T* px = reinterpret_cast<const T*>(p.x) + (r0 + slot) * p.xs + col0;
+      float k[W], s1[W], s2[W];
+      A::unpack(A::load(px), k);
+#pragma unroll
+      for (int j = 0; j < W; ++j) { s1[j] = 0.f; s2[j] = 0.f; }
+      auto add_row = [&](const Raw& raw) {
+        const uint32_t ws[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          unsigned short h0, h1;
+          halves(ws[i], h0, h1);
+          const float d0 = E::sub_wide(h0, k[2 * i]), d1 = E::sub_wide(h1, k[2 * i + 1]);
+          s1[2 * i] += d0; s2[2 * i] = fmaf(d0, d0, s2[2 * i]);
+          s1[2 * i + 1] += d1; s2[2 * i + 1] = fmaf(d1, d1, s2[2 * i + 1]);
+        }
+      };
+      long long f = r0 + slot;
+      for (; f + (UB - 1) * ns < r1; f += UB * ns) {
+        Raw raw[UB];
+#pragma unroll
+        for (int u = 0; u < UB; ++u, px += xstep) raw[u] = A::load_hint(px, keep);
+#pragma unroll
+        for (int u = 0; u < UB; ++u) add_row(raw[u]);
+      }
+      for (; f < r1; f += ns, px += xstep) add_row(A::load_hint(px, keep));
+      const float n = static_cast<float>((r1 - (r0 + slot) + ns - 1) / ns);
+      const float inv_n = __frcp_rn(n);
+#pragma unroll
+      for (int j = 0; j < W; ++j) {
+        const float m = s1[j] * inv_n;                        // mean - K
+        run.a[j] = k[j] + m;
+        run.b[j] = fmaxf(fmaf(-s1[j], m, s2[j]), 0.f);
+      }
+    }
+  } else if (active) {
     const T* px = reinterpret_cast<const T*>(p.x) + (r0 + slot) * p.xs + col0;
     long long f = r0 + slot;
     for (; f + (UB - 1) * ns < r1; f += UB * ns) {
