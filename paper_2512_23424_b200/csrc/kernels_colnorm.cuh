@@ -124,7 +124,11 @@ __global__ void __launch_bounds__(kAxisThreads, 4) col_stat_kernel(const ColPara
     const int nbase = static_cast<int>(n / ns), nrem = static_cast<int>(n % ns);
     float mean = 0.f;
     for (int i = 0; i < ns; ++i) mean = fmaf(static_cast<float>(nbase + (i < nrem ? 1 : 0)), part[0][i * cw + threadIdx.x], mean);
-    mean *= 1.0f / static_cast<float>(n);
+    {
+      // (weighted sum / n with one residual step: the rounded 1 / n alone would bias every block's mean the same way)
+      const float nf = static_cast<float>(n), inv_n = 1.0f / nf, q = mean * inv_n;
+      mean = fmaf(fmaf(-q, nf, mean), inv_n, q);
+    }
     float m2 = 0.f;
     for (int i = 0; i < ns; ++i) {
       const float d = part[0][i * cw + threadIdx.x] - mean;

@@ -16,6 +16,25 @@
 
 namespace akg {
 
+// s / N for the N values of a thread.  Unless N is a power of two the rounded reciprocal is off by up to half an
+// ulp, and the product s * (1 / N) is off the same way in every thread of every row: a bias of the row mean of
+// up to 2^-24 |mean| that no merge averages out.  It shows where |mean| is many standard deviations (mean / std
+// = 30: results next to zero were off by 6e-6, beyond two ulps of a 16-bit result); one residual step takes it out.
+template <int N> __device__ __forceinline__ float thread_mean(float s) {
+  constexpr float inv = 1.0f / N;
+  const float q = s * inv;
+  if constexpr ((N & (N - 1)) == 0) return q;
+  return fmaf(fmaf(-q, static_cast<float>(N), s), inv, q);
+}
+
+// Mean of the NW warp means held by lanes 0 .. NW - 1 (mw; `mine` marks them): lane 0's value plus the mean of
+// the differences from it, so that the rounded 1 / NW (inv_warps; NW is any number up to 32) and the rounding of
+// the sum act on the differences only, not on the mean's own magnitude.
+__device__ __forceinline__ float mean_of_warp_means(float mw, bool mine, float inv_warps) {
+  const float ref = __shfl_sync(0xffffffffu, mw, 0);
+  return fmaf(warp_sum(mine ? mw - ref : 0.f), inv_warps, ref);
+}
+
 // Occupancy target of the register-resident kernels: at least 1024 threads per SM, i.e.
 // at most 64 registers per thread (occupancy, not instruction count, bounds them next).
 template <int THREADS> constexpr int kRegMinBlocks = (1024 / THREADS) > 0 ? (1024 / THREADS) : 1;
@@ -73,7 +92,7 @@ __device__ __forceinline__ void norm_row_full(const RowParams& p, long long row,
     float s0 = 0.f, s1 = 0.f;
 #pragma unroll
     for (int i = 0; i < N; i += 2) { s0 += v[i]; s1 += v[i + 1]; }
-    float mu = (s0 + s1) * (1.0f / N);
+    float mu = thread_mean<N>(s0 + s1);
     float q0 = 0.f, q1 = 0.f;
 #pragma unroll
     for (int i = 0; i < N; i += 2) {
@@ -168,7 +187,7 @@ __device__ __forceinline__ void flex_row_stats(const float (&v)[N], float (*red)
     float s0 = 0.f, s1 = 0.f;
 #pragma unroll
     for (int i = 0; i < N; i += 2) { s0 += v[i]; s1 += v[i + 1]; }
-    float mu = (s0 + s1) * (1.0f / N);
+    float mu = thread_mean<N>(s0 + s1);
     float q0 = 0.f, q1 = 0.f;
 #pragma unroll
     for (int i = 0; i < N; i += 2) {
@@ -193,7 +212,7 @@ __device__ __forceinline__ void flex_row_stats(const float (&v)[N], float (*red)
     const bool mine = static_cast<int>(threadIdx.x & 31) < NW;
     const float mw = mine ? red[0][threadIdx.x & 31] : 0.f;
     const float qsum = warp_sum(mine ? red[1][threadIdx.x & 31] : 0.f);
-    mean = warp_sum(mw) * inv_warps;
+    mean = mean_of_warp_means(mw, mine, inv_warps);
     const float d = mine ? mw - mean : 0.f;
     const float dev = warp_sum(d * d);
     rstd = rsqrt_refined(fmaf(fmaf(dev, 32.0f * N, qsum), inv_cols, eps));
@@ -229,7 +248,7 @@ __device__ __forceinline__ void flex_merge(float mu, float m2, int n, float (*re
     const bool mine = static_cast<int>(threadIdx.x & 31) < NW;
     const float mw = mine ? red[0][threadIdx.x & 31] : 0.f;
     const float qsum = warp_sum(mine ? red[1][threadIdx.x & 31] : 0.f);
-    mean = warp_sum(mw) * inv_warps;
+    mean = mean_of_warp_means(mw, mine, inv_warps);
     const float d = mine ? mw - mean : 0.f;
     const float dev = warp_sum(d * d);
     rstd = rsqrt_refined(fmaf(fmaf(dev, 32.0f * static_cast<float>(n), qsum), inv_cols, eps));
@@ -295,7 +314,7 @@ __global__ void __launch_bounds__(1024, 1) reg_norm_packed(const RowParams p, co
           s1 = E::add_wide(h1, s1);
         }
       }
-      mu = (s0 + s1) * (1.0f / N);
+      mu = thread_mean<N>(s0 + s1);
       float q0 = 0.f, q1 = 0.f;
 #pragma unroll
       for (int k = 0; k < VPT; ++k) {

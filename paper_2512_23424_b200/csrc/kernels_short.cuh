@@ -139,7 +139,10 @@ __global__ void __launch_bounds__(kShortThreads, 8) short_rows_kernel(const RowP
         for (int k = 0; k < K; ++k)
 #pragma unroll
           for (int j = 0; j < EPV; j += 2) { s0 += v[k][j]; s1 += v[k][j + 1]; }
-        mean = group_sum<L>(s0 + s1) * inv_cols;
+        const float sum = group_sum<L>(s0 + s1);
+        mean = sum * inv_cols;
+        // (one residual step: the rounded 1 / cols would bias every row's mean the same way, by up to 2^-24 |mean|)
+        mean = fmaf(fmaf(-mean, static_cast<float>(p.cols), sum), inv_cols, mean);
         float q0 = 0.f, q1 = 0.f;
 #pragma unroll
         for (int k = 0; k < K; ++k) {

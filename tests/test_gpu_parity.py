@@ -142,6 +142,21 @@ def test_shape_sweep(op, dtype):
         check_workload(w)
 
 
+# LayerNorm rows whose mean is thirty standard deviations from zero: a mean that is off by one part in 2^24
+# (a thread's sum times a rounded 1 / 24, 1 / 56, ...; warp means times a rounded 1 / 3, 1 / 7, ...) moves the
+# results next to zero by more than two ulps of a 16-bit type.  Shapes with a number of values per thread and a
+# number of warps per row that are no powers of two, and short rows (1 / cols).
+@pytest.mark.parametrize("dtype,rows,cols,seed,affine", [
+    (wl.BF16, 585, 5376, 112391494, True), (wl.F16, 585, 5376, 98737495, True), (wl.F16, 585, 5376, 98737495, False),
+    (wl.BF16, 585, 5376, 5, True), (wl.BF16, 585, 10752, 5, True), (wl.BF16, 2000, 768, 6, True),
+    (wl.BF16, 4100, 264, 7, True), (wl.F16, 4100, 200, 8, True), (wl.F32, 300, 5120, 9, True),
+    (wl.F32, 300, 2560, 10, True)])
+def test_layernorm_mean_far_from_zero(dtype, rows, cols, seed, affine):
+    base = wl.make_random("layernorm", wl.F32 if dtype == wl.F16 else dtype, rows, cols, seed, loc=-3.0, scale=0.1,
+                          affine=affine)
+    check_workload(wl.as_f16(base) if dtype == wl.F16 else base, variants=["auto"])
+
+
 @pytest.mark.parametrize("op", ["softmax", "log_softmax", "layernorm", "rmsnorm"])
 @pytest.mark.parametrize("dtype", [wl.F32, wl.BF16])
 def test_strides_offsets_and_no_stray_writes(op, dtype):
