@@ -101,8 +101,10 @@ __device__ __forceinline__ void axis_merge_slots(const float* q0, const float* q
     for (int i = 0; i < ns; ++i)
       bb = fmaf(q1[i * cw], OP == OP_SOFTMAX ? ex2_approx(q0[i * cw] - ms) : exp_diff(q0[i * cw], ms), bb);
   } else if (OP == OP_LAYERNORM) {
-    for (int i = 0; i < ns; ++i) a = fmaf(static_cast<float>(nbase + (i < nrem ? 1 : 0)), q0[i * cw], a);
-    a *= inv_f;
+    // (the first slot's mean plus the weighted mean of the differences from it: see axis_merge_column)
+    const float ref = q0[0];
+    for (int i = 0; i < ns; ++i) a = fmaf(static_cast<float>(nbase + (i < nrem ? 1 : 0)), q0[i * cw] - ref, a);
+    a = fmaf(a, inv_f, ref);
     for (int i = 0; i < ns; ++i) {
       const float d = q0[i * cw] - a;
       bb += fmaf(static_cast<float>(nbase + (i < nrem ? 1 : 0)) * d, d, q1[i * cw]);

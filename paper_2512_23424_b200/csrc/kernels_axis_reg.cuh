@@ -123,11 +123,15 @@ __device__ __forceinline__ void axis_merge_column(const float* q0, const float* 
     for (int i = 0; i < nf; ++i)
       bb = fmaf(q1[i * CW], OP == OP_SOFTMAX ? ex2_approx(q0[i * CW] - ms) : exp_diff(q0[i * CW], ms), bb);
   } else if (OP == OP_LAYERNORM) {
+    // The mean as the first partial mean plus the weighted mean of the differences from it: summing the partial
+    // means themselves rounds at the magnitude of count x |mean| and the rounded 1 / F biases the quotient, which
+    // together put 1e-6 |mean| into the mean of a thousand rows (results off by 2e-5 where mean / std = 30).
+    const float ref = q0[0];
     if (nrem == 0) {                       // equal counts: mean of means, M2 = sum M2_i + n sum d_i^2
 #pragma unroll 4
-      for (int i = 0; i < nf; ++i) a += q0[i * CW];
+      for (int i = 0; i < nf; ++i) a += q0[i * CW] - ref;
       const float nb = static_cast<float>(nbase);
-      a *= nb * inv_f;
+      a = fmaf(a, nb * inv_f, ref);
       float dd = 0.f;
 #pragma unroll 4
       for (int i = 0; i < nf; ++i) {
@@ -137,8 +141,8 @@ __device__ __forceinline__ void axis_merge_column(const float* q0, const float* 
       }
       bb = fmaf(nb, dd, bb);
     } else {
-      for (int i = 0; i < nf; ++i) a = fmaf(static_cast<float>(nbase + (i < nrem ? 1 : 0)), q0[i * CW], a);
-      a *= inv_f;
+      for (int i = 0; i < nf; ++i) a = fmaf(static_cast<float>(nbase + (i < nrem ? 1 : 0)), q0[i * CW] - ref, a);
+      a = fmaf(a, inv_f, ref);
       for (int i = 0; i < nf; ++i) {
         const float d = q0[i * CW] - a;
         bb += fmaf(static_cast<float>(nbase + (i < nrem ? 1 : 0)) * d, d, q1[i * CW]);
@@ -241,18 +245,26 @@ __device__ __forceinline__ void axis_reg_load(const T* px, long long xstep, bool
       sa[j] = (FULL || nt > 0) ? k[j] + m : 0.f;
     }
   } else if (OP == OP_LAYERNORM) {
+    // fp32 storage: the exact two sweeps, the mean as the thread's first row plus the mean of the differences
+    // from it.  (The plain sum of R values rounds at R |mean| and the rounded 1 / nt biases the quotient: with
+    // 3 to 16 rows per column and mean / std = 30 the results were off by three to five times what the
+    // rounding of the mean itself costs.)
+    float k[W];
+    A::unpack(raw[0], k);
 #pragma unroll
     for (int j = 0; j < W; ++j) { sa[j] = 0.f; sb[j] = 0.f; }
 #pragma unroll
-    for (int r = 0; r < R; ++r) {
-      float v[W];
-      A::unpack(raw[r], v);
+    for (int r = 1; r < R; ++r) {
+      if (FULL || r < nt) {
+        float v[W];
+        A::unpack(raw[r], v);
 #pragma unroll
-      for (int j = 0; j < W; ++j) sa[j] += v[j];             // rows not held are zeros
+        for (int j = 0; j < W; ++j) sa[j] += v[j] - k[j];
+      }
     }
     const float inv_nt = FULL ? (1.0f / R) : ((nt > 0) ? __frcp_rn(static_cast<float>(nt)) : 0.f);
 #pragma unroll
-    for (int j = 0; j < W; ++j) sa[j] *= inv_nt;
+    for (int j = 0; j < W; ++j) sa[j] = (FULL || nt > 0) ? fmaf(sa[j], inv_nt, k[j]) : 0.f;
 #pragma unroll
     for (int r = 0; r < R; ++r) {
       if (FULL || r < nt) {

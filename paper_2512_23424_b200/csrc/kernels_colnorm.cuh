@@ -122,13 +122,13 @@ __global__ void __launch_bounds__(kAxisThreads, 4) col_stat_kernel(const ColPara
   if (static_cast<int>(threadIdx.x) < cw && c < p.cols) {
     const long long n = r1 - r0;
     const int nbase = static_cast<int>(n / ns), nrem = static_cast<int>(n % ns);
+    // the first slot's mean plus the weighted mean of the differences from it: the sum of count x mean itself
+    // would round at n |mean| and the rounded 1 / n would bias every block's quotient the same way
+    const float ref = part[0][threadIdx.x];
     float mean = 0.f;
-    for (int i = 0; i < ns; ++i) mean = fmaf(static_cast<float>(nbase + (i < nrem ? 1 : 0)), part[0][i * cw + threadIdx.x], mean);
-    {
-      // (weighted sum / n with one residual step: the rounded 1 / n alone would bias every block's mean the same way)
-      const float nf = static_cast<float>(n), inv_n = 1.0f / nf, q = mean * inv_n;
-      mean = fmaf(fmaf(-q, nf, mean), inv_n, q);
-    }
+    for (int i = 0; i < ns; ++i)
+      mean = fmaf(static_cast<float>(nbase + (i < nrem ? 1 : 0)), part[0][i * cw + threadIdx.x] - ref, mean);
+    mean = fmaf(mean, 1.0f / static_cast<float>(n), ref);
     float m2 = 0.f;
     for (int i = 0; i < ns; ++i) {
       const float d = part[0][i * cw + threadIdx.x] - mean;

@@ -54,6 +54,36 @@ def test_axis_shapes(op, dtype):
         check(op, dtype, x, g, b, got, eps, f"axis {op} {outer}x{red}x{inner} [{akg.last_kernel()}]")
 
 
+# LayerNorm lines whose mean lies thirty standard deviations from zero.  The mean has to come out within an ulp
+# or so: partial means merged as "first partial + weighted mean of the differences from it", the thread's own
+# mean as "first row + mean of the differences".  (Summing the values, or count x partial mean, rounds at the
+# magnitude count x |mean|, and a rounded 1 / count biases the quotient: 2e-5 on fp32 results before.)  Only
+# the element-wise bound is asserted: the relative criterion of Eq. 2-3 has no meaning for the results next
+# to zero of such lines.
+@pytest.mark.parametrize("dtype", [wl.F32, wl.BF16])
+def test_axis_layernorm_mean_far_from_zero(dtype):
+    eps = 1e-5
+    kernels = set()
+    for i, (outer, red, inner) in enumerate([(3, 16, 1024), (2, 1000, 1024), (2, 257, 8), (1, 1000, 8), (4, 512, 8),
+                                             (2, 64, 4096), (2, 100, 264)]):
+        rng = np.random.default_rng(700 + i)
+        x = rng.normal(-3.0, 0.1, size=(outer, red, inner)).astype(np.float32)
+        g = rng.uniform(0.5, 1.5, red).astype(np.float32)
+        b = rng.normal(0, 0.1, red).astype(np.float32)
+        if dtype == wl.BF16:
+            x, g, b = wl.f32_to_bf16_bits(x), wl.f32_to_bf16_bits(g), wl.f32_to_bf16_bits(b)
+        out = binding.rowop_axis("layernorm", to_torch(x.reshape(outer * red, inner), dtype).view(outer, red, inner),
+                                 gamma=to_torch(g, dtype), beta=to_torch(b, dtype), eps=eps)
+        torch.cuda.synchronize()
+        kernels.add(akg.last_kernel().split("<")[0])
+        got = to_numpy(out.view(outer * red, inner)).reshape(outer, red, inner)
+        ref = oracle.rowop_axis("layernorm", x, g, b, eps=float(np.float32(eps)), nthreads=8)
+        what = f"axis layernorm {outer}x{red}x{inner} [{akg.last_kernel()}]"
+        w = wl.Workload(what, "layernorm", dtype, outer * inner, red, as_lines(x), eps=eps, gamma=g, beta=b)
+        compare(as_lines(got), as_lines(ref), dtype, what, cancel_magnitude(w, as_lines(ref)))
+    assert kernels == {"axis", "axis_reg"}
+
+
 @pytest.mark.parametrize("op", ["softmax", "rmsnorm"])
 @pytest.mark.parametrize("dtype", [wl.F32, wl.BF16])
 def test_axis_strides_in_place_and_padding(op, dtype):
